@@ -1,0 +1,183 @@
+/*
+ * qless.h -- C ABI of the QLESS hot path for NVIDIA B200 (sm_100a).
+ *
+ * QLESS (arXiv 2502.01703) values training examples by the similarity of their
+ * projected, quantised LoRA gradients to validation gradients. This library is
+ * the data-parallel hot path of that method:
+ *
+ *   qless_project_quantize  gradient -> Adam direction -> random projection
+ *                           -> L2 normalise -> absmax b-bit codes (+ scale)
+ *   qless_score             codes x validation codes -> influence scores
+ *   qless_select_topk       scores -> indices of the top fraction
+ *
+ * Naming. The paper projects R^d -> R^k; to avoid a clash this header calls the
+ * gradient dimension P and the projected dimension d (d = 8192 in the paper's
+ * Sec. 4.1), N / V the numbers of training / validation examples, C the number
+ * of checkpoints, T the number of target tasks, b = `bits` the code width.
+ *
+ * Conventions for every call, unless an argument says otherwise:
+ *  - pointers are DEVICE pointers into memory the caller owns; "host" marks the
+ *    exceptions. The library allocates nothing that outlives a call; scratch is
+ *    the caller's `workspace` (size from the matching *_workspace() query,
+ *    256-byte aligned).
+ *  - calls enqueue work on `cuda_stream` (a cudaStream_t cast to void*, NULL =
+ *    default stream) and return without synchronising. Host arrays are read
+ *    before the call returns.
+ *  - every precondition is checked before anything is launched; a violation
+ *    returns a status and leaves all buffers untouched. Calls with zero rows
+ *    succeed and touch nothing. No exception crosses this boundary.
+ *  - qless_last_error() gives a thread-local, human readable description of the
+ *    last non-OK status returned on this thread.
+ */
+#ifndef QLESS_H_
+#define QLESS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    QLESS_OK = 0,
+    QLESS_ERR_INVALID_ARG = 1, /* NULL where a buffer is required, negative size, bad offsets ... */
+    QLESS_ERR_UNSUPPORTED = 2, /* bits not in {1,2,4,8}; d or P not a multiple of 128; d > 8192 ... */
+    QLESS_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or smaller than the query says */
+    QLESS_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed; text in qless_last_error() */
+    QLESS_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up (see qless_check) */
+} qless_status;
+
+typedef enum { QLESS_F32 = 0, QLESS_BF16 = 1 } qless_dtype;
+
+/* Adam hyper-parameters of the training-gradient prologue. step = 0 switches the bias
+ * correction off (it is a uniform factor that normalisation removes, except through eps). */
+typedef struct {
+    float beta1;  /* 0.9   */
+    float beta2;  /* 0.999 */
+    float eps;    /* 1e-8  */
+    int64_t step; /* 0     */
+} qless_adam_cfg;
+
+const char* qless_last_error(void);
+
+/* Reads and clears the device-side timeout flag after synchronising `cuda_stream`. Kernels that
+ * wait on asynchronous copies or tensor-core completion give up after a bounded number of polls,
+ * set the flag and exit; results of that call are then invalid. Returns QLESS_OK,
+ * QLESS_ERR_TIMEOUT or QLESS_ERR_CUDA. */
+qless_status qless_check(void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Stage 1 + 2: datastore construction (paper Sec. 2.2 Eq. 1-2, Sec. 3.1, Eq. 4-5).
+ *
+ * For each of the n gradient rows g (row-major [n, P], leading dimension ld_grads elements):
+ *   Gamma = Adam direction of g given the checkpoint's moments (Sec. 2.2 "Adam training gradient
+ *           Gamma(z; theta)"):  m' = b1 m + (1-b1) g, v' = b2 v + (1-b2) g^2, (bias-corrected if
+ *           step > 0), Gamma = m' / (sqrt(v') + eps), computed in fp32 and rounded to bf16.
+ *           adam_m = adam_v = NULL selects the SGD (validation) gradient: Gamma = bf16(g).
+ *   y     = R Gamma (Eq. 1), R in {+-1/sqrt(d)}^{d x P} Rademacher. R is never stored: entry
+ *           (r, j) is bit t = j mod 128 of the Philox4x32-10 block with counter
+ *           (j / 128, r, 0, 0) and key (seed low, seed high); within 32-bit output word t / 32
+ *           the bit index is 15 - (u / 2) + 16 (u mod 2), u = t mod 32; bit 1 means -1.
+ *           bf16 x bf16 products, fp32 accumulation, one fp32 multiply by 1/sqrt(d).
+ *   yhat  = y / ||y||_2 (Eq. 2).
+ *   S     = max_m |yhat_m|; alpha = 2^(b-1) - 1; q_m = round_half_even(alpha yhat_m / S) (Eq. 4-5);
+ *           b = 1: q_m = -1 if yhat_m < 0 else +1 (sign quantiser). A zero vector gives S = 0 and
+ *           all-zero codes.
+ * Outputs (all optional except codes and scales):
+ *   codes      [n, d*bits/8] bytes, dense little-endian packing: b=8 one int8 per code; b=4 code m in
+ *              bits [4(m&1), +4) of byte m>>1; b=2 code m in bits [2(m&3), +2) of byte m>>2 (two's
+ *              complement fields); b=1 code m is bit m&7 of byte m>>3, bit 1 <=> -1.
+ *   scales     [n] fp32, the absmax S of the normalised vector (the "single scale factor" of Sec. 3.1).
+ *   code_sumsq [n] int32, sum_m q_m^2 = ||q||^2 of Eq. 6 (NULL to skip).
+ *   proj_out   [n, d] fp32, the un-normalised projection y (NULL to skip; test tap).
+ * The same seed must be used for every vector that will be scored together.
+ * Requirements: d % 128 == 0, 128 <= d <= 8192; P % 128 == 0; P < 2^39; grads 16-byte aligned and
+ * ld_grads % 8 == 0; bits in {1,2,4,8}; codes 16-byte aligned.
+ * ------------------------------------------------------------------------------------------ */
+size_t qless_project_quantize_workspace(int64_t n, int64_t P, int32_t d, int32_t bits);
+
+qless_status qless_project_quantize(
+    const void* grads, qless_dtype dtype, int64_t n, int64_t ld_grads,
+    const float* adam_m, const float* adam_v, const qless_adam_cfg* adam /* host, NULL = defaults */,
+    int64_t P, int32_t d, uint64_t seed, int32_t bits,
+    void* codes, float* scales, int32_t* code_sumsq, float* proj_out,
+    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Stage 2 alone (Eq. 2, Eq. 4-5, packing) on fp32 rows x [n, d]; normalize = 0 skips Eq. 2 so that
+ * already-normalised rows can be fed. Same outputs and packing as above. Needs no workspace. */
+qless_status qless_quantize(
+    const float* x, int64_t n, int32_t d, int32_t normalize, int32_t bits,
+    void* codes, float* scales, int32_t* code_sumsq, void* cuda_stream);
+
+/* Stage 1a alone: the Adam prologue. gamma_out [n, P] bf16 (raw 16-bit patterns), row-major, leading
+ * dimension P. Same reading of Gamma as above. */
+qless_status qless_adam_gamma(
+    const void* grads, qless_dtype dtype, int64_t n, int64_t ld_grads,
+    const float* adam_m, const float* adam_v, const qless_adam_cfg* adam /* host */,
+    int64_t P, void* gamma_out, void* cuda_stream);
+
+/* Entries of the projection matrix as the kernels generate them: out [nr, nj] int8 (+1 / -1) for
+ * rows r0 .. r0+nr-1 and columns j0 .. j0+nj-1 of sqrt(d) R (entry map above). */
+qless_status qless_philox_entries(
+    uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj, int8_t* out, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Stage 3: influence scores over the quantised datastore (paper Eq. 6-7; aggregation as in LESS,
+ * which the paper follows: "cumulative influence scores", Sec. 4.1).
+ *
+ *   D_i[t, v]  = sum_m q_{t,i,m} q_{v,i,m}                 integer, exact (b = 1: d - 2 popcount(xor))
+ *   sim_i[t,v] = D_i / (||q_{t,i}|| ||q_{v,i}||)            mode COSINE (Eq. 6-7); a vector whose scale
+ *                                                          is 0 is the zero vector and contributes 0
+ *              = (S_t/alpha)(S_v/alpha) D_i                mode DEQUANT (alpha := 1 at b = 1): inner
+ *                                                          product of the reconstructed vectors (Eq. 3)
+ *   A[t, j]    = sum_i eta_i * mean_{v in task j} sim_i[t, v]
+ *   score[t]   = max_j A[t, j]
+ *
+ * train_codes [C][N][d*bits/8] with checkpoint stride train_ckpt_stride_bytes (>= N*d*bits/8, multiple
+ * of 16); val_codes likewise with V. train_scales [C][N], val_scales [C][V]. train_sumsq / val_sumsq
+ * [C][N] / [C][V] int32 as produced by qless_project_quantize; NULL = recomputed from the codes.
+ * lr_weights: host [C] (eta_i, used as given). task_offsets: host [T+1], strictly increasing,
+ * [0] = 0, [T] = V. scores [N] fp32; per_task [N, T] fp32 or NULL.
+ * Requirements: d % 128 == 0, d <= 8192; 1 <= V <= 4096; 1 <= T <= 64; 1 <= C <= 64.
+ * ------------------------------------------------------------------------------------------ */
+typedef enum { QLESS_SCORE_COSINE = 0, QLESS_SCORE_DEQUANT = 1 } qless_score_mode;
+
+size_t qless_score_workspace(int64_t N, int32_t V, int32_t C, int32_t T, int32_t d, int32_t bits);
+
+qless_status qless_score(
+    const void* train_codes, int64_t train_ckpt_stride_bytes,
+    const void* val_codes, int64_t val_ckpt_stride_bytes,
+    const float* train_scales, const float* val_scales,
+    const int32_t* train_sumsq, const int32_t* val_sumsq,
+    const float* lr_weights /* host */, const int32_t* task_offsets /* host */,
+    int64_t N, int32_t V, int32_t C, int32_t T, int32_t d, int32_t bits, qless_score_mode mode,
+    float* scores, float* per_task,
+    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* The integer numerators alone, for one checkpoint: dots [nt, V] int32 = D[t0 + t, v] computed by the
+ * same kernels that feed qless_score. train_codes [>= t0+nt, d*bits/8], val_codes [V, d*bits/8]. */
+size_t qless_score_dots_workspace(int64_t nt, int32_t V, int32_t d, int32_t bits);
+
+qless_status qless_score_dots(
+    const void* train_codes, const void* val_codes, int64_t t0, int64_t nt, int32_t V,
+    int32_t d, int32_t bits, int32_t* dots, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Stage 4: top-k selection ("Select the top 5% of training data", Sec. 4.1).
+ *
+ *   k = floor(frac * N + 1e-6) clamped to [0, N], written to *k_out (host) before the call returns.
+ *   Total order on fp32: by value, -0 below +0, every NaN below -inf; equal scores are admitted by
+ *   ascending index. indices [k] int64 receives the selected indices in ascending order.
+ * Requirements: 0 <= frac <= 1; N < 2^31.
+ * ------------------------------------------------------------------------------------------ */
+size_t qless_select_topk_workspace(int64_t N);
+
+qless_status qless_select_topk(
+    const float* scores, int64_t N, double frac, int64_t* indices, int64_t* k_out /* host */,
+    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QLESS_H_ */
