@@ -1,0 +1,363 @@
+// C ABI of the QLESS library: argument validation, workspace carving and kernel sequencing.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <vector>
+
+#include "qless_kernels.h"
+
+namespace qless {
+
+static thread_local char t_err[512] = "";
+
+qless_status fail(qless_status st, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(t_err, sizeof(t_err), fmt, ap);
+    va_end(ap);
+    return st;
+}
+
+qless_status cuda_fail(cudaError_t e, const char* what)
+{
+    snprintf(t_err, sizeof(t_err), "CUDA error %d (%s) in %s", (int)e, cudaGetErrorString(e), what);
+    return QLESS_ERR_CUDA;
+}
+
+int sm_count()
+{
+    static thread_local int cached_dev = -1, cached = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (dev != cached_dev) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached = n; cached_dev = dev;
+    }
+    return cached;
+}
+
+__device__ unsigned int g_timeout_flag = 0;
+
+unsigned int* timeout_flag_ptr()
+{
+    static thread_local int cached_dev = -1;
+    static thread_local unsigned int* p = nullptr;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev != cached_dev || p == nullptr) {
+        void* q = nullptr;
+        if (cudaGetSymbolAddress(&q, g_timeout_flag) != cudaSuccess) return nullptr;
+        p = reinterpret_cast<unsigned int*>(q); cached_dev = dev;
+    }
+    return p;
+}
+
+static bool valid_bits(int b) { return b == 1 || b == 2 || b == 4 || b == 8; }
+static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+static qless_status make_adam(const qless_adam_cfg* cfg, AdamParams* ap)
+{
+    qless_adam_cfg c = {0.9f, 0.999f, 1e-8f, 0};
+    if (cfg) c = *cfg;
+    QLESS_REQUIRE(c.beta1 >= 0.f && c.beta1 < 1.f && c.beta2 >= 0.f && c.beta2 < 1.f && c.eps >= 0.f && c.step >= 0,
+                  QLESS_ERR_INVALID_ARG, "adam config out of range (beta in [0,1), eps >= 0, step >= 0)");
+    ap->beta1 = c.beta1; ap->beta2 = c.beta2; ap->eps = c.eps;
+    ap->omb1 = 1.0f - c.beta1; ap->omb2 = 1.0f - c.beta2;
+    ap->bias_correct = c.step > 0;
+    ap->c1 = ap->c2 = 1.0f;
+    if (c.step > 0) {
+        ap->c1 = (float)(1.0 - std::pow((double)c.beta1, (double)c.step));
+        ap->c2 = (float)(1.0 - std::pow((double)c.beta2, (double)c.step));
+    }
+    return QLESS_OK;
+}
+
+static qless_status check_grads(const void* grads, qless_dtype dtype, int64_t n, int64_t ld, const float* m,
+                                const float* v, int64_t P)
+{
+    QLESS_REQUIRE(n >= 0 && P > 0, QLESS_ERR_INVALID_ARG, "n must be >= 0 and P > 0 (n=%lld, P=%lld)", (long long)n, (long long)P);
+    QLESS_REQUIRE(dtype == QLESS_F32 || dtype == QLESS_BF16, QLESS_ERR_INVALID_ARG, "dtype must be QLESS_F32 or QLESS_BF16");
+    QLESS_REQUIRE(P % 128 == 0, QLESS_ERR_UNSUPPORTED, "P must be a multiple of 128 (P=%lld)", (long long)P);
+    QLESS_REQUIRE(P < ((int64_t)1 << 39), QLESS_ERR_UNSUPPORTED, "P must be < 2^39");
+    QLESS_REQUIRE((m == nullptr) == (v == nullptr), QLESS_ERR_INVALID_ARG, "adam_m and adam_v must both be given or both be NULL");
+    if (n == 0) return QLESS_OK;
+    QLESS_REQUIRE(grads != nullptr, QLESS_ERR_INVALID_ARG, "grads is NULL");
+    QLESS_REQUIRE(ld >= P && ld % 8 == 0, QLESS_ERR_INVALID_ARG, "ld_grads must be >= P and a multiple of 8 (ld=%lld)", (long long)ld);
+    QLESS_REQUIRE(aligned(grads, 16) && aligned(m, 16) && aligned(v, 16), QLESS_ERR_INVALID_ARG, "grads, adam_m, adam_v must be 16-byte aligned");
+    return QLESS_OK;
+}
+
+struct PqWorkspace {
+    size_t gamma_off, part_off, total;
+    ProjectPlan plan;
+};
+
+static PqWorkspace pq_layout(int64_t n, int64_t P, int32_t d)
+{
+    PqWorkspace w;
+    w.plan = plan_projection(n, P, d);
+    w.gamma_off = 0;
+    w.part_off = align_up((size_t)n * (size_t)P * sizeof(__nv_bfloat16), 256);
+    w.total = w.part_off + align_up((size_t)w.plan.num_chunks * (size_t)n * (size_t)d * sizeof(float), 256);
+    return w;
+}
+
+}  // namespace qless
+
+using namespace qless;
+
+extern "C" {
+
+const char* qless_last_error(void) { return t_err; }
+
+qless_status qless_check(void* cuda_stream)
+{
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    unsigned int* flag = timeout_flag_ptr();
+    QLESS_REQUIRE(flag != nullptr, QLESS_ERR_CUDA, "cannot resolve the device timeout flag");
+    unsigned int h = 0;
+    QLESS_CUDA_TRY(cudaMemcpyAsync(&h, flag, sizeof(h), cudaMemcpyDeviceToHost, st));
+    QLESS_CUDA_TRY(cudaStreamSynchronize(st));
+    if (h != 0) {
+        QLESS_CUDA_TRY(cudaMemsetAsync(flag, 0, sizeof(h), st));
+        QLESS_CUDA_TRY(cudaStreamSynchronize(st));
+        return fail(QLESS_ERR_TIMEOUT, "a device-side bounded wait gave up (code 0x%x); results of that call are invalid", h);
+    }
+    return QLESS_OK;
+}
+
+size_t qless_project_quantize_workspace(int64_t n, int64_t P, int32_t d, int32_t bits)
+{
+    (void)bits;
+    if (n <= 0 || P <= 0 || d <= 0) return 256;
+    return pq_layout(n, P, d).total;
+}
+
+qless_status qless_project_quantize(const void* grads, qless_dtype dtype, int64_t n, int64_t ld_grads,
+                                    const float* adam_m, const float* adam_v, const qless_adam_cfg* adam,
+                                    int64_t P, int32_t d, uint64_t seed, int32_t bits, void* codes, float* scales,
+                                    int32_t* code_sumsq, float* proj_out, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream)
+{
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    qless_status s = check_grads(grads, dtype, n, ld_grads, adam_m, adam_v, P);
+    if (s != QLESS_OK) return s;
+    QLESS_REQUIRE(valid_bits(bits), QLESS_ERR_UNSUPPORTED, "bits must be 1, 2, 4 or 8 (bits=%d)", bits);
+    QLESS_REQUIRE(d >= 128 && d <= 8192 && d % 128 == 0, QLESS_ERR_UNSUPPORTED, "d must be a multiple of 128 in [128, 8192] (d=%d)", d);
+    AdamParams ap;
+    s = make_adam(adam, &ap);
+    if (s != QLESS_OK) return s;
+    if (n == 0) return QLESS_OK;
+    QLESS_REQUIRE(codes != nullptr && scales != nullptr, QLESS_ERR_INVALID_ARG, "codes and scales are required");
+    QLESS_REQUIRE(aligned(codes, 16) && aligned(proj_out, 16), QLESS_ERR_INVALID_ARG, "codes and proj_out must be 16-byte aligned");
+    const PqWorkspace w = pq_layout(n, P, d);
+    QLESS_REQUIRE(workspace != nullptr && aligned(workspace, 256), QLESS_ERR_WORKSPACE, "workspace must be non-NULL and 256-byte aligned");
+    QLESS_REQUIRE(workspace_bytes >= w.total, QLESS_ERR_WORKSPACE, "workspace too small: %zu bytes given, %zu needed", workspace_bytes, w.total);
+
+    uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+    const __nv_bfloat16* gamma;
+    int64_t ld = P;
+    if (dtype == QLESS_BF16 && adam_m == nullptr) {
+        gamma = reinterpret_cast<const __nv_bfloat16*>(grads);       // Gamma = g, already bf16
+        ld = ld_grads;
+    } else {
+        __nv_bfloat16* gbuf = reinterpret_cast<__nv_bfloat16*>(ws + w.gamma_off);
+        QLESS_CUDA_TRY(launch_adam_gamma(grads, dtype, n, ld_grads, adam_m, adam_v, ap, P, gbuf, st));
+        gamma = gbuf;
+    }
+    float* part = reinterpret_cast<float*>(ws + w.part_off);
+    QLESS_CUDA_TRY(launch_project_simt(gamma, ld, w.plan, seed, part, st));
+    const float inv_sqrt_d = 1.0f / sqrtf((float)d);
+    QLESS_CUDA_TRY(launch_quantize(part, w.plan.num_chunks, inv_sqrt_d, n, d, 1, bits, codes, scales, code_sumsq, proj_out, st));
+    return QLESS_OK;
+}
+
+qless_status qless_quantize(const float* x, int64_t n, int32_t d, int32_t normalize, int32_t bits, void* codes,
+                            float* scales, int32_t* code_sumsq, void* cuda_stream)
+{
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    QLESS_REQUIRE(n >= 0, QLESS_ERR_INVALID_ARG, "n must be >= 0");
+    QLESS_REQUIRE(valid_bits(bits), QLESS_ERR_UNSUPPORTED, "bits must be 1, 2, 4 or 8 (bits=%d)", bits);
+    QLESS_REQUIRE(d >= 128 && d <= 8192 && d % 128 == 0, QLESS_ERR_UNSUPPORTED, "d must be a multiple of 128 in [128, 8192] (d=%d)", d);
+    if (n == 0) return QLESS_OK;
+    QLESS_REQUIRE(x != nullptr && codes != nullptr && scales != nullptr, QLESS_ERR_INVALID_ARG, "x, codes and scales are required");
+    QLESS_REQUIRE(aligned(x, 16) && aligned(codes, 16), QLESS_ERR_INVALID_ARG, "x and codes must be 16-byte aligned");
+    QLESS_CUDA_TRY(launch_quantize(x, 1, 1.0f, n, d, normalize ? 1 : 0, bits, codes, scales, code_sumsq, nullptr, st));
+    return QLESS_OK;
+}
+
+qless_status qless_adam_gamma(const void* grads, qless_dtype dtype, int64_t n, int64_t ld_grads, const float* adam_m,
+                              const float* adam_v, const qless_adam_cfg* adam, int64_t P, void* gamma_out,
+                              void* cuda_stream)
+{
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    qless_status s = check_grads(grads, dtype, n, ld_grads, adam_m, adam_v, P);
+    if (s != QLESS_OK) return s;
+    AdamParams ap;
+    s = make_adam(adam, &ap);
+    if (s != QLESS_OK) return s;
+    if (n == 0) return QLESS_OK;
+    QLESS_REQUIRE(gamma_out != nullptr && aligned(gamma_out, 16), QLESS_ERR_INVALID_ARG, "gamma_out must be non-NULL and 16-byte aligned");
+    QLESS_CUDA_TRY(launch_adam_gamma(grads, dtype, n, ld_grads, adam_m, adam_v, ap, P,
+                                     reinterpret_cast<__nv_bfloat16*>(gamma_out), st));
+    return QLESS_OK;
+}
+
+qless_status qless_philox_entries(uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj, int8_t* out,
+                                  void* cuda_stream)
+{
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    QLESS_REQUIRE(r0 >= 0 && nr >= 0 && j0 >= 0 && nj >= 0, QLESS_ERR_INVALID_ARG, "negative range");
+    QLESS_REQUIRE(r0 + nr <= ((int64_t)1 << 32) && j0 + nj <= ((int64_t)1 << 39), QLESS_ERR_UNSUPPORTED, "row < 2^32 and column < 2^39 required");
+    if (nr == 0 || nj == 0) return QLESS_OK;
+    QLESS_REQUIRE(out != nullptr, QLESS_ERR_INVALID_ARG, "out is NULL");
+    QLESS_CUDA_TRY(launch_philox_entries(seed, r0, nr, j0, nj, out, st));
+    return QLESS_OK;
+}
+
+// ---- scoring -----------------------------------------------------------------------------------
+
+static qless_status check_score_shape(int64_t N, int32_t V, int32_t d, int32_t bits)
+{
+    QLESS_REQUIRE(N >= 0, QLESS_ERR_INVALID_ARG, "N must be >= 0");
+    QLESS_REQUIRE(valid_bits(bits), QLESS_ERR_UNSUPPORTED, "bits must be 1, 2, 4 or 8 (bits=%d)", bits);
+    QLESS_REQUIRE(d >= 128 && d <= 8192 && d % 128 == 0, QLESS_ERR_UNSUPPORTED, "d must be a multiple of 128 in [128, 8192] (d=%d)", d);
+    QLESS_REQUIRE(V >= 1 && V <= 4096, QLESS_ERR_UNSUPPORTED, "V must be in [1, 4096] (V=%d)", V);
+    return QLESS_OK;
+}
+
+struct ScoreWs { size_t tmult, vmult, eta, off, total; };
+static ScoreWs score_layout(int64_t N, int32_t V, int32_t C, int32_t T)
+{
+    ScoreWs w;
+    w.tmult = 0;
+    w.vmult = w.tmult + align_up((size_t)C * (size_t)N * 4, 256);
+    w.eta = w.vmult + align_up((size_t)C * (size_t)V * 4, 256);
+    w.off = w.eta + align_up((size_t)C * (size_t)T * 4, 256);
+    w.total = w.off + align_up((size_t)(T + 1) * 4, 256);
+    return w;
+}
+
+size_t qless_score_workspace(int64_t N, int32_t V, int32_t C, int32_t T, int32_t d, int32_t bits)
+{
+    (void)d; (void)bits;
+    if (N < 0 || V <= 0 || C <= 0 || T <= 0) return 256;
+    return score_layout(N, V, C, T).total;
+}
+
+qless_status qless_score(const void* train_codes, int64_t train_ckpt_stride_bytes, const void* val_codes,
+                         int64_t val_ckpt_stride_bytes, const float* train_scales, const float* val_scales,
+                         const int32_t* train_sumsq, const int32_t* val_sumsq, const float* lr_weights,
+                         const int32_t* task_offsets, int64_t N, int32_t V, int32_t C, int32_t T, int32_t d,
+                         int32_t bits, qless_score_mode mode, float* scores, float* per_task, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream)
+{
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    qless_status s = check_score_shape(N, V, d, bits);
+    if (s != QLESS_OK) return s;
+    QLESS_REQUIRE(C >= 1 && C <= 64, QLESS_ERR_UNSUPPORTED, "C must be in [1, 64] (C=%d)", C);
+    QLESS_REQUIRE(T >= 1 && T <= 64, QLESS_ERR_UNSUPPORTED, "T must be in [1, 64] (T=%d)", T);
+    QLESS_REQUIRE(mode == QLESS_SCORE_COSINE || mode == QLESS_SCORE_DEQUANT, QLESS_ERR_INVALID_ARG, "unknown score mode");
+    QLESS_REQUIRE(lr_weights != nullptr && task_offsets != nullptr, QLESS_ERR_INVALID_ARG, "lr_weights and task_offsets (host) are required");
+    QLESS_REQUIRE(task_offsets[0] == 0 && task_offsets[T] == V, QLESS_ERR_INVALID_ARG, "task_offsets must start at 0 and end at V");
+    for (int j = 0; j < T; ++j)
+        QLESS_REQUIRE(task_offsets[j + 1] > task_offsets[j], QLESS_ERR_INVALID_ARG, "task_offsets must be strictly increasing (task %d)", j);
+    const int64_t row_bytes = (int64_t)d * bits / 8;
+    QLESS_REQUIRE(train_ckpt_stride_bytes >= N * row_bytes && train_ckpt_stride_bytes % 16 == 0 &&
+                  val_ckpt_stride_bytes >= V * row_bytes && val_ckpt_stride_bytes % 16 == 0,
+                  QLESS_ERR_INVALID_ARG, "checkpoint strides must cover a checkpoint and be multiples of 16");
+    if (N == 0) return QLESS_OK;
+    QLESS_REQUIRE(train_codes && val_codes && train_scales && val_scales && scores, QLESS_ERR_INVALID_ARG, "codes, scales and scores are required");
+    QLESS_REQUIRE(aligned(train_codes, 16) && aligned(val_codes, 16), QLESS_ERR_INVALID_ARG, "code arrays must be 16-byte aligned");
+    const ScoreWs w = score_layout(N, V, C, T);
+    QLESS_REQUIRE(workspace != nullptr && aligned(workspace, 256), QLESS_ERR_WORKSPACE, "workspace must be non-NULL and 256-byte aligned");
+    QLESS_REQUIRE(workspace_bytes >= w.total, QLESS_ERR_WORKSPACE, "workspace too small: %zu bytes given, %zu needed", workspace_bytes, w.total);
+
+    uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+    float* tmult = reinterpret_cast<float*>(ws + w.tmult);
+    float* vmult = reinterpret_cast<float*>(ws + w.vmult);
+    float* d_eta = reinterpret_cast<float*>(ws + w.eta);
+    int32_t* d_off = reinterpret_cast<int32_t*>(ws + w.off);
+
+    std::vector<float> eoc((size_t)C * T);
+    for (int i = 0; i < C; ++i)
+        for (int j = 0; j < T; ++j)
+            eoc[(size_t)i * T + j] = lr_weights[i] / (float)(task_offsets[j + 1] - task_offsets[j]);
+    // pageable host sources: the runtime stages them before returning, so the vectors may die here
+    QLESS_CUDA_TRY(cudaMemcpyAsync(d_eta, eoc.data(), eoc.size() * 4, cudaMemcpyHostToDevice, st));
+    QLESS_CUDA_TRY(cudaMemcpyAsync(d_off, task_offsets, (size_t)(T + 1) * 4, cudaMemcpyHostToDevice, st));
+    QLESS_CUDA_TRY(launch_multipliers(reinterpret_cast<const uint8_t*>(train_codes), train_ckpt_stride_bytes, train_scales,
+                                      train_sumsq, N, C, d, bits, (int)mode, tmult, st));
+    QLESS_CUDA_TRY(launch_multipliers(reinterpret_cast<const uint8_t*>(val_codes), val_ckpt_stride_bytes, val_scales,
+                                      val_sumsq, V, C, d, bits, (int)mode, vmult, st));
+    ScoreArgs a;
+    a.train = reinterpret_cast<const uint8_t*>(train_codes); a.train_stride = train_ckpt_stride_bytes;
+    a.val = reinterpret_cast<const uint8_t*>(val_codes); a.val_stride = val_ckpt_stride_bytes;
+    a.train_mult = tmult; a.val_mult = vmult; a.eta_over_cnt = d_eta; a.task_off = d_off;
+    a.N = N; a.V = V; a.C = C; a.T = T; a.d = d; a.bits = bits;
+    a.scores = scores; a.per_task = per_task; a.dots = nullptr;
+    QLESS_CUDA_TRY(launch_score_simt(a, st));
+    return QLESS_OK;
+}
+
+size_t qless_score_dots_workspace(int64_t nt, int32_t V, int32_t d, int32_t bits)
+{
+    (void)nt; (void)V; (void)d; (void)bits;
+    return 256;
+}
+
+qless_status qless_score_dots(const void* train_codes, const void* val_codes, int64_t t0, int64_t nt, int32_t V,
+                              int32_t d, int32_t bits, int32_t* dots, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream)
+{
+    (void)workspace; (void)workspace_bytes;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    qless_status s = check_score_shape(nt, V, d, bits);
+    if (s != QLESS_OK) return s;
+    QLESS_REQUIRE(t0 >= 0, QLESS_ERR_INVALID_ARG, "t0 must be >= 0");
+    if (nt == 0) return QLESS_OK;
+    QLESS_REQUIRE(train_codes && val_codes && dots, QLESS_ERR_INVALID_ARG, "train_codes, val_codes and dots are required");
+    QLESS_REQUIRE(aligned(train_codes, 16) && aligned(val_codes, 16), QLESS_ERR_INVALID_ARG, "code arrays must be 16-byte aligned");
+    const int64_t row_bytes = (int64_t)d * bits / 8;
+    ScoreArgs a;
+    a.train = reinterpret_cast<const uint8_t*>(train_codes) + t0 * row_bytes; a.train_stride = 0;
+    a.val = reinterpret_cast<const uint8_t*>(val_codes); a.val_stride = 0;
+    a.train_mult = nullptr; a.val_mult = nullptr; a.eta_over_cnt = nullptr; a.task_off = nullptr;
+    a.N = nt; a.V = V; a.C = 1; a.T = 1; a.d = d; a.bits = bits;
+    a.scores = nullptr; a.per_task = nullptr; a.dots = dots;
+    QLESS_CUDA_TRY(launch_score_simt(a, st));
+    return QLESS_OK;
+}
+
+// ---- selection ---------------------------------------------------------------------------------
+
+size_t qless_select_topk_workspace(int64_t N) { return select_workspace_bytes(N); }
+
+qless_status qless_select_topk(const float* scores, int64_t N, double frac, int64_t* indices, int64_t* k_out,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    QLESS_REQUIRE(N >= 0 && N < ((int64_t)1 << 31), QLESS_ERR_INVALID_ARG, "N must be in [0, 2^31)");
+    QLESS_REQUIRE(frac >= 0.0 && frac <= 1.0, QLESS_ERR_INVALID_ARG, "frac must be in [0, 1]");   // also rejects NaN
+    QLESS_REQUIRE(k_out != nullptr, QLESS_ERR_INVALID_ARG, "k_out (host) is required");
+    double kf = std::floor(frac * (double)N + 1e-6);
+    if (kf < 0.0) kf = 0.0;
+    if (kf > (double)N) kf = (double)N;
+    const int64_t k = (int64_t)kf;
+    if (k > 0) {
+        QLESS_REQUIRE(scores != nullptr && indices != nullptr, QLESS_ERR_INVALID_ARG, "scores and indices are required");
+        QLESS_REQUIRE(aligned(scores, 16), QLESS_ERR_INVALID_ARG, "scores must be 16-byte aligned");
+        QLESS_REQUIRE(workspace != nullptr && aligned(workspace, 256), QLESS_ERR_WORKSPACE, "workspace must be non-NULL and 256-byte aligned");
+        QLESS_REQUIRE(workspace_bytes >= select_workspace_bytes(N), QLESS_ERR_WORKSPACE, "workspace too small: %zu bytes given, %zu needed",
+                      workspace_bytes, select_workspace_bytes(N));
+    }
+    *k_out = k;
+    if (k == 0) return QLESS_OK;
+    QLESS_CUDA_TRY(launch_select_topk(scores, N, k, indices, workspace, st));
+    return QLESS_OK;
+}
+
+}  // extern "C"

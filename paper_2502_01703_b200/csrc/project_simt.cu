@@ -1,0 +1,98 @@
+// Projection (Eq. 1) on the CUDA cores: a plain tiled kernel used for shapes the tensor-core kernel
+// does not take. part[s][i][r] = sum_{j in chunk s} Gamma[i][j] * sign(r, j).
+#include "qless_kernels.h"
+
+namespace qless {
+
+namespace {
+
+constexpr int PS_DR = 64;     // projected rows per block
+constexpr int PS_GR = 32;     // gradient rows per block
+constexpr int PS_T = 256;
+
+__global__ void __launch_bounds__(PS_T)
+project_simt_kernel(const __nv_bfloat16* __restrict__ gamma, int64_t ld, int64_t n, int64_t P, int32_t d,
+                    int64_t chunk, uint64_t seed, float* __restrict__ part)
+{
+    __shared__ __align__(16) float s_g[PS_GR][128];
+    const int tid = threadIdx.x;
+    const int tr = tid & (PS_DR - 1), ti = tid >> 6;           // ti = 0..3, 8 gradient rows each
+    const uint32_t r = blockIdx.x * PS_DR + tr;
+    const int64_t i0 = (int64_t)blockIdx.y * PS_GR;
+    const int64_t k0 = (int64_t)blockIdx.z * chunk;
+    const int64_t k1 = min(P, k0 + chunk);
+    float acc[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc[u] = 0.0f;
+
+    for (int64_t kb = k0; kb < k1; kb += 128) {
+        __syncthreads();
+        // 32 rows x 128 columns of Gamma -> fp32 in shared memory (rows >= n read as zero)
+        for (int e = tid; e < PS_GR * 64; e += PS_T) {
+            const int row = e >> 6, cp = e & 63;
+            float2 f = make_float2(0.f, 0.f);
+            if (i0 + row < n) {
+                const uint32_t w = *reinterpret_cast<const uint32_t*>(gamma + (i0 + row) * ld + kb + 2 * cp);
+                f.x = __uint_as_float(w << 16);
+                f.y = __uint_as_float(w & 0xFFFF0000u);
+            }
+            *reinterpret_cast<float2*>(&s_g[row][2 * cp]) = f;
+        }
+        __syncthreads();
+        uint32_t w[4];
+        rademacher_block(seed, r, (uint32_t)(kb >> 7), w);
+#pragma unroll
+        for (int wi = 0; wi < 4; ++wi) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {               // 4 columns at a time
+                uint32_t sm[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int u = q * 4 + c;
+                    const int beta = 15 - (u >> 1) + 16 * (u & 1);
+                    sm[c] = ((w[wi] >> beta) & 1u) << 31;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const float4 g = *reinterpret_cast<const float4*>(&s_g[ti * 8 + u][wi * 32 + q * 4]);
+                    acc[u] += __uint_as_float(__float_as_uint(g.x) ^ sm[0]);
+                    acc[u] += __uint_as_float(__float_as_uint(g.y) ^ sm[1]);
+                    acc[u] += __uint_as_float(__float_as_uint(g.z) ^ sm[2]);
+                    acc[u] += __uint_as_float(__float_as_uint(g.w) ^ sm[3]);
+                }
+            }
+        }
+    }
+    float* out = part + (int64_t)blockIdx.z * n * d;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const int64_t i = i0 + ti * 8 + u;
+        if (i < n) out[i * d + r] = acc[u];
+    }
+}
+
+}  // namespace
+
+ProjectPlan plan_projection(int64_t n, int64_t P, int32_t d)
+{
+    ProjectPlan pl;
+    pl.n = n; pl.P = P; pl.d = d;
+    int64_t chunk = P < 32768 ? P : 32768;
+    const int64_t tiles = (int64_t)(d / 128) * ((n + 255) / 256);
+    while (chunk > 2048 && chunk % 256 == 0 && tiles * ((P + chunk - 1) / chunk) < 2 * (int64_t)sm_count())
+        chunk >>= 1;
+    pl.chunk = chunk;
+    pl.num_chunks = (int32_t)((P + chunk - 1) / chunk);
+    return pl;
+}
+
+cudaError_t launch_project_simt(const __nv_bfloat16* gamma, int64_t ld, const ProjectPlan& pl, uint64_t seed,
+                                float* part, cudaStream_t st)
+{
+    if (pl.n == 0) return cudaSuccess;
+    dim3 grid((unsigned)(pl.d / PS_DR), (unsigned)((pl.n + PS_GR - 1) / PS_GR), (unsigned)pl.num_chunks);
+    project_simt_kernel<<<grid, PS_T, 0, st>>>(gamma, ld, pl.n, pl.P, pl.d, pl.chunk, seed, part);
+    return cudaGetLastError();
+}
+
+}  // namespace qless

@@ -1,0 +1,111 @@
+// Adam prologue (Gamma) and the stand-alone generator of projection-matrix entries.
+#include "qless_kernels.h"
+
+namespace qless {
+
+// Gamma_j = m'/(sqrt(v')+eps), m' = b1 m + (1-b1) g, v' = b2 v + (1-b2) g^2, every operation a
+// separately rounded IEEE fp32 operation (no fused multiply-add), result rounded to bf16 (RNE).
+__device__ __forceinline__ float adam_dir(float g, float m, float v, const AdamParams& ap)
+{
+    float m1 = __fadd_rn(__fmul_rn(ap.beta1, m), __fmul_rn(ap.omb1, g));
+    float v1 = __fadd_rn(__fmul_rn(ap.beta2, v), __fmul_rn(ap.omb2, __fmul_rn(g, g)));
+    if (ap.bias_correct) { m1 = __fdiv_rn(m1, ap.c1); v1 = __fdiv_rn(v1, ap.c2); }
+    const float den = __fadd_rn(__fsqrt_rn(v1), ap.eps);
+    return __fdiv_rn(m1, den);
+}
+
+// One thread handles 8 consecutive columns of one row: 16-byte bf16 loads/stores, 2x16-byte fp32.
+template <bool BF16_IN, bool ADAM>
+__global__ void __launch_bounds__(256)
+adam_gamma_kernel(const void* __restrict__ grads, int64_t n, int64_t ld, const float* __restrict__ m,
+                  const float* __restrict__ v, AdamParams ap, int64_t P, __nv_bfloat16* __restrict__ gamma)
+{
+    const int64_t groups_per_row = P >> 3;
+    const int64_t total = n * groups_per_row;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = idx / groups_per_row;
+        const int64_t j0 = (idx - row * groups_per_row) << 3;
+        float g[8];
+        if (BF16_IN) {
+            const uint4 raw = *reinterpret_cast<const uint4*>(
+                reinterpret_cast<const __nv_bfloat16*>(grads) + row * ld + j0);
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                g[2 * k] = __uint_as_float(w[k] << 16);
+                g[2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u);
+            }
+        } else {
+            const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(grads) + row * ld + j0);
+            const float4 a = p[0], b = p[1];
+            g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w; g[4] = b.x; g[5] = b.y; g[6] = b.z; g[7] = b.w;
+        }
+        if (ADAM) {
+            const float4 m0 = *reinterpret_cast<const float4*>(m + j0), m1 = *reinterpret_cast<const float4*>(m + j0 + 4);
+            const float4 v0 = *reinterpret_cast<const float4*>(v + j0), v1 = *reinterpret_cast<const float4*>(v + j0 + 4);
+            const float mm[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+            const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+            for (int k = 0; k < 8; ++k) g[k] = adam_dir(g[k], mm[k], vv[k], ap);
+        }
+        uint32_t o[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const __nv_bfloat162 pr = __floats2bfloat162_rn(g[2 * k], g[2 * k + 1]);
+            o[k] = *reinterpret_cast<const uint32_t*>(&pr);
+        }
+        *reinterpret_cast<uint4*>(gamma + row * P + j0) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+cudaError_t launch_adam_gamma(const void* grads, qless_dtype dtype, int64_t n, int64_t ld, const float* m,
+                              const float* v, const AdamParams& ap, int64_t P, __nv_bfloat16* gamma,
+                              cudaStream_t st)
+{
+    if (n == 0 || P == 0) return cudaSuccess;
+    const int64_t total = n * (P >> 3);
+    const int threads = 256;
+    int64_t blocks = (total + threads - 1) / threads;
+    const int64_t cap = (int64_t)sm_count() * 16;
+    if (blocks > cap) blocks = cap;
+    const bool adam = (m != nullptr);
+    if (dtype == QLESS_BF16) {
+        if (adam) adam_gamma_kernel<true, true><<<(unsigned)blocks, threads, 0, st>>>(grads, n, ld, m, v, ap, P, gamma);
+        else adam_gamma_kernel<true, false><<<(unsigned)blocks, threads, 0, st>>>(grads, n, ld, m, v, ap, P, gamma);
+    } else {
+        if (adam) adam_gamma_kernel<false, true><<<(unsigned)blocks, threads, 0, st>>>(grads, n, ld, m, v, ap, P, gamma);
+        else adam_gamma_kernel<false, false><<<(unsigned)blocks, threads, 0, st>>>(grads, n, ld, m, v, ap, P, gamma);
+    }
+    return cudaGetLastError();
+}
+
+// out[a][b] = sign(r0 + a, j0 + b) as int8.
+__global__ void philox_entries_kernel(uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj,
+                                      int8_t* __restrict__ out)
+{
+    const int64_t total = nr * nj;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t a = idx / nj, b = idx - a * nj;
+        const uint64_t j = (uint64_t)(j0 + b);
+        uint32_t w[4];
+        rademacher_block(seed, (uint32_t)(r0 + a), (uint32_t)(j >> 7), w);
+        const uint32_t t = (uint32_t)(j & 127u);
+        out[idx] = (int8_t)rademacher_sign_of(w[t >> 5], (int)(t & 31u));
+    }
+}
+
+cudaError_t launch_philox_entries(uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj, int8_t* out,
+                                  cudaStream_t st)
+{
+    const int64_t total = nr * nj;
+    if (total == 0) return cudaSuccess;
+    int64_t blocks = (total + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 16;
+    if (blocks > cap) blocks = cap;
+    philox_entries_kernel<<<(unsigned)blocks, 256, 0, st>>>(seed, r0, nr, j0, nj, out);
+    return cudaGetLastError();
+}
+
+}  // namespace qless

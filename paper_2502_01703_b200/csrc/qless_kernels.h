@@ -1,0 +1,64 @@
+// Internal launch interface between the C ABI (api.cu) and the kernel translation units.
+#pragma once
+#include "qless_common.cuh"
+
+namespace qless {
+
+struct AdamParams {
+    float beta1, beta2, eps;
+    float omb1, omb2;      // 1 - beta1, 1 - beta2 (fp32 subtraction, as written in the formula)
+    float c1, c2;          // bias-correction divisors (1 if step == 0)
+    int   bias_correct;
+};
+
+// Gamma[n, P] (bf16) from gradient rows; m/v NULL => bf16(g).
+cudaError_t launch_adam_gamma(const void* grads, qless_dtype dtype, int64_t n, int64_t ld,
+                              const float* m, const float* v, const AdamParams& ap, int64_t P,
+                              __nv_bfloat16* gamma, cudaStream_t st);
+
+cudaError_t launch_philox_entries(uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj,
+                                  int8_t* out, cudaStream_t st);
+
+// Projection partial sums: part[s][i][r] = sum over K-chunk s of Gamma[i][j] * sign(r, j), fp32,
+// s = 0 .. num_chunks-1, chunk s covering columns [s*chunk, min(P, (s+1)*chunk)).
+struct ProjectPlan {
+    int64_t n, P;
+    int32_t d;
+    int64_t chunk;        // K-chunk length (multiple of 128)
+    int32_t num_chunks;
+};
+ProjectPlan plan_projection(int64_t n, int64_t P, int32_t d);
+cudaError_t launch_project_simt(const __nv_bfloat16* gamma, int64_t ld, const ProjectPlan& pl,
+                                uint64_t seed, float* part, cudaStream_t st);
+
+// Stage 2. x = inv_scale-scaled sum of `num_parts` partial arrays [num_parts][n][d] (num_parts = 1,
+// scale = 1 for plain rows). Writes proj_out (optional), codes, scales, sumsq (optional).
+cudaError_t launch_quantize(const float* parts, int32_t num_parts, float scale, int64_t n, int32_t d,
+                            int normalize, int32_t bits, void* codes, float* scales, int32_t* sumsq,
+                            float* proj_out, cudaStream_t st);
+
+// Stage 3.
+struct ScoreArgs {
+    const uint8_t* train; int64_t train_stride;   // bytes per checkpoint
+    const uint8_t* val;   int64_t val_stride;
+    const float* train_mult;    // [C][N] per-vector multipliers
+    const float* val_mult;      // [C][V]
+    const float* eta_over_cnt;  // device [C][T]: eta_i / |task j|
+    const int32_t* task_off;    // device [T+1]
+    int64_t N; int32_t V, C, T, d, bits;
+    float* scores; float* per_task;
+    int32_t* dots;              // if non-NULL: write raw integer dots [N][V] of checkpoint 0 only
+};
+cudaError_t launch_score_simt(const ScoreArgs& a, cudaStream_t st);
+// multipliers: mult = (scale == 0) ? 0 : 1/sqrt(sumsq) (cosine) or scale/alpha (dequant);
+// sumsq NULL => recomputed from codes.
+cudaError_t launch_multipliers(const uint8_t* codes, int64_t ckpt_stride, const float* scales,
+                               const int32_t* sumsq, int64_t rows, int32_t C, int32_t d, int32_t bits,
+                               int mode, float* mult, cudaStream_t st);
+
+// Stage 4.
+size_t select_workspace_bytes(int64_t N);
+cudaError_t launch_select_topk(const float* scores, int64_t N, int64_t k, int64_t* indices,
+                               void* ws, cudaStream_t st);
+
+}  // namespace qless

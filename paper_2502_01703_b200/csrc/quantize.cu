@@ -1,0 +1,188 @@
+// Stage 2: (sum of projection partials) -> L2 normalise (Eq. 2) -> absmax b-bit codes (Eq. 4-5) -> pack.
+// HBM-bound: each row is read once (4*d bytes per partial) and d*b/8 + 8 bytes are written.
+#include "qless_kernels.h"
+
+namespace qless {
+
+namespace {
+
+constexpr int QT = 256;        // threads per row
+constexpr int QMAX_V4 = 8;     // float4 chunks per thread  => d <= 256 * 8 * 4 = 8192
+
+__device__ __forceinline__ double warp_sum(double x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
+    return x;
+}
+__device__ __forceinline__ float warp_max(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xFFFFFFFFu, x, o));
+    return x;
+}
+__device__ __forceinline__ int warp_sum_i(int x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
+    return x;
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(QT)
+quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale, int64_t n, int32_t d,
+                int normalize, uint8_t* __restrict__ codes, float* __restrict__ scales,
+                int32_t* __restrict__ sumsq, float* __restrict__ proj_out)
+{
+    __shared__ double s_d[QT / 32];
+    __shared__ float s_f[QT / 32];
+    __shared__ int s_i[QT / 32];
+    __shared__ __align__(16) uint8_t s_out[8192];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nv4 = d >> 2;                       // float4 chunks per row (multiple of 32)
+    const int64_t part_stride = n * (int64_t)d;
+    const int row_bytes = d * BITS / 8;
+
+    for (int64_t row = blockIdx.x; row < n; row += gridDim.x) {
+        float4 x[QMAX_V4];
+        // ---- load + fixed-order sum of partials, scaled once ----
+#pragma unroll
+        for (int k = 0; k < QMAX_V4; ++k) {
+            const int c = tid + k * QT;
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c < nv4) {
+                const float4* p = reinterpret_cast<const float4*>(parts + row * d) + c;
+                a = __ldcs(p);
+                for (int s = 1; s < num_parts; ++s) {
+                    const float4 b = __ldcs(reinterpret_cast<const float4*>(parts + s * part_stride + row * d) + c);
+                    a.x = __fadd_rn(a.x, b.x); a.y = __fadd_rn(a.y, b.y);
+                    a.z = __fadd_rn(a.z, b.z); a.w = __fadd_rn(a.w, b.w);
+                }
+                if (scale != 1.0f) {
+                    a.x = __fmul_rn(a.x, scale); a.y = __fmul_rn(a.y, scale);
+                    a.z = __fmul_rn(a.z, scale); a.w = __fmul_rn(a.w, scale);
+                }
+                if (proj_out) __stcs(reinterpret_cast<float4*>(proj_out + row * d) + c, a);
+            }
+            x[k] = a;
+        }
+        // ---- Eq. 2: norm in double, one fp32 reciprocal, one fp32 multiply per element ----
+        bool zero_vec = false;
+        if (normalize) {
+            double acc = 0.0;
+#pragma unroll
+            for (int k = 0; k < QMAX_V4; ++k) {
+                acc += (double)x[k].x * (double)x[k].x; acc += (double)x[k].y * (double)x[k].y;
+                acc += (double)x[k].z * (double)x[k].z; acc += (double)x[k].w * (double)x[k].w;
+            }
+            acc = warp_sum(acc);
+            if (lane == 0) s_d[warp] = acc;
+            __syncthreads();
+            double tot = 0.0;
+#pragma unroll
+            for (int w = 0; w < QT / 32; ++w) tot += s_d[w];
+            const float nrm = (float)sqrt(tot);
+            if (nrm == 0.0f) {
+                zero_vec = true;
+            } else {
+                const float rn = __fdiv_rn(1.0f, nrm);
+#pragma unroll
+                for (int k = 0; k < QMAX_V4; ++k) {
+                    x[k].x = __fmul_rn(x[k].x, rn); x[k].y = __fmul_rn(x[k].y, rn);
+                    x[k].z = __fmul_rn(x[k].z, rn); x[k].w = __fmul_rn(x[k].w, rn);
+                }
+            }
+        }
+        // ---- Eq. 4: S = max |x| ----
+        float mx = 0.0f;
+#pragma unroll
+        for (int k = 0; k < QMAX_V4; ++k)
+            mx = fmaxf(fmaxf(mx, fmaxf(fabsf(x[k].x), fabsf(x[k].y))), fmaxf(fabsf(x[k].z), fabsf(x[k].w)));
+        mx = warp_max(mx);
+        if (lane == 0) s_f[warp] = mx;
+        __syncthreads();
+        float S = 0.0f;
+#pragma unroll
+        for (int w = 0; w < QT / 32; ++w) S = fmaxf(S, s_f[w]);
+        if (zero_vec) S = 0.0f;
+
+        // ---- Eq. 5 + pack into shared memory ----
+        constexpr int ALPHA = (BITS == 1) ? 1 : ((1 << (BITS - 1)) - 1);
+        const float r = (S > 0.0f) ? __fdiv_rn((float)ALPHA, S) : 0.0f;
+        int ss = 0;
+#pragma unroll
+        for (int k = 0; k < QMAX_V4; ++k) {
+            const int c = tid + k * QT;
+            if (c < nv4) {      // warp-uniform: nv4 is a multiple of 32
+                const float e[4] = {x[k].x, x[k].y, x[k].z, x[k].w};
+                int q[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (BITS == 1) {
+                        q[u] = (S > 0.0f) ? ((e[u] < 0.0f) ? -1 : 1) : 0;
+                    } else {
+                        int t = __float2int_rn(__fmul_rn(e[u], r));
+                        t = max(-ALPHA, min(ALPHA, t));
+                        q[u] = t;
+                    }
+                    ss += q[u] * q[u];
+                }
+                if (BITS == 8) {
+                    const uint32_t w = (uint32_t)(q[0] & 0xFF) | ((uint32_t)(q[1] & 0xFF) << 8) |
+                                       ((uint32_t)(q[2] & 0xFF) << 16) | ((uint32_t)(q[3] & 0xFF) << 24);
+                    reinterpret_cast<uint32_t*>(s_out)[c] = w;
+                } else if (BITS == 4) {
+                    const uint32_t w = (uint32_t)(q[0] & 0xF) | ((uint32_t)(q[1] & 0xF) << 4) |
+                                       ((uint32_t)(q[2] & 0xF) << 8) | ((uint32_t)(q[3] & 0xF) << 12);
+                    reinterpret_cast<uint16_t*>(s_out)[c] = (uint16_t)w;
+                } else if (BITS == 2) {
+                    const uint32_t w = (uint32_t)(q[0] & 0x3) | ((uint32_t)(q[1] & 0x3) << 2) |
+                                       ((uint32_t)(q[2] & 0x3) << 4) | ((uint32_t)(q[3] & 0x3) << 6);
+                    s_out[c] = (uint8_t)w;
+                } else {
+                    uint32_t nib = (q[0] < 0 ? 1u : 0u) | (q[1] < 0 ? 2u : 0u) | (q[2] < 0 ? 4u : 0u) | (q[3] < 0 ? 8u : 0u);
+                    const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, nib, 1);
+                    if ((lane & 1) == 0) s_out[c >> 1] = (uint8_t)(nib | (hi << 4));
+                }
+            }
+        }
+        ss = warp_sum_i(ss);
+        if (lane == 0) s_i[warp] = ss;
+        __syncthreads();       // s_out and s_i complete
+        if (tid == 0) {
+            int tot = 0;
+#pragma unroll
+            for (int w = 0; w < QT / 32; ++w) tot += s_i[w];
+            scales[row] = S;
+            if (sumsq) sumsq[row] = tot;
+        }
+        // ---- 128-bit coalesced stores of the packed row ----
+        uint4* dst = reinterpret_cast<uint4*>(codes + row * (int64_t)row_bytes);
+        const uint4* src = reinterpret_cast<const uint4*>(s_out);
+        for (int i = tid; i < (row_bytes >> 4); i += QT) __stcs(dst + i, src[i]);
+        __syncthreads();       // before the next row reuses shared memory
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_quantize(const float* parts, int32_t num_parts, float scale, int64_t n, int32_t d,
+                            int normalize, int32_t bits, void* codes, float* scales, int32_t* sumsq,
+                            float* proj_out, cudaStream_t st)
+{
+    if (n == 0) return cudaSuccess;
+    int64_t blocks = n;
+    const int64_t cap = (int64_t)sm_count() * 8 * 4;
+    if (blocks > cap) blocks = cap;
+    uint8_t* c = reinterpret_cast<uint8_t*>(codes);
+    switch (bits) {
+        case 8: quantize_kernel<8><<<(unsigned)blocks, QT, 0, st>>>(parts, num_parts, scale, n, d, normalize, c, scales, sumsq, proj_out); break;
+        case 4: quantize_kernel<4><<<(unsigned)blocks, QT, 0, st>>>(parts, num_parts, scale, n, d, normalize, c, scales, sumsq, proj_out); break;
+        case 2: quantize_kernel<2><<<(unsigned)blocks, QT, 0, st>>>(parts, num_parts, scale, n, d, normalize, c, scales, sumsq, proj_out); break;
+        default: quantize_kernel<1><<<(unsigned)blocks, QT, 0, st>>>(parts, num_parts, scale, n, d, normalize, c, scales, sumsq, proj_out); break;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace qless
