@@ -1,0 +1,329 @@
+#!/usr/bin/env python
+"""Benchmark of the QLESS hot path: gradients projected + quantised per second at P = 2^23, d = 8192.
+
+One step = one batch of 256 bf16 per-example gradients through the whole path: Adam prologue ->
+Philox-Rademacher projection -> normalise -> 4-bit absmax codes (qless_project_quantize), then the
+batch's codes scored against a resident 448-vector validation store in 3 tasks (qless_score) and the
+top 5 % selected (qless_select_topk). Inputs are seeded synthetic data (Student-t(3) entries with
+lognormal row scales); the batch (4.3 GB) is far larger than L2, so no flush is needed between steps.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0). With --gpus N > 1 (launched by torch.distributed.run, one rank per
+GPU) every rank works on its own batches: weak scaling, no data-path collective.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOAD = "c2_project_quantize"
+N_VAL, TASKS, FRAC = 448, [64, 128, 256], 0.05
+SEED = 20250203
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_burst=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        sm.sort()
+        return dict(sm_mhz=sm[len(sm) // 2] if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def run_reference(args):
+    """The CPU oracle timed as it stands on a bounded sample of the same workload (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2502_01703_b200 import workloads as W
+    cfg = W.CONFIGS[WORKLOAD]
+    P, d, bits = cfg["P"], cfg["d"], cfg["bits"]
+    n_rows, n_coords = 1, 16
+    g = W.student_t_gradients(n_rows, P, seed=SEED, dtype=torch.bfloat16).float().numpy()
+    m, v = [t.numpy() for t in W.adam_moments(P, seed=SEED + 1)]
+    coords = np.arange(n_coords, dtype=np.int32) * (d // n_coords)
+
+    def step():
+        t0 = time.perf_counter()
+        gam = oracle.adam_gamma(g, m, v)
+        t1 = time.perf_counter()
+        y = oracle.project_rows(gam, d, SEED, coords)
+        t2 = time.perf_counter()
+        full = np.resize(y, (n_rows, d)).astype(np.float32)
+        oracle.quantize_rows(full, bits, normalize=True)
+        t3 = time.perf_counter()
+        # seconds one gradient would take through the full path (projection is linear in d)
+        return ((t1 - t0) + (t2 - t1) * (d / n_coords) + (t3 - t2)) / n_rows
+
+    for _ in range(args.warmup):
+        step()
+    per_grad = [step() for _ in range(args.steps)]
+    sec = sum(per_grad) / len(per_grad)
+    value = 1.0 / sec
+    sample = (f"{n_rows} gradient row(s) at full P=2^23 through Adam prologue, projection onto {n_coords} of {d} "
+              f"output coordinates (scaled x{d // n_coords}), normalise+quantise of a full row; single thread")
+    line = dict(impl="reference", metric="grads projected+quantized/s (P=2^23,d=8192)", value=value, unit="grads/s",
+                n_gpus=args.gpus, steps=args.steps, warmup=args.warmup, ms_per_step=sec * cfg["batch_rows"] * 1e3,
+                higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=WORKLOAD, batch_rows=cfg["batch_rows"], P=P, d=d, bits=bits),
+                cpu_baseline=dict(value=value, unit="grads/s", cores=1, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit="grads/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+def cpu_baseline():
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2502_01703_b200 import workloads as W
+    cfg = W.CONFIGS[WORKLOAD]
+    P, d, bits = cfg["P"], cfg["d"], cfg["bits"]
+    n_rows, n_coords = 4, 128
+    g = W.student_t_gradients(n_rows, P, seed=SEED, dtype=torch.bfloat16).float().numpy()
+    m, v = [t.numpy() for t in W.adam_moments(P, seed=SEED + 1)]
+    coords = np.arange(n_coords, dtype=np.int32) * (d // n_coords)
+    t0 = time.perf_counter()
+    gam = oracle.adam_gamma(g, m, v)
+    t1 = time.perf_counter()
+    y = oracle.project_rows(gam, d, SEED, coords)
+    t2 = time.perf_counter()
+    oracle.quantize_rows(np.resize(y, (n_rows, d)).astype(np.float32), bits, normalize=True)
+    t3 = time.perf_counter()
+    sec_per_grad = ((t1 - t0) + (t2 - t1) * (d / n_coords) + (t3 - t2)) / n_rows
+    return dict(value=1.0 / sec_per_grad, unit="grads/s", cores=1, kind="oracle",
+                sample=(f"{n_rows} gradient rows at full P=2^23, projection onto {n_coords} of {d} output coordinates "
+                        f"(scaled x{d // n_coords}; the work is linear in d), {t3 - t0:.1f} s of CPU time, single thread"))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2502_01703_b200 import binding as B
+    from paper_2502_01703_b200 import workloads as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus != world and world > 1:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    B.lib()    # fails loudly if the CUDA library is missing
+    cfg = W.CONFIGS[WORKLOAD]
+    n, P, d, bits = cfg["batch_rows"], cfg["P"], cfg["d"], cfg["bits"]
+    rb = d * bits // 8
+    off = W.task_offsets(TASKS).tolist()
+
+    # ---- synthetic inputs, resident in HBM before the timed region ----
+    g = W.student_t_gradients(n, P, seed=SEED + 100 * rank, device=dev, dtype=torch.bfloat16)
+    m, v = W.adam_moments(P, seed=SEED + 1, device=dev)
+    g_val = W.student_t_gradients(N_VAL, P, seed=SEED + 2, device=dev, dtype=torch.bfloat16)
+    ws = torch.empty(B.qless_project_quantize_workspace(max(n, 256), P, d, bits), dtype=torch.uint8, device=dev)
+    val_codes = torch.empty((1, N_VAL, rb), dtype=torch.uint8, device=dev)
+    val_scales = torch.empty((1, N_VAL), dtype=torch.float32, device=dev)
+    val_sumsq = torch.empty((1, N_VAL), dtype=torch.int32, device=dev)
+    for r0 in range(0, N_VAL, 256):
+        r1 = min(N_VAL, r0 + 256)
+        B.qless_project_quantize(g_val[r0:r1], d, SEED, bits, workspace=ws,
+                                 out=dict(codes=val_codes[0, r0:r1], scales=val_scales[0, r0:r1],
+                                          sumsq=val_sumsq[0, r0:r1]))
+    del g_val
+    out = dict(codes=torch.empty((n, rb), dtype=torch.uint8, device=dev),
+               scales=torch.empty(n, dtype=torch.float32, device=dev),
+               sumsq=torch.empty(n, dtype=torch.int32, device=dev))
+    scores = torch.empty(n, dtype=torch.float32, device=dev)
+    indices = torch.empty(n, dtype=torch.int64, device=dev)
+    ws_score = torch.empty(B.qless_score_workspace(n, N_VAL, 1, len(TASKS), d, bits), dtype=torch.uint8, device=dev)
+    ws_sel = torch.empty(B.qless_select_topk_workspace(n), dtype=torch.uint8, device=dev)
+
+    def step():
+        B.qless_project_quantize(g, d, SEED, bits, m, v, out=out, workspace=ws)
+        B.qless_score(out["codes"].unsqueeze(0), val_codes, out["scales"].unsqueeze(0), val_scales, [1.0], off,
+                      d, bits, train_sumsq=out["sumsq"].unsqueeze(0), val_sumsq=val_sumsq, scores=scores,
+                      workspace=ws_score)
+        return B.qless_select_topk(scores, FRAC, indices=indices, workspace=ws_sel)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    B.qless_check()
+
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    launches0 = B.qless_kernel_launches()
+    B.qless_profile_enable(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    prof = B.qless_profile_collect()
+    B.qless_profile_enable(False)
+    launches = B.qless_kernel_launches() - launches0
+    B.qless_check()
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+
+    # ---- end to end through the host-buffer entry point (rank-local; host->device copies timed) ----
+    e2e = None
+    if not args.no_e2e:
+        g_host = torch.empty((n, P), dtype=torch.bfloat16).pin_memory()
+        g_host.copy_(g)
+        host_out = dict(codes=torch.empty((n, rb), dtype=torch.uint8).pin_memory(),
+                        scales=torch.empty(n, dtype=torch.float32).pin_memory(),
+                        sumsq=torch.empty(n, dtype=torch.int32).pin_memory())
+        idx_host = torch.empty(n, dtype=torch.int64).pin_memory()
+        ws_host = torch.empty(B.qless_project_quantize_host_workspace(n, P, d, bits, B.BF16), dtype=torch.uint8, device=dev)
+        del ws
+        k_sel = int(FRAC * n + 1e-6)
+
+        def step_e2e():
+            B.qless_project_quantize_host(g_host, d, SEED, bits, m, v, out=host_out, workspace=ws_host, device=dev)
+            out["codes"].copy_(host_out["codes"], non_blocking=True)
+            out["scales"].copy_(host_out["scales"], non_blocking=True)
+            out["sumsq"].copy_(host_out["sumsq"], non_blocking=True)
+            B.qless_score(out["codes"].unsqueeze(0), val_codes, out["scales"].unsqueeze(0), val_scales, [1.0], off,
+                          d, bits, train_sumsq=out["sumsq"].unsqueeze(0), val_sumsq=val_sumsq, scores=scores,
+                          workspace=ws_score)
+            sel = B.qless_select_topk(scores, FRAC, indices=indices, workspace=ws_sel)
+            idx_host[:sel.numel()].copy_(sel, non_blocking=True)
+
+        for _ in range(min(args.warmup, 2)):
+            step_e2e()
+        barrier()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for _ in range(args.e2e_steps):
+            step_e2e()
+        f1.record()
+        barrier()
+        ms_e2e = f0.elapsed_time(f1)
+        if world > 1:
+            t = torch.tensor([ms_e2e], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        h2d = n * P * 2 + n * rb + 2 * n * 4
+        d2h = n * rb + 2 * n * 4 + k_sel * 8
+        e2e = dict(value=world * n * args.e2e_steps / (ms_e2e * 1e-3), unit="grads/s", h2d_bytes_per_step=h2d,
+                   d2h_bytes_per_step=d2h, steps=args.e2e_steps, ms_per_step=ms_e2e / args.e2e_steps)
+
+    if rank == 0:
+        peaks = load_peaks()
+        value = world * n * args.steps / (ms_total * 1e-3)
+        proj_ms, proj_cnt = prof.get("project", (0.0, 0))
+        flops = 2.0 * n * P * d
+        achieved = flops / (proj_ms / max(proj_cnt, 1) * 1e-3) / 1e12 if proj_cnt else None
+        roofline = dict(bound="tensor", kernel="project", achieved=achieved, peak=peaks["bf16_sustained"],
+                        unit="TFLOP/s", frac=(achieved / peaks["bf16_sustained"]) if achieved else None,
+                        traffic=None, peak_source=f"{peaks['source']} (sustained bf16; burst {peaks['bf16_burst']})",
+                        flops_per_launch=flops, ms_per_launch=proj_ms / max(proj_cnt, 1))
+        line = dict(metric="grads projected+quantized/s (P=2^23,d=8192)", value=value, unit="grads/s",
+                    n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=ms_total / args.steps,
+                    higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
+                    config=dict(workload=WORKLOAD, batch_rows=n, P=P, d=d, bits=bits, val_rows=N_VAL, tasks=TASKS,
+                                select_frac=FRAC, l2="inputs larger than L2 (4.3 GB batch), no flush"),
+                    clocks=clocks, gpu_launches=launches, roofline=roofline,
+                    stages_ms_per_step={k: ms / args.steps for k, (ms, c) in prof.items()},
+                    e2e=e2e)
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline()
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

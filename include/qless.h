@@ -67,6 +67,16 @@ const char* qless_last_error(void);
  * QLESS_ERR_TIMEOUT or QLESS_ERR_CUDA. */
 qless_status qless_check(void* cuda_stream);
 
+/* Per-kernel timing for benchmarks (no counterpart in the paper; measurement aid). While enabled on the
+ * calling thread, every kernel the library launches is bracketed by CUDA events on the call's stream.
+ * qless_profile_collect synchronises those events, writes "name=milliseconds*launches;..." (time summed
+ * per kernel name since the last collect) into buf (NUL-terminated, truncated to buflen) and clears the
+ * record. Enabling costs two event records per launch; leave it off otherwise. */
+qless_status qless_profile_enable(int32_t on);
+/* Number of kernels this library has launched in this process so far (all threads). */
+uint64_t qless_kernel_launches(void);
+qless_status qless_profile_collect(char* buf /* host */, size_t buflen);
+
 /* ------------------------------------------------------------------------------------------
  * Stage 1 + 2: datastore construction (paper Sec. 2.2 Eq. 1-2, Sec. 3.1, Eq. 4-5).
  *
@@ -102,6 +112,22 @@ qless_status qless_project_quantize(
     const float* adam_m, const float* adam_v, const qless_adam_cfg* adam /* host, NULL = defaults */,
     int64_t P, int32_t d, uint64_t seed, int32_t bits,
     void* codes, float* scales, int32_t* code_sumsq, float* proj_out,
+    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* The same computation for callers whose gradients live in HOST memory (pinned memory makes the copies
+ * asynchronous). grads [n, P] (ld_grads elements per row), codes, scales, code_sumsq are HOST pointers;
+ * adam_m / adam_v stay DEVICE pointers (one copy per checkpoint serves every batch). The call copies the
+ * batch to the device workspace, runs qless_project_quantize there and copies the results back, all on
+ * `cuda_stream`; the host buffers must stay valid until the stream has drained. Workspace size:
+ * qless_project_quantize_host_workspace. Definition of the operation: as qless_project_quantize
+ * (Eq. 1-2, Eq. 4-5). */
+size_t qless_project_quantize_host_workspace(int64_t n, int64_t P, int32_t d, int32_t bits, qless_dtype dtype);
+
+qless_status qless_project_quantize_host(
+    const void* grads_host, qless_dtype dtype, int64_t n, int64_t ld_grads,
+    const float* adam_m, const float* adam_v, const qless_adam_cfg* adam /* host, NULL = defaults */,
+    int64_t P, int32_t d, uint64_t seed, int32_t bits,
+    void* codes_host, float* scales_host, int32_t* code_sumsq_host /* NULL to skip */,
     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Stage 2 alone (Eq. 2, Eq. 4-5, packing) on fp32 rows x [n, d]; normalize = 0 skips Eq. 2 so that

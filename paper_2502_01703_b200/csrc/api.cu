@@ -3,6 +3,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <atomic>
 #include <vector>
 
 #include "qless_kernels.h"
@@ -25,6 +26,9 @@ qless_status cuda_fail(cudaError_t e, const char* what)
     snprintf(t_err, sizeof(t_err), "CUDA error %d (%s) in %s", (int)e, cudaGetErrorString(e), what);
     return QLESS_ERR_CUDA;
 }
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
 int sm_count()
 {
@@ -53,6 +57,26 @@ unsigned int* timeout_flag_ptr()
         p = reinterpret_cast<unsigned int*>(q); cached_dev = dev;
     }
     return p;
+}
+
+// ---- per-kernel event timing ---------------------------------------------------------------------
+struct ProfRec { const char* name; cudaEvent_t a, b; };
+static thread_local bool t_prof_on = false;
+static thread_local std::vector<ProfRec> t_prof;
+
+ProfileScope::ProfileScope(const char* name, cudaStream_t st) : name_(name), st_(st), slot_(-1)
+{
+    if (!t_prof_on) return;
+    ProfRec r; r.name = name;
+    if (cudaEventCreate(&r.a) != cudaSuccess) return;
+    if (cudaEventCreate(&r.b) != cudaSuccess) { cudaEventDestroy(r.a); return; }
+    cudaEventRecord(r.a, st);
+    t_prof.push_back(r);
+    slot_ = (int)t_prof.size() - 1;
+}
+ProfileScope::~ProfileScope()
+{
+    if (slot_ >= 0) cudaEventRecord(t_prof[slot_].b, st_);
 }
 
 static bool valid_bits(int b) { return b == 1 || b == 2 || b == 4 || b == 8; }
@@ -129,6 +153,39 @@ qless_status qless_check(void* cuda_stream)
     return QLESS_OK;
 }
 
+uint64_t qless_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+qless_status qless_profile_enable(int32_t on)
+{
+    t_prof_on = on != 0;
+    return QLESS_OK;
+}
+
+qless_status qless_profile_collect(char* buf, size_t buflen)
+{
+    QLESS_REQUIRE(buf != nullptr && buflen > 0, QLESS_ERR_INVALID_ARG, "buf is required");
+    struct Acc { const char* name; double ms; int count; };
+    std::vector<Acc> acc;
+    for (auto& r : t_prof) {
+        float ms = 0.f;
+        cudaEventSynchronize(r.b);
+        if (cudaEventElapsedTime(&ms, r.a, r.b) != cudaSuccess) ms = 0.f;
+        cudaEventDestroy(r.a); cudaEventDestroy(r.b);
+        bool found = false;
+        for (auto& a : acc) if (strcmp(a.name, r.name) == 0) { a.ms += ms; a.count++; found = true; break; }
+        if (!found) acc.push_back({r.name, ms, 1});
+    }
+    t_prof.clear();
+    size_t pos = 0;
+    buf[0] = 0;
+    for (auto& a : acc) {
+        int w = snprintf(buf + pos, buflen - pos, "%s=%.6f*%d;", a.name, a.ms, a.count);
+        if (w < 0 || (size_t)w >= buflen - pos) break;
+        pos += (size_t)w;
+    }
+    return QLESS_OK;
+}
+
 size_t qless_project_quantize_workspace(int64_t n, int64_t P, int32_t d, int32_t bits)
 {
     (void)bits;
@@ -165,13 +222,59 @@ qless_status qless_project_quantize(const void* grads, qless_dtype dtype, int64_
         ld = ld_grads;
     } else {
         __nv_bfloat16* gbuf = reinterpret_cast<__nv_bfloat16*>(ws + w.gamma_off);
-        QLESS_CUDA_TRY(launch_adam_gamma(grads, dtype, n, ld_grads, adam_m, adam_v, ap, P, gbuf, st));
+        { ProfileScope ps("adam_gamma", st);
+          QLESS_CUDA_TRY(launch_adam_gamma(grads, dtype, n, ld_grads, adam_m, adam_v, ap, P, gbuf, st)); }
         gamma = gbuf;
     }
     float* part = reinterpret_cast<float*>(ws + w.part_off);
-    QLESS_CUDA_TRY(launch_project_simt(gamma, ld, w.plan, seed, part, st));
+    { ProfileScope ps("project", st);
+      QLESS_CUDA_TRY(launch_project_simt(gamma, ld, w.plan, seed, part, st)); }
     const float inv_sqrt_d = 1.0f / sqrtf((float)d);
-    QLESS_CUDA_TRY(launch_quantize(part, w.plan.num_chunks, inv_sqrt_d, n, d, 1, bits, codes, scales, code_sumsq, proj_out, st));
+    { ProfileScope ps("quantize", st);
+      QLESS_CUDA_TRY(launch_quantize(part, w.plan.num_chunks, inv_sqrt_d, n, d, 1, bits, codes, scales, code_sumsq, proj_out, st)); }
+    return QLESS_OK;
+}
+
+size_t qless_project_quantize_host_workspace(int64_t n, int64_t P, int32_t d, int32_t bits, qless_dtype dtype)
+{
+    if (n <= 0 || P <= 0 || d <= 0) return 256;
+    const size_t esz = (dtype == QLESS_BF16) ? 2 : 4;
+    return align_up((size_t)n * (size_t)P * esz, 256) + align_up((size_t)n * (size_t)d * bits / 8, 256) +
+           2 * align_up((size_t)n * 4, 256) + qless_project_quantize_workspace(n, P, d, bits);
+}
+
+qless_status qless_project_quantize_host(const void* grads_host, qless_dtype dtype, int64_t n, int64_t ld_grads,
+                                         const float* adam_m, const float* adam_v, const qless_adam_cfg* adam,
+                                         int64_t P, int32_t d, uint64_t seed, int32_t bits, void* codes_host,
+                                         float* scales_host, int32_t* code_sumsq_host, void* workspace,
+                                         size_t workspace_bytes, void* cuda_stream)
+{
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    QLESS_REQUIRE(n >= 0 && P > 0 && d > 0, QLESS_ERR_INVALID_ARG, "n >= 0, P > 0, d > 0 required");
+    QLESS_REQUIRE(dtype == QLESS_F32 || dtype == QLESS_BF16, QLESS_ERR_INVALID_ARG, "dtype must be QLESS_F32 or QLESS_BF16");
+    QLESS_REQUIRE(valid_bits(bits), QLESS_ERR_UNSUPPORTED, "bits must be 1, 2, 4 or 8 (bits=%d)", bits);
+    if (n == 0) return QLESS_OK;
+    QLESS_REQUIRE(grads_host && codes_host && scales_host, QLESS_ERR_INVALID_ARG, "grads_host, codes_host and scales_host are required");
+    QLESS_REQUIRE(ld_grads >= P, QLESS_ERR_INVALID_ARG, "ld_grads must be >= P");
+    const size_t need = qless_project_quantize_host_workspace(n, P, d, bits, dtype);
+    QLESS_REQUIRE(workspace != nullptr && aligned(workspace, 256), QLESS_ERR_WORKSPACE, "workspace must be non-NULL and 256-byte aligned");
+    QLESS_REQUIRE(workspace_bytes >= need, QLESS_ERR_WORKSPACE, "workspace too small: %zu bytes given, %zu needed", workspace_bytes, need);
+    const size_t esz = (dtype == QLESS_BF16) ? 2 : 4;
+    uint8_t* p = reinterpret_cast<uint8_t*>(workspace);
+    void* d_grads = p; p += align_up((size_t)n * (size_t)P * esz, 256);
+    void* d_codes = p; p += align_up((size_t)n * (size_t)d * bits / 8, 256);
+    float* d_scales = reinterpret_cast<float*>(p); p += align_up((size_t)n * 4, 256);
+    int32_t* d_sumsq = reinterpret_cast<int32_t*>(p); p += align_up((size_t)n * 4, 256);
+    const size_t inner = workspace_bytes - (size_t)(p - reinterpret_cast<uint8_t*>(workspace));
+    QLESS_CUDA_TRY(cudaMemcpy2DAsync(d_grads, (size_t)P * esz, grads_host, (size_t)ld_grads * esz, (size_t)P * esz,
+                                     (size_t)n, cudaMemcpyHostToDevice, st));
+    qless_status s = qless_project_quantize(d_grads, dtype, n, P, adam_m, adam_v, adam, P, d, seed, bits, d_codes,
+                                            d_scales, code_sumsq_host ? d_sumsq : nullptr, nullptr, p, inner, cuda_stream);
+    if (s != QLESS_OK) return s;
+    QLESS_CUDA_TRY(cudaMemcpyAsync(codes_host, d_codes, (size_t)n * (size_t)d * bits / 8, cudaMemcpyDeviceToHost, st));
+    QLESS_CUDA_TRY(cudaMemcpyAsync(scales_host, d_scales, (size_t)n * 4, cudaMemcpyDeviceToHost, st));
+    if (code_sumsq_host)
+        QLESS_CUDA_TRY(cudaMemcpyAsync(code_sumsq_host, d_sumsq, (size_t)n * 4, cudaMemcpyDeviceToHost, st));
     return QLESS_OK;
 }
 
@@ -185,7 +288,8 @@ qless_status qless_quantize(const float* x, int64_t n, int32_t d, int32_t normal
     if (n == 0) return QLESS_OK;
     QLESS_REQUIRE(x != nullptr && codes != nullptr && scales != nullptr, QLESS_ERR_INVALID_ARG, "x, codes and scales are required");
     QLESS_REQUIRE(aligned(x, 16) && aligned(codes, 16), QLESS_ERR_INVALID_ARG, "x and codes must be 16-byte aligned");
-    QLESS_CUDA_TRY(launch_quantize(x, 1, 1.0f, n, d, normalize ? 1 : 0, bits, codes, scales, code_sumsq, nullptr, st));
+    { ProfileScope ps("quantize", st);
+      QLESS_CUDA_TRY(launch_quantize(x, 1, 1.0f, n, d, normalize ? 1 : 0, bits, codes, scales, code_sumsq, nullptr, st)); }
     return QLESS_OK;
 }
 
@@ -299,7 +403,8 @@ qless_status qless_score(const void* train_codes, int64_t train_ckpt_stride_byte
     a.train_mult = tmult; a.val_mult = vmult; a.eta_over_cnt = d_eta; a.task_off = d_off;
     a.N = N; a.V = V; a.C = C; a.T = T; a.d = d; a.bits = bits;
     a.scores = scores; a.per_task = per_task; a.dots = nullptr;
-    QLESS_CUDA_TRY(launch_score_simt(a, st));
+    { ProfileScope ps("score", st);
+      QLESS_CUDA_TRY(launch_score_simt(a, st)); }
     return QLESS_OK;
 }
 
@@ -356,7 +461,8 @@ qless_status qless_select_topk(const float* scores, int64_t N, double frac, int6
     }
     *k_out = k;
     if (k == 0) return QLESS_OK;
-    QLESS_CUDA_TRY(launch_select_topk(scores, N, k, indices, workspace, st));
+    { ProfileScope ps("select", st);
+      QLESS_CUDA_TRY(launch_select_topk(scores, N, k, indices, workspace, st)); }
     return QLESS_OK;
 }
 

@@ -92,6 +92,7 @@ cudaError_t launch_project_simt(const __nv_bfloat16* gamma, int64_t ld, const Pr
     if (pl.n == 0) return cudaSuccess;
     dim3 grid((unsigned)(pl.d / PS_DR), (unsigned)((pl.n + PS_GR - 1) / PS_GR), (unsigned)pl.num_chunks);
     project_simt_kernel<<<grid, PS_T, 0, st>>>(gamma, ld, pl.n, pl.P, pl.d, pl.chunk, seed, part);
+    count_launches(1);
     return cudaGetLastError();
 }
 

@@ -77,6 +77,7 @@ cudaError_t launch_adam_gamma(const void* grads, qless_dtype dtype, int64_t n, i
         if (adam) adam_gamma_kernel<false, true><<<(unsigned)blocks, threads, 0, st>>>(grads, n, ld, m, v, ap, P, gamma);
         else adam_gamma_kernel<false, false><<<(unsigned)blocks, threads, 0, st>>>(grads, n, ld, m, v, ap, P, gamma);
     }
+    count_launches(1);
     return cudaGetLastError();
 }
 
@@ -105,6 +106,7 @@ cudaError_t launch_philox_entries(uint64_t seed, int64_t r0, int64_t nr, int64_t
     const int64_t cap = (int64_t)sm_count() * 16;
     if (blocks > cap) blocks = cap;
     philox_entries_kernel<<<(unsigned)blocks, 256, 0, st>>>(seed, r0, nr, j0, nj, out);
+    count_launches(1);
     return cudaGetLastError();
 }
 

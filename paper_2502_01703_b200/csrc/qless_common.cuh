@@ -27,6 +27,15 @@ qless_status cuda_fail(cudaError_t e, const char* what);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Optional per-kernel event timing (see qless_profile_enable). Usage: { ProfileScope ps("name", st); launch; }
+struct ProfileScope {
+    ProfileScope(const char* name, cudaStream_t st);
+    ~ProfileScope();
+    const char* name_; cudaStream_t st_; int slot_;
+};
+
+void count_launches(int n);   // bookkeeping behind qless_kernel_launches()
+
 int sm_count();   // SM count of the current device (cached)
 
 // Address of the device-side timeout word that kernels with bounded waits set when they give up.

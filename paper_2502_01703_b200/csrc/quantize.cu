@@ -182,6 +182,7 @@ cudaError_t launch_quantize(const float* parts, int32_t num_parts, float scale, 
         case 2: quantize_kernel<2><<<(unsigned)blocks, QT, 0, st>>>(parts, num_parts, scale, n, d, normalize, c, scales, sumsq, proj_out); break;
         default: quantize_kernel<1><<<(unsigned)blocks, QT, 0, st>>>(parts, num_parts, scale, n, d, normalize, c, scales, sumsq, proj_out); break;
     }
+    count_launches(1);
     return cudaGetLastError();
 }
 

@@ -227,6 +227,7 @@ cudaError_t launch_score_simt(const ScoreArgs& a, cudaStream_t st)
         default: QLESS_LAUNCH_SCORE(1) break;
     }
 #undef QLESS_LAUNCH_SCORE
+    count_launches(1);
     return cudaGetLastError();
 }
 
@@ -243,6 +244,7 @@ cudaError_t launch_multipliers(const uint8_t* codes, int64_t ckpt_stride, const 
         case 2: multipliers_kernel<2><<<grid, 256, 0, st>>>(codes, ckpt_stride, scales, sumsq, rows, C, d, mode, mult); break;
         default: multipliers_kernel<1><<<grid, 256, 0, st>>>(codes, ckpt_stride, scales, sumsq, rows, C, d, mode, mult); break;
     }
+    count_launches(1);
     return cudaGetLastError();
 }
 

@@ -222,6 +222,7 @@ cudaError_t launch_select_topk(const float* scores, int64_t N, int64_t k, int64_
     select_count_kernel<<<(unsigned)nblk, SEL_T, 0, st>>>(scores, N, w.state, w.blk_cnt);
     select_block_scan_kernel<<<1, 1024, 0, st>>>(w.blk_cnt, nblk, w.blk_off);
     select_write_kernel<<<(unsigned)nblk, SEL_T, 0, st>>>(scores, N, w.state, w.blk_off, indices);
+    count_launches(9);
     return cudaGetLastError();
 }
 

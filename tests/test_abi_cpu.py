@@ -1,0 +1,112 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the header
+declares, and rejects bad arguments with a status before touching the device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2502_01703_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    from paper_2502_01703_b200 import build
+    build.build()
+    return B.lib()
+
+
+def test_exports_every_declared_symbol(L):
+    text = ""
+    inc = os.path.join(ROOT, "include")
+    for name in sorted(os.listdir(inc)):
+        if name.endswith(".h"):
+            text += open(os.path.join(inc, name)).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = sorted(set(re.findall(r"\b(qless_[a-z0-9_]+)\s*\(", text)))
+    assert len(declared) >= 13
+    for sym in declared:
+        assert hasattr(L, sym), sym
+    assert sorted(B.EXPORTS) == [s for s in declared if s in B.EXPORTS]
+    for sym in B.EXPORTS:
+        assert sym in declared
+
+
+def test_workspace_queries_are_pure_host_functions(L):
+    assert B.qless_project_quantize_workspace(0, 1024, 512, 8) >= 256
+    a = B.qless_project_quantize_workspace(256, 1 << 23, 8192, 4)
+    assert a >= 256 * (1 << 23) * 2 + 256 * 8192 * 4
+    assert a % 256 == 0
+    assert B.qless_score_workspace(270_000, 448, 4, 3, 8192, 8) >= 4 * 270_000 * 4
+    assert B.qless_select_topk_workspace(1000) >= 3 * 2048 * 4
+    assert B.qless_select_topk_workspace(1 << 28) < (1 << 28)
+
+
+def _status(call):
+    try:
+        call()
+    except B.QlessError as e:
+        return e.status
+    return 0
+
+
+def test_bad_arguments_return_statuses_before_any_launch(L):
+    null = None
+    # bits
+    st = L.qless_quantize(null, 4, 512, 1, 3, null, null, null, null)
+    assert st == B.ERR_UNSUPPORTED and b"bits" in L.qless_last_error()
+    # d not a multiple of 128 / too large
+    assert L.qless_quantize(null, 4, 500, 1, 8, null, null, null, null) == B.ERR_UNSUPPORTED
+    assert L.qless_quantize(null, 4, 16384, 1, 8, null, null, null, null) == B.ERR_UNSUPPORTED
+    # required pointers
+    assert L.qless_quantize(null, 4, 512, 1, 8, null, null, null, null) == B.ERR_INVALID_ARG
+    # zero rows succeed without touching anything
+    assert L.qless_quantize(null, 0, 512, 1, 8, null, null, null, null) == B.QLESS_OK
+    # negative sizes
+    assert L.qless_quantize(null, -1, 512, 1, 8, null, null, null, null) == B.ERR_INVALID_ARG
+    # projection: P not multiple of 128, one moment missing
+    st = L.qless_project_quantize(null, B.F32, 1, 1000, null, null, None, 1000, 512, 1, 8, null, null, null, null, null, 0, null)
+    assert st == B.ERR_UNSUPPORTED
+    st = L.qless_project_quantize(null, B.F32, 1, 1024, C.c_void_p(16), null, None, 1024, 512, 1, 8, null, null, null, null, null, 0, null)
+    assert st == B.ERR_INVALID_ARG
+    st = L.qless_project_quantize(null, 7, 1, 1024, null, null, None, 1024, 512, 1, 8, null, null, null, null, null, 0, null)
+    assert st == B.ERR_INVALID_ARG
+    # workspace missing / too small (pointers are never dereferenced: the call stops first)
+    fake = C.c_void_p(4096)
+    st = L.qless_project_quantize(fake, B.F32, 2, 1024, null, null, None, 1024, 512, 1, 8, fake, fake, null, null, null, 0, null)
+    assert st == B.ERR_WORKSPACE
+    st = L.qless_project_quantize(fake, B.F32, 2, 1024, null, null, None, 1024, 512, 1, 8, fake, fake, null, null, fake, 16, null)
+    assert st == B.ERR_WORKSPACE and b"too small" in L.qless_last_error()
+    # adam config out of range
+    cfg = B.AdamCfg(1.5, 0.999, 1e-8, 0)
+    st = L.qless_project_quantize(fake, B.F32, 2, 1024, fake, fake, C.byref(cfg), 1024, 512, 1, 8, fake, fake, null, null, fake, 1 << 30, null)
+    assert st == B.ERR_INVALID_ARG
+    # select: frac out of range, NaN
+    k = C.c_int64(-1)
+    assert L.qless_select_topk(null, 10, 1.5, null, C.byref(k), null, 0, null) == B.ERR_INVALID_ARG
+    assert L.qless_select_topk(null, 10, float("nan"), null, C.byref(k), null, 0, null) == B.ERR_INVALID_ARG
+    assert L.qless_select_topk(null, 10, 0.5, null, None, null, 0, null) == B.ERR_INVALID_ARG
+    # k = 0 succeeds and reports it
+    assert L.qless_select_topk(null, 10, 0.0, null, C.byref(k), null, 0, null) == B.QLESS_OK and k.value == 0
+    assert L.qless_select_topk(null, 0, 0.5, null, C.byref(k), null, 0, null) == B.QLESS_OK and k.value == 0
+    # score: task offsets
+    eta = (C.c_float * 2)(1.0, 0.5)
+    def score(off, V=8, T=2, Cn=2, bits=8, d=128):
+        o = (C.c_int32 * (T + 1))(*off)
+        return L.qless_score(fake, 4096, fake, 4096, fake, fake, null, null, eta, o, 4, V, Cn, T, d, bits, 0,
+                             fake, null, null, 0, null)
+    assert score([0, 4, 7]) == B.ERR_INVALID_ARG          # does not end at V
+    assert score([0, 4, 4]) == B.ERR_INVALID_ARG          # empty task
+    assert score([1, 4, 8]) == B.ERR_INVALID_ARG
+    assert score([0, 4, 8], bits=5) == B.ERR_UNSUPPORTED
+    assert score([0, 4, 8]) == B.ERR_WORKSPACE            # valid shapes, no workspace given
+    assert score([0, 4, 8], V=8, d=130) == B.ERR_UNSUPPORTED
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="build the CUDA library"):
+        B.lib()
