@@ -203,6 +203,36 @@ qless_status qless_select_topk(
     const float* scores, int64_t N, double frac, int64_t* indices, int64_t* k_out /* host */,
     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Top-k selection for callers that cannot allocate device memory. (The paper has no counterpart: this
+ * is a packaging variant of qless_select_topk, same result, same ordering rules.)
+ *
+ * Who needs it: code that runs where a cudaMalloc is not an option -- inside a region whose memory is
+ * fully budgeted by a pool the caller does not own (a serving process with a fixed arena, a plug-in
+ * loaded into somebody else's process), or on a path where an allocation's implicit device
+ * synchronisation would stall other streams. qless_select_topk asks such callers for a workspace they
+ * cannot produce; this entry point brings its own.
+ *
+ * The scratch of the radix select (histograms, selection state, per-block counts and offsets) lives in a
+ * fixed array in device global memory that is part of the library image: 74 KiB on every GPU that loads
+ * the library, held until the process exits. That bounds the input: N <= QLESS_SELECT_STATIC_MAX_N
+ * (4 194 304 scores); a larger N is refused with QLESS_ERR_UNSUPPORTED and a message that names the limit.
+ * The call makes no cudaMalloc / cudaFree and calls nothing that allocates; inputs and outputs are still
+ * the caller's (scores [N] fp32 device, 16-byte aligned; indices [k] int64 device; k_out host).
+ *
+ * First call on each device: the library looks up the array's device address (once per device, with that
+ * device current). Make that first call outside any stream capture; later calls only enqueue kernels and
+ * one memset on `cuda_stream`.
+ * Sharing: every call on a device uses the same array. The parts that must start at zero are cleared at
+ * the start of each call and the rest is overwritten before it is read, so back-to-back calls on one
+ * stream are independent. Two calls that overlap on the GPU (different streams, or host threads feeding
+ * different streams) race on the array and give undefined results: serialise them.
+ */
+#define QLESS_SELECT_STATIC_MAX_N (1 << 22)
+
+qless_status qless_select_topk_static(
+    const float* scores, int64_t N, double frac, int64_t* indices, int64_t* k_out /* host */,
+    void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,8 +23,9 @@ EXPORTS = [
     "qless_quantize", "qless_adam_gamma", "qless_philox_entries", "qless_score_workspace", "qless_score",
     "qless_score_dots_workspace", "qless_score_dots", "qless_select_topk_workspace", "qless_select_topk",
     "qless_project_quantize_host_workspace", "qless_project_quantize_host", "qless_profile_enable",
-    "qless_profile_collect", "qless_kernel_launches",
+    "qless_profile_collect", "qless_kernel_launches", "qless_select_topk_static",
 ]
+SELECT_STATIC_MAX_N = 1 << 22
 
 
 class AdamCfg(C.Structure):
@@ -88,6 +89,8 @@ def lib():
         L.qless_select_topk_workspace.argtypes = [i64]
         L.qless_select_topk.restype = C.c_int
         L.qless_select_topk.argtypes = [vp, i64, C.c_double, vp, C.POINTER(i64), vp, sz, vp]
+        L.qless_select_topk_static.restype = C.c_int
+        L.qless_select_topk_static.argtypes = [vp, i64, C.c_double, vp, C.POINTER(i64), vp]
         _lib = L
     return _lib
 
@@ -294,4 +297,15 @@ def qless_select_topk(scores, frac, indices=None, workspace=None, stream=None):
     k = C.c_int64(0)
     _check(lib().qless_select_topk(_ptr(scores), N, float(frac), _ptr(indices), C.byref(k), _ptr(ws),
                                    ws.numel(), _stream(stream)))
+    return indices[:k.value]
+
+
+def qless_select_topk_static(scores, frac, indices, stream=None):
+    """Allocation-free variant of qless_select_topk for N <= SELECT_STATIC_MAX_N: the scratch is a fixed
+    array inside the library, so the caller passes only the input and a preallocated int64 `indices`
+    tensor with room for k entries. Returns a view of the first k entries; nothing is allocated here
+    either. Calls that overlap on the GPU share that array and must be serialised by the caller."""
+    k = C.c_int64(0)
+    _check(lib().qless_select_topk_static(_ptr(scores), scores.numel(), float(frac), _ptr(indices), C.byref(k),
+                                          _stream(stream)))
     return indices[:k.value]

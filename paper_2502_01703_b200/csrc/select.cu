@@ -2,6 +2,9 @@
 // Three histogram passes (11 + 11 + 10 bits) fix the k-th largest key T exactly and the number of
 // keys equal to T that are admitted (smallest indices first); the compaction writes the indices of
 // {key > T} and of the admitted ties in ascending order.
+#include <cmath>
+#include <mutex>
+
 #include "qless_kernels.h"
 
 namespace qless {
@@ -227,3 +230,73 @@ cudaError_t launch_select_topk(const float* scores, int64_t N, int64_t k, int64_
 }
 
 }  // namespace qless
+
+// ------------------------------------------------------------------------------------------------
+// Selection without any allocation: the scratch of the radix select lives in a fixed device array.
+// ------------------------------------------------------------------------------------------------
+
+namespace qless {
+namespace {
+
+// 3 histograms (24 KiB) + state (256 B) + per-block offsets and counts for MAX_N / 2048 = 2048 blocks
+// (32 KiB + 16 KiB) = 73 984 bytes; rounded up. Resident on every GPU that loads the library.
+constexpr size_t kStaticScratchBytes = 74 * 1024;
+static __device__ __align__(256) unsigned char g_select_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mu;
+void* g_scratch_addr[kMaxDevices] = {};
+
+// Device address of g_select_scratch on the current device. In host code the array's name only
+// stands for the symbol; the address kernels can use has to be asked for, once per device.
+qless_status static_scratch(void** out)
+{
+    int dev = 0;
+    QLESS_CUDA_TRY(cudaGetDevice(&dev));
+    QLESS_REQUIRE(dev >= 0 && dev < kMaxDevices, QLESS_ERR_UNSUPPORTED, "device ordinal %d beyond %d", dev, kMaxDevices);
+    std::lock_guard<std::mutex> lk(g_scratch_mu);
+    if (g_scratch_addr[dev] == nullptr) {
+        void* p = nullptr;
+        QLESS_CUDA_TRY(cudaGetSymbolAddress(&p, g_select_scratch));
+        QLESS_REQUIRE(p != nullptr, QLESS_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+        g_scratch_addr[dev] = p;
+    }
+    *out = g_scratch_addr[dev];
+    return QLESS_OK;
+}
+
+}  // namespace
+
+}  // namespace qless
+
+extern "C" qless_status qless_select_topk_static(const float* scores, int64_t N, double frac, int64_t* indices,
+                                                 int64_t* k_out, void* cuda_stream)
+{
+    using namespace qless;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    QLESS_REQUIRE(N >= 0, QLESS_ERR_INVALID_ARG, "N must be >= 0");
+    QLESS_REQUIRE(N <= (int64_t)QLESS_SELECT_STATIC_MAX_N, QLESS_ERR_UNSUPPORTED,
+                  "qless_select_topk_static handles at most %d scores (N=%lld); use qless_select_topk with a workspace",
+                  (int)QLESS_SELECT_STATIC_MAX_N, (long long)N);
+    QLESS_REQUIRE(frac >= 0.0 && frac <= 1.0, QLESS_ERR_INVALID_ARG, "frac must be in [0, 1]");
+    QLESS_REQUIRE(k_out != nullptr, QLESS_ERR_INVALID_ARG, "k_out (host) is required");
+    double kf = std::floor(frac * (double)N + 1e-6);
+    if (kf < 0.0) kf = 0.0;
+    if (kf > (double)N) kf = (double)N;
+    const int64_t k = (int64_t)kf;
+    if (k > 0) {
+        QLESS_REQUIRE(scores != nullptr && indices != nullptr, QLESS_ERR_INVALID_ARG, "scores and indices are required");
+        QLESS_REQUIRE((reinterpret_cast<uintptr_t>(scores) % 16) == 0, QLESS_ERR_INVALID_ARG, "scores must be 16-byte aligned");
+        static_assert(kStaticScratchBytes >= 3 * 2048 * 4 + 256 + 2048 * 16 + 2048 * 8, "scratch array too small");
+        QLESS_REQUIRE(select_workspace_bytes(N) <= kStaticScratchBytes, QLESS_ERR_UNSUPPORTED, "internal: scratch array too small");
+    }
+    *k_out = k;
+    if (k == 0) return QLESS_OK;
+    void* scratch = nullptr;
+    qless_status s = static_scratch(&scratch);
+    if (s != QLESS_OK) return s;
+    // The histograms are cleared inside; the state and the per-block arrays are rewritten in full for
+    // this N before they are read, so nothing of the previous call's contents is used.
+    QLESS_CUDA_TRY(launch_select_topk(scores, N, k, indices, scratch, st));
+    return QLESS_OK;
+}
