@@ -130,6 +130,12 @@ qless_status qless_project_quantize_host(
     void* codes_host, float* scales_host, int32_t* code_sumsq_host /* NULL to skip */,
     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Test hook: which kernel computes the projection of Eq. 1 in qless_project_quantize. 0 (default): the
+ * tcgen05 tensor-core kernel; 1: a plain CUDA-core kernel of the same definition, kept so that the
+ * tensor-core result can be cross-checked on the device at sizes the CPU oracle only samples (it is
+ * also what runs when P >= 2^31). Process-wide. */
+qless_status qless_set_projection_path(int32_t path);
+
 /* Stage 2 alone (Eq. 2, Eq. 4-5, packing) on fp32 rows x [n, d]; normalize = 0 skips Eq. 2 so that
  * already-normalised rows can be fed. Same outputs and packing as above. Needs no workspace. */
 qless_status qless_quantize(

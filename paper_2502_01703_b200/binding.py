@@ -24,6 +24,7 @@ EXPORTS = [
     "qless_score_dots_workspace", "qless_score_dots", "qless_select_topk_workspace", "qless_select_topk",
     "qless_project_quantize_host_workspace", "qless_project_quantize_host", "qless_profile_enable",
     "qless_profile_collect", "qless_kernel_launches", "qless_select_topk_static",
+    "qless_set_projection_path",
 ]
 SELECT_STATIC_MAX_N = 1 << 22
 
@@ -89,6 +90,8 @@ def lib():
         L.qless_select_topk_workspace.argtypes = [i64]
         L.qless_select_topk.restype = C.c_int
         L.qless_select_topk.argtypes = [vp, i64, C.c_double, vp, C.POINTER(i64), vp, sz, vp]
+        L.qless_set_projection_path.restype = C.c_int
+        L.qless_set_projection_path.argtypes = [i32]
         L.qless_select_topk_static.restype = C.c_int
         L.qless_select_topk_static.argtypes = [vp, i64, C.c_double, vp, C.POINTER(i64), vp]
         _lib = L
@@ -309,3 +312,8 @@ def qless_select_topk_static(scores, frac, indices, stream=None):
     _check(lib().qless_select_topk_static(_ptr(scores), scores.numel(), float(frac), _ptr(indices), C.byref(k),
                                           _stream(stream)))
     return indices[:k.value]
+
+
+def qless_set_projection_path(path):
+    """0 = tensor-core projection kernel (default), 1 = CUDA-core cross-check kernel."""
+    _check(lib().qless_set_projection_path(int(path)))

@@ -7,6 +7,7 @@
 #include <vector>
 
 #include "qless_kernels.h"
+#include "tc_common.cuh"
 
 namespace qless {
 
@@ -79,6 +80,8 @@ ProfileScope::~ProfileScope()
     if (slot_ >= 0) cudaEventRecord(t_prof[slot_].b, st_);
 }
 
+static std::atomic<int> g_projection_path{0};   // 0 = tensor cores, 1 = CUDA cores (cross-check hook)
+
 static bool valid_bits(int b) { return b == 1 || b == 2 || b == 4 || b == 8; }
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -150,6 +153,13 @@ qless_status qless_check(void* cuda_stream)
         QLESS_CUDA_TRY(cudaStreamSynchronize(st));
         return fail(QLESS_ERR_TIMEOUT, "a device-side bounded wait gave up (code 0x%x); results of that call are invalid", h);
     }
+    return QLESS_OK;
+}
+
+qless_status qless_set_projection_path(int32_t path)
+{
+    QLESS_REQUIRE(path == 0 || path == 1, QLESS_ERR_INVALID_ARG, "path must be 0 (tensor cores) or 1 (CUDA cores)");
+    g_projection_path.store(path);
     return QLESS_OK;
 }
 
@@ -227,8 +237,18 @@ qless_status qless_project_quantize(const void* grads, qless_dtype dtype, int64_
         gamma = gbuf;
     }
     float* part = reinterpret_cast<float*>(ws + w.part_off);
-    { ProfileScope ps("project", st);
-      QLESS_CUDA_TRY(launch_project_simt(gamma, ld, w.plan, seed, part, st)); }
+    if (g_projection_path == 0 && P < ((int64_t)1 << 31)) {
+        CUtensorMap tmap;
+        s = make_tmap_2d_sw128(&tmap, gamma, 2, (uint64_t)P, (uint64_t)n, (uint64_t)ld * 2, 64, 256);
+        if (s != QLESS_OK) return s;
+        unsigned int* flag = timeout_flag_ptr();
+        QLESS_REQUIRE(flag != nullptr, QLESS_ERR_CUDA, "cannot resolve the device timeout flag");
+        ProfileScope ps("project", st);
+        QLESS_CUDA_TRY(launch_project_tc(tmap, w.plan, seed, part, flag, st));
+    } else {
+        ProfileScope ps("project", st);
+        QLESS_CUDA_TRY(launch_project_simt(gamma, ld, w.plan, seed, part, st));
+    }
     const float inv_sqrt_d = 1.0f / sqrtf((float)d);
     { ProfileScope ps("quantize", st);
       QLESS_CUDA_TRY(launch_quantize(part, w.plan.num_chunks, inv_sqrt_d, n, d, 1, bits, codes, scales, code_sumsq, proj_out, st)); }

@@ -75,12 +75,15 @@ project_simt_kernel(const __nv_bfloat16* __restrict__ gamma, int64_t ld, int64_t
 
 ProjectPlan plan_projection(int64_t n, int64_t P, int32_t d)
 {
+    // K-chunk length: a power of two in [1024, 65536] (so every chunk starts on a Philox block and a chain
+    // of fp32 accumulations never exceeds 4096 tensor-core steps), the largest that still gives every SM
+    // about four work items of (256 gradient rows x 128 projected coordinates x chunk).
     ProjectPlan pl;
     pl.n = n; pl.P = P; pl.d = d;
-    int64_t chunk = P < 32768 ? P : 32768;
     const int64_t tiles = (int64_t)(d / 128) * ((n + 255) / 256);
-    while (chunk > 2048 && chunk % 256 == 0 && tiles * ((P + chunk - 1) / chunk) < 2 * (int64_t)sm_count())
-        chunk >>= 1;
+    int64_t chunk = 65536;
+    while (chunk > 1024 && tiles * ((P + chunk - 1) / chunk) < 4 * (int64_t)sm_count()) chunk >>= 1;
+    if (chunk > P) chunk = P;
     pl.chunk = chunk;
     pl.num_chunks = (int32_t)((P + chunk - 1) / chunk);
     return pl;

@@ -1,0 +1,230 @@
+// Projection (Eq. 1) on the 5th-generation tensor cores.
+//
+//   part[s][i][r] = sum_{j in K-chunk s} Gamma[i][j] * sign(r, j)          (bf16 x bf16 -> fp32)
+//
+// as a GEMM with the roles chosen for the hardware: the M side (128 TMEM lanes) is a tile of 128
+// projected coordinates r, whose +-1.0 operand rows are generated from Philox straight into tensor
+// memory (no shared-memory traffic, no swizzle); the N side is a tile of up to 256 gradient rows,
+// streamed K-major from global memory by TMA into 128-byte-swizzled shared memory. The accumulator
+// (128 x 256 fp32) occupies TMEM columns 0..255, four 128-deep stages of the sign operand occupy
+// columns 256..511. Each CTA is persistent and walks work items (gradient tile, K-chunk, r tile)
+// K-chunk-major, so that at any time all CTAs read the same slab of Gamma (L2 reuse); after each
+// K-chunk the accumulator is drained to a per-chunk partial, which bounds the length of any fp32
+// accumulation chain and makes the final sum order fixed.
+//
+// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer (+ TMEM allocation), warps 2-5 sign
+// generators, warps 6-9 accumulator drain. All waits are bounded; a wait that gives up raises the
+// device timeout word and every role leaves its loop.
+#include "qless_kernels.h"
+#include "tc_common.cuh"
+
+namespace qless {
+
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128;                 // projected coordinates per tile (UMMA M)
+constexpr int BN = 256;                 // gradient rows per tile (UMMA N)
+constexpr int BK = 64;                  // K per shared-memory stage (128 bytes of bf16)
+constexpr int SB = 6;                   // shared-memory stages of the gradient operand
+constexpr int SA = 4;                   // TMEM stages of the sign operand, 128 K each (64 columns)
+constexpr int B_STAGE_BYTES = BN * BK * 2;     // 32 KiB
+constexpr int TMEM_COLS = 512;
+constexpr int D_COL = 0, A_COL = 256;
+constexpr int NTHREADS = 320;
+constexpr uint32_t IDESC = make_idesc(/*D=F32*/ 1, /*A=BF16*/ 1, /*B=BF16*/ 1, BM, BN);
+
+struct __align__(8) Barriers {
+    uint64_t b_full[SB], b_empty[SB], a_full[SA], a_empty[SA], d_full, d_empty;
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)SB * B_STAGE_BYTES + sizeof(Barriers);
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int32_t d, int64_t P, int64_t chunk,
+                  int32_t num_chunks, uint64_t seed, float* __restrict__ part, unsigned int* __restrict__ timeout_word)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Barriers* bars = reinterpret_cast<Barriers*>(smem + (size_t)SB * B_STAGE_BYTES);
+    volatile uint32_t* abort_flag = &bars->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_dt = d / BM;
+    const int num_nt = (int)((n + BN - 1) / BN);
+    const int64_t num_items = (int64_t)num_nt * num_chunks * num_dt;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < SB; ++s) { mbar_init(smem_u32(&bars->b_full[s]), 1); mbar_init(smem_u32(&bars->b_empty[s]), 1); }
+        for (int s = 0; s < SA; ++s) { mbar_init(smem_u32(&bars->a_full[s]), 128); mbar_init(smem_u32(&bars->a_empty[s]), 1); }
+        mbar_init(smem_u32(&bars->d_full), 1);
+        mbar_init(smem_u32(&bars->d_empty), 128);
+        bars->abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tmap_gamma);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&bars->tmem_base), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = bars->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------- TMA producer -------------------------------
+        if (lane == 0) {
+            uint32_t it = 0;     // global stage counter
+            bool ok = true;
+            for (int64_t item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+                const int64_t nt = item / ((int64_t)num_chunks * num_dt);
+                const int kc = (int)((item / num_dt) % num_chunks);
+                const int64_t k0 = (int64_t)kc * chunk;
+                const int nkb = (int)((min(P, k0 + chunk) - k0) / BK);
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % SB;
+                    const uint32_t ph = (it / SB) & 1u;
+                    if (!mbar_wait(smem_u32(&bars->b_empty[s]), ph ^ 1u, abort_flag, timeout_word, TO_PRODUCER)) { ok = false; break; }
+                    const uint32_t full = smem_u32(&bars->b_full[s]);
+                    mbar_arrive_expect_tx(full, B_STAGE_BYTES);
+                    tma_load_2d(smem_u32(smem + (size_t)s * B_STAGE_BYTES), &tmap_gamma, full,
+                                (int32_t)(k0 + (int64_t)kb * BK), (int32_t)(nt * BN));
+                }
+            }
+            if (!ok) {
+                // leave no copy in flight behind us: give every armed stage a bounded chance to land
+                for (int s = 0; s < SB; ++s)
+                    for (uint32_t t = 0; t < (1u << 16); ++t)
+                        if (mbar_try_wait(smem_u32(&bars->b_full[s]), 0) || mbar_try_wait(smem_u32(&bars->b_full[s]), 1)) break;
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------- MMA issuer -------------------------------
+        if (lane == 0) {
+            uint32_t itb = 0, ita = 0, n_item = 0;
+            bool ok = true;
+            for (int64_t item = blockIdx.x; item < num_items && ok; item += gridDim.x, ++n_item) {
+                const int kc = (int)((item / num_dt) % num_chunks);
+                const int64_t k0 = (int64_t)kc * chunk;
+                const int nkb = (int)((min(P, k0 + chunk) - k0) / BK);
+                if (!mbar_wait(smem_u32(&bars->d_empty), (n_item & 1u) ^ 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
+                tc_fence_after();
+                for (int kb = 0; kb < nkb; ++kb, ++itb) {
+                    const int sb = itb % SB;
+                    if (!mbar_wait(smem_u32(&bars->b_full[sb]), (itb / SB) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
+                    const int sa = ita % SA;
+                    if ((kb & 1) == 0) {
+                        if (!mbar_wait(smem_u32(&bars->a_full[sa]), (ita / SA) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
+                    }
+                    tc_fence_after();
+                    const uint64_t bdesc = make_smem_desc_sw128(smem_u32(smem + (size_t)sb * B_STAGE_BYTES));
+                    const uint32_t a_addr = tmem_base + A_COL + sa * 64 + (kb & 1) * 32;
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        mma_f16_ts(tmem_base + D_COL, a_addr + k * 8, bdesc + (uint64_t)(k * 2), IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+                    mma_commit(smem_u32(&bars->b_empty[sb]));
+                    if (kb & 1) { mma_commit(smem_u32(&bars->a_empty[sa])); ++ita; }
+                }
+                if (ok) mma_commit(smem_u32(&bars->d_full));
+            }
+        }
+    } else if (warp < 6) {
+        // ------------------------------- sign generators -------------------------------
+        const int q = warp & 3;                                  // TMEM lane quadrant this warp may access
+        uint32_t ita = 0;
+        bool ok = true;
+        for (int64_t item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+            const int dt = (int)(item % num_dt);
+            const int kc = (int)((item / num_dt) % num_chunks);
+            const int64_t k0 = (int64_t)kc * chunk;
+            const int nka = (int)((min(P, k0 + chunk) - k0) / 128);
+            const uint32_t r = (uint32_t)(dt * BM + q * 32 + lane);
+            for (int ka = 0; ka < nka; ++ka, ++ita) {
+                const int sa = ita % SA;
+                uint32_t w[4];
+                rademacher_block(seed, r, (uint32_t)((k0 >> 7) + ka), w);     // overlaps with the wait below
+                ok = mbar_wait(smem_u32(&bars->a_empty[sa]), ((ita / SA) & 1u) ^ 1u, abort_flag, timeout_word, TO_GENERATOR);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + A_COL + sa * 64;
+#pragma unroll
+                for (int wi = 0; wi < 4; ++wi) {
+                    uint32_t v[16];
+#pragma unroll
+                    for (int p = 0; p < 16; ++p) v[p] = rademacher_bf16x2(w[wi], p);
+                    tmem_st_x16(taddr + wi * 16, v);
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars->a_full[sa]));
+            }
+        }
+    } else {
+        // ------------------------------- accumulator drain -------------------------------
+        const int q = warp & 3;
+        uint32_t n_item = 0;
+        bool ok = true;
+        for (int64_t item = blockIdx.x; item < num_items && ok; item += gridDim.x, ++n_item) {
+            const int dt = (int)(item % num_dt);
+            const int kc = (int)((item / num_dt) % num_chunks);
+            const int64_t nt = item / ((int64_t)num_chunks * num_dt);
+            ok = mbar_wait(smem_u32(&bars->d_full), n_item & 1u, abort_flag, timeout_word, TO_EPILOGUE);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            float* out = part + ((int64_t)kc * n + nt * BN) * d + dt * BM + q * 32 + lane;
+            const int64_t rows_here = min((int64_t)BN, n - nt * BN);
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + D_COL;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld_x32(taddr + c0, v);
+                tmem_wait_ld();
+                if (c0 + 32 == BN) {          // accumulator fully read: hand it back before the stores
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&bars->d_empty));
+                }
+#pragma unroll
+                for (int k = 0; k < 32; ++k)
+                    if (c0 + k < rows_here) __stcs(out + (int64_t)(c0 + k) * d, __uint_as_float(v[k]));
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace
+
+size_t project_tc_smem_bytes() { return SMEM_BYTES; }
+
+cudaError_t launch_project_tc(const CUtensorMap& tmap, const ProjectPlan& pl, uint64_t seed, float* part,
+                              unsigned int* timeout_word, cudaStream_t st)
+{
+    if (pl.n == 0) return cudaSuccess;
+    static thread_local bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(project_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int64_t items = (int64_t)((pl.n + BN - 1) / BN) * pl.num_chunks * (pl.d / BM);
+    int64_t grid = sm_count();
+    if (grid > items) grid = items;
+    project_tc_kernel<<<(unsigned)grid, NTHREADS, SMEM_BYTES, st>>>(tmap, pl.n, pl.d, pl.P, pl.chunk, pl.num_chunks, seed,
+                                                                    part, timeout_word);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+}  // namespace qless

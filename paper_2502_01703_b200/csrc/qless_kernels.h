@@ -1,5 +1,7 @@
 // Internal launch interface between the C ABI (api.cu) and the kernel translation units.
 #pragma once
+#include <cuda.h>
+
 #include "qless_common.cuh"
 
 namespace qless {
@@ -30,6 +32,10 @@ struct ProjectPlan {
 ProjectPlan plan_projection(int64_t n, int64_t P, int32_t d);
 cudaError_t launch_project_simt(const __nv_bfloat16* gamma, int64_t ld, const ProjectPlan& pl,
                                 uint64_t seed, float* part, cudaStream_t st);
+
+// Tensor-core projection (project_tc.cu). The tensor map describes Gamma [n, P] bf16 with a 64 x 256 box.
+cudaError_t launch_project_tc(const CUtensorMap& tmap, const ProjectPlan& pl, uint64_t seed, float* part,
+                              unsigned int* timeout_word, cudaStream_t st);
 
 // Stage 2. x = inv_scale-scaled sum of `num_parts` partial arrays [num_parts][n][d] (num_parts = 1,
 // scale = 1 for plain rows). Writes proj_out (optional), codes, scales, sumsq (optional).
