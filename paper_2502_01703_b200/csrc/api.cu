@@ -225,21 +225,14 @@ qless_status qless_project_quantize(const void* grads, qless_dtype dtype, int64_
     QLESS_REQUIRE(workspace_bytes >= w.total, QLESS_ERR_WORKSPACE, "workspace too small: %zu bytes given, %zu needed", workspace_bytes, w.total);
 
     uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
-    const __nv_bfloat16* gamma;
-    int64_t ld = P;
-    if (dtype == QLESS_BF16 && adam_m == nullptr) {
-        gamma = reinterpret_cast<const __nv_bfloat16*>(grads);       // Gamma = g, already bf16
-        ld = ld_grads;
-    } else {
-        __nv_bfloat16* gbuf = reinterpret_cast<__nv_bfloat16*>(ws + w.gamma_off);
-        { ProfileScope ps("adam_gamma", st);
-          QLESS_CUDA_TRY(launch_adam_gamma(grads, dtype, n, ld_grads, adam_m, adam_v, ap, P, gbuf, st)); }
-        gamma = gbuf;
-    }
+    // Pre-pass: Gamma as bf16 in the K-blocked layout the projection streams ([P/64][n][64]).
+    __nv_bfloat16* gamma = reinterpret_cast<__nv_bfloat16*>(ws + w.gamma_off);
+    { ProfileScope ps("adam_gamma", st);
+      QLESS_CUDA_TRY(launch_adam_gamma(grads, dtype, n, ld_grads, adam_m, adam_v, ap, P, gamma, true, st)); }
     float* part = reinterpret_cast<float*>(ws + w.part_off);
-    if (g_projection_path == 0 && P < ((int64_t)1 << 31)) {
+    if (g_projection_path == 0 && (P / 64) * n < ((int64_t)1 << 31)) {
         CUtensorMap tmap;
-        s = make_tmap_2d_sw128(&tmap, gamma, 2, (uint64_t)P, (uint64_t)n, (uint64_t)ld * 2, 64, 256);
+        s = make_tmap_2d_sw128(&tmap, gamma, 2, 64, (uint64_t)(P / 64) * (uint64_t)n, 128, 64, 256);
         if (s != QLESS_OK) return s;
         unsigned int* flag = timeout_flag_ptr();
         QLESS_REQUIRE(flag != nullptr, QLESS_ERR_CUDA, "cannot resolve the device timeout flag");
@@ -247,7 +240,7 @@ qless_status qless_project_quantize(const void* grads, qless_dtype dtype, int64_
         QLESS_CUDA_TRY(launch_project_tc(tmap, w.plan, seed, part, flag, st));
     } else {
         ProfileScope ps("project", st);
-        QLESS_CUDA_TRY(launch_project_simt(gamma, ld, w.plan, seed, part, st));
+        QLESS_CUDA_TRY(launch_project_simt(gamma, w.plan, seed, part, st));
     }
     const float inv_sqrt_d = 1.0f / sqrtf((float)d);
     { ProfileScope ps("quantize", st);
@@ -326,7 +319,7 @@ qless_status qless_adam_gamma(const void* grads, qless_dtype dtype, int64_t n, i
     if (n == 0) return QLESS_OK;
     QLESS_REQUIRE(gamma_out != nullptr && aligned(gamma_out, 16), QLESS_ERR_INVALID_ARG, "gamma_out must be non-NULL and 16-byte aligned");
     QLESS_CUDA_TRY(launch_adam_gamma(grads, dtype, n, ld_grads, adam_m, adam_v, ap, P,
-                                     reinterpret_cast<__nv_bfloat16*>(gamma_out), st));
+                                     reinterpret_cast<__nv_bfloat16*>(gamma_out), false, st));
     return QLESS_OK;
 }
 

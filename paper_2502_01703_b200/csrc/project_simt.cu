@@ -11,7 +11,7 @@ constexpr int PS_GR = 32;     // gradient rows per block
 constexpr int PS_T = 256;
 
 __global__ void __launch_bounds__(PS_T)
-project_simt_kernel(const __nv_bfloat16* __restrict__ gamma, int64_t ld, int64_t n, int64_t P, int32_t d,
+project_simt_kernel(const __nv_bfloat16* __restrict__ gamma, int64_t n, int64_t P, int32_t d,
                     int64_t chunk, uint64_t seed, float* __restrict__ part)
 {
     __shared__ __align__(16) float s_g[PS_GR][128];
@@ -32,7 +32,8 @@ project_simt_kernel(const __nv_bfloat16* __restrict__ gamma, int64_t ld, int64_t
             const int row = e >> 6, cp = e & 63;
             float2 f = make_float2(0.f, 0.f);
             if (i0 + row < n) {
-                const uint32_t w = *reinterpret_cast<const uint32_t*>(gamma + (i0 + row) * ld + kb + 2 * cp);
+                const int64_t j = kb + 2 * cp;     // tiled layout [P/64][n][64]
+                const uint32_t w = *reinterpret_cast<const uint32_t*>(gamma + ((((j >> 6) * n + (i0 + row)) << 6) + (j & 63)));
                 f.x = __uint_as_float(w << 16);
                 f.y = __uint_as_float(w & 0xFFFF0000u);
             }
@@ -89,12 +90,12 @@ ProjectPlan plan_projection(int64_t n, int64_t P, int32_t d)
     return pl;
 }
 
-cudaError_t launch_project_simt(const __nv_bfloat16* gamma, int64_t ld, const ProjectPlan& pl, uint64_t seed,
+cudaError_t launch_project_simt(const __nv_bfloat16* gamma, const ProjectPlan& pl, uint64_t seed,
                                 float* part, cudaStream_t st)
 {
     if (pl.n == 0) return cudaSuccess;
     dim3 grid((unsigned)(pl.d / PS_DR), (unsigned)((pl.n + PS_GR - 1) / PS_GR), (unsigned)pl.num_chunks);
-    project_simt_kernel<<<grid, PS_T, 0, st>>>(gamma, ld, pl.n, pl.P, pl.d, pl.chunk, seed, part);
+    project_simt_kernel<<<grid, PS_T, 0, st>>>(gamma, pl.n, pl.P, pl.d, pl.chunk, seed, part);
     count_launches(1);
     return cudaGetLastError();
 }

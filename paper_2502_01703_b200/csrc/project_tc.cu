@@ -5,7 +5,8 @@
 // as a GEMM with the roles chosen for the hardware: the M side (128 TMEM lanes) is a tile of 128
 // projected coordinates r, whose +-1.0 operand rows are generated from Philox straight into tensor
 // memory (no shared-memory traffic, no swizzle); the N side is a tile of up to 256 gradient rows,
-// streamed K-major from global memory by TMA into 128-byte-swizzled shared memory. The accumulator
+// streamed by TMA from a K-blocked copy of Gamma ([P/64][n][64], so that each 256 x 64 operand tile is one
+// contiguous 32 KiB span) into 128-byte-swizzled shared memory. The accumulator
 // (128 x 256 fp32) occupies TMEM columns 0..255, four 128-deep stages of the sign operand occupy
 // columns 256..511. Each CTA is persistent and walks work items (gradient tile, K-chunk, r tile)
 // K-chunk-major, so that at any time all CTAs read the same slab of Gamma (L2 reuse); after each
@@ -91,8 +92,10 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                     if (!mbar_wait(smem_u32(&bars->b_empty[s]), ph ^ 1u, abort_flag, timeout_word, TO_PRODUCER)) { ok = false; break; }
                     const uint32_t full = smem_u32(&bars->b_full[s]);
                     mbar_arrive_expect_tx(full, B_STAGE_BYTES);
-                    tma_load_2d(smem_u32(smem + (size_t)s * B_STAGE_BYTES), &tmap_gamma, full,
-                                (int32_t)(k0 + (int64_t)kb * BK), (int32_t)(nt * BN));
+                    // tiled Gamma: K block kb64 holds its n rows of 64 columns contiguously
+                    const int64_t kb64 = (k0 >> 6) + kb;
+                    tma_load_2d(smem_u32(smem + (size_t)s * B_STAGE_BYTES), &tmap_gamma, full, 0,
+                                (int32_t)(kb64 * n + nt * BN));
                 }
             }
             if (!ok) {

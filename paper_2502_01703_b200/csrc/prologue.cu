@@ -15,7 +15,7 @@ __device__ __forceinline__ float adam_dir(float g, float m, float v, const AdamP
 }
 
 // One thread handles 8 consecutive columns of one row: 16-byte bf16 loads/stores, 2x16-byte fp32.
-template <bool BF16_IN, bool ADAM>
+template <bool BF16_IN, bool ADAM, bool TILED>
 __global__ void __launch_bounds__(256)
 adam_gamma_kernel(const void* __restrict__ grads, int64_t n, int64_t ld, const float* __restrict__ m,
                   const float* __restrict__ v, AdamParams ap, int64_t P, __nv_bfloat16* __restrict__ gamma)
@@ -55,13 +55,16 @@ adam_gamma_kernel(const void* __restrict__ grads, int64_t n, int64_t ld, const f
             const __nv_bfloat162 pr = __floats2bfloat162_rn(g[2 * k], g[2 * k + 1]);
             o[k] = *reinterpret_cast<const uint32_t*>(&pr);
         }
-        *reinterpret_cast<uint4*>(gamma + row * P + j0) = make_uint4(o[0], o[1], o[2], o[3]);
+        // TILED: [K block of 64 columns][row][64] so that a (256 rows x 64 columns) operand tile is one
+        // contiguous 32 KiB span; otherwise plain row-major [n, P].
+        const int64_t dst = TILED ? (((j0 >> 6) * n + row) << 6) + (j0 & 63) : row * P + j0;
+        *reinterpret_cast<uint4*>(gamma + dst) = make_uint4(o[0], o[1], o[2], o[3]);
     }
 }
 
 cudaError_t launch_adam_gamma(const void* grads, qless_dtype dtype, int64_t n, int64_t ld, const float* m,
                               const float* v, const AdamParams& ap, int64_t P, __nv_bfloat16* gamma,
-                              cudaStream_t st)
+                              bool tiled, cudaStream_t st)
 {
     if (n == 0 || P == 0) return cudaSuccess;
     const int64_t total = n * (P >> 3);
@@ -70,13 +73,17 @@ cudaError_t launch_adam_gamma(const void* grads, qless_dtype dtype, int64_t n, i
     const int64_t cap = (int64_t)sm_count() * 16;
     if (blocks > cap) blocks = cap;
     const bool adam = (m != nullptr);
-    if (dtype == QLESS_BF16) {
-        if (adam) adam_gamma_kernel<true, true><<<(unsigned)blocks, threads, 0, st>>>(grads, n, ld, m, v, ap, P, gamma);
-        else adam_gamma_kernel<true, false><<<(unsigned)blocks, threads, 0, st>>>(grads, n, ld, m, v, ap, P, gamma);
-    } else {
-        if (adam) adam_gamma_kernel<false, true><<<(unsigned)blocks, threads, 0, st>>>(grads, n, ld, m, v, ap, P, gamma);
-        else adam_gamma_kernel<false, false><<<(unsigned)blocks, threads, 0, st>>>(grads, n, ld, m, v, ap, P, gamma);
-    }
+#define QLESS_AG(B, A, T) adam_gamma_kernel<B, A, T><<<(unsigned)blocks, threads, 0, st>>>(grads, n, ld, m, v, ap, P, gamma)
+    const bool bf = (dtype == QLESS_BF16);
+    if (bf && adam && tiled) QLESS_AG(true, true, true);
+    else if (bf && adam) QLESS_AG(true, true, false);
+    else if (bf && tiled) QLESS_AG(true, false, true);
+    else if (bf) QLESS_AG(true, false, false);
+    else if (adam && tiled) QLESS_AG(false, true, true);
+    else if (adam) QLESS_AG(false, true, false);
+    else if (tiled) QLESS_AG(false, false, true);
+    else QLESS_AG(false, false, false);
+#undef QLESS_AG
     count_launches(1);
     return cudaGetLastError();
 }

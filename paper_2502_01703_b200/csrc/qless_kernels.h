@@ -13,10 +13,11 @@ struct AdamParams {
     int   bias_correct;
 };
 
-// Gamma[n, P] (bf16) from gradient rows; m/v NULL => bf16(g).
+// Gamma (bf16) from gradient rows; m/v NULL => bf16(g). tiled = false: row-major [n, P];
+// tiled = true: [P/64][n][64] (element (i, j) at ((j/64)*n + i)*64 + j%64), the layout the projection reads.
 cudaError_t launch_adam_gamma(const void* grads, qless_dtype dtype, int64_t n, int64_t ld,
                               const float* m, const float* v, const AdamParams& ap, int64_t P,
-                              __nv_bfloat16* gamma, cudaStream_t st);
+                              __nv_bfloat16* gamma, bool tiled, cudaStream_t st);
 
 cudaError_t launch_philox_entries(uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj,
                                   int8_t* out, cudaStream_t st);
@@ -30,10 +31,11 @@ struct ProjectPlan {
     int32_t num_chunks;
 };
 ProjectPlan plan_projection(int64_t n, int64_t P, int32_t d);
-cudaError_t launch_project_simt(const __nv_bfloat16* gamma, int64_t ld, const ProjectPlan& pl,
+cudaError_t launch_project_simt(const __nv_bfloat16* gamma_tiled, const ProjectPlan& pl,
                                 uint64_t seed, float* part, cudaStream_t st);
 
-// Tensor-core projection (project_tc.cu). The tensor map describes Gamma [n, P] bf16 with a 64 x 256 box.
+// Tensor-core projection (project_tc.cu). The tensor map describes tiled Gamma as [(P/64)*n][64] bf16 with a
+// 64 x 256 box.
 cudaError_t launch_project_tc(const CUtensorMap& tmap, const ProjectPlan& pl, uint64_t seed, float* part,
                               unsigned int* timeout_word, cudaStream_t st);
 
