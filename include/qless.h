@@ -136,6 +136,11 @@ qless_status qless_project_quantize_host(
  * also what runs when P >= 2^31). Process-wide. */
 qless_status qless_set_projection_path(int32_t path);
 
+/* Test hook, as above, for the integer similarity of 8-, 4- and 2-bit codes in qless_score and
+ * qless_score_dots: 0 (default) tcgen05 int8 kernel (used when T <= 8), 1 CUDA-core kernel. 1-bit codes
+ * always use the XOR + population-count kernel. Process-wide. */
+qless_status qless_set_score_path(int32_t path);
+
 /* Stage 2 alone (Eq. 2, Eq. 4-5, packing) on fp32 rows x [n, d]; normalize = 0 skips Eq. 2 so that
  * already-normalised rows can be fed. Same outputs and packing as above. Needs no workspace. */
 qless_status qless_quantize(

@@ -24,7 +24,7 @@ EXPORTS = [
     "qless_score_dots_workspace", "qless_score_dots", "qless_select_topk_workspace", "qless_select_topk",
     "qless_project_quantize_host_workspace", "qless_project_quantize_host", "qless_profile_enable",
     "qless_profile_collect", "qless_kernel_launches", "qless_select_topk_static",
-    "qless_set_projection_path",
+    "qless_set_projection_path", "qless_set_score_path",
 ]
 SELECT_STATIC_MAX_N = 1 << 22
 
@@ -90,6 +90,8 @@ def lib():
         L.qless_select_topk_workspace.argtypes = [i64]
         L.qless_select_topk.restype = C.c_int
         L.qless_select_topk.argtypes = [vp, i64, C.c_double, vp, C.POINTER(i64), vp, sz, vp]
+        L.qless_set_score_path.restype = C.c_int
+        L.qless_set_score_path.argtypes = [i32]
         L.qless_set_projection_path.restype = C.c_int
         L.qless_set_projection_path.argtypes = [i32]
         L.qless_select_topk_static.restype = C.c_int
@@ -317,3 +319,8 @@ def qless_select_topk_static(scores, frac, indices, stream=None):
 def qless_set_projection_path(path):
     """0 = tensor-core projection kernel (default), 1 = CUDA-core cross-check kernel."""
     _check(lib().qless_set_projection_path(int(path)))
+
+
+def qless_set_score_path(path):
+    """0 = tensor-core scoring kernel for 8/4/2-bit codes (default), 1 = CUDA-core kernel."""
+    _check(lib().qless_set_score_path(int(path)))

@@ -80,6 +80,7 @@ ProfileScope::~ProfileScope()
     if (slot_ >= 0) cudaEventRecord(t_prof[slot_].b, st_);
 }
 
+static std::atomic<int> g_score_path{0};        // 0 = tensor cores for 8/4/2-bit codes, 1 = CUDA cores
 static std::atomic<int> g_projection_path{0};   // 0 = tensor cores, 1 = CUDA cores (cross-check hook)
 
 static bool valid_bits(int b) { return b == 1 || b == 2 || b == 4 || b == 8; }
@@ -160,6 +161,13 @@ qless_status qless_set_projection_path(int32_t path)
 {
     QLESS_REQUIRE(path == 0 || path == 1, QLESS_ERR_INVALID_ARG, "path must be 0 (tensor cores) or 1 (CUDA cores)");
     g_projection_path.store(path);
+    return QLESS_OK;
+}
+
+qless_status qless_set_score_path(int32_t path)
+{
+    QLESS_REQUIRE(path == 0 || path == 1, QLESS_ERR_INVALID_ARG, "path must be 0 (tensor cores) or 1 (CUDA cores)");
+    g_score_path.store(path);
     return QLESS_OK;
 }
 
@@ -346,23 +354,23 @@ static qless_status check_score_shape(int64_t N, int32_t V, int32_t d, int32_t b
     return QLESS_OK;
 }
 
-struct ScoreWs { size_t tmult, vmult, eta, off, total; };
-static ScoreWs score_layout(int64_t N, int32_t V, int32_t C, int32_t T)
+struct ScoreWs { size_t tmult, vmult, eta, off, vunp, total; };
+static ScoreWs score_layout(int64_t N, int32_t V, int32_t C, int32_t T, int32_t d, int32_t bits)
 {
     ScoreWs w;
     w.tmult = 0;
     w.vmult = w.tmult + align_up((size_t)C * (size_t)N * 4, 256);
     w.eta = w.vmult + align_up((size_t)C * (size_t)V * 4, 256);
     w.off = w.eta + align_up((size_t)C * (size_t)T * 4, 256);
-    w.total = w.off + align_up((size_t)(T + 1) * 4, 256);
+    w.vunp = w.off + align_up((size_t)(T + 1) * 4, 256);
+    w.total = w.vunp + (bits == 1 ? 0 : score_tc_workspace_bytes(V, C, d, bits));
     return w;
 }
 
 size_t qless_score_workspace(int64_t N, int32_t V, int32_t C, int32_t T, int32_t d, int32_t bits)
 {
-    (void)d; (void)bits;
-    if (N < 0 || V <= 0 || C <= 0 || T <= 0) return 256;
-    return score_layout(N, V, C, T).total;
+    if (N < 0 || V <= 0 || C <= 0 || T <= 0 || d <= 0) return 256;
+    return score_layout(N, V, C, T, d, bits).total;
 }
 
 qless_status qless_score(const void* train_codes, int64_t train_ckpt_stride_bytes, const void* val_codes,
@@ -389,7 +397,7 @@ qless_status qless_score(const void* train_codes, int64_t train_ckpt_stride_byte
     if (N == 0) return QLESS_OK;
     QLESS_REQUIRE(train_codes && val_codes && train_scales && val_scales && scores, QLESS_ERR_INVALID_ARG, "codes, scales and scores are required");
     QLESS_REQUIRE(aligned(train_codes, 16) && aligned(val_codes, 16), QLESS_ERR_INVALID_ARG, "code arrays must be 16-byte aligned");
-    const ScoreWs w = score_layout(N, V, C, T);
+    const ScoreWs w = score_layout(N, V, C, T, d, bits);
     QLESS_REQUIRE(workspace != nullptr && aligned(workspace, 256), QLESS_ERR_WORKSPACE, "workspace must be non-NULL and 256-byte aligned");
     QLESS_REQUIRE(workspace_bytes >= w.total, QLESS_ERR_WORKSPACE, "workspace too small: %zu bytes given, %zu needed", workspace_bytes, w.total);
 
@@ -416,22 +424,30 @@ qless_status qless_score(const void* train_codes, int64_t train_ckpt_stride_byte
     a.train_mult = tmult; a.val_mult = vmult; a.eta_over_cnt = d_eta; a.task_off = d_off;
     a.N = N; a.V = V; a.C = C; a.T = T; a.d = d; a.bits = bits;
     a.scores = scores; a.per_task = per_task; a.dots = nullptr;
-    { ProfileScope ps("score", st);
-      QLESS_CUDA_TRY(launch_score_simt(a, st)); }
+    if (bits != 1 && g_score_path == 0 && score_tc_supported(T)) {
+        unsigned int* flag = timeout_flag_ptr();
+        QLESS_REQUIRE(flag != nullptr, QLESS_ERR_CUDA, "cannot resolve the device timeout flag");
+        ProfileScope ps("score", st);
+        s = launch_score_tc(a, ws + w.vunp, flag, st);
+        if (s != QLESS_OK) return s;
+    } else {
+        ProfileScope ps("score", st);
+        QLESS_CUDA_TRY(launch_score_simt(a, st));
+    }
     return QLESS_OK;
 }
 
 size_t qless_score_dots_workspace(int64_t nt, int32_t V, int32_t d, int32_t bits)
 {
-    (void)nt; (void)V; (void)d; (void)bits;
-    return 256;
+    (void)nt;
+    if (V <= 0 || d <= 0 || bits == 1) return 256;
+    return 256 + score_tc_workspace_bytes(V, 1, d, bits);
 }
 
 qless_status qless_score_dots(const void* train_codes, const void* val_codes, int64_t t0, int64_t nt, int32_t V,
                               int32_t d, int32_t bits, int32_t* dots, void* workspace, size_t workspace_bytes,
                               void* cuda_stream)
 {
-    (void)workspace; (void)workspace_bytes;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     qless_status s = check_score_shape(nt, V, d, bits);
     if (s != QLESS_OK) return s;
@@ -446,7 +462,17 @@ qless_status qless_score_dots(const void* train_codes, const void* val_codes, in
     a.train_mult = nullptr; a.val_mult = nullptr; a.eta_over_cnt = nullptr; a.task_off = nullptr;
     a.N = nt; a.V = V; a.C = 1; a.T = 1; a.d = d; a.bits = bits;
     a.scores = nullptr; a.per_task = nullptr; a.dots = dots;
-    QLESS_CUDA_TRY(launch_score_simt(a, st));
+    if (bits != 1 && g_score_path == 0) {
+        const size_t need = qless_score_dots_workspace(nt, V, d, bits);
+        QLESS_REQUIRE(workspace != nullptr && aligned(workspace, 256), QLESS_ERR_WORKSPACE, "workspace must be non-NULL and 256-byte aligned");
+        QLESS_REQUIRE(workspace_bytes >= need, QLESS_ERR_WORKSPACE, "workspace too small: %zu bytes given, %zu needed", workspace_bytes, need);
+        unsigned int* flag = timeout_flag_ptr();
+        QLESS_REQUIRE(flag != nullptr, QLESS_ERR_CUDA, "cannot resolve the device timeout flag");
+        s = launch_score_tc(a, reinterpret_cast<uint8_t*>(workspace), flag, st);
+        if (s != QLESS_OK) return s;
+    } else {
+        QLESS_CUDA_TRY(launch_score_simt(a, st));
+    }
     return QLESS_OK;
 }
 

@@ -58,6 +58,10 @@ struct ScoreArgs {
     int32_t* dots;              // if non-NULL: write raw integer dots [N][V] of checkpoint 0 only
 };
 cudaError_t launch_score_simt(const ScoreArgs& a, cudaStream_t st);
+// Tensor-core scoring for bits in {8, 4, 2} (score_tc.cu). T must be <= 8 (score_tc_supported).
+bool score_tc_supported(int32_t T);
+size_t score_tc_workspace_bytes(int32_t V, int32_t C, int32_t d, int32_t bits);
+qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned int* timeout_word, cudaStream_t st);
 // multipliers: mult = (scale == 0) ? 0 : 1/sqrt(sumsq) (cosine) or scale/alpha (dequant);
 // sumsq NULL => recomputed from codes.
 cudaError_t launch_multipliers(const uint8_t* codes, int64_t ckpt_stride, const float* scales,

@@ -1,0 +1,417 @@
+// Stage 3 for 8-, 4- and 2-bit codes on the tensor cores (tcgen05.mma kind::i8, int32 accumulators in TMEM).
+//
+// One CTA owns a tile of 128 train rows (UMMA M). For each checkpoint it streams the tile's codes and the
+// validation codes K-block by K-block (128 codes = 128 bytes per row per block, 128-byte-swizzled K-major
+// operands) and accumulates D[t, v] = sum_m q_t,m q_v,m for up to 512 validation vectors at once (two MMAs
+// of N <= 256 per K step). After the last K block of a checkpoint the epilogue warps read the accumulator
+// (thread = train row), apply the per-vector multipliers (Eq. 6), form the per-task means and add
+// eta_i * mean to the running per-task sums; after the last checkpoint they take the max over tasks.
+// The N x V x C similarity tensor never exists in memory.
+//
+// 8-bit train codes go from global memory to the MMA operand buffer by TMA. 4- and 2-bit train codes
+// arrive packed (TMA, no swizzle) in a staging buffer; four unpack warps sign-extend them to int8 and
+// write the swizzled operand rows themselves (generic-proxy stores + fence.proxy.async). Validation codes
+// are unpacked once per call into a workspace (they are a few MB and stay in L2). Inside a 128-code block
+// the unpackers place the codes in a fixed permutation, the same for both operands, which an inner
+// product does not see.
+//
+// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer (+ TMEM allocation), warps 2-5 unpack
+// (idle for 8-bit), warps 6-9 epilogue. All waits are bounded.
+#include "qless_kernels.h"
+#include "tc_common.cuh"
+
+namespace qless {
+
+namespace {
+
+using namespace tc;
+
+constexpr int TM = 128;                    // train rows per tile
+constexpr int KB = 128;                    // codes (= unpacked bytes) per row per K block
+constexpr int A_STAGE = TM * KB;           // 16 KiB
+constexpr int MAX_STAGES = 8;
+constexpr int NTHREADS = 320;
+constexpr int TMAX = 8;                    // tasks held in registers by the epilogue
+
+struct ScoreTcParams {
+    int64_t N;
+    int32_t V, C, T, d, bits;
+    int32_t vpad;               // validation rows per tile, multiple of 16, <= 512
+    int32_t n1, n2;             // MMA N of the two halves (n1 + n2 = vpad)
+    int32_t nA, nB, nP;         // pipeline depths: operand A, operand B, packed staging
+    const float* train_mult;    // [C][N]
+    const float* val_mult;      // [C][V]
+    const float* eta_over_cnt;  // [C][T]
+    const int32_t* task_off;    // [T+1]
+    float* scores;
+    float* per_task;
+    int32_t* dots;              // raw integer dots [N][V] (C = 1) instead of scores
+    unsigned int* timeout_word;
+};
+
+struct __align__(8) ScoreBars {
+    uint64_t a_full[MAX_STAGES], a_empty[MAX_STAGES], b_full[MAX_STAGES], b_empty[MAX_STAGES];
+    uint64_t p_full[MAX_STAGES], p_empty[MAX_STAGES], d_full, d_empty;
+    uint32_t tmem_base, abort_flag;
+    int32_t task_off[65];
+    float mv[512];
+};
+
+// 8 packed 4-bit codes -> two words of four int8 (low nibbles, high nibbles)
+__device__ __forceinline__ void unpack4(uint32_t w, uint32_t& lo, uint32_t& hi)
+{
+    lo = __vsub4((w & 0x0F0F0F0Fu) ^ 0x08080808u, 0x08080808u);
+    hi = __vsub4(((w >> 4) & 0x0F0F0F0Fu) ^ 0x08080808u, 0x08080808u);
+}
+// 16 packed 2-bit codes -> four words of four int8 (field f of every byte -> word f)
+__device__ __forceinline__ void unpack2(uint32_t w, uint32_t (&o)[4])
+{
+#pragma unroll
+    for (int f = 0; f < 4; ++f) o[f] = __vsub4(((w >> (2 * f)) & 0x03030303u) ^ 0x02020202u, 0x02020202u);
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(NTHREADS, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_constant__ CUtensorMap tmap_val1,
+                const __grid_constant__ CUtensorMap tmap_val2, const ScoreTcParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int b_stage = p.vpad * KB;                       // bytes; multiple of 2048
+    constexpr int P_STAGE = (BITS == 8) ? 0 : TM * 16 * BITS;     // packed staging bytes per stage
+    uint8_t* sA = smem;
+    uint8_t* sB = sA + (size_t)p.nA * A_STAGE;
+    uint8_t* sP = sB + (size_t)p.nB * b_stage;
+    ScoreBars* bars = reinterpret_cast<ScoreBars*>(sP + (size_t)p.nP * P_STAGE);
+    volatile uint32_t* abort_flag = &bars->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nkb = p.d / KB;
+    const int num_vt = (p.V + p.vpad - 1) / p.vpad;
+    const int64_t num_tiles = (p.N + TM - 1) / TM;
+    const uint32_t idesc1 = make_idesc(/*D=S32*/ 2, /*A=S8*/ 1, /*B=S8*/ 1, TM, p.n1);
+    const uint32_t idesc2 = make_idesc(2, 1, 1, TM, p.n2 > 0 ? p.n2 : 16);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MAX_STAGES; ++s) {
+            mbar_init(smem_u32(&bars->a_full[s]), BITS == 8 ? 1 : 128);
+            mbar_init(smem_u32(&bars->a_empty[s]), 1);
+            mbar_init(smem_u32(&bars->b_full[s]), 1);
+            mbar_init(smem_u32(&bars->b_empty[s]), 1);
+            mbar_init(smem_u32(&bars->p_full[s]), 1);
+            mbar_init(smem_u32(&bars->p_empty[s]), 128);
+        }
+        mbar_init(smem_u32(&bars->d_full), 1);
+        mbar_init(smem_u32(&bars->d_empty), 128);
+        bars->abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tmap_train); prefetch_tmap(&tmap_val1); prefetch_tmap(&tmap_val2);
+    }
+    if (p.task_off != nullptr)
+        for (int j = threadIdx.x; j <= p.T; j += NTHREADS) bars->task_off[j] = p.task_off[j];
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&bars->tmem_base), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = bars->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------- TMA producer -------------------------------
+        if (lane == 0) {
+            uint32_t itA = 0, itB = 0;      // stage counters (A counts staging stages when BITS < 8)
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                for (int vt = 0; vt < num_vt && ok; ++vt)
+                    for (int i = 0; i < p.C && ok; ++i)
+                        for (int kb = 0; kb < nkb; ++kb, ++itA, ++itB) {
+                            // train operand (or its packed form)
+                            if (BITS == 8) {
+                                const int s = itA % p.nA;
+                                if (!mbar_wait(smem_u32(&bars->a_empty[s]), ((itA / p.nA) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) { ok = false; break; }
+                                const uint32_t full = smem_u32(&bars->a_full[s]);
+                                mbar_arrive_expect_tx(full, A_STAGE);
+                                tma_load_3d(smem_u32(sA + (size_t)s * A_STAGE), &tmap_train, full, kb * KB, (int32_t)(tile * TM), i);
+                            } else {
+                                const int s = itA % p.nP;
+                                if (!mbar_wait(smem_u32(&bars->p_empty[s]), ((itA / p.nP) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) { ok = false; break; }
+                                const uint32_t full = smem_u32(&bars->p_full[s]);
+                                mbar_arrive_expect_tx(full, P_STAGE);
+                                tma_load_3d(smem_u32(sP + (size_t)s * P_STAGE), &tmap_train, full, kb * 16 * BITS, (int32_t)(tile * TM), i);
+                            }
+                            // validation operand (int8, possibly from the unpacked workspace copy)
+                            const int sb = itB % p.nB;
+                            if (!mbar_wait(smem_u32(&bars->b_empty[sb]), ((itB / p.nB) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) { ok = false; break; }
+                            const uint32_t bfull = smem_u32(&bars->b_full[sb]);
+                            mbar_arrive_expect_tx(bfull, (uint32_t)b_stage);
+                            uint8_t* dstB = sB + (size_t)sb * b_stage;
+                            tma_load_3d(smem_u32(dstB), &tmap_val1, bfull, kb * KB, vt * p.vpad, i);
+                            if (p.n2 > 0) tma_load_3d(smem_u32(dstB + (size_t)p.n1 * KB), &tmap_val2, bfull, kb * KB, vt * p.vpad + p.n1, i);
+                        }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------- MMA issuer -------------------------------
+        if (lane == 0) {
+            uint32_t itA = 0, itB = 0, n_acc = 0;
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x)
+                for (int vt = 0; vt < num_vt && ok; ++vt)
+                    for (int i = 0; i < p.C && ok; ++i, ++n_acc) {
+                        if (!mbar_wait(smem_u32(&bars->d_empty), (n_acc & 1u) ^ 1u, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
+                        tc_fence_after();
+                        for (int kb = 0; kb < nkb; ++kb, ++itA, ++itB) {
+                            const int sa = itA % p.nA, sb = itB % p.nB;
+                            if (!mbar_wait(smem_u32(&bars->a_full[sa]), (itA / p.nA) & 1u, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
+                            if (!mbar_wait(smem_u32(&bars->b_full[sb]), (itB / p.nB) & 1u, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
+                            tc_fence_after();
+                            const uint64_t adesc = make_smem_desc_sw128(smem_u32(sA + (size_t)sa * A_STAGE));
+                            const uint64_t bdesc1 = make_smem_desc_sw128(smem_u32(sB + (size_t)sb * b_stage));
+                            const uint64_t bdesc2 = make_smem_desc_sw128(smem_u32(sB + (size_t)sb * b_stage + (size_t)p.n1 * KB));
+#pragma unroll
+                            for (int k = 0; k < KB / 32; ++k) {
+                                const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
+                                mma_i8_ss(tmem_base, adesc + (uint64_t)(k * 2), bdesc1 + (uint64_t)(k * 2), idesc1, acc);
+                                if (p.n2 > 0) mma_i8_ss(tmem_base + p.n1, adesc + (uint64_t)(k * 2), bdesc2 + (uint64_t)(k * 2), idesc2, acc);
+                            }
+                            mma_commit(smem_u32(&bars->a_empty[sa]));
+                            mma_commit(smem_u32(&bars->b_empty[sb]));
+                        }
+                        if (ok) mma_commit(smem_u32(&bars->d_full));
+                    }
+        }
+    } else if (warp < 6) {
+        // ------------------------------- unpack warps (4- and 2-bit train codes) -------------------------------
+        if (BITS != 8) {
+            const int row = (warp - 2) * 32 + lane;               // row of the 128-row tile
+            uint32_t it = 0;
+            bool ok = true;
+            const int64_t my_tiles = (num_tiles > blockIdx.x) ? (num_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+            const int64_t total = my_tiles * num_vt * p.C * nkb;
+            for (int64_t q = 0; q < total && ok; ++q, ++it) {
+                const int sp = it % p.nP, sa = it % p.nA;
+                ok = mbar_wait(smem_u32(&bars->p_full[sp]), (it / p.nP) & 1u, abort_flag, p.timeout_word, TO_UNPACK);
+                ok = ok && mbar_wait(smem_u32(&bars->a_empty[sa]), ((it / p.nA) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_UNPACK);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                const uint4* src = reinterpret_cast<const uint4*>(sP + (size_t)sp * P_STAGE + (size_t)row * (16 * BITS));
+                uint8_t* dst_row = sA + (size_t)sa * A_STAGE + (size_t)row * KB;
+                uint32_t out[32];
+#pragma unroll
+                for (int c = 0; c < (16 * BITS) / 16; ++c) {
+                    const uint4 w = src[c];
+                    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (BITS == 4) {
+                            unpack4(ww[u], out[(c * 4 + u) * 2], out[(c * 4 + u) * 2 + 1]);
+                        } else {
+                            uint32_t o4[4];
+                            unpack2(ww[u], o4);
+#pragma unroll
+                            for (int f = 0; f < 4; ++f) out[(c * 4 + u) * 4 + f] = o4[f];
+                        }
+                    }
+                }
+                // swizzled operand row: 16-byte chunk c of row r lives at chunk position c ^ (r & 7)
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    *reinterpret_cast<uint4*>(dst_row + ((c ^ (row & 7)) << 4)) =
+                        make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
+                fence_proxy_async_smem();                    // make the stores visible to the tensor core's reads
+                mbar_arrive(smem_u32(&bars->a_full[sa]));
+                mbar_arrive(smem_u32(&bars->p_empty[sp]));
+            }
+        }
+    } else {
+        // ------------------------------- epilogue -------------------------------
+        const int q = warp & 3;
+        const int tl = q * 32 + lane;                        // row of the tile = TMEM lane
+        const int et = threadIdx.x - 6 * 32;                 // 0..127 among the epilogue threads
+        uint32_t n_acc = 0;
+        bool ok = true;
+        for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            const int64_t t = tile * TM + tl;
+            float A[TMAX];
+#pragma unroll
+            for (int j = 0; j < TMAX; ++j) A[j] = 0.0f;
+            for (int vt = 0; vt < num_vt && ok; ++vt) {
+                const int v0 = vt * p.vpad;
+                const int vcount = min(p.vpad, p.V - v0);
+                for (int i = 0; i < p.C && ok; ++i, ++n_acc) {
+                    if (p.dots == nullptr) {
+                        // this checkpoint's validation multipliers -> shared memory (epilogue threads only)
+                        asm volatile("bar.sync 1, 128;" ::: "memory");
+                        for (int v = et; v < p.vpad; v += 128) bars->mv[v] = (v < vcount) ? p.val_mult[(int64_t)i * p.V + v0 + v] : 0.0f;
+                        asm volatile("bar.sync 1, 128;" ::: "memory");
+                    }
+                    ok = mbar_wait(smem_u32(&bars->d_full), n_acc & 1u, abort_flag, p.timeout_word, TO_EPILOGUE);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+                    const float mt = (p.dots == nullptr && t < p.N) ? p.train_mult[(int64_t)i * p.N + t] : 0.0f;
+                    int j = 0;
+                    if (p.dots == nullptr) while (j < p.T - 1 && bars->task_off[j + 1] <= v0) ++j;
+                    float task_sum = 0.0f;
+#pragma unroll 1
+                    for (int c0 = 0; c0 < p.vpad; c0 += 32) {
+                        uint32_t v[32];
+                        tmem_ld_x32(taddr + c0, v);
+                        tmem_wait_ld();
+                        if (c0 + 32 >= p.vpad) {              // accumulator fully read: release it
+                            tc_fence_before();
+                            mbar_arrive(smem_u32(&bars->d_empty));
+                        }
+                        if (p.dots != nullptr) {
+                            if (t < p.N) {
+#pragma unroll
+                                for (int k = 0; k < 32; ++k)
+                                    if (c0 + k < vcount) p.dots[t * p.V + v0 + c0 + k] = (int32_t)v[k];
+                            }
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < 32; ++k) {
+                                const int col = c0 + k;
+                                if (col < vcount) {
+                                    if (v0 + col >= bars->task_off[j + 1]) {       // task j complete
+                                        const float add = task_sum * mt * p.eta_over_cnt[i * p.T + j];
+#pragma unroll
+                                        for (int jj = 0; jj < TMAX; ++jj) if (jj == j) A[jj] += add;
+                                        task_sum = 0.0f;
+                                        ++j;
+                                    }
+                                    task_sum += __fmul_rn((float)(int32_t)v[k], bars->mv[col]);
+                                }
+                            }
+                        }
+                    }
+                    if (p.dots == nullptr) {
+                        const float add = task_sum * mt * p.eta_over_cnt[i * p.T + j];
+#pragma unroll
+                        for (int jj = 0; jj < TMAX; ++jj) if (jj == j) A[jj] += add;
+                    }
+                }
+            }
+            if (ok && p.dots == nullptr && t < p.N) {
+                float best = A[0];
+#pragma unroll
+                for (int jj = 1; jj < TMAX; ++jj) if (jj < p.T) best = fmaxf(best, A[jj]);
+                p.scores[t] = best;
+                if (p.per_task) {
+#pragma unroll
+                    for (int jj = 0; jj < TMAX; ++jj) if (jj < p.T) p.per_task[t * p.T + jj] = A[jj];
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// Validation codes -> int8 [C][V][d] in the permutation the train-side unpack warps use.
+template <int BITS>
+__global__ void unpack_val_kernel(const uint8_t* __restrict__ codes, int64_t ckpt_stride, int32_t V, int32_t C, int32_t d,
+                                  uint8_t* __restrict__ out)
+{
+    const int words_per_row = d * BITS / 32;
+    const int64_t total = (int64_t)C * V * words_per_row;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t rowid = idx / words_per_row;
+        const int wq = (int)(idx - rowid * words_per_row);
+        const int64_t i = rowid / V, v = rowid - i * V;
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(codes + i * ckpt_stride + v * (int64_t)(d * BITS / 8) + 4 * wq);
+        uint32_t* o = reinterpret_cast<uint32_t*>(out + rowid * d) + wq * (8 / BITS);
+        if (BITS == 4) { unpack4(w, o[0], o[1]); }
+        else { uint32_t o4[4]; unpack2(w, o4); o[0] = o4[0]; o[1] = o4[1]; o[2] = o4[2]; o[3] = o4[3]; }
+    }
+}
+
+}  // namespace
+
+bool score_tc_supported(int32_t T) { return T <= TMAX; }
+
+size_t score_tc_workspace_bytes(int32_t V, int32_t C, int32_t d, int32_t bits)
+{
+    return bits == 8 ? 0 : align_up((size_t)C * V * d, 256);
+}
+
+// a.dots != NULL: raw dots of one checkpoint. val_unpacked: workspace of score_tc_workspace_bytes (bits < 8).
+qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned int* timeout_word, cudaStream_t st)
+{
+    if (a.N == 0) return QLESS_OK;
+    ScoreTcParams p;
+    p.N = a.N; p.V = a.V; p.C = a.C; p.T = a.T; p.d = a.d; p.bits = a.bits;
+    const int vpad_all = (a.V + 15) / 16 * 16;
+    p.vpad = vpad_all < 512 ? vpad_all : 512;
+    p.n1 = p.vpad < 256 ? p.vpad : 256;
+    p.n2 = p.vpad - p.n1;
+    const int64_t row_bytes = (int64_t)a.d * a.bits / 8;
+
+    // shared-memory plan
+    const size_t budget = 227 * 1024 - 1024 - sizeof(ScoreBars) - 64;
+    const size_t b_stage = (size_t)p.vpad * KB;
+    const size_t p_stage = a.bits == 8 ? 0 : (size_t)TM * 16 * a.bits;
+    int nA = 2, nB = 2, nP = a.bits == 8 ? 0 : 2;
+    auto used = [&]() { return (size_t)nA * A_STAGE + (size_t)nB * b_stage + (size_t)nP * p_stage; };
+    bool grew = true;
+    while (grew) {        // grow the deepest-latency pipelines round-robin while they fit
+        grew = false;
+        if (nB < MAX_STAGES && used() + b_stage <= budget) { ++nB; grew = true; }
+        if (a.bits == 8 && nA < nB && used() + A_STAGE <= budget) { ++nA; grew = true; }
+        if (a.bits != 8 && nP < MAX_STAGES && nP < nB && used() + p_stage <= budget) { ++nP; grew = true; }
+    }
+    if (a.bits != 8 && used() + A_STAGE <= budget && nA < 3) ++nA;
+    p.nA = nA; p.nB = nB; p.nP = nP > 0 ? nP : 1;
+    const size_t smem = 1024 + used() + sizeof(ScoreBars);
+
+    p.train_mult = a.train_mult; p.val_mult = a.val_mult; p.eta_over_cnt = a.eta_over_cnt; p.task_off = a.task_off;
+    p.scores = a.scores; p.per_task = a.per_task; p.dots = a.dots; p.timeout_word = timeout_word;
+
+    const uint8_t* val_src = a.val;
+    int64_t val_row = row_bytes, val_stride = a.val_stride;
+    if (a.bits != 8) {
+        const int64_t total_words = (int64_t)a.C * a.V * (row_bytes / 4);
+        int64_t blocks = (total_words + 255) / 256;
+        if (blocks > (int64_t)sm_count() * 8) blocks = (int64_t)sm_count() * 8;
+        if (a.bits == 4) unpack_val_kernel<4><<<(unsigned)blocks, 256, 0, st>>>(a.val, a.val_stride, a.V, a.C, a.d, val_unpacked);
+        else unpack_val_kernel<2><<<(unsigned)blocks, 256, 0, st>>>(a.val, a.val_stride, a.V, a.C, a.d, val_unpacked);
+        count_launches(1);
+        val_src = val_unpacked; val_row = a.d; val_stride = (int64_t)a.V * a.d;
+    }
+    CUtensorMap tm_train, tm_v1, tm_v2;
+    qless_status s;
+    const int64_t tstride = a.C > 1 ? a.train_stride : (int64_t)a.N * row_bytes;
+    s = make_tmap_3d_u8(&tm_train, a.train, (uint64_t)row_bytes, (uint64_t)a.N, (uint64_t)a.C, (uint64_t)row_bytes,
+                        (uint64_t)tstride, a.bits == 8 ? 128 : 16 * a.bits, TM, a.bits == 8);
+    if (s != QLESS_OK) return s;
+    const int64_t vstride = a.C > 1 ? val_stride : (int64_t)a.V * val_row;
+    s = make_tmap_3d_u8(&tm_v1, val_src, (uint64_t)val_row, (uint64_t)a.V, (uint64_t)a.C, (uint64_t)val_row, (uint64_t)vstride, 128, p.n1, true);
+    if (s != QLESS_OK) return s;
+    s = make_tmap_3d_u8(&tm_v2, val_src, (uint64_t)val_row, (uint64_t)a.V, (uint64_t)a.C, (uint64_t)val_row, (uint64_t)vstride, 128,
+                        p.n2 > 0 ? p.n2 : 16, true);
+    if (s != QLESS_OK) return s;
+
+    const int64_t tiles = (a.N + TM - 1) / TM;
+    int64_t grid = sm_count();
+    if (grid > tiles) grid = tiles;
+#define QLESS_LAUNCH_SCORE_TC(B)                                                                                    \
+    QLESS_CUDA_TRY(cudaFuncSetAttribute(score_tc_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+    score_tc_kernel<B><<<(unsigned)grid, NTHREADS, smem, st>>>(tm_train, tm_v1, tm_v2, p);
+    if (a.bits == 8) { QLESS_LAUNCH_SCORE_TC(8) }
+    else if (a.bits == 4) { QLESS_LAUNCH_SCORE_TC(4) }
+    else { QLESS_LAUNCH_SCORE_TC(2) }
+#undef QLESS_LAUNCH_SCORE_TC
+    count_launches(1);
+    QLESS_CUDA_TRY(cudaGetLastError());
+    return QLESS_OK;
+}
+
+}  // namespace qless

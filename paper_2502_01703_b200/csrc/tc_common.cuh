@@ -68,6 +68,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const CUtensorMap
         ::"r"(smem_dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap* tmap, uint32_t bar, int32_t c0,
+                                            int32_t c1, int32_t c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tmap)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
@@ -167,5 +175,11 @@ __device__ __forceinline__ void mma_commit(uint32_t bar)
 // elem_bytes in {1, 2}; box_inner * elem_bytes must be 128.
 qless_status make_tmap_2d_sw128(CUtensorMap* out, const void* base, int elem_bytes, uint64_t inner, uint64_t outer,
                                 uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer);
+
+// Host: 3-D byte tensor map [outer2][outer1][inner bytes] (uint8 elements). swizzle128 = true needs a 128-byte
+// wide box; otherwise the box lands in shared memory as plain rows of box_inner bytes (a multiple of 16).
+qless_status make_tmap_3d_u8(CUtensorMap* out, const void* base, uint64_t inner_bytes, uint64_t outer1, uint64_t outer2,
+                             uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t box_inner, uint32_t box_outer1,
+                             bool swizzle128);
 
 }  // namespace qless
