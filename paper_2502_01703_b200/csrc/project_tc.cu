@@ -49,7 +49,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                   int32_t num_chunks, uint64_t seed, float* __restrict__ part, unsigned int* __restrict__ timeout_word)
 {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);    // 1 KiB aligned, still a shared pointer
     Barriers* bars = reinterpret_cast<Barriers*>(smem + (size_t)SB * B_STAGE_BYTES);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 

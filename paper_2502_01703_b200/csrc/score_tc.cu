@@ -54,7 +54,7 @@ struct __align__(8) ScoreBars {
     uint64_t p_full[MAX_STAGES], p_empty[MAX_STAGES], d_full, d_empty;
     uint32_t tmem_base, abort_flag;
     int32_t task_off[65];
-    float mv[512];
+    __align__(16) float mv[512];
 };
 
 // 8 packed 4-bit codes -> two words of four int8 (low nibbles, high nibbles)
@@ -76,7 +76,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 const __grid_constant__ CUtensorMap tmap_val2, const ScoreTcParams p)
 {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);    // 1 KiB aligned, still a shared pointer
     const int b_stage = p.vpad * KB;                       // bytes; multiple of 2048
     constexpr int P_STAGE = (BITS == 8) ? 0 : TM * 16 * BITS;     // packed staging bytes per stage
     uint8_t* sA = smem;
@@ -255,6 +255,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                     const float mt = (p.dots == nullptr && t < p.N) ? p.train_mult[(int64_t)i * p.N + t] : 0.0f;
                     int j = 0;
                     if (p.dots == nullptr) while (j < p.T - 1 && bars->task_off[j + 1] <= v0) ++j;
+                    int next_b = (p.dots == nullptr) ? bars->task_off[j + 1] - v0 : 0x7FFFFFFF;   // first column of task j+1
                     float task_sum = 0.0f;
 #pragma unroll 1
                     for (int c0 = 0; c0 < p.vpad; c0 += 32) {
@@ -272,23 +273,36 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                                     if (c0 + k < vcount) p.dots[t * p.V + v0 + c0 + k] = (int32_t)v[k];
                             }
                         } else {
+                            // columns >= vcount carry a zero multiplier, so they add nothing
+                            float x[32];
 #pragma unroll
-                            for (int k = 0; k < 32; ++k) {
-                                const int col = c0 + k;
-                                if (col < vcount) {
-                                    if (v0 + col >= bars->task_off[j + 1]) {       // task j complete
+                            for (int k4 = 0; k4 < 8; ++k4) {
+                                const float4 m4 = *reinterpret_cast<const float4*>(&bars->mv[c0 + 4 * k4]);
+                                x[4 * k4 + 0] = __fmul_rn((float)(int32_t)v[4 * k4 + 0], m4.x);
+                                x[4 * k4 + 1] = __fmul_rn((float)(int32_t)v[4 * k4 + 1], m4.y);
+                                x[4 * k4 + 2] = __fmul_rn((float)(int32_t)v[4 * k4 + 2], m4.z);
+                                x[4 * k4 + 3] = __fmul_rn((float)(int32_t)v[4 * k4 + 3], m4.w);
+                            }
+                            if (next_b >= c0 + 32) {          // whole chunk inside task j (the common case)
+#pragma unroll
+                                for (int k = 0; k < 32; ++k) task_sum += x[k];
+                            } else {
+#pragma unroll
+                                for (int k = 0; k < 32; ++k) {
+                                    if (c0 + k == next_b && j < p.T) {   // task j complete
                                         const float add = task_sum * mt * p.eta_over_cnt[i * p.T + j];
 #pragma unroll
                                         for (int jj = 0; jj < TMAX; ++jj) if (jj == j) A[jj] += add;
                                         task_sum = 0.0f;
                                         ++j;
+                                        next_b = (j < p.T) ? bars->task_off[j + 1] - v0 : 0x7FFFFFFF;
                                     }
-                                    task_sum += __fmul_rn((float)(int32_t)v[k], bars->mv[col]);
+                                    task_sum += x[k];
                                 }
                             }
                         }
                     }
-                    if (p.dots == nullptr) {
+                    if (p.dots == nullptr && j < p.T) {
                         const float add = task_sum * mt * p.eta_over_cnt[i * p.T + j];
 #pragma unroll
                         for (int jj = 0; jj < TMAX; ++jj) if (jj == j) A[jj] += add;
