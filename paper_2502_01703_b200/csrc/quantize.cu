@@ -29,7 +29,7 @@ __device__ __forceinline__ int warp_sum_i(int x)
 }
 
 template <int BITS>
-__global__ void __launch_bounds__(QT)
+__global__ void __launch_bounds__(QT, 5)
 quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale, int64_t n, int32_t d,
                 int normalize, uint8_t* __restrict__ codes, float* __restrict__ scales,
                 int32_t* __restrict__ sumsq, float* __restrict__ proj_out)
@@ -67,45 +67,36 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
             }
             x[k] = a;
         }
-        // ---- Eq. 2: norm in double, one fp32 reciprocal, one fp32 multiply per element ----
-        bool zero_vec = false;
-        if (normalize) {
-            double acc = 0.0;
+        // ---- one block reduction for both Eq. 2 and Eq. 4: sum of squares (double) and max |x| of the raw row.
+        // yhat_m = fl(x_m * rn) is monotone in |x_m|, so max_m |yhat_m| = fl(max_m |x_m| * rn) exactly.
+        double acc = 0.0;
+        float mx = 0.0f;
 #pragma unroll
-            for (int k = 0; k < QMAX_V4; ++k) {
+        for (int k = 0; k < QMAX_V4; ++k) {
+            if (normalize) {
                 acc += (double)x[k].x * (double)x[k].x; acc += (double)x[k].y * (double)x[k].y;
                 acc += (double)x[k].z * (double)x[k].z; acc += (double)x[k].w * (double)x[k].w;
             }
-            acc = warp_sum(acc);
-            if (lane == 0) s_d[warp] = acc;
-            __syncthreads();
-            double tot = 0.0;
-#pragma unroll
-            for (int w = 0; w < QT / 32; ++w) tot += s_d[w];
-            const float nrm = (float)sqrt(tot);
-            if (nrm == 0.0f) {
-                zero_vec = true;
-            } else {
-                const float rn = __fdiv_rn(1.0f, nrm);
-#pragma unroll
-                for (int k = 0; k < QMAX_V4; ++k) {
-                    x[k].x = __fmul_rn(x[k].x, rn); x[k].y = __fmul_rn(x[k].y, rn);
-                    x[k].z = __fmul_rn(x[k].z, rn); x[k].w = __fmul_rn(x[k].w, rn);
-                }
-            }
-        }
-        // ---- Eq. 4: S = max |x| ----
-        float mx = 0.0f;
-#pragma unroll
-        for (int k = 0; k < QMAX_V4; ++k)
             mx = fmaxf(fmaxf(mx, fmaxf(fabsf(x[k].x), fabsf(x[k].y))), fmaxf(fabsf(x[k].z), fabsf(x[k].w)));
+        }
+        if (normalize) acc = warp_sum(acc);
         mx = warp_max(mx);
-        if (lane == 0) s_f[warp] = mx;
+        if (lane == 0) { s_d[warp] = acc; s_f[warp] = mx; }
         __syncthreads();
+        double tot = 0.0;
         float S = 0.0f;
 #pragma unroll
-        for (int w = 0; w < QT / 32; ++w) S = fmaxf(S, s_f[w]);
-        if (zero_vec) S = 0.0f;
+        for (int w = 0; w < QT / 32; ++w) { tot += s_d[w]; S = fmaxf(S, s_f[w]); }
+        float rn = 1.0f;
+        if (normalize) {
+            const float nrm = (float)sqrt(tot);
+            if (nrm == 0.0f) {
+                S = 0.0f;                               // zero vector
+            } else {
+                rn = __fdiv_rn(1.0f, nrm);
+                S = __fmul_rn(S, rn);
+            }
+        }
 
         // ---- Eq. 5 + pack into shared memory ----
         constexpr int ALPHA = (BITS == 1) ? 1 : ((1 << (BITS - 1)) - 1);
@@ -115,7 +106,7 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
         for (int k = 0; k < QMAX_V4; ++k) {
             const int c = tid + k * QT;
             if (c < nv4) {      // warp-uniform: nv4 is a multiple of 32
-                const float e[4] = {x[k].x, x[k].y, x[k].z, x[k].w};
+                const float e[4] = {__fmul_rn(x[k].x, rn), __fmul_rn(x[k].y, rn), __fmul_rn(x[k].z, rn), __fmul_rn(x[k].w, rn)};
                 int q[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {

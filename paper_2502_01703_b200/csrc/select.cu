@@ -64,24 +64,42 @@ select_hist_kernel(const float* __restrict__ scores, int64_t N, const SelectStat
         if (s_h[i]) atomicAdd(&hist[i], s_h[i]);
 }
 
-// One block: walk the histogram from the top bin down to the bin that holds the k_rem-th largest key.
+// One block of 1024 threads: find the bin that holds the k_rem-th largest key, counting from the top bin
+// down (block-wide prefix sum over the reversed histogram).
 template <int PASS>
-__global__ void select_scan_kernel(const uint32_t* __restrict__ hist, SelectState* __restrict__ state, int64_t k)
+__global__ void __launch_bounds__(1024)
+select_scan_kernel(const uint32_t* __restrict__ hist, SelectState* __restrict__ state, int64_t k)
 {
-    if (threadIdx.x != 0) return;
     constexpr int NB = (PASS == 2) ? 1024 : 2048;
     constexpr int SHIFT = (PASS == 2) ? 10 : 11;
-    int64_t k_rem = (PASS == 0) ? k : state->k_rem;
+    constexpr int PER = NB / 1024;
+    __shared__ int64_t s_w[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t k_rem = (PASS == 0) ? k : state->k_rem;
     const uint32_t prefix = (PASS == 0) ? 0u : state->prefix;
-    int64_t above = 0;
-    int b = NB - 1;
-    for (; b > 0; --b) {
-        const int64_t c = hist[b];
-        if (above + c >= k_rem) break;
-        above += c;
+    int64_t c[PER];
+    int64_t mine = 0;
+#pragma unroll
+    for (int u = 0; u < PER; ++u) { c[u] = hist[NB - 1 - (tid * PER + u)]; mine += c[u]; }
+    int64_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int64_t a = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += a;
     }
-    state->prefix = (prefix << SHIFT) | (uint32_t)b;
-    state->k_rem = k_rem - above;
+    if (lane == 31) s_w[warp] = inc;
+    __syncthreads();            // also orders every thread's read of *state before the single write below
+    int64_t pre = inc - mine;
+    for (int w = 0; w < warp; ++w) pre += s_w[w];
+#pragma unroll
+    for (int u = 0; u < PER; ++u) {
+        if (pre < k_rem && k_rem <= pre + c[u]) {       // exactly one (thread, u) satisfies this
+            const int b = NB - 1 - (tid * PER + u);
+            state->prefix = (prefix << SHIFT) | (uint32_t)b;
+            state->k_rem = k_rem - pre;
+        }
+        pre += c[u];
+    }
 }
 
 __global__ void __launch_bounds__(SEL_T)
@@ -216,11 +234,11 @@ cudaError_t launch_select_topk(const float* scores, int64_t N, int64_t k, int64_
     if (hb > cap) hb = cap;
     if (hb < 1) hb = 1;
     select_hist_kernel<0><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, w.state, w.hist);
-    select_scan_kernel<0><<<1, 32, 0, st>>>(w.hist, w.state, k);
+    select_scan_kernel<0><<<1, 1024, 0, st>>>(w.hist, w.state, k);
     select_hist_kernel<1><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, w.state, w.hist + 2048);
-    select_scan_kernel<1><<<1, 32, 0, st>>>(w.hist + 2048, w.state, k);
+    select_scan_kernel<1><<<1, 1024, 0, st>>>(w.hist + 2048, w.state, k);
     select_hist_kernel<2><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, w.state, w.hist + 4096);
-    select_scan_kernel<2><<<1, 32, 0, st>>>(w.hist + 4096, w.state, k);
+    select_scan_kernel<2><<<1, 1024, 0, st>>>(w.hist + 4096, w.state, k);
     const int64_t nblk = sel_nblk(N);
     select_count_kernel<<<(unsigned)nblk, SEL_T, 0, st>>>(scores, N, w.state, w.blk_cnt);
     select_block_scan_kernel<<<1, 1024, 0, st>>>(w.blk_cnt, nblk, w.blk_off);
