@@ -240,7 +240,7 @@ qless_status qless_project_quantize(const void* grads, qless_dtype dtype, int64_
     float* part = reinterpret_cast<float*>(ws + w.part_off);
     if (g_projection_path == 0 && (P / 64) * n < ((int64_t)1 << 31)) {
         CUtensorMap tmap;
-        s = make_tmap_2d_sw128(&tmap, gamma, 2, 64, (uint64_t)(P / 64) * (uint64_t)n, 128, 64, 256);
+        s = make_tmap_2d_sw128(&tmap, gamma, 2, 64, (uint64_t)(P / 64) * (uint64_t)n, 128, 64, 128);
         if (s != QLESS_OK) return s;
         unsigned int* flag = timeout_flag_ptr();
         QLESS_REQUIRE(flag != nullptr, QLESS_ERR_CUDA, "cannot resolve the device timeout flag");

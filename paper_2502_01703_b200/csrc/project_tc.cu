@@ -2,20 +2,23 @@
 //
 //   part[s][i][r] = sum_{j in K-chunk s} Gamma[i][j] * sign(r, j)          (bf16 x bf16 -> fp32)
 //
-// as a GEMM with the roles chosen for the hardware: the M side (128 TMEM lanes) is a tile of 128
-// projected coordinates r, whose +-1.0 operand rows are generated from Philox straight into tensor
-// memory (no shared-memory traffic, no swizzle); the N side is a tile of up to 256 gradient rows,
-// streamed by TMA from a K-blocked copy of Gamma ([P/64][n][64], so that each 256 x 64 operand tile is one
-// contiguous 32 KiB span) into 128-byte-swizzled shared memory. The accumulator
-// (128 x 256 fp32) occupies TMEM columns 0..255, four 128-deep stages of the sign operand occupy
-// columns 256..511. Each CTA is persistent and walks work items (gradient tile, K-chunk, r tile)
-// K-chunk-major, so that at any time all CTAs read the same slab of Gamma (L2 reuse); after each
-// K-chunk the accumulator is drained to a per-chunk partial, which bounds the length of any fp32
-// accumulation chain and makes the final sum order fixed.
+// as a GEMM with the roles chosen for the hardware. Two CTAs on neighbouring SMs form a pair and run
+// one 256 x 256 x K tensor-core tile (tcgen05.mma cta_group::2). The M side (2 x 128 TMEM lanes) is a
+// tile of 256 projected coordinates r, 128 per CTA, whose +-1.0 operand rows each CTA generates from
+// Philox straight into its own tensor memory (no shared-memory traffic, no swizzle). The N side is a tile
+// of up to 256 gradient rows, of which each CTA streams half (128 rows) by TMA from a K-blocked copy of
+// Gamma ([P/64][n][64], so that each 128 x 64 operand tile is one contiguous 16 KiB span) into
+// 128-byte-swizzled shared memory: pairing halves the bytes every SM pulls from L2 and the shared-memory
+// traffic of the gradient operand. In each CTA the accumulator (128 x 256 fp32) occupies TMEM columns
+// 0..255 and four 128-deep stages of the sign operand occupy columns 256..511. Pairs are persistent and
+// walk work items (gradient tile, K-chunk, r tile) K-chunk-major, so that at any time all pairs read the
+// same slab of Gamma (L2 reuse); after each K-chunk the accumulator is drained to a per-chunk partial,
+// which bounds the length of any fp32 accumulation chain and makes the final sum order fixed.
 //
-// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer (+ TMEM allocation), warps 2-5 sign
-// generators, warps 6-9 accumulator drain. All waits are bounded; a wait that gives up raises the
-// device timeout word and every role leaves its loop.
+// Warp roles (320 threads per CTA): warp 0 TMA producer, warp 1 MMA issuer (leader CTA only; + TMEM
+// allocation in both), warps 2-5 sign generators, warps 6-9 accumulator drain. The leader's barriers
+// collect the arrivals of both CTAs; tcgen05.commit releases stages in both CTAs at once. All waits are
+// bounded; a wait that gives up raises the device timeout word and every role leaves its loop.
 #include "qless_kernels.h"
 #include "tc_common.cuh"
 
@@ -25,16 +28,16 @@ namespace {
 
 using namespace tc;
 
-constexpr int BM = 128;                 // projected coordinates per tile (UMMA M)
-constexpr int BN = 256;                 // gradient rows per tile (UMMA N)
+constexpr int BM = 128;                 // projected coordinates per CTA (UMMA M = 256 per pair)
+constexpr int BN = 256;                 // gradient rows per tile (UMMA N), 128 of them staged by each CTA
 constexpr int BK = 64;                  // K per shared-memory stage (128 bytes of bf16)
-constexpr int SB = 6;                   // shared-memory stages of the gradient operand
+constexpr int SB = 12;                  // shared-memory stages of the gradient operand
 constexpr int SA = 4;                   // TMEM stages of the sign operand, 128 K each (64 columns)
-constexpr int B_STAGE_BYTES = BN * BK * 2;     // 32 KiB
+constexpr int B_STAGE_BYTES = (BN / 2) * BK * 2;     // 16 KiB per CTA
 constexpr int TMEM_COLS = 512;
 constexpr int D_COL = 0, A_COL = 256;
 constexpr int NTHREADS = 320;
-constexpr uint32_t IDESC = make_idesc(/*D=F32*/ 1, /*A=BF16*/ 1, /*B=BF16*/ 1, BM, BN);
+constexpr uint32_t IDESC = make_idesc(/*D=F32*/ 1, /*A=BF16*/ 1, /*B=BF16*/ 1, 2 * BM, BN);
 
 struct __align__(8) Barriers {
     uint64_t b_full[SB], b_empty[SB], a_full[SA], a_empty[SA], d_full, d_empty;
@@ -44,7 +47,7 @@ struct __align__(8) Barriers {
 
 constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)SB * B_STAGE_BYTES + sizeof(Barriers);
 
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int32_t d, int64_t P, int64_t chunk,
                   int32_t num_chunks, uint64_t seed, float* __restrict__ part, unsigned int* __restrict__ timeout_word)
 {
@@ -54,25 +57,29 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_dt = d / BM;
+    const uint32_t rank = cluster_ctarank();            // 0 = leader of the pair
+    const int64_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int num_dt = (d + 2 * BM - 1) / (2 * BM);     // tiles of 256 projected coordinates
     const int num_nt = (int)((n + BN - 1) / BN);
     const int64_t num_items = (int64_t)num_nt * num_chunks * num_dt;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < SB; ++s) { mbar_init(smem_u32(&bars->b_full[s]), 1); mbar_init(smem_u32(&bars->b_empty[s]), 1); }
-        for (int s = 0; s < SA; ++s) { mbar_init(smem_u32(&bars->a_full[s]), 128); mbar_init(smem_u32(&bars->a_empty[s]), 1); }
+        // a_full / d_empty of the leader collect one arrival per generator / drain warp of both CTAs
+        for (int s = 0; s < SA; ++s) { mbar_init(smem_u32(&bars->a_full[s]), 8); mbar_init(smem_u32(&bars->a_empty[s]), 1); }
         mbar_init(smem_u32(&bars->d_full), 1);
-        mbar_init(smem_u32(&bars->d_empty), 128);
+        mbar_init(smem_u32(&bars->d_empty), 8);
         bars->abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmap_gamma);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(&bars->tmem_base), TMEM_COLS);
-        tmem_relinquish();
+        tmem_alloc_pair(smem_u32(&bars->tmem_base), TMEM_COLS);
+        tmem_relinquish_pair();
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();                 // both CTAs' barriers are initialised before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
 
@@ -81,7 +88,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
         if (lane == 0) {
             uint32_t it = 0;     // global stage counter
             bool ok = true;
-            for (int64_t item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+            for (int64_t item = pair; item < num_items && ok; item += num_pairs) {
                 const int64_t nt = item / ((int64_t)num_chunks * num_dt);
                 const int kc = (int)((item / num_dt) % num_chunks);
                 const int64_t k0 = (int64_t)kc * chunk;
@@ -89,13 +96,15 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % SB;
                     const uint32_t ph = (it / SB) & 1u;
-                    if (!mbar_wait(smem_u32(&bars->b_empty[s]), ph ^ 1u, abort_flag, timeout_word, TO_PRODUCER)) { ok = false; break; }
-                    const uint32_t full = smem_u32(&bars->b_full[s]);
-                    mbar_arrive_expect_tx(full, B_STAGE_BYTES);
-                    // tiled Gamma: K block kb64 holds its n rows of 64 columns contiguously
+                    if (!mbar_wait_cluster(smem_u32(&bars->b_empty[s]), ph ^ 1u, abort_flag, timeout_word, TO_PRODUCER)) { ok = false; break; }
+                    // both halves of the stage complete on the leader's barrier, which expects their sum
+                    const uint32_t full = map_to_cta(smem_u32(&bars->b_full[s]), 0);
+                    if (rank == 0) mbar_arrive_expect_tx(smem_u32(&bars->b_full[s]), 2 * B_STAGE_BYTES);
+                    // tiled Gamma: K block kb64 holds its n rows of 64 columns contiguously; this CTA takes
+                    // rows [rank*128, rank*128 + 128) of the 256-row tile
                     const int64_t kb64 = (k0 >> 6) + kb;
-                    tma_load_2d(smem_u32(smem + (size_t)s * B_STAGE_BYTES), &tmap_gamma, full, 0,
-                                (int32_t)(kb64 * n + nt * BN));
+                    tma_load_2d_pair(smem_u32(smem + (size_t)s * B_STAGE_BYTES), &tmap_gamma, full, 0,
+                                     (int32_t)(kb64 * n + nt * BN + rank * (BN / 2)));
                 }
             }
             if (!ok) {
@@ -103,36 +112,37 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 for (int s = 0; s < SB; ++s)
                     for (uint32_t t = 0; t < (1u << 16); ++t)
                         if (mbar_try_wait(smem_u32(&bars->b_full[s]), 0) || mbar_try_wait(smem_u32(&bars->b_full[s]), 1)) break;
+                for (volatile int spin = 0; spin < (1 << 16); ++spin) { }    // the peer's barrier sees our copies: give them time to land
             }
         }
     } else if (warp == 1) {
         // ------------------------------- MMA issuer -------------------------------
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
             uint32_t itb = 0, ita = 0, n_item = 0;
             bool ok = true;
-            for (int64_t item = blockIdx.x; item < num_items && ok; item += gridDim.x, ++n_item) {
+            for (int64_t item = pair; item < num_items && ok; item += num_pairs, ++n_item) {
                 const int kc = (int)((item / num_dt) % num_chunks);
                 const int64_t k0 = (int64_t)kc * chunk;
                 const int nkb = (int)((min(P, k0 + chunk) - k0) / BK);
-                if (!mbar_wait(smem_u32(&bars->d_empty), (n_item & 1u) ^ 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
+                if (!mbar_wait_cluster(smem_u32(&bars->d_empty), (n_item & 1u) ^ 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
                 tc_fence_after();
                 for (int kb = 0; kb < nkb; ++kb, ++itb) {
                     const int sb = itb % SB;
-                    if (!mbar_wait(smem_u32(&bars->b_full[sb]), (itb / SB) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
+                    if (!mbar_wait_cluster(smem_u32(&bars->b_full[sb]), (itb / SB) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
                     const int sa = ita % SA;
                     if ((kb & 1) == 0) {
-                        if (!mbar_wait(smem_u32(&bars->a_full[sa]), (ita / SA) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
+                        if (!mbar_wait_cluster(smem_u32(&bars->a_full[sa]), (ita / SA) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
                     }
                     tc_fence_after();
                     const uint64_t bdesc = make_smem_desc_sw128(smem_u32(smem + (size_t)sb * B_STAGE_BYTES));
                     const uint32_t a_addr = tmem_base + A_COL + sa * 64 + (kb & 1) * 32;
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)
-                        mma_f16_ts(tmem_base + D_COL, a_addr + k * 8, bdesc + (uint64_t)(k * 2), IDESC, (kb > 0 || k > 0) ? 1u : 0u);
-                    mma_commit(smem_u32(&bars->b_empty[sb]));
-                    if (kb & 1) { mma_commit(smem_u32(&bars->a_empty[sa])); ++ita; }
+                        mma_f16_ts_pair(tmem_base + D_COL, a_addr + k * 8, bdesc + (uint64_t)(k * 2), IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+                    mma_commit_pair(smem_u32(&bars->b_empty[sb]));
+                    if (kb & 1) { mma_commit_pair(smem_u32(&bars->a_empty[sa])); ++ita; }
                 }
-                if (ok) mma_commit(smem_u32(&bars->d_full));
+                if (ok) mma_commit_pair(smem_u32(&bars->d_full));
             }
         }
     } else if (warp < 6) {
@@ -140,8 +150,8 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
         const int q = warp & 3;                                  // TMEM lane quadrant this warp may access
         uint32_t ita = 0;
         bool ok = true;
-        for (int64_t item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
-            const int dt = (int)(item % num_dt);
+        for (int64_t item = pair; item < num_items && ok; item += num_pairs) {
+            const int dt = (int)(item % num_dt) * 2 + (int)rank;           // this CTA's 128 projected coordinates
             const int kc = (int)((item / num_dt) % num_chunks);
             const int64_t k0 = (int64_t)kc * chunk;
             const int nka = (int)((min(P, k0 + chunk) - k0) / 128);
@@ -150,7 +160,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 const int sa = ita % SA;
                 uint32_t w[4];
                 rademacher_block(seed, r, (uint32_t)((k0 >> 7) + ka), w);     // overlaps with the wait below
-                ok = mbar_wait(smem_u32(&bars->a_empty[sa]), ((ita / SA) & 1u) ^ 1u, abort_flag, timeout_word, TO_GENERATOR);
+                ok = mbar_wait_cluster(smem_u32(&bars->a_empty[sa]), ((ita / SA) & 1u) ^ 1u, abort_flag, timeout_word, TO_GENERATOR);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
@@ -164,7 +174,8 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 }
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(smem_u32(&bars->a_full[sa]));
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->a_full[sa]), 0));
             }
         }
     } else {
@@ -172,16 +183,16 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
         const int q = warp & 3;
         uint32_t n_item = 0;
         bool ok = true;
-        for (int64_t item = blockIdx.x; item < num_items && ok; item += gridDim.x, ++n_item) {
-            const int dt = (int)(item % num_dt);
+        for (int64_t item = pair; item < num_items && ok; item += num_pairs, ++n_item) {
+            const int dt = (int)(item % num_dt) * 2 + (int)rank;
             const int kc = (int)((item / num_dt) % num_chunks);
             const int64_t nt = item / ((int64_t)num_chunks * num_dt);
-            ok = mbar_wait(smem_u32(&bars->d_full), n_item & 1u, abort_flag, timeout_word, TO_EPILOGUE);
+            ok = mbar_wait_cluster(smem_u32(&bars->d_full), n_item & 1u, abort_flag, timeout_word, TO_EPILOGUE);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after();
             float* out = part + ((int64_t)kc * n + nt * BN) * d + dt * BM + q * 32 + lane;
-            const int64_t rows_here = min((int64_t)BN, n - nt * BN);
+            const int64_t rows_here = (dt * BM < d) ? min((int64_t)BN, n - nt * BN) : 0;   // d = 128 (mod 256): last half tile is empty
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + D_COL;
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
@@ -190,7 +201,8 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 tmem_wait_ld();
                 if (c0 + 32 == BN) {          // accumulator fully read: hand it back before the stores
                     tc_fence_before();
-                    mbar_arrive(smem_u32(&bars->d_empty));
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->d_empty), 0));
                 }
 #pragma unroll
                 for (int k = 0; k < 32; ++k)
@@ -201,9 +213,10 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
 
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();                 // neither CTA frees tensor memory or exits while its peer may still touch it
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
     }
 }
 
@@ -215,15 +228,11 @@ cudaError_t launch_project_tc(const CUtensorMap& tmap, const ProjectPlan& pl, ui
                               unsigned int* timeout_word, cudaStream_t st)
 {
     if (pl.n == 0) return cudaSuccess;
-    static thread_local bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(project_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
-    const int64_t items = (int64_t)((pl.n + BN - 1) / BN) * pl.num_chunks * (pl.d / BM);
-    int64_t grid = sm_count();
-    if (grid > items) grid = items;
+    cudaError_t e = cudaFuncSetAttribute(project_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    const int64_t items = (int64_t)((pl.n + BN - 1) / BN) * pl.num_chunks * ((pl.d + 2 * BM - 1) / (2 * BM));
+    int64_t grid = (sm_count() / 2) * 2;               // CTA pairs
+    if (grid > 2 * items) grid = 2 * items;
     project_tc_kernel<<<(unsigned)grid, NTHREADS, SMEM_BYTES, st>>>(tmap, pl.n, pl.d, pl.P, pl.chunk, pl.num_chunks, seed,
                                                                     part, timeout_word);
     count_launches(1);

@@ -35,7 +35,7 @@ cudaError_t launch_project_simt(const __nv_bfloat16* gamma_tiled, const ProjectP
                                 uint64_t seed, float* part, cudaStream_t st);
 
 // Tensor-core projection (project_tc.cu). The tensor map describes tiled Gamma as [(P/64)*n][64] bf16 with a
-// 64 x 256 box.
+// 64 x 128 box.
 cudaError_t launch_project_tc(const CUtensorMap& tmap, const ProjectPlan& pl, uint64_t seed, float* part,
                               unsigned int* timeout_word, cudaStream_t st);
 
