@@ -24,7 +24,7 @@ EXPORTS = [
     "qless_score_dots_workspace", "qless_score_dots", "qless_select_topk_workspace", "qless_select_topk",
     "qless_project_quantize_host_workspace", "qless_project_quantize_host", "qless_profile_enable",
     "qless_profile_collect", "qless_kernel_launches", "qless_select_topk_static",
-    "qless_set_projection_path", "qless_set_score_path",
+    "qless_set_projection_path", "qless_set_score_path", "qless_microbench",
 ]
 SELECT_STATIC_MAX_N = 1 << 22
 
@@ -90,6 +90,8 @@ def lib():
         L.qless_select_topk_workspace.argtypes = [i64]
         L.qless_select_topk.restype = C.c_int
         L.qless_select_topk.argtypes = [vp, i64, C.c_double, vp, C.POINTER(i64), vp, sz, vp]
+        L.qless_microbench.restype = C.c_int
+        L.qless_microbench.argtypes = [i32, i32, C.POINTER(C.c_float), C.POINTER(C.c_double), vp, sz, vp]
         L.qless_set_score_path.restype = C.c_int
         L.qless_set_score_path.argtypes = [i32]
         L.qless_set_projection_path.restype = C.c_int
@@ -324,3 +326,15 @@ def qless_set_projection_path(path):
 def qless_set_score_path(path):
     """0 = tensor-core scoring kernel for 8/4/2-bit codes (default), 1 = CUDA-core kernel."""
     _check(lib().qless_set_score_path(int(path)))
+
+
+MICROBENCH = {"bf16_ss": 0, "bf16_ts": 1, "i8_ss": 2, "bf16_ss_pair": 3, "bf16_ts_pair": 4, "i8_ss_pair": 5, "popc": 6}
+
+
+def qless_microbench(what, iters, device="cuda", stream=None):
+    """(milliseconds, operations) of one peak-rate micro-benchmark; `what` is a key of MICROBENCH."""
+    ms, ops = C.c_float(0), C.c_double(0)
+    scratch = torch.empty(4 << 20, dtype=torch.uint8, device=device)
+    _check(lib().qless_microbench(MICROBENCH[what], int(iters), C.byref(ms), C.byref(ops), _ptr(scratch), scratch.numel(),
+                                  _stream(stream)))
+    return ms.value, ops.value

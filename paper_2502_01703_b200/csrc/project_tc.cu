@@ -15,8 +15,8 @@
 // same slab of Gamma (L2 reuse); after each K-chunk the accumulator is drained to a per-chunk partial,
 // which bounds the length of any fp32 accumulation chain and makes the final sum order fixed.
 //
-// Warp roles (320 threads per CTA): warp 0 TMA producer, warp 1 MMA issuer (leader CTA only; + TMEM
-// allocation in both), warps 2-5 sign generators, warps 6-9 accumulator drain. The leader's barriers
+// Warp roles (448 threads per CTA): warp 0 TMA producer, warp 1 MMA issuer (leader CTA only; + TMEM
+// allocation in both), warps 2-5 and 10-13 sign generators, warps 6-9 accumulator drain. The leader's barriers
 // collect the arrivals of both CTAs; tcgen05.commit releases stages in both CTAs at once. All waits are
 // bounded; a wait that gives up raises the device timeout word and every role leaves its loop.
 #include "qless_kernels.h"
@@ -36,7 +36,7 @@ constexpr int SA = 4;                   // TMEM stages of the sign operand, 128 
 constexpr int B_STAGE_BYTES = (BN / 2) * BK * 2;     // 16 KiB per CTA
 constexpr int TMEM_COLS = 512;
 constexpr int D_COL = 0, A_COL = 256;
-constexpr int NTHREADS = 320;
+constexpr int NTHREADS = 448;
 constexpr uint32_t IDESC = make_idesc(/*D=F32*/ 1, /*A=BF16*/ 1, /*B=BF16*/ 1, 2 * BM, BN);
 
 struct __align__(8) Barriers {
@@ -145,9 +145,12 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 if (ok) mma_commit_pair(smem_u32(&bars->d_full));
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 6 || warp >= 10) {
         // ------------------------------- sign generators -------------------------------
+        // two groups of four warps (2-5 and 10-13) take alternate 128-deep stages, so that the latency of one
+        // stage (Philox chain, TMEM store, barrier round trip) overlaps the next
         const int q = warp & 3;                                  // TMEM lane quadrant this warp may access
+        const uint32_t grp = (warp >= 10) ? 1u : 0u;
         uint32_t ita = 0;
         bool ok = true;
         for (int64_t item = pair; item < num_items && ok; item += num_pairs) {
@@ -157,6 +160,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
             const int nka = (int)((min(P, k0 + chunk) - k0) / 128);
             const uint32_t r = (uint32_t)(dt * BM + q * 32 + lane);
             for (int ka = 0; ka < nka; ++ka, ++ita) {
+                if ((ita & 1u) != grp) continue;
                 const int sa = ita % SA;
                 uint32_t w[4];
                 rademacher_block(seed, r, (uint32_t)((k0 >> 7) + ka), w);     // overlaps with the wait below
