@@ -30,10 +30,11 @@ using namespace tc;
 
 constexpr int BM = 128;                 // projected coordinates per CTA (UMMA M = 256 per pair)
 constexpr int BN = 256;                 // gradient rows per tile (UMMA N), 128 of them staged by each CTA
-constexpr int BK = 64;                  // K per shared-memory stage (128 bytes of bf16)
-constexpr int SB = 12;                  // shared-memory stages of the gradient operand
+constexpr int BK = 128;                 // K per shared-memory stage: two 64-column (128-byte) swizzle panels
+constexpr int SB = 6;                   // shared-memory stages of the gradient operand
 constexpr int SA = 4;                   // TMEM stages of the sign operand, 128 K each (64 columns)
-constexpr int B_STAGE_BYTES = (BN / 2) * BK * 2;     // 16 KiB per CTA
+constexpr int B_PANEL_BYTES = (BN / 2) * 64 * 2;      // 16 KiB: 128 rows x 64 columns
+constexpr int B_STAGE_BYTES = 2 * B_PANEL_BYTES;      // 32 KiB per CTA
 constexpr int TMEM_COLS = 512;
 constexpr int D_COL = 0, A_COL = 256;
 constexpr int NTHREADS = 448;
@@ -102,9 +103,11 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                     if (rank == 0) mbar_arrive_expect_tx(smem_u32(&bars->b_full[s]), 2 * B_STAGE_BYTES);
                     // tiled Gamma: K block kb64 holds its n rows of 64 columns contiguously; this CTA takes
                     // rows [rank*128, rank*128 + 128) of the 256-row tile
-                    const int64_t kb64 = (k0 >> 6) + kb;
-                    tma_load_2d_pair(smem_u32(smem + (size_t)s * B_STAGE_BYTES), &tmap_gamma, full, 0,
-                                     (int32_t)(kb64 * n + nt * BN + rank * (BN / 2)));
+                    const int64_t kb64 = (k0 >> 6) + 2 * kb;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_2d_pair(smem_u32(smem + (size_t)s * B_STAGE_BYTES + h * B_PANEL_BYTES), &tmap_gamma, full, 0,
+                                         (int32_t)((kb64 + h) * n + nt * BN + rank * (BN / 2)));
                 }
             }
             if (!ok) {
@@ -130,17 +133,17 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                     const int sb = itb % SB;
                     if (!mbar_wait_cluster(smem_u32(&bars->b_full[sb]), (itb / SB) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
                     const int sa = ita % SA;
-                    if ((kb & 1) == 0) {
-                        if (!mbar_wait_cluster(smem_u32(&bars->a_full[sa]), (ita / SA) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
-                    }
+                    if (!mbar_wait_cluster(smem_u32(&bars->a_full[sa]), (ita / SA) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
                     tc_fence_after();
-                    const uint64_t bdesc = make_smem_desc_sw128(smem_u32(smem + (size_t)sb * B_STAGE_BYTES));
-                    const uint32_t a_addr = tmem_base + A_COL + sa * 64 + (kb & 1) * 32;
+                    const uint32_t a_addr = tmem_base + A_COL + sa * 64;
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        mma_f16_ts_pair(tmem_base + D_COL, a_addr + k * 8, bdesc + (uint64_t)(k * 2), IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+                    for (int k = 0; k < BK / 16; ++k) {
+                        const uint64_t bdesc = make_smem_desc_sw128(smem_u32(smem + (size_t)sb * B_STAGE_BYTES + (k >> 2) * B_PANEL_BYTES));
+                        mma_f16_ts_pair(tmem_base + D_COL, a_addr + k * 8, bdesc + (uint64_t)((k & 3) * 2), IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+                    }
                     mma_commit_pair(smem_u32(&bars->b_empty[sb]));
-                    if (kb & 1) { mma_commit_pair(smem_u32(&bars->a_empty[sa])); ++ita; }
+                    mma_commit_pair(smem_u32(&bars->a_empty[sa]));
+                    ++ita;
                 }
                 if (ok) mma_commit_pair(smem_u32(&bars->d_full));
             }
