@@ -30,11 +30,11 @@ using namespace tc;
 
 constexpr int BM = 128;                 // projected coordinates per CTA (UMMA M = 256 per pair)
 constexpr int BN = 256;                 // gradient rows per tile (UMMA N), 128 of them staged by each CTA
-constexpr int BK = 128;                 // K per shared-memory stage: two 64-column (128-byte) swizzle panels
-constexpr int SB = 6;                   // shared-memory stages of the gradient operand
+constexpr int BK = 256;                 // K per shared-memory stage: four 64-column (128-byte) swizzle panels
+constexpr int SB = 3;                   // shared-memory stages of the gradient operand
 constexpr int SA = 4;                   // TMEM stages of the sign operand, 128 K each (64 columns)
 constexpr int B_PANEL_BYTES = (BN / 2) * 64 * 2;      // 16 KiB: 128 rows x 64 columns
-constexpr int B_STAGE_BYTES = 2 * B_PANEL_BYTES;      // 32 KiB per CTA
+constexpr int B_STAGE_BYTES = (BK / 64) * B_PANEL_BYTES;      // 64 KiB per CTA
 constexpr int TMEM_COLS = 512;
 constexpr int D_COL = 0, A_COL = 256;
 constexpr int NTHREADS = 448;
@@ -93,19 +93,20 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 const int64_t nt = item / ((int64_t)num_chunks * num_dt);
                 const int kc = (int)((item / num_dt) % num_chunks);
                 const int64_t k0 = (int64_t)kc * chunk;
-                const int nkb = (int)((min(P, k0 + chunk) - k0) / BK);
+                const int64_t klen = min(P, k0 + chunk) - k0;              // multiple of 128
+                const int nkb = (int)((klen + BK - 1) / BK);
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % SB;
                     const uint32_t ph = (it / SB) & 1u;
                     if (!mbar_wait_cluster(smem_u32(&bars->b_empty[s]), ph ^ 1u, abort_flag, timeout_word, TO_PRODUCER)) { ok = false; break; }
                     // both halves of the stage complete on the leader's barrier, which expects their sum
+                    const int panels = (int)min((int64_t)(BK / 64), (klen - (int64_t)kb * BK) >> 6);   // a chunk may end on half a stage
                     const uint32_t full = map_to_cta(smem_u32(&bars->b_full[s]), 0);
-                    if (rank == 0) mbar_arrive_expect_tx(smem_u32(&bars->b_full[s]), 2 * B_STAGE_BYTES);
+                    if (rank == 0) mbar_arrive_expect_tx(smem_u32(&bars->b_full[s]), 2 * panels * B_PANEL_BYTES);
                     // tiled Gamma: K block kb64 holds its n rows of 64 columns contiguously; this CTA takes
                     // rows [rank*128, rank*128 + 128) of the 256-row tile
-                    const int64_t kb64 = (k0 >> 6) + 2 * kb;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h)
+                    const int64_t kb64 = (k0 >> 6) + (BK / 64) * kb;
+                    for (int h = 0; h < panels; ++h)
                         tma_load_2d_pair(smem_u32(smem + (size_t)s * B_STAGE_BYTES + h * B_PANEL_BYTES), &tmap_gamma, full, 0,
                                          (int32_t)((kb64 + h) * n + nt * BN + rank * (BN / 2)));
                 }
@@ -126,24 +127,28 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
             for (int64_t item = pair; item < num_items && ok; item += num_pairs, ++n_item) {
                 const int kc = (int)((item / num_dt) % num_chunks);
                 const int64_t k0 = (int64_t)kc * chunk;
-                const int nkb = (int)((min(P, k0 + chunk) - k0) / BK);
+                const int64_t klen = min(P, k0 + chunk) - k0;
+                const int nkb = (int)((klen + BK - 1) / BK);
                 if (!mbar_wait_cluster(smem_u32(&bars->d_empty), (n_item & 1u) ^ 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
                 tc_fence_after();
                 for (int kb = 0; kb < nkb; ++kb, ++itb) {
                     const int sb = itb % SB;
                     if (!mbar_wait_cluster(smem_u32(&bars->b_full[sb]), (itb / SB) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
-                    const int sa = ita % SA;
-                    if (!mbar_wait_cluster(smem_u32(&bars->a_full[sa]), (ita / SA) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a_addr = tmem_base + A_COL + sa * 64;
+                    const int nh = (int)min((int64_t)(BK / 128), (klen - (int64_t)kb * BK) >> 7);
+                    for (int h = 0; h < nh && ok; ++h, ++ita) {                // one 128-deep sign stage at a time
+                        const int sa = ita % SA;
+                        if (!mbar_wait_cluster(smem_u32(&bars->a_full[sa]), (ita / SA) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t a_addr = tmem_base + A_COL + sa * 64;
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k) {
-                        const uint64_t bdesc = make_smem_desc_sw128(smem_u32(smem + (size_t)sb * B_STAGE_BYTES + (k >> 2) * B_PANEL_BYTES));
-                        mma_f16_ts_pair(tmem_base + D_COL, a_addr + k * 8, bdesc + (uint64_t)((k & 3) * 2), IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+                        for (int k = 0; k < 8; ++k) {
+                            const uint64_t bdesc = make_smem_desc_sw128(smem_u32(smem + (size_t)sb * B_STAGE_BYTES + (2 * h + (k >> 2)) * B_PANEL_BYTES));
+                            mma_f16_ts_pair(tmem_base + D_COL, a_addr + k * 8, bdesc + (uint64_t)((k & 3) * 2), IDESC, (kb > 0 || h > 0 || k > 0) ? 1u : 0u);
+                        }
+                        mma_commit_pair(smem_u32(&bars->a_empty[sa]));
                     }
+                    if (!ok) break;
                     mma_commit_pair(smem_u32(&bars->b_empty[sb]));
-                    mma_commit_pair(smem_u32(&bars->a_empty[sa]));
-                    ++ita;
                 }
                 if (ok) mma_commit_pair(smem_u32(&bars->d_full));
             }
