@@ -5,21 +5,41 @@ namespace qless {
 
 // Gamma_j = m'/(sqrt(v')+eps), m' = b1 m + (1-b1) g, v' = b2 v + (1-b2) g^2, every operation a
 // separately rounded IEEE fp32 operation (no fused multiply-add), result rounded to bf16 (RNE).
-__device__ __forceinline__ float adam_dir(float g, float m, float v, const AdamParams& ap)
+// bm = fl(b1 m), bv = fl(b2 v) are passed in because they are the same for every row of the batch.
+//
+// The IEEE square root and division are the expensive part, and the result only keeps 8 bits. So the
+// quotient is first formed with the approximate reciprocal units (a few ulp of error); unless that value
+// lies close to a bf16 rounding boundary (or outside the normal range) its bf16 rounding is already the one
+// the exact sequence gives, and the exact sequence runs only for the rare remaining elements. The value
+// returned always rounds to the same bf16 as the exact one.
+__device__ __forceinline__ float adam_dir(float g, float bm, float bv, const AdamParams& ap)
 {
-    float m1 = __fadd_rn(__fmul_rn(ap.beta1, m), __fmul_rn(ap.omb1, g));
-    float v1 = __fadd_rn(__fmul_rn(ap.beta2, v), __fmul_rn(ap.omb2, __fmul_rn(g, g)));
-    if (ap.bias_correct) { m1 = __fdiv_rn(m1, ap.c1); v1 = __fdiv_rn(v1, ap.c2); }
+    float m1 = __fadd_rn(bm, __fmul_rn(ap.omb1, g));
+    float v1 = __fadd_rn(bv, __fmul_rn(ap.omb2, __fmul_rn(g, g)));
+    if (!ap.bias_correct) {
+        float rs, rc;
+        asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rs) : "f"(v1));
+        const float den_a = __fadd_rn(__fmul_rn(v1, rs), ap.eps);          // v1 = 0 gives NaN: handled below
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(den_a));
+        const float q = __fmul_rn(m1, rc);
+        const int lo = (int)(__float_as_uint(q) & 0xFFFFu);
+        const float aq = fabsf(q);
+        // NaN fails every comparison, so it takes the exact path too
+        const bool safe = (abs(lo - 0x8000) > 32) && den_a > 1e-30f && den_a < 1e30f && aq > 1e-30f && aq < 1e30f;
+        if (safe) return q;
+    } else {
+        m1 = __fdiv_rn(m1, ap.c1); v1 = __fdiv_rn(v1, ap.c2);
+    }
     const float den = __fadd_rn(__fsqrt_rn(v1), ap.eps);
     return __fdiv_rn(m1, den);
 }
 
 // One thread handles 8 consecutive columns (16-byte bf16 accesses) of AG_ROWS consecutive rows, so the
 // moments m, v (shared by every row of the batch) are read once per AG_ROWS rows instead of once per row.
-constexpr int AG_ROWS = 8;
+constexpr int AG_ROWS = 4;
 
 template <bool BF16_IN, bool ADAM, bool TILED>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 adam_gamma_kernel(const void* __restrict__ grads, int64_t n, int64_t ld, const float* __restrict__ m,
                   const float* __restrict__ v, AdamParams ap, int64_t P, __nv_bfloat16* __restrict__ gamma)
 {
@@ -37,6 +57,8 @@ adam_gamma_kernel(const void* __restrict__ grads, int64_t n, int64_t ld, const f
             const float4 v0 = __ldg(reinterpret_cast<const float4*>(v + j0)), v1 = __ldg(reinterpret_cast<const float4*>(v + j0 + 4));
             mm[0] = m0.x; mm[1] = m0.y; mm[2] = m0.z; mm[3] = m0.w; mm[4] = m1.x; mm[5] = m1.y; mm[6] = m1.z; mm[7] = m1.w;
             vv[0] = v0.x; vv[1] = v0.y; vv[2] = v0.z; vv[3] = v0.w; vv[4] = v1.x; vv[5] = v1.y; vv[6] = v1.z; vv[7] = v1.w;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) { mm[k] = __fmul_rn(ap.beta1, mm[k]); vv[k] = __fmul_rn(ap.beta2, vv[k]); }
         }
         // issue every row's loads before any arithmetic (memory-level parallelism)
         uint4 raw[AG_ROWS][BF16_IN ? 1 : 2];
