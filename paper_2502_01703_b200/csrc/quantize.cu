@@ -45,6 +45,11 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
     const int row_bytes = d * BITS / 8;
 
     for (int64_t row = blockIdx.x; row < n; row += gridDim.x) {
+        // ask L2 for the row this CTA will take next, so that its loads find it there
+        if (tid == 0 && row + gridDim.x < n) {
+            for (int s = 0; s < num_parts; ++s)
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(parts + s * part_stride + (row + gridDim.x) * d), "r"(d * 4) : "memory");
+        }
         float4 x[QMAX_V4];
         // ---- load + fixed-order sum of partials, scaled once ----
 #pragma unroll
@@ -107,34 +112,34 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
             const int c = tid + k * QT;
             if (c < nv4) {      // warp-uniform: nv4 is a multiple of 32
                 const float e[4] = {__fmul_rn(x[k].x, rn), __fmul_rn(x[k].y, rn), __fmul_rn(x[k].z, rn), __fmul_rn(x[k].w, rn)};
-                int q[4];
+                if (BITS == 1) {
+                    uint32_t nib = 0;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (BITS == 1) {
-                        q[u] = (S > 0.0f) ? ((e[u] < 0.0f) ? -1 : 1) : 0;
-                    } else {
-                        int t = __float2int_rn(__fmul_rn(e[u], r));
-                        t = max(-ALPHA, min(ALPHA, t));
-                        q[u] = t;
-                    }
-                    ss += q[u] * q[u];
-                }
-                if (BITS == 8) {
-                    const uint32_t w = (uint32_t)(q[0] & 0xFF) | ((uint32_t)(q[1] & 0xFF) << 8) |
-                                       ((uint32_t)(q[2] & 0xFF) << 16) | ((uint32_t)(q[3] & 0xFF) << 24);
-                    reinterpret_cast<uint32_t*>(s_out)[c] = w;
-                } else if (BITS == 4) {
-                    const uint32_t w = (uint32_t)(q[0] & 0xF) | ((uint32_t)(q[1] & 0xF) << 4) |
-                                       ((uint32_t)(q[2] & 0xF) << 8) | ((uint32_t)(q[3] & 0xF) << 12);
-                    reinterpret_cast<uint16_t*>(s_out)[c] = (uint16_t)w;
-                } else if (BITS == 2) {
-                    const uint32_t w = (uint32_t)(q[0] & 0x3) | ((uint32_t)(q[1] & 0x3) << 2) |
-                                       ((uint32_t)(q[2] & 0x3) << 4) | ((uint32_t)(q[3] & 0x3) << 6);
-                    s_out[c] = (uint8_t)w;
-                } else {
-                    uint32_t nib = (q[0] < 0 ? 1u : 0u) | (q[1] < 0 ? 2u : 0u) | (q[2] < 0 ? 4u : 0u) | (q[3] < 0 ? 8u : 0u);
+                    for (int u = 0; u < 4; ++u) nib |= (S > 0.0f && e[u] < 0.0f) ? (1u << u) : 0u;
+                    ss += (S > 0.0f) ? 4 : 0;
                     const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, nib, 1);
                     if ((lane & 1) == 0) s_out[c >> 1] = (uint8_t)(nib | (hi << 4));
+                } else {
+                    // round-half-even to an integer by adding 1.5 * 2^23: the sum's low mantissa bits are the
+                    // two's-complement code (|yhat r| <= alpha (1 + 2^-23), so no clamp is needed)
+                    uint32_t t[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) t[u] = __float_as_uint(__fadd_rn(__fmul_rn(e[u], r), 12582912.0f));
+                    // low bytes of the four sums -> one word of four int8 codes
+                    const uint32_t w8 = __byte_perm(__byte_perm(t[0], t[1], 0x0040), __byte_perm(t[2], t[3], 0x0040), 0x5410);
+                    ss = __dp4a((int)w8, (int)w8, ss);
+                    if (BITS == 8) {
+                        reinterpret_cast<uint32_t*>(s_out)[c] = w8;
+                    } else if (BITS == 4) {
+                        const uint32_t n4 = w8 & 0x0F0F0F0Fu;
+                        const uint32_t u4 = n4 | (n4 >> 4);                    // bytes 0 and 2 hold two nibbles each
+                        reinterpret_cast<uint16_t*>(s_out)[c] = (uint16_t)__byte_perm(u4, 0u, 0x4420);
+                    } else {
+                        const uint32_t n2 = w8 & 0x03030303u;
+                        const uint32_t u2 = n2 | (n2 >> 6);                    // byte 0: codes 0,1 ; byte 2: codes 2,3
+                        const uint32_t v2 = u2 | (u2 >> 12);                   // byte 0: codes 0..3
+                        s_out[c] = (uint8_t)(v2 & 0xFFu);
+                    }
                 }
             }
         }
