@@ -1,9 +1,11 @@
 // Stage 3 for 8-, 4- and 2-bit codes on the tensor cores (tcgen05.mma kind::i8, int32 accumulators in TMEM).
 //
-// One CTA owns a tile of 128 train rows (UMMA M). For each checkpoint it streams the tile's codes and the
-// validation codes K-block by K-block (128 codes = 128 bytes per row per block, 128-byte-swizzled K-major
-// operands) and accumulates D[t, v] = sum_m q_t,m q_v,m for up to 512 validation vectors at once (two MMAs
-// of N <= 256 per K step). After the last K block of a checkpoint the epilogue warps read the accumulator
+// Two CTAs on neighbouring SMs form a pair (cta_group::2) and own a tile of 256 train rows (UMMA M), 128
+// per CTA. For each checkpoint the pair streams the tile's codes and the validation codes K-block by
+// K-block (128 codes = 128 bytes per row per block, 128-byte-swizzled K-major operands) and accumulates
+// D[t, v] = sum_m q_t,m q_v,m for up to 512 validation vectors at once (two MMAs of N <= 256 per K step);
+// each CTA stages only half of the validation rows of every MMA, which halves what an SM pulls from L2.
+// After the last K block of a checkpoint the epilogue warps of each CTA read their half of the accumulator
 // (thread = train row), apply the per-vector multipliers (Eq. 6), form the per-task means and add
 // eta_i * mean to the running per-task sums; after the last checkpoint they take the max over tasks.
 // The N x V x C similarity tensor never exists in memory.
@@ -15,8 +17,13 @@
 // the unpackers place the codes in a fixed permutation, the same for both operands, which an inner
 // product does not see.
 //
-// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer (+ TMEM allocation), warps 2-5 unpack
-// (idle for 8-bit), warps 6-9 epilogue. All waits are bounded.
+// One barrier per pipeline stage on the leader CTA collects everything the MMAs of that stage need (TMA
+// bytes of both CTAs, and the unpack warps' arrivals); one tcgen05.commit releases the stage in both CTAs:
+// the single MMA-issuing thread runs at the tensor pipe's own pace, so every other instruction it executes
+// is lost tensor time.
+//
+// Warp roles (320 threads per CTA): warp 0 TMA producer, warp 1 MMA issuer (leader only; + TMEM
+// allocation), warps 2-5 unpack (idle for 8-bit), warps 6-9 epilogue. All waits are bounded.
 #include "qless_kernels.h"
 #include "tc_common.cuh"
 
@@ -38,7 +45,7 @@ struct ScoreTcParams {
     int32_t V, C, T, d, bits;
     int32_t vpad;               // validation rows per tile, multiple of 16, <= 512
     int32_t n1, n2;             // MMA N of the two halves (n1 + n2 = vpad)
-    int32_t nA, nB, nP;         // pipeline depths: operand A, operand B, packed staging
+    int32_t nS, nP;             // pipeline depths: operand stages (A + B), packed staging
     const float* train_mult;    // [C][N]
     const float* val_mult;      // [C][V]
     const float* eta_over_cnt;  // [C][T]
@@ -50,7 +57,7 @@ struct ScoreTcParams {
 };
 
 struct __align__(8) ScoreBars {
-    uint64_t a_full[MAX_STAGES], a_empty[MAX_STAGES], b_full[MAX_STAGES], b_empty[MAX_STAGES];
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES];
     uint64_t p_full[MAX_STAGES], p_empty[MAX_STAGES], d_full, d_empty;
     uint32_t tmem_base, abort_flag;
     int32_t task_off[65];
@@ -71,38 +78,39 @@ __device__ __forceinline__ void unpack2(uint32_t w, uint32_t (&o)[4])
 }
 
 template <int BITS>
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_constant__ CUtensorMap tmap_val1,
                 const __grid_constant__ CUtensorMap tmap_val2, const ScoreTcParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);    // 1 KiB aligned, still a shared pointer
-    const int b_stage = p.vpad * KB;                       // bytes; multiple of 2048
+    const int bh1 = (p.n1 / 2) * KB, bh2 = (p.n2 / 2) * KB;      // bytes of this CTA's rows of the two MMA halves
+    const int stage_bytes = A_STAGE + bh1 + bh2;                  // multiple of 1024
     constexpr int P_STAGE = (BITS == 8) ? 0 : TM * 16 * BITS;     // packed staging bytes per stage
-    uint8_t* sA = smem;
-    uint8_t* sB = sA + (size_t)p.nA * A_STAGE;
-    uint8_t* sP = sB + (size_t)p.nB * b_stage;
+    uint8_t* sS = smem;                                           // stage s: [A 16 KiB][B half 1][B half 2]
+    uint8_t* sP = sS + (size_t)p.nS * stage_bytes;
     ScoreBars* bars = reinterpret_cast<ScoreBars*>(sP + (size_t)p.nP * P_STAGE);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int64_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
     const int nkb = p.d / KB;
     const int num_vt = (p.V + p.vpad - 1) / p.vpad;
-    const int64_t num_tiles = (p.N + TM - 1) / TM;
-    const uint32_t idesc1 = make_idesc(/*D=S32*/ 2, /*A=S8*/ 1, /*B=S8*/ 1, TM, p.n1);
-    const uint32_t idesc2 = make_idesc(2, 1, 1, TM, p.n2 > 0 ? p.n2 : 16);
+    const int64_t num_tiles = (p.N + 2 * TM - 1) / (2 * TM);      // tiles of 256 train rows
+    const uint32_t idesc1 = make_idesc(/*D=S32*/ 2, /*A=S8*/ 1, /*B=S8*/ 1, 2 * TM, p.n1);
+    const uint32_t idesc2 = make_idesc(2, 1, 1, 2 * TM, p.n2 > 0 ? p.n2 : 16);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_STAGES; ++s) {
-            mbar_init(smem_u32(&bars->a_full[s]), BITS == 8 ? 1 : 128);
-            mbar_init(smem_u32(&bars->a_empty[s]), 1);
-            mbar_init(smem_u32(&bars->b_full[s]), 1);
-            mbar_init(smem_u32(&bars->b_empty[s]), 1);
+            // leader's full[s]: the producer's expect_tx arrival (+ one arrival per unpack warp of both CTAs)
+            mbar_init(smem_u32(&bars->full[s]), BITS == 8 ? 1 : 9);
+            mbar_init(smem_u32(&bars->empty[s]), 1);
             mbar_init(smem_u32(&bars->p_full[s]), 1);
-            mbar_init(smem_u32(&bars->p_empty[s]), 128);
+            mbar_init(smem_u32(&bars->p_empty[s]), 4);
         }
         mbar_init(smem_u32(&bars->d_full), 1);
-        mbar_init(smem_u32(&bars->d_empty), 128);
+        mbar_init(smem_u32(&bars->d_empty), 8);
         bars->abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmap_train); prefetch_tmap(&tmap_val1); prefetch_tmap(&tmap_val2);
@@ -110,94 +118,91 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
     if (p.task_off != nullptr)
         for (int j = threadIdx.x; j <= p.T; j += NTHREADS) bars->task_off[j] = p.task_off[j];
     if (warp == 1) {
-        tmem_alloc(smem_u32(&bars->tmem_base), 512);
-        tmem_relinquish();
+        tmem_alloc_pair(smem_u32(&bars->tmem_base), 512);
+        tmem_relinquish_pair();
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
 
     if (warp == 0) {
         // ------------------------------- TMA producer -------------------------------
         if (lane == 0) {
-            uint32_t itA = 0, itB = 0;      // stage counters (A counts staging stages when BITS < 8)
+            uint32_t it = 0;
             bool ok = true;
-            for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            const uint32_t tx_total = 2u * (uint32_t)((BITS == 8 ? A_STAGE : 0) + bh1 + bh2);   // both CTAs
+            for (int64_t tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+                const int32_t row0 = (int32_t)(tile * 2 * TM + rank * TM);
                 for (int vt = 0; vt < num_vt && ok; ++vt)
                     for (int i = 0; i < p.C && ok; ++i)
-                        for (int kb = 0; kb < nkb; ++kb, ++itA, ++itB) {
-                            // train operand (or its packed form)
+                        for (int kb = 0; kb < nkb; ++kb, ++it) {
+                            const int s = it % p.nS;
+                            if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), ((it / p.nS) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) { ok = false; break; }
+                            const uint32_t full = map_to_cta(smem_u32(&bars->full[s]), 0);
+                            if (rank == 0) mbar_arrive_expect_tx(smem_u32(&bars->full[s]), tx_total);
+                            uint8_t* st = sS + (size_t)s * stage_bytes;
                             if (BITS == 8) {
-                                const int s = itA % p.nA;
-                                if (!mbar_wait(smem_u32(&bars->a_empty[s]), ((itA / p.nA) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) { ok = false; break; }
-                                const uint32_t full = smem_u32(&bars->a_full[s]);
-                                mbar_arrive_expect_tx(full, A_STAGE);
-                                tma_load_3d(smem_u32(sA + (size_t)s * A_STAGE), &tmap_train, full, kb * KB, (int32_t)(tile * TM), i);
+                                tma_load_3d_pair(smem_u32(st), &tmap_train, full, kb * KB, row0, i);
                             } else {
-                                const int s = itA % p.nP;
-                                if (!mbar_wait(smem_u32(&bars->p_empty[s]), ((itA / p.nP) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) { ok = false; break; }
-                                const uint32_t full = smem_u32(&bars->p_full[s]);
-                                mbar_arrive_expect_tx(full, P_STAGE);
-                                tma_load_3d(smem_u32(sP + (size_t)s * P_STAGE), &tmap_train, full, kb * 16 * BITS, (int32_t)(tile * TM), i);
+                                const int sp = it % p.nP;
+                                if (!mbar_wait(smem_u32(&bars->p_empty[sp]), ((it / p.nP) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) { ok = false; break; }
+                                const uint32_t pfull = smem_u32(&bars->p_full[sp]);
+                                mbar_arrive_expect_tx(pfull, P_STAGE);
+                                tma_load_3d(smem_u32(sP + (size_t)sp * P_STAGE), &tmap_train, pfull, kb * 16 * BITS, row0, i);
                             }
-                            // validation operand (int8, possibly from the unpacked workspace copy)
-                            const int sb = itB % p.nB;
-                            if (!mbar_wait(smem_u32(&bars->b_empty[sb]), ((itB / p.nB) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) { ok = false; break; }
-                            const uint32_t bfull = smem_u32(&bars->b_full[sb]);
-                            mbar_arrive_expect_tx(bfull, (uint32_t)b_stage);
-                            uint8_t* dstB = sB + (size_t)sb * b_stage;
-                            tma_load_3d(smem_u32(dstB), &tmap_val1, bfull, kb * KB, vt * p.vpad, i);
-                            if (p.n2 > 0) tma_load_3d(smem_u32(dstB + (size_t)p.n1 * KB), &tmap_val2, bfull, kb * KB, vt * p.vpad + p.n1, i);
+                            // this CTA's rows of the validation operand of each MMA half
+                            tma_load_3d_pair(smem_u32(st + A_STAGE), &tmap_val1, full, kb * KB, vt * p.vpad + (int)rank * (p.n1 / 2), i);
+                            if (p.n2 > 0)
+                                tma_load_3d_pair(smem_u32(st + A_STAGE + bh1), &tmap_val2, full, kb * KB, vt * p.vpad + p.n1 + (int)rank * (p.n2 / 2), i);
                         }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------- MMA issuer -------------------------------
-        if (lane == 0) {
-            uint32_t itA = 0, itB = 0, n_acc = 0;
+        // ------------------------------- MMA issuer (leader CTA) -------------------------------
+        if (lane == 0 && rank == 0) {
+            uint32_t it = 0, n_acc = 0;
             bool ok = true;
-            for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x)
+            for (int64_t tile = pair; tile < num_tiles && ok; tile += num_pairs)
                 for (int vt = 0; vt < num_vt && ok; ++vt)
                     for (int i = 0; i < p.C && ok; ++i, ++n_acc) {
-                        if (!mbar_wait(smem_u32(&bars->d_empty), (n_acc & 1u) ^ 1u, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
-                        tc_fence_after();
-                        for (int kb = 0; kb < nkb; ++kb, ++itA, ++itB) {
-                            const int sa = itA % p.nA, sb = itB % p.nB;
-                            if (!mbar_wait(smem_u32(&bars->a_full[sa]), (itA / p.nA) & 1u, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
-                            if (!mbar_wait(smem_u32(&bars->b_full[sb]), (itB / p.nB) & 1u, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
+                        if (!mbar_wait_cluster(smem_u32(&bars->d_empty), (n_acc & 1u) ^ 1u, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
+                        for (int kb = 0; kb < nkb; ++kb, ++it) {
+                            const int s = it % p.nS;
+                            if (!mbar_wait_cluster(smem_u32(&bars->full[s]), (it / p.nS) & 1u, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
                             tc_fence_after();
-                            const uint64_t adesc = make_smem_desc_sw128(smem_u32(sA + (size_t)sa * A_STAGE));
-                            const uint64_t bdesc1 = make_smem_desc_sw128(smem_u32(sB + (size_t)sb * b_stage));
-                            const uint64_t bdesc2 = make_smem_desc_sw128(smem_u32(sB + (size_t)sb * b_stage + (size_t)p.n1 * KB));
+                            const uint32_t st = smem_u32(sS + (size_t)s * stage_bytes);
+                            const uint64_t adesc = make_smem_desc_sw128(st);
+                            const uint64_t bdesc1 = make_smem_desc_sw128(st + A_STAGE);
+                            const uint64_t bdesc2 = make_smem_desc_sw128(st + A_STAGE + bh1);
 #pragma unroll
                             for (int k = 0; k < KB / 32; ++k) {
                                 const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
-                                mma_i8_ss(tmem_base, adesc + (uint64_t)(k * 2), bdesc1 + (uint64_t)(k * 2), idesc1, acc);
-                                if (p.n2 > 0) mma_i8_ss(tmem_base + p.n1, adesc + (uint64_t)(k * 2), bdesc2 + (uint64_t)(k * 2), idesc2, acc);
+                                mma_i8_ss_pair(tmem_base, adesc + (uint64_t)(k * 2), bdesc1 + (uint64_t)(k * 2), idesc1, acc);
+                                if (p.n2 > 0) mma_i8_ss_pair(tmem_base + p.n1, adesc + (uint64_t)(k * 2), bdesc2 + (uint64_t)(k * 2), idesc2, acc);
                             }
-                            mma_commit(smem_u32(&bars->a_empty[sa]));
-                            mma_commit(smem_u32(&bars->b_empty[sb]));
+                            mma_commit_pair(smem_u32(&bars->empty[s]));
                         }
-                        if (ok) mma_commit(smem_u32(&bars->d_full));
+                        if (ok) mma_commit_pair(smem_u32(&bars->d_full));
                     }
         }
     } else if (warp < 6) {
         // ------------------------------- unpack warps (4- and 2-bit train codes) -------------------------------
         if (BITS != 8) {
-            const int row = (warp - 2) * 32 + lane;               // row of the 128-row tile
+            const int row = (warp - 2) * 32 + lane;               // row of this CTA's 128-row half tile
             uint32_t it = 0;
             bool ok = true;
-            const int64_t my_tiles = (num_tiles > blockIdx.x) ? (num_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+            const int64_t my_tiles = (num_tiles > pair) ? (num_tiles - pair + num_pairs - 1) / num_pairs : 0;
             const int64_t total = my_tiles * num_vt * p.C * nkb;
             for (int64_t q = 0; q < total && ok; ++q, ++it) {
-                const int sp = it % p.nP, sa = it % p.nA;
+                const int sp = it % p.nP, s = it % p.nS;
                 ok = mbar_wait(smem_u32(&bars->p_full[sp]), (it / p.nP) & 1u, abort_flag, p.timeout_word, TO_UNPACK);
-                ok = ok && mbar_wait(smem_u32(&bars->a_empty[sa]), ((it / p.nA) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_UNPACK);
+                ok = ok && mbar_wait_cluster(smem_u32(&bars->empty[s]), ((it / p.nS) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_UNPACK);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 const uint4* src = reinterpret_cast<const uint4*>(sP + (size_t)sp * P_STAGE + (size_t)row * (16 * BITS));
-                uint8_t* dst_row = sA + (size_t)sa * A_STAGE + (size_t)row * KB;
+                uint8_t* dst_row = sS + (size_t)s * stage_bytes + (size_t)row * KB;
                 uint32_t out[32];
 #pragma unroll
                 for (int c = 0; c < (16 * BITS) / 16; ++c) {
@@ -221,8 +226,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                     *reinterpret_cast<uint4*>(dst_row + ((c ^ (row & 7)) << 4)) =
                         make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
                 fence_proxy_async_smem();                    // make the stores visible to the tensor core's reads
-                mbar_arrive(smem_u32(&bars->a_full[sa]));
-                mbar_arrive(smem_u32(&bars->p_empty[sp]));
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive_cluster(map_to_cta(smem_u32(&bars->full[s]), 0));
+                    mbar_arrive(smem_u32(&bars->p_empty[sp]));
+                }
             }
         }
     } else {
@@ -232,8 +240,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
         const int et = threadIdx.x - 6 * 32;                 // 0..127 among the epilogue threads
         uint32_t n_acc = 0;
         bool ok = true;
-        for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-            const int64_t t = tile * TM + tl;
+        for (int64_t tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+            const int64_t t = tile * 2 * TM + rank * TM + tl;
             float A[TMAX];
 #pragma unroll
             for (int j = 0; j < TMAX; ++j) A[j] = 0.0f;
@@ -247,7 +255,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         for (int v = et; v < p.vpad; v += 128) bars->mv[v] = (v < vcount) ? p.val_mult[(int64_t)i * p.V + v0 + v] : 0.0f;
                         asm volatile("bar.sync 1, 128;" ::: "memory");
                     }
-                    ok = mbar_wait(smem_u32(&bars->d_full), n_acc & 1u, abort_flag, p.timeout_word, TO_EPILOGUE);
+                    ok = mbar_wait_cluster(smem_u32(&bars->d_full), n_acc & 1u, abort_flag, p.timeout_word, TO_EPILOGUE);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     tc_fence_after();
@@ -264,7 +272,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         tmem_wait_ld();
                         if (c0 + 32 >= p.vpad) {              // accumulator fully read: release it
                             tc_fence_before();
-                            mbar_arrive(smem_u32(&bars->d_empty));
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->d_empty), 0));
                         }
                         if (p.dots != nullptr) {
                             if (t < p.N) {
@@ -324,9 +333,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
 
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();                 // neither CTA frees tensor memory or exits while its peer may still touch it
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 512);
+        tmem_dealloc_pair(tmem_base, 512);
     }
 }
 
@@ -369,22 +379,16 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     p.n2 = p.vpad - p.n1;
     const int64_t row_bytes = (int64_t)a.d * a.bits / 8;
 
-    // shared-memory plan
+    // shared-memory plan: as many operand stages as fit (each: 16 KiB of train rows + this CTA's validation rows)
     const size_t budget = 227 * 1024 - 1024 - sizeof(ScoreBars) - 64;
-    const size_t b_stage = (size_t)p.vpad * KB;
+    const size_t stage = (size_t)A_STAGE + (size_t)(p.vpad / 2) * KB;
     const size_t p_stage = a.bits == 8 ? 0 : (size_t)TM * 16 * a.bits;
-    int nA = 2, nB = 2, nP = a.bits == 8 ? 0 : 2;
-    auto used = [&]() { return (size_t)nA * A_STAGE + (size_t)nB * b_stage + (size_t)nP * p_stage; };
-    bool grew = true;
-    while (grew) {        // grow the deepest-latency pipelines round-robin while they fit
-        grew = false;
-        if (nB < MAX_STAGES && used() + b_stage <= budget) { ++nB; grew = true; }
-        if (a.bits == 8 && nA < nB && used() + A_STAGE <= budget) { ++nA; grew = true; }
-        if (a.bits != 8 && nP < MAX_STAGES && nP < nB && used() + p_stage <= budget) { ++nP; grew = true; }
-    }
-    if (a.bits != 8 && used() + A_STAGE <= budget && nA < 3) ++nA;
-    p.nA = nA; p.nB = nB; p.nP = nP > 0 ? nP : 1;
-    const size_t smem = 1024 + used() + sizeof(ScoreBars);
+    int nP = a.bits == 8 ? 0 : 3;
+    int nS = (int)((budget - (size_t)nP * p_stage) / stage);
+    if (nS > MAX_STAGES) nS = MAX_STAGES;
+    QLESS_REQUIRE(nS >= 2, QLESS_ERR_UNSUPPORTED, "internal: not enough shared memory for two pipeline stages");
+    p.nS = nS; p.nP = nP > 0 ? nP : 1;
+    const size_t smem = 1024 + (size_t)nS * stage + (size_t)nP * p_stage + sizeof(ScoreBars);
 
     p.train_mult = a.train_mult; p.val_mult = a.val_mult; p.eta_over_cnt = a.eta_over_cnt; p.task_off = a.task_off;
     p.scores = a.scores; p.per_task = a.per_task; p.dots = a.dots; p.timeout_word = timeout_word;
@@ -404,18 +408,18 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     qless_status s;
     const int64_t tstride = a.C > 1 ? a.train_stride : (int64_t)a.N * row_bytes;
     s = make_tmap_3d_u8(&tm_train, a.train, (uint64_t)row_bytes, (uint64_t)a.N, (uint64_t)a.C, (uint64_t)row_bytes,
-                        (uint64_t)tstride, a.bits == 8 ? 128 : 16 * a.bits, TM, a.bits == 8);
+                        (uint64_t)tstride, a.bits == 8 ? 128 : 16 * a.bits, TM, a.bits == 8);     // this CTA's 128 rows
     if (s != QLESS_OK) return s;
     const int64_t vstride = a.C > 1 ? val_stride : (int64_t)a.V * val_row;
-    s = make_tmap_3d_u8(&tm_v1, val_src, (uint64_t)val_row, (uint64_t)a.V, (uint64_t)a.C, (uint64_t)val_row, (uint64_t)vstride, 128, p.n1, true);
+    s = make_tmap_3d_u8(&tm_v1, val_src, (uint64_t)val_row, (uint64_t)a.V, (uint64_t)a.C, (uint64_t)val_row, (uint64_t)vstride, 128, p.n1 / 2, true);
     if (s != QLESS_OK) return s;
     s = make_tmap_3d_u8(&tm_v2, val_src, (uint64_t)val_row, (uint64_t)a.V, (uint64_t)a.C, (uint64_t)val_row, (uint64_t)vstride, 128,
-                        p.n2 > 0 ? p.n2 : 16, true);
+                        p.n2 > 0 ? p.n2 / 2 : 8, true);
     if (s != QLESS_OK) return s;
 
-    const int64_t tiles = (a.N + TM - 1) / TM;
-    int64_t grid = sm_count();
-    if (grid > tiles) grid = tiles;
+    const int64_t tiles = (a.N + 2 * TM - 1) / (2 * TM);
+    int64_t grid = (sm_count() / 2) * 2;            // CTA pairs
+    if (grid > 2 * tiles) grid = 2 * tiles;
 #define QLESS_LAUNCH_SCORE_TC(B)                                                                                    \
     QLESS_CUDA_TRY(cudaFuncSetAttribute(score_tc_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
     score_tc_kernel<B><<<(unsigned)grid, NTHREADS, smem, st>>>(tm_train, tm_v1, tm_v2, p);
