@@ -22,8 +22,8 @@
 // the single MMA-issuing thread runs at the tensor pipe's own pace, so every other instruction it executes
 // is lost tensor time.
 //
-// Warp roles (320 threads per CTA): warp 0 TMA producer, warp 1 MMA issuer (leader only; + TMEM
-// allocation), warps 2-5 unpack (idle for 8-bit), warps 6-9 epilogue. All waits are bounded.
+// Warp roles (448 threads per CTA): warp 0 TMA producer, warp 1 MMA issuer (leader only; + TMEM
+// allocation), warps 2-5 and 10-13 unpack (idle for 8-bit), warps 6-9 epilogue. All waits are bounded.
 #include "qless_kernels.h"
 #include "tc_common.cuh"
 
@@ -37,7 +37,7 @@ constexpr int TM = 128;                    // train rows per tile
 constexpr int KB = 128;                    // codes (= unpacked bytes) per row per K block
 constexpr int A_STAGE = TM * KB;           // 16 KiB
 constexpr int MAX_STAGES = 8;
-constexpr int NTHREADS = 320;
+constexpr int NTHREADS = 448;
 constexpr int TMAX = 8;                    // tasks held in registers by the epilogue
 
 struct ScoreTcParams {
@@ -133,25 +133,43 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
             uint32_t it = 0;
             bool ok = true;
             const uint32_t tx_total = 2u * (uint32_t)((BITS == 8 ? A_STAGE : 0) + bh1 + bh2);   // both CTAs
+            const int64_t my_tiles = (num_tiles > pair) ? (num_tiles - pair + num_pairs - 1) / num_pairs : 0;
+            const int64_t total = my_tiles * num_vt * p.C * nkb;
+            // Packed train codes run ahead of the operand stages in their own ring: the load for iteration q is
+            // issued as soon as ring slot q % nP is free, not when operand stage q % nS is.
+            int64_t pq = 0;                     // next packed load to issue
+            // blocking = false: issue only if the ring slot is already free (returns false otherwise)
+            auto issue_packed = [&](int64_t q, bool blocking) -> bool {
+                const int sp = (int)(q % p.nP);
+                const uint32_t par = (uint32_t)((q / p.nP) & 1) ^ 1u;
+                if (blocking) { if (!mbar_wait(smem_u32(&bars->p_empty[sp]), par, abort_flag, p.timeout_word, TO_PRODUCER)) return false; }
+                else if (!mbar_try_wait(smem_u32(&bars->p_empty[sp]), par)) return false;
+                const int kb = (int)(q % nkb);
+                const int i = (int)((q / nkb) % p.C);
+                const int64_t tile = pair + (q / ((int64_t)nkb * p.C * num_vt)) * num_pairs;
+                const uint32_t pfull = smem_u32(&bars->p_full[sp]);
+                mbar_arrive_expect_tx(pfull, P_STAGE);
+                tma_load_3d(smem_u32(sP + (size_t)sp * P_STAGE), &tmap_train, pfull, kb * 16 * BITS, (int32_t)(tile * 2 * TM + rank * TM), i);
+                return true;
+            };
+
             for (int64_t tile = pair; tile < num_tiles && ok; tile += num_pairs) {
                 const int32_t row0 = (int32_t)(tile * 2 * TM + rank * TM);
                 for (int vt = 0; vt < num_vt && ok; ++vt)
                     for (int i = 0; i < p.C && ok; ++i)
                         for (int kb = 0; kb < nkb; ++kb, ++it) {
+                            if (BITS != 8) {
+                                // the packed codes of this iteration must be on their way; those of the next few if a slot is free
+                                while (pq <= (int64_t)it && ok) { ok = issue_packed(pq, true); ++pq; }
+                                if (!ok) break;
+                                while (pq < total && pq < (int64_t)it + p.nP && issue_packed(pq, false)) ++pq;
+                            }
                             const int s = it % p.nS;
                             if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), ((it / p.nS) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) { ok = false; break; }
                             const uint32_t full = map_to_cta(smem_u32(&bars->full[s]), 0);
                             if (rank == 0) mbar_arrive_expect_tx(smem_u32(&bars->full[s]), tx_total);
                             uint8_t* st = sS + (size_t)s * stage_bytes;
-                            if (BITS == 8) {
-                                tma_load_3d_pair(smem_u32(st), &tmap_train, full, kb * KB, row0, i);
-                            } else {
-                                const int sp = it % p.nP;
-                                if (!mbar_wait(smem_u32(&bars->p_empty[sp]), ((it / p.nP) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) { ok = false; break; }
-                                const uint32_t pfull = smem_u32(&bars->p_full[sp]);
-                                mbar_arrive_expect_tx(pfull, P_STAGE);
-                                tma_load_3d(smem_u32(sP + (size_t)sp * P_STAGE), &tmap_train, pfull, kb * 16 * BITS, row0, i);
-                            }
+                            if (BITS == 8) tma_load_3d_pair(smem_u32(st), &tmap_train, full, kb * KB, row0, i);
                             // this CTA's rows of the validation operand of each MMA half
                             tma_load_3d_pair(smem_u32(st + A_STAGE), &tmap_val1, full, kb * KB, vt * p.vpad + (int)rank * (p.n1 / 2), i);
                             if (p.n2 > 0)
@@ -187,15 +205,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         if (ok) mma_commit_pair(smem_u32(&bars->d_full));
                     }
         }
-    } else if (warp < 6) {
+    } else if (warp < 6 || warp >= 10) {
         // ------------------------------- unpack warps (4- and 2-bit train codes) -------------------------------
+        // two groups of four warps (2-5 and 10-13) take alternate K blocks, so that the barrier round trips of
+        // one block overlap the unpacking of the next
         if (BITS != 8) {
-            const int row = (warp - 2) * 32 + lane;               // row of this CTA's 128-row half tile
+            const int row = ((warp - 2) & 3) * 32 + lane;         // row of this CTA's 128-row half tile
+            const uint32_t grp = (warp >= 10) ? 1u : 0u;
             uint32_t it = 0;
             bool ok = true;
             const int64_t my_tiles = (num_tiles > pair) ? (num_tiles - pair + num_pairs - 1) / num_pairs : 0;
             const int64_t total = my_tiles * num_vt * p.C * nkb;
             for (int64_t q = 0; q < total && ok; ++q, ++it) {
+                if ((it & 1u) != grp) continue;
                 const int sp = it % p.nP, s = it % p.nS;
                 ok = mbar_wait(smem_u32(&bars->p_full[sp]), (it / p.nP) & 1u, abort_flag, p.timeout_word, TO_UNPACK);
                 ok = ok && mbar_wait_cluster(smem_u32(&bars->empty[s]), ((it / p.nS) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_UNPACK);
@@ -383,7 +405,7 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     const size_t budget = 227 * 1024 - 1024 - sizeof(ScoreBars) - 64;
     const size_t stage = (size_t)A_STAGE + (size_t)(p.vpad / 2) * KB;
     const size_t p_stage = a.bits == 8 ? 0 : (size_t)TM * 16 * a.bits;
-    int nP = a.bits == 8 ? 0 : 3;
+    int nP = a.bits == 8 ? 0 : 4;
     int nS = (int)((budget - (size_t)nP * p_stage) / stage);
     if (nS > MAX_STAGES) nS = MAX_STAGES;
     QLESS_REQUIRE(nS >= 2, QLESS_ERR_UNSUPPORTED, "internal: not enough shared memory for two pipeline stages");
