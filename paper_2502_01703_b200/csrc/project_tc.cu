@@ -187,7 +187,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->a_full[sa]), 0));
+                if (lane == 0) mbar_arrive_leader_tmem(smem_u32(&bars->a_full[sa]), rank);
             }
         }
     } else {
@@ -214,7 +214,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 if (c0 + 32 == BN) {          // accumulator fully read: hand it back before the stores
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->d_empty), 0));
+                    if (lane == 0) mbar_arrive_leader_tmem(smem_u32(&bars->d_empty), rank);
                 }
 #pragma unroll
                 for (int k = 0; k < 32; ++k)

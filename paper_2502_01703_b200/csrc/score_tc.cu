@@ -11,11 +11,13 @@
 // The N x V x C similarity tensor never exists in memory.
 //
 // 8-bit train codes go from global memory to the MMA operand buffer by TMA. 4- and 2-bit train codes
-// arrive packed (TMA, no swizzle) in a staging buffer; four unpack warps sign-extend them to int8 and
-// write the swizzled operand rows themselves (generic-proxy stores + fence.proxy.async). Validation codes
-// are unpacked once per call into a workspace (they are a few MB and stay in L2). Inside a 128-code block
-// the unpackers place the codes in a fixed permutation, the same for both operands, which an inner
-// product does not see.
+// arrive packed (TMA, no swizzle) in a staging ring; unpack warps (thread = train row = TMEM lane)
+// sign-extend them to int8 and store them straight into tensor memory, from where the MMA takes its A
+// operand: no shared-memory write, no swizzle, no proxy fence. The accumulator leaves 64 of the 512 TMEM
+// columns free, enough for two 128-code blocks of A, so at these widths a validation tile holds at most 448
+// vectors. Validation codes are unpacked once per call into a workspace (they are a few MB and stay in L2).
+// Inside a 128-code block the unpackers place the codes in a fixed permutation, the same for both
+// operands, which an inner product does not see.
 //
 // One barrier per pipeline stage on the leader CTA collects everything the MMAs of that stage need (TMA
 // bytes of both CTAs, and the unpack warps' arrivals); one tcgen05.commit releases the stage in both CTAs:
@@ -39,6 +41,7 @@ constexpr int A_STAGE = TM * KB;           // 16 KiB
 constexpr int MAX_STAGES = 8;
 constexpr int NTHREADS = 448;
 constexpr int TMAX = 8;                    // tasks held in registers by the epilogue
+constexpr int A_TMEM_COL = 448;            // sub-byte widths: two 32-column slots of unpacked train codes
 
 struct ScoreTcParams {
     int64_t N;
@@ -85,7 +88,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);    // 1 KiB aligned, still a shared pointer
     const int bh1 = (p.n1 / 2) * KB, bh2 = (p.n2 / 2) * KB;      // bytes of this CTA's rows of the two MMA halves
-    const int stage_bytes = A_STAGE + bh1 + bh2;                  // multiple of 1024
+    constexpr int A_SMEM = (BITS == 8) ? A_STAGE : 0;              // sub-byte widths keep A in tensor memory
+    const int stage_bytes = A_SMEM + bh1 + bh2;                   // multiple of 1024
     constexpr int P_STAGE = (BITS == 8) ? 0 : TM * 16 * BITS;     // packed staging bytes per stage
     uint8_t* sS = smem;                                           // stage s: [A 16 KiB][B half 1][B half 2]
     uint8_t* sP = sS + (size_t)p.nS * stage_bytes;
@@ -171,9 +175,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                             uint8_t* st = sS + (size_t)s * stage_bytes;
                             if (BITS == 8) tma_load_3d_pair(smem_u32(st), &tmap_train, full, kb * KB, row0, i);
                             // this CTA's rows of the validation operand of each MMA half
-                            tma_load_3d_pair(smem_u32(st + A_STAGE), &tmap_val1, full, kb * KB, vt * p.vpad + (int)rank * (p.n1 / 2), i);
+                            tma_load_3d_pair(smem_u32(st + A_SMEM), &tmap_val1, full, kb * KB, vt * p.vpad + (int)rank * (p.n1 / 2), i);
                             if (p.n2 > 0)
-                                tma_load_3d_pair(smem_u32(st + A_STAGE + bh1), &tmap_val2, full, kb * KB, vt * p.vpad + p.n1 + (int)rank * (p.n2 / 2), i);
+                                tma_load_3d_pair(smem_u32(st + A_SMEM + bh1), &tmap_val2, full, kb * KB, vt * p.vpad + p.n1 + (int)rank * (p.n2 / 2), i);
                         }
             }
         }
@@ -192,13 +196,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                             tc_fence_after();
                             const uint32_t st = smem_u32(sS + (size_t)s * stage_bytes);
                             const uint64_t adesc = make_smem_desc_sw128(st);
-                            const uint64_t bdesc1 = make_smem_desc_sw128(st + A_STAGE);
-                            const uint64_t bdesc2 = make_smem_desc_sw128(st + A_STAGE + bh1);
+                            const uint64_t bdesc1 = make_smem_desc_sw128(st + A_SMEM);
+                            const uint64_t bdesc2 = make_smem_desc_sw128(st + A_SMEM + bh1);
+                            const uint32_t a_tmem = tmem_base + A_TMEM_COL + (it & 1u) * 32;
 #pragma unroll
                             for (int k = 0; k < KB / 32; ++k) {
                                 const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
-                                mma_i8_ss_pair(tmem_base, adesc + (uint64_t)(k * 2), bdesc1 + (uint64_t)(k * 2), idesc1, acc);
-                                if (p.n2 > 0) mma_i8_ss_pair(tmem_base + p.n1, adesc + (uint64_t)(k * 2), bdesc2 + (uint64_t)(k * 2), idesc2, acc);
+                                if (BITS == 8) {
+                                    mma_i8_ss_pair(tmem_base, adesc + (uint64_t)(k * 2), bdesc1 + (uint64_t)(k * 2), idesc1, acc);
+                                    if (p.n2 > 0) mma_i8_ss_pair(tmem_base + p.n1, adesc + (uint64_t)(k * 2), bdesc2 + (uint64_t)(k * 2), idesc2, acc);
+                                } else {
+                                    mma_i8_ts_pair(tmem_base, a_tmem + k * 8, bdesc1 + (uint64_t)(k * 2), idesc1, acc);
+                                    if (p.n2 > 0) mma_i8_ts_pair(tmem_base + p.n1, a_tmem + k * 8, bdesc2 + (uint64_t)(k * 2), idesc2, acc);
+                                }
                             }
                             mma_commit_pair(smem_u32(&bars->empty[s]));
                         }
@@ -210,7 +220,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
         // two groups of four warps (2-5 and 10-13) take alternate K blocks, so that the barrier round trips of
         // one block overlap the unpacking of the next
         if (BITS != 8) {
-            const int row = ((warp - 2) & 3) * 32 + lane;         // row of this CTA's 128-row half tile
+            const int row = (warp & 3) * 32 + lane;               // row of this CTA's 128-row half tile = TMEM lane
             const uint32_t grp = (warp >= 10) ? 1u : 0u;
             uint32_t it = 0;
             bool ok = true;
@@ -220,11 +230,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 if ((it & 1u) != grp) continue;
                 const int sp = it % p.nP, s = it % p.nS;
                 ok = mbar_wait(smem_u32(&bars->p_full[sp]), (it / p.nP) & 1u, abort_flag, p.timeout_word, TO_UNPACK);
-                ok = ok && mbar_wait_cluster(smem_u32(&bars->empty[s]), ((it / p.nS) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_UNPACK);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
+                // unpack into registers first: this needs only the packed bytes, not the TMEM slot
                 const uint4* src = reinterpret_cast<const uint4*>(sP + (size_t)sp * P_STAGE + (size_t)row * (16 * BITS));
-                uint8_t* dst_row = sS + (size_t)s * stage_bytes + (size_t)row * KB;
                 uint32_t out[32];
 #pragma unroll
                 for (int c = 0; c < (16 * BITS) / 16; ++c) {
@@ -242,17 +251,28 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         }
                     }
                 }
-                // swizzled operand row: 16-byte chunk c of row r lives at chunk position c ^ (r & 7)
-#pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    *reinterpret_cast<uint4*>(dst_row + ((c ^ (row & 7)) << 4)) =
-                        make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
-                fence_proxy_async_smem();                    // make the stores visible to the tensor core's reads
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive_cluster(map_to_cta(smem_u32(&bars->full[s]), 0));
-                    mbar_arrive(smem_u32(&bars->p_empty[sp]));
+                if (lane == 0) mbar_arrive(smem_u32(&bars->p_empty[sp]));      // staging slot read: the producer may refill it
+                // TMEM slot it % 2 is free once the MMAs of K block it - 2 have completed, which is what releases
+                // operand stage (it - 2) % nS (nS > 2, so that barrier cannot run a whole phase ahead of us)
+                if (it >= 2)
+                    ok = mbar_wait_cluster(smem_u32(&bars->empty[(it - 2) % p.nS]), ((it - 2) / p.nS) & 1u, abort_flag, p.timeout_word, TO_UNPACK);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                // this thread's row of the A operand: TMEM lane = row, column c = codes 4c .. 4c+3 of the block
+                const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + A_TMEM_COL + (it & 1u) * 32;
+                {
+                    uint32_t lo16[16], hi16[16];
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) { lo16[c] = out[c]; hi16[c] = out[16 + c]; }
+                    tmem_st_x16(taddr, lo16);
+                    tmem_st_x16(taddr + 16, hi16);
                 }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_leader_tmem(smem_u32(&bars->full[s]), rank);
             }
         }
     } else {
@@ -295,7 +315,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         if (c0 + 32 >= p.vpad) {              // accumulator fully read: release it
                             tc_fence_before();
                             __syncwarp();
-                            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->d_empty), 0));
+                            if (lane == 0) mbar_arrive_leader_tmem(smem_u32(&bars->d_empty), rank);
                         }
                         if (p.dots != nullptr) {
                             if (t < p.N) {
@@ -396,19 +416,20 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     ScoreTcParams p;
     p.N = a.N; p.V = a.V; p.C = a.C; p.T = a.T; p.d = a.d; p.bits = a.bits;
     const int vpad_all = (a.V + 15) / 16 * 16;
-    p.vpad = vpad_all < 512 ? vpad_all : 512;
+    const int vcap = a.bits == 8 ? 512 : A_TMEM_COL;        // sub-byte widths keep 64 TMEM columns for the A operand
+    p.vpad = vpad_all < vcap ? vpad_all : vcap;
     p.n1 = p.vpad < 256 ? p.vpad : 256;
     p.n2 = p.vpad - p.n1;
     const int64_t row_bytes = (int64_t)a.d * a.bits / 8;
 
     // shared-memory plan: as many operand stages as fit (each: 16 KiB of train rows + this CTA's validation rows)
     const size_t budget = 227 * 1024 - 1024 - sizeof(ScoreBars) - 64;
-    const size_t stage = (size_t)A_STAGE + (size_t)(p.vpad / 2) * KB;
+    const size_t stage = (a.bits == 8 ? (size_t)A_STAGE : 0) + (size_t)(p.vpad / 2) * KB;
     const size_t p_stage = a.bits == 8 ? 0 : (size_t)TM * 16 * a.bits;
     int nP = a.bits == 8 ? 0 : 4;
     int nS = (int)((budget - (size_t)nP * p_stage) / stage);
     if (nS > MAX_STAGES) nS = MAX_STAGES;
-    QLESS_REQUIRE(nS >= 2, QLESS_ERR_UNSUPPORTED, "internal: not enough shared memory for two pipeline stages");
+    QLESS_REQUIRE(nS >= 3, QLESS_ERR_UNSUPPORTED, "internal: not enough shared memory for two pipeline stages");
     p.nS = nS; p.nP = nP > 0 ? nP : 1;
     const size_t smem = 1024 + (size_t)nS * stage + (size_t)nP * p_stage + sizeof(ScoreBars);
 

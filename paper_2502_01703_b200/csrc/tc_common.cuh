@@ -83,6 +83,19 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// Arrival that only has to order tensor-memory accesses (already ordered by tcgen05.wait / tcgen05.fence),
+// on the leader's barrier: a plain CTA-scope arrive in the leader, a relaxed cluster-scope one in the peer.
+// (A release at cluster scope costs about 1500 clocks; these arrivals sit on the critical path of a stage.)
+__device__ __forceinline__ void mbar_arrive_leader_tmem(uint32_t own_bar, uint32_t rank)
+{
+    if (rank == 0) {
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(own_bar) : "memory");
+    } else {
+        uint32_t r;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(r) : "r"(own_bar));
+        asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0], 1;" ::"r"(r) : "memory");
+    }
+}
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
@@ -96,11 +109,14 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
     return ok != 0;
 }
 // Bounded wait on an own barrier whose arrivals may come from the peer CTA.
+// backoff_ns > 0: sleep between polls, so that a warp in a long wait leaves the issue slots to the warps
+// that share its scheduler.
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                                  unsigned int* timeout_word, uint32_t code)
+                                                  unsigned int* timeout_word, uint32_t code, uint32_t backoff_ns = 0)
 {
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
         if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (backoff_ns) __nanosleep(backoff_ns);
         if ((it & 255u) == 255u && *abort_flag) return false;
     }
     *abort_flag = 1u;
@@ -154,6 +170,16 @@ __device__ __forceinline__ void mma_i8_ss_pair(uint32_t d_tmem, uint64_t a_desc,
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Pair MMA with the int8 A operand in tensor memory (lane = row, four codes per 32-bit column).
+__device__ __forceinline__ void mma_i8_ts_pair(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 // Arrive, once every MMA issued so far has completed, on the barrier at this offset in BOTH CTAs of the pair.
