@@ -49,6 +49,7 @@ struct ScoreTcParams {
     int32_t vpad;               // validation rows per tile, multiple of 16, <= 512
     int32_t n1, n2;             // MMA N of the two halves (n1 + n2 = vpad)
     int32_t nS, nP;             // pipeline depths: operand stages (A + B), packed staging
+    int32_t epi_groups;         // 1 or 2 groups of four epilogue warps (2: each takes half of the columns)
     const float* train_mult;    // [C][N]
     const float* val_mult;      // [C][V]
     const float* eta_over_cnt;  // [C][T]
@@ -65,6 +66,7 @@ struct __align__(8) ScoreBars {
     uint32_t tmem_base, abort_flag;
     int32_t task_off[65];
     __align__(16) float mv[512];
+    float comb[TM][6];          // per-task partial sums handed from the second epilogue group to the first
 };
 
 // 8 packed 4-bit codes -> two words of four int8 (low nibbles, high nibbles)
@@ -114,7 +116,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
             mbar_init(smem_u32(&bars->p_empty[s]), 4);
         }
         mbar_init(smem_u32(&bars->d_full), 1);
-        mbar_init(smem_u32(&bars->d_empty), 8);
+        mbar_init(smem_u32(&bars->d_empty), 8 * p.epi_groups);     // one arrival per epilogue warp of both CTAs
         bars->abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmap_train); prefetch_tmap(&tmap_val1); prefetch_tmap(&tmap_val2);
@@ -215,7 +217,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         if (ok) mma_commit_pair(smem_u32(&bars->d_full));
                     }
         }
-    } else if (warp < 6 || warp >= 10) {
+    } else if (BITS != 8 && (warp < 6 || warp >= 10)) {
         // ------------------------------- unpack warps (4- and 2-bit train codes) -------------------------------
         // two groups of four warps (2-5 and 10-13) take alternate K blocks, so that the barrier round trips of
         // one block overlap the unpacking of the next
@@ -275,11 +277,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 if (lane == 0) mbar_arrive_leader_tmem(smem_u32(&bars->full[s]), rank);
             }
         }
-    } else {
+    } else if (warp >= 6 && warp < 10 || (warp < 6 && p.epi_groups == 2)) {
         // ------------------------------- epilogue -------------------------------
+        // warps 6-9 (group 0) and, for 8-bit codes where they have nothing to unpack, warps 2-5 (group 1): with two
+        // groups each reads half of the accumulator's columns, which halves the time the tensor pipe waits for it
         const int q = warp & 3;
         const int tl = q * 32 + lane;                        // row of the tile = TMEM lane
-        const int et = threadIdx.x - 6 * 32;                 // 0..127 among the epilogue threads
+        const int eg = (warp >= 6) ? 0 : 1;
+        const int et = eg * 128 + tl;                        // index among the epilogue threads
+        const int nthr_e = 128 * p.epi_groups;
+        const int nch = (p.vpad + 31) / 32;                  // 32-column chunks of the accumulator
+        const int ch_lo = (p.epi_groups == 2 && eg == 1) ? (nch + 1) / 2 : 0;
+        const int ch_hi = (p.epi_groups == 2 && eg == 0) ? (nch + 1) / 2 : nch;
         uint32_t n_acc = 0;
         bool ok = true;
         for (int64_t tile = pair; tile < num_tiles && ok; tile += num_pairs) {
@@ -293,9 +302,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 for (int i = 0; i < p.C && ok; ++i, ++n_acc) {
                     if (p.dots == nullptr) {
                         // this checkpoint's validation multipliers -> shared memory (epilogue threads only)
-                        asm volatile("bar.sync 1, 128;" ::: "memory");
-                        for (int v = et; v < p.vpad; v += 128) bars->mv[v] = (v < vcount) ? p.val_mult[(int64_t)i * p.V + v0 + v] : 0.0f;
-                        asm volatile("bar.sync 1, 128;" ::: "memory");
+                        asm volatile("bar.sync 1, %0;" ::"r"(nthr_e) : "memory");
+                        for (int v = et; v < p.vpad; v += nthr_e) bars->mv[v] = (v < vcount) ? p.val_mult[(int64_t)i * p.V + v0 + v] : 0.0f;
+                        asm volatile("bar.sync 1, %0;" ::"r"(nthr_e) : "memory");
                     }
                     ok = mbar_wait_cluster(smem_u32(&bars->d_full), n_acc & 1u, abort_flag, p.timeout_word, TO_EPILOGUE);
                     ok = __all_sync(0xFFFFFFFFu, ok);
@@ -304,15 +313,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
                     const float mt = (p.dots == nullptr && t < p.N) ? p.train_mult[(int64_t)i * p.N + t] : 0.0f;
                     int j = 0;
-                    if (p.dots == nullptr) while (j < p.T - 1 && bars->task_off[j + 1] <= v0) ++j;
+                    if (p.dots == nullptr) while (j < p.T - 1 && bars->task_off[j + 1] <= v0 + ch_lo * 32) ++j;
                     int next_b = (p.dots == nullptr) ? bars->task_off[j + 1] - v0 : 0x7FFFFFFF;   // first column of task j+1
                     float task_sum = 0.0f;
 #pragma unroll 1
-                    for (int c0 = 0; c0 < p.vpad; c0 += 32) {
+                    for (int c0 = ch_lo * 32; c0 < ch_hi * 32; c0 += 32) {
                         uint32_t v[32];
                         tmem_ld_x32(taddr + c0, v);
                         tmem_wait_ld();
-                        if (c0 + 32 >= p.vpad) {              // accumulator fully read: release it
+                        if (c0 + 32 >= ch_hi * 32) {          // this warp's share of the accumulator is read: release it
                             tc_fence_before();
                             __syncwarp();
                             if (lane == 0) mbar_arrive_leader_tmem(smem_u32(&bars->d_empty), rank);
@@ -360,7 +369,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                     }
                 }
             }
-            if (ok && p.dots == nullptr && t < p.N) {
+            if (ok && p.dots == nullptr && p.epi_groups == 2) {      // add the second group's partial sums to the first's
+                if (eg == 1) {
+#pragma unroll
+                    for (int jj = 0; jj < 6; ++jj) bars->comb[tl][jj] = A[jj];
+                }
+                asm volatile("bar.sync 3, 256;" ::: "memory");
+                if (eg == 0) {
+#pragma unroll
+                    for (int jj = 0; jj < 6; ++jj) A[jj] += bars->comb[tl][jj];
+                }
+            }
+            if (ok && p.dots == nullptr && t < p.N && eg == 0) {
                 float best = A[0];
 #pragma unroll
                 for (int jj = 1; jj < TMAX; ++jj) if (jj < p.T) best = fmaxf(best, A[jj]);
@@ -431,6 +451,7 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     if (nS > MAX_STAGES) nS = MAX_STAGES;
     QLESS_REQUIRE(nS >= 3, QLESS_ERR_UNSUPPORTED, "internal: not enough shared memory for two pipeline stages");
     p.nS = nS; p.nP = nP > 0 ? nP : 1;
+    p.epi_groups = (a.bits == 8 && a.T <= 6) ? 2 : 1;
     const size_t smem = 1024 + (size_t)nS * stage + (size_t)nP * p_stage + sizeof(ScoreBars);
 
     p.train_mult = a.train_mult; p.val_mult = a.val_mult; p.eta_over_cnt = a.eta_over_cnt; p.task_off = a.task_off;
