@@ -157,6 +157,127 @@ def cpu_baseline():
                         f"(scaled x{d // n_coords}; the work is linear in d), {t3 - t0:.1f} s of CPU time, single thread"))
 
 
+def _time_ms(torch, fn, iters, warm=1):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def stage_measurements(torch, B, W, dev, peaks):
+    """The other kernels of the path at the sizes where their roofline is observable: quantise on 65 536 rows,
+    scoring on the 270 K x 448 x 4-checkpoint store per bit width and on the 2 M-row 1-bit store, selection on
+    2^28 scores. Each entry gives the CUDA-event time of the library call and the achieved fraction of the
+    relevant measured peak (HBM copy bandwidth, or the library's own tcgen05 int8 / XOR+POPC micro-benchmark)."""
+    out = {}
+    # measured peaks of units the driver did not measure
+    ms, ops = B.qless_microbench("i8_ss_pair", 20000, device=dev)
+    i8_peak = ops / ms / 1e9            # Tops/s
+    ms, ops = B.qless_microbench("popc", 20000, device=dev)
+    popc_peak = ops / ms / 1e9          # T word-ops/s
+    ms, ops = B.qless_microbench("bf16_ts_pair", 20000, device=dev)
+    out["microbench"] = dict(int8_tops=i8_peak, popc_xor_add_twordops=popc_peak, bf16_tcgen05_tflops=ops / ms / 1e9,
+                             note="back-to-back tcgen05.mma / XOR+POPC+IADD on all SMs, burst")
+    d = 8192
+    # ---- quantise ----
+    n = 65536
+    x = torch.randn((n, d), device=dev)
+    q = {}
+    for bits in (8, 4, 2, 1):
+        t = _time_ms(torch, lambda: B.qless_quantize(x, bits), 5)
+        byts = n * (4 * d + d * bits // 8 + 8)
+        q[str(bits)] = dict(ms=t, gbs=byts / t / 1e6, frac_of_hbm=byts / t / 1e6 / peaks["hbm_gbs"])
+    out["quantize_65536x8192"] = q
+    del x
+    # ---- scoring, config 3 ----
+    cfg = W.CONFIGS["c3_score_sweep"]
+    N, C, V = cfg["N"], cfg["C"], sum(cfg["tasks"])
+    off = W.task_offsets(cfg["tasks"]).tolist()
+    store = {b: dict(tc=torch.empty((C, N, d * b // 8), dtype=torch.uint8, device=dev),
+                     vc=torch.empty((C, V, d * b // 8), dtype=torch.uint8, device=dev),
+                     ts=torch.empty((C, N), device=dev), vs=torch.empty((C, V), device=dev),
+                     tq=torch.empty((C, N), dtype=torch.int32, device=dev), vq=torch.empty((C, V), dtype=torch.int32, device=dev))
+             for b in cfg["bits"]}
+    chunk = 16384
+    for r0 in range(0, N, chunk):
+        r1 = min(N, r0 + chunk)
+        xs = W.lowrank_gaussian_features(r1 - r0, d, C, seed=SEED + 7 + r0, device=dev)
+        for i in range(C):
+            for b in cfg["bits"]:
+                st = store[b]
+                st["tc"][i, r0:r1], st["ts"][i, r0:r1], st["tq"][i, r0:r1] = B.qless_quantize(xs[i], b)
+    xs = W.lowrank_gaussian_features(V, d, C, seed=SEED + 8, device=dev)
+    for i in range(C):
+        for b in cfg["bits"]:
+            st = store[b]
+            st["vc"][i], st["vs"][i], st["vq"][i] = B.qless_quantize(xs[i], b)
+    del xs
+    sc = torch.empty(N, device=dev)
+    res = {}
+    for b in cfg["bits"]:
+        st = store[b]
+        ws = torch.empty(B.qless_score_workspace(N, V, C, len(off) - 1, d, b), dtype=torch.uint8, device=dev)
+        t = _time_ms(torch, lambda: B.qless_score(st["tc"], st["vc"], st["ts"], st["vs"], cfg["lr"], off, d, b,
+                                                  train_sumsq=st["tq"], val_sumsq=st["vq"], scores=sc, workspace=ws), 5)
+        e = dict(ms=t, scores_per_s=N * V / (t * 1e-3), pair_dots_per_s=N * V * C / (t * 1e-3))
+        if b == 1:
+            wops = N * V * C * (d / 32)
+            e.update(bound="alu", achieved_twordops=wops / t / 1e9, frac_of_popc_peak=wops / t / 1e9 / popc_peak)
+        else:
+            iops = 2.0 * N * V * C * d
+            e.update(bound="tensor", achieved_tops=iops / t / 1e9, frac_of_int8_peak=iops / t / 1e9 / i8_peak)
+        res[str(b)] = e
+    out["score_c3_270000x448x4"] = res
+    idx = torch.empty(N, dtype=torch.int64, device=dev)
+    wsel = torch.empty(B.qless_select_topk_workspace(N), dtype=torch.uint8, device=dev)
+    out["select_c3_270000_top5pct"] = dict(ms=_time_ms(torch, lambda: B.qless_select_topk(sc, cfg["frac"], indices=idx, workspace=wsel), 20))
+    del store, sc
+    # ---- 1-bit scale-up, config 4 ----
+    cfg = W.CONFIGS["c4_onebit_scaleup"]
+    N = cfg["N"]
+    tc = torch.empty((C, N, d // 8), dtype=torch.uint8, device=dev)
+    ts = torch.empty((C, N), device=dev); tq = torch.empty((C, N), dtype=torch.int32, device=dev)
+    vc = torch.empty((C, V, d // 8), dtype=torch.uint8, device=dev)
+    vs = torch.empty((C, V), device=dev); vq = torch.empty((C, V), dtype=torch.int32, device=dev)
+    chunk = 32768
+    for r0 in range(0, N, chunk):
+        r1 = min(N, r0 + chunk)
+        xs = W.lowrank_gaussian_features(r1 - r0, d, C, seed=SEED + 9 + r0, device=dev)
+        for i in range(C):
+            tc[i, r0:r1], ts[i, r0:r1], tq[i, r0:r1] = B.qless_quantize(xs[i], 1)
+    xs = W.lowrank_gaussian_features(V, d, C, seed=SEED + 10, device=dev)
+    for i in range(C):
+        vc[i], vs[i], vq[i] = B.qless_quantize(xs[i], 1)
+    del xs
+    sc = torch.empty(N, device=dev)
+    ws = torch.empty(B.qless_score_workspace(N, V, C, len(off) - 1, d, 1), dtype=torch.uint8, device=dev)
+    t = _time_ms(torch, lambda: B.qless_score(tc, vc, ts, vs, cfg["lr"], off, d, 1, train_sumsq=tq, val_sumsq=vq,
+                                              scores=sc, workspace=ws), 2)
+    wops = N * V * C * (d / 32)
+    out["score_c4_2000000x448x4_1bit"] = dict(ms=t, scores_per_s=N * V / (t * 1e-3), bound="alu",
+                                              achieved_twordops=wops / t / 1e9, frac_of_popc_peak=wops / t / 1e9 / popc_peak)
+    idx = torch.empty(N, dtype=torch.int64, device=dev)
+    wsel = torch.empty(B.qless_select_topk_workspace(N), dtype=torch.uint8, device=dev)
+    out["select_c4_2000000_top1pct"] = dict(ms=_time_ms(torch, lambda: B.qless_select_topk(sc, cfg["frac"], indices=idx, workspace=wsel), 20))
+    del tc, sc, idx
+    # ---- selection at a size where HBM bandwidth is observable ----
+    N = 1 << 28
+    s = torch.randn(N, device=dev)
+    idx = torch.empty(N // 16, dtype=torch.int64, device=dev)
+    wsel = torch.empty(B.qless_select_topk_workspace(N), dtype=torch.uint8, device=dev)
+    t = _time_ms(torch, lambda: B.qless_select_topk(s, 0.05, indices=idx, workspace=wsel), 3)
+    out["select_2^28_top5pct"] = dict(ms=t, gbs_algorithmic=4.0 * N / t / 1e6, frac_of_hbm=4.0 * N / t / 1e6 / peaks["hbm_gbs"],
+                                      note="algorithmic bytes = 4N (every score read once)")
+    B.qless_check()
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -302,6 +423,10 @@ def run_ours(args):
                     clocks=clocks, gpu_launches=launches, roofline=roofline,
                     stages_ms_per_step={k: ms / args.steps for k, (ms, c) in prof.items()},
                     e2e=e2e)
+        if world == 1 and not args.no_stages:
+            del g, out
+            torch.cuda.empty_cache()
+            line["stages"] = stage_measurements(torch, B, W, dev, peaks)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline()
         print(json.dumps(line))
@@ -318,6 +443,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-stages", action="store_true", help="skip the per-kernel measurements at their own sizes")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
