@@ -140,7 +140,7 @@ def cpu_baseline():
     from paper_2502_01703_b200 import workloads as W
     cfg = W.CONFIGS[WORKLOAD]
     P, d, bits = cfg["P"], cfg["d"], cfg["bits"]
-    n_rows, n_coords = 4, 128
+    n_rows, n_coords = 4, 512
     g = W.student_t_gradients(n_rows, P, seed=SEED, dtype=torch.bfloat16).float().numpy()
     m, v = [t.numpy() for t in W.adam_moments(P, seed=SEED + 1)]
     coords = np.arange(n_coords, dtype=np.int32) * (d // n_coords)
