@@ -157,6 +157,22 @@ def cpu_baseline():
                         f"(scaled x{d // n_coords}; the work is linear in d), {t3 - t0:.1f} s of CPU time, single thread"))
 
 
+def max_over_ranks(ms_local, dist=None, device=None):
+    """Timing rule for N > 1: every rank measures its own replica on its own device; the job's time is the
+    slowest rank's (all-reduce MAX). Replicas share no data, so this is the only collective of the benchmark."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(ms_local)
+    import torch
+    t = torch.tensor([float(ms_local)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank_per_step, steps, world, ms_total):
+    """Weak scaling: every rank processes its own units; value = all ranks' units / slowest rank's time."""
+    return world * units_per_rank_per_step * steps / (ms_total * 1e-3)
+
+
 def _time_ms(torch, fn, iters, warm=1):
     for _ in range(warm):
         fn()
@@ -357,10 +373,7 @@ def run_ours(args):
     B.qless_profile_enable(False)
     launches = B.qless_kernel_launches() - launches0
     B.qless_check()
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dist if world > 1 else None, dev)
 
     # ---- end to end through the host-buffer entry point (rank-local; host->device copies timed) ----
     e2e = None
@@ -396,18 +409,15 @@ def run_ours(args):
         f1.record()
         barrier()
         ms_e2e = f0.elapsed_time(f1)
-        if world > 1:
-            t = torch.tensor([ms_e2e], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e = max_over_ranks(ms_e2e, dist if world > 1 else None, dev)
         h2d = n * P * 2 + n * rb + 2 * n * 4
         d2h = n * rb + 2 * n * 4 + k_sel * 8
-        e2e = dict(value=world * n * args.e2e_steps / (ms_e2e * 1e-3), unit="grads/s", h2d_bytes_per_step=h2d,
+        e2e = dict(value=whole_job_rate(n, args.e2e_steps, world, ms_e2e), unit="grads/s", h2d_bytes_per_step=h2d,
                    d2h_bytes_per_step=d2h, steps=args.e2e_steps, ms_per_step=ms_e2e / args.e2e_steps)
 
     if rank == 0:
         peaks = load_peaks()
-        value = world * n * args.steps / (ms_total * 1e-3)
+        value = whole_job_rate(n, args.steps, world, ms_total)
         proj_ms, proj_cnt = prof.get("project", (0.0, 0))
         flops = 2.0 * n * P * d
         achieved = flops / (proj_ms / max(proj_cnt, 1) * 1e-3) / 1e12 if proj_cnt else None
