@@ -24,7 +24,7 @@ EXPORTS = [
     "qless_score_dots_workspace", "qless_score_dots", "qless_select_topk_workspace", "qless_select_topk",
     "qless_project_quantize_host_workspace", "qless_project_quantize_host", "qless_profile_enable",
     "qless_profile_collect", "qless_kernel_launches", "qless_select_topk_static",
-    "qless_set_projection_path", "qless_set_score_path", "qless_microbench",
+    "qless_set_projection_path", "qless_set_score_path", "qless_set_select_path", "qless_microbench",
 ]
 SELECT_STATIC_MAX_N = 1 << 22
 
@@ -94,6 +94,8 @@ def lib():
         L.qless_microbench.argtypes = [i32, i32, C.POINTER(C.c_float), C.POINTER(C.c_double), vp, sz, vp]
         L.qless_set_score_path.restype = C.c_int
         L.qless_set_score_path.argtypes = [i32]
+        L.qless_set_select_path.restype = C.c_int
+        L.qless_set_select_path.argtypes = [i32]
         L.qless_set_projection_path.restype = C.c_int
         L.qless_set_projection_path.argtypes = [i32]
         L.qless_select_topk_static.restype = C.c_int
@@ -321,6 +323,11 @@ def qless_select_topk_static(scores, frac, indices, stream=None):
 def qless_set_projection_path(path):
     """0 = tensor-core projection kernel (default), 1 = CUDA-core cross-check kernel."""
     _check(lib().qless_set_projection_path(int(path)))
+
+
+def qless_set_select_path(path):
+    """0 = by size (default), 1 = multi-pass select at every N, 2 = sampled bracket forced too high."""
+    _check(lib().qless_set_select_path(int(path)))
 
 
 def qless_set_score_path(path):

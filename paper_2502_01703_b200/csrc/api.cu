@@ -171,6 +171,13 @@ qless_status qless_set_score_path(int32_t path)
     return QLESS_OK;
 }
 
+qless_status qless_set_select_path(int32_t path)
+{
+    QLESS_REQUIRE(path >= 0 && path <= 2, QLESS_ERR_INVALID_ARG, "path must be 0 (by size), 1 (multi-pass) or 2 (bracket forced too high)");
+    set_select_path(path);
+    return QLESS_OK;
+}
+
 uint64_t qless_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
 qless_status qless_profile_enable(int32_t on)

@@ -72,5 +72,7 @@ cudaError_t launch_multipliers(const uint8_t* codes, int64_t ckpt_stride, const 
 size_t select_workspace_bytes(int64_t N);
 cudaError_t launch_select_topk(const float* scores, int64_t N, int64_t k, int64_t* indices,
                                void* ws, cudaStream_t st);
+// 0: path by size; 1: multi-pass select at every N; 2: sampled bracket forced too high (exercises the fallback).
+void set_select_path(int mode);
 
 }  // namespace qless

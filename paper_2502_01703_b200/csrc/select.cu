@@ -29,14 +29,23 @@ struct SelectWs {
     int64_t* blk_off;     // [nblk][2]  exclusive prefix (gt, eq)
 };
 
+// A kernel whose gate is closed returns at once: the launches of the bracketed path and of its
+// fallback are both enqueued, and a flag written on the device decides which of the two does the work.
+struct Gate {
+    const uint32_t* flag;     // nullptr: always open
+    uint32_t want;
+    __device__ __forceinline__ bool closed() const { return flag != nullptr && *flag != want; }
+};
+
 __host__ __device__ inline int64_t sel_nblk(int64_t N) { return (N + SEL_CHUNK - 1) / SEL_CHUNK; }
 
 template <int PASS>
 __global__ void __launch_bounds__(SEL_T)
 select_hist_kernel(const float* __restrict__ scores, int64_t N, const SelectState* __restrict__ state,
-                   uint32_t* __restrict__ hist)
+                   uint32_t* __restrict__ hist, Gate gate)
 {
     __shared__ uint32_t s_h[2048];
+    if (gate.closed()) return;
     for (int i = threadIdx.x; i < 2048; i += SEL_T) s_h[i] = 0;
     __syncthreads();
     const uint32_t prefix = (PASS == 0) ? 0u : state->prefix;
@@ -68,8 +77,10 @@ select_hist_kernel(const float* __restrict__ scores, int64_t N, const SelectStat
 // down (block-wide prefix sum over the reversed histogram).
 template <int PASS>
 __global__ void __launch_bounds__(1024)
-select_scan_kernel(const uint32_t* __restrict__ hist, SelectState* __restrict__ state, int64_t k)
+select_scan_kernel(const uint32_t* __restrict__ hist, SelectState* __restrict__ state, int64_t k, Gate gate,
+                   uint32_t* __restrict__ short_flag)
 {
+    if (gate.closed()) return;
     constexpr int NB = (PASS == 2) ? 1024 : 2048;
     constexpr int SHIFT = (PASS == 2) ? 10 : 11;
     constexpr int PER = NB / 1024;
@@ -100,15 +111,19 @@ select_scan_kernel(const uint32_t* __restrict__ hist, SelectState* __restrict__ 
         }
         pre += c[u];
     }
+    // fewer than k_rem keys in the whole histogram: no bin was chosen; tell the caller
+    if (short_flag != nullptr && tid == 1023 && pre < k_rem) *short_flag = 1u;
 }
 
 __global__ void __launch_bounds__(SEL_T)
-select_count_kernel(const float* __restrict__ scores, int64_t N, const SelectState* __restrict__ state,
-                    int32_t* __restrict__ blk_cnt)
+select_count_kernel(const float* __restrict__ scores, int64_t N, int64_t nblk, const SelectState* __restrict__ state,
+                    int32_t* __restrict__ blk_cnt, Gate gate)
 {
     __shared__ int s_gt[SEL_T / 32], s_eq[SEL_T / 32];
+    if (gate.closed()) return;
     const uint32_t T = state->prefix;
-    const int64_t base = (int64_t)blockIdx.x * SEL_CHUNK + threadIdx.x * SEL_EPT;
+    for (int64_t blk = blockIdx.x; blk < nblk; blk += gridDim.x) {
+    const int64_t base = blk * SEL_CHUNK + threadIdx.x * SEL_EPT;
     int gt = 0, eq = 0;
 #pragma unroll
     for (int u = 0; u < SEL_EPT; ++u) {
@@ -125,50 +140,54 @@ select_count_kernel(const float* __restrict__ scores, int64_t N, const SelectSta
     if (threadIdx.x == 0) {
         int a = 0, b = 0;
         for (int w = 0; w < SEL_T / 32; ++w) { a += s_gt[w]; b += s_eq[w]; }
-        blk_cnt[2 * blockIdx.x] = a; blk_cnt[2 * blockIdx.x + 1] = b;
+        blk_cnt[2 * blk] = a; blk_cnt[2 * blk + 1] = b;
+    }
+    __syncthreads();
     }
 }
 
-// Exclusive prefix sums over blocks (one block of 1024 threads, sequential over tiles of 1024 blocks).
+// Exclusive prefix sums over blocks: one block of 1024 threads, thread t sums its run of consecutive
+// entries, the block scans the 1024 run totals, and each thread writes the prefixes of its run.
 __global__ void __launch_bounds__(1024)
-select_block_scan_kernel(const int32_t* __restrict__ blk_cnt, int64_t nblk, int64_t* __restrict__ blk_off)
+select_block_scan_kernel(const int32_t* __restrict__ blk_cnt, int64_t nblk, int64_t* __restrict__ blk_off, Gate gate)
 {
+    if (gate.closed()) return;
     __shared__ int64_t s_w[2][32];
-    __shared__ int64_t s_carry[2];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) { s_carry[0] = 0; s_carry[1] = 0; }
-    __syncthreads();
-    for (int64_t base = 0; base < nblk; base += 1024) {
-        const int64_t b = base + threadIdx.x;
-        int64_t v[2] = {0, 0};
-        if (b < nblk) { v[0] = blk_cnt[2 * b]; v[1] = blk_cnt[2 * b + 1]; }
-        int64_t inc[2] = {v[0], v[1]};
+    const int64_t per = (nblk + 1023) / 1024;
+    const int64_t b0 = threadIdx.x * per, b1 = (b0 + per < nblk) ? b0 + per : nblk;
+    const int2* cnt2 = reinterpret_cast<const int2*>(blk_cnt);
+    int64_t v0 = 0, v1 = 0;
+    for (int64_t b = b0; b < b1; ++b) { const int2 c = cnt2[b]; v0 += c.x; v1 += c.y; }
+    int64_t i0 = v0, i1 = v1;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int64_t a0 = __shfl_up_sync(0xFFFFFFFFu, inc[0], o), a1 = __shfl_up_sync(0xFFFFFFFFu, inc[1], o);
-            if (lane >= o) { inc[0] += a0; inc[1] += a1; }
-        }
-        if (lane == 31) { s_w[0][warp] = inc[0]; s_w[1][warp] = inc[1]; }
-        __syncthreads();
-        int64_t wo[2] = {0, 0};
-        for (int w = 0; w < warp; ++w) { wo[0] += s_w[0][w]; wo[1] += s_w[1][w]; }
-        const int64_t c0 = s_carry[0], c1 = s_carry[1];
-        if (b < nblk) { blk_off[2 * b] = c0 + wo[0] + inc[0] - v[0]; blk_off[2 * b + 1] = c1 + wo[1] + inc[1] - v[1]; }
-        __syncthreads();
-        if (threadIdx.x == 1023) { s_carry[0] = c0 + wo[0] + inc[0]; s_carry[1] = c1 + wo[1] + inc[1]; }
-        __syncthreads();
+    for (int o = 1; o < 32; o <<= 1) {
+        const int64_t a0 = __shfl_up_sync(0xFFFFFFFFu, i0, o), a1 = __shfl_up_sync(0xFFFFFFFFu, i1, o);
+        if (lane >= o) { i0 += a0; i1 += a1; }
+    }
+    if (lane == 31) { s_w[0][warp] = i0; s_w[1][warp] = i1; }
+    __syncthreads();
+    int64_t r0 = i0 - v0, r1 = i1 - v1;
+    for (int w = 0; w < warp; ++w) { r0 += s_w[0][w]; r1 += s_w[1][w]; }
+    longlong2* off2 = reinterpret_cast<longlong2*>(blk_off);
+    for (int64_t b = b0; b < b1; ++b) {
+        const int2 c = cnt2[b];
+        off2[b] = make_longlong2(r0, r1);
+        r0 += c.x; r1 += c.y;
     }
 }
 
 __global__ void __launch_bounds__(SEL_T)
-select_write_kernel(const float* __restrict__ scores, int64_t N, const SelectState* __restrict__ state,
-                    const int64_t* __restrict__ blk_off, int64_t* __restrict__ indices)
+select_write_kernel(const float* __restrict__ scores, int64_t N, int64_t nblk, const SelectState* __restrict__ state,
+                    const int64_t* __restrict__ blk_off, int64_t* __restrict__ indices, Gate gate)
 {
     __shared__ int s_gt[SEL_T / 32], s_eq[SEL_T / 32];
+    if (gate.closed()) return;
     const uint32_t T = state->prefix;
     const int64_t k_ties = state->k_rem;
-    const int64_t base = (int64_t)blockIdx.x * SEL_CHUNK + threadIdx.x * SEL_EPT;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int64_t blk = blockIdx.x; blk < nblk; blk += gridDim.x) {
+    const int64_t base = blk * SEL_CHUNK + threadIdx.x * SEL_EPT;
     uint32_t fgt = 0, feq = 0;
 #pragma unroll
     for (int u = 0; u < SEL_EPT; ++u) {
@@ -187,8 +206,8 @@ select_write_kernel(const float* __restrict__ scores, int64_t N, const SelectSta
     }
     if (lane == 31) { s_gt[warp] = igt; s_eq[warp] = ieq; }
     __syncthreads();
-    int64_t gt_before = blk_off[2 * blockIdx.x] + igt - gt;
-    int64_t eq_before = blk_off[2 * blockIdx.x + 1] + ieq - eq;
+    int64_t gt_before = blk_off[2 * blk] + igt - gt;
+    int64_t eq_before = blk_off[2 * blk + 1] + ieq - eq;
     for (int w = 0; w < warp; ++w) { gt_before += s_gt[w]; eq_before += s_eq[w]; }
 #pragma unroll
     for (int u = 0; u < SEL_EPT; ++u) {
@@ -198,6 +217,280 @@ select_write_kernel(const float* __restrict__ scores, int64_t N, const SelectSta
             indices[pos] = base + u;
         }
         gt_before += g; eq_before += e;
+    }
+    __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Large N: two reads of the scores instead of five. A stratified sample brackets the k-th largest
+// key from below (lo); one pass over the scores copies every key >= lo, in index order, into the
+// segment of its 4096-score chunk; the radix select and the ordered compaction then run on those
+// candidates alone (a few per cent of N, resident in L2). If fewer than k candidates turn up (the
+// bracket was too high: probability below 1e-8 for scores in any order, since the offset inside
+// each stratum is hashed) a flag opens the gates of the exact multi-pass path enqueued behind.
+// ------------------------------------------------------------------------------------------------
+
+constexpr int SG_T = 256;
+constexpr int SG_CH = 4096;                     // scores per chunk = capacity of its candidate segment
+constexpr int SG_SAMPLE = 16384;                // strata (one sampled score each)
+constexpr int64_t SG_MIN_N = (int64_t)1 << 22;  // above this the bracketed path is used
+
+struct BracketState {
+    uint32_t lo_key;              // candidates are the keys >= lo_key
+    uint32_t fallback;            // 1: fewer than k candidates, the exact path must run
+    unsigned long long n_cand;
+};
+
+struct BracketWs {
+    uint32_t* hist;               // [6][2048]: 0..2 candidates, 3..5 fallback
+    SelectState* state;           // 256-byte region; BracketState sits 64 bytes in
+    BracketState* bstate;
+    int64_t* blk_off;             // sized for the fallback's 2048-score blocks
+    int32_t* blk_cnt;
+    uint32_t* chunk_cnt;          // [nchunk]
+    uint16_t* seg_off;            // [nchunk][SG_CH] offset of the candidate inside its chunk
+    uint32_t* seg_key;            // [nchunk][SG_CH]
+};
+
+__host__ __device__ inline int64_t sg_nchunk(int64_t N) { return (N + SG_CH - 1) / SG_CH; }
+
+__device__ __forceinline__ uint32_t mix32(uint32_t x)
+{
+    x ^= x >> 16; x *= 0x7FEB352Du; x ^= x >> 15; x *= 0x846CA68Bu; x ^= x >> 16;
+    return x;
+}
+
+// One block: sample one score per stratum, find the r-th largest sampled key in shared memory
+// (three histogram rounds), r = expected rank of the k-th largest + 6 standard deviations + 8.
+__global__ void __launch_bounds__(1024)
+select_sample_kernel(const float* __restrict__ scores, int64_t N, int64_t k, BracketState* __restrict__ bs,
+                     int force_short)
+{
+    extern __shared__ uint32_t s_key[];          // [SG_SAMPLE]
+    __shared__ uint32_t s_h[2048];
+    __shared__ int s_w[32];
+    __shared__ uint32_t s_prefix;
+    __shared__ int s_rem;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t per = N / SG_SAMPLE;           // >= 256 for every N this path takes
+    for (int j = tid; j < SG_SAMPLE; j += 1024) {
+        const int64_t pos = (int64_t)j * per + (int64_t)(mix32(0x9E3779B9u * (uint32_t)j + 0x85EBCA6Bu) % (uint64_t)per);
+        s_key[j] = order_key(__float_as_uint(__ldg(scores + pos)));
+    }
+    const double p = (double)k / (double)N;
+    const double ks = ceil(p * (double)SG_SAMPLE);
+    const double rr = ks + ceil(6.0 * sqrt(ks * (1.0 - p))) + 8.0;
+    if (force_short) { if (tid == 0) bs->lo_key = 0xFF800000u; return; }      // key of +inf
+    if (rr >= (double)SG_SAMPLE) { if (tid == 0) bs->lo_key = 0u; return; }     // every score is a candidate
+    if (tid == 0) { s_prefix = 0u; s_rem = (int)rr; }
+    __syncthreads();
+#pragma unroll 1
+    for (int round = 0; round < 3; ++round) {
+        const int shift = (round == 0) ? 21 : (round == 1) ? 10 : 0;
+        const int bits = (round == 2) ? 10 : 11;
+        const uint32_t mask = (1u << bits) - 1u;
+        for (int i = tid; i < 2048; i += 1024) s_h[i] = 0;
+        __syncthreads();
+        const uint32_t prefix = s_prefix;
+        const int rem = s_rem;
+        for (int j = tid; j < SG_SAMPLE; j += 1024) {
+            const uint32_t key = s_key[j];
+            if (round == 0 || (key >> (shift + bits)) == prefix) atomicAdd(&s_h[(key >> shift) & mask], 1u);
+        }
+        __syncthreads();
+        // prefix sum from the top bin down: thread t owns bins 2047-2t and 2046-2t
+        const int c0 = (int)s_h[2047 - 2 * tid], c1 = (int)s_h[2046 - 2 * tid];
+        int inc = c0 + c1;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int a = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= o) inc += a;
+        }
+        if (lane == 31) s_w[warp] = inc;
+        __syncthreads();
+        int pre = inc - c0 - c1;
+        for (int w = 0; w < warp; ++w) pre += s_w[w];
+        if (pre < rem && rem <= pre + c0) { s_prefix = (prefix << bits) | (uint32_t)(2047 - 2 * tid); s_rem = rem - pre; }
+        else if (pre + c0 < rem && rem <= pre + c0 + c1) { s_prefix = (prefix << bits) | (uint32_t)(2046 - 2 * tid); s_rem = rem - pre - c0; }
+        __syncthreads();
+    }
+    if (tid == 0) bs->lo_key = s_prefix;
+}
+
+// The second (and last) read of the scores: candidates of each chunk, in index order, to the chunk's
+// segment; their top-11-bit histogram for the first round of the radix select.
+// The test runs on s = key ^ 0x80000000 read as a signed integer (two operations per score from the
+// raw bits; NaNs with the sign bit clear land above +inf and are cut off by the range check).
+// Warp w of the block owns scores [512 w, 512 w + 512) of the chunk, lane l the four at 128 j + 4 l of
+// each of its four loads j, so that positions follow from one packed warp scan (a byte per load).
+__global__ void __launch_bounds__(SG_T)
+select_gather_kernel(const float* __restrict__ scores, int64_t N, BracketState* __restrict__ bs,
+                     uint32_t* __restrict__ seg_key, uint16_t* __restrict__ seg_off,
+                     uint32_t* __restrict__ chunk_cnt, uint32_t* __restrict__ hist0)
+{
+    __shared__ uint32_t s_h[2048];
+    __shared__ uint32_t s_wtot[2][SG_T / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int i = tid; i < 2048; i += SG_T) s_h[i] = 0;
+    __syncthreads();
+    const uint32_t lo = bs->lo_key;
+    const uint32_t lo_s = lo ^ 0x80000000u;
+    const uint32_t range = (lo == 0u) ? 0xFFFFFFFFu : (0x7F800000u - lo_s);     // lo == 0: NaNs are candidates too
+    const int64_t nchunk = sg_nchunk(N);
+    unsigned long long mine = 0;
+    int par = 0;
+    for (int64_t c = blockIdx.x; c < nchunk; c += gridDim.x, par ^= 1) {
+        const int64_t base = c * SG_CH;
+        const int wofs = warp * 512 + lane * 4;
+        uint32_t sv[4][4];
+        uint32_t flags[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t i = base + wofs + j * 128;
+            uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+            uint32_t valid = 0;
+            if (i + 3 < N) { raw = __ldcs(reinterpret_cast<const uint4*>(scores + i)); valid = 0xFu; }
+            else {
+                if (i < N) { raw.x = __float_as_uint(scores[i]); valid |= 1u; }
+                if (i + 1 < N) { raw.y = __float_as_uint(scores[i + 1]); valid |= 2u; }
+                if (i + 2 < N) { raw.z = __float_as_uint(scores[i + 2]); valid |= 4u; }
+            }
+            const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+            uint32_t f = 0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                sv[j][u] = r[u] ^ ((uint32_t)((int32_t)r[u] >> 31) & 0x7FFFFFFFu);
+                if (sv[j][u] - lo_s <= range) f |= 1u << u;
+            }
+            flags[j] = f & valid;
+        }
+        const uint32_t cnt = (uint32_t)__popc(flags[0]) | ((uint32_t)__popc(flags[1]) << 8) |
+                             ((uint32_t)__popc(flags[2]) << 16) | ((uint32_t)__popc(flags[3]) << 24);
+        uint32_t inc = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t a = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= o) inc += a;
+        }
+        const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31);       // per-load totals of this warp (<= 128 each)
+        const uint32_t t0 = tot & 0xFFu, t1 = (tot >> 8) & 0xFFu, t2 = (tot >> 16) & 0xFFu, t3 = tot >> 24;
+        const uint32_t wtot = t0 + t1 + t2 + t3;
+        if (lane == 0) s_wtot[par][warp] = wtot;
+        __syncthreads();                // one barrier per chunk: the two buffers alternate
+        uint32_t wbase = 0, ctot = 0;
+#pragma unroll
+        for (int w = 0; w < SG_T / 32; ++w) {
+            const uint32_t t = s_wtot[par][w];
+            ctot += t;
+            if (w < warp) wbase += t;
+        }
+        if (flags[0] | flags[1] | flags[2] | flags[3]) {
+            const uint32_t excl = inc - cnt;
+            const uint32_t lbase[4] = {wbase, wbase + t0, wbase + t0 + t1, wbase + t0 + t1 + t2};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (flags[j]) {
+                    uint32_t pos = lbase[j] + ((excl >> (8 * j)) & 0xFFu);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if ((flags[j] >> u) & 1u) {
+                            // back to the key; a NaN (only reachable with lo == 0) has key 0
+                            const uint32_t sk = sv[j][u];
+                            const bool is_nan = (sk > 0x7F800000u && sk < 0x80000000u) || (sk >= 0x80000000u && sk < 0x807FFFFFu);
+                            const uint32_t key = is_nan ? 0u : (sk ^ 0x80000000u);
+                            seg_key[base + pos] = key;
+                            seg_off[base + pos] = (uint16_t)(wofs + j * 128 + u);
+                            atomicAdd(&s_h[key >> 21], 1u);
+                            ++pos;
+                        }
+                    }
+                }
+            }
+        }
+        if (tid == 0) { chunk_cnt[c] = ctot; mine += ctot; }
+    }
+    __syncthreads();
+    for (int i = tid; i < 2048; i += SG_T)
+        if (s_h[i]) atomicAdd(&hist0[i], s_h[i]);
+    if (tid == 0 && mine) atomicAdd(&bs->n_cand, mine);
+}
+
+// Radix-select rounds 2 and 3 on the candidates: one warp per chunk segment.
+template <int PASS>
+__global__ void __launch_bounds__(SG_T)
+cand_hist_kernel(const uint32_t* __restrict__ seg_key, const uint32_t* __restrict__ chunk_cnt, int64_t nchunk,
+                 const SelectState* __restrict__ state, uint32_t* __restrict__ hist, Gate gate)
+{
+    __shared__ uint32_t s_h[2048];
+    if (gate.closed()) return;
+    for (int i = threadIdx.x; i < 2048; i += SG_T) s_h[i] = 0;
+    __syncthreads();
+    const uint32_t prefix = state->prefix;
+    const int lane = threadIdx.x & 31;
+    const int64_t nwarp = (int64_t)gridDim.x * (SG_T / 32);
+    for (int64_t c = (int64_t)blockIdx.x * (SG_T / 32) + (threadIdx.x >> 5); c < nchunk; c += nwarp) {
+        const int cnt = (int)chunk_cnt[c];
+        const uint32_t* seg = seg_key + c * SG_CH;
+        for (int j = lane; j < cnt; j += 32) {
+            const uint32_t key = seg[j];
+            if (PASS == 1) { if ((key >> 21) == prefix) atomicAdd(&s_h[(key >> 10) & 0x7FFu], 1u); }
+            else { if ((key >> 10) == prefix) atomicAdd(&s_h[key & 0x3FFu], 1u); }
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 2048; i += SG_T)
+        if (s_h[i]) atomicAdd(&hist[i], s_h[i]);
+}
+
+__global__ void __launch_bounds__(SG_T)
+cand_count_kernel(const uint32_t* __restrict__ seg_key, const uint32_t* __restrict__ chunk_cnt, int64_t nchunk,
+                  const SelectState* __restrict__ state, int32_t* __restrict__ blk_cnt, Gate gate)
+{
+    if (gate.closed()) return;
+    const uint32_t T = state->prefix;
+    const int lane = threadIdx.x & 31;
+    const int64_t nwarp = (int64_t)gridDim.x * (SG_T / 32);
+    for (int64_t c = (int64_t)blockIdx.x * (SG_T / 32) + (threadIdx.x >> 5); c < nchunk; c += nwarp) {
+        const int cnt = (int)chunk_cnt[c];
+        const uint32_t* seg = seg_key + c * SG_CH;
+        int gt = 0, eq = 0;
+        for (int j = lane; j < cnt; j += 32) {
+            const uint32_t key = seg[j];
+            gt += (key > T); eq += (key == T);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { gt += __shfl_xor_sync(0xFFFFFFFFu, gt, o); eq += __shfl_xor_sync(0xFFFFFFFFu, eq, o); }
+        if (lane == 0) { blk_cnt[2 * c] = gt; blk_cnt[2 * c + 1] = eq; }
+    }
+}
+
+__global__ void __launch_bounds__(SG_T)
+cand_write_kernel(const uint32_t* __restrict__ seg_key, const uint16_t* __restrict__ seg_off,
+                  const uint32_t* __restrict__ chunk_cnt, int64_t nchunk, const SelectState* __restrict__ state,
+                  const int64_t* __restrict__ blk_off, int64_t* __restrict__ indices, Gate gate)
+{
+    if (gate.closed()) return;
+    const uint32_t T = state->prefix;
+    const int64_t k_ties = state->k_rem;
+    const int lane = threadIdx.x & 31;
+    const uint32_t lt = (1u << lane) - 1u;
+    const int64_t nwarp = (int64_t)gridDim.x * (SG_T / 32);
+    for (int64_t c = (int64_t)blockIdx.x * (SG_T / 32) + (threadIdx.x >> 5); c < nchunk; c += nwarp) {
+        const int cnt = (int)chunk_cnt[c];
+        const uint32_t* seg = seg_key + c * SG_CH;
+        const uint16_t* off = seg_off + c * SG_CH;
+        int64_t gt_run = blk_off[2 * c], eq_run = blk_off[2 * c + 1];
+        for (int j0 = 0; j0 < cnt; j0 += 32) {
+            const int j = j0 + lane;
+            const uint32_t key = (j < cnt) ? seg[j] : 0u;
+            const bool g = (j < cnt) && key > T, e = (j < cnt) && key == T;
+            const uint32_t bg = __ballot_sync(0xFFFFFFFFu, g), be = __ballot_sync(0xFFFFFFFFu, e);
+            const int64_t gt_before = gt_run + __popc(bg & lt), eq_before = eq_run + __popc(be & lt);
+            if (g || (e && eq_before < k_ties))
+                indices[gt_before + (eq_before < k_ties ? eq_before : k_ties)] = c * SG_CH + off[j];
+            gt_run += __popc(bg); eq_run += __popc(be);
+        }
     }
 }
 
@@ -213,38 +506,121 @@ SelectWs carve(void* ws, int64_t N)
     return w;
 }
 
-}  // namespace
-
-size_t select_workspace_bytes(int64_t N)
+size_t compact_workspace_bytes(int64_t N)
 {
     const int64_t nblk = sel_nblk(N > 0 ? N : 1);
     return 3 * 2048 * sizeof(uint32_t) + 256 + align_up((size_t)nblk * 2 * sizeof(int64_t), 256) +
            align_up((size_t)nblk * 2 * sizeof(int32_t), 256);
 }
 
-cudaError_t launch_select_topk(const float* scores, int64_t N, int64_t k, int64_t* indices, void* ws,
-                               cudaStream_t st)
+BracketWs carve_bracket(void* ws, int64_t N)
 {
-    if (N == 0 || k == 0) return cudaSuccess;
-    SelectWs w = carve(ws, N);
-    cudaError_t e = cudaMemsetAsync(w.hist, 0, 3 * 2048 * sizeof(uint32_t), st);
-    if (e != cudaSuccess) return e;
+    BracketWs w;
+    uint8_t* p = reinterpret_cast<uint8_t*>(ws);
+    w.hist = reinterpret_cast<uint32_t*>(p); p += 6 * 2048 * sizeof(uint32_t);
+    w.state = reinterpret_cast<SelectState*>(p);
+    w.bstate = reinterpret_cast<BracketState*>(p + 64); p += 256;
+    const int64_t nblk = sel_nblk(N), nchunk = sg_nchunk(N);
+    w.blk_off = reinterpret_cast<int64_t*>(p); p += align_up((size_t)nblk * 2 * sizeof(int64_t), 256);
+    w.blk_cnt = reinterpret_cast<int32_t*>(p); p += align_up((size_t)nblk * 2 * sizeof(int32_t), 256);
+    w.chunk_cnt = reinterpret_cast<uint32_t*>(p); p += align_up((size_t)nchunk * sizeof(uint32_t), 256);
+    w.seg_off = reinterpret_cast<uint16_t*>(p); p += align_up((size_t)nchunk * SG_CH * sizeof(uint16_t), 256);
+    w.seg_key = reinterpret_cast<uint32_t*>(p);
+    return w;
+}
+
+size_t bracket_workspace_bytes(int64_t N)
+{
+    const int64_t nblk = sel_nblk(N), nchunk = sg_nchunk(N);
+    return 6 * 2048 * sizeof(uint32_t) + 256 + align_up((size_t)nblk * 2 * sizeof(int64_t), 256) +
+           align_up((size_t)nblk * 2 * sizeof(int32_t), 256) + align_up((size_t)nchunk * sizeof(uint32_t), 256) +
+           align_up((size_t)nchunk * SG_CH * sizeof(uint16_t), 256) + (size_t)nchunk * SG_CH * sizeof(uint32_t);
+}
+
+// The exact multi-pass path on the scores themselves (five reads). hist: three cleared histograms.
+cudaError_t launch_multipass(const float* scores, int64_t N, int64_t k, int64_t* indices, uint32_t* hist,
+                             SelectState* state, int32_t* blk_cnt, int64_t* blk_off, Gate gate, cudaStream_t st)
+{
     int64_t hb = (N / 4 + SEL_T - 1) / SEL_T;
     const int64_t cap = (int64_t)sm_count() * 8;
     if (hb > cap) hb = cap;
     if (hb < 1) hb = 1;
-    select_hist_kernel<0><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, w.state, w.hist);
-    select_scan_kernel<0><<<1, 1024, 0, st>>>(w.hist, w.state, k);
-    select_hist_kernel<1><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, w.state, w.hist + 2048);
-    select_scan_kernel<1><<<1, 1024, 0, st>>>(w.hist + 2048, w.state, k);
-    select_hist_kernel<2><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, w.state, w.hist + 4096);
-    select_scan_kernel<2><<<1, 1024, 0, st>>>(w.hist + 4096, w.state, k);
+    select_hist_kernel<0><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, state, hist, gate);
+    select_scan_kernel<0><<<1, 1024, 0, st>>>(hist, state, k, gate, nullptr);
+    select_hist_kernel<1><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, state, hist + 2048, gate);
+    select_scan_kernel<1><<<1, 1024, 0, st>>>(hist + 2048, state, k, gate, nullptr);
+    select_hist_kernel<2><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, state, hist + 4096, gate);
+    select_scan_kernel<2><<<1, 1024, 0, st>>>(hist + 4096, state, k, gate, nullptr);
     const int64_t nblk = sel_nblk(N);
-    select_count_kernel<<<(unsigned)nblk, SEL_T, 0, st>>>(scores, N, w.state, w.blk_cnt);
-    select_block_scan_kernel<<<1, 1024, 0, st>>>(w.blk_cnt, nblk, w.blk_off);
-    select_write_kernel<<<(unsigned)nblk, SEL_T, 0, st>>>(scores, N, w.state, w.blk_off, indices);
+    const int64_t cap2 = (int64_t)sm_count() * 32;
+    const unsigned cg = (unsigned)(nblk < cap2 ? nblk : cap2);
+    select_count_kernel<<<cg, SEL_T, 0, st>>>(scores, N, nblk, state, blk_cnt, gate);
+    select_block_scan_kernel<<<1, 1024, 0, st>>>(blk_cnt, nblk, blk_off, gate);
+    select_write_kernel<<<cg, SEL_T, 0, st>>>(scores, N, nblk, state, blk_off, indices, gate);
     count_launches(9);
     return cudaGetLastError();
+}
+
+cudaError_t launch_bracketed(const float* scores, int64_t N, int64_t k, int64_t* indices, void* ws, bool force_short,
+                             cudaStream_t st)
+{
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(select_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        SG_SAMPLE * (int)sizeof(uint32_t));
+    });
+    if (attr_err != cudaSuccess) return attr_err;
+    BracketWs w = carve_bracket(ws, N);
+    cudaError_t e = cudaMemsetAsync(w.hist, 0, 6 * 2048 * sizeof(uint32_t) + 256, st);
+    if (e != cudaSuccess) return e;
+    const int64_t nchunk = sg_nchunk(N);
+    const int64_t cap = (int64_t)sm_count() * 8;
+    const unsigned gb = (unsigned)(nchunk < cap ? nchunk : cap);
+    const int64_t wb = (nchunk + SG_T / 32 - 1) / (SG_T / 32);
+    const unsigned cb = (unsigned)(wb < cap ? wb : cap);
+    const Gate none{nullptr, 0u};
+    const Gate ok{&w.bstate->fallback, 0u};          // enough candidates: select among them
+    const Gate fb{&w.bstate->fallback, 1u};          // too few: exact path on the scores
+    select_sample_kernel<<<1, 1024, SG_SAMPLE * sizeof(uint32_t), st>>>(scores, N, k, w.bstate, force_short ? 1 : 0);
+    select_gather_kernel<<<gb, SG_T, 0, st>>>(scores, N, w.bstate, w.seg_key, w.seg_off, w.chunk_cnt, w.hist);
+    select_scan_kernel<0><<<1, 1024, 0, st>>>(w.hist, w.state, k, none, &w.bstate->fallback);
+    cand_hist_kernel<1><<<cb, SG_T, 0, st>>>(w.seg_key, w.chunk_cnt, nchunk, w.state, w.hist + 2048, ok);
+    select_scan_kernel<1><<<1, 1024, 0, st>>>(w.hist + 2048, w.state, k, ok, nullptr);
+    cand_hist_kernel<2><<<cb, SG_T, 0, st>>>(w.seg_key, w.chunk_cnt, nchunk, w.state, w.hist + 4096, ok);
+    select_scan_kernel<2><<<1, 1024, 0, st>>>(w.hist + 4096, w.state, k, ok, nullptr);
+    cand_count_kernel<<<cb, SG_T, 0, st>>>(w.seg_key, w.chunk_cnt, nchunk, w.state, w.blk_cnt, ok);
+    select_block_scan_kernel<<<1, 1024, 0, st>>>(w.blk_cnt, nchunk, w.blk_off, ok);
+    cand_write_kernel<<<cb, SG_T, 0, st>>>(w.seg_key, w.seg_off, w.chunk_cnt, nchunk, w.state, w.blk_off, indices, ok);
+    count_launches(10);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return launch_multipass(scores, N, k, indices, w.hist + 3 * 2048, w.state, w.blk_cnt, w.blk_off, fb, st);
+}
+
+int g_select_path = 0;     // 0: by size; 1: multi-pass always; 2: bracketed with a bracket that is too high
+
+}  // namespace
+
+void set_select_path(int mode) { g_select_path = mode; }
+
+static bool use_bracket(int64_t N) { return g_select_path != 1 && N > SG_MIN_N; }
+
+size_t select_workspace_bytes(int64_t N)
+{
+    if (N > SG_MIN_N) return bracket_workspace_bytes(N);     // whatever the path chosen at launch time
+    return compact_workspace_bytes(N);
+}
+
+cudaError_t launch_select_topk(const float* scores, int64_t N, int64_t k, int64_t* indices, void* ws,
+                               cudaStream_t st)
+{
+    if (N == 0 || k == 0) return cudaSuccess;
+    if (use_bracket(N)) return launch_bracketed(scores, N, k, indices, ws, g_select_path == 2, st);
+    SelectWs w = carve(ws, N);
+    cudaError_t e = cudaMemsetAsync(w.hist, 0, 3 * 2048 * sizeof(uint32_t), st);
+    if (e != cudaSuccess) return e;
+    return launch_multipass(scores, N, k, indices, w.hist, w.state, w.blk_cnt, w.blk_off, Gate{nullptr, 0u}, st);
 }
 
 }  // namespace qless

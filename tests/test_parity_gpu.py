@@ -277,6 +277,46 @@ def test_topk_ties_and_special_values():
     assert _np(B.qless_select_topk(q, 0.75)).tolist() == [1, 2, 3]
 
 
+def _large_scores(kind, N, seed):
+    gen = torch.Generator(device=DEV); gen.manual_seed(seed)
+    if kind == "gauss":
+        return torch.randn(N, generator=gen, device=DEV)
+    if kind == "ties":
+        return torch.round(torch.randn(N, generator=gen, device=DEV) * 8) / 8
+    if kind == "const":
+        return torch.full((N,), -1.25, device=DEV)
+    if kind == "ascending":
+        return torch.arange(N, device=DEV, dtype=torch.float32) * (1.0 / 1024)
+    if kind == "descending":
+        return -torch.arange(N, device=DEV, dtype=torch.float32) * (1.0 / 1024)
+    if kind == "spike":       # almost all scores equal, a few thousand larger ones packed into one stretch
+        s = torch.zeros(N, device=DEV)
+        s[N // 3: N // 3 + 5000] = torch.rand(5000, generator=gen, device=DEV) + 1.0
+        return s
+    raise ValueError(kind)
+
+
+# Above 2^22 scores the selection brackets the k-th largest key from a sample, gathers the candidates
+# in one pass and selects among them; the three paths must return the oracle's set, in order.
+@pytest.mark.parametrize("kind,N", [("gauss", (1 << 22) + 1), ("gauss", 5_000_003), ("ties", 6_000_000),
+                                     ("const", (1 << 22) + 4097), ("ascending", 4_500_000),
+                                     ("descending", 4_500_001), ("spike", 5_000_000), ("gauss", (1 << 24) + 77)])
+def test_topk_large_bracketed(kind, N):
+    s = _large_scores(kind, N, 95 + N % 1000)
+    s_np = _np(s)
+    for frac in (1e-6, 0.0005, 0.05, 0.5, 1.0):
+        want = oracle.select_topk(s_np, frac)
+        got = _np(B.qless_select_topk(s, frac))
+        assert got.shape == want.shape and np.array_equal(got, want), (kind, N, frac)
+    try:
+        for path in (1, 2):
+            B.qless_set_select_path(path)
+            got = _np(B.qless_select_topk(s, 0.05))
+            assert np.array_equal(got, oracle.select_topk(s_np, 0.05)), (kind, N, path)
+    finally:
+        B.qless_set_select_path(0)
+
+
 # ----------------------------------------------------------------------------------------------
 # Config 1: tiny end to end (1000 train + 64 val, P = 8192 fp32, d = 512, 8-bit, 2 checkpoints,
 # lr [1, 0.5], 2 tasks of 32, top 5 %)
