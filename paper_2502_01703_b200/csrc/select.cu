@@ -320,48 +320,67 @@ select_sample_kernel(const float* __restrict__ scores, int64_t N, int64_t k, Bra
 
 // The second (and last) read of the scores: candidates of each chunk, in index order, to the chunk's
 // segment; their top-11-bit histogram for the first round of the radix select.
-// The test runs on s = key ^ 0x80000000 read as a signed integer (two operations per score from the
-// raw bits; NaNs with the sign bit clear land above +inf and are cut off by the range check).
+// The test runs on s = key ^ 0x80000000 read as a signed integer: lo_s <= s <= s(+inf), one subtraction
+// and one unsigned compare. For a bracket above zero (POS) s is the raw bit pattern itself: negative
+// scores and NaNs fall outside the range by themselves. Otherwise s takes two more operations per score.
 // Warp w of the block owns scores [512 w, 512 w + 512) of the chunk, lane l the four at 128 j + 4 l of
-// each of its four loads j, so that positions follow from one packed warp scan (a byte per load).
-__global__ void __launch_bounds__(SG_T)
-select_gather_kernel(const float* __restrict__ scores, int64_t N, BracketState* __restrict__ bs,
-                     uint32_t* __restrict__ seg_key, uint16_t* __restrict__ seg_off,
-                     uint32_t* __restrict__ chunk_cnt, uint32_t* __restrict__ hist0)
+// each of its four 16-byte pieces j, so that positions follow from one packed warp scan (a byte per
+// piece). Each thread fetches its own pieces with cp.async into a ring of SG_RING chunks, two chunks
+// ahead of the one it works on: enough bytes in flight per SM without holding them in registers.
+constexpr int SG_RING = 3;
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, int src_bytes)
 {
-    __shared__ uint32_t s_h[2048];
-    __shared__ uint32_t s_wtot[2][SG_T / 32];
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int KEEP> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(KEEP) : "memory"); }
+
+template <bool POS>
+__device__ __forceinline__ void gather_chunks(const float* __restrict__ scores, int64_t N, uint32_t lo,
+                                              uint32_t* __restrict__ seg_key, uint16_t* __restrict__ seg_off,
+                                              uint32_t* __restrict__ chunk_cnt, uint32_t* s_h, uint32_t (*s_wtot)[SG_T / 32],
+                                              uint32_t* s_ring, unsigned long long& mine)
+{
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int i = tid; i < 2048; i += SG_T) s_h[i] = 0;
-    __syncthreads();
-    const uint32_t lo = bs->lo_key;
     const uint32_t lo_s = lo ^ 0x80000000u;
     const uint32_t range = (lo == 0u) ? 0xFFFFFFFFu : (0x7F800000u - lo_s);     // lo == 0: NaNs are candidates too
     const int64_t nchunk = sg_nchunk(N);
-    unsigned long long mine = 0;
-    int par = 0;
+    const int wofs = warp * 512 + lane * 4;
+
+    // fetch of chunk c into a ring slot: pieces beyond N are zero-filled (src_bytes counts what exists)
+    auto fetch = [&](int64_t c, int slot) {
+        if (c < nchunk) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int64_t i = c * SG_CH + wofs + j * 128;
+                const int64_t left = N - i;
+                const int nb = left >= 4 ? 16 : (left > 0 ? (int)left * 4 : 0);
+                cp_async16(s_ring + slot * SG_CH + wofs + j * 128, nb ? (const void*)(scores + i) : (const void*)scores, nb);
+            }
+        }
+        cp_async_commit();          // a group per step, empty or not, keeps the wait count fixed
+    };
+    fetch(blockIdx.x, 0);
+    fetch((int64_t)blockIdx.x + gridDim.x, 1);
+    int slot = 0, par = 0;
     for (int64_t c = blockIdx.x; c < nchunk; c += gridDim.x, par ^= 1) {
+        fetch(c + 2 * (int64_t)gridDim.x, slot == 0 ? 2 : slot - 1);      // the slot consumed one step ago
+        cp_async_wait<2>();                                             // this thread's pieces of chunk c have landed
         const int64_t base = c * SG_CH;
-        const int wofs = warp * 512 + lane * 4;
-        uint32_t sv[4][4];
+        const uint32_t* mychunk = s_ring + slot * SG_CH + wofs;
         uint32_t flags[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int64_t i = base + wofs + j * 128;
-            uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-            uint32_t valid = 0;
-            if (i + 3 < N) { raw = __ldcs(reinterpret_cast<const uint4*>(scores + i)); valid = 0xFu; }
-            else {
-                if (i < N) { raw.x = __float_as_uint(scores[i]); valid |= 1u; }
-                if (i + 1 < N) { raw.y = __float_as_uint(scores[i + 1]); valid |= 2u; }
-                if (i + 2 < N) { raw.z = __float_as_uint(scores[i + 2]); valid |= 4u; }
-            }
+            const uint4 raw = *reinterpret_cast<const uint4*>(mychunk + j * 128);
+            const int64_t left = N - (base + wofs + j * 128);
+            const uint32_t valid = left >= 4 ? 0xFu : (left > 0 ? (1u << (int)left) - 1u : 0u);
             const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
             uint32_t f = 0;
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                sv[j][u] = r[u] ^ ((uint32_t)((int32_t)r[u] >> 31) & 0x7FFFFFFFu);
-                if (sv[j][u] - lo_s <= range) f |= 1u << u;
+                const uint32_t sv = POS ? r[u] : (r[u] ^ ((uint32_t)((int32_t)r[u] >> 31) & 0x7FFFFFFFu));
+                if (sv - lo_s <= range) f |= 1u << u;
             }
             flags[j] = f & valid;
         }
@@ -373,11 +392,10 @@ select_gather_kernel(const float* __restrict__ scores, int64_t N, BracketState* 
             const uint32_t a = __shfl_up_sync(0xFFFFFFFFu, inc, o);
             if (lane >= o) inc += a;
         }
-        const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31);       // per-load totals of this warp (<= 128 each)
+        const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31);       // per-piece totals of this warp (<= 128 each)
         const uint32_t t0 = tot & 0xFFu, t1 = (tot >> 8) & 0xFFu, t2 = (tot >> 16) & 0xFFu, t3 = tot >> 24;
-        const uint32_t wtot = t0 + t1 + t2 + t3;
-        if (lane == 0) s_wtot[par][warp] = wtot;
-        __syncthreads();                // one barrier per chunk: the two buffers alternate
+        if (lane == 0) s_wtot[par][warp] = t0 + t1 + t2 + t3;
+        __syncthreads();                // one barrier per chunk: the two total buffers alternate
         uint32_t wbase = 0, ctot = 0;
 #pragma unroll
         for (int w = 0; w < SG_T / 32; ++w) {
@@ -385,31 +403,48 @@ select_gather_kernel(const float* __restrict__ scores, int64_t N, BracketState* 
             ctot += t;
             if (w < warp) wbase += t;
         }
-        if (flags[0] | flags[1] | flags[2] | flags[3]) {
-            const uint32_t excl = inc - cnt;
-            const uint32_t lbase[4] = {wbase, wbase + t0, wbase + t0 + t1, wbase + t0 + t1 + t2};
+        const uint32_t excl = inc - cnt;
+        const uint32_t lbase[4] = {wbase, wbase + t0, wbase + t0 + t1, wbase + t0 + t1 + t2};
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (flags[j]) {
-                    uint32_t pos = lbase[j] + ((excl >> (8 * j)) & 0xFFu);
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        if ((flags[j] >> u) & 1u) {
-                            // back to the key; a NaN (only reachable with lo == 0) has key 0
-                            const uint32_t sk = sv[j][u];
-                            const bool is_nan = (sk > 0x7F800000u && sk < 0x80000000u) || (sk >= 0x80000000u && sk < 0x807FFFFFu);
-                            const uint32_t key = is_nan ? 0u : (sk ^ 0x80000000u);
-                            seg_key[base + pos] = key;
-                            seg_off[base + pos] = (uint16_t)(wofs + j * 128 + u);
-                            atomicAdd(&s_h[key >> 21], 1u);
-                            ++pos;
-                        }
-                    }
-                }
+        for (int j = 0; j < 4; ++j) {
+            uint32_t f = flags[j];
+            int64_t pos = base + lbase[j] + ((excl >> (8 * j)) & 0xFFu);
+            while (f) {
+                const int u = __ffs((int)f) - 1;
+                f &= f - 1u;
+                const uint32_t r = mychunk[j * 128 + u];
+                // the key; a NaN (only reachable with lo == 0) has key 0
+                uint32_t key;
+                if (POS) key = r | 0x80000000u;
+                else key = order_key(r);
+                seg_key[pos] = key;
+                seg_off[pos] = (uint16_t)(wofs + j * 128 + u);
+                atomicAdd(&s_h[key >> 21], 1u);
+                ++pos;
             }
         }
         if (tid == 0) { chunk_cnt[c] = ctot; mine += ctot; }
+        slot = (slot == SG_RING - 1) ? 0 : slot + 1;
     }
+    cp_async_wait<0>();
+}
+
+__global__ void __launch_bounds__(SG_T, 4)
+select_gather_kernel(const float* __restrict__ scores, int64_t N, BracketState* __restrict__ bs,
+                     uint32_t* __restrict__ seg_key, uint16_t* __restrict__ seg_off,
+                     uint32_t* __restrict__ chunk_cnt, uint32_t* __restrict__ hist0)
+{
+    extern __shared__ __align__(16) uint8_t s_dyn[];      // ring of SG_RING chunks of raw scores
+    __shared__ uint32_t s_h[2048];
+    __shared__ uint32_t s_wtot[2][SG_T / 32];
+    const int tid = threadIdx.x;
+    for (int i = tid; i < 2048; i += SG_T) s_h[i] = 0;
+    __syncthreads();
+    const uint32_t lo = bs->lo_key;
+    unsigned long long mine = 0;
+    uint32_t* s_ring = reinterpret_cast<uint32_t*>(s_dyn);
+    if (lo > 0x80000000u) gather_chunks<true>(scores, N, lo, seg_key, seg_off, chunk_cnt, s_h, s_wtot, s_ring, mine);
+    else gather_chunks<false>(scores, N, lo, seg_key, seg_off, chunk_cnt, s_h, s_wtot, s_ring, mine);
     __syncthreads();
     for (int i = tid; i < 2048; i += SG_T)
         if (s_h[i]) atomicAdd(&hist0[i], s_h[i]);
@@ -569,6 +604,9 @@ cudaError_t launch_bracketed(const float* scores, int64_t N, int64_t k, int64_t*
     std::call_once(once, [] {
         attr_err = cudaFuncSetAttribute(select_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         SG_SAMPLE * (int)sizeof(uint32_t));
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(select_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            SG_RING * SG_CH * (int)sizeof(uint32_t));
     });
     if (attr_err != cudaSuccess) return attr_err;
     BracketWs w = carve_bracket(ws, N);
@@ -576,14 +614,15 @@ cudaError_t launch_bracketed(const float* scores, int64_t N, int64_t k, int64_t*
     if (e != cudaSuccess) return e;
     const int64_t nchunk = sg_nchunk(N);
     const int64_t cap = (int64_t)sm_count() * 8;
-    const unsigned gb = (unsigned)(nchunk < cap ? nchunk : cap);
+    const int64_t gcap = (int64_t)sm_count() * 4;          // the gather kernel's resident blocks (48 KiB ring each)
+    const unsigned gb = (unsigned)(nchunk < gcap ? nchunk : gcap);
     const int64_t wb = (nchunk + SG_T / 32 - 1) / (SG_T / 32);
     const unsigned cb = (unsigned)(wb < cap ? wb : cap);
     const Gate none{nullptr, 0u};
     const Gate ok{&w.bstate->fallback, 0u};          // enough candidates: select among them
     const Gate fb{&w.bstate->fallback, 1u};          // too few: exact path on the scores
     select_sample_kernel<<<1, 1024, SG_SAMPLE * sizeof(uint32_t), st>>>(scores, N, k, w.bstate, force_short ? 1 : 0);
-    select_gather_kernel<<<gb, SG_T, 0, st>>>(scores, N, w.bstate, w.seg_key, w.seg_off, w.chunk_cnt, w.hist);
+    select_gather_kernel<<<gb, SG_T, SG_RING * SG_CH * sizeof(uint32_t), st>>>(scores, N, w.bstate, w.seg_key, w.seg_off, w.chunk_cnt, w.hist);
     select_scan_kernel<0><<<1, 1024, 0, st>>>(w.hist, w.state, k, none, &w.bstate->fallback);
     cand_hist_kernel<1><<<cb, SG_T, 0, st>>>(w.seg_key, w.chunk_cnt, nchunk, w.state, w.hist + 2048, ok);
     select_scan_kernel<1><<<1, 1024, 0, st>>>(w.hist + 2048, w.state, k, ok, nullptr);
