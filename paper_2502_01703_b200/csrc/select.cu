@@ -318,20 +318,23 @@ select_sample_kernel(const float* __restrict__ scores, int64_t N, int64_t k, Bra
     if (tid == 0) bs->lo_key = s_prefix;
 }
 
-// The second (and last) read of the scores: candidates of each chunk, in index order, to the chunk's
-// segment; their top-11-bit histogram for the first round of the radix select.
+// The second (and last) read of the scores: the candidates of each 4096-score chunk go to the chunk's
+// segment (key and offset inside the chunk, in no particular order: the final write restores index
+// order from the offsets), and their top-11-bit histogram feeds the first round of the radix select.
 // The test runs on s = key ^ 0x80000000 read as a signed integer: lo_s <= s <= s(+inf), one subtraction
 // and one unsigned compare. For a bracket above zero (POS) s is the raw bit pattern itself: negative
 // scores and NaNs fall outside the range by themselves. Otherwise s takes two more operations per score.
-// Warp w of the block owns scores [512 w, 512 w + 512) of the chunk, lane l the four at 128 j + 4 l of
-// each of its four 16-byte pieces j, so that positions follow from one packed warp scan (a byte per
-// piece). Each thread fetches its own pieces with cp.async into a ring of SG_RING chunks, two chunks
-// ahead of the one it works on: enough bytes in flight per SM without holding them in registers.
+// A warp owns whole chunks and walks each in eight steps of 512 scores (16 per lane, as four 16-byte
+// pieces 128 scores apart), with no block-wide barrier; a warp scan of the per-lane counts gives each
+// lane its run in the segment. Each lane fetches its own pieces with cp.async into a ring of three
+// steps, two steps ahead of the one it works on: enough bytes in flight per SM without registers.
 constexpr int SG_RING = 3;
+constexpr int SG_STEP = 512;                    // scores per warp step
+constexpr int SG_STEPS = SG_CH / SG_STEP;       // 8
 
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, int src_bytes)
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc, int src_bytes)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc), "r"(src_bytes) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gsrc), "r"(src_bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int KEEP> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(KEEP) : "memory"); }
@@ -339,92 +342,100 @@ template <int KEEP> __device__ __forceinline__ void cp_async_wait() { asm volati
 template <bool POS>
 __device__ __forceinline__ void gather_chunks(const float* __restrict__ scores, int64_t N, uint32_t lo,
                                               uint32_t* __restrict__ seg_key, uint16_t* __restrict__ seg_off,
-                                              uint32_t* __restrict__ chunk_cnt, uint32_t* s_h, uint32_t (*s_wtot)[SG_T / 32],
-                                              uint32_t* s_ring, unsigned long long& mine)
+                                              uint32_t* __restrict__ chunk_cnt, uint32_t* s_h, uint32_t* __restrict__ hist0,
+                                              uint32_t* s_ring /* this warp's [SG_RING][SG_STEP] */, unsigned long long& mine)
 {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int lane = threadIdx.x & 31;
     const uint32_t lo_s = lo ^ 0x80000000u;
     const uint32_t range = (lo == 0u) ? 0xFFFFFFFFu : (0x7F800000u - lo_s);     // lo == 0: NaNs are candidates too
     const int64_t nchunk = sg_nchunk(N);
-    const int wofs = warp * 512 + lane * 4;
+    const int64_t gwarp = (int64_t)blockIdx.x * (SG_T / 32) + (threadIdx.x >> 5);
+    const int64_t nwarp = (int64_t)gridDim.x * (SG_T / 32);
+    const uint32_t ring_u32 = (uint32_t)__cvta_generic_to_shared(s_ring) + lane * 16;
 
-    // fetch of chunk c into a ring slot: pieces beyond N are zero-filled (src_bytes counts what exists)
-    auto fetch = [&](int64_t c, int slot) {
-        if (c < nchunk) {
+    // fetch cursor: two steps ahead of the work cursor
+    int64_t fc = gwarp; int fsub = 0, fslot = 0;
+    auto fetch = [&]() {
+        if (fc < nchunk) {
+            const int64_t i0 = fc * SG_CH + fsub * SG_STEP;          // first score of the step
+            const float* src = scores + i0 + lane * 4;
+            const uint32_t dst = ring_u32 + fslot * (SG_STEP * 4);
+            if (N - i0 >= SG_STEP) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int64_t i = c * SG_CH + wofs + j * 128;
-                const int64_t left = N - i;
-                const int nb = left >= 4 ? 16 : (left > 0 ? (int)left * 4 : 0);
-                cp_async16(s_ring + slot * SG_CH + wofs + j * 128, nb ? (const void*)(scores + i) : (const void*)scores, nb);
+                for (int j = 0; j < 4; ++j) cp_async16(dst + j * 512, src + j * 128, 16);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {                        // pieces beyond N are zero-filled
+                    const int64_t left = N - (i0 + lane * 4 + j * 128);
+                    const int nb = left >= 4 ? 16 : (left > 0 ? (int)left * 4 : 0);
+                    cp_async16(dst + j * 512, nb ? (const void*)(src + j * 128) : (const void*)scores, nb);
+                }
             }
         }
         cp_async_commit();          // a group per step, empty or not, keeps the wait count fixed
+        fslot = (fslot == SG_RING - 1) ? 0 : fslot + 1;
+        if (++fsub == SG_STEPS) { fsub = 0; fc += nwarp; }
     };
-    fetch(blockIdx.x, 0);
-    fetch((int64_t)blockIdx.x + gridDim.x, 1);
-    int slot = 0, par = 0;
-    for (int64_t c = blockIdx.x; c < nchunk; c += gridDim.x, par ^= 1) {
-        fetch(c + 2 * (int64_t)gridDim.x, slot == 0 ? 2 : slot - 1);      // the slot consumed one step ago
-        cp_async_wait<2>();                                             // this thread's pieces of chunk c have landed
-        const int64_t base = c * SG_CH;
-        const uint32_t* mychunk = s_ring + slot * SG_CH + wofs;
-        uint32_t flags[4];
+    fetch();
+    fetch();
+    int slot = 0;
+    for (int64_t c = gwarp; c < nchunk; c += nwarp) {
+        uint32_t* kp = seg_key + c * SG_CH;
+        uint16_t* op = seg_off + c * SG_CH;
+        uint32_t run = 0;
+#pragma unroll 1
+        for (int sub = 0; sub < SG_STEPS; ++sub) {
+            fetch();
+            cp_async_wait<2>();                                       // this lane's pieces of the step have landed
+            const uint32_t* mine_s = s_ring + slot * SG_STEP + lane * 4;
+            const int64_t i0 = c * SG_CH + sub * SG_STEP;
+            uint32_t F = 0;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const uint4 raw = *reinterpret_cast<const uint4*>(mychunk + j * 128);
-            const int64_t left = N - (base + wofs + j * 128);
-            const uint32_t valid = left >= 4 ? 0xFu : (left > 0 ? (1u << (int)left) - 1u : 0u);
-            const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
-            uint32_t f = 0;
+            for (int j = 0; j < 4; ++j) {
+                const uint4 raw = *reinterpret_cast<const uint4*>(mine_s + j * 128);
+                const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const uint32_t sv = POS ? r[u] : (r[u] ^ ((uint32_t)((int32_t)r[u] >> 31) & 0x7FFFFFFFu));
-                if (sv - lo_s <= range) f |= 1u << u;
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t sv = POS ? r[u] : (r[u] ^ ((uint32_t)((int32_t)r[u] >> 31) & 0x7FFFFFFFu));
+                    if (sv - lo_s <= range) F |= 1u << (4 * j + u);
+                }
             }
-            flags[j] = f & valid;
-        }
-        const uint32_t cnt = (uint32_t)__popc(flags[0]) | ((uint32_t)__popc(flags[1]) << 8) |
-                             ((uint32_t)__popc(flags[2]) << 16) | ((uint32_t)__popc(flags[3]) << 24);
-        uint32_t inc = cnt;
+            if (N - i0 < SG_STEP) {                                   // ragged end: drop what lies beyond N
+                uint32_t valid = 0;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t a = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-            if (lane >= o) inc += a;
-        }
-        const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31);       // per-piece totals of this warp (<= 128 each)
-        const uint32_t t0 = tot & 0xFFu, t1 = (tot >> 8) & 0xFFu, t2 = (tot >> 16) & 0xFFu, t3 = tot >> 24;
-        if (lane == 0) s_wtot[par][warp] = t0 + t1 + t2 + t3;
-        __syncthreads();                // one barrier per chunk: the two total buffers alternate
-        uint32_t wbase = 0, ctot = 0;
+                for (int j = 0; j < 4; ++j) {
+                    const int64_t left = N - (i0 + lane * 4 + j * 128);
+                    valid |= (left >= 4 ? 0xFu : (left > 0 ? (1u << (int)left) - 1u : 0u)) << (4 * j);
+                }
+                F &= valid;
+            }
+            const uint32_t cnt = (uint32_t)__popc(F);
+            uint32_t inc = cnt;
 #pragma unroll
-        for (int w = 0; w < SG_T / 32; ++w) {
-            const uint32_t t = s_wtot[par][w];
-            ctot += t;
-            if (w < warp) wbase += t;
-        }
-        const uint32_t excl = inc - cnt;
-        const uint32_t lbase[4] = {wbase, wbase + t0, wbase + t0 + t1, wbase + t0 + t1 + t2};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            uint32_t f = flags[j];
-            int64_t pos = base + lbase[j] + ((excl >> (8 * j)) & 0xFFu);
-            while (f) {
-                const int u = __ffs((int)f) - 1;
-                f &= f - 1u;
-                const uint32_t r = mychunk[j * 128 + u];
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t a = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                if (lane >= o) inc += a;
+            }
+            const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31);
+            uint32_t pos = run + inc - cnt;
+            const uint32_t obase = (uint32_t)(sub * SG_STEP + lane * 4);
+            while (F) {
+                const int b = __ffs((int)F) - 1;
+                F &= F - 1u;
+                const uint32_t e = (uint32_t)((b >> 2) * 128 + (b & 3));
+                const uint32_t r = mine_s[e];
                 // the key; a NaN (only reachable with lo == 0) has key 0
-                uint32_t key;
-                if (POS) key = r | 0x80000000u;
-                else key = order_key(r);
-                seg_key[pos] = key;
-                seg_off[pos] = (uint16_t)(wofs + j * 128 + u);
-                atomicAdd(&s_h[key >> 21], 1u);
+                const uint32_t key = POS ? (r | 0x80000000u) : order_key(r);
+                kp[pos] = key;
+                op[pos] = (uint16_t)(obase + e);
+                if (POS || key >= 0x80000000u) atomicAdd(&s_h[(key >> 21) - 1024u], 1u);
+                else atomicAdd(&hist0[key >> 21], 1u);          // negative scores and NaNs: rare as candidates
                 ++pos;
             }
+            run += tot;
+            slot = (slot == SG_RING - 1) ? 0 : slot + 1;
         }
-        if (tid == 0) { chunk_cnt[c] = ctot; mine += ctot; }
-        slot = (slot == SG_RING - 1) ? 0 : slot + 1;
+        if (lane == 0) { chunk_cnt[c] = run; mine += run; }
     }
     cp_async_wait<0>();
 }
@@ -434,21 +445,20 @@ select_gather_kernel(const float* __restrict__ scores, int64_t N, BracketState* 
                      uint32_t* __restrict__ seg_key, uint16_t* __restrict__ seg_off,
                      uint32_t* __restrict__ chunk_cnt, uint32_t* __restrict__ hist0)
 {
-    extern __shared__ __align__(16) uint8_t s_dyn[];      // ring of SG_RING chunks of raw scores
-    __shared__ uint32_t s_h[2048];
-    __shared__ uint32_t s_wtot[2][SG_T / 32];
+    extern __shared__ __align__(16) uint8_t s_dyn[];      // per warp: ring of SG_RING steps of raw scores
+    __shared__ uint32_t s_h[1024];           // bins 1024..2047: keys of scores with the sign bit clear
     const int tid = threadIdx.x;
-    for (int i = tid; i < 2048; i += SG_T) s_h[i] = 0;
+    for (int i = tid; i < 1024; i += SG_T) s_h[i] = 0;
     __syncthreads();
     const uint32_t lo = bs->lo_key;
     unsigned long long mine = 0;
-    uint32_t* s_ring = reinterpret_cast<uint32_t*>(s_dyn);
-    if (lo > 0x80000000u) gather_chunks<true>(scores, N, lo, seg_key, seg_off, chunk_cnt, s_h, s_wtot, s_ring, mine);
-    else gather_chunks<false>(scores, N, lo, seg_key, seg_off, chunk_cnt, s_h, s_wtot, s_ring, mine);
+    uint32_t* s_ring = reinterpret_cast<uint32_t*>(s_dyn) + (tid >> 5) * (SG_RING * SG_STEP);
+    if (lo > 0x80000000u) gather_chunks<true>(scores, N, lo, seg_key, seg_off, chunk_cnt, s_h, hist0, s_ring, mine);
+    else gather_chunks<false>(scores, N, lo, seg_key, seg_off, chunk_cnt, s_h, hist0, s_ring, mine);
     __syncthreads();
-    for (int i = tid; i < 2048; i += SG_T)
-        if (s_h[i]) atomicAdd(&hist0[i], s_h[i]);
-    if (tid == 0 && mine) atomicAdd(&bs->n_cand, mine);
+    for (int i = tid; i < 1024; i += SG_T)
+        if (s_h[i]) atomicAdd(&hist0[1024 + i], s_h[i]);
+    if ((tid & 31) == 0 && mine) atomicAdd(&bs->n_cand, mine);
 }
 
 // Radix-select rounds 2 and 3 on the candidates: one warp per chunk segment.
@@ -500,32 +510,67 @@ cand_count_kernel(const uint32_t* __restrict__ seg_key, const uint32_t* __restri
     }
 }
 
+// Final write: a warp per chunk marks the offsets of {key > T} and of {key == T} in two 4096-bit maps
+// in shared memory, which puts the segment's unordered candidates back in index order; each lane then
+// walks its 128 bits, and the running counts (block offsets + warp scan) give every index its place.
 __global__ void __launch_bounds__(SG_T)
 cand_write_kernel(const uint32_t* __restrict__ seg_key, const uint16_t* __restrict__ seg_off,
                   const uint32_t* __restrict__ chunk_cnt, int64_t nchunk, const SelectState* __restrict__ state,
                   const int64_t* __restrict__ blk_off, int64_t* __restrict__ indices, Gate gate)
 {
+    __shared__ __align__(16) uint32_t s_bm[SG_T / 32][2][SG_CH / 32];
     if (gate.closed()) return;
     const uint32_t T = state->prefix;
     const int64_t k_ties = state->k_rem;
-    const int lane = threadIdx.x & 31;
-    const uint32_t lt = (1u << lane) - 1u;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t* bm_gt = s_bm[warp][0];
+    uint32_t* bm_eq = s_bm[warp][1];
     const int64_t nwarp = (int64_t)gridDim.x * (SG_T / 32);
-    for (int64_t c = (int64_t)blockIdx.x * (SG_T / 32) + (threadIdx.x >> 5); c < nchunk; c += nwarp) {
+    for (int64_t c = (int64_t)blockIdx.x * (SG_T / 32) + warp; c < nchunk; c += nwarp) {
         const int cnt = (int)chunk_cnt[c];
+        if (cnt == 0) continue;
         const uint32_t* seg = seg_key + c * SG_CH;
         const uint16_t* off = seg_off + c * SG_CH;
-        int64_t gt_run = blk_off[2 * c], eq_run = blk_off[2 * c + 1];
-        for (int j0 = 0; j0 < cnt; j0 += 32) {
-            const int j = j0 + lane;
-            const uint32_t key = (j < cnt) ? seg[j] : 0u;
-            const bool g = (j < cnt) && key > T, e = (j < cnt) && key == T;
-            const uint32_t bg = __ballot_sync(0xFFFFFFFFu, g), be = __ballot_sync(0xFFFFFFFFu, e);
-            const int64_t gt_before = gt_run + __popc(bg & lt), eq_before = eq_run + __popc(be & lt);
-            if (g || (e && eq_before < k_ties))
-                indices[gt_before + (eq_before < k_ties ? eq_before : k_ties)] = c * SG_CH + off[j];
-            gt_run += __popc(bg); eq_run += __popc(be);
+        reinterpret_cast<uint4*>(bm_gt)[lane] = make_uint4(0u, 0u, 0u, 0u);
+        reinterpret_cast<uint4*>(bm_eq)[lane] = make_uint4(0u, 0u, 0u, 0u);
+        __syncwarp();
+        for (int j = lane; j < cnt; j += 32) {
+            const uint32_t key = seg[j];
+            if (key >= T) {
+                const uint32_t o = off[j];
+                atomicOr((key > T ? bm_gt : bm_eq) + (o >> 5), 1u << (o & 31u));
+            }
         }
+        __syncwarp();
+        const uint4 g4 = reinterpret_cast<const uint4*>(bm_gt)[lane];
+        const uint4 e4 = reinterpret_cast<const uint4*>(bm_eq)[lane];
+        const uint32_t g[4] = {g4.x, g4.y, g4.z, g4.w}, e[4] = {e4.x, e4.y, e4.z, e4.w};
+        const int cg = __popc(g[0]) + __popc(g[1]) + __popc(g[2]) + __popc(g[3]);
+        const int ce = __popc(e[0]) + __popc(e[1]) + __popc(e[2]) + __popc(e[3]);
+        int ig = cg, ie = ce;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int a = __shfl_up_sync(0xFFFFFFFFu, ig, o), b2 = __shfl_up_sync(0xFFFFFFFFu, ie, o);
+            if (lane >= o) { ig += a; ie += b2; }
+        }
+        int64_t gt_before = blk_off[2 * c] + (ig - cg), eq_before = blk_off[2 * c + 1] + (ie - ce);
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            uint32_t m = g[w] | e[w];
+            const int64_t ibase = c * SG_CH + (lane * 4 + w) * 32;
+            while (m) {
+                const int b = __ffs((int)m) - 1;
+                m &= m - 1u;
+                if ((g[w] >> b) & 1u) {
+                    indices[gt_before + (eq_before < k_ties ? eq_before : k_ties)] = ibase + b;
+                    ++gt_before;
+                } else {
+                    if (eq_before < k_ties) indices[gt_before + eq_before] = ibase + b;
+                    ++eq_before;
+                }
+            }
+        }
+        __syncwarp();       // the maps are cleared again for the warp's next chunk
     }
 }
 
@@ -606,7 +651,7 @@ cudaError_t launch_bracketed(const float* scores, int64_t N, int64_t k, int64_t*
                                         SG_SAMPLE * (int)sizeof(uint32_t));
         if (attr_err == cudaSuccess)
             attr_err = cudaFuncSetAttribute(select_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            SG_RING * SG_CH * (int)sizeof(uint32_t));
+                                            (SG_T / 32) * SG_RING * SG_STEP * (int)sizeof(uint32_t));
     });
     if (attr_err != cudaSuccess) return attr_err;
     BracketWs w = carve_bracket(ws, N);
@@ -615,14 +660,15 @@ cudaError_t launch_bracketed(const float* scores, int64_t N, int64_t k, int64_t*
     const int64_t nchunk = sg_nchunk(N);
     const int64_t cap = (int64_t)sm_count() * 8;
     const int64_t gcap = (int64_t)sm_count() * 4;          // the gather kernel's resident blocks (48 KiB ring each)
-    const unsigned gb = (unsigned)(nchunk < gcap ? nchunk : gcap);
+    const int64_t gneed = (nchunk + SG_T / 32 - 1) / (SG_T / 32);       // a warp per chunk
+    const unsigned gb = (unsigned)(gneed < gcap ? gneed : gcap);
     const int64_t wb = (nchunk + SG_T / 32 - 1) / (SG_T / 32);
     const unsigned cb = (unsigned)(wb < cap ? wb : cap);
     const Gate none{nullptr, 0u};
     const Gate ok{&w.bstate->fallback, 0u};          // enough candidates: select among them
     const Gate fb{&w.bstate->fallback, 1u};          // too few: exact path on the scores
     select_sample_kernel<<<1, 1024, SG_SAMPLE * sizeof(uint32_t), st>>>(scores, N, k, w.bstate, force_short ? 1 : 0);
-    select_gather_kernel<<<gb, SG_T, SG_RING * SG_CH * sizeof(uint32_t), st>>>(scores, N, w.bstate, w.seg_key, w.seg_off, w.chunk_cnt, w.hist);
+    select_gather_kernel<<<gb, SG_T, (SG_T / 32) * SG_RING * SG_STEP * sizeof(uint32_t), st>>>(scores, N, w.bstate, w.seg_key, w.seg_off, w.chunk_cnt, w.hist);
     select_scan_kernel<0><<<1, 1024, 0, st>>>(w.hist, w.state, k, none, &w.bstate->fallback);
     cand_hist_kernel<1><<<cb, SG_T, 0, st>>>(w.seg_key, w.chunk_cnt, nchunk, w.state, w.hist + 2048, ok);
     select_scan_kernel<1><<<1, 1024, 0, st>>>(w.hist + 2048, w.state, k, ok, nullptr);
