@@ -146,34 +146,135 @@ select_count_kernel(const float* __restrict__ scores, int64_t N, int64_t nblk, c
     }
 }
 
-// Exclusive prefix sums over blocks: one block of 1024 threads, thread t sums its run of consecutive
-// entries, the block scans the 1024 run totals, and each thread writes the prefixes of its run.
+// Exclusive prefix sums over blocks: one block of 32 warps. Warp w scans its run of consecutive entries
+// in coalesced tiles of 32 (shuffle scan, running total carried along) and writes run-local prefixes;
+// after the 32 run totals are combined, a second sweep adds each run's base.
 __global__ void __launch_bounds__(1024)
 select_block_scan_kernel(const int32_t* __restrict__ blk_cnt, int64_t nblk, int64_t* __restrict__ blk_off, Gate gate)
 {
     if (gate.closed()) return;
     __shared__ int64_t s_w[2][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t per = (nblk + 1023) / 1024;
-    const int64_t b0 = threadIdx.x * per, b1 = (b0 + per < nblk) ? b0 + per : nblk;
+    const int64_t per = ((nblk + 31) / 32 + 31) / 32 * 32;          // entries per warp, a multiple of 32
+    const int64_t b0 = warp * per, b1 = (b0 + per < nblk) ? b0 + per : nblk;
     const int2* cnt2 = reinterpret_cast<const int2*>(blk_cnt);
-    int64_t v0 = 0, v1 = 0;
-    for (int64_t b = b0; b < b1; ++b) { const int2 c = cnt2[b]; v0 += c.x; v1 += c.y; }
-    int64_t i0 = v0, i1 = v1;
+    longlong2* off2 = reinterpret_cast<longlong2*>(blk_off);
+    int64_t run0 = 0, run1 = 0;
+    constexpr int NB = 8;                           // tiles fetched together: one memory round trip per batch
+    for (int64_t t = b0; t < b1; t += 32 * NB) {
+        int2 c[NB];
+#pragma unroll
+        for (int q = 0; q < NB; ++q) {
+            const int64_t b = t + q * 32 + lane;
+            c[q] = (b < b1) ? cnt2[b] : make_int2(0, 0);
+        }
+#pragma unroll
+        for (int q = 0; q < NB; ++q) {
+            const int64_t b = t + q * 32 + lane;
+            int i0 = c[q].x, i1 = c[q].y;           // a tile sums to at most 32 * 4096
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int a0 = __shfl_up_sync(0xFFFFFFFFu, i0, o), a1 = __shfl_up_sync(0xFFFFFFFFu, i1, o);
+                if (lane >= o) { i0 += a0; i1 += a1; }
+            }
+            if (b < b1) off2[b] = make_longlong2(run0 + (i0 - c[q].x), run1 + (i1 - c[q].y));
+            run0 += __shfl_sync(0xFFFFFFFFu, i0, 31);
+            run1 += __shfl_sync(0xFFFFFFFFu, i1, 31);
+        }
+    }
+    if (lane == 0) { s_w[0][warp] = run0; s_w[1][warp] = run1; }
+    __syncthreads();
+    if (warp == 0) return;
+    int64_t base0 = 0, base1 = 0;
+    for (int w = 0; w < warp; ++w) { base0 += s_w[0][w]; base1 += s_w[1][w]; }
+    for (int64_t t = b0; t < b1; t += 32 * NB) {
+        longlong2 v[NB];
+#pragma unroll
+        for (int q = 0; q < NB; ++q) {
+            const int64_t b = t + q * 32 + lane;
+            if (b < b1) v[q] = off2[b];             // this lane's own writes of the first sweep
+        }
+#pragma unroll
+        for (int q = 0; q < NB; ++q) {
+            const int64_t b = t + q * 32 + lane;
+            if (b < b1) { v[q].x += base0; v[q].y += base1; off2[b] = v[q]; }
+        }
+    }
+}
+
+// The same prefix sums for many blocks, spread over the GPU (one SM alone is bound by its own memory
+// bandwidth): tiles of 1024 entries are scanned by a block each, which also leaves the tile's total;
+// a second launch adds to every tile the sum of the totals of the tiles before it.
+__global__ void __launch_bounds__(1024)
+select_tile_scan_kernel(const int32_t* __restrict__ blk_cnt, int64_t nblk, int64_t* __restrict__ blk_off,
+                        int64_t* __restrict__ tile_tot, Gate gate)
+{
+    if (gate.closed()) return;
+    __shared__ int s_w[2][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t b = (int64_t)blockIdx.x * 1024 + threadIdx.x;
+    int2 c = make_int2(0, 0);
+    if (b < nblk) c = reinterpret_cast<const int2*>(blk_cnt)[b];
+    int i0 = c.x, i1 = c.y;                         // a tile sums to at most 1024 * 4096
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        const int64_t a0 = __shfl_up_sync(0xFFFFFFFFu, i0, o), a1 = __shfl_up_sync(0xFFFFFFFFu, i1, o);
+        const int a0 = __shfl_up_sync(0xFFFFFFFFu, i0, o), a1 = __shfl_up_sync(0xFFFFFFFFu, i1, o);
         if (lane >= o) { i0 += a0; i1 += a1; }
     }
     if (lane == 31) { s_w[0][warp] = i0; s_w[1][warp] = i1; }
     __syncthreads();
-    int64_t r0 = i0 - v0, r1 = i1 - v1;
-    for (int w = 0; w < warp; ++w) { r0 += s_w[0][w]; r1 += s_w[1][w]; }
-    longlong2* off2 = reinterpret_cast<longlong2*>(blk_off);
-    for (int64_t b = b0; b < b1; ++b) {
-        const int2 c = cnt2[b];
-        off2[b] = make_longlong2(r0, r1);
-        r0 += c.x; r1 += c.y;
+    const int w0 = s_w[0][lane], w1 = s_w[1][lane];
+    int p0 = w0, p1 = w1;                           // every warp scans the 32 warp totals
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int a0 = __shfl_up_sync(0xFFFFFFFFu, p0, o), a1 = __shfl_up_sync(0xFFFFFFFFu, p1, o);
+        if (lane >= o) { p0 += a0; p1 += a1; }
+    }
+    const int base0 = __shfl_sync(0xFFFFFFFFu, p0 - w0, warp), base1 = __shfl_sync(0xFFFFFFFFu, p1 - w1, warp);
+    if (b < nblk) reinterpret_cast<longlong2*>(blk_off)[b] = make_longlong2((int64_t)(base0 + i0 - c.x), (int64_t)(base1 + i1 - c.y));
+    if (threadIdx.x == 1023)
+        reinterpret_cast<longlong2*>(tile_tot)[blockIdx.x] = make_longlong2((int64_t)(base0 + i0), (int64_t)(base1 + i1));
+}
+
+__global__ void __launch_bounds__(1024)
+select_tile_add_kernel(int64_t nblk, int64_t* __restrict__ blk_off, const int64_t* __restrict__ tile_tot, Gate gate)
+{
+    if (gate.closed()) return;
+    if (blockIdx.x == 0) return;
+    __shared__ int64_t s_w[2][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int64_t a0 = 0, a1 = 0;
+    for (int64_t t = threadIdx.x; t < (int64_t)blockIdx.x; t += 1024) {
+        const longlong2 v = reinterpret_cast<const longlong2*>(tile_tot)[t];
+        a0 += v.x; a1 += v.y;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { a0 += __shfl_xor_sync(0xFFFFFFFFu, a0, o); a1 += __shfl_xor_sync(0xFFFFFFFFu, a1, o); }
+    if (lane == 0) { s_w[0][warp] = a0; s_w[1][warp] = a1; }
+    __syncthreads();
+    int64_t base0 = 0, base1 = 0;
+#pragma unroll
+    for (int w = 0; w < 32; ++w) { base0 += s_w[0][w]; base1 += s_w[1][w]; }
+    const int64_t b = (int64_t)blockIdx.x * 1024 + threadIdx.x;
+    if (b < nblk) {
+        longlong2 v = reinterpret_cast<longlong2*>(blk_off)[b];
+        v.x += base0; v.y += base1;
+        reinterpret_cast<longlong2*>(blk_off)[b] = v;
+    }
+}
+
+// Prefix sums over the per-block counts: one launch for a few thousand blocks, two beyond.
+inline void launch_block_scan(const int32_t* blk_cnt, int64_t nblk, int64_t* blk_off, int64_t* tile_tot, Gate gate,
+                              cudaStream_t st)
+{
+    if (tile_tot == nullptr || nblk <= 4096) {
+        select_block_scan_kernel<<<1, 1024, 0, st>>>(blk_cnt, nblk, blk_off, gate);
+        count_launches(1);
+    } else {
+        const unsigned tiles = (unsigned)((nblk + 1023) / 1024);
+        select_tile_scan_kernel<<<tiles, 1024, 0, st>>>(blk_cnt, nblk, blk_off, tile_tot, gate);
+        select_tile_add_kernel<<<tiles, 1024, 0, st>>>(nblk, blk_off, tile_tot, gate);
+        count_launches(2);
     }
 }
 
@@ -248,6 +349,8 @@ struct BracketWs {
     BracketState* bstate;
     int64_t* blk_off;             // sized for the fallback's 2048-score blocks
     int32_t* blk_cnt;
+    int64_t* tile_tot;            // [ceil(nblk / 1024)][2] totals of the block-count tiles
+    uint32_t* sample_key;         // [SG_SAMPLE]
     uint32_t* chunk_cnt;          // [nchunk]
     uint16_t* seg_off;            // [nchunk][SG_CH] offset of the candidate inside its chunk
     uint32_t* seg_key;            // [nchunk][SG_CH]
@@ -261,61 +364,53 @@ __device__ __forceinline__ uint32_t mix32(uint32_t x)
     return x;
 }
 
-// One block: sample one score per stratum, find the r-th largest sampled key in shared memory
-// (three histogram rounds), r = expected rank of the k-th largest + 6 standard deviations + 8.
+// First launch of the bracketed path, spread over the GPU: clears the histograms and the state, and
+// fetches one score per stratum (16384 scattered reads: far too many misses for one SM to keep in flight).
+__global__ void __launch_bounds__(256)
+select_init_kernel(const float* __restrict__ scores, int64_t N, uint32_t* __restrict__ clear, int clear_words,
+                   uint32_t* __restrict__ sample_key)
+{
+    const int j = blockIdx.x * 256 + threadIdx.x;           // grid covers SG_SAMPLE threads
+    for (int i = j; i < clear_words; i += SG_SAMPLE) clear[i] = 0u;
+    const int64_t per = N / SG_SAMPLE;                      // >= 256 for every N this path takes
+    // offset inside the stratum: hash scaled to [0, per) (per < 2^32 for every N below 2^46)
+    const int64_t pos = (int64_t)j * per + (int64_t)(((uint64_t)mix32(0x9E3779B9u * (uint32_t)j + 0x85EBCA6Bu) * (uint64_t)per) >> 32);
+    sample_key[j] = order_key(__float_as_uint(__ldg(scores + pos)));
+}
+
+// One block: the r-th largest sampled key by bisection on the key's bits, largest t with
+// #{key >= t} >= r: 32 block-wide counts over 16 keys per thread held in registers.
+// r = expected rank of the k-th largest + 6 standard deviations + 8.
 __global__ void __launch_bounds__(1024)
-select_sample_kernel(const float* __restrict__ scores, int64_t N, int64_t k, BracketState* __restrict__ bs,
+select_sample_kernel(const uint32_t* __restrict__ sample_key, int64_t N, int64_t k, BracketState* __restrict__ bs,
                      int force_short)
 {
-    extern __shared__ uint32_t s_key[];          // [SG_SAMPLE]
-    __shared__ uint32_t s_h[2048];
-    __shared__ int s_w[32];
-    __shared__ uint32_t s_prefix;
-    __shared__ int s_rem;
+    constexpr int PER_T = SG_SAMPLE / 1024;
+    __shared__ int s_cnt[2][32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t per = N / SG_SAMPLE;           // >= 256 for every N this path takes
-    for (int j = tid; j < SG_SAMPLE; j += 1024) {
-        const int64_t pos = (int64_t)j * per + (int64_t)(mix32(0x9E3779B9u * (uint32_t)j + 0x85EBCA6Bu) % (uint64_t)per);
-        s_key[j] = order_key(__float_as_uint(__ldg(scores + pos)));
-    }
     const double p = (double)k / (double)N;
     const double ks = ceil(p * (double)SG_SAMPLE);
     const double rr = ks + ceil(6.0 * sqrt(ks * (1.0 - p))) + 8.0;
     if (force_short) { if (tid == 0) bs->lo_key = 0xFF800000u; return; }      // key of +inf
     if (rr >= (double)SG_SAMPLE) { if (tid == 0) bs->lo_key = 0u; return; }     // every score is a candidate
-    if (tid == 0) { s_prefix = 0u; s_rem = (int)rr; }
-    __syncthreads();
-#pragma unroll 1
-    for (int round = 0; round < 3; ++round) {
-        const int shift = (round == 0) ? 21 : (round == 1) ? 10 : 0;
-        const int bits = (round == 2) ? 10 : 11;
-        const uint32_t mask = (1u << bits) - 1u;
-        for (int i = tid; i < 2048; i += 1024) s_h[i] = 0;
-        __syncthreads();
-        const uint32_t prefix = s_prefix;
-        const int rem = s_rem;
-        for (int j = tid; j < SG_SAMPLE; j += 1024) {
-            const uint32_t key = s_key[j];
-            if (round == 0 || (key >> (shift + bits)) == prefix) atomicAdd(&s_h[(key >> shift) & mask], 1u);
-        }
-        __syncthreads();
-        // prefix sum from the top bin down: thread t owns bins 2047-2t and 2046-2t
-        const int c0 = (int)s_h[2047 - 2 * tid], c1 = (int)s_h[2046 - 2 * tid];
-        int inc = c0 + c1;
+    const int r = (int)rr;
+    uint32_t v[PER_T];
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int a = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-            if (lane >= o) inc += a;
-        }
-        if (lane == 31) s_w[warp] = inc;
-        __syncthreads();
-        int pre = inc - c0 - c1;
-        for (int w = 0; w < warp; ++w) pre += s_w[w];
-        if (pre < rem && rem <= pre + c0) { s_prefix = (prefix << bits) | (uint32_t)(2047 - 2 * tid); s_rem = rem - pre; }
-        else if (pre + c0 < rem && rem <= pre + c0 + c1) { s_prefix = (prefix << bits) | (uint32_t)(2046 - 2 * tid); s_rem = rem - pre - c0; }
-        __syncthreads();
+    for (int i = 0; i < PER_T; ++i) v[i] = sample_key[tid + i * 1024];
+    uint32_t t = 0;
+#pragma unroll 1
+    for (int bit = 31; bit >= 0; --bit) {
+        const uint32_t cand = t | (1u << bit);
+        int c = 0;
+#pragma unroll
+        for (int i = 0; i < PER_T; ++i) c += (v[i] >= cand);
+        c = __reduce_add_sync(0xFFFFFFFFu, c);
+        if (lane == 0) s_cnt[bit & 1][warp] = c;
+        __syncthreads();                    // the two count buffers alternate: one barrier per bit
+        const int total = __reduce_add_sync(0xFFFFFFFFu, s_cnt[bit & 1][lane]);
+        if (total >= r) t = cand;
     }
-    if (tid == 0) bs->lo_key = s_prefix;
+    if (tid == 0) bs->lo_key = t;
 }
 
 // The second (and last) read of the scores: the candidates of each 4096-score chunk go to the chunk's
@@ -461,7 +556,55 @@ select_gather_kernel(const float* __restrict__ scores, int64_t N, BracketState* 
     if ((tid & 31) == 0 && mine) atomicAdd(&bs->n_cand, mine);
 }
 
-// Radix-select rounds 2 and 3 on the candidates: one warp per chunk segment.
+// The kernels below walk the candidate segments with one warp per chunk. A segment holds a few hundred
+// entries, so the walk is bound by memory round trips, not bytes: each warp fetches the first CB * 32
+// keys of its NEXT chunk (and the count of the one after) before it works on the current one.
+constexpr int CB = 8;
+
+struct SegCursor {
+    const uint32_t* __restrict__ seg_key;
+    const uint32_t* __restrict__ chunk_cnt;
+    int64_t nchunk, nwarp, c;
+    int lane;
+    int cnt, cnt_next;                  // of chunk c and of chunk c + nwarp
+    uint32_t k[CB], k_next[CB];         // first batch of chunk c / c + nwarp (lanes beyond the count: unspecified)
+
+    __device__ __forceinline__ void fetch_keys(int64_t chunk, int n, uint32_t (&dst)[CB]) const
+    {
+        const uint32_t* seg = seg_key + chunk * SG_CH;
+#pragma unroll
+        for (int q = 0; q < CB; ++q) {
+            const int j = q * 32 + lane;
+            if (j < n) dst[q] = __ldg(seg + j);
+        }
+    }
+    __device__ __forceinline__ void start(const uint32_t* sk, const uint32_t* cc, int64_t n)
+    {
+        seg_key = sk; chunk_cnt = cc; nchunk = n;
+        lane = threadIdx.x & 31;
+        nwarp = (int64_t)gridDim.x * (blockDim.x >> 5);
+        c = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+        cnt = (c < nchunk) ? (int)__ldg(chunk_cnt + c) : 0;
+        cnt_next = (c + nwarp < nchunk) ? (int)__ldg(chunk_cnt + c + nwarp) : 0;
+        if (c < nchunk) fetch_keys(c, cnt, k);
+    }
+    __device__ __forceinline__ bool valid() const { return c < nchunk; }
+    // issue the loads for the chunks ahead; call before working on chunk c
+    __device__ __forceinline__ int prefetch()
+    {
+        const int cnt_after = (c + 2 * nwarp < nchunk) ? (int)__ldg(chunk_cnt + c + 2 * nwarp) : 0;
+        if (c + nwarp < nchunk) fetch_keys(c + nwarp, cnt_next, k_next);
+        return cnt_after;
+    }
+    __device__ __forceinline__ void advance(int cnt_after)
+    {
+        c += nwarp; cnt = cnt_next; cnt_next = cnt_after;
+#pragma unroll
+        for (int q = 0; q < CB; ++q) k[q] = k_next[q];
+    }
+};
+
+// Radix-select rounds 2 and 3 on the candidates.
 template <int PASS>
 __global__ void __launch_bounds__(SG_T)
 cand_hist_kernel(const uint32_t* __restrict__ seg_key, const uint32_t* __restrict__ chunk_cnt, int64_t nchunk,
@@ -472,16 +615,19 @@ cand_hist_kernel(const uint32_t* __restrict__ seg_key, const uint32_t* __restric
     for (int i = threadIdx.x; i < 2048; i += SG_T) s_h[i] = 0;
     __syncthreads();
     const uint32_t prefix = state->prefix;
-    const int lane = threadIdx.x & 31;
-    const int64_t nwarp = (int64_t)gridDim.x * (SG_T / 32);
-    for (int64_t c = (int64_t)blockIdx.x * (SG_T / 32) + (threadIdx.x >> 5); c < nchunk; c += nwarp) {
-        const int cnt = (int)chunk_cnt[c];
-        const uint32_t* seg = seg_key + c * SG_CH;
-        for (int j = lane; j < cnt; j += 32) {
-            const uint32_t key = seg[j];
-            if (PASS == 1) { if ((key >> 21) == prefix) atomicAdd(&s_h[(key >> 10) & 0x7FFu], 1u); }
-            else { if ((key >> 10) == prefix) atomicAdd(&s_h[key & 0x3FFu], 1u); }
-        }
+    auto add = [&](uint32_t key) {
+        if (PASS == 1) { if ((key >> 21) == prefix) atomicAdd(&s_h[(key >> 10) & 0x7FFu], 1u); }
+        else { if ((key >> 10) == prefix) atomicAdd(&s_h[key & 0x3FFu], 1u); }
+    };
+    SegCursor cur;
+    for (cur.start(seg_key, chunk_cnt, nchunk); cur.valid();) {
+        const int after = cur.prefetch();
+#pragma unroll
+        for (int q = 0; q < CB; ++q)
+            if (q * 32 + cur.lane < cur.cnt) add(cur.k[q]);
+        const uint32_t* seg = seg_key + cur.c * SG_CH;
+        for (int j = CB * 32 + cur.lane; j < cur.cnt; j += 32) add(seg[j]);       // segments longer than a batch
+        cur.advance(after);
     }
     __syncthreads();
     for (int i = threadIdx.x; i < 2048; i += SG_T)
@@ -494,83 +640,102 @@ cand_count_kernel(const uint32_t* __restrict__ seg_key, const uint32_t* __restri
 {
     if (gate.closed()) return;
     const uint32_t T = state->prefix;
-    const int lane = threadIdx.x & 31;
-    const int64_t nwarp = (int64_t)gridDim.x * (SG_T / 32);
-    for (int64_t c = (int64_t)blockIdx.x * (SG_T / 32) + (threadIdx.x >> 5); c < nchunk; c += nwarp) {
-        const int cnt = (int)chunk_cnt[c];
-        const uint32_t* seg = seg_key + c * SG_CH;
+    SegCursor cur;
+    for (cur.start(seg_key, chunk_cnt, nchunk); cur.valid();) {
+        const int after = cur.prefetch();
         int gt = 0, eq = 0;
-        for (int j = lane; j < cnt; j += 32) {
-            const uint32_t key = seg[j];
-            gt += (key > T); eq += (key == T);
-        }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) { gt += __shfl_xor_sync(0xFFFFFFFFu, gt, o); eq += __shfl_xor_sync(0xFFFFFFFFu, eq, o); }
-        if (lane == 0) { blk_cnt[2 * c] = gt; blk_cnt[2 * c + 1] = eq; }
+        for (int q = 0; q < CB; ++q)
+            if (q * 32 + cur.lane < cur.cnt) { gt += (cur.k[q] > T); eq += (cur.k[q] == T); }
+        const uint32_t* seg = seg_key + cur.c * SG_CH;
+        for (int j = CB * 32 + cur.lane; j < cur.cnt; j += 32) { const uint32_t key = seg[j]; gt += (key > T); eq += (key == T); }
+        gt = __reduce_add_sync(0xFFFFFFFFu, gt);
+        eq = __reduce_add_sync(0xFFFFFFFFu, eq);
+        if (cur.lane == 0) *reinterpret_cast<int2*>(blk_cnt + 2 * cur.c) = make_int2(gt, eq);
+        cur.advance(after);
     }
 }
 
 // Final write: a warp per chunk marks the offsets of {key > T} and of {key == T} in two 4096-bit maps
-// in shared memory, which puts the segment's unordered candidates back in index order; each lane then
-// walks its 128 bits, and the running counts (block offsets + warp scan) give every index its place.
+// in shared memory, which puts the segment's unordered candidates back in index order: the number of
+// set bits below a candidate's offset (a per-word prefix plus a masked population count) is how many
+// of the chunk's larger or equal-key scores come before it, and with the chunk's offsets that is its
+// place in the output.
 __global__ void __launch_bounds__(SG_T)
 cand_write_kernel(const uint32_t* __restrict__ seg_key, const uint16_t* __restrict__ seg_off,
                   const uint32_t* __restrict__ chunk_cnt, int64_t nchunk, const SelectState* __restrict__ state,
                   const int64_t* __restrict__ blk_off, int64_t* __restrict__ indices, Gate gate)
 {
     __shared__ __align__(16) uint32_t s_bm[SG_T / 32][2][SG_CH / 32];
+    __shared__ __align__(16) uint16_t s_pre[SG_T / 32][2][SG_CH / 32];      // set bits in the words before
     if (gate.closed()) return;
     const uint32_t T = state->prefix;
     const int64_t k_ties = state->k_rem;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t* bm_gt = s_bm[warp][0];
     uint32_t* bm_eq = s_bm[warp][1];
-    const int64_t nwarp = (int64_t)gridDim.x * (SG_T / 32);
-    for (int64_t c = (int64_t)blockIdx.x * (SG_T / 32) + warp; c < nchunk; c += nwarp) {
-        const int cnt = (int)chunk_cnt[c];
-        if (cnt == 0) continue;
+    uint16_t* pre_gt = s_pre[warp][0];
+    uint16_t* pre_eq = s_pre[warp][1];
+    SegCursor cur;
+    for (cur.start(seg_key, chunk_cnt, nchunk); cur.valid();) {
+        const int after = cur.prefetch();
+        const int64_t c = cur.c;
+        const int cnt = cur.cnt;
+        if (cnt == 0) { cur.advance(after); continue; }
         const uint32_t* seg = seg_key + c * SG_CH;
         const uint16_t* off = seg_off + c * SG_CH;
+        const longlong2 base2 = *reinterpret_cast<const longlong2*>(blk_off + 2 * c);
+        // offsets of the first batch, for the entries that are selected or tied (all loads issued together)
+        uint32_t o[CB];
+#pragma unroll
+        for (int q = 0; q < CB; ++q) {
+            const int j = q * 32 + lane;
+            o[q] = (j < cnt && cur.k[q] >= T) ? (uint32_t)off[j] : 0xFFFFFFFFu;
+        }
         reinterpret_cast<uint4*>(bm_gt)[lane] = make_uint4(0u, 0u, 0u, 0u);
         reinterpret_cast<uint4*>(bm_eq)[lane] = make_uint4(0u, 0u, 0u, 0u);
         __syncwarp();
-        for (int j = lane; j < cnt; j += 32) {
+#pragma unroll
+        for (int q = 0; q < CB; ++q)
+            if (o[q] != 0xFFFFFFFFu) atomicOr((cur.k[q] > T ? bm_gt : bm_eq) + (o[q] >> 5), 1u << (o[q] & 31u));
+        for (int j = CB * 32 + lane; j < cnt; j += 32) {                 // segments longer than a batch
             const uint32_t key = seg[j];
-            if (key >= T) {
-                const uint32_t o = off[j];
-                atomicOr((key > T ? bm_gt : bm_eq) + (o >> 5), 1u << (o & 31u));
-            }
+            if (key >= T) { const uint32_t oo = off[j]; atomicOr((key > T ? bm_gt : bm_eq) + (oo >> 5), 1u << (oo & 31u)); }
         }
         __syncwarp();
         const uint4 g4 = reinterpret_cast<const uint4*>(bm_gt)[lane];
         const uint4 e4 = reinterpret_cast<const uint4*>(bm_eq)[lane];
-        const uint32_t g[4] = {g4.x, g4.y, g4.z, g4.w}, e[4] = {e4.x, e4.y, e4.z, e4.w};
-        const int cg = __popc(g[0]) + __popc(g[1]) + __popc(g[2]) + __popc(g[3]);
-        const int ce = __popc(e[0]) + __popc(e[1]) + __popc(e[2]) + __popc(e[3]);
+        const int pg[4] = {__popc(g4.x), __popc(g4.y), __popc(g4.z), __popc(g4.w)};
+        const int pe[4] = {__popc(e4.x), __popc(e4.y), __popc(e4.z), __popc(e4.w)};
+        const int cg = pg[0] + pg[1] + pg[2] + pg[3], ce = pe[0] + pe[1] + pe[2] + pe[3];
         int ig = cg, ie = ce;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int a = __shfl_up_sync(0xFFFFFFFFu, ig, o), b2 = __shfl_up_sync(0xFFFFFFFFu, ie, o);
-            if (lane >= o) { ig += a; ie += b2; }
+        for (int sh = 1; sh < 32; sh <<= 1) {
+            const int a2 = __shfl_up_sync(0xFFFFFFFFu, ig, sh), b2 = __shfl_up_sync(0xFFFFFFFFu, ie, sh);
+            if (lane >= sh) { ig += a2; ie += b2; }
         }
-        int64_t gt_before = blk_off[2 * c] + (ig - cg), eq_before = blk_off[2 * c + 1] + (ie - ce);
+        ig -= cg; ie -= ce;
+        reinterpret_cast<uint2*>(pre_gt)[lane] = make_uint2((uint32_t)ig | ((uint32_t)(ig + pg[0]) << 16),
+                                                            (uint32_t)(ig + pg[0] + pg[1]) | ((uint32_t)(ig + pg[0] + pg[1] + pg[2]) << 16));
+        reinterpret_cast<uint2*>(pre_eq)[lane] = make_uint2((uint32_t)ie | ((uint32_t)(ie + pe[0]) << 16),
+                                                            (uint32_t)(ie + pe[0] + pe[1]) | ((uint32_t)(ie + pe[0] + pe[1] + pe[2]) << 16));
+        __syncwarp();
+        auto place = [&](uint32_t key, uint32_t oo) {
+            const uint32_t w = oo >> 5, below = (1u << (oo & 31u)) - 1u;
+            const int64_t gt_before = base2.x + pre_gt[w] + __popc(bm_gt[w] & below);
+            const int64_t eq_before = base2.y + pre_eq[w] + __popc(bm_eq[w] & below);
+            if (key > T) indices[gt_before + (eq_before < k_ties ? eq_before : k_ties)] = c * SG_CH + oo;
+            else if (eq_before < k_ties) indices[gt_before + eq_before] = c * SG_CH + oo;
+        };
 #pragma unroll
-        for (int w = 0; w < 4; ++w) {
-            uint32_t m = g[w] | e[w];
-            const int64_t ibase = c * SG_CH + (lane * 4 + w) * 32;
-            while (m) {
-                const int b = __ffs((int)m) - 1;
-                m &= m - 1u;
-                if ((g[w] >> b) & 1u) {
-                    indices[gt_before + (eq_before < k_ties ? eq_before : k_ties)] = ibase + b;
-                    ++gt_before;
-                } else {
-                    if (eq_before < k_ties) indices[gt_before + eq_before] = ibase + b;
-                    ++eq_before;
-                }
-            }
+        for (int q = 0; q < CB; ++q)
+            if (o[q] != 0xFFFFFFFFu) place(cur.k[q], o[q]);
+        for (int j = CB * 32 + lane; j < cnt; j += 32) {
+            const uint32_t key = seg[j];
+            if (key >= T) place(key, off[j]);
         }
         __syncwarp();       // the maps are cleared again for the warp's next chunk
+        cur.advance(after);
     }
 }
 
@@ -603,6 +768,8 @@ BracketWs carve_bracket(void* ws, int64_t N)
     const int64_t nblk = sel_nblk(N), nchunk = sg_nchunk(N);
     w.blk_off = reinterpret_cast<int64_t*>(p); p += align_up((size_t)nblk * 2 * sizeof(int64_t), 256);
     w.blk_cnt = reinterpret_cast<int32_t*>(p); p += align_up((size_t)nblk * 2 * sizeof(int32_t), 256);
+    w.tile_tot = reinterpret_cast<int64_t*>(p); p += align_up((size_t)((nblk + 1023) / 1024) * 2 * sizeof(int64_t), 256);
+    w.sample_key = reinterpret_cast<uint32_t*>(p); p += SG_SAMPLE * sizeof(uint32_t);
     w.chunk_cnt = reinterpret_cast<uint32_t*>(p); p += align_up((size_t)nchunk * sizeof(uint32_t), 256);
     w.seg_off = reinterpret_cast<uint16_t*>(p); p += align_up((size_t)nchunk * SG_CH * sizeof(uint16_t), 256);
     w.seg_key = reinterpret_cast<uint32_t*>(p);
@@ -613,13 +780,14 @@ size_t bracket_workspace_bytes(int64_t N)
 {
     const int64_t nblk = sel_nblk(N), nchunk = sg_nchunk(N);
     return 6 * 2048 * sizeof(uint32_t) + 256 + align_up((size_t)nblk * 2 * sizeof(int64_t), 256) +
-           align_up((size_t)nblk * 2 * sizeof(int32_t), 256) + align_up((size_t)nchunk * sizeof(uint32_t), 256) +
+           align_up((size_t)nblk * 2 * sizeof(int32_t), 256) + align_up((size_t)((nblk + 1023) / 1024) * 2 * sizeof(int64_t), 256) +
+           SG_SAMPLE * sizeof(uint32_t) + align_up((size_t)nchunk * sizeof(uint32_t), 256) +
            align_up((size_t)nchunk * SG_CH * sizeof(uint16_t), 256) + (size_t)nchunk * SG_CH * sizeof(uint32_t);
 }
 
 // The exact multi-pass path on the scores themselves (five reads). hist: three cleared histograms.
 cudaError_t launch_multipass(const float* scores, int64_t N, int64_t k, int64_t* indices, uint32_t* hist,
-                             SelectState* state, int32_t* blk_cnt, int64_t* blk_off, Gate gate, cudaStream_t st)
+                             SelectState* state, int32_t* blk_cnt, int64_t* blk_off, int64_t* tile_tot, Gate gate, cudaStream_t st)
 {
     int64_t hb = (N / 4 + SEL_T - 1) / SEL_T;
     const int64_t cap = (int64_t)sm_count() * 8;
@@ -635,9 +803,9 @@ cudaError_t launch_multipass(const float* scores, int64_t N, int64_t k, int64_t*
     const int64_t cap2 = (int64_t)sm_count() * 32;
     const unsigned cg = (unsigned)(nblk < cap2 ? nblk : cap2);
     select_count_kernel<<<cg, SEL_T, 0, st>>>(scores, N, nblk, state, blk_cnt, gate);
-    select_block_scan_kernel<<<1, 1024, 0, st>>>(blk_cnt, nblk, blk_off, gate);
+    launch_block_scan(blk_cnt, nblk, blk_off, tile_tot, gate, st);
     select_write_kernel<<<cg, SEL_T, 0, st>>>(scores, N, nblk, state, blk_off, indices, gate);
-    count_launches(9);
+    count_launches(8);
     return cudaGetLastError();
 }
 
@@ -647,16 +815,12 @@ cudaError_t launch_bracketed(const float* scores, int64_t N, int64_t k, int64_t*
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(select_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        SG_SAMPLE * (int)sizeof(uint32_t));
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(select_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        attr_err = cudaFuncSetAttribute(select_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             (SG_T / 32) * SG_RING * SG_STEP * (int)sizeof(uint32_t));
     });
     if (attr_err != cudaSuccess) return attr_err;
     BracketWs w = carve_bracket(ws, N);
-    cudaError_t e = cudaMemsetAsync(w.hist, 0, 6 * 2048 * sizeof(uint32_t) + 256, st);
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
     const int64_t nchunk = sg_nchunk(N);
     const int64_t cap = (int64_t)sm_count() * 8;
     const int64_t gcap = (int64_t)sm_count() * 4;          // the gather kernel's resident blocks (48 KiB ring each)
@@ -667,7 +831,8 @@ cudaError_t launch_bracketed(const float* scores, int64_t N, int64_t k, int64_t*
     const Gate none{nullptr, 0u};
     const Gate ok{&w.bstate->fallback, 0u};          // enough candidates: select among them
     const Gate fb{&w.bstate->fallback, 1u};          // too few: exact path on the scores
-    select_sample_kernel<<<1, 1024, SG_SAMPLE * sizeof(uint32_t), st>>>(scores, N, k, w.bstate, force_short ? 1 : 0);
+    select_init_kernel<<<SG_SAMPLE / 256, 256, 0, st>>>(scores, N, w.hist, 6 * 2048 + 64, w.sample_key);     // histograms + state
+    select_sample_kernel<<<1, 1024, 0, st>>>(w.sample_key, N, k, w.bstate, force_short ? 1 : 0);
     select_gather_kernel<<<gb, SG_T, (SG_T / 32) * SG_RING * SG_STEP * sizeof(uint32_t), st>>>(scores, N, w.bstate, w.seg_key, w.seg_off, w.chunk_cnt, w.hist);
     select_scan_kernel<0><<<1, 1024, 0, st>>>(w.hist, w.state, k, none, &w.bstate->fallback);
     cand_hist_kernel<1><<<cb, SG_T, 0, st>>>(w.seg_key, w.chunk_cnt, nchunk, w.state, w.hist + 2048, ok);
@@ -675,12 +840,12 @@ cudaError_t launch_bracketed(const float* scores, int64_t N, int64_t k, int64_t*
     cand_hist_kernel<2><<<cb, SG_T, 0, st>>>(w.seg_key, w.chunk_cnt, nchunk, w.state, w.hist + 4096, ok);
     select_scan_kernel<2><<<1, 1024, 0, st>>>(w.hist + 4096, w.state, k, ok, nullptr);
     cand_count_kernel<<<cb, SG_T, 0, st>>>(w.seg_key, w.chunk_cnt, nchunk, w.state, w.blk_cnt, ok);
-    select_block_scan_kernel<<<1, 1024, 0, st>>>(w.blk_cnt, nchunk, w.blk_off, ok);
+    launch_block_scan(w.blk_cnt, nchunk, w.blk_off, w.tile_tot, ok, st);
     cand_write_kernel<<<cb, SG_T, 0, st>>>(w.seg_key, w.seg_off, w.chunk_cnt, nchunk, w.state, w.blk_off, indices, ok);
-    count_launches(10);
+    count_launches(10);          // the prefix-sum launches count themselves
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    return launch_multipass(scores, N, k, indices, w.hist + 3 * 2048, w.state, w.blk_cnt, w.blk_off, fb, st);
+    return launch_multipass(scores, N, k, indices, w.hist + 3 * 2048, w.state, w.blk_cnt, w.blk_off, w.tile_tot, fb, st);
 }
 
 int g_select_path = 0;     // 0: by size; 1: multi-pass always; 2: bracketed with a bracket that is too high
@@ -705,7 +870,7 @@ cudaError_t launch_select_topk(const float* scores, int64_t N, int64_t k, int64_
     SelectWs w = carve(ws, N);
     cudaError_t e = cudaMemsetAsync(w.hist, 0, 3 * 2048 * sizeof(uint32_t), st);
     if (e != cudaSuccess) return e;
-    return launch_multipass(scores, N, k, indices, w.hist, w.state, w.blk_cnt, w.blk_off, Gate{nullptr, 0u}, st);
+    return launch_multipass(scores, N, k, indices, w.hist, w.state, w.blk_cnt, w.blk_off, nullptr, Gate{nullptr, 0u}, st);
 }
 
 }  // namespace qless
