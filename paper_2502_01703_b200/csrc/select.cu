@@ -612,7 +612,7 @@ cand_hist_kernel(const uint32_t* __restrict__ seg_key, const uint32_t* __restric
 {
     __shared__ uint32_t s_h[2048];
     if (gate.closed()) return;
-    for (int i = threadIdx.x; i < 2048; i += SG_T) s_h[i] = 0;
+    for (int i = threadIdx.x; i < 2048; i += blockDim.x) s_h[i] = 0;
     __syncthreads();
     const uint32_t prefix = state->prefix;
     auto add = [&](uint32_t key) {
@@ -630,7 +630,7 @@ cand_hist_kernel(const uint32_t* __restrict__ seg_key, const uint32_t* __restric
         cur.advance(after);
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < 2048; i += SG_T)
+    for (int i = threadIdx.x; i < 2048; i += blockDim.x)
         if (s_h[i]) atomicAdd(&hist[i], s_h[i]);
 }
 
@@ -720,12 +720,16 @@ cand_write_kernel(const uint32_t* __restrict__ seg_key, const uint16_t* __restri
         reinterpret_cast<uint2*>(pre_eq)[lane] = make_uint2((uint32_t)ie | ((uint32_t)(ie + pe[0]) << 16),
                                                             (uint32_t)(ie + pe[0] + pe[1]) | ((uint32_t)(ie + pe[0] + pe[1] + pe[2]) << 16));
         __syncwarp();
+        // place = (larger keys before) + min(ties before, k_ties): the chunk's own part of both in 32 bits
+        const int64_t room64 = k_ties - base2.y;                                  // ties this chunk may still admit
+        const uint32_t room = room64 <= 0 ? 0u : (room64 >= SG_CH ? (uint32_t)SG_CH : (uint32_t)room64);
+        int64_t* out = indices + base2.x + (base2.y < k_ties ? base2.y : k_ties);
+        const int64_t ibase = c * SG_CH;
         auto place = [&](uint32_t key, uint32_t oo) {
             const uint32_t w = oo >> 5, below = (1u << (oo & 31u)) - 1u;
-            const int64_t gt_before = base2.x + pre_gt[w] + __popc(bm_gt[w] & below);
-            const int64_t eq_before = base2.y + pre_eq[w] + __popc(bm_eq[w] & below);
-            if (key > T) indices[gt_before + (eq_before < k_ties ? eq_before : k_ties)] = c * SG_CH + oo;
-            else if (eq_before < k_ties) indices[gt_before + eq_before] = c * SG_CH + oo;
+            const uint32_t g_loc = pre_gt[w] + __popc(bm_gt[w] & below);
+            const uint32_t e_loc = pre_eq[w] + __popc(bm_eq[w] & below);
+            if (key > T || e_loc < room) out[g_loc + (e_loc < room ? e_loc : room)] = ibase + oo;
         };
 #pragma unroll
         for (int q = 0; q < CB; ++q)
