@@ -24,6 +24,11 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes of one projection launch per projected coordinate (dram__bytes_read.sum + dram__bytes_write.sum of
+# project_tc_kernel): one ncu capture at n = 256, d = 8192, P = 2^20 gave 735.3 MB + 120.2 MB; both parts grow in
+# proportion to P (the Gamma batch read, and one fp32 partial per 65 536-coordinate chunk written).
+PROJECT_TRAFFIC_BYTES_PER_P = (735.292672e6 + 120.235264e6) / 1048576.0
+PROJECT_TRAFFIC_SOURCE = "ncu capture at n=256, d=8192, P=2^20, scaled by P (profiles/project_tc_kernel__n256_P2e20_d8192.md)"
 WORKLOAD = "c2_project_quantize"
 N_VAL, TASKS, FRAC = 448, [64, 128, 256], 0.05
 SEED = 20250203
@@ -423,7 +428,7 @@ def run_ours(args):
         achieved = flops / (proj_ms / max(proj_cnt, 1) * 1e-3) / 1e12 if proj_cnt else None
         roofline = dict(bound="tensor", kernel="project", achieved=achieved, peak=peaks["bf16_sustained"],
                         unit="TFLOP/s", frac=(achieved / peaks["bf16_sustained"]) if achieved else None,
-                        traffic=None, peak_source=f"{peaks['source']} (sustained bf16; burst {peaks['bf16_burst']})",
+                        traffic=PROJECT_TRAFFIC_BYTES_PER_P * P, traffic_source=PROJECT_TRAFFIC_SOURCE, peak_source=f"{peaks['source']} (sustained bf16; burst {peaks['bf16_burst']})",
                         flops_per_launch=flops, ms_per_launch=proj_ms / max(proj_cnt, 1))
         line = dict(metric="grads projected+quantized/s (P=2^23,d=8192)", value=value, unit="grads/s",
                     n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=ms_total / args.steps,
