@@ -34,8 +34,8 @@ __device__ __forceinline__ float adam_dir(float g, float bm, float bv, const Ada
     return __fdiv_rn(m1, den);
 }
 
-// One thread handles 8 consecutive columns (16-byte bf16 accesses) of AG_ROWS consecutive rows, so the
-// moments m, v (shared by every row of the batch) are read once per AG_ROWS rows instead of once per row.
+// One thread handles 8 consecutive columns (16-byte bf16 accesses); AG_ROWS is the number of consecutive
+// rows whose loads it issues together.
 constexpr int AG_ROWS = 4;
 
 template <bool BF16_IN, bool ADAM, bool TILED>
@@ -43,68 +43,70 @@ __global__ void __launch_bounds__(256, 4)
 adam_gamma_kernel(const void* __restrict__ grads, int64_t n, int64_t ld, const float* __restrict__ m,
                   const float* __restrict__ v, AdamParams ap, int64_t P, __nv_bfloat16* __restrict__ gamma)
 {
+    // A thread owns 8 consecutive coordinates and walks down all n rows, AG_ROWS at a time: the moments of its
+    // coordinates are read from memory once per batch and stay in registers.
     const int64_t groups_per_row = P >> 3;
-    const int64_t row_groups = (n + AG_ROWS - 1) / AG_ROWS;
-    const int64_t total = row_groups * groups_per_row;
-    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-         idx += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t rg = idx / groups_per_row;
-        const int64_t j0 = (idx - rg * groups_per_row) << 3;
-        const int64_t row0 = rg * AG_ROWS;
+    for (int64_t cg = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; cg < groups_per_row;
+         cg += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t j0 = cg << 3;
         float mm[8], vv[8];
         if (ADAM) {
-            const float4 m0 = __ldg(reinterpret_cast<const float4*>(m + j0)), m1 = __ldg(reinterpret_cast<const float4*>(m + j0 + 4));
-            const float4 v0 = __ldg(reinterpret_cast<const float4*>(v + j0)), v1 = __ldg(reinterpret_cast<const float4*>(v + j0 + 4));
+            const float4 m0 = __ldcs(reinterpret_cast<const float4*>(m + j0)), m1 = __ldcs(reinterpret_cast<const float4*>(m + j0 + 4));
+            const float4 v0 = __ldcs(reinterpret_cast<const float4*>(v + j0)), v1 = __ldcs(reinterpret_cast<const float4*>(v + j0 + 4));
             mm[0] = m0.x; mm[1] = m0.y; mm[2] = m0.z; mm[3] = m0.w; mm[4] = m1.x; mm[5] = m1.y; mm[6] = m1.z; mm[7] = m1.w;
             vv[0] = v0.x; vv[1] = v0.y; vv[2] = v0.z; vv[3] = v0.w; vv[4] = v1.x; vv[5] = v1.y; vv[6] = v1.z; vv[7] = v1.w;
 #pragma unroll
             for (int k = 0; k < 8; ++k) { mm[k] = __fmul_rn(ap.beta1, mm[k]); vv[k] = __fmul_rn(ap.beta2, vv[k]); }
         }
-        // issue every row's loads before any arithmetic (memory-level parallelism)
-        uint4 raw[AG_ROWS][BF16_IN ? 1 : 2];
+        // TILED: [K block of 64 columns][row][64] so that a (256 rows x 64 columns) operand tile is one
+        // contiguous 32 KiB span; otherwise plain row-major [n, P].
+        __nv_bfloat16* out = TILED ? gamma + (((j0 >> 6) * n) << 6) + (j0 & 63) : gamma + j0;
+        const int64_t out_ld = TILED ? 64 : P;
+#pragma unroll 1
+        for (int64_t row0 = 0; row0 < n; row0 += AG_ROWS) {
+            // issue every row's loads before any arithmetic (memory-level parallelism)
+            uint4 raw[AG_ROWS][BF16_IN ? 1 : 2];
 #pragma unroll
-        for (int r = 0; r < AG_ROWS; ++r) {
-            if (row0 + r < n) {
-                if (BF16_IN) {
-                    raw[r][0] = __ldcs(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(grads) + (row0 + r) * ld + j0));
-                } else {
-                    const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(grads) + (row0 + r) * ld + j0);
-                    raw[r][0] = __ldcs(p);
-                    raw[r][BF16_IN ? 0 : 1] = __ldcs(p + 1);
+            for (int r = 0; r < AG_ROWS; ++r) {
+                if (row0 + r < n) {
+                    if (BF16_IN) {
+                        raw[r][0] = __ldcs(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(grads) + (row0 + r) * ld + j0));
+                    } else {
+                        const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(grads) + (row0 + r) * ld + j0);
+                        raw[r][0] = __ldcs(p);
+                        raw[r][BF16_IN ? 0 : 1] = __ldcs(p + 1);
+                    }
                 }
             }
-        }
 #pragma unroll
-        for (int r = 0; r < AG_ROWS; ++r) {
-            const int64_t row = row0 + r;
-            if (row >= n) break;
-            float g[8];
-            if (BF16_IN) {
-                const uint32_t w[4] = {raw[r][0].x, raw[r][0].y, raw[r][0].z, raw[r][0].w};
+            for (int r = 0; r < AG_ROWS; ++r) {
+                const int64_t row = row0 + r;
+                if (row >= n) break;
+                float g[8];
+                if (BF16_IN) {
+                    const uint32_t w[4] = {raw[r][0].x, raw[r][0].y, raw[r][0].z, raw[r][0].w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        g[2 * k] = __uint_as_float(w[k] << 16);
+                        g[2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u);
+                    }
+                } else {
+                    const uint4 a = raw[r][0], b = raw[r][BF16_IN ? 0 : 1];
+                    g[0] = __uint_as_float(a.x); g[1] = __uint_as_float(a.y); g[2] = __uint_as_float(a.z); g[3] = __uint_as_float(a.w);
+                    g[4] = __uint_as_float(b.x); g[5] = __uint_as_float(b.y); g[6] = __uint_as_float(b.z); g[7] = __uint_as_float(b.w);
+                }
+                if (ADAM) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) g[k] = adam_dir(g[k], mm[k], vv[k], ap);
+                }
+                uint32_t o[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    g[2 * k] = __uint_as_float(w[k] << 16);
-                    g[2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u);
+                    const __nv_bfloat162 pr = __floats2bfloat162_rn(g[2 * k], g[2 * k + 1]);
+                    o[k] = *reinterpret_cast<const uint32_t*>(&pr);
                 }
-            } else {
-                const uint4 a = raw[r][0], b = raw[r][BF16_IN ? 0 : 1];
-                g[0] = __uint_as_float(a.x); g[1] = __uint_as_float(a.y); g[2] = __uint_as_float(a.z); g[3] = __uint_as_float(a.w);
-                g[4] = __uint_as_float(b.x); g[5] = __uint_as_float(b.y); g[6] = __uint_as_float(b.z); g[7] = __uint_as_float(b.w);
+                *reinterpret_cast<uint4*>(out + row * out_ld) = make_uint4(o[0], o[1], o[2], o[3]);
             }
-            if (ADAM) {
-#pragma unroll
-                for (int k = 0; k < 8; ++k) g[k] = adam_dir(g[k], mm[k], vv[k], ap);
-            }
-            uint32_t o[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const __nv_bfloat162 pr = __floats2bfloat162_rn(g[2 * k], g[2 * k + 1]);
-                o[k] = *reinterpret_cast<const uint32_t*>(&pr);
-            }
-            // TILED: [K block of 64 columns][row][64] so that a (256 rows x 64 columns) operand tile is one
-            // contiguous 32 KiB span; otherwise plain row-major [n, P].
-            const int64_t dst = TILED ? (((j0 >> 6) * n + row) << 6) + (j0 & 63) : row * P + j0;
-            *reinterpret_cast<uint4*>(gamma + dst) = make_uint4(o[0], o[1], o[2], o[3]);
         }
     }
 }
@@ -114,7 +116,7 @@ cudaError_t launch_adam_gamma(const void* grads, qless_dtype dtype, int64_t n, i
                               bool tiled, cudaStream_t st)
 {
     if (n == 0 || P == 0) return cudaSuccess;
-    const int64_t total = ((n + AG_ROWS - 1) / AG_ROWS) * (P >> 3);
+    const int64_t total = P >> 3;          // a thread per group of 8 coordinates
     const int threads = 256;
     int64_t blocks = (total + threads - 1) / threads;
     const int64_t cap = (int64_t)sm_count() * 16;
