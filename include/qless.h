@@ -81,7 +81,8 @@ qless_status qless_profile_collect(char* buf /* host */, size_t buflen);
  * vendor tool has measured on the machine at hand). `what`: 0 / 1 / 2 = back-to-back tcgen05.mma on every SM
  * with operands resident on chip: bf16 with both operands in shared memory / bf16 with A in tensor memory /
  * int8; 3 / 4 / 5 = the same three on CTA pairs (cta_group::2); 6 = the XOR + POPC + IADD mix of 1-bit
- * scoring on the integer pipes (scratch: device buffer of >= 8 KiB per SM). Runs the kernel twice and times
+ * scoring on the integer pipes (scratch: device buffer of >= 8 KiB per SM); 7 = int8 on CTA pairs with A in
+ * tensor memory. Runs the kernel twice and times
  * the second run with CUDA events on `cuda_stream` (synchronises it). *ms_out: milliseconds; *ops_out:
  * operations executed (2 x multiply-accumulates, or word operations for 6). Host pointers. */
 qless_status qless_microbench(int32_t what, int32_t iters, float* ms_out, double* ops_out, void* scratch,

@@ -14,7 +14,8 @@ using namespace tc;
 
 struct __align__(8) MbBars { uint64_t done; uint32_t tmem_base; uint32_t abort_flag; };
 
-// KIND: 0 = bf16 A,B in shared memory; 1 = bf16 A in tensor memory; 2 = int8 A,B in shared memory.
+// KIND: 0 = bf16 A,B in shared memory; 1 = bf16 A in tensor memory; 2 = int8 A,B in shared memory;
+//       3 = int8 A in tensor memory.
 // PAIR: 0 = one CTA per 128 x 256 tile; 1 = CTA pair per 256 x 256 tile (cta_group::2).
 template <int KIND, int PAIR>
 __global__ void __launch_bounds__(128, 1)
@@ -31,7 +32,7 @@ mma_peak_kernel(int iters, unsigned int* timeout_word)
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
 
     for (int i = threadIdx.x; i < (A_BYTES + B_BYTES) / 4; i += blockDim.x)
-        reinterpret_cast<uint32_t*>(smem)[i] = (KIND == 2) ? (0x01FF02FEu ^ (uint32_t)(i * 0x01010101u & 0x03030303u))
+        reinterpret_cast<uint32_t*>(smem)[i] = (KIND >= 2) ? (0x01FF02FEu ^ (uint32_t)(i * 0x01010101u & 0x03030303u))
                                                             : ((i & 1) ? 0x3F80BF80u : 0xBF803F80u);
     if (threadIdx.x == 0) { mbar_init(smem_u32(&bars->done), 1); bars->abort_flag = 0; fence_barrier_init(); }
     if (warp == 0) {
@@ -44,13 +45,14 @@ mma_peak_kernel(int iters, unsigned int* timeout_word)
     if (PAIR) cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
-    if (KIND == 1) {                                        // A operand: 64 columns of +-1.0 pairs in every lane
+    if (KIND == 1 || KIND == 3) {                           // A operand: 64 columns (bf16 +-1.0 pairs, or small int8) in every lane
         const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + 256;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             uint32_t v[16];
 #pragma unroll
-            for (int k = 0; k < 16; ++k) v[k] = ((lane + k) & 1) ? 0x3F80BF80u : 0xBF803F80u;
+            for (int k = 0; k < 16; ++k) v[k] = (KIND == 3) ? (0x01FF02FEu ^ (uint32_t)((lane + k) & 3) * 0x01010101u)
+                                                            : (((lane + k) & 1) ? 0x3F80BF80u : 0xBF803F80u);
             tmem_st_x16(taddr + c * 16, v);
         }
         tmem_wait_st();
@@ -62,7 +64,7 @@ mma_peak_kernel(int iters, unsigned int* timeout_word)
 
     if (threadIdx.x == 0 && rank == 0) {
         constexpr uint32_t M = PAIR ? 256 : 128;
-        const uint32_t idesc = (KIND == 2) ? make_idesc(2, 1, 1, M, 256) : make_idesc(1, 1, 1, M, 256);
+        const uint32_t idesc = (KIND >= 2) ? make_idesc(2, 1, 1, M, 256) : make_idesc(1, 1, 1, M, 256);
         const uint64_t adesc = make_smem_desc_sw128(smem_u32(sA));
         const uint64_t bdesc = make_smem_desc_sw128(smem_u32(sB));
         for (int it = 0; it < iters; ++it) {
@@ -77,6 +79,8 @@ mma_peak_kernel(int iters, unsigned int* timeout_word)
                 } else if (KIND == 1) {
                     if (PAIR) mma_f16_ts_pair(tmem_base, tmem_base + 256 + 8 * k, bdesc + (uint64_t)(2 * k), idesc, acc);
                     else mma_f16_ts(tmem_base, tmem_base + 256 + 8 * k, bdesc + (uint64_t)(2 * k), idesc, acc);
+                } else if (KIND == 3) {
+                    if (PAIR) mma_i8_ts_pair(tmem_base, tmem_base + 256 + 8 * k, bdesc + (uint64_t)(2 * k), idesc, acc);
                 } else {
                     if (PAIR) mma_i8_ss_pair(tmem_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, acc);
                     else mma_i8_ss(tmem_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, acc);
@@ -158,7 +162,7 @@ extern "C" qless_status qless_microbench(int32_t what, int32_t iters, float* ms_
             if (what == 0) { QLESS_MB_LAUNCH(0) } else if (what == 1) { QLESS_MB_LAUNCH(1) } else { QLESS_MB_LAUNCH(2) }
 #undef QLESS_MB_LAUNCH
             ops = (double)sms * iters * 4.0 * 2.0 * 128 * 256 * (what == 2 ? 32 : 16);
-        } else if (what >= 3 && what <= 5) {
+        } else if ((what >= 3 && what <= 5) || what == 7) {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3((unsigned)(sms / 2 * 2)); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = smem; cfg.stream = st;
             cudaLaunchAttribute attr; attr.id = cudaLaunchAttributeClusterDimension; attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
@@ -166,9 +170,9 @@ extern "C" qless_status qless_microbench(int32_t what, int32_t iters, float* ms_
 #define QLESS_MB_LAUNCH(K)                                                                                           \
             err = cudaFuncSetAttribute(mma_peak_kernel<K, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
             if (err == cudaSuccess) err = cudaLaunchKernelEx(&cfg, mma_peak_kernel<K, 1>, (int)iters, flag);
-            if (what == 3) { QLESS_MB_LAUNCH(0) } else if (what == 4) { QLESS_MB_LAUNCH(1) } else { QLESS_MB_LAUNCH(2) }
+            if (what == 3) { QLESS_MB_LAUNCH(0) } else if (what == 4) { QLESS_MB_LAUNCH(1) } else if (what == 5) { QLESS_MB_LAUNCH(2) } else { QLESS_MB_LAUNCH(3) }
 #undef QLESS_MB_LAUNCH
-            ops = (double)(sms / 2) * iters * 4.0 * 2.0 * 256 * 256 * (what == 5 ? 32 : 16);
+            ops = (double)(sms / 2) * iters * 4.0 * 2.0 * 256 * 256 * (what == 5 || what == 7 ? 32 : 16);
         } else if (what == 6) {
             const size_t need = (size_t)sms * 8 * 256 * sizeof(uint32_t);
             QLESS_REQUIRE(scratch != nullptr && scratch_bytes >= need, QLESS_ERR_WORKSPACE, "scratch of %zu bytes required", need);

@@ -82,6 +82,13 @@ __device__ __forceinline__ void unpack2(uint32_t w, uint32_t (&o)[4])
     for (int f = 0; f < 4; ++f) o[f] = __vsub4(((w >> (2 * f)) & 0x03030303u) ^ 0x02020202u, 0x02020202u);
 }
 
+// Position in a ring of n slots: slot index and the parity of its current use. Advanced by comparison, not by
+// division: the role loops below run on single threads whose every instruction is on the critical path.
+struct Ring {
+    uint32_t slot = 0, parity = 0;
+    __device__ __forceinline__ void next(uint32_t n) { if (++slot == n) { slot = 0; parity ^= 1u; } }
+};
+
 template <int BITS>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_constant__ CUtensorMap tmap_val1,
@@ -144,34 +151,36 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
             // Packed train codes run ahead of the operand stages in their own ring: the load for iteration q is
             // issued as soon as ring slot q % nP is free, not when operand stage q % nS is.
             int64_t pq = 0;                     // next packed load to issue
-            // blocking = false: issue only if the ring slot is already free (returns false otherwise)
-            auto issue_packed = [&](int64_t q, bool blocking) -> bool {
-                const int sp = (int)(q % p.nP);
-                const uint32_t par = (uint32_t)((q / p.nP) & 1) ^ 1u;
-                if (blocking) { if (!mbar_wait(smem_u32(&bars->p_empty[sp]), par, abort_flag, p.timeout_word, TO_PRODUCER)) return false; }
-                else if (!mbar_try_wait(smem_u32(&bars->p_empty[sp]), par)) return false;
-                const int kb = (int)(q % nkb);
-                const int i = (int)((q / nkb) % p.C);
-                const int64_t tile = pair + (q / ((int64_t)nkb * p.C * num_vt)) * num_pairs;
+            Ring pring;                         // its ring slot
+            int p_kb = 0, p_i = 0, p_vt = 0;    // and its K block, checkpoint, validation tile and train tile
+            int64_t p_tile = pair;
+            // blocking = false: issue only if the ring slot is already free (one look at the barrier, no suspension)
+            auto issue_packed = [&](bool blocking) -> bool {
+                const uint32_t sp = pring.slot;
+                if (blocking) { if (!mbar_wait(smem_u32(&bars->p_empty[sp]), pring.parity ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) return false; }
+                else if (!mbar_test_wait(smem_u32(&bars->p_empty[sp]), pring.parity ^ 1u)) return false;
                 const uint32_t pfull = smem_u32(&bars->p_full[sp]);
                 mbar_arrive_expect_tx(pfull, P_STAGE);
-                tma_load_3d(smem_u32(sP + (size_t)sp * P_STAGE), &tmap_train, pfull, kb * 16 * BITS, (int32_t)(tile * 2 * TM + rank * TM), i);
+                tma_load_3d(smem_u32(sP + (size_t)sp * P_STAGE), &tmap_train, pfull, p_kb * 16 * BITS, (int32_t)(p_tile * 2 * TM + rank * TM), p_i);
+                ++pq; pring.next((uint32_t)p.nP);
+                if (++p_kb == nkb) { p_kb = 0; if (++p_i == p.C) { p_i = 0; if (++p_vt == num_vt) { p_vt = 0; p_tile += num_pairs; } } }
                 return true;
             };
+            Ring st_ring;
 
             for (int64_t tile = pair; tile < num_tiles && ok; tile += num_pairs) {
                 const int32_t row0 = (int32_t)(tile * 2 * TM + rank * TM);
                 for (int vt = 0; vt < num_vt && ok; ++vt)
                     for (int i = 0; i < p.C && ok; ++i)
-                        for (int kb = 0; kb < nkb; ++kb, ++it) {
+                        for (int kb = 0; kb < nkb; ++kb, ++it, st_ring.next((uint32_t)p.nS)) {
                             if (BITS != 8) {
                                 // the packed codes of this iteration must be on their way; those of the next few if a slot is free
-                                while (pq <= (int64_t)it && ok) { ok = issue_packed(pq, true); ++pq; }
+                                while (pq <= (int64_t)it && ok) ok = issue_packed(true);
                                 if (!ok) break;
-                                while (pq < total && pq < (int64_t)it + p.nP && issue_packed(pq, false)) ++pq;
+                                while (pq < total && pq < (int64_t)it + p.nP && issue_packed(false)) {}
                             }
-                            const int s = it % p.nS;
-                            if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), ((it / p.nS) & 1u) ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) { ok = false; break; }
+                            const int s = (int)st_ring.slot;
+                            if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), st_ring.parity ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) { ok = false; break; }
                             const uint32_t full = map_to_cta(smem_u32(&bars->full[s]), 0);
                             if (rank == 0) mbar_arrive_expect_tx(smem_u32(&bars->full[s]), tx_total);
                             uint8_t* st = sS + (size_t)s * stage_bytes;
@@ -187,14 +196,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
         // ------------------------------- MMA issuer (leader CTA) -------------------------------
         if (lane == 0 && rank == 0) {
             uint32_t it = 0, n_acc = 0;
+            Ring st_ring;
             bool ok = true;
             for (int64_t tile = pair; tile < num_tiles && ok; tile += num_pairs)
                 for (int vt = 0; vt < num_vt && ok; ++vt)
                     for (int i = 0; i < p.C && ok; ++i, ++n_acc) {
                         if (!mbar_wait_cluster(smem_u32(&bars->d_empty), (n_acc & 1u) ^ 1u, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
-                        for (int kb = 0; kb < nkb; ++kb, ++it) {
-                            const int s = it % p.nS;
-                            if (!mbar_wait_cluster(smem_u32(&bars->full[s]), (it / p.nS) & 1u, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
+                        for (int kb = 0; kb < nkb; ++kb, ++it, st_ring.next((uint32_t)p.nS)) {
+                            const int s = (int)st_ring.slot;
+                            if (!mbar_wait_cluster(smem_u32(&bars->full[s]), st_ring.parity, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
                             tc_fence_after();
                             const uint32_t st = smem_u32(sS + (size_t)s * stage_bytes);
                             const uint64_t adesc = make_smem_desc_sw128(st);
@@ -228,10 +238,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
             bool ok = true;
             const int64_t my_tiles = (num_tiles > pair) ? (num_tiles - pair + num_pairs - 1) / num_pairs : 0;
             const int64_t total = my_tiles * num_vt * p.C * nkb;
-            for (int64_t q = 0; q < total && ok; ++q, ++it) {
+            Ring st_ring, lag_ring, pring;              // operand stage of K block it, of K block it - 2, packed slot
+            for (int64_t q = 0; q < total && ok; ++q, ++it, st_ring.next((uint32_t)p.nS), pring.next((uint32_t)p.nP)) {
+                if (it >= 3) lag_ring.next((uint32_t)p.nS);      // lag_ring = position of K block it - 2
                 if ((it & 1u) != grp) continue;
-                const int sp = it % p.nP, s = it % p.nS;
-                ok = mbar_wait(smem_u32(&bars->p_full[sp]), (it / p.nP) & 1u, abort_flag, p.timeout_word, TO_UNPACK);
+                const int sp = (int)pring.slot, s = (int)st_ring.slot;
+                ok = mbar_wait(smem_u32(&bars->p_full[sp]), pring.parity, abort_flag, p.timeout_word, TO_UNPACK);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 // unpack into registers first: this needs only the packed bytes, not the TMEM slot
@@ -253,12 +265,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         }
                     }
                 }
+                // the slot is refilled by TMA (async proxy) once every reader has arrived: the reads above (generic
+                // proxy, their values not yet consumed) have to be ordered before that write
+                fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bars->p_empty[sp]));      // staging slot read: the producer may refill it
                 // TMEM slot it % 2 is free once the MMAs of K block it - 2 have completed, which is what releases
                 // operand stage (it - 2) % nS (nS > 2, so that barrier cannot run a whole phase ahead of us)
                 if (it >= 2)
-                    ok = mbar_wait_cluster(smem_u32(&bars->empty[(it - 2) % p.nS]), ((it - 2) / p.nS) & 1u, abort_flag, p.timeout_word, TO_UNPACK);
+                    ok = mbar_wait_cluster(smem_u32(&bars->empty[lag_ring.slot]), lag_ring.parity, abort_flag, p.timeout_word, TO_UNPACK);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
