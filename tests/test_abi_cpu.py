@@ -104,6 +104,17 @@ def test_bad_arguments_return_statuses_before_any_launch(L):
     assert score([0, 4, 8], bits=5) == B.ERR_UNSUPPORTED
     assert score([0, 4, 8]) == B.ERR_WORKSPACE            # valid shapes, no workspace given
     assert score([0, 4, 8], V=8, d=130) == B.ERR_UNSUPPORTED
+    # test hooks that choose a kernel variant: only the documented values
+    for hook, bad in ((L.qless_set_projection_path, 2), (L.qless_set_score_path, -1), (L.qless_set_select_path, 3)):
+        assert hook(bad) == B.ERR_INVALID_ARG
+        assert hook(0) == B.QLESS_OK
+    # micro-benchmarks: unknown kind, missing outputs (checked before anything is launched)
+    ms, ops = C.c_float(0), C.c_double(0)
+    assert L.qless_microbench(0, 10, None, C.byref(ops), null, 0, null) == B.ERR_INVALID_ARG
+    assert L.qless_microbench(0, 0, C.byref(ms), C.byref(ops), null, 0, null) == B.ERR_INVALID_ARG
+    # selection without a workspace: sizes beyond the built-in scratch are refused
+    assert L.qless_select_topk_static(null, (1 << 22) + 1, 0.5, null, C.byref(k), null) == B.ERR_UNSUPPORTED
+    assert L.qless_select_topk_static(null, 10, 0.0, null, C.byref(k), null) == B.QLESS_OK and k.value == 0
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
