@@ -1,4 +1,5 @@
 // C ABI of the QLESS library: argument validation, workspace carving and kernel sequencing.
+#include <mutex>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -133,6 +134,53 @@ static PqWorkspace pq_layout(int64_t n, int64_t P, int32_t d)
     return w;
 }
 
+// Adam prologue and projection of the columns [j0, j0 + len) of a batch whose full plan is `full` (j0 and len
+// multiples of full.chunk, except that the last range may end at P): Gamma goes to its place in the K-blocked
+// buffer [P/64][n][64], the partial sums to the chunks of that range. Everything is enqueued on st.
+static qless_status project_columns(const void* grads, qless_dtype dtype, int64_t n, int64_t ld_grads, const float* adam_m,
+                                    const float* adam_v, const AdamParams& ap, const ProjectPlan& full, int64_t j0,
+                                    int64_t len, uint64_t seed, __nv_bfloat16* gamma, float* part, cudaStream_t st)
+{
+    const size_t esz = (dtype == QLESS_BF16) ? 2 : 4;
+    const void* g_slab = reinterpret_cast<const uint8_t*>(grads) + (size_t)j0 * esz;
+    __nv_bfloat16* gamma_slab = gamma + (j0 / 64) * n * 64;
+    // Pre-pass: Gamma as bf16 in the K-blocked layout the projection streams
+    { ProfileScope ps("adam_gamma", st);
+      QLESS_CUDA_TRY(launch_adam_gamma(g_slab, dtype, n, ld_grads, adam_m ? adam_m + j0 : nullptr, adam_v ? adam_v + j0 : nullptr,
+                                       ap, len, gamma_slab, true, st)); }
+    ProjectPlan pl = full;
+    pl.P = len; pl.k_base = j0;
+    pl.num_chunks = (int32_t)((len + full.chunk - 1) / full.chunk);
+    float* part_slab = part + (j0 / full.chunk) * n * (int64_t)full.d;
+    if (g_projection_path == 0 && (len / 64) * n < ((int64_t)1 << 31)) {
+        CUtensorMap tmap;
+        qless_status s = make_tmap_2d_sw128(&tmap, gamma_slab, 2, 64, (uint64_t)(len / 64) * (uint64_t)n, 128, 64, 128);
+        if (s != QLESS_OK) return s;
+        unsigned int* flag = timeout_flag_ptr();
+        QLESS_REQUIRE(flag != nullptr, QLESS_ERR_CUDA, "cannot resolve the device timeout flag");
+        ProfileScope ps("project", st);
+        QLESS_CUDA_TRY(launch_project_tc(tmap, pl, seed, part_slab, flag, st));
+    } else {
+        ProfileScope ps("project", st);
+        QLESS_CUDA_TRY(launch_project_simt(gamma_slab, pl, seed, part_slab, st));
+    }
+    return QLESS_OK;
+}
+
+// A stream of the library's own per device, for copies that run beside the caller's stream.
+static qless_status copy_stream(cudaStream_t* out)
+{
+    static std::mutex mu;
+    static cudaStream_t streams[64] = {};
+    int dev = 0;
+    QLESS_CUDA_TRY(cudaGetDevice(&dev));
+    QLESS_REQUIRE(dev >= 0 && dev < 64, QLESS_ERR_UNSUPPORTED, "device ordinal %d beyond 64", dev);
+    std::lock_guard<std::mutex> lk(mu);
+    if (streams[dev] == nullptr) QLESS_CUDA_TRY(cudaStreamCreateWithFlags(&streams[dev], cudaStreamNonBlocking));
+    *out = streams[dev];
+    return QLESS_OK;
+}
+
 }  // namespace qless
 
 using namespace qless;
@@ -240,23 +288,10 @@ qless_status qless_project_quantize(const void* grads, qless_dtype dtype, int64_
     QLESS_REQUIRE(workspace_bytes >= w.total, QLESS_ERR_WORKSPACE, "workspace too small: %zu bytes given, %zu needed", workspace_bytes, w.total);
 
     uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
-    // Pre-pass: Gamma as bf16 in the K-blocked layout the projection streams ([P/64][n][64]).
     __nv_bfloat16* gamma = reinterpret_cast<__nv_bfloat16*>(ws + w.gamma_off);
-    { ProfileScope ps("adam_gamma", st);
-      QLESS_CUDA_TRY(launch_adam_gamma(grads, dtype, n, ld_grads, adam_m, adam_v, ap, P, gamma, true, st)); }
     float* part = reinterpret_cast<float*>(ws + w.part_off);
-    if (g_projection_path == 0 && (P / 64) * n < ((int64_t)1 << 31)) {
-        CUtensorMap tmap;
-        s = make_tmap_2d_sw128(&tmap, gamma, 2, 64, (uint64_t)(P / 64) * (uint64_t)n, 128, 64, 128);
-        if (s != QLESS_OK) return s;
-        unsigned int* flag = timeout_flag_ptr();
-        QLESS_REQUIRE(flag != nullptr, QLESS_ERR_CUDA, "cannot resolve the device timeout flag");
-        ProfileScope ps("project", st);
-        QLESS_CUDA_TRY(launch_project_tc(tmap, w.plan, seed, part, flag, st));
-    } else {
-        ProfileScope ps("project", st);
-        QLESS_CUDA_TRY(launch_project_simt(gamma, w.plan, seed, part, st));
-    }
+    s = project_columns(grads, dtype, n, ld_grads, adam_m, adam_v, ap, w.plan, 0, P, seed, gamma, part, st);
+    if (s != QLESS_OK) return s;
     const float inv_sqrt_d = 1.0f / sqrtf((float)d);
     { ProfileScope ps("quantize", st);
       QLESS_CUDA_TRY(launch_quantize(part, w.plan.num_chunks, inv_sqrt_d, n, d, 1, bits, codes, scales, code_sumsq, proj_out, st)); }
@@ -294,11 +329,51 @@ qless_status qless_project_quantize_host(const void* grads_host, qless_dtype dty
     float* d_scales = reinterpret_cast<float*>(p); p += align_up((size_t)n * 4, 256);
     int32_t* d_sumsq = reinterpret_cast<int32_t*>(p); p += align_up((size_t)n * 4, 256);
     const size_t inner = workspace_bytes - (size_t)(p - reinterpret_cast<uint8_t*>(workspace));
-    QLESS_CUDA_TRY(cudaMemcpy2DAsync(d_grads, (size_t)P * esz, grads_host, (size_t)ld_grads * esz, (size_t)P * esz,
-                                     (size_t)n, cudaMemcpyHostToDevice, st));
-    qless_status s = qless_project_quantize(d_grads, dtype, n, P, adam_m, adam_v, adam, P, d, seed, bits, d_codes,
-                                            d_scales, code_sumsq_host ? d_sumsq : nullptr, nullptr, p, inner, cuda_stream);
+    // The batch crosses the host link in column slabs on a stream of the library's own; the prologue and the
+    // projection of a slab run on the caller's stream while the next slab is copied. The staging buffer holds the
+    // whole batch, so slabs never overwrite each other; the first copy waits for what the caller's stream had
+    // queued before this call (an earlier call may still be reading the buffer).
+    AdamParams ap;
+    qless_status s = make_adam(adam, &ap);
     if (s != QLESS_OK) return s;
+    QLESS_REQUIRE((adam_m == nullptr) == (adam_v == nullptr), QLESS_ERR_INVALID_ARG, "adam_m and adam_v must both be given or both be NULL");
+    QLESS_REQUIRE(P % 128 == 0 && P < ((int64_t)1 << 39), QLESS_ERR_UNSUPPORTED, "P must be a multiple of 128 below 2^39 (P=%lld)", (long long)P);
+    QLESS_REQUIRE(d >= 128 && d <= 8192 && d % 128 == 0, QLESS_ERR_UNSUPPORTED, "d must be a multiple of 128 in [128, 8192] (d=%d)", d);
+    QLESS_REQUIRE(aligned(adam_m, 16) && aligned(adam_v, 16), QLESS_ERR_INVALID_ARG, "adam_m, adam_v must be 16-byte aligned");
+    const PqWorkspace w = pq_layout(n, P, d);
+    QLESS_REQUIRE(inner >= w.total, QLESS_ERR_WORKSPACE, "internal: workspace accounting");
+    __nv_bfloat16* gamma = reinterpret_cast<__nv_bfloat16*>(p + w.gamma_off);
+    float* part = reinterpret_cast<float*>(p + w.part_off);
+    cudaStream_t cs = nullptr;
+    s = copy_stream(&cs);
+    if (s != QLESS_OK) return s;
+    // about eight slabs, each a whole number of K chunks
+    int64_t chunks_per_slab = (w.plan.num_chunks + 7) / 8;
+    if (chunks_per_slab < 1) chunks_per_slab = 1;
+    const int64_t slab = chunks_per_slab * w.plan.chunk;
+    cudaEvent_t ev_entry = nullptr, ev_slab = nullptr;
+    QLESS_CUDA_TRY(cudaEventCreateWithFlags(&ev_entry, cudaEventDisableTiming));
+    cudaError_t ce = cudaEventRecord(ev_entry, st);
+    if (ce == cudaSuccess) ce = cudaStreamWaitEvent(cs, ev_entry, 0);
+    cudaEventDestroy(ev_entry);             // released once the recorded work has completed
+    if (ce != cudaSuccess) return cuda_fail(ce, "event set-up of the host path");
+    for (int64_t j0 = 0; j0 < P; j0 += slab) {
+        const int64_t len = (P - j0 < slab) ? P - j0 : slab;
+        ce = cudaMemcpy2DAsync(reinterpret_cast<uint8_t*>(d_grads) + (size_t)j0 * esz, (size_t)P * esz,
+                               reinterpret_cast<const uint8_t*>(grads_host) + (size_t)j0 * esz, (size_t)ld_grads * esz,
+                               (size_t)len * esz, (size_t)n, cudaMemcpyHostToDevice, cs);
+        if (ce == cudaSuccess) ce = cudaEventCreateWithFlags(&ev_slab, cudaEventDisableTiming);
+        if (ce != cudaSuccess) return cuda_fail(ce, "host-to-device copy of a column slab");
+        ce = cudaEventRecord(ev_slab, cs);
+        if (ce == cudaSuccess) ce = cudaStreamWaitEvent(st, ev_slab, 0);
+        cudaEventDestroy(ev_slab);
+        if (ce != cudaSuccess) return cuda_fail(ce, "ordering a column slab before its projection");
+        s = project_columns(d_grads, dtype, n, P, adam_m, adam_v, ap, w.plan, j0, len, seed, gamma, part, st);
+        if (s != QLESS_OK) return s;
+    }
+    { ProfileScope ps("quantize", st);
+      QLESS_CUDA_TRY(launch_quantize(part, w.plan.num_chunks, 1.0f / sqrtf((float)d), n, d, 1, bits, d_codes, d_scales,
+                                     code_sumsq_host ? d_sumsq : nullptr, nullptr, st)); }
     QLESS_CUDA_TRY(cudaMemcpyAsync(codes_host, d_codes, (size_t)n * (size_t)d * bits / 8, cudaMemcpyDeviceToHost, st));
     QLESS_CUDA_TRY(cudaMemcpyAsync(scales_host, d_scales, (size_t)n * 4, cudaMemcpyDeviceToHost, st));
     if (code_sumsq_host)

@@ -12,7 +12,7 @@ constexpr int PS_T = 256;
 
 __global__ void __launch_bounds__(PS_T)
 project_simt_kernel(const __nv_bfloat16* __restrict__ gamma, int64_t n, int64_t P, int32_t d,
-                    int64_t chunk, uint64_t seed, float* __restrict__ part)
+                    int64_t chunk, uint32_t kblk_base, uint64_t seed, float* __restrict__ part)
 {
     __shared__ __align__(16) float s_g[PS_GR][128];
     const int tid = threadIdx.x;
@@ -41,7 +41,7 @@ project_simt_kernel(const __nv_bfloat16* __restrict__ gamma, int64_t n, int64_t 
         }
         __syncthreads();
         uint32_t w[4];
-        rademacher_block(seed, r, (uint32_t)(kb >> 7), w);
+        rademacher_block(seed, r, kblk_base + (uint32_t)(kb >> 7), w);
 #pragma unroll
         for (int wi = 0; wi < 4; ++wi) {
 #pragma unroll
@@ -80,7 +80,7 @@ ProjectPlan plan_projection(int64_t n, int64_t P, int32_t d)
     // of fp32 accumulations never exceeds 4096 tensor-core steps), the largest that still gives every SM
     // about four work items of (256 gradient rows x 128 projected coordinates x chunk).
     ProjectPlan pl;
-    pl.n = n; pl.P = P; pl.d = d;
+    pl.n = n; pl.P = P; pl.d = d; pl.k_base = 0;
     const int64_t tiles = (int64_t)(d / 128) * ((n + 255) / 256);
     int64_t chunk = 65536;
     while (chunk > 1024 && tiles * ((P + chunk - 1) / chunk) < 4 * (int64_t)sm_count()) chunk >>= 1;
@@ -95,7 +95,7 @@ cudaError_t launch_project_simt(const __nv_bfloat16* gamma, const ProjectPlan& p
 {
     if (pl.n == 0) return cudaSuccess;
     dim3 grid((unsigned)(pl.d / PS_DR), (unsigned)((pl.n + PS_GR - 1) / PS_GR), (unsigned)pl.num_chunks);
-    project_simt_kernel<<<grid, PS_T, 0, st>>>(gamma, pl.n, pl.P, pl.d, pl.chunk, seed, part);
+    project_simt_kernel<<<grid, PS_T, 0, st>>>(gamma, pl.n, pl.P, pl.d, pl.chunk, (uint32_t)(pl.k_base >> 7), seed, part);
     count_launches(1);
     return cudaGetLastError();
 }

@@ -50,7 +50,8 @@ constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)SB * B_STAGE_BY
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int32_t d, int64_t P, int64_t chunk,
-                  int32_t num_chunks, uint64_t seed, float* __restrict__ part, unsigned int* __restrict__ timeout_word)
+                  int32_t num_chunks, uint32_t kblk_base, uint64_t seed, float* __restrict__ part,
+                  unsigned int* __restrict__ timeout_word)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);    // 1 KiB aligned, still a shared pointer
@@ -171,7 +172,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 if ((ita & 1u) != grp) continue;
                 const int sa = ita % SA;
                 uint32_t w[4];
-                rademacher_block(seed, r, (uint32_t)((k0 >> 7) + ka), w);     // overlaps with the wait below
+                rademacher_block(seed, r, kblk_base + (uint32_t)((k0 >> 7) + ka), w);     // overlaps with the wait below
                 ok = mbar_wait_cluster(smem_u32(&bars->a_empty[sa]), ((ita / SA) & 1u) ^ 1u, abort_flag, timeout_word, TO_GENERATOR);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
@@ -245,8 +246,8 @@ cudaError_t launch_project_tc(const CUtensorMap& tmap, const ProjectPlan& pl, ui
     const int64_t items = (int64_t)((pl.n + BN - 1) / BN) * pl.num_chunks * ((pl.d + 2 * BM - 1) / (2 * BM));
     int64_t grid = (sm_count() / 2) * 2;               // CTA pairs
     if (grid > 2 * items) grid = 2 * items;
-    project_tc_kernel<<<(unsigned)grid, NTHREADS, SMEM_BYTES, st>>>(tmap, pl.n, pl.d, pl.P, pl.chunk, pl.num_chunks, seed,
-                                                                    part, timeout_word);
+    project_tc_kernel<<<(unsigned)grid, NTHREADS, SMEM_BYTES, st>>>(tmap, pl.n, pl.d, pl.P, pl.chunk, pl.num_chunks,
+                                                                    (uint32_t)(pl.k_base >> 7), seed, part, timeout_word);
     count_launches(1);
     return cudaGetLastError();
 }

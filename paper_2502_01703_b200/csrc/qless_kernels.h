@@ -29,6 +29,7 @@ struct ProjectPlan {
     int32_t d;
     int64_t chunk;        // K-chunk length (multiple of 128)
     int32_t num_chunks;
+    int64_t k_base;       // absolute index of the first column given (a multiple of chunk): offsets the Philox counters
 };
 ProjectPlan plan_projection(int64_t n, int64_t P, int32_t d);
 cudaError_t launch_project_simt(const __nv_bfloat16* gamma_tiled, const ProjectPlan& pl,

@@ -249,6 +249,35 @@ def test_scores_edge_shapes():
 
 
 # ----------------------------------------------------------------------------------------------
+# Host-buffer entry: the batch is copied in column slabs that overlap the projection of earlier slabs;
+# codes, scales and code norms must be those of the device-buffer entry, bit for bit.
+# ----------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n,P,d,bits,dtype,adam", [
+    (40, 32768, 256, 4, torch.bfloat16, True),       # 32 K chunks -> 8 slabs of 4
+    (33, 4736, 128, 8, torch.float32, False),        # 5 chunks, the last one ragged -> 5 slabs
+    (5, 1024, 512, 1, torch.float32, True),          # a single chunk -> one slab
+    (300, 65536, 1024, 2, torch.bfloat16, True),     # two gradient-row tiles
+])
+def test_host_entry_matches_device_entry(n, P, d, bits, dtype, adam):
+    g = W.student_t_gradients(n, P, seed=61 + n, device="cpu").to(dtype)
+    pitch = P + 64                                            # rows of the host buffer need not be contiguous
+    host = torch.zeros((n, pitch), dtype=dtype).pin_memory()
+    host[:, :P] = g
+    m = v = cfg = None
+    if adam:
+        m, v = W.adam_moments(P, seed=62, device=DEV)
+        cfg = dict(beta1=0.9, beta2=0.999, eps=1e-8, step=0)
+    dev_out = B.qless_project_quantize(g.to(DEV), d, 777, bits, adam_m=m, adam_v=v, adam=cfg)
+    for rep in range(2):                                      # the second call reuses the staging buffers
+        host_out = B.qless_project_quantize_host(host[:, :P], d, 777, bits, adam_m=m, adam_v=v, adam=cfg, device=DEV)
+        torch.cuda.synchronize()
+        assert np.array_equal(host_out["codes"].numpy(), _np(dev_out["codes"]))
+        assert np.array_equal(host_out["scales"].numpy(), _np(dev_out["scales"]))
+        assert np.array_equal(host_out["sumsq"].numpy(), _np(dev_out["sumsq"]))
+
+
+# ----------------------------------------------------------------------------------------------
 # Top-k (bit-exact index sets, ascending order)
 # ----------------------------------------------------------------------------------------------
 
