@@ -22,11 +22,13 @@ __device__ __forceinline__ float adam_dir(float g, float bm, float bv, const Ada
         const float den_a = __fadd_rn(__fmul_rn(v1, rs), ap.eps);          // v1 = 0 gives NaN: handled below
         asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(den_a));
         const float q = __fmul_rn(m1, rc);
-        const int lo = (int)(__float_as_uint(q) & 0xFFFFu);
-        const float aq = fabsf(q);
-        // NaN fails every comparison, so it takes the exact path too
-        const bool safe = (abs(lo - 0x8000) > 32) && den_a > 1e-30f && den_a < 1e30f && aq > 1e-30f && aq < 1e30f;
-        if (safe) return q;
+        // Safe if q is well inside the normal range (biased exponent in [28, 226]: zeros, subnormals, infinities
+        // and NaNs all fall outside; so does every case in which den_a or its reciprocal left the normal range,
+        // since q is then 0, infinite or NaN) and its low 16 bits are more than 32 away from the bf16 tie 0x8000.
+        const uint32_t qb = __float_as_uint(q);
+        const bool in_range = (((qb >> 23) & 0xFFu) - 28u) <= 198u;
+        const bool off_tie = ((qb - 0x7FE0u) & 0xFFFFu) > 0x40u;
+        if (in_range && off_tie) return q;
     } else {
         m1 = __fdiv_rn(m1, ap.c1); v1 = __fdiv_rn(v1, ap.c2);
     }
