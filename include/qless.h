@@ -147,9 +147,10 @@ qless_status qless_project_quantize_host(
  * also what runs when P >= 2^31). Process-wide. */
 qless_status qless_set_projection_path(int32_t path);
 
-/* Test hook, as above, for the integer similarity of 8-, 4- and 2-bit codes in qless_score and
- * qless_score_dots: 0 (default) tcgen05 int8 kernel (used when T <= 8), 1 CUDA-core kernel. 1-bit codes
- * always use the XOR + population-count kernel. Process-wide. */
+/* Test hook, as above, for the integer similarity in qless_score and qless_score_dots: 0 (default) the
+ * tcgen05 int8 kernel for every code width (used when T <= 8; sub-byte codes, sign bits included, are expanded
+ * to int8 on the way), 1 the CUDA-core kernels (dp4a for 8-, 4- and 2-bit codes, XOR + population count for
+ * 1-bit codes). Process-wide. */
 qless_status qless_set_score_path(int32_t path);
 
 /* Test hook for qless_select_topk. 0 (default): for N > 2^22 a sampled lower bracket of the k-th largest

@@ -445,7 +445,7 @@ static ScoreWs score_layout(int64_t N, int32_t V, int32_t C, int32_t T, int32_t 
     w.eta = w.vmult + align_up((size_t)C * (size_t)V * 4, 256);
     w.off = w.eta + align_up((size_t)C * (size_t)T * 4, 256);
     w.vunp = w.off + align_up((size_t)(T + 1) * 4, 256);
-    w.total = w.vunp + (bits == 1 ? 0 : score_tc_workspace_bytes(V, C, d, bits));
+    w.total = w.vunp + score_tc_workspace_bytes(V, C, d, bits);
     return w;
 }
 
@@ -506,7 +506,7 @@ qless_status qless_score(const void* train_codes, int64_t train_ckpt_stride_byte
     a.train_mult = tmult; a.val_mult = vmult; a.eta_over_cnt = d_eta; a.task_off = d_off;
     a.N = N; a.V = V; a.C = C; a.T = T; a.d = d; a.bits = bits;
     a.scores = scores; a.per_task = per_task; a.dots = nullptr;
-    if (bits != 1 && g_score_path == 0 && score_tc_supported(T)) {
+    if (g_score_path == 0 && score_tc_supported(T)) {
         unsigned int* flag = timeout_flag_ptr();
         QLESS_REQUIRE(flag != nullptr, QLESS_ERR_CUDA, "cannot resolve the device timeout flag");
         ProfileScope ps("score", st);
@@ -522,7 +522,7 @@ qless_status qless_score(const void* train_codes, int64_t train_ckpt_stride_byte
 size_t qless_score_dots_workspace(int64_t nt, int32_t V, int32_t d, int32_t bits)
 {
     (void)nt;
-    if (V <= 0 || d <= 0 || bits == 1) return 256;
+    if (V <= 0 || d <= 0) return 256;
     return 256 + score_tc_workspace_bytes(V, 1, d, bits);
 }
 
@@ -544,7 +544,7 @@ qless_status qless_score_dots(const void* train_codes, const void* val_codes, in
     a.train_mult = nullptr; a.val_mult = nullptr; a.eta_over_cnt = nullptr; a.task_off = nullptr;
     a.N = nt; a.V = V; a.C = 1; a.T = 1; a.d = d; a.bits = bits;
     a.scores = nullptr; a.per_task = nullptr; a.dots = dots;
-    if (bits != 1 && g_score_path == 0) {
+    if (g_score_path == 0) {
         const size_t need = qless_score_dots_workspace(nt, V, d, bits);
         QLESS_REQUIRE(workspace != nullptr && aligned(workspace, 256), QLESS_ERR_WORKSPACE, "workspace must be non-NULL and 256-byte aligned");
         QLESS_REQUIRE(workspace_bytes >= need, QLESS_ERR_WORKSPACE, "workspace too small: %zu bytes given, %zu needed", workspace_bytes, need);

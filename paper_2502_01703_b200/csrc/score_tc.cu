@@ -1,4 +1,5 @@
-// Stage 3 for 8-, 4- and 2-bit codes on the tensor cores (tcgen05.mma kind::i8, int32 accumulators in TMEM).
+// Stage 3 on the tensor cores (tcgen05.mma kind::i8, int32 accumulators in TMEM) for every code width: 8-bit
+// codes as they are, 4-, 2- and 1-bit codes (sign bits as +-1) expanded to int8 on the way.
 //
 // Two CTAs on neighbouring SMs form a pair (cta_group::2) and own a tile of 256 train rows (UMMA M), 128
 // per CTA. For each checkpoint the pair streams the tile's codes and the validation codes K-block by
@@ -10,7 +11,7 @@
 // eta_i * mean to the running per-task sums; after the last checkpoint they take the max over tasks.
 // The N x V x C similarity tensor never exists in memory.
 //
-// 8-bit train codes go from global memory to the MMA operand buffer by TMA. 4- and 2-bit train codes
+// 8-bit train codes go from global memory to the MMA operand buffer by TMA. 4-, 2- and 1-bit train codes
 // arrive packed (TMA, no swizzle) in a staging ring; unpack warps (thread = train row = TMEM lane)
 // sign-extend them to int8 and store them straight into tensor memory, from where the MMA takes its A
 // operand: no shared-memory write, no swizzle, no proxy fence. The accumulator leaves 64 of the 512 TMEM
@@ -88,6 +89,12 @@ struct Ring {
     uint32_t slot = 0, parity = 0;
     __device__ __forceinline__ void next(uint32_t n) { if (++slot == n) { slot = 0; parity ^= 1u; } }
 };
+
+// 4 sign bits (bit set = negative) -> one word of four int8 +-1: the multiply copies bit i to byte i
+__device__ __forceinline__ uint32_t unpack1_nibble(uint32_t nib)
+{
+    return 0x01010101u + ((nib * 0x00204081u) & 0x01010101u) * 0xFEu;
+}
 
 template <int BITS>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
@@ -257,6 +264,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                     for (int u = 0; u < 4; ++u) {
                         if (BITS == 4) {
                             unpack4(ww[u], out[(c * 4 + u) * 2], out[(c * 4 + u) * 2 + 1]);
+                        } else if (BITS == 1) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) out[u * 8 + j] = unpack1_nibble((ww[u] >> (4 * j)) & 0xFu);
                         } else {
                             uint32_t o4[4];
                             unpack2(ww[u], o4);
@@ -431,6 +441,10 @@ __global__ void unpack_val_kernel(const uint8_t* __restrict__ codes, int64_t ckp
         const uint32_t w = *reinterpret_cast<const uint32_t*>(codes + i * ckpt_stride + v * (int64_t)(d * BITS / 8) + 4 * wq);
         uint32_t* o = reinterpret_cast<uint32_t*>(out + rowid * d) + wq * (8 / BITS);
         if (BITS == 4) { unpack4(w, o[0], o[1]); }
+        else if (BITS == 1) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) o[j] = unpack1_nibble((w >> (4 * j)) & 0xFu);
+        }
         else { uint32_t o4[4]; unpack2(w, o4); o[0] = o4[0]; o[1] = o4[1]; o[2] = o4[2]; o[3] = o4[3]; }
     }
 }
@@ -479,6 +493,7 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
         int64_t blocks = (total_words + 255) / 256;
         if (blocks > (int64_t)sm_count() * 8) blocks = (int64_t)sm_count() * 8;
         if (a.bits == 4) unpack_val_kernel<4><<<(unsigned)blocks, 256, 0, st>>>(a.val, a.val_stride, a.V, a.C, a.d, val_unpacked);
+        else if (a.bits == 1) unpack_val_kernel<1><<<(unsigned)blocks, 256, 0, st>>>(a.val, a.val_stride, a.V, a.C, a.d, val_unpacked);
         else unpack_val_kernel<2><<<(unsigned)blocks, 256, 0, st>>>(a.val, a.val_stride, a.V, a.C, a.d, val_unpacked);
         count_launches(1);
         val_src = val_unpacked; val_row = a.d; val_stride = (int64_t)a.V * a.d;
@@ -504,6 +519,7 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     score_tc_kernel<B><<<(unsigned)grid, NTHREADS, smem, st>>>(tm_train, tm_v1, tm_v2, p);
     if (a.bits == 8) { QLESS_LAUNCH_SCORE_TC(8) }
     else if (a.bits == 4) { QLESS_LAUNCH_SCORE_TC(4) }
+    else if (a.bits == 1) { QLESS_LAUNCH_SCORE_TC(1) }
     else { QLESS_LAUNCH_SCORE_TC(2) }
 #undef QLESS_LAUNCH_SCORE_TC
     count_launches(1);

@@ -234,6 +234,29 @@ def test_scores_match_oracle(bits, mode):
     assert torch.equal(got2, got)
 
 
+# The CUDA-core kernels (dp4a for 8/4/2-bit codes, XOR + population count for 1-bit codes) stay in the library as
+# a second implementation of the same integer similarity: they must agree with the oracle as the tensor-core
+# kernel does, and with the tensor-core kernel bit for bit on the raw dots.
+@pytest.mark.parametrize("bits", [8, 4, 2, 1])
+def test_score_cuda_core_path(bits):
+    C, N, V, d = 2, 300, 200, 1024
+    eta, off = [1.0, 0.5], [0, 50, 200]
+    tc, vc, ts, vs, tss, vss = _make_store(bits, C, N, V, d, seed=65)
+    dots_tc = _np(B.qless_score_dots(tc[0], vc[0], d, bits))
+    scores_tc = _np(B.qless_score(tc, vc, ts, vs, eta, off, d, bits))
+    try:
+        B.qless_set_score_path(1)
+        dots_cc = _np(B.qless_score_dots(tc[0], vc[0], d, bits))
+        scores_cc = _np(B.qless_score(tc, vc, ts, vs, eta, off, d, bits))
+    finally:
+        B.qless_set_score_path(0)
+    want_dots = oracle.dots(_np(tc[0]), _np(vc[0]), d, bits)
+    assert np.array_equal(dots_cc, want_dots) and np.array_equal(dots_tc, want_dots)
+    want = oracle.score(_np(tc), _np(vc), _np(ts), _np(vs), eta, off, d, bits)
+    assert np.abs(scores_cc - want).max() <= SCORE_TOL * sum(eta)
+    assert np.abs(scores_tc - want).max() <= SCORE_TOL * sum(eta)
+
+
 def test_scores_edge_shapes():
     for (C, N, V, T) in [(1, 1, 1, 1), (2, 64, 128, 1), (1, 65, 129, 2), (4, 10, 448, 3)]:
         d, bits = 256, 4
