@@ -227,6 +227,27 @@ def score(train_codes, val_codes, train_scales, val_scales, eta, task_offsets, d
     return (scores, per_task) if want_per_task else scores
 
 
+def score_16bit(train, val, eta, task_offsets, want_per_task=False):
+    """The 16-bit LESS baseline (Eq. 3 with the aggregation of Sec. 4.1), written out: train [C, N, d] and
+    val [C, V, d] hold the stored vectors (values that a 16-bit store can hold, passed as floats);
+    score[t] = max_j sum_i eta_i * mean_{v in task j} <x_t,i, x_v,i> / (||x_t,i|| ||x_v,i||), in fp64; a zero
+    vector has cosine 0 with everything."""
+    train = np.asarray(train, np.float64); val = np.asarray(val, np.float64)
+    eta = np.asarray(eta, np.float64); off = np.asarray(task_offsets, np.int64)
+    Cn, N, d = train.shape
+    T = off.size - 1
+    per_task = np.zeros((N, T), np.float64)
+    for i in range(Cn):
+        tn = np.sqrt((train[i] * train[i]).sum(axis=1)); vn = np.sqrt((val[i] * val[i]).sum(axis=1))
+        inner = train[i] @ val[i].T
+        denom = tn[:, None] * vn[None, :]
+        cos = np.divide(inner, denom, out=np.zeros_like(inner), where=denom > 0)
+        for j in range(T):
+            per_task[:, j] += eta[i] * cos[:, off[j]:off[j + 1]].mean(axis=1)
+    scores = per_task.max(axis=1)
+    return (scores, per_task) if want_per_task else scores
+
+
 def topk_count(N, frac):
     return int(lib().qlo_topk_count(int(N), float(frac)))
 

@@ -509,3 +509,46 @@ def test_project_quantize_is_the_composition_of_its_stages():
         if bits == 1:
             for i in range(n):
                 assert np.array_equal(oracle.unpack(codes[i], d, 1) < 0, y[i] < 0)
+
+
+# ----------------------------------------------------------------------------------------------
+# 16-bit LESS baseline (Eq. 3): pinned to closed forms and to the already-pinned integer cosine
+# ----------------------------------------------------------------------------------------------
+
+def test_score_16bit_closed_forms():
+    d = 64
+    e = np.eye(d)
+    # one checkpoint, one task of two validation vectors e0, e1; train rows: e0, (e0+e1), -e1, zero
+    train = np.stack([e[0], e[0] + e[1], -e[1], np.zeros(d)])[None]
+    val = np.stack([e[0], e[1]])[None]
+    s, pt = oracle.score_16bit(train, val, [2.0], [0, 2], want_per_task=True)
+    want = 2.0 * np.array([0.5, np.sqrt(0.5), -0.5, 0.0])
+    assert np.allclose(s, want, rtol=0, atol=1e-15) and pt.shape == (4, 1)
+    # scaling any stored vector by a positive constant changes nothing (Eq. 2 / Eq. 3 normalise)
+    s2 = oracle.score_16bit(train * np.array([3.0, 0.25, 7.0, 1.0])[None, :, None], val * 5.0, [2.0], [0, 2])
+    assert np.allclose(s2, want, rtol=0, atol=1e-15)
+    # two tasks: the maximum over tasks of the per-task means
+    s3, pt3 = oracle.score_16bit(train, val, [1.0], [0, 1, 2], want_per_task=True)
+    assert np.allclose(pt3, [[1, 0], [np.sqrt(0.5), np.sqrt(0.5)], [0, -1], [0, 0]], atol=1e-15)
+    assert np.allclose(s3, [1, np.sqrt(0.5), 0, 0], atol=1e-15)
+    # checkpoints add with their learning rates
+    s4 = oracle.score_16bit(np.concatenate([train, train]), np.concatenate([val, val]), [1.0, 0.5], [0, 2])
+    assert np.allclose(s4, 0.75 * want, atol=1e-15)
+
+
+def test_score_16bit_equals_integer_cosine_on_code_valued_vectors():
+    # Vectors whose entries are the 8-bit codes themselves (exact in a 16-bit float): Eq. 3 on them is the
+    # integer cosine of Eq. 6-7, which the quantised scorer of the oracle computes independently.
+    rng = np.random.default_rng(7)
+    C, N, V, d = 2, 37, 12, 256
+    x_t = rng.standard_normal((C, N, d)).astype(np.float32); x_v = rng.standard_normal((C, V, d)).astype(np.float32)
+    tc = np.empty((C, N, d), np.uint8); vc = np.empty((C, V, d), np.uint8)
+    ts = np.empty((C, N), np.float32); vs = np.empty((C, V), np.float32)
+    for i in range(C):
+        tc[i], ts[i], _ = oracle.quantize_rows(x_t[i], 8)
+        vc[i], vs[i], _ = oracle.quantize_rows(x_v[i], 8)
+    eta, off = [1.0, 0.5], [0, 5, 12]
+    want = oracle.score(tc, vc, ts, vs, eta, off, d, 8)
+    got = oracle.score_16bit(tc.view(np.int8).astype(np.float64), vc.view(np.int8).astype(np.float64), eta, off)
+    assert np.abs(got - want).max() <= 2e-6          # the quantised scorer rounds to fp32
+
