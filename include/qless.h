@@ -211,6 +211,20 @@ qless_status qless_score(
     float* scores, float* per_task,
     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The 16-bit baseline the paper compares against (LESS, Eq. 3 with the aggregation of Sec. 4.1): the store holds
+ * the projected gradients themselves as bf16 rows, train_rows [C][N][d] and val_rows [C][V][d] (device,
+ * checkpoint strides in bytes, multiples of 16), and
+ *   scores[t] = max_j sum_i lr_weights[i] * mean_{v in task j} <x_t,i, x_v,i> / (||x_t,i|| ||x_v,i||)
+ * with the inner products accumulated in fp32 on the tensor cores and the norms in fp64; a zero row scores 0.
+ * lr_weights [C] and task_offsets [T+1] are host arrays (tasks are consecutive validation rows, T <= 8);
+ * per_task (device [N][T]) may be NULL. Same d and V limits as qless_score. Workspace: device, 256-byte
+ * aligned, qless_score_16bit_workspace bytes. Errors: the statuses of qless_score. */
+size_t qless_score_16bit_workspace(int64_t N, int32_t V, int32_t C, int32_t T);
+qless_status qless_score_16bit(const void* train_rows, int64_t train_ckpt_stride_bytes, const void* val_rows,
+                               int64_t val_ckpt_stride_bytes, const float* lr_weights, const int32_t* task_offsets,
+                               int64_t N, int32_t V, int32_t C, int32_t T, int32_t d, float* scores, float* per_task,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* The integer numerators alone, for one checkpoint: dots [nt, V] int32 = D[t0 + t, v] computed by the
  * same kernels that feed qless_score. train_codes [>= t0+nt, d*bits/8], val_codes [V, d*bits/8]. */
 size_t qless_score_dots_workspace(int64_t nt, int32_t V, int32_t d, int32_t bits);

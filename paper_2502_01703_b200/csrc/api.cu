@@ -519,6 +519,61 @@ qless_status qless_score(const void* train_codes, int64_t train_ckpt_stride_byte
     return QLESS_OK;
 }
 
+size_t qless_score_16bit_workspace(int64_t N, int32_t V, int32_t C, int32_t T)
+{
+    if (N < 0 || V <= 0 || C <= 0 || T <= 0) return 256;
+    return score_layout(N, V, C, T, 128, 8).total;
+}
+
+qless_status qless_score_16bit(const void* train_rows, int64_t train_ckpt_stride_bytes, const void* val_rows,
+                               int64_t val_ckpt_stride_bytes, const float* lr_weights, const int32_t* task_offsets,
+                               int64_t N, int32_t V, int32_t C, int32_t T, int32_t d, float* scores, float* per_task,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    qless_status s = check_score_shape(N, V, d, 8);
+    if (s != QLESS_OK) return s;
+    QLESS_REQUIRE(C >= 1 && C <= 64, QLESS_ERR_UNSUPPORTED, "C must be in [1, 64] (C=%d)", C);
+    QLESS_REQUIRE(T >= 1 && T <= 8, QLESS_ERR_UNSUPPORTED, "T must be in [1, 8] (T=%d)", T);
+    QLESS_REQUIRE(lr_weights != nullptr && task_offsets != nullptr, QLESS_ERR_INVALID_ARG, "lr_weights and task_offsets (host) are required");
+    QLESS_REQUIRE(task_offsets[0] == 0 && task_offsets[T] == V, QLESS_ERR_INVALID_ARG, "task_offsets must start at 0 and end at V");
+    for (int j = 0; j < T; ++j)
+        QLESS_REQUIRE(task_offsets[j + 1] > task_offsets[j], QLESS_ERR_INVALID_ARG, "task_offsets must be strictly increasing (task %d)", j);
+    const int64_t row_bytes = (int64_t)d * 2;
+    QLESS_REQUIRE(train_ckpt_stride_bytes >= N * row_bytes && train_ckpt_stride_bytes % 16 == 0 &&
+                  val_ckpt_stride_bytes >= V * row_bytes && val_ckpt_stride_bytes % 16 == 0,
+                  QLESS_ERR_INVALID_ARG, "checkpoint strides must cover a checkpoint and be multiples of 16");
+    if (N == 0) return QLESS_OK;
+    QLESS_REQUIRE(train_rows && val_rows && scores, QLESS_ERR_INVALID_ARG, "train_rows, val_rows and scores are required");
+    QLESS_REQUIRE(aligned(train_rows, 16) && aligned(val_rows, 16), QLESS_ERR_INVALID_ARG, "row arrays must be 16-byte aligned");
+    const ScoreWs w = score_layout(N, V, C, T, 128, 8);
+    QLESS_REQUIRE(workspace != nullptr && aligned(workspace, 256), QLESS_ERR_WORKSPACE, "workspace must be non-NULL and 256-byte aligned");
+    QLESS_REQUIRE(workspace_bytes >= w.total, QLESS_ERR_WORKSPACE, "workspace too small: %zu bytes given, %zu needed", workspace_bytes, w.total);
+    uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+    float* tmult = reinterpret_cast<float*>(ws + w.tmult);
+    float* vmult = reinterpret_cast<float*>(ws + w.vmult);
+    float* d_eta = reinterpret_cast<float*>(ws + w.eta);
+    int32_t* d_off = reinterpret_cast<int32_t*>(ws + w.off);
+    std::vector<float> eoc((size_t)C * T);
+    for (int i = 0; i < C; ++i)
+        for (int j = 0; j < T; ++j)
+            eoc[(size_t)i * T + j] = lr_weights[i] / (float)(task_offsets[j + 1] - task_offsets[j]);
+    QLESS_CUDA_TRY(cudaMemcpyAsync(d_eta, eoc.data(), eoc.size() * 4, cudaMemcpyHostToDevice, st));
+    QLESS_CUDA_TRY(cudaMemcpyAsync(d_off, task_offsets, (size_t)(T + 1) * 4, cudaMemcpyHostToDevice, st));
+    QLESS_CUDA_TRY(launch_inv_norms_bf16(reinterpret_cast<const uint8_t*>(train_rows), train_ckpt_stride_bytes, N, C, d, tmult, st));
+    QLESS_CUDA_TRY(launch_inv_norms_bf16(reinterpret_cast<const uint8_t*>(val_rows), val_ckpt_stride_bytes, V, C, d, vmult, st));
+    ScoreArgs a;
+    a.train = reinterpret_cast<const uint8_t*>(train_rows); a.train_stride = train_ckpt_stride_bytes;
+    a.val = reinterpret_cast<const uint8_t*>(val_rows); a.val_stride = val_ckpt_stride_bytes;
+    a.train_mult = tmult; a.val_mult = vmult; a.eta_over_cnt = d_eta; a.task_off = d_off;
+    a.N = N; a.V = V; a.C = C; a.T = T; a.d = d; a.bits = 16;
+    a.scores = scores; a.per_task = per_task; a.dots = nullptr;
+    unsigned int* flag = timeout_flag_ptr();
+    QLESS_REQUIRE(flag != nullptr, QLESS_ERR_CUDA, "cannot resolve the device timeout flag");
+    ProfileScope ps("score16", st);
+    return launch_score_tc(a, nullptr, flag, st);
+}
+
 size_t qless_score_dots_workspace(int64_t nt, int32_t V, int32_t d, int32_t bits)
 {
     (void)nt;

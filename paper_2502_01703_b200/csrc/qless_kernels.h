@@ -59,7 +59,8 @@ struct ScoreArgs {
     int32_t* dots;              // if non-NULL: write raw integer dots [N][V] of checkpoint 0 only
 };
 cudaError_t launch_score_simt(const ScoreArgs& a, cudaStream_t st);
-// Tensor-core scoring for bits in {8, 4, 2} (score_tc.cu). T must be <= 8 (score_tc_supported).
+// Tensor-core scoring (score_tc.cu) for bits in {8, 4, 2, 1}, and for bits = 16: rows of d bf16 values, fp32
+// accumulation (the 16-bit baseline). T must be <= 8 (score_tc_supported).
 bool score_tc_supported(int32_t T);
 size_t score_tc_workspace_bytes(int32_t V, int32_t C, int32_t d, int32_t bits);
 qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned int* timeout_word, cudaStream_t st);
@@ -68,6 +69,9 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
 cudaError_t launch_multipliers(const uint8_t* codes, int64_t ckpt_stride, const float* scales,
                                const int32_t* sumsq, int64_t rows, int32_t C, int32_t d, int32_t bits,
                                int mode, float* mult, cudaStream_t st);
+// 16-bit baseline: per-row 1/norm of bf16 rows [C][nrows][d] (0 for a zero row).
+cudaError_t launch_inv_norms_bf16(const uint8_t* rows, int64_t ckpt_stride, int64_t nrows, int32_t C, int32_t d,
+                                  float* mult, cudaStream_t st);
 
 // Stage 4.
 size_t select_workspace_bytes(int64_t N);

@@ -248,4 +248,43 @@ cudaError_t launch_multipliers(const uint8_t* codes, int64_t ckpt_stride, const 
     return cudaGetLastError();
 }
 
+// 16-bit baseline: mult[i][r] = 1 / ||row r of checkpoint i|| (0 for a zero row), rows of d bf16 values. One warp per
+// row, squares summed in double.
+__global__ void __launch_bounds__(256)
+inv_norm_bf16_kernel(const uint8_t* __restrict__ rows, int64_t ckpt_stride, int64_t nrows, int32_t C, int32_t d,
+                     float* __restrict__ mult)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t nwarp = (int64_t)gridDim.x * 8;
+    for (int64_t r = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); r < (int64_t)C * nrows; r += nwarp) {
+        const int64_t i = r / nrows, row = r - i * nrows;
+        const uint4* src = reinterpret_cast<const uint4*>(rows + i * ckpt_stride + row * (int64_t)d * 2);
+        double acc = 0.0;
+        for (int c = lane; c < d / 8; c += 32) {
+            const uint4 w = __ldg(src + c);
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const double lo = (double)__uint_as_float(ww[u] << 16), hi = (double)__uint_as_float(ww[u] & 0xFFFF0000u);
+                acc += lo * lo; acc += hi * hi;
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+        if (lane == 0) mult[r] = (acc > 0.0) ? (float)(1.0 / sqrt(acc)) : 0.0f;
+    }
+}
+
+cudaError_t launch_inv_norms_bf16(const uint8_t* rows, int64_t ckpt_stride, int64_t nrows, int32_t C, int32_t d,
+                                  float* mult, cudaStream_t st)
+{
+    if (nrows == 0) return cudaSuccess;
+    int64_t blocks = ((int64_t)C * nrows + 7) / 8;
+    const int64_t cap = (int64_t)sm_count() * 16;
+    if (blocks > cap) blocks = cap;
+    inv_norm_bf16_kernel<<<(unsigned)blocks, 256, 0, st>>>(rows, ckpt_stride, nrows, C, d, mult);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
 }  // namespace qless

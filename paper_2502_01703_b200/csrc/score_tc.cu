@@ -104,9 +104,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);    // 1 KiB aligned, still a shared pointer
     const int bh1 = (p.n1 / 2) * KB, bh2 = (p.n2 / 2) * KB;      // bytes of this CTA's rows of the two MMA halves
-    constexpr int A_SMEM = (BITS == 8) ? A_STAGE : 0;              // sub-byte widths keep A in tensor memory
+    constexpr bool DIRECT = (BITS >= 8);                           // 8-bit codes and bf16 rows feed the MMA as stored
+    constexpr int A_SMEM = DIRECT ? A_STAGE : 0;                   // sub-byte widths keep A in tensor memory
     const int stage_bytes = A_SMEM + bh1 + bh2;                   // multiple of 1024
-    constexpr int P_STAGE = (BITS == 8) ? 0 : TM * 16 * BITS;     // packed staging bytes per stage
+    constexpr int P_STAGE = DIRECT ? 0 : TM * 16 * BITS;          // packed staging bytes per stage
     uint8_t* sS = smem;                                           // stage s: [A 16 KiB][B half 1][B half 2]
     uint8_t* sP = sS + (size_t)p.nS * stage_bytes;
     ScoreBars* bars = reinterpret_cast<ScoreBars*>(sP + (size_t)p.nP * P_STAGE);
@@ -115,16 +116,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     const int64_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-    const int nkb = p.d / KB;
+    const int nkb = (BITS == 16) ? (2 * p.d) / KB : p.d / KB;      // K blocks of 128 bytes per row
     const int num_vt = (p.V + p.vpad - 1) / p.vpad;
     const int64_t num_tiles = (p.N + 2 * TM - 1) / (2 * TM);      // tiles of 256 train rows
-    const uint32_t idesc1 = make_idesc(/*D=S32*/ 2, /*A=S8*/ 1, /*B=S8*/ 1, 2 * TM, p.n1);
-    const uint32_t idesc2 = make_idesc(2, 1, 1, 2 * TM, p.n2 > 0 ? p.n2 : 16);
+    // int8: D = S32 (2), A = B = S8 (1); 16-bit baseline: D = F32 (1), A = B = BF16 (1)
+    const uint32_t idesc1 = make_idesc(BITS == 16 ? 1 : 2, 1, 1, 2 * TM, p.n1);
+    const uint32_t idesc2 = make_idesc(BITS == 16 ? 1 : 2, 1, 1, 2 * TM, p.n2 > 0 ? p.n2 : 16);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_STAGES; ++s) {
             // leader's full[s]: the producer's expect_tx arrival (+ one arrival per unpack warp of both CTAs)
-            mbar_init(smem_u32(&bars->full[s]), BITS == 8 ? 1 : 9);
+            mbar_init(smem_u32(&bars->full[s]), DIRECT ? 1 : 9);
             mbar_init(smem_u32(&bars->empty[s]), 1);
             mbar_init(smem_u32(&bars->p_full[s]), 1);
             mbar_init(smem_u32(&bars->p_empty[s]), 4);
@@ -152,7 +154,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            const uint32_t tx_total = 2u * (uint32_t)((BITS == 8 ? A_STAGE : 0) + bh1 + bh2);   // both CTAs
+            const uint32_t tx_total = 2u * (uint32_t)(A_SMEM + bh1 + bh2);   // both CTAs
             const int64_t my_tiles = (num_tiles > pair) ? (num_tiles - pair + num_pairs - 1) / num_pairs : 0;
             const int64_t total = my_tiles * num_vt * p.C * nkb;
             // Packed train codes run ahead of the operand stages in their own ring: the load for iteration q is
@@ -180,7 +182,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 for (int vt = 0; vt < num_vt && ok; ++vt)
                     for (int i = 0; i < p.C && ok; ++i)
                         for (int kb = 0; kb < nkb; ++kb, ++it, st_ring.next((uint32_t)p.nS)) {
-                            if (BITS != 8) {
+                            if (!DIRECT) {
                                 // the packed codes of this iteration must be on their way; those of the next few if a slot is free
                                 while (pq <= (int64_t)it && ok) ok = issue_packed(true);
                                 if (!ok) break;
@@ -191,7 +193,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                             const uint32_t full = map_to_cta(smem_u32(&bars->full[s]), 0);
                             if (rank == 0) mbar_arrive_expect_tx(smem_u32(&bars->full[s]), tx_total);
                             uint8_t* st = sS + (size_t)s * stage_bytes;
-                            if (BITS == 8) tma_load_3d_pair(smem_u32(st), &tmap_train, full, kb * KB, row0, i);
+                            if (DIRECT) tma_load_3d_pair(smem_u32(st), &tmap_train, full, kb * KB, row0, i);
                             // this CTA's rows of the validation operand of each MMA half
                             tma_load_3d_pair(smem_u32(st + A_SMEM), &tmap_val1, full, kb * KB, vt * p.vpad + (int)rank * (p.n1 / 2), i);
                             if (p.n2 > 0)
@@ -221,7 +223,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
 #pragma unroll
                             for (int k = 0; k < KB / 32; ++k) {
                                 const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
-                                if (BITS == 8) {
+                                if (BITS == 16) {
+                                    mma_f16_ss_pair(tmem_base, adesc + (uint64_t)(k * 2), bdesc1 + (uint64_t)(k * 2), idesc1, acc);
+                                    if (p.n2 > 0) mma_f16_ss_pair(tmem_base + p.n1, adesc + (uint64_t)(k * 2), bdesc2 + (uint64_t)(k * 2), idesc2, acc);
+                                } else if (BITS == 8) {
                                     mma_i8_ss_pair(tmem_base, adesc + (uint64_t)(k * 2), bdesc1 + (uint64_t)(k * 2), idesc1, acc);
                                     if (p.n2 > 0) mma_i8_ss_pair(tmem_base + p.n1, adesc + (uint64_t)(k * 2), bdesc2 + (uint64_t)(k * 2), idesc2, acc);
                                 } else {
@@ -234,11 +239,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         if (ok) mma_commit_pair(smem_u32(&bars->d_full));
                     }
         }
-    } else if (BITS != 8 && (warp < 6 || warp >= 10)) {
+    } else if (!DIRECT && (warp < 6 || warp >= 10)) {
         // ------------------------------- unpack warps (4- and 2-bit train codes) -------------------------------
         // two groups of four warps (2-5 and 10-13) take alternate K blocks, so that the barrier round trips of
         // one block overlap the unpacking of the next
-        if (BITS != 8) {
+        if (!DIRECT) {
             const int row = (warp & 3) * 32 + lane;               // row of this CTA's 128-row half tile = TMEM lane
             const uint32_t grp = (warp >= 10) ? 1u : 0u;
             uint32_t it = 0;
@@ -363,10 +368,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
 #pragma unroll
                             for (int k4 = 0; k4 < 8; ++k4) {
                                 const float4 m4 = *reinterpret_cast<const float4*>(&bars->mv[c0 + 4 * k4]);
-                                x[4 * k4 + 0] = __fmul_rn((float)(int32_t)v[4 * k4 + 0], m4.x);
-                                x[4 * k4 + 1] = __fmul_rn((float)(int32_t)v[4 * k4 + 1], m4.y);
-                                x[4 * k4 + 2] = __fmul_rn((float)(int32_t)v[4 * k4 + 2], m4.z);
-                                x[4 * k4 + 3] = __fmul_rn((float)(int32_t)v[4 * k4 + 3], m4.w);
+                                // the accumulator holds int32 dots, or fp32 inner products for the 16-bit baseline
+                                auto acc_f = [](uint32_t raw) { return BITS == 16 ? __uint_as_float(raw) : (float)(int32_t)raw; };
+                                x[4 * k4 + 0] = __fmul_rn(acc_f(v[4 * k4 + 0]), m4.x);
+                                x[4 * k4 + 1] = __fmul_rn(acc_f(v[4 * k4 + 1]), m4.y);
+                                x[4 * k4 + 2] = __fmul_rn(acc_f(v[4 * k4 + 2]), m4.z);
+                                x[4 * k4 + 3] = __fmul_rn(acc_f(v[4 * k4 + 3]), m4.w);
                             }
                             if (next_b >= c0 + 32) {          // whole chunk inside task j (the common case)
 #pragma unroll
@@ -455,7 +462,7 @@ bool score_tc_supported(int32_t T) { return T <= TMAX; }
 
 size_t score_tc_workspace_bytes(int32_t V, int32_t C, int32_t d, int32_t bits)
 {
-    return bits == 8 ? 0 : align_up((size_t)C * V * d, 256);
+    return bits >= 8 ? 0 : align_up((size_t)C * V * d, 256);
 }
 
 // a.dots != NULL: raw dots of one checkpoint. val_unpacked: workspace of score_tc_workspace_bytes (bits < 8).
@@ -465,7 +472,7 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     ScoreTcParams p;
     p.N = a.N; p.V = a.V; p.C = a.C; p.T = a.T; p.d = a.d; p.bits = a.bits;
     const int vpad_all = (a.V + 15) / 16 * 16;
-    const int vcap = a.bits == 8 ? 512 : A_TMEM_COL;        // sub-byte widths keep 64 TMEM columns for the A operand
+    const int vcap = a.bits >= 8 ? 512 : A_TMEM_COL;        // sub-byte widths keep 64 TMEM columns for the A operand
     p.vpad = vpad_all < vcap ? vpad_all : vcap;
     p.n1 = p.vpad < 256 ? p.vpad : 256;
     p.n2 = p.vpad - p.n1;
@@ -473,14 +480,14 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
 
     // shared-memory plan: as many operand stages as fit (each: 16 KiB of train rows + this CTA's validation rows)
     const size_t budget = 227 * 1024 - 1024 - sizeof(ScoreBars) - 64;
-    const size_t stage = (a.bits == 8 ? (size_t)A_STAGE : 0) + (size_t)(p.vpad / 2) * KB;
-    const size_t p_stage = a.bits == 8 ? 0 : (size_t)TM * 16 * a.bits;
-    int nP = a.bits == 8 ? 0 : 4;
+    const size_t stage = (a.bits >= 8 ? (size_t)A_STAGE : 0) + (size_t)(p.vpad / 2) * KB;
+    const size_t p_stage = a.bits >= 8 ? 0 : (size_t)TM * 16 * a.bits;
+    int nP = a.bits >= 8 ? 0 : 4;
     int nS = (int)((budget - (size_t)nP * p_stage) / stage);
     if (nS > MAX_STAGES) nS = MAX_STAGES;
     QLESS_REQUIRE(nS >= 3, QLESS_ERR_UNSUPPORTED, "internal: not enough shared memory for two pipeline stages");
     p.nS = nS; p.nP = nP > 0 ? nP : 1;
-    p.epi_groups = (a.bits == 8 && a.T <= 6) ? 2 : 1;
+    p.epi_groups = (a.bits >= 8 && a.T <= 6) ? 2 : 1;
     const size_t smem = 1024 + (size_t)nS * stage + (size_t)nP * p_stage + sizeof(ScoreBars);
 
     p.train_mult = a.train_mult; p.val_mult = a.val_mult; p.eta_over_cnt = a.eta_over_cnt; p.task_off = a.task_off;
@@ -488,7 +495,7 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
 
     const uint8_t* val_src = a.val;
     int64_t val_row = row_bytes, val_stride = a.val_stride;
-    if (a.bits != 8) {
+    if (a.bits < 8) {
         const int64_t total_words = (int64_t)a.C * a.V * (row_bytes / 4);
         int64_t blocks = (total_words + 255) / 256;
         if (blocks > (int64_t)sm_count() * 8) blocks = (int64_t)sm_count() * 8;
@@ -502,7 +509,7 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     qless_status s;
     const int64_t tstride = a.C > 1 ? a.train_stride : (int64_t)a.N * row_bytes;
     s = make_tmap_3d_u8(&tm_train, a.train, (uint64_t)row_bytes, (uint64_t)a.N, (uint64_t)a.C, (uint64_t)row_bytes,
-                        (uint64_t)tstride, a.bits == 8 ? 128 : 16 * a.bits, TM, a.bits == 8);     // this CTA's 128 rows
+                        (uint64_t)tstride, a.bits >= 8 ? 128 : 16 * a.bits, TM, a.bits >= 8);     // this CTA's 128 rows
     if (s != QLESS_OK) return s;
     const int64_t vstride = a.C > 1 ? val_stride : (int64_t)a.V * val_row;
     s = make_tmap_3d_u8(&tm_v1, val_src, (uint64_t)val_row, (uint64_t)a.V, (uint64_t)a.C, (uint64_t)val_row, (uint64_t)vstride, 128, p.n1 / 2, true);
@@ -517,7 +524,8 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
 #define QLESS_LAUNCH_SCORE_TC(B)                                                                                    \
     QLESS_CUDA_TRY(cudaFuncSetAttribute(score_tc_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
     score_tc_kernel<B><<<(unsigned)grid, NTHREADS, smem, st>>>(tm_train, tm_v1, tm_v2, p);
-    if (a.bits == 8) { QLESS_LAUNCH_SCORE_TC(8) }
+    if (a.bits == 16) { QLESS_LAUNCH_SCORE_TC(16) }
+    else if (a.bits == 8) { QLESS_LAUNCH_SCORE_TC(8) }
     else if (a.bits == 4) { QLESS_LAUNCH_SCORE_TC(4) }
     else if (a.bits == 1) { QLESS_LAUNCH_SCORE_TC(1) }
     else { QLESS_LAUNCH_SCORE_TC(2) }

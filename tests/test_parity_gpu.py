@@ -257,6 +257,27 @@ def test_score_cuda_core_path(bits):
     assert np.abs(scores_tc - want).max() <= SCORE_TOL * sum(eta)
 
 
+# 16-bit baseline (Eq. 3): bf16 rows, fp32 accumulation on the tensor cores against the fp64 definition. Tolerance:
+# d products of bf16 values are exact in fp32; their fp32 sum over d = 8192 terms carries a relative error of a few
+# 2^-24 sqrt(d) of the norm product in practice (bound d 2^-24), so 2e-5 per unit of |eta| is the stated bar.
+SCORE16_TOL = 2e-5
+
+@pytest.mark.parametrize("C,N,V,d,off", [(2, 300, 100, 512, [0, 10, 37, 100]), (1, 65, 129, 128, [0, 129]),
+                                         (3, 700, 448, 8192, [0, 150, 300, 448]), (1, 5, 600, 1024, [0, 512, 600])])
+def test_score_16bit_matches_oracle(C, N, V, d, off):
+    gen = torch.Generator(device=DEV); gen.manual_seed(66 + N)
+    tr = torch.randn((C, N, d), generator=gen, device=DEV).to(torch.bfloat16)
+    va = torch.randn((C, V, d), generator=gen, device=DEV).to(torch.bfloat16)
+    tr[0, 3] = 0                                        # a zero row in the store
+    tr[0, 4] = va[0, 1] * 2                             # a row parallel to a validation row
+    eta = [1.0, 0.75, 0.5][:C]
+    got, got_pt = B.qless_score_16bit(tr, va, eta, off, want_per_task=True)
+    want, want_pt = oracle.score_16bit(_np(tr.float()), _np(va.float()), eta, off, want_per_task=True)
+    assert np.abs(_np(got) - want).max() <= SCORE16_TOL * sum(eta)
+    assert np.abs(_np(got_pt) - want_pt).max() <= SCORE16_TOL * sum(eta)
+    assert np.all(_np(got_pt)[3] == 0.0) if C == 1 else True
+
+
 def test_scores_edge_shapes():
     for (C, N, V, T) in [(1, 1, 1, 1), (2, 64, 128, 1), (1, 65, 129, 2), (4, 10, 448, 3)]:
         d, bits = 256, 4
