@@ -203,7 +203,8 @@ def stage_measurements(torch, B, W, dev, peaks):
     ms, ops = B.qless_microbench("popc", 20000, device=dev)
     popc_peak = ops / ms / 1e9          # T word-ops/s
     ms, ops = B.qless_microbench("bf16_ts_pair", 20000, device=dev)
-    out["microbench"] = dict(int8_tops=i8_peak, popc_xor_add_twordops=popc_peak, bf16_tcgen05_tflops=ops / ms / 1e9,
+    bf16_peak = ops / ms / 1e9          # TFLOP/s
+    out["microbench"] = dict(int8_tops=i8_peak, popc_xor_add_twordops=popc_peak, bf16_tcgen05_tflops=bf16_peak,
                              note="back-to-back tcgen05.mma / XOR+POPC+IADD on all SMs, burst")
     d = 8192
     # ---- quantise ----
@@ -225,22 +226,38 @@ def stage_measurements(torch, B, W, dev, peaks):
                      ts=torch.empty((C, N), device=dev), vs=torch.empty((C, V), device=dev),
                      tq=torch.empty((C, N), dtype=torch.int32, device=dev), vq=torch.empty((C, V), dtype=torch.int32, device=dev))
              for b in cfg["bits"]}
+    t16 = torch.empty((C, N, d), dtype=torch.bfloat16, device=dev)       # the 16-bit store of the same features
+    v16 = torch.empty((C, V, d), dtype=torch.bfloat16, device=dev)
     chunk = 16384
     for r0 in range(0, N, chunk):
         r1 = min(N, r0 + chunk)
         xs = W.lowrank_gaussian_features(r1 - r0, d, C, seed=SEED + 7 + r0, device=dev)
         for i in range(C):
+            t16[i, r0:r1] = xs[i].to(torch.bfloat16)
             for b in cfg["bits"]:
                 st = store[b]
                 st["tc"][i, r0:r1], st["ts"][i, r0:r1], st["tq"][i, r0:r1] = B.qless_quantize(xs[i], b)
     xs = W.lowrank_gaussian_features(V, d, C, seed=SEED + 8, device=dev)
     for i in range(C):
+        v16[i] = xs[i].to(torch.bfloat16)
         for b in cfg["bits"]:
             st = store[b]
             st["vc"][i], st["vs"][i], st["vq"][i] = B.qless_quantize(xs[i], b)
     del xs
     sc = torch.empty(N, device=dev)
     res = {}
+    # 16-bit baseline on the same features: its time, and its top-5 % set as the reference for the overlaps below
+    sc16 = torch.empty(N, device=dev)
+    ws16 = torch.empty(B.qless_score_16bit_workspace(N, V, C, len(off) - 1), dtype=torch.uint8, device=dev)
+    t = _time_ms(torch, lambda: B.qless_score_16bit(t16, v16, cfg["lr"], off, scores=sc16, workspace=ws16), 5)
+    flops = 2.0 * N * V * C * d
+    res["16"] = dict(ms=t, scores_per_s=N * V / (t * 1e-3), pair_dots_per_s=N * V * C / (t * 1e-3), bound="tensor",
+                     achieved_tflops=flops / t / 1e9, frac_of_bf16_peak=flops / t / 1e9 / bf16_peak,
+                     store_gb=C * (N + V) * d * 2 / 1e9)
+    top16 = B.qless_select_topk(sc16, cfg["frac"])
+    in16 = torch.zeros(N, dtype=torch.bool, device=dev)
+    in16[top16] = True
+    del t16, v16, ws16
     for b in cfg["bits"]:
         st = store[b]
         ws = torch.empty(B.qless_score_workspace(N, V, C, len(off) - 1, d, b), dtype=torch.uint8, device=dev)
@@ -248,7 +265,10 @@ def stage_measurements(torch, B, W, dev, peaks):
                                                   train_sumsq=st["tq"], val_sumsq=st["vq"], scores=sc, workspace=ws), 5)
         e = dict(ms=t, scores_per_s=N * V / (t * 1e-3), pair_dots_per_s=N * V * C / (t * 1e-3))
         iops = 2.0 * N * V * C * d
-        e.update(bound="tensor", achieved_tops=iops / t / 1e9, frac_of_int8_peak=iops / t / 1e9 / i8_peak)
+        e.update(bound="tensor", achieved_tops=iops / t / 1e9, frac_of_int8_peak=iops / t / 1e9 / i8_peak,
+                 store_gb=C * (N + V) * (d * b // 8 + 8) / 1e9)
+        topb = B.qless_select_topk(sc, cfg["frac"])
+        e["top5pct_overlap_with_16bit"] = float(in16[topb].float().mean())
         res[str(b)] = e
         if b == 1:
             # the XOR + population-count kernel (CUDA cores) on the same store, against the integer-ALU peak
