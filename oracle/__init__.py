@@ -4,7 +4,10 @@ TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the benchmark's
 CPU-baseline leg may import this package; the CUDA library never does, and this
 package never imports the CUDA library. Every function here only marshals numpy
 arrays into the C routine of the same name; the arithmetic is in the C file,
-each routine citing the equation of the paper it restates.
+each routine citing the equation of the paper it restates. Two functions are plain numpy instead, written out
+below: score_16bit (Eq. 3) and quantize_absmean_rows. The latter is PARITY UNPINNED as far as the formula goes:
+the paper names absmean quantisation (Sec. 6, Table 3) without giving it, so the function states one reading and
+is pinned only to what the paper and the arithmetic fix (see its docstring).
 """
 import ctypes as C
 import os
@@ -189,6 +192,46 @@ def quantize_rows(x, bits, normalize=True):
     lib().qlo_quantize_rows(_p(x, _f32p), n, d, bits, 1 if normalize else 0,
                             _p(codes, _u8p), _p(scales, _f32p), _p(sumsq, _i32p))
     return codes, scales, sumsq
+
+
+ABSMEAN_STEP = {2: 1.0, 4: 0.5, 8: 1.0 / 32.0}      # quantisation step in units of the mean absolute value
+
+
+def quantize_absmean_rows(x, bits, normalize=True):
+    """Absmean variant of Eq. 4-5 (Sec. 6, Table 3; the paper gives no formula: PARITY UNPINNED, this is the
+    reading): with yhat the (optionally L2-normalised, Eq. 2) row in fp32,
+        gamma = fp32( sum_m |yhat_m| (in fp64) / d ),   Delta = gamma * c_b,  c_2 = 1, c_4 = 1/2, c_8 = 1/32,
+        q_m   = clamp( round_half_even( fp32(yhat_m * fp32(1 / Delta)) ), -alpha, alpha ),  alpha = 2^(b-1) - 1,
+    and the stored scale is S = fp32(alpha * Delta), so that q_m * S / alpha dequantises as for absmax codes.
+    b = 2 is the ternary round-and-clip of x / mean|x|; the constants for b = 4, 8 put the clip point at
+    3.5 and about 4 mean absolute values. b = 1 is the sign code of Eq. 5 (no scale enters). A zero row gives
+    zero codes and S = 0. Returns (codes uint8 [n, d*bits/8], scales fp32 [n], sumsq int32 [n])."""
+    x = _c(x, np.float32)
+    n, d = x.shape
+    if bits == 1:
+        return quantize_rows(x, 1, normalize)
+    alpha = 2 ** (bits - 1) - 1
+    codes = np.empty((n, d * bits // 8), np.uint8)
+    scales = np.empty(n, np.float32)
+    sumsq = np.empty(n, np.int32)
+    for r in range(n):
+        yh = normalize_row(x[r]) if normalize else x[r]
+        gamma = np.float32(np.abs(yh.astype(np.float64)).sum() / d)
+        if not gamma > 0:
+            codes[r] = 0; scales[r] = 0; sumsq[r] = 0
+            continue
+        delta = np.float32(gamma * np.float32(ABSMEAN_STEP[bits]))
+        rcp = np.float32(1.0) / delta
+        t = (yh * rcp).astype(np.float32)
+        q = np.clip(np.rint(t), -alpha, alpha).astype(np.int8)
+        codes[r] = pack(q, bits)
+        scales[r] = np.float32(alpha) * delta
+        sumsq[r] = int((q.astype(np.int64) ** 2).sum())
+    return codes, scales, sumsq
+
+
+def normalize_row(y):
+    return normalize(y)[0]
 
 
 def dot(a, b):

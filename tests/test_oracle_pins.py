@@ -552,3 +552,53 @@ def test_score_16bit_equals_integer_cosine_on_code_valued_vectors():
     got = oracle.score_16bit(tc.view(np.int8).astype(np.float64), vc.view(np.int8).astype(np.float64), eta, off)
     assert np.abs(got - want).max() <= 2e-6          # the quantised scorer rounds to fp32
 
+
+# ----------------------------------------------------------------------------------------------
+# Absmean quantiser (Sec. 6, Table 3). The paper gives no formula, so parity for it is unpinned; what
+# can be pinned is the arithmetic of the stated reading and the one property the paper claims.
+# ----------------------------------------------------------------------------------------------
+
+def test_absmean_hand_example_and_invariants():
+    x = np.array([[0.5, -1.5, 2.0, 0.0] * 32], np.float32)          # mean |x| = 1 exactly
+    c2, s2, q2 = oracle.quantize_absmean_rows(x, 2, normalize=False)
+    assert oracle.unpack(c2[0], 128, 2)[:4].tolist() == [0, -1, 1, 0]         # 0.5 ties to even, +-1.5 and 2 clip
+    assert s2[0] == 1.0 and q2[0] == 64
+    c4, s4, q4 = oracle.quantize_absmean_rows(x, 4, normalize=False)
+    assert oracle.unpack(c4[0], 128, 4)[:4].tolist() == [1, -3, 4, 0] and s4[0] == 3.5
+    c8, s8, _ = oracle.quantize_absmean_rows(x, 8, normalize=False)
+    assert oracle.unpack(c8[0], 128, 8)[:4].tolist() == [16, -48, 64, 0] and s8[0] == np.float32(127 / 32)
+    # a power-of-two rescaling of the row changes the scale, not the codes; dequantisation error <= Delta / 2
+    rng = np.random.default_rng(3)
+    y = rng.standard_normal((5, 512)).astype(np.float32)
+    for bits in (2, 4, 8):
+        a = oracle.quantize_absmean_rows(y, bits, normalize=False)
+        b = oracle.quantize_absmean_rows(y * np.float32(0.25), bits, normalize=False)
+        assert np.array_equal(a[0], b[0]) and np.array_equal(a[1] * np.float32(0.25), b[1])
+        alpha = 2 ** (bits - 1) - 1
+        for r in range(5):
+            q = oracle.unpack(a[0][r], 512, bits).astype(np.float64)
+            delta = float(a[1][r]) / alpha
+            inside = np.abs(q) < alpha
+            assert np.abs(q * delta - y[r])[inside].max() <= delta / 2 * (1 + 1e-6)
+    z = oracle.quantize_absmean_rows(np.zeros((1, 128), np.float32), 4)
+    assert not z[0].any() and z[1][0] == 0 and z[2][0] == 0
+    # 1 bit: the sign code itself
+    assert np.array_equal(oracle.quantize_absmean_rows(y, 1)[0], oracle.quantize_rows(y, 1)[0])
+
+
+def test_absmean_keeps_more_nonzero_codes_than_absmax_at_low_width():
+    # The property the paper states for near-Gaussian rows (Sec. 6): at 2 and 4 bits absmax sends most coordinates
+    # to the zero bin, absmean does not. For z ~ N(0,1), d = 8192: absmax 2-bit keeps |z| > max/2 (about 2 sigma,
+    # under 10 %); absmean 2-bit keeps |z| > mean|z| / 2 = 0.399 sigma: 2 (1 - Phi(0.399)) = 0.690.
+    rng = np.random.default_rng(11)
+    y = rng.standard_normal((8, 8192)).astype(np.float32)
+    for bits, lo_mean, hi_max in ((2, 0.67, 0.10), (4, 0.82, 0.80)):
+        cm = oracle.quantize_absmean_rows(y, bits)[0]
+        cx = oracle.quantize_rows(y, bits)[0]
+        nz_mean = np.mean([np.count_nonzero(oracle.unpack(cm[r], 8192, bits)) for r in range(8)]) / 8192
+        nz_max = np.mean([np.count_nonzero(oracle.unpack(cx[r], 8192, bits)) for r in range(8)]) / 8192
+        assert nz_mean > lo_mean and nz_max < hi_max and nz_mean > nz_max
+    cm = oracle.quantize_absmean_rows(y, 2)[0]
+    nz = np.mean([np.count_nonzero(oracle.unpack(cm[r], 8192, 2)) for r in range(8)]) / 8192
+    assert abs(nz - 0.690) < 0.01
+
