@@ -282,10 +282,34 @@ def stage_measurements(torch, B, W, dev, peaks):
             res["1_popc"] = dict(ms=t, scores_per_s=N * V / (t * 1e-3), pair_dots_per_s=N * V * C / (t * 1e-3), bound="alu",
                                  achieved_twordops=wops / t / 1e9, frac_of_popc_peak=wops / t / 1e9 / popc_peak)
     out["score_c3_270000x448x4"] = res
+    # absmean codes of the same features (Sec. 6, Table 3): only the selection overlap is of interest, the kernels
+    # that score them are the ones timed above
+    del store
+    am = {}
+    for b in (8, 4, 2):
+        tcb = torch.empty((C, N, d * b // 8), dtype=torch.uint8, device=dev); tsb = torch.empty((C, N), device=dev)
+        tqb = torch.empty((C, N), dtype=torch.int32, device=dev)
+        vcb = torch.empty((C, V, d * b // 8), dtype=torch.uint8, device=dev); vsb = torch.empty((C, V), device=dev)
+        vqb = torch.empty((C, V), dtype=torch.int32, device=dev)
+        for r0 in range(0, N, chunk):
+            r1 = min(N, r0 + chunk)
+            xs = W.lowrank_gaussian_features(r1 - r0, d, C, seed=SEED + 7 + r0, device=dev)
+            for i in range(C):
+                tcb[i, r0:r1], tsb[i, r0:r1], tqb[i, r0:r1] = B.qless_quantize_absmean(xs[i], b)
+        xs = W.lowrank_gaussian_features(V, d, C, seed=SEED + 8, device=dev)
+        for i in range(C):
+            vcb[i], vsb[i], vqb[i] = B.qless_quantize_absmean(xs[i], b)
+        del xs
+        ws = torch.empty(B.qless_score_workspace(N, V, C, len(off) - 1, d, b), dtype=torch.uint8, device=dev)
+        B.qless_score(tcb, vcb, tsb, vsb, cfg["lr"], off, d, b, train_sumsq=tqb, val_sumsq=vqb, scores=sc, workspace=ws)
+        topb = B.qless_select_topk(sc, cfg["frac"])
+        am[str(b)] = dict(top5pct_overlap_with_16bit=float(in16[topb].float().mean()))
+        del tcb, vcb, ws
+    out["absmean_c3_overlap"] = am
     idx = torch.empty(N, dtype=torch.int64, device=dev)
     wsel = torch.empty(B.qless_select_topk_workspace(N), dtype=torch.uint8, device=dev)
     out["select_c3_270000_top5pct"] = dict(ms=_time_ms(torch, lambda: B.qless_select_topk(sc, cfg["frac"], indices=idx, workspace=wsel), 20))
-    del store, sc
+    del sc
     # ---- 1-bit scale-up, config 4 ----
     cfg = W.CONFIGS["c4_onebit_scaleup"]
     N = cfg["N"]

@@ -166,6 +166,14 @@ qless_status qless_quantize(
     const float* x, int64_t n, int32_t d, int32_t normalize, int32_t bits,
     void* codes, float* scales, int32_t* code_sumsq, void* cuda_stream);
 
+/* Absmean variant of the same stage (Sec. 6, Table 3). The paper names it without a formula; the reading built
+ * here: gamma = mean_m |yhat_m|, Delta = gamma * c_b with c_2 = 1, c_4 = 1/2, c_8 = 1/32,
+ * q_m = clamp(round_half_even(yhat_m / Delta), -alpha, alpha); scales[r] = alpha * Delta, so that q * scale / alpha
+ * dequantises as for absmax codes and qless_score takes such a store unchanged. bits = 1 is the sign code.
+ * Same arguments, packing, limits and errors as qless_quantize. */
+qless_status qless_quantize_absmean(const float* x, int64_t n, int32_t d, int32_t normalize, int32_t bits, void* codes,
+                                    float* scales, int32_t* code_sumsq, void* cuda_stream);
+
 /* Stage 1a alone: the Adam prologue. gamma_out [n, P] bf16 (raw 16-bit patterns), row-major, leading
  * dimension P. Same reading of Gamma as above. */
 qless_status qless_adam_gamma(

@@ -20,7 +20,7 @@ COSINE, DEQUANT = 0, 1
 
 EXPORTS = [
     "qless_last_error", "qless_check", "qless_project_quantize_workspace", "qless_project_quantize",
-    "qless_quantize", "qless_adam_gamma", "qless_philox_entries", "qless_score_workspace", "qless_score",
+    "qless_quantize", "qless_quantize_absmean", "qless_adam_gamma", "qless_philox_entries", "qless_score_workspace", "qless_score",
     "qless_score_16bit_workspace", "qless_score_16bit", "qless_score_dots_workspace", "qless_score_dots", "qless_select_topk_workspace", "qless_select_topk",
     "qless_project_quantize_host_workspace", "qless_project_quantize_host", "qless_profile_enable",
     "qless_profile_collect", "qless_kernel_launches", "qless_select_topk_static",
@@ -73,6 +73,8 @@ def lib():
         L.qless_profile_collect.argtypes = [C.c_char_p, sz]
         L.qless_quantize.restype = C.c_int
         L.qless_quantize.argtypes = [vp, i64, i32, i32, i32, vp, vp, vp, vp]
+        L.qless_quantize_absmean.restype = C.c_int
+        L.qless_quantize_absmean.argtypes = [vp, i64, i32, i32, i32, vp, vp, vp, vp]
         L.qless_adam_gamma.restype = C.c_int
         L.qless_adam_gamma.argtypes = [vp, C.c_int, i64, i64, vp, vp, C.POINTER(AdamCfg), i64, vp, vp]
         L.qless_philox_entries.restype = C.c_int
@@ -236,6 +238,18 @@ def qless_quantize(x, bits, normalize=True, want_sumsq=True, stream=None):
     sumsq = torch.empty(n, dtype=torch.int32, device=dev) if want_sumsq else None
     _check(lib().qless_quantize(_ptr(x), n, d, 1 if normalize else 0, bits, _ptr(codes), _ptr(scales),
                                 _ptr(sumsq), _stream(stream)))
+    return codes, scales, sumsq
+
+
+def qless_quantize_absmean(x, bits, normalize=True, want_sumsq=True, stream=None):
+    """As qless_quantize, with the scale taken from the mean absolute value of the row."""
+    n, d = x.shape
+    dev = x.device
+    codes = torch.empty((n, d * bits // 8), dtype=torch.uint8, device=dev)
+    scales = torch.empty(n, dtype=torch.float32, device=dev)
+    sumsq = torch.empty(n, dtype=torch.int32, device=dev) if want_sumsq else None
+    _check(lib().qless_quantize_absmean(_ptr(x), n, d, 1 if normalize else 0, bits, _ptr(codes), _ptr(scales),
+                                        _ptr(sumsq), _stream(stream)))
     return codes, scales, sumsq
 
 

@@ -396,6 +396,21 @@ qless_status qless_quantize(const float* x, int64_t n, int32_t d, int32_t normal
     return QLESS_OK;
 }
 
+qless_status qless_quantize_absmean(const float* x, int64_t n, int32_t d, int32_t normalize, int32_t bits, void* codes,
+                                    float* scales, int32_t* code_sumsq, void* cuda_stream)
+{
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    QLESS_REQUIRE(n >= 0, QLESS_ERR_INVALID_ARG, "n must be >= 0");
+    QLESS_REQUIRE(valid_bits(bits), QLESS_ERR_UNSUPPORTED, "bits must be 1, 2, 4 or 8 (bits=%d)", bits);
+    QLESS_REQUIRE(d >= 128 && d <= 8192 && d % 128 == 0, QLESS_ERR_UNSUPPORTED, "d must be a multiple of 128 in [128, 8192] (d=%d)", d);
+    if (n == 0) return QLESS_OK;
+    QLESS_REQUIRE(x != nullptr && codes != nullptr && scales != nullptr, QLESS_ERR_INVALID_ARG, "x, codes and scales are required");
+    QLESS_REQUIRE(aligned(x, 16) && aligned(codes, 16), QLESS_ERR_INVALID_ARG, "x and codes must be 16-byte aligned");
+    { ProfileScope ps("quantize_absmean", st);
+      QLESS_CUDA_TRY(launch_quantize_absmean(x, n, d, normalize ? 1 : 0, bits, codes, scales, code_sumsq, st)); }
+    return QLESS_OK;
+}
+
 qless_status qless_adam_gamma(const void* grads, qless_dtype dtype, int64_t n, int64_t ld_grads, const float* adam_m,
                               const float* adam_v, const qless_adam_cfg* adam, int64_t P, void* gamma_out,
                               void* cuda_stream)

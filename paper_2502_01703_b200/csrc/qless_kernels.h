@@ -42,6 +42,9 @@ cudaError_t launch_project_tc(const CUtensorMap& tmap, const ProjectPlan& pl, ui
 
 // Stage 2. x = inv_scale-scaled sum of `num_parts` partial arrays [num_parts][n][d] (num_parts = 1,
 // scale = 1 for plain rows). Writes proj_out (optional), codes, scales, sumsq (optional).
+// Absmean variant of the same stage on plain fp32 rows (scale from the mean absolute value).
+cudaError_t launch_quantize_absmean(const float* x, int64_t n, int32_t d, int normalize, int32_t bits, void* codes,
+                                    float* scales, int32_t* sumsq, cudaStream_t st);
 cudaError_t launch_quantize(const float* parts, int32_t num_parts, float scale, int64_t n, int32_t d,
                             int normalize, int32_t bits, void* codes, float* scales, int32_t* sumsq,
                             float* proj_out, cudaStream_t st);

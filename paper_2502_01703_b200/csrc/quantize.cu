@@ -28,7 +28,9 @@ __device__ __forceinline__ int warp_sum_i(int x)
     return x;
 }
 
-template <int BITS>
+// ABSMEAN: the scale comes from the mean absolute value of the row instead of its maximum (see the absmean
+// branch below); BITS = 1 has no scale and is always instantiated with ABSMEAN = false.
+template <int BITS, bool ABSMEAN = false>
 __global__ void __launch_bounds__(QT, 5)
 quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale, int64_t n, int32_t d,
                 int normalize, uint8_t* __restrict__ codes, float* __restrict__ scales,
@@ -105,7 +107,29 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
 
         // ---- Eq. 5 + pack into shared memory ----
         constexpr int ALPHA = (BITS == 1) ? 1 : ((1 << (BITS - 1)) - 1);
-        const float r = (S > 0.0f) ? __fdiv_rn((float)ALPHA, S) : 0.0f;
+        float r = (S > 0.0f) ? __fdiv_rn((float)ALPHA, S) : 0.0f;
+        if (ABSMEAN) {
+            // gamma = mean |yhat| (sum in double), Delta = gamma * c_b (c_2 = 1, c_4 = 1/2, c_8 = 1/32),
+            // q = clamp(rne(yhat / Delta), -alpha, alpha); the stored scale alpha * Delta dequantises like an absmax one
+            double sa = 0.0;
+#pragma unroll
+            for (int k = 0; k < QMAX_V4; ++k) {
+                sa += (double)fabsf(__fmul_rn(x[k].x, rn)); sa += (double)fabsf(__fmul_rn(x[k].y, rn));
+                sa += (double)fabsf(__fmul_rn(x[k].z, rn)); sa += (double)fabsf(__fmul_rn(x[k].w, rn));
+            }
+            sa = warp_sum(sa);
+            __syncthreads();                 // everyone has read s_d of the first reduction
+            if (lane == 0) s_d[warp] = sa;
+            __syncthreads();
+            double ta = 0.0;
+#pragma unroll
+            for (int w = 0; w < QT / 32; ++w) ta += s_d[w];
+            const float gamma = (float)(ta / (double)d);
+            constexpr float CB = (BITS == 2) ? 1.0f : (BITS == 4) ? 0.5f : 0.03125f;
+            const float delta = __fmul_rn(gamma, CB);
+            r = (gamma > 0.0f) ? __fdiv_rn(1.0f, delta) : 0.0f;
+            S = (gamma > 0.0f) ? __fmul_rn((float)ALPHA, delta) : 0.0f;
+        }
         int ss = 0;
 #pragma unroll
         for (int k = 0; k < QMAX_V4; ++k) {
@@ -124,7 +148,11 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
                     // two's-complement code (|yhat r| <= alpha (1 + 2^-23), so no clamp is needed)
                     uint32_t t[4];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) t[u] = __float_as_uint(__fadd_rn(__fmul_rn(e[u], r), 12582912.0f));
+                    for (int u = 0; u < 4; ++u) {
+                        float v = __fmul_rn(e[u], r);
+                        if (ABSMEAN) v = fminf(fmaxf(v, -(float)ALPHA), (float)ALPHA);      // clip (integers: rounding commutes)
+                        t[u] = __float_as_uint(__fadd_rn(v, 12582912.0f));
+                    }
                     // low bytes of the four sums -> one word of four int8 codes
                     const uint32_t w8 = __byte_perm(__byte_perm(t[0], t[1], 0x0040), __byte_perm(t[2], t[3], 0x0040), 0x5410);
                     ss = __dp4a((int)w8, (int)w8, ss);
@@ -162,6 +190,24 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
 }
 
 }  // namespace
+
+cudaError_t launch_quantize_absmean(const float* x, int64_t n, int32_t d, int normalize, int32_t bits, void* codes,
+                                    float* scales, int32_t* sumsq, cudaStream_t st)
+{
+    if (n == 0) return cudaSuccess;
+    int64_t blocks = n;
+    const int64_t cap = (int64_t)sm_count() * 8 * 4;
+    if (blocks > cap) blocks = cap;
+    uint8_t* c = reinterpret_cast<uint8_t*>(codes);
+    switch (bits) {
+        case 8: quantize_kernel<8, true><<<(unsigned)blocks, QT, 0, st>>>(x, 1, 1.0f, n, d, normalize, c, scales, sumsq, nullptr); break;
+        case 4: quantize_kernel<4, true><<<(unsigned)blocks, QT, 0, st>>>(x, 1, 1.0f, n, d, normalize, c, scales, sumsq, nullptr); break;
+        case 2: quantize_kernel<2, true><<<(unsigned)blocks, QT, 0, st>>>(x, 1, 1.0f, n, d, normalize, c, scales, sumsq, nullptr); break;
+        default: quantize_kernel<1><<<(unsigned)blocks, QT, 0, st>>>(x, 1, 1.0f, n, d, normalize, c, scales, sumsq, nullptr); break;
+    }
+    count_launches(1);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_quantize(const float* parts, int32_t num_parts, float scale, int64_t n, int32_t d,
                             int normalize, int32_t bits, void* codes, float* scales, int32_t* sumsq,

@@ -116,6 +116,43 @@ def test_quantize_with_normalisation_near_tie_audit(bits):
         assert np.all(np.abs(np.abs(pos - np.floor(pos)) - 0.5) < 1e-5)
 
 
+# Absmean variant: same protocol as above. The mean absolute value is reduced in another order than the oracle's
+# (both in fp64), so codes may differ only where yhat / Delta sits within 1e-5 of a rounding boundary, by one level.
+@pytest.mark.parametrize("bits", [8, 4, 2, 1])
+@pytest.mark.parametrize("normalize", [False, True])
+def test_quantize_absmean_matches_oracle(bits, normalize):
+    n, d = 200, 8192
+    y = _np(W.student_t_gradients(n, d, seed=33, device=DEV)) * np.float32(1e-2)
+    y[5] = 0.0
+    y[6, :] = np.tile(np.array([0.5, -1.5, 2.0, 0.0], np.float32), d // 4)      # mean |x| = 1: ties and clipping
+    codes, scales, sumsq = B.qless_quantize_absmean(torch.from_numpy(y).to(DEV), bits, normalize=normalize)
+    wc, ws, wss = oracle.quantize_absmean_rows(y, bits, normalize=normalize)
+    codes, scales, sumsq = _np(codes), _np(scales), _np(sumsq)
+    assert np.allclose(scales, ws, rtol=3e-7, atol=0)
+    if not normalize:
+        assert np.array_equal(codes[6], wc[6]) and scales[6] == ws[6]
+    bad_rows = np.where((codes != wc).any(axis=1))[0]
+    assert len(bad_rows) <= 3, f"{len(bad_rows)} rows differ"
+    alpha = 2 ** (bits - 1) - 1 if bits > 1 else 1
+    for r in bad_rows:
+        qa = oracle.unpack(codes[r], d, bits).astype(np.int32)
+        qb = oracle.unpack(wc[r], d, bits).astype(np.int32)
+        diff = np.where(qa != qb)[0]
+        assert bits > 1 and np.abs(qa - qb).max() == 1
+        yh = (oracle.normalize(y[r])[0] if normalize else y[r]).astype(np.float64)
+        pos = alpha * yh[diff] / float(ws[r])
+        assert np.all(np.abs(np.abs(pos - np.floor(pos)) - 0.5) < 1e-5)
+    ok = np.setdiff1d(np.arange(n), bad_rows)
+    assert np.array_equal(sumsq[ok], wss[ok])
+    # such a store goes through the scorer unchanged
+    if bits == 4 and normalize:
+        tc = torch.from_numpy(wc[:64].copy()).to(DEV).unsqueeze(0); vc = torch.from_numpy(wc[64:96].copy()).to(DEV).unsqueeze(0)
+        ts = torch.from_numpy(ws[:64].copy()).to(DEV).unsqueeze(0); vs = torch.from_numpy(ws[64:96].copy()).to(DEV).unsqueeze(0)
+        got = B.qless_score(tc, vc, ts, vs, [1.0], [0, 32], d, bits)
+        want = oracle.score(wc[None, :64], wc[None, 64:96], ws[None, :64], ws[None, 64:96], [1.0], [0, 32], d, bits)
+        assert np.abs(_np(got) - want).max() <= SCORE_TOL
+
+
 def test_quantize_edge_shapes():
     for n in (0, 1, 2):
         x = torch.randn((n, 256), device=DEV)
