@@ -315,6 +315,36 @@ def test_score_16bit_matches_oracle(C, N, V, d, off):
     assert np.all(_np(got_pt)[3] == 0.0) if C == 1 else True
 
 
+# Un-normalised (TracIn-style, Sec. 2.1) scores need no kernel of their own: rows quantised without Eq. 2 keep their
+# length in the scale, and the DEQUANT mode sums eta <S_t q_t / alpha, S_v q_v / alpha>. Checked against the oracle on the
+# same codes (1e-5 relative) and against the fp64 inner products of the rows themselves (8-bit quantisation error).
+def test_unnormalised_scores_through_dequant_mode():
+    C, N, V, d, bits = 2, 200, 64, 1024, 8
+    gen = torch.Generator(device=DEV); gen.manual_seed(68)
+    lens_t = torch.rand((C, N, 1), generator=gen, device=DEV) * 4 + 0.25
+    lens_v = torch.rand((C, V, 1), generator=gen, device=DEV) * 2 + 0.5
+    xt = torch.randn((C, N, d), generator=gen, device=DEV) * lens_t / np.sqrt(d)
+    xv = torch.randn((C, V, d), generator=gen, device=DEV) * lens_v / np.sqrt(d)
+    xv = xv + 0.5 * xt[:, :V]                                  # correlated, so that scores are not all near zero
+    tc = torch.empty((C, N, d), dtype=torch.uint8, device=DEV); vc = torch.empty((C, V, d), dtype=torch.uint8, device=DEV)
+    ts = torch.empty((C, N), device=DEV); vs = torch.empty((C, V), device=DEV)
+    for i in range(C):
+        tc[i], ts[i], _ = B.qless_quantize(xt[i], bits, normalize=False)
+        vc[i], vs[i], _ = B.qless_quantize(xv[i], bits, normalize=False)
+    eta, off = [1.0, 0.5], [0, 20, 64]
+    got, got_pt = B.qless_score(tc, vc, ts, vs, eta, off, d, bits, mode=B.DEQUANT, want_per_task=True)
+    want, want_pt = oracle.score(_np(tc), _np(vc), _np(ts), _np(vs), eta, off, d, bits, mode=B.DEQUANT, want_per_task=True)
+    scale = float(np.abs(want_pt).max())
+    assert np.abs(_np(got_pt) - want_pt).max() <= SCORE_TOL * sum(eta) * scale
+    exact = np.zeros((N, 2))
+    for i in range(C):
+        ip = _np(xt[i]).astype(np.float64) @ _np(xv[i]).astype(np.float64).T
+        for j in range(2):
+            exact[:, j] += eta[i] * ip[:, off[j]:off[j + 1]].mean(axis=1)
+    assert np.abs(_np(got_pt) - exact).max() <= 0.02 * np.abs(exact).max()
+    assert np.abs(_np(got) - exact.max(axis=1)).max() <= 0.02 * np.abs(exact).max()
+
+
 def test_scores_edge_shapes():
     for (C, N, V, T) in [(1, 1, 1, 1), (2, 64, 128, 1), (1, 65, 129, 2), (4, 10, 448, 3)]:
         d, bits = 256, 4
