@@ -134,11 +134,11 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 tc_fence_after();
                 for (int kb = 0; kb < nkb; ++kb, ++itb) {
                     const int sb = itb % SB;
-                    if (!mbar_wait_cluster(smem_u32(&bars->b_full[sb]), (itb / SB) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
+                    if (!mbar_wait(smem_u32(&bars->b_full[sb]), (itb / SB) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
                     const int nh = (int)min((int64_t)(BK / 128), (klen - (int64_t)kb * BK) >> 7);
                     for (int h = 0; h < nh && ok; ++h, ++ita) {                // one 128-deep sign stage at a time
                         const int sa = ita % SA;
-                        if (!mbar_wait_cluster(smem_u32(&bars->a_full[sa]), (ita / SA) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
+                        if (!mbar_wait(smem_u32(&bars->a_full[sa]), (ita / SA) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t a_addr = tmem_base + A_COL + sa * 64;
 #pragma unroll
