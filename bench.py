@@ -197,7 +197,7 @@ def stage_measurements(torch, B, W, dev, peaks):
     2^28 scores. Each entry gives the CUDA-event time of the library call and the achieved fraction of the
     relevant measured peak (HBM copy bandwidth, or the library's own tcgen05 int8 / XOR+POPC micro-benchmark)."""
     out = {}
-    # measured peaks of units the driver did not measure
+    # measured peaks of the units that have no externally measured figure (int8 tensor pipe, integer ALU mix)
     ms, ops = B.qless_microbench("i8_ss_pair", 20000, device=dev)
     i8_peak = ops / ms / 1e9            # Tops/s
     ms, ops = B.qless_microbench("popc", 20000, device=dev)
