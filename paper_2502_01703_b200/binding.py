@@ -21,7 +21,7 @@ COSINE, DEQUANT = 0, 1
 EXPORTS = [
     "qless_last_error", "qless_check", "qless_project_quantize_workspace", "qless_project_quantize",
     "qless_quantize", "qless_quantize_absmean", "qless_adam_gamma", "qless_philox_entries", "qless_score_workspace", "qless_score",
-    "qless_score_16bit_workspace", "qless_score_16bit", "qless_score_dots_workspace", "qless_score_dots", "qless_select_topk_workspace", "qless_select_topk",
+    "qless_score_16bit_workspace", "qless_score_16bit", "qless_inv_norms_16bit", "qless_score_dots_workspace", "qless_score_dots", "qless_select_topk_workspace", "qless_select_topk",
     "qless_project_quantize_host_workspace", "qless_project_quantize_host", "qless_profile_enable",
     "qless_profile_collect", "qless_kernel_launches", "qless_select_topk_static",
     "qless_set_projection_path", "qless_set_score_path", "qless_set_select_path", "qless_microbench",
@@ -87,8 +87,10 @@ def lib():
         L.qless_score_16bit_workspace.restype = sz
         L.qless_score_16bit_workspace.argtypes = [i64, i32, i32, i32]
         L.qless_score_16bit.restype = C.c_int
-        L.qless_score_16bit.argtypes = [vp, i64, vp, i64, C.POINTER(C.c_float), C.POINTER(i32), i64, i32, i32, i32, i32,
-                                        vp, vp, vp, sz, vp]
+        L.qless_score_16bit.argtypes = [vp, i64, vp, i64, vp, vp, C.POINTER(C.c_float), C.POINTER(i32), i64, i32, i32, i32,
+                                        i32, vp, vp, vp, sz, vp]
+        L.qless_inv_norms_16bit.restype = C.c_int
+        L.qless_inv_norms_16bit.argtypes = [vp, i64, i64, i32, i32, vp, vp]
         L.qless_score_dots_workspace.restype = sz
         L.qless_score_dots_workspace.argtypes = [i64, i32, i32, i32]
         L.qless_score_dots.restype = C.c_int
@@ -298,8 +300,16 @@ def qless_score_16bit_workspace(N, V, Cn, T):
     return int(lib().qless_score_16bit_workspace(N, V, Cn, T))
 
 
+def qless_inv_norms_16bit(rows, stream=None):
+    """rows bf16 [C, n, d] -> 1 / ||row|| as f32 [C, n] (0 for a zero row)."""
+    Cn, n, d = rows.shape
+    out = torch.empty((Cn, n), dtype=torch.float32, device=rows.device)
+    _check(lib().qless_inv_norms_16bit(_ptr(rows), rows.stride(0) * 2, n, Cn, d, _ptr(out), _stream(stream)))
+    return out
+
+
 def qless_score_16bit(train_rows, val_rows, lr_weights, task_offsets, want_per_task=False, scores=None,
-                      workspace=None, stream=None):
+                      workspace=None, stream=None, train_inv_norms=None, val_inv_norms=None):
     """The 16-bit baseline: train_rows bf16 [C, N, d], val_rows bf16 [C, V, d] (checkpoint stride taken from the
     tensors); lr_weights / task_offsets: host sequences."""
     assert train_rows.dtype == torch.bfloat16 and val_rows.dtype == torch.bfloat16
@@ -314,7 +324,8 @@ def qless_score_16bit(train_rows, val_rows, lr_weights, task_offsets, want_per_t
     per_task = torch.empty((N, T), dtype=torch.float32, device=dev) if want_per_task else None
     ws = _workspace(qless_score_16bit_workspace(N, V, Cn, T), dev, workspace)
     _check(lib().qless_score_16bit(_ptr(train_rows), train_rows.stride(0) * 2 if Cn > 0 else 0, _ptr(val_rows),
-                                   val_rows.stride(0) * 2, eta, off, N, V, Cn, T, d, _ptr(scores), _ptr(per_task),
+                                   val_rows.stride(0) * 2, _ptr(train_inv_norms), _ptr(val_inv_norms), eta, off, N, V, Cn, T,
+                                   d, _ptr(scores), _ptr(per_task),
                                    _ptr(ws), ws.numel(), _stream(stream)))
     return (scores, per_task) if want_per_task else scores
 

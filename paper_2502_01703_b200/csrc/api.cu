@@ -540,8 +540,23 @@ size_t qless_score_16bit_workspace(int64_t N, int32_t V, int32_t C, int32_t T)
     return score_layout(N, V, C, T, 128, 8).total;
 }
 
+qless_status qless_inv_norms_16bit(const void* rows, int64_t ckpt_stride_bytes, int64_t nrows, int32_t C, int32_t d,
+                                   float* inv_norms, void* cuda_stream)
+{
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    QLESS_REQUIRE(nrows >= 0 && C >= 1, QLESS_ERR_INVALID_ARG, "nrows >= 0 and C >= 1 required");
+    QLESS_REQUIRE(d >= 128 && d <= 8192 && d % 128 == 0, QLESS_ERR_UNSUPPORTED, "d must be a multiple of 128 in [128, 8192] (d=%d)", d);
+    QLESS_REQUIRE(ckpt_stride_bytes >= nrows * (int64_t)d * 2 && ckpt_stride_bytes % 16 == 0, QLESS_ERR_INVALID_ARG,
+                  "checkpoint stride must cover a checkpoint and be a multiple of 16");
+    if (nrows == 0) return QLESS_OK;
+    QLESS_REQUIRE(rows != nullptr && inv_norms != nullptr && aligned(rows, 16), QLESS_ERR_INVALID_ARG, "rows (16-byte aligned) and inv_norms are required");
+    QLESS_CUDA_TRY(launch_inv_norms_bf16(reinterpret_cast<const uint8_t*>(rows), ckpt_stride_bytes, nrows, C, d, inv_norms, st));
+    return QLESS_OK;
+}
+
 qless_status qless_score_16bit(const void* train_rows, int64_t train_ckpt_stride_bytes, const void* val_rows,
-                               int64_t val_ckpt_stride_bytes, const float* lr_weights, const int32_t* task_offsets,
+                               int64_t val_ckpt_stride_bytes, const float* train_inv_norms, const float* val_inv_norms,
+                               const float* lr_weights, const int32_t* task_offsets,
                                int64_t N, int32_t V, int32_t C, int32_t T, int32_t d, float* scores, float* per_task,
                                void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
@@ -575,12 +590,16 @@ qless_status qless_score_16bit(const void* train_rows, int64_t train_ckpt_stride
             eoc[(size_t)i * T + j] = lr_weights[i] / (float)(task_offsets[j + 1] - task_offsets[j]);
     QLESS_CUDA_TRY(cudaMemcpyAsync(d_eta, eoc.data(), eoc.size() * 4, cudaMemcpyHostToDevice, st));
     QLESS_CUDA_TRY(cudaMemcpyAsync(d_off, task_offsets, (size_t)(T + 1) * 4, cudaMemcpyHostToDevice, st));
-    QLESS_CUDA_TRY(launch_inv_norms_bf16(reinterpret_cast<const uint8_t*>(train_rows), train_ckpt_stride_bytes, N, C, d, tmult, st));
-    QLESS_CUDA_TRY(launch_inv_norms_bf16(reinterpret_cast<const uint8_t*>(val_rows), val_ckpt_stride_bytes, V, C, d, vmult, st));
+    // the norms are a pass over the whole store: a caller that keeps them beside the store passes them in
+    if (train_inv_norms == nullptr)
+        QLESS_CUDA_TRY(launch_inv_norms_bf16(reinterpret_cast<const uint8_t*>(train_rows), train_ckpt_stride_bytes, N, C, d, tmult, st));
+    if (val_inv_norms == nullptr)
+        QLESS_CUDA_TRY(launch_inv_norms_bf16(reinterpret_cast<const uint8_t*>(val_rows), val_ckpt_stride_bytes, V, C, d, vmult, st));
     ScoreArgs a;
     a.train = reinterpret_cast<const uint8_t*>(train_rows); a.train_stride = train_ckpt_stride_bytes;
     a.val = reinterpret_cast<const uint8_t*>(val_rows); a.val_stride = val_ckpt_stride_bytes;
-    a.train_mult = tmult; a.val_mult = vmult; a.eta_over_cnt = d_eta; a.task_off = d_off;
+    a.train_mult = train_inv_norms ? train_inv_norms : tmult; a.val_mult = val_inv_norms ? val_inv_norms : vmult;
+    a.eta_over_cnt = d_eta; a.task_off = d_off;
     a.N = N; a.V = V; a.C = C; a.T = T; a.d = d; a.bits = 16;
     a.scores = scores; a.per_task = per_task; a.dots = nullptr;
     unsigned int* flag = timeout_flag_ptr();

@@ -313,6 +313,9 @@ def test_score_16bit_matches_oracle(C, N, V, d, off):
     assert np.abs(_np(got) - want).max() <= SCORE16_TOL * sum(eta)
     assert np.abs(_np(got_pt) - want_pt).max() <= SCORE16_TOL * sum(eta)
     assert np.all(_np(got_pt)[3] == 0.0) if C == 1 else True
+    # norms kept beside the store give the same scores
+    got2 = B.qless_score_16bit(tr, va, eta, off, train_inv_norms=B.qless_inv_norms_16bit(tr), val_inv_norms=B.qless_inv_norms_16bit(va))
+    assert torch.equal(got2, got)
 
 
 # Un-normalised (TracIn-style, Sec. 2.1) scores need no kernel of their own: rows quantised without Eq. 2 keep their
