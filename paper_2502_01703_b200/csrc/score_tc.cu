@@ -213,7 +213,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         if (!mbar_wait_cluster(smem_u32(&bars->d_empty), (n_acc & 1u) ^ 1u, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
                         for (int kb = 0; kb < nkb; ++kb, ++it, st_ring.next((uint32_t)p.nS)) {
                             const int s = (int)st_ring.slot;
-                            if (!mbar_wait_cluster(smem_u32(&bars->full[s]), st_ring.parity, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
+                            if (!mbar_wait(smem_u32(&bars->full[s]), st_ring.parity, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
                             tc_fence_after();
                             const uint32_t st = smem_u32(sS + (size_t)s * stage_bytes);
                             const uint64_t adesc = make_smem_desc_sw128(st);
@@ -288,7 +288,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 // TMEM slot it % 2 is free once the MMAs of K block it - 2 have completed, which is what releases
                 // operand stage (it - 2) % nS (nS > 2, so that barrier cannot run a whole phase ahead of us)
                 if (it >= 2)
-                    ok = mbar_wait_cluster(smem_u32(&bars->empty[lag_ring.slot]), lag_ring.parity, abort_flag, p.timeout_word, TO_UNPACK);
+                    ok = mbar_wait(smem_u32(&bars->empty[lag_ring.slot]), lag_ring.parity, abort_flag, p.timeout_word, TO_UNPACK);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
