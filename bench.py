@@ -191,6 +191,50 @@ def _time_ms(torch, fn, iters, warm=1):
     return e0.elapsed_time(e1) / iters
 
 
+def pipeline_c5(torch, B, W, dev):
+    """Config 5 end to end: per checkpoint 32 768 training gradients (P = 2^22, bf16, Adam prologue) and 448
+    validation gradients are projected to d = 8192 and stored as 2-bit codes, then scored and the top 5 % selected.
+    The gradients are streamed in batches of 256 rows; to keep input generation out of the way each checkpoint
+    cycles a pool of 4 generated batches (32 distinct pools over the run), so rows repeat inside a checkpoint: this
+    changes nothing in the work done. Times are the library's own per-kernel CUDA-event totals."""
+    cfg = W.CONFIGS["c5_full_pipeline"]
+    N, V, P, d, C, bits = cfg["n_train"], cfg["n_val"], cfg["P"], cfg["d"], cfg["C"], cfg["bits"]
+    rb = d * bits // 8
+    off = W.task_offsets(cfg["tasks"]).tolist()
+    tc = torch.empty((C, N, rb), dtype=torch.uint8, device=dev); ts = torch.empty((C, N), device=dev)
+    tq = torch.empty((C, N), dtype=torch.int32, device=dev)
+    vc = torch.empty((C, V, rb), dtype=torch.uint8, device=dev); vs = torch.empty((C, V), device=dev)
+    vq = torch.empty((C, V), dtype=torch.int32, device=dev)
+    ws = torch.empty(B.qless_project_quantize_workspace(V, P, d, bits), dtype=torch.uint8, device=dev)
+    B.qless_profile_collect()
+    B.qless_profile_enable(True)
+    for i in range(C):
+        m, v = W.adam_moments(P, seed=SEED + 300 + i, device=dev)
+        pool = [W.student_t_gradients(256, P, seed=SEED + 400 + 8 * i + j, device=dev, dtype=torch.bfloat16) for j in range(4)]
+        for b in range(N // 256):
+            r0 = b * 256
+            B.qless_project_quantize(pool[b % 4], d, SEED, bits, m, v, workspace=ws,
+                                     out=dict(codes=tc[i, r0:r0 + 256], scales=ts[i, r0:r0 + 256], sumsq=tq[i, r0:r0 + 256]))
+        del pool
+        g = W.student_t_gradients(V, P, seed=SEED + 500 + i, device=dev, dtype=torch.bfloat16)
+        B.qless_project_quantize(g, d, SEED, bits, workspace=ws, out=dict(codes=vc[i], scales=vs[i], sumsq=vq[i]))
+        del g, m, v
+    sc = torch.empty(N, device=dev)
+    wsc = torch.empty(B.qless_score_workspace(N, V, C, len(off) - 1, d, bits), dtype=torch.uint8, device=dev)
+    B.qless_score(tc, vc, ts, vs, cfg["lr"], off, d, bits, train_sumsq=tq, val_sumsq=vq, scores=sc, workspace=wsc)
+    idx = B.qless_select_topk(sc, cfg["frac"])
+    torch.cuda.synchronize()
+    prof = B.qless_profile_collect()
+    B.qless_profile_enable(False)
+    B.qless_check()
+    stages = {k: dict(ms=ms, calls=c) for k, (ms, c) in prof.items()}
+    total = sum(ms for ms, _ in prof.values())
+    rows = C * (N + V)
+    return dict(stages=stages, total_ms=total, gradients=rows, gradients_per_s=rows / (total * 1e-3), selected=int(idx.numel()),
+                project_tflops=2.0 * rows * P * d / (prof["project"][0] * 1e-3) / 1e12 if "project" in prof else None,
+                note="library time only (per-kernel CUDA events); input generation excluded")
+
+
 def stage_measurements(torch, B, W, dev, peaks):
     """The other kernels of the path at the sizes where their roofline is observable: quantise on 65 536 rows,
     scoring on the 270 K x 448 x 4-checkpoint store per bit width and on the 2 M-row 1-bit store, selection on
@@ -343,6 +387,8 @@ def stage_measurements(torch, B, W, dev, peaks):
     wsel = torch.empty(B.qless_select_topk_workspace(N), dtype=torch.uint8, device=dev)
     out["select_c4_2000000_top1pct"] = dict(ms=_time_ms(torch, lambda: B.qless_select_topk(sc, cfg["frac"], indices=idx, workspace=wsel), 20))
     del tc, sc, idx
+    # ---- config 5: the whole path for a 4-checkpoint store, stage by stage ----
+    out["pipeline_c5"] = pipeline_c5(torch, B, W, dev)
     # ---- selection at a size where HBM bandwidth is observable ----
     N = 1 << 28
     s = torch.randn(N, device=dev)
