@@ -109,7 +109,7 @@ qless_status qless_microbench(int32_t what, int32_t iters, float* ms_out, double
  *   codes      [n, d*bits/8] bytes, dense little-endian packing: b=8 one int8 per code; b=4 code m in
  *              bits [4(m&1), +4) of byte m>>1; b=2 code m in bits [2(m&3), +2) of byte m>>2 (two's
  *              complement fields); b=1 code m is bit m&7 of byte m>>3, bit 1 <=> -1.
- *   scales     [n] fp32, the absmax S of the normalised vector (the "single scale factor" of Sec. 3.1).
+ *   scales     [n] fp32, the absmax S of the normalised vector (the one scale per vector of Sec. 3.1).
  *   code_sumsq [n] int32, sum_m q_m^2 = ||q||^2 of Eq. 6 (NULL to skip).
  *   proj_out   [n, d] fp32, the un-normalised projection y (NULL to skip; test tap).
  * The same seed must be used for every vector that will be scored together.
@@ -188,7 +188,7 @@ qless_status qless_philox_entries(
 
 /* ------------------------------------------------------------------------------------------
  * Stage 3: influence scores over the quantised datastore (paper Eq. 6-7; aggregation as in LESS,
- * which the paper follows: "cumulative influence scores", Sec. 4.1).
+ * which the paper follows when it accumulates influence over the validation data, Sec. 4.1).
  *
  *   D_i[t, v]  = sum_m q_{t,i,m} q_{v,i,m}                 integer, exact (b = 1: d - 2 popcount(xor))
  *   sim_i[t,v] = D_i / (||q_{t,i}|| ||q_{v,i}||)            mode COSINE (Eq. 6-7); a vector whose scale
@@ -247,7 +247,7 @@ qless_status qless_score_dots(
     int32_t d, int32_t bits, int32_t* dots, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
- * Stage 4: top-k selection ("Select the top 5% of training data", Sec. 4.1).
+ * Stage 4: top-k selection (the top 5 % of the training data by score, Sec. 4.1).
  *
  *   k = floor(frac * N + 1e-6) clamped to [0, N], written to *k_out (host) before the call returns.
  *   Total order on fp32: by value, -0 below +0, every NaN below -inf; equal scores are admitted by

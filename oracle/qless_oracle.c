@@ -369,7 +369,7 @@ void qlo_dots(const uint8_t* train_codes, const uint8_t* val_codes, int64_t t0, 
 /*   Inf(z, z') = sum_i eta_i <qhat_z',i , qhat_z,i>                 (Eq. 7)  */
 /*   A[z, j]   = sum_i eta_i * mean_{z' in task j} <qhat_z',i, qhat_z,i>      */
 /*   score[z]  = max_j A[z, j]                                                */
-/* ("cumulative influence scores", Sec. 4.1; mean-per-task / max-over-tasks   */
+/* (influence accumulated over the validation data, Sec. 4.1; mean-per-task / max-over-tasks   */
 /* is the LESS rule the paper inherits.)                                      */
 /* mode 0 (cosine): as above; a vector whose stored scale S is 0 is the zero  */
 /*   vector and contributes 0.                                                */
