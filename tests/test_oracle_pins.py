@@ -228,7 +228,7 @@ def test_sign_quantizer_and_zero_vector():
 
 
 def test_zero_bin_occupancy_of_absmax_on_gaussians():
-    # Sec. 5 ("Analyzing Sparsity Effects of Absmax Quantization"): for Gaussian-like values most
+    # Sec. 5 (the paragraph on the sparsity that absmax quantisation induces): for Gaussian-like values most
     # entries fall in the zero bin at low bit widths; 1-bit has no zero bin.
     # Closed form: P(q = 0) = P(|x| < S/(2 alpha)) = erf(S / (2 alpha sigma sqrt 2)).
     x = np.random.default_rng(8).standard_normal(8192).astype(np.float32)
