@@ -104,6 +104,21 @@ def test_bad_arguments_return_statuses_before_any_launch(L):
     assert score([0, 4, 8], bits=5) == B.ERR_UNSUPPORTED
     assert score([0, 4, 8]) == B.ERR_WORKSPACE            # valid shapes, no workspace given
     assert score([0, 4, 8], V=8, d=130) == B.ERR_UNSUPPORTED
+    # the widened entry points check their arguments in the same way
+    assert L.qless_quantize_absmean(null, 4, 500, 1, 8, null, null, null, null) == B.ERR_UNSUPPORTED
+    assert L.qless_quantize_absmean(null, 4, 512, 1, 3, null, null, null, null) == B.ERR_UNSUPPORTED
+    assert L.qless_quantize_absmean(null, 4, 512, 1, 4, null, null, null, null) == B.ERR_INVALID_ARG
+    assert L.qless_quantize_absmean(null, 0, 512, 1, 4, null, null, null, null) == B.QLESS_OK
+    o3 = (C.c_int32 * 3)(0, 4, 8)
+    def score16(V=8, T=2, d=128, off=o3, ws=null, wsb=0):
+        return L.qless_score_16bit(fake, 4096, fake, 4096, null, null, eta, off, 4, V, 2, T, d, fake, null, ws, wsb, null)
+    assert score16(d=130) == B.ERR_UNSUPPORTED
+    assert score16(T=9, off=(C.c_int32 * 10)(*range(10))) == B.ERR_UNSUPPORTED
+    assert score16(off=(C.c_int32 * 3)(0, 4, 7)) == B.ERR_INVALID_ARG
+    assert score16() == B.ERR_WORKSPACE
+    assert B.qless_score_16bit_workspace(1000, 64, 2, 3) >= 2 * 1000 * 4
+    assert L.qless_inv_norms_16bit(fake, 16, 4, 1, 128, fake, null) == B.ERR_INVALID_ARG      # stride does not cover a checkpoint
+    assert L.qless_inv_norms_16bit(null, 4096, 0, 1, 128, null, null) == B.QLESS_OK
     # test hooks that choose a kernel variant: only the documented values
     for hook, bad in ((L.qless_set_projection_path, 2), (L.qless_set_score_path, -1), (L.qless_set_select_path, 3)):
         assert hook(bad) == B.ERR_INVALID_ARG
