@@ -383,6 +383,16 @@ def stage_measurements(torch, B, W, dev, peaks):
     iops = 2.0 * N * V * C * d
     out["score_c4_2000000x448x4_1bit"] = dict(ms=t, scores_per_s=N * V / (t * 1e-3), bound="tensor",
                                               achieved_tops=iops / t / 1e9, frac_of_int8_peak=iops / t / 1e9 / i8_peak)
+    # the same store through the XOR + population-count kernel (CUDA cores), against the integer-ALU peak
+    B.qless_set_score_path(1)
+    try:
+        t = _time_ms(torch, lambda: B.qless_score(tc, vc, ts, vs, cfg["lr"], off, d, 1, train_sumsq=tq, val_sumsq=vq,
+                                                  scores=sc, workspace=ws), 2)
+    finally:
+        B.qless_set_score_path(0)
+    wops = N * V * C * (d / 32)
+    out["score_c4_2000000x448x4_1bit_popc"] = dict(ms=t, scores_per_s=N * V / (t * 1e-3), bound="alu",
+                                                   achieved_twordops=wops / t / 1e9, frac_of_popc_peak=wops / t / 1e9 / popc_peak)
     idx = torch.empty(N, dtype=torch.int64, device=dev)
     wsel = torch.empty(B.qless_select_topk_workspace(N), dtype=torch.uint8, device=dev)
     out["select_c4_2000000_top1pct"] = dict(ms=_time_ms(torch, lambda: B.qless_select_topk(sc, cfg["frac"], indices=idx, workspace=wsel), 20))
