@@ -153,11 +153,12 @@ qless_status qless_set_projection_path(int32_t path);
  * 1-bit codes). Process-wide. */
 qless_status qless_set_score_path(int32_t path);
 
-/* Test hook for qless_select_topk. 0 (default): for N > 2^22 a sampled lower bracket of the k-th largest
- * key, one gather pass and a radix select on the gathered candidates (two reads of the scores), with the
- * multi-pass select enqueued behind it as a device-gated fallback; for smaller N the multi-pass select
- * (five reads). 1: multi-pass at every N. 2: the bracket is forced above every key, so that the fallback
- * does the work. The result is the same in all three. Process-wide. */
+/* Test hook for qless_select_topk. 0 (default): up to 360 448 scores one launch of a thread-block cluster that
+ * keeps the keys in shared memory (one read, no workspace used); up to 2^22 the multi-pass radix select (five
+ * reads); above, a sampled lower bracket of the k-th largest key, one gather pass and a radix select on the
+ * gathered candidates (two reads), with the multi-pass select enqueued behind it as a device-gated fallback.
+ * 1: multi-pass at every N. 2: as 0, with the bracket forced above every key, so that the fallback does the
+ * work. The result is the same in all three. Process-wide. */
 qless_status qless_set_select_path(int32_t path);
 
 /* Stage 2 alone (Eq. 2, Eq. 4-5, packing) on fp32 rows x [n, d]; normalize = 0 skips Eq. 2 so that

@@ -6,6 +6,7 @@
 #include <mutex>
 
 #include "qless_kernels.h"
+#include "tc_common.cuh"
 
 namespace qless {
 
@@ -743,6 +744,127 @@ cand_write_kernel(const uint32_t* __restrict__ seg_key, const uint16_t* __restri
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Small N (every workload of the paper): one thread-block cluster of eight CTAs does the whole selection
+// in one launch. Each CTA loads its contiguous slice of the scores once and keeps the keys in shared
+// memory; the three radix rounds build per-CTA histograms there and every CTA sums the eight histograms
+// through distributed shared memory; the slice totals of {key > T}, {key == T} are exchanged the same way
+// and each CTA writes its part of the answer in index order. One read of the scores, no workspace, and the
+// only waits are the hardware cluster barrier.
+// ------------------------------------------------------------------------------------------------
+constexpr int CL_CTAS = 8;
+constexpr int CL_T = 1024;
+constexpr int CL_CAP = 45056;                              // keys per CTA held in shared memory (176 KiB)
+constexpr int64_t CL_MAX_N = (int64_t)CL_CTAS * CL_CAP;    // 360 448 scores
+
+__device__ __forceinline__ uint32_t ld_dsmem_u32(uint32_t cluster_addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(cluster_addr) : "memory");
+    return v;
+}
+
+__global__ void __cluster_dims__(CL_CTAS, 1, 1) __launch_bounds__(CL_T, 1)
+select_cluster_kernel(const float* __restrict__ scores, int64_t N, int64_t k, int64_t* __restrict__ indices)
+{
+    extern __shared__ uint32_t s_key[];                    // [CL_CAP] keys of this CTA's slice
+    __shared__ uint32_t s_hist2[2][2048];                  // alternating per round: one cluster barrier per round suffices
+    __shared__ int64_t s_w[2][32];
+    __shared__ uint32_t s_bin;
+    __shared__ int64_t s_krem;
+    __shared__ int s_tot[2];                               // this slice's counts of {key > T}, {key == T}
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t rank = tc::cluster_ctarank();
+    const int64_t per = ((N + CL_CTAS - 1) / CL_CTAS + 3) & ~(int64_t)3;          // slice length, a multiple of 4
+    const int64_t i0 = (int64_t)rank * per;
+    const int n_loc = (int)((i0 >= N) ? 0 : ((N - i0 < per) ? N - i0 : per));
+    for (int i = tid; i < n_loc; i += CL_T) s_key[i] = order_key(__float_as_uint(__ldg(scores + i0 + i)));
+    __syncthreads();
+
+    uint32_t prefix = 0;
+    int64_t k_rem = k;
+#pragma unroll 1
+    for (int round = 0; round < 3; ++round) {
+        const int shift = (round == 0) ? 21 : (round == 1) ? 10 : 0;
+        const int bits = (round == 2) ? 10 : 11;
+        const uint32_t mask = (1u << bits) - 1u;
+        uint32_t* s_hist = s_hist2[round & 1];
+        for (int i = tid; i < 2048; i += CL_T) s_hist[i] = 0;
+        __syncthreads();
+        for (int i = tid; i < n_loc; i += CL_T) {
+            const uint32_t key = s_key[i];
+            if (round == 0 || (key >> (shift + bits)) == prefix) atomicAdd(&s_hist[(key >> shift) & mask], 1u);
+        }
+        __syncthreads();
+        tc::cluster_sync_all();                           // all eight histograms of this round complete
+        // every CTA sums the eight histograms and finds the bin of the k_rem-th largest key: thread t owns, from the
+        // top, bins 2047-2t and 2046-2t (rounds 0, 1) or bin 1023-t (round 2)
+        const int nb = 1 << bits;
+        const int per_t = nb / CL_T;                      // 2 or 1
+        int64_t c[2] = {0, 0};
+        for (int u = 0; u < per_t; ++u) {
+            const int b = nb - 1 - (tid * per_t + u);
+            const uint32_t own = tc::smem_u32(&s_hist[b]);
+            int64_t sum = 0;
+#pragma unroll
+            for (uint32_t r = 0; r < CL_CTAS; ++r) sum += ld_dsmem_u32(tc::map_to_cta(own, r));
+            c[u] = sum;
+        }
+        const int64_t mine = c[0] + c[1];
+        int64_t inc = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int64_t a = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= o) inc += a;
+        }
+        if (lane == 31) s_w[0][warp] = inc;
+        __syncthreads();
+        int64_t pre = inc - mine;
+        for (int w = 0; w < warp; ++w) pre += s_w[0][w];
+        for (int u = 0; u < per_t; ++u) {
+            if (pre < k_rem && k_rem <= pre + c[u]) { s_bin = (uint32_t)(nb - 1 - (tid * per_t + u)); s_krem = k_rem - pre; }
+            pre += c[u];
+        }
+        __syncthreads();
+        prefix = (prefix << bits) | s_bin;
+        k_rem = s_krem;
+        // no barrier here: the next round fills the other histogram buffer, and this one is cleared again only after
+        // the next round's cluster barrier, which every CTA reaches after it has finished reading it
+    }
+    const uint32_t T = prefix;
+    const int64_t k_ties = k_rem;
+
+    // thread t owns a run of consecutive keys of the slice (odd length: no shared-memory bank conflicts)
+    const int len = ((n_loc + CL_T - 1) / CL_T) | 1;
+    const int j0 = tid * len, j1 = (j0 + len < n_loc) ? j0 + len : n_loc;
+    int gt = 0, eq = 0;
+    for (int j = j0; j < j1; ++j) { const uint32_t key = s_key[j]; gt += (key > T); eq += (key == T); }
+    int ig = gt, ie = eq;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int a = __shfl_up_sync(0xFFFFFFFFu, ig, o), b = __shfl_up_sync(0xFFFFFFFFu, ie, o);
+        if (lane >= o) { ig += a; ie += b; }
+    }
+    if (lane == 31) { s_w[0][warp] = ig; s_w[1][warp] = ie; }
+    __syncthreads();
+    int64_t gt_before = ig - gt, eq_before = ie - eq;
+    for (int w = 0; w < warp; ++w) { gt_before += s_w[0][w]; eq_before += s_w[1][w]; }
+    if (tid == CL_T - 1) { s_tot[0] = (int)(gt_before + gt); s_tot[1] = (int)(eq_before + eq); }
+    __syncthreads();
+    tc::cluster_sync_all();                               // slice totals visible to the other CTAs
+    for (uint32_t r = 0; r < rank; ++r) {
+        gt_before += (int)ld_dsmem_u32(tc::map_to_cta(tc::smem_u32(&s_tot[0]), r));
+        eq_before += (int)ld_dsmem_u32(tc::map_to_cta(tc::smem_u32(&s_tot[1]), r));
+    }
+    for (int j = j0; j < j1; ++j) {
+        const uint32_t key = s_key[j];
+        const bool g = key > T, e = key == T;
+        if (g || (e && eq_before < k_ties)) indices[gt_before + (eq_before < k_ties ? eq_before : k_ties)] = i0 + j;
+        gt_before += g; eq_before += e;
+    }
+    tc::cluster_sync_all();                               // no CTA leaves while another may still read its shared memory
+}
+
 SelectWs carve(void* ws, int64_t N)
 {
     SelectWs w;
@@ -870,6 +992,17 @@ cudaError_t launch_select_topk(const float* scores, int64_t N, int64_t k, int64_
                                cudaStream_t st)
 {
     if (N == 0 || k == 0) return cudaSuccess;
+    if (g_select_path != 1 && N <= CL_MAX_N) {
+        static std::once_flag once;
+        static cudaError_t attr_err = cudaSuccess;
+        std::call_once(once, [] {
+            attr_err = cudaFuncSetAttribute(select_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CL_CAP * (int)sizeof(uint32_t));
+        });
+        if (attr_err != cudaSuccess) return attr_err;
+        select_cluster_kernel<<<CL_CTAS, CL_T, CL_CAP * sizeof(uint32_t), st>>>(scores, N, k, indices);
+        count_launches(1);
+        return cudaGetLastError();
+    }
     if (use_bracket(N)) return launch_bracketed(scores, N, k, indices, ws, g_select_path == 2, st);
     SelectWs w = carve(ws, N);
     cudaError_t e = cudaMemsetAsync(w.hist, 0, 3 * 2048 * sizeof(uint32_t), st);

@@ -395,7 +395,7 @@ def test_host_entry_matches_device_entry(n, P, d, bits, dtype, adam):
 # Top-k (bit-exact index sets, ascending order)
 # ----------------------------------------------------------------------------------------------
 
-@pytest.mark.parametrize("N", [1, 2, 63, 1000, 2048, 2049, 100_003, 1 << 21])
+@pytest.mark.parametrize("N", [1, 2, 7, 8, 9, 63, 1000, 2048, 2049, 100_003, 270_000, 360_448, 360_449, 1 << 21])
 @pytest.mark.parametrize("frac", [0.0, 0.01, 0.05, 0.5, 1.0])
 def test_topk_matches_oracle(N, frac):
     gen = torch.Generator(device=DEV); gen.manual_seed(80 + N)
@@ -403,6 +403,12 @@ def test_topk_matches_oracle(N, frac):
     got = _np(B.qless_select_topk(s, frac))
     want = oracle.select_topk(_np(s), frac)
     assert np.array_equal(got, want)
+    # up to 360 448 scores the default is the one-launch cluster kernel; the multi-pass kernels must agree with it
+    try:
+        B.qless_set_select_path(1)
+        assert np.array_equal(_np(B.qless_select_topk(s, frac)), want)
+    finally:
+        B.qless_set_select_path(0)
 
 
 def test_topk_ties_and_special_values():
