@@ -52,6 +52,12 @@ def _declare(L):
     L.qlo_project_rows.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_int32, C.c_uint64, _i32p,
                                    C.c_int32, _f32p]
     L.qlo_project_rows.restype = None
+    L.qlo_gaussian_entry_exact.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64]
+    L.qlo_gaussian_entry_exact.restype = C.c_double
+    L.qlo_gaussian_row.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64, C.c_uint64, _f32p]
+    L.qlo_gaussian_row.restype = None
+    L.qlo_project_gaussian.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_int32, C.c_uint64, _f32p]
+    L.qlo_project_gaussian.restype = None
     L.qlo_normalize.argtypes = [_f32p, C.c_int32, _f32p]
     L.qlo_normalize.restype = C.c_float
     L.qlo_quantize.argtypes = [_f32p, C.c_int32, C.c_int32, _i8p, _i32p]
@@ -138,6 +144,28 @@ def project(gamma, d, seed):
     n, P = gamma.shape
     y = np.empty((n, d), np.float32)
     lib().qlo_project(_p(gamma, _f32p), n, P, d, int(seed), _p(y, _f32p))
+    return y
+
+
+def gaussian_entry_exact(seed, r, j):
+    """Entry z_{r,j} of the Gaussian matrix before its rounding to bf16 (float64)."""
+    return float(lib().qlo_gaussian_entry_exact(int(seed), int(r), int(j)))
+
+
+def gaussian_rows(seed, r0, nr, j0, nj):
+    """fp32 [nr, nj]: the bf16-rounded entries z_{r,j} for r in [r0, r0+nr), j in [j0, j0+nj)."""
+    out = np.empty((nr, nj), np.float32)
+    for a in range(nr):
+        lib().qlo_gaussian_row(int(seed), int(r0 + a), int(j0), int(nj), _p(out[a], _f32p))
+    return out
+
+
+def project_gaussian(gamma, d, seed):
+    """Eq. 1 with the Gaussian matrix: fp32 [n, d]."""
+    gamma = _c(gamma, np.float32)
+    n, P = gamma.shape
+    y = np.empty((n, d), np.float32)
+    lib().qlo_project_gaussian(_p(gamma, _f32p), n, P, d, int(seed), _p(y, _f32p))
     return y
 
 

@@ -17,8 +17,9 @@
  * Pins (what fixes each function independently of this file) live in
  * tests/test_oracle_pins.py.
  *
- * Parity unpinned: the Adam hyper-parameters (beta1, beta2, eps) and the map
- * from a Philox output bit to a matrix entry are conventions of this library,
+ * Parity unpinned: the Adam hyper-parameters (beta1, beta2, eps) and the maps
+ * from Philox output to a matrix entry (Rademacher bit, Gaussian pair) are
+ * conventions of this library,
  * not statements of the paper; the paper cannot pin them. Everything else has
  * at least one pin.
  *
@@ -201,6 +202,67 @@ void qlo_project_rows(const float* gamma, int64_t n, int64_t P, int32_t d, uint6
         }
     }
     free(s);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Gaussian projection matrix (the other distribution Sec. 2.4 allows for R): */
+/* R_rj = z_rj / sqrt(d), z_rj ~ N(0, 1), again a pure function of            */
+/* (seed, r, j) and never stored.                                             */
+/*                                                                            */
+/* Entry map (library convention): the four entries j = 4q .. 4q+3 of row r   */
+/* come from ONE Philox call with                                             */
+/*     counter = (q mod 2^32, r, q div 2^32, 1),  key = seed as above         */
+/* (the last counter word keeps this stream apart from the Rademacher one).   */
+/* Output words (w0, w1) give entries 4q, 4q+1 and (w2, w3) give 4q+2, 4q+3   */
+/* by the Box-Muller transform (Box and Muller, Ann. Math. Statist. 1958):    */
+/*     u1 = (floor(wa / 2^9) + 1/2) / 2^23,  u2 = (floor(wb / 2^9) + 1/2) / 2^23 */
+/*     z_even = sqrt(-2 ln u1) cos(2 pi u2),  z_odd = sqrt(-2 ln u1) sin(2 pi u2) */
+/* (both uniforms lie strictly inside (0, 1) and are exact in binary32).      */
+/* The entry that enters the contraction is z rounded to bf16, because the    */
+/* projection multiplies bf16 operands.                                       */
+/* ------------------------------------------------------------------------- */
+
+/* The entry before rounding, in double. */
+double qlo_gaussian_entry_exact(uint64_t seed, uint32_t r, uint64_t j)
+{
+    uint64_t q = j >> 2;
+    uint32_t ctr[4] = { (uint32_t)(q & 0xFFFFFFFFu), r, (uint32_t)(q >> 32), 1u };
+    uint32_t key[2] = { (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32) };
+    uint32_t w[4];
+    qlo_philox4x32_10(ctr, key, w);
+    uint32_t wa = (j & 2u) ? w[2] : w[0];
+    uint32_t wb = (j & 2u) ? w[3] : w[1];
+    double u1 = ((double)(wa >> 9) + 0.5) / 8388608.0;
+    double u2 = ((double)(wb >> 9) + 0.5) / 8388608.0;
+    double rho = sqrt(-2.0 * log(u1));
+    double ang = 2.0 * 3.14159265358979323846 * u2;
+    return (j & 1u) ? rho * sin(ang) : rho * cos(ang);
+}
+
+/* Entries of row r for columns j0 .. j0+nj-1 as they enter the contraction:  */
+/* fp32 holding bf16-representable values.                                    */
+void qlo_gaussian_row(uint64_t seed, uint32_t r, uint64_t j0, uint64_t nj, float* out)
+{
+    for (uint64_t i = 0; i < nj; ++i)
+        out[i] = qlo_round_to_bf16((float)qlo_gaussian_entry_exact(seed, r, j0 + i));
+}
+
+/* Eq. 1 with the Gaussian matrix: y_r = (sum_j Gamma_j z_rj) / sqrt(d), the   */
+/* sum in double over j ascending, the scale the fp32 value of 1/sqrt(d).     */
+void qlo_project_gaussian(const float* gamma, int64_t n, int64_t P, int32_t d, uint64_t seed, float* y)
+{
+    float* z = (float*)malloc(sizeof(float) * (size_t)P);
+    float inv_sqrt_d = 1.0f / sqrtf((float)d);
+    for (int32_t r = 0; r < d; ++r) {
+        qlo_gaussian_row(seed, (uint32_t)r, 0, (uint64_t)P, z);
+        for (int64_t i = 0; i < n; ++i) {
+            const float* gi = gamma + i * P;
+            double acc = 0.0;
+            for (int64_t j = 0; j < P; ++j) acc += (double)gi[j] * (double)z[j];
+            y[i * (int64_t)d + r] = (float)(acc * (double)inv_sqrt_d);
+        }
+    }
+    free(z);
 }
 
 /* ------------------------------------------------------------------------- */

@@ -602,3 +602,79 @@ def test_absmean_keeps_more_nonzero_codes_than_absmax_at_low_width():
     nz = np.mean([np.count_nonzero(oracle.unpack(cm[r], 8192, 2)) for r in range(8)]) / 8192
     assert abs(nz - 0.690) < 0.01
 
+
+
+# ----------------------------------------------------------------------------------------------
+# Gaussian projection matrix (the other distribution Sec. 2.4 allows): parity unpinned as far as
+# the Philox-to-entry map goes (a convention); the transform and the distribution are pinned here
+# ----------------------------------------------------------------------------------------------
+
+def test_gaussian_entries_are_the_box_muller_images_of_their_philox_words():
+    # invert the transform: z_even^2 + z_odd^2 = -2 ln u1 and atan2(z_odd, z_even) = 2 pi u2, with u1, u2
+    # rebuilt here from the Philox words of the block's own counter (catches swapped words, sin/cos, a
+    # missing factor 2 or pi, a wrong counter word)
+    seed = 0xFEED_0000_BEEF
+    key = [seed & 0xFFFFFFFF, seed >> 32]
+    for r in (0, 5, 4095):
+        for q in (0, 1, 1000, 2 ** 32 + 3):
+            w = [int(x) for x in oracle.philox4x32_10([q % 2 ** 32, r, q >> 32, 1], key)]
+            z = [oracle.gaussian_entry_exact(seed, r, 4 * q + t) for t in range(4)]
+            for (wa, wb, ze, zo) in ((w[0], w[1], z[0], z[1]), (w[2], w[3], z[2], z[3])):
+                u1 = ((wa >> 9) + 0.5) / 2 ** 23
+                u2 = ((wb >> 9) + 0.5) / 2 ** 23
+                assert 0.0 < u1 < 1.0 and 0.0 < u2 < 1.0
+                assert math.isclose(ze * ze + zo * zo, -2.0 * math.log(u1), rel_tol=1e-12)
+                ang = math.atan2(zo, ze) % (2 * math.pi)
+                assert math.isclose(ang, 2 * math.pi * u2, rel_tol=0, abs_tol=1e-9)
+    # the row generator returns the same entries rounded to bf16 (torch's rounding)
+    row = oracle.gaussian_rows(seed, 7, 1, 8, 64)[0]
+    want = torch.tensor([oracle.gaussian_entry_exact(seed, 7, 8 + i) for i in range(64)],
+                        dtype=torch.float32).to(torch.bfloat16).float().numpy()
+    assert np.array_equal(row, want)
+
+
+def test_gaussian_entries_follow_the_standard_normal_law():
+    from scipy import stats
+    seed = 2025
+    z = np.array([[oracle.gaussian_entry_exact(seed, r, j) for j in range(4096)] for r in range(16)])
+    flat = z.reshape(-1)                                # 65 536 entries
+    n = flat.size
+    assert abs(flat.mean()) <= 5 / math.sqrt(n)
+    assert abs(flat.var() - 1.0) <= 5 * math.sqrt(2.0 / n)
+    assert abs((flat ** 4).mean() - 3.0) <= 5 * math.sqrt(96.0 / n)
+    assert stats.kstest(flat, "norm").pvalue > 1e-3
+    # even and odd entries (the cosine and the sine branch) separately, and their independence
+    assert stats.kstest(flat[0::2], "norm").pvalue > 1e-3
+    assert stats.kstest(flat[1::2], "norm").pvalue > 1e-3
+    assert abs(np.corrcoef(flat[0::2], flat[1::2])[0, 1]) <= 5 / math.sqrt(n / 2)
+    # rows are uncorrelated with each other and with the Rademacher matrix of the same seed
+    c = np.corrcoef(z)
+    assert np.abs(c - np.eye(16)).max() <= 5 / math.sqrt(4096)
+    s = oracle.rademacher_rows(seed, 0, 16, 0, 4096).astype(np.float64)
+    assert np.abs((z * s).mean(1)).max() <= 5 / math.sqrt(4096)
+    # bf16 rounding (8 significand bits) moves an entry by at most half an ulp, under 2^-8 of its size
+    zb = oracle.gaussian_rows(seed, 0, 16, 0, 4096).astype(np.float64)
+    assert np.all(np.abs(zb - z) <= np.abs(z) * 2.0 ** -8)
+
+
+def test_gaussian_projection_basis_vector_matmul_and_jl():
+    P, d, seed, n = 1024, 256, 31, 9
+    # a basis vector returns its column of the matrix, scaled by the fp32 value of 1/sqrt(d)
+    for j in (0, 3, 4, 1023):
+        e = np.zeros((1, P), np.float32)
+        e[0, j] = 1.0
+        y = oracle.project_gaussian(e, d, seed)[0]
+        col = oracle.gaussian_rows(seed, 0, d, j, 1)[:, 0].astype(np.float64)
+        assert np.array_equal(y, (col * float(np.float32(1.0) / np.sqrt(np.float32(d)))).astype(np.float32))
+    # library routine: numpy matmul with the explicitly generated matrix
+    x = oracle.round_to_bf16(workloads.student_t_gradients(n, P, seed=6).numpy())
+    R = oracle.gaussian_rows(seed, 0, d, 0, P).astype(np.float64)
+    want = (x.astype(np.float64) @ R.T) / math.sqrt(d)
+    got = oracle.project_gaussian(x, d, seed).astype(np.float64)
+    assert np.allclose(got, want, rtol=1e-6, atol=1e-6 * np.abs(want).max())
+    # Johnson-Lindenstrauss: ||Rx||^2 / ||x||^2 is chi^2_d / d for a Gaussian matrix: mean 1, s.d. sqrt(2/d)
+    xn = (x.astype(np.float64) ** 2).sum(1)
+    ratio = (got ** 2).sum(1) / xn
+    assert np.all(np.abs(ratio - 1.0) <= 5 * math.sqrt(2.0 / d))
+    ip_x = x.astype(np.float64) @ x.astype(np.float64).T
+    assert np.all(np.abs(got @ got.T - ip_x) <= 5 * np.sqrt(np.outer(xn, xn)) / math.sqrt(d))
