@@ -407,6 +407,28 @@ def stage_measurements(torch, B, W, dev, peaks):
     t = _time_ms(torch, lambda: B.qless_select_topk(s, 0.05, indices=idx, workspace=wsel), 3)
     out["select_2^28_top5pct"] = dict(ms=t, gbs_algorithmic=4.0 * N / t / 1e6, frac_of_hbm=4.0 * N / t / 1e6 / peaks["hbm_gbs"],
                                       note="algorithmic bytes = 4N (every score read once)")
+    del s, idx, wsel
+    # ---- projection with the Gaussian matrix (the distribution Sec. 2.4 names beside Rademacher) ----
+    n, P = 256, 1 << 20
+    g = W.student_t_gradients(n, P, seed=SEED + 600, device=dev, dtype=torch.bfloat16)
+    ws = torch.empty(B.qless_project_quantize_workspace(n, P, d, 4), dtype=torch.uint8, device=dev)
+    pq = {}
+    for name, kind in (("rademacher", B.RADEMACHER), ("gaussian", B.GAUSSIAN)):
+        B.qless_set_projection_matrix(kind)
+        try:
+            B.qless_profile_collect()
+            B.qless_profile_enable(True)
+            for _ in range(4):
+                B.qless_project_quantize(g, d, SEED, 4, workspace=ws)
+            torch.cuda.synchronize()
+            prof = B.qless_profile_collect()
+        finally:
+            B.qless_profile_enable(False)
+            B.qless_set_projection_matrix(B.RADEMACHER)
+        t = prof["project"][0] / prof["project"][1]
+        pq[name] = dict(ms=t, tflops=2.0 * n * P * d / t / 1e9, grads_per_s=n / (t * 1e-3))
+    pq["note"] = "projection kernel alone, 256 bf16 rows, P = 2^20; the Gaussian matrix is bounded by its generator warps"
+    out["project_256x2^20_by_matrix"] = pq
     B.qless_check()
     return out
 

@@ -187,6 +187,26 @@ qless_status qless_adam_gamma(
 qless_status qless_philox_entries(
     uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj, int8_t* out, void* cuda_stream);
 
+/* Which random matrix R the projection of Eq. 1 uses in qless_project_quantize and
+ * qless_project_quantize_host (Sec. 2.4 leaves the distribution open between Gaussian and Rademacher).
+ * QLESS_MATRIX_RADEMACHER (default): entries +-1/sqrt(d), entry map above. QLESS_MATRIX_GAUSSIAN: entries
+ * z/sqrt(d) with z standard normal, rounded to bf16 (the operand type of the contraction): the four entries of
+ * row r in columns 4q .. 4q+3 come from one Philox4x32-10 call with counter (q mod 2^32, r, q div 2^32, 1) and
+ * the same key; output words (w0, w1) give columns 4q, 4q+1 and (w2, w3) give 4q+2, 4q+3 by the Box-Muller
+ * transform z_even = sqrt(-2 ln u1) cos(2 pi u2), z_odd = sqrt(-2 ln u1) sin(2 pi u2) with
+ * u = (floor(w / 2^9) + 1/2) / 2^23. The logarithm, square root, sine and cosine are evaluated in fp32, so an
+ * entry may differ from the correctly rounded one by one bf16 step where it falls next to a rounding boundary.
+ * The generator, not the tensor pipe, bounds this variant (about 100 times the instructions per entry).
+ * Process-wide; stores built with different matrices (or seeds) must not be scored against each other.
+ * Returns QLESS_ERR_INVALID_ARG for any other value. */
+enum { QLESS_MATRIX_RADEMACHER = 0, QLESS_MATRIX_GAUSSIAN = 1 };
+qless_status qless_set_projection_matrix(int32_t kind);
+
+/* Entries of the Gaussian matrix as the kernels generate them: out [nr, nj] fp32 (device; bf16-representable
+ * values of sqrt(d) R) for rows r0 .. r0+nr-1 and columns j0 .. j0+nj-1; j0 must be a multiple of 4. */
+qless_status qless_gaussian_entries(
+    uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj, float* out, void* cuda_stream);
+
 /* ------------------------------------------------------------------------------------------
  * Stage 3: influence scores over the quantised datastore (paper Eq. 6-7; aggregation as in LESS,
  * which the paper follows when it accumulates influence over the validation data, Sec. 4.1).

@@ -25,7 +25,9 @@ EXPORTS = [
     "qless_project_quantize_host_workspace", "qless_project_quantize_host", "qless_profile_enable",
     "qless_profile_collect", "qless_kernel_launches", "qless_select_topk_static",
     "qless_set_projection_path", "qless_set_score_path", "qless_set_select_path", "qless_microbench",
+    "qless_set_projection_matrix", "qless_gaussian_entries",
 ]
+RADEMACHER, GAUSSIAN = 0, 1
 SELECT_STATIC_MAX_N = 1 << 22
 
 
@@ -107,6 +109,10 @@ def lib():
         L.qless_set_select_path.argtypes = [i32]
         L.qless_set_projection_path.restype = C.c_int
         L.qless_set_projection_path.argtypes = [i32]
+        L.qless_set_projection_matrix.restype = C.c_int
+        L.qless_set_projection_matrix.argtypes = [i32]
+        L.qless_gaussian_entries.restype = C.c_int
+        L.qless_gaussian_entries.argtypes = [C.c_uint64, i64, i64, i64, i64, vp, vp]
         L.qless_select_topk_static.restype = C.c_int
         L.qless_select_topk_static.argtypes = [vp, i64, C.c_double, vp, C.POINTER(i64), vp]
         _lib = L
@@ -269,6 +275,12 @@ def qless_philox_entries(seed, r0, nr, j0, nj, device="cuda", stream=None):
     return out
 
 
+def qless_gaussian_entries(seed, r0, nr, j0, nj, device="cuda", stream=None):
+    out = torch.empty((nr, nj), dtype=torch.float32, device=device)
+    _check(lib().qless_gaussian_entries(seed, r0, nr, j0, nj, _ptr(out), _stream(stream)))
+    return out
+
+
 def qless_score_workspace(N, V, Cn, T, d, bits):
     return int(lib().qless_score_workspace(N, V, Cn, T, d, bits))
 
@@ -378,6 +390,11 @@ def qless_select_topk_static(scores, frac, indices, stream=None):
 def qless_set_projection_path(path):
     """0 = tensor-core projection kernel (default), 1 = CUDA-core cross-check kernel."""
     _check(lib().qless_set_projection_path(int(path)))
+
+
+def qless_set_projection_matrix(kind):
+    """RADEMACHER (0, default: the method's matrix) or GAUSSIAN (1): the random matrix of the projection."""
+    _check(lib().qless_set_projection_matrix(int(kind)))
 
 
 def qless_set_select_path(path):

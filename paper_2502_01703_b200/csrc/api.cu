@@ -83,6 +83,7 @@ ProfileScope::~ProfileScope()
 
 static std::atomic<int> g_score_path{0};        // 0 = tensor cores for 8/4/2-bit codes, 1 = CUDA cores
 static std::atomic<int> g_projection_path{0};   // 0 = tensor cores, 1 = CUDA cores (cross-check hook)
+static std::atomic<int> g_projection_matrix{0}; // 0 = Rademacher (the method), 1 = Gaussian
 
 static bool valid_bits(int b) { return b == 1 || b == 2 || b == 4 || b == 8; }
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -150,6 +151,7 @@ static qless_status project_columns(const void* grads, qless_dtype dtype, int64_
                                        ap, len, gamma_slab, true, st)); }
     ProjectPlan pl = full;
     pl.P = len; pl.k_base = j0;
+    pl.gaussian = (g_projection_matrix == 1);
     pl.num_chunks = (int32_t)((len + full.chunk - 1) / full.chunk);
     float* part_slab = part + (j0 / full.chunk) * n * (int64_t)full.d;
     if (g_projection_path == 0 && (len / 64) * n < ((int64_t)1 << 31)) {
@@ -209,6 +211,27 @@ qless_status qless_set_projection_path(int32_t path)
 {
     QLESS_REQUIRE(path == 0 || path == 1, QLESS_ERR_INVALID_ARG, "path must be 0 (tensor cores) or 1 (CUDA cores)");
     g_projection_path.store(path);
+    return QLESS_OK;
+}
+
+qless_status qless_set_projection_matrix(int32_t kind)
+{
+    QLESS_REQUIRE(kind == QLESS_MATRIX_RADEMACHER || kind == QLESS_MATRIX_GAUSSIAN, QLESS_ERR_INVALID_ARG,
+                  "kind must be QLESS_MATRIX_RADEMACHER (0) or QLESS_MATRIX_GAUSSIAN (1)");
+    g_projection_matrix.store(kind);
+    return QLESS_OK;
+}
+
+qless_status qless_gaussian_entries(uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj, float* out,
+                                    void* cuda_stream)
+{
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    QLESS_REQUIRE(r0 >= 0 && nr >= 0 && j0 >= 0 && nj >= 0, QLESS_ERR_INVALID_ARG, "negative range");
+    QLESS_REQUIRE(j0 % 4 == 0, QLESS_ERR_INVALID_ARG, "j0 must be a multiple of 4 (j0=%lld)", (long long)j0);
+    QLESS_REQUIRE(r0 + nr <= ((int64_t)1 << 32) && j0 + nj <= ((int64_t)1 << 39), QLESS_ERR_UNSUPPORTED, "row < 2^32 and column < 2^39 required");
+    if (nr == 0 || nj == 0) return QLESS_OK;
+    QLESS_REQUIRE(out != nullptr, QLESS_ERR_INVALID_ARG, "out is NULL");
+    QLESS_CUDA_TRY(launch_gaussian_entries(seed, r0, nr, j0, nj, out, st));
     return QLESS_OK;
 }
 

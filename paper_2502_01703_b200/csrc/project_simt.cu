@@ -10,6 +10,7 @@ constexpr int PS_DR = 64;     // projected rows per block
 constexpr int PS_GR = 32;     // gradient rows per block
 constexpr int PS_T = 256;
 
+template <bool GAUSS>
 __global__ void __launch_bounds__(PS_T)
 project_simt_kernel(const __nv_bfloat16* __restrict__ gamma, int64_t n, int64_t P, int32_t d,
                     int64_t chunk, uint32_t kblk_base, uint64_t seed, float* __restrict__ part)
@@ -40,26 +41,42 @@ project_simt_kernel(const __nv_bfloat16* __restrict__ gamma, int64_t n, int64_t 
             *reinterpret_cast<float2*>(&s_g[row][2 * cp]) = f;
         }
         __syncthreads();
+        const uint32_t blk = kblk_base + (uint32_t)(kb >> 7);
         uint32_t w[4];
-        rademacher_block(seed, r, kblk_base + (uint32_t)(kb >> 7), w);
+        if (!GAUSS) rademacher_block(seed, r, blk, w);
 #pragma unroll
         for (int wi = 0; wi < 4; ++wi) {
-#pragma unroll
+#pragma unroll 2
             for (int q = 0; q < 8; ++q) {               // 4 columns at a time
-                uint32_t sm[4];
+                if (GAUSS) {
+                    uint32_t lo, hi;
+                    gaussian_quad_bf16x2(seed, r, (blk << 5) | (uint32_t)(wi * 8 + q), blk >> 27, lo, hi);
+                    const float z0 = __uint_as_float(lo << 16), z1 = __uint_as_float(lo & 0xFFFF0000u);
+                    const float z2 = __uint_as_float(hi << 16), z3 = __uint_as_float(hi & 0xFFFF0000u);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int u = q * 4 + c;
-                    const int beta = 15 - (u >> 1) + 16 * (u & 1);
-                    sm[c] = ((w[wi] >> beta) & 1u) << 31;
-                }
+                    for (int u = 0; u < 8; ++u) {
+                        const float4 g = *reinterpret_cast<const float4*>(&s_g[ti * 8 + u][wi * 32 + q * 4]);
+                        acc[u] = fmaf(g.x, z0, acc[u]);
+                        acc[u] = fmaf(g.y, z1, acc[u]);
+                        acc[u] = fmaf(g.z, z2, acc[u]);
+                        acc[u] = fmaf(g.w, z3, acc[u]);
+                    }
+                } else {
+                    uint32_t sm[4];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const float4 g = *reinterpret_cast<const float4*>(&s_g[ti * 8 + u][wi * 32 + q * 4]);
-                    acc[u] += __uint_as_float(__float_as_uint(g.x) ^ sm[0]);
-                    acc[u] += __uint_as_float(__float_as_uint(g.y) ^ sm[1]);
-                    acc[u] += __uint_as_float(__float_as_uint(g.z) ^ sm[2]);
-                    acc[u] += __uint_as_float(__float_as_uint(g.w) ^ sm[3]);
+                    for (int c = 0; c < 4; ++c) {
+                        const int u = q * 4 + c;
+                        const int beta = 15 - (u >> 1) + 16 * (u & 1);
+                        sm[c] = ((w[wi] >> beta) & 1u) << 31;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const float4 g = *reinterpret_cast<const float4*>(&s_g[ti * 8 + u][wi * 32 + q * 4]);
+                        acc[u] += __uint_as_float(__float_as_uint(g.x) ^ sm[0]);
+                        acc[u] += __uint_as_float(__float_as_uint(g.y) ^ sm[1]);
+                        acc[u] += __uint_as_float(__float_as_uint(g.z) ^ sm[2]);
+                        acc[u] += __uint_as_float(__float_as_uint(g.w) ^ sm[3]);
+                    }
                 }
             }
         }
@@ -80,7 +97,7 @@ ProjectPlan plan_projection(int64_t n, int64_t P, int32_t d)
     // of fp32 accumulations never exceeds 4096 tensor-core steps), the largest that still gives every SM
     // about four work items of (256 gradient rows x 128 projected coordinates x chunk).
     ProjectPlan pl;
-    pl.n = n; pl.P = P; pl.d = d; pl.k_base = 0;
+    pl.n = n; pl.P = P; pl.d = d; pl.k_base = 0; pl.gaussian = false;
     const int64_t tiles = (int64_t)(d / 128) * ((n + 255) / 256);
     int64_t chunk = 65536;
     while (chunk > 1024 && tiles * ((P + chunk - 1) / chunk) < 4 * (int64_t)sm_count()) chunk >>= 1;
@@ -95,7 +112,10 @@ cudaError_t launch_project_simt(const __nv_bfloat16* gamma, const ProjectPlan& p
 {
     if (pl.n == 0) return cudaSuccess;
     dim3 grid((unsigned)(pl.d / PS_DR), (unsigned)((pl.n + PS_GR - 1) / PS_GR), (unsigned)pl.num_chunks);
-    project_simt_kernel<<<grid, PS_T, 0, st>>>(gamma, pl.n, pl.P, pl.d, pl.chunk, (uint32_t)(pl.k_base >> 7), seed, part);
+    if (pl.gaussian)
+        project_simt_kernel<true><<<grid, PS_T, 0, st>>>(gamma, pl.n, pl.P, pl.d, pl.chunk, (uint32_t)(pl.k_base >> 7), seed, part);
+    else
+        project_simt_kernel<false><<<grid, PS_T, 0, st>>>(gamma, pl.n, pl.P, pl.d, pl.chunk, (uint32_t)(pl.k_base >> 7), seed, part);
     count_launches(1);
     return cudaGetLastError();
 }

@@ -48,6 +48,9 @@ struct __align__(8) Barriers {
 
 constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)SB * B_STAGE_BYTES + sizeof(Barriers);
 
+// GAUSS = false: the Rademacher matrix of the method; true: Gaussian entries (Box-Muller on Philox words, bf16),
+// which cost the generator warps about a hundred times more instructions per entry.
+template <bool GAUSS>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int32_t d, int64_t P, int64_t chunk,
                   int32_t num_chunks, uint32_t kblk_base, uint64_t seed, float* __restrict__ part,
@@ -171,19 +174,35 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
             for (int ka = 0; ka < nka; ++ka, ++ita) {
                 if ((ita & 1u) != grp) continue;
                 const int sa = ita % SA;
-                uint32_t w[4];
-                rademacher_block(seed, r, kblk_base + (uint32_t)((k0 >> 7) + ka), w);     // overlaps with the wait below
-                ok = mbar_wait_cluster(smem_u32(&bars->a_empty[sa]), ((ita / SA) & 1u) ^ 1u, abort_flag, timeout_word, TO_GENERATOR);
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) break;
-                tc_fence_after();
+                const uint32_t blk = kblk_base + (uint32_t)((k0 >> 7) + ka);      // 128-column block of the matrix
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + A_COL + sa * 64;
+                if constexpr (GAUSS) {
+                    uint32_t v[4][16];                                            // generated before the slot is waited for
 #pragma unroll
-                for (int wi = 0; wi < 4; ++wi) {
-                    uint32_t v[16];
+                    for (int wi = 0; wi < 4; ++wi)
 #pragma unroll
-                    for (int p = 0; p < 16; ++p) v[p] = rademacher_bf16x2(w[wi], p);
-                    tmem_st_x16(taddr + wi * 16, v);
+                        for (int c = 0; c < 8; ++c)
+                            gaussian_quad_bf16x2(seed, r, (blk << 5) | (uint32_t)(wi * 8 + c), blk >> 27, v[wi][2 * c], v[wi][2 * c + 1]);
+                    ok = mbar_wait_cluster(smem_u32(&bars->a_empty[sa]), ((ita / SA) & 1u) ^ 1u, abort_flag, timeout_word, TO_GENERATOR);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int wi = 0; wi < 4; ++wi) tmem_st_x16(taddr + wi * 16, v[wi]);
+                } else {
+                    uint32_t w[4];
+                    rademacher_block(seed, r, blk, w);     // overlaps with the wait below
+                    ok = mbar_wait_cluster(smem_u32(&bars->a_empty[sa]), ((ita / SA) & 1u) ^ 1u, abort_flag, timeout_word, TO_GENERATOR);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int wi = 0; wi < 4; ++wi) {
+                        uint32_t v[16];
+#pragma unroll
+                        for (int p = 0; p < 16; ++p) v[p] = rademacher_bf16x2(w[wi], p);
+                        tmem_st_x16(taddr + wi * 16, v);
+                    }
                 }
                 tmem_wait_st();
                 tc_fence_before();
@@ -241,13 +260,18 @@ cudaError_t launch_project_tc(const CUtensorMap& tmap, const ProjectPlan& pl, ui
                               unsigned int* timeout_word, cudaStream_t st)
 {
     if (pl.n == 0) return cudaSuccess;
-    cudaError_t e = cudaFuncSetAttribute(project_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(pl.gaussian ? project_tc_kernel<true> : project_tc_kernel<false>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
     if (e != cudaSuccess) return e;
     const int64_t items = (int64_t)((pl.n + BN - 1) / BN) * pl.num_chunks * ((pl.d + 2 * BM - 1) / (2 * BM));
     int64_t grid = (sm_count() / 2) * 2;               // CTA pairs
     if (grid > 2 * items) grid = 2 * items;
-    project_tc_kernel<<<(unsigned)grid, NTHREADS, SMEM_BYTES, st>>>(tmap, pl.n, pl.d, pl.P, pl.chunk, pl.num_chunks,
-                                                                    (uint32_t)(pl.k_base >> 7), seed, part, timeout_word);
+    if (pl.gaussian)
+        project_tc_kernel<true><<<(unsigned)grid, NTHREADS, SMEM_BYTES, st>>>(tmap, pl.n, pl.d, pl.P, pl.chunk, pl.num_chunks,
+                                                                              (uint32_t)(pl.k_base >> 7), seed, part, timeout_word);
+    else
+        project_tc_kernel<false><<<(unsigned)grid, NTHREADS, SMEM_BYTES, st>>>(tmap, pl.n, pl.d, pl.P, pl.chunk, pl.num_chunks,
+                                                                               (uint32_t)(pl.k_base >> 7), seed, part, timeout_word);
     count_launches(1);
     return cudaGetLastError();
 }

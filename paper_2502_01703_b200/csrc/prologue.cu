@@ -168,4 +168,37 @@ cudaError_t launch_philox_entries(uint64_t seed, int64_t r0, int64_t nr, int64_t
     return cudaGetLastError();
 }
 
+// out[a][b] = z(r0 + a, j0 + b) of the Gaussian matrix, as fp32 (values are bf16-representable). One thread per
+// group of four columns; j0 is a multiple of 4.
+__global__ void gaussian_entries_kernel(uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj,
+                                        float* __restrict__ out)
+{
+    const int64_t quads = (nj + 3) / 4;
+    const int64_t total = nr * quads;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t a = idx / quads, b = idx - a * quads;
+        const uint64_t q = (uint64_t)(j0 >> 2) + (uint64_t)b;
+        uint32_t lo, hi;
+        gaussian_quad_bf16x2(seed, (uint32_t)(r0 + a), (uint32_t)q, (uint32_t)(q >> 32), lo, hi);
+        const float z[4] = {__uint_as_float(lo << 16), __uint_as_float(lo & 0xFFFF0000u),
+                            __uint_as_float(hi << 16), __uint_as_float(hi & 0xFFFF0000u)};
+        for (int t = 0; t < 4; ++t)
+            if (4 * b + t < nj) out[a * nj + 4 * b + t] = z[t];
+    }
+}
+
+cudaError_t launch_gaussian_entries(uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj, float* out,
+                                    cudaStream_t st)
+{
+    const int64_t total = nr * ((nj + 3) / 4);
+    if (total == 0) return cudaSuccess;
+    int64_t blocks = (total + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 16;
+    if (blocks > cap) blocks = cap;
+    gaussian_entries_kernel<<<(unsigned)blocks, 256, 0, st>>>(seed, r0, nr, j0, nj, out);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
 }  // namespace qless

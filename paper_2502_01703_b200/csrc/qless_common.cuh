@@ -83,6 +83,33 @@ __host__ __device__ __forceinline__ int rademacher_sign_of(uint32_t word, int u)
     return ((word >> beta) & 1u) ? -1 : 1;
 }
 
+// Gaussian matrix (the other distribution Sec. 2.4 allows): the four entries of row r in columns 4q .. 4q+3 come
+// from one Philox call with counter (q mod 2^32, r, q div 2^32, 1); output words (w0, w1) give columns 4q, 4q+1 and
+// (w2, w3) give 4q+2, 4q+3 by the Box-Muller transform of u = (floor(w / 2^9) + 1/2) / 2^23 (exact in fp32,
+// strictly inside (0, 1)): z_even = sqrt(-2 ln u1) cos(2 pi u2), z_odd = sqrt(-2 ln u1) sin(2 pi u2). The entries
+// are rounded to bf16, the operand type of the contraction; lo packs columns 4q, 4q+1 (4q in the low half),
+// hi packs 4q+2, 4q+3.
+#ifdef __CUDACC__
+__device__ __forceinline__ uint32_t box_muller_bf16x2(uint32_t wa, uint32_t wb)
+{
+    const float u1 = ((float)(wa >> 9) + 0.5f) * 1.1920928955078125e-07f;        // 2^-23
+    const float two_u2 = ((float)(wb >> 9) + 0.5f) * 2.384185791015625e-07f;     // 2^-22
+    const float rho = sqrtf(-2.0f * logf(u1));
+    float sn, cs;
+    sincospif(two_u2, &sn, &cs);
+    const __nv_bfloat162 z = __floats2bfloat162_rn(rho * cs, rho * sn);
+    return *reinterpret_cast<const uint32_t*>(&z);
+}
+__device__ __forceinline__ void gaussian_quad_bf16x2(uint64_t seed, uint32_t r, uint32_t q_lo, uint32_t q_hi,
+                                                     uint32_t& lo, uint32_t& hi)
+{
+    uint32_t w[4];
+    philox4x32_10(q_lo, r, q_hi, 1u, (uint32_t)seed, (uint32_t)(seed >> 32), w);
+    lo = box_muller_bf16x2(w[0], w[1]);
+    hi = box_muller_bf16x2(w[2], w[3]);
+}
+#endif
+
 // Order-preserving key of an fp32 score: larger key <=> larger score; -0 < +0; NaN lowest.
 __host__ __device__ __forceinline__ uint32_t order_key(uint32_t bits)
 {

@@ -21,6 +21,9 @@ cudaError_t launch_adam_gamma(const void* grads, qless_dtype dtype, int64_t n, i
 
 cudaError_t launch_philox_entries(uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj,
                                   int8_t* out, cudaStream_t st);
+// Entries of the Gaussian matrix as fp32 (bf16-representable values); j0 a multiple of 4.
+cudaError_t launch_gaussian_entries(uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj,
+                                    float* out, cudaStream_t st);
 
 // Projection partial sums: part[s][i][r] = sum over K-chunk s of Gamma[i][j] * sign(r, j), fp32,
 // s = 0 .. num_chunks-1, chunk s covering columns [s*chunk, min(P, (s+1)*chunk)).
@@ -30,6 +33,7 @@ struct ProjectPlan {
     int64_t chunk;        // K-chunk length (multiple of 128)
     int32_t num_chunks;
     int64_t k_base;       // absolute index of the first column given (a multiple of chunk): offsets the Philox counters
+    bool gaussian;        // entries of R: false = Rademacher +-1 (the method), true = standard normal (bf16)
 };
 ProjectPlan plan_projection(int64_t n, int64_t P, int32_t d);
 cudaError_t launch_project_simt(const __nv_bfloat16* gamma_tiled, const ProjectPlan& pl,

@@ -224,6 +224,85 @@ def test_projection_is_deterministic_and_handles_empty_batch():
 
 
 # ----------------------------------------------------------------------------------------------
+# Gaussian projection matrix (the other distribution Sec. 2.4 allows for R)
+# ----------------------------------------------------------------------------------------------
+
+@pytest.fixture
+def gaussian_matrix():
+    B.qless_set_projection_matrix(B.GAUSSIAN)
+    try:
+        yield
+    finally:
+        B.qless_set_projection_matrix(B.RADEMACHER)
+        B.qless_set_projection_path(0)
+
+
+@pytest.mark.parametrize("seed,r0,nr,j0,nj", [
+    (0, 0, 8, 0, 512), (0x9E3779B97F4A7C15, 5, 3, 120, 301), (42, 8190, 2, (1 << 23) - 200, 200),
+    (7, 0, 1, 4, 1), (7, 100, 130, 64, 130), (3, 1, 2, (1 << 36) + 8, 64),
+])
+def test_gaussian_entries_match_oracle(seed, r0, nr, j0, nj):
+    # The device evaluates ln, sqrt, sin and cos in fp32, the oracle in fp64: an entry may land on the other side
+    # of a bf16 rounding boundary. Such entries must be rare and differ by exactly one bf16 step; all others are
+    # bit-identical.
+    got = _np(B.qless_gaussian_entries(seed, r0, nr, j0, nj))
+    want = oracle.gaussian_rows(seed, r0, nr, j0, nj)
+    gb = (got.view(np.uint32) >> 16).astype(np.int64)
+    wb = (want.view(np.uint32) >> 16).astype(np.int64)
+    assert np.all((got.view(np.uint32) & 0xFFFF) == 0)          # bf16-representable
+    diff = np.abs(gb - wb)
+    assert diff.max() <= 1
+    assert (diff != 0).sum() <= max(1, int(2e-3 * got.size)), (int((diff != 0).sum()), got.size)
+
+
+@pytest.mark.parametrize("n,P,d,dtype,use_adam", [
+    (37, 1024, 256, torch.float32, True),
+    (300, 4096, 128, torch.bfloat16, True),
+    (5, 2048 + 128, 512, torch.bfloat16, False),
+    (64, 1 << 16, 256, torch.bfloat16, True),
+])
+def test_gaussian_projection_matches_oracle(gaussian_matrix, n, P, d, dtype, use_adam):
+    seed = 0xBADC0DE
+    g = W.student_t_gradients(n, P, seed=44, device=DEV, dtype=dtype)
+    m, v = W.adam_moments(P, seed=45, device=DEV)
+    out = B.qless_project_quantize(g, d, seed, 4, m if use_adam else None, v if use_adam else None, want_proj=True)
+    B.qless_check()
+    gamma = oracle.adam_gamma(_np(g.float()), _np(m) if use_adam else None, _np(v) if use_adam else None)
+    want = oracle.project_gaussian(gamma, d, seed)
+    rel_l2, rel_max = _proj_err(_np(out["proj"]), want)
+    assert rel_l2 <= PROJ_TOL and rel_max <= PROJ_TOL, (rel_l2, rel_max)
+    # the integer stages downstream are the same kernels: oracle quantiser on the GPU's own projection
+    wc, ws, _ = oracle.quantize_rows(_np(out["proj"]), 4, normalize=True)
+    assert (_np(out["codes"]) == wc).all(axis=1).sum() >= n - 1
+    assert np.allclose(_np(out["scales"]), ws, rtol=3e-7)
+    # the CUDA-core kernel generates the same entries: only the fp32 summation order differs
+    B.qless_set_projection_path(1)
+    ref = B.qless_project_quantize(g, d, seed, 4, m if use_adam else None, v if use_adam else None, want_proj=True)
+    e_l2, e_max = _proj_err(_np(out["proj"]), _np(ref["proj"]))
+    assert e_l2 <= 1e-5 and e_max <= 1e-5, (e_l2, e_max)
+
+
+def test_gaussian_projection_of_basis_vectors_and_switch_back(gaussian_matrix):
+    # e_j projects to column j of the matrix the entry hook returns, scaled by the fp32 value of 1/sqrt(d)
+    P, d, seed = 1024, 256, 78
+    js = [0, 1, 2, 3, 127, 128, 1023]
+    g = torch.zeros((len(js), P), dtype=torch.bfloat16, device=DEV)
+    for a, j in enumerate(js):
+        g[a, j] = 1.0
+    proj = _np(B.qless_project_quantize(g, d, seed, 8, want_proj=True)["proj"])
+    for a, j in enumerate(js):
+        col = _np(B.qless_gaussian_entries(seed, 0, d, j - j % 4, 4))[:, j % 4]
+        assert np.array_equal(proj[a], col * np.float32(1.0 / np.sqrt(np.float32(d))))
+    # switching back restores the Rademacher matrix
+    B.qless_set_projection_matrix(B.RADEMACHER)
+    proj = _np(B.qless_project_quantize(g, d, seed, 8, want_proj=True)["proj"])
+    col = oracle.rademacher_rows(seed, 0, d, 0, 1)[:, 0].astype(np.float32)
+    assert np.array_equal(proj[0], col * np.float32(1.0 / np.sqrt(np.float32(d))))
+    with pytest.raises(B.QlessError):
+        B.qless_set_projection_matrix(2)
+
+
+# ----------------------------------------------------------------------------------------------
 # Integer similarity and aggregated scores
 # ----------------------------------------------------------------------------------------------
 
