@@ -92,12 +92,16 @@ __host__ __device__ __forceinline__ int rademacher_sign_of(uint32_t word, int u)
 #ifdef __CUDACC__
 __device__ __forceinline__ uint32_t box_muller_bf16x2(uint32_t wa, uint32_t wb)
 {
-    const float u1 = ((float)(wa >> 9) + 0.5f) * 1.1920928955078125e-07f;        // 2^-23
-    const float two_u2 = ((float)(wb >> 9) + 0.5f) * 2.384185791015625e-07f;     // 2^-22
-    const float rho = sqrtf(-2.0f * logf(u1));
-    float sn, cs;
-    sincospif(two_u2, &sn, &cs);
-    const __nv_bfloat162 z = __floats2bfloat162_rn(rho * cs, rho * sn);
+    // The generator warps bound this variant, so the transform runs on the special-function units: log2, square
+    // root, sine and cosine each one approximate instruction (absolute error about 2^-21 with the angle brought
+    // into (-pi, pi): cos(2 pi u2) = -cos(2 pi (u2 - 1/2)), likewise the sine), well inside half a bf16 step except
+    // for entries that sit next to a rounding boundary.
+    const float u1 = ((float)(wa >> 9) + 0.5f) * 1.1920928955078125e-07f;                 // 2^-23, exact
+    const float t = ((float)((int)(wb >> 9) - (1 << 22)) + 0.5f) * 1.1920928955078125e-07f;   // u2 - 1/2, exact
+    float rho;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rho) : "f"(-2.0f * __logf(u1)));
+    const float ang = 6.283185307179586f * t;
+    const __nv_bfloat162 z = __floats2bfloat162_rn(-rho * __cosf(ang), -rho * __sinf(ang));
     return *reinterpret_cast<const uint32_t*>(&z);
 }
 __device__ __forceinline__ void gaussian_quad_bf16x2(uint64_t seed, uint32_t r, uint32_t q_lo, uint32_t q_hi,

@@ -1,6 +1,6 @@
 """Run one stage of the hot path at a chosen shape on synthetic inputs (for profiling a small case).
 
-    python -m paper_2502_01703_b200.run_case project  --n 256 --P 1048576 --d 8192 --bits 4 --iters 3
+    python -m paper_2502_01703_b200.run_case project  --n 256 --P 1048576 --d 8192 --bits 4 --iters 3   (--matrix gaussian)
     python -m paper_2502_01703_b200.run_case quantize --n 32768 --d 8192 --bits 4
     python -m paper_2502_01703_b200.run_case score    --N 20000 --V 448 --C 4 --d 8192 --bits 8     (16: the bf16 baseline)
     python -m paper_2502_01703_b200.run_case select   --N 67108864 --frac 0.05
@@ -28,9 +28,11 @@ def main():
     ap.add_argument("--frac", type=float, default=0.05)
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--no-adam", action="store_true")
+    ap.add_argument("--matrix", choices=["rademacher", "gaussian"], default="rademacher", help="random matrix of the projection")
     a = ap.parse_args()
     dev = "cuda"
     if a.stage == "project":
+        B.qless_set_projection_matrix(B.GAUSSIAN if a.matrix == "gaussian" else B.RADEMACHER)
         g = W.student_t_gradients(a.n, a.P, seed=1, device=dev, dtype=torch.bfloat16)
         m, v = (None, None) if a.no_adam else W.adam_moments(a.P, seed=2, device=dev)
         ws = torch.empty(B.qless_project_quantize_workspace(a.n, a.P, a.d, a.bits), dtype=torch.uint8, device=dev)
