@@ -248,8 +248,20 @@ def stage_measurements(torch, B, W, dev, peaks):
     popc_peak = ops / ms / 1e9          # T word-ops/s
     ms, ops = B.qless_microbench("bf16_ts_pair", 20000, device=dev)
     bf16_peak = ops / ms / 1e9          # TFLOP/s
+    ms, ops = B.qless_microbench("i8_ss_pair_n448", 20000, device=dev)
+    i8_n448 = ops / ms / 1e9            # Tops/s in the two-MMA shape of 8-bit scoring at 448 validation vectors
+    ms, byts = B.qless_microbench("tma_l2_stream", 20000, device=dev)
+    l2_gbs = byts / ms / 1e6            # GB/s from L2 into shared memory, TMA alone
     out["microbench"] = dict(int8_tops=i8_peak, popc_xor_add_twordops=popc_peak, bf16_tcgen05_tflops=bf16_peak,
-                             note="back-to-back tcgen05.mma / XOR+POPC+IADD on all SMs, burst")
+                             int8_tops_scoring_shape_n448=i8_n448, tma_l2_to_smem_gbs=l2_gbs,
+                             note="back-to-back tcgen05.mma / XOR+POPC+IADD on all SMs, burst; TMA streaming from an L2-resident buffer")
+    # the same int8 micro-benchmark held for about two seconds, clocks sampled: the tensor pipe under the power cap
+    smp = ClockSampler(torch.cuda.current_device())
+    smp.start()
+    ms, ops = B.qless_microbench("i8_ss_pair", 4_000_000, device=dev)
+    ck = smp.stop()
+    i8_sustained = ops / ms / 1e9
+    out["microbench"].update(int8_tops_sustained=i8_sustained, int8_sustained_clocks=ck)
     d = 8192
     # ---- quantise ----
     n = 65536
@@ -300,6 +312,17 @@ def stage_measurements(torch, B, W, dev, peaks):
         iops = 2.0 * N * V * C * d
         e.update(bound="tensor", achieved_tops=iops / t / 1e9, frac_of_int8_peak=iops / t / 1e9 / i8_peak,
                  store_gb=C * (N + V) * (d * b // 8 + 8) / 1e9)
+        # the same call repeated for over a second with the clocks sampled, against the sustained micro-benchmark
+        smp = ClockSampler(torch.cuda.current_device())
+        smp.start()
+        ts_ = _time_ms(torch, lambda: B.qless_score(st["tc"], st["vc"], st["ts"], st["vs"], cfg["lr"], off, d, b,
+                                                    train_sumsq=st["tq"], val_sumsq=st["vq"], scores=sc, workspace=ws), 400, warm=0)
+        ck = smp.stop()
+        e.update(ms_sustained=ts_, frac_of_int8_sustained=iops / ts_ / 1e9 / i8_sustained, sustained_clocks=ck)
+        if ck.get("sm_mhz") and ck.get("sm_max_mhz"):
+            # the micro-benchmark holds the maximum clock (its operands never change, so it draws little power); the
+            # scoring kernel runs under the power cap: its rate against the tensor peak at the clock it actually had
+            e.update(frac_of_int8_peak_at_sustained_clock=iops / ts_ / 1e9 / (i8_sustained * ck["sm_mhz"] / ck["sm_max_mhz"]))
         tops[b] = B.qless_select_topk(sc, cfg["frac"])
         res[str(b)] = e
         if b == 1:

@@ -82,9 +82,15 @@ qless_status qless_profile_collect(char* buf /* host */, size_t buflen);
  * with operands resident on chip: bf16 with both operands in shared memory / bf16 with A in tensor memory /
  * int8; 3 / 4 / 5 = the same three on CTA pairs (cta_group::2); 6 = the XOR + POPC + IADD mix of 1-bit
  * scoring on the integer pipes (scratch: device buffer of >= 8 KiB per SM); 7 = int8 on CTA pairs with A in
- * tensor memory. Runs the kernel twice and times
+ * tensor memory; 8 = int8 on CTA pairs in the shape 8-bit scoring issues for 448 validation vectors (per K step
+ * one MMA of N = 256 and one of N = 192 that re-read the same A from shared memory); 9 = TMA alone streaming
+ * 48 KiB stages from an L2-resident buffer into shared memory on every SM, nothing consuming them (scratch:
+ * 16-byte aligned device buffer of >= 4 MiB, QLESS_ERR_WORKSPACE otherwise); 10 = 8 and 9 together as 8-bit
+ * scoring runs them (the MMAs of one K block committed at once, one 48 KiB stage per K block streamed into other
+ * shared memory three stages ahead, the MMAs never waiting for data; same scratch; operations counted are the
+ * MMAs'); 11 = the kernel of 10 with the copies switched off. Runs the kernel twice and times
  * the second run with CUDA events on `cuda_stream` (synchronises it). *ms_out: milliseconds; *ops_out:
- * operations executed (2 x multiply-accumulates, or word operations for 6). Host pointers. */
+ * operations executed (2 x multiply-accumulates; word operations for 6; bytes moved for 9). Host pointers. */
 qless_status qless_microbench(int32_t what, int32_t iters, float* ms_out, double* ops_out, void* scratch,
                               size_t scratch_bytes, void* cuda_stream);
 

@@ -15,7 +15,8 @@ using namespace tc;
 struct __align__(8) MbBars { uint64_t done; uint32_t tmem_base; uint32_t abort_flag; };
 
 // KIND: 0 = bf16 A,B in shared memory; 1 = bf16 A in tensor memory; 2 = int8 A,B in shared memory;
-//       3 = int8 A in tensor memory.
+//       3 = int8 A in tensor memory; 4 = int8 A,B in shared memory in the shape the 8-bit scoring kernel issues
+//       for 448 validation vectors (pair only): per K step one MMA of N = 256 and one of N = 192 on the same A.
 // PAIR: 0 = one CTA per 128 x 256 tile; 1 = CTA pair per 256 x 256 tile (cta_group::2).
 template <int KIND, int PAIR>
 __global__ void __launch_bounds__(128, 1)
@@ -24,7 +25,7 @@ mma_peak_kernel(int iters, unsigned int* timeout_word)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     constexpr int A_BYTES = 128 * 128;                      // 128 rows x 128 bytes (one swizzle panel)
-    constexpr int B_BYTES = (PAIR ? 128 : 256) * 128;
+    constexpr int B_BYTES = (KIND == 4 ? 224 : PAIR ? 128 : 256) * 128;
     uint8_t* sA = smem;
     uint8_t* sB = smem + A_BYTES;
     MbBars* bars = reinterpret_cast<MbBars*>(sB + B_BYTES);
@@ -65,8 +66,10 @@ mma_peak_kernel(int iters, unsigned int* timeout_word)
     if (threadIdx.x == 0 && rank == 0) {
         constexpr uint32_t M = PAIR ? 256 : 128;
         const uint32_t idesc = (KIND >= 2) ? make_idesc(2, 1, 1, M, 256) : make_idesc(1, 1, 1, M, 256);
+        const uint32_t idesc192 = make_idesc(2, 1, 1, M, 192);
         const uint64_t adesc = make_smem_desc_sw128(smem_u32(sA));
         const uint64_t bdesc = make_smem_desc_sw128(smem_u32(sB));
+        const uint64_t bdesc192 = make_smem_desc_sw128(smem_u32(sB + 128 * 128));    // this CTA's 96 rows of the second MMA
         for (int it = 0; it < iters; ++it) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {                   // four K steps of 32 bytes inside the 128-byte panel
@@ -81,6 +84,11 @@ mma_peak_kernel(int iters, unsigned int* timeout_word)
                     else mma_f16_ts(tmem_base, tmem_base + 256 + 8 * k, bdesc + (uint64_t)(2 * k), idesc, acc);
                 } else if (KIND == 3) {
                     if (PAIR) mma_i8_ts_pair(tmem_base, tmem_base + 256 + 8 * k, bdesc + (uint64_t)(2 * k), idesc, acc);
+                } else if (KIND == 4) {
+                    if (PAIR) {
+                        mma_i8_ss_pair(tmem_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, acc);
+                        mma_i8_ss_pair(tmem_base + 256, adesc + (uint64_t)(2 * k), bdesc192 + (uint64_t)(2 * k), idesc192, acc);
+                    }
                 } else {
                     if (PAIR) mma_i8_ss_pair(tmem_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, acc);
                     else mma_i8_ss(tmem_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, acc);
@@ -97,6 +105,139 @@ mma_peak_kernel(int iters, unsigned int* timeout_word)
     if (warp == 0) {
         tc_fence_after();
         if (PAIR) tmem_dealloc_pair(tmem_base, 512); else tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// L2 -> shared memory streaming rate of TMA alone: every CTA keeps TS_STAGES stages of three 128-row x 128-byte
+// boxes (48 KiB, the operand bytes of one K block of 8-bit scoring, rounded up) in flight from a buffer of
+// 512 rows x 8192 bytes that stays in L2, and nothing consumes them.
+constexpr int TS_STAGES = 4;
+constexpr int TS_BOX = 128 * 128;
+struct __align__(8) TsBars { uint64_t full[TS_STAGES]; uint32_t abort_flag; };
+
+__global__ void __launch_bounds__(128, 1)
+tma_stream_kernel(const __grid_constant__ CUtensorMap tmap, int iters, unsigned int* timeout_word)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    TsBars* bars = reinterpret_cast<TsBars*>(smem + (size_t)TS_STAGES * 3 * TS_BOX);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < TS_STAGES; ++s) mbar_init(smem_u32(&bars->full[s]), 1);
+        bars->abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tmap);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        bool ok = true;
+        uint32_t tile = blockIdx.x * 7u;
+        for (int it = 0; it < iters && ok; ++it) {
+            const int s = it % TS_STAGES;
+            const uint32_t bar = smem_u32(&bars->full[s]);
+            if (it >= TS_STAGES) ok = mbar_wait(bar, (uint32_t)(it / TS_STAGES - 1) & 1u, &bars->abort_flag, timeout_word, TO_PRODUCER);
+            if (!ok) break;
+            mbar_arrive_expect_tx(bar, 3 * TS_BOX);
+#pragma unroll
+            for (int b = 0; b < 3; ++b, ++tile)
+                tma_load_3d(smem_u32(smem + (size_t)(s * 3 + b) * TS_BOX), &tmap, bar, (int32_t)(tile & 63u) * 128,
+                            (int32_t)((tile >> 6) & 3u) * 128, 0);
+        }
+        // every armed stage lands before the CTA leaves (bounded)
+        const int issued = ok ? iters : 0;
+        for (int it = (issued > TS_STAGES ? issued - TS_STAGES : 0); it < issued; ++it)
+            mbar_wait(smem_u32(&bars->full[it % TS_STAGES]), (uint32_t)(it / TS_STAGES) & 1u, &bars->abort_flag, timeout_word, TO_PRODUCER);
+        if (!ok)
+            for (int s = 0; s < TS_STAGES; ++s)
+                for (uint32_t t = 0; t < (1u << 16); ++t)
+                    if (mbar_try_wait(smem_u32(&bars->full[s]), 0) || mbar_try_wait(smem_u32(&bars->full[s]), 1)) break;
+    }
+    __syncthreads();
+}
+
+// The two together, as 8-bit scoring runs them: the leader of a CTA pair issues the int8 MMAs of one K block
+// (4 K steps x (N = 256, N = 192), operands resident in shared memory) back to back and commits once per K block;
+// in both CTAs a second thread streams one 48 KiB stage per K block from L2 into other shared memory, MX_STAGES
+// ahead, re-arming a stage when the commit of the K block that "used" it has arrived. The MMAs never wait for
+// data: what this measures is how much the copies landing in shared memory slow the tensor pipe's operand reads.
+constexpr int MX_STAGES = 3;
+struct __align__(8) MxBars { uint64_t done, full[MX_STAGES], empty[MX_STAGES]; uint32_t tmem_base; uint32_t abort_flag; };
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128, 1)
+mma_tma_mix_kernel(const __grid_constant__ CUtensorMap tmap, int iters, int with_copies, unsigned int* timeout_word)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    constexpr int A_BYTES = 128 * 128, B_BYTES = 224 * 128;
+    uint8_t* sA = smem;
+    uint8_t* sB = smem + A_BYTES;
+    uint8_t* sS = smem + A_BYTES + 32 * 1024;               // stream stages, 1 KiB aligned
+    MxBars* bars = reinterpret_cast<MxBars*>(sS + (size_t)MX_STAGES * 3 * TS_BOX);
+    const int warp = threadIdx.x >> 5;
+    const uint32_t rank = cluster_ctarank();
+
+    for (int i = threadIdx.x; i < (A_BYTES + B_BYTES) / 4; i += blockDim.x)
+        reinterpret_cast<uint32_t*>(smem)[i] = 0x01FF02FEu ^ (uint32_t)(i * 0x01010101u & 0x03030303u);
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars->done), 1);
+        for (int s = 0; s < MX_STAGES; ++s) { mbar_init(smem_u32(&bars->full[s]), 1); mbar_init(smem_u32(&bars->empty[s]), 1); }
+        bars->abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tmap);
+    }
+    if (warp == 0) { tmem_alloc_pair(smem_u32(&bars->tmem_base), 512); tmem_relinquish_pair(); }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = bars->tmem_base;
+
+    if (threadIdx.x == 0 && rank == 0) {
+        const uint32_t idesc = make_idesc(2, 1, 1, 256, 256), idesc192 = make_idesc(2, 1, 1, 256, 192);
+        const uint64_t adesc = make_smem_desc_sw128(smem_u32(sA));
+        const uint64_t bdesc = make_smem_desc_sw128(smem_u32(sB));
+        const uint64_t bdesc192 = make_smem_desc_sw128(smem_u32(sB + 128 * 128));
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t acc = (it > 0 || k > 0) ? 1u : 0u;
+                mma_i8_ss_pair(tmem_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, acc);
+                mma_i8_ss_pair(tmem_base + 256, adesc + (uint64_t)(2 * k), bdesc192 + (uint64_t)(2 * k), idesc192, acc);
+            }
+            mma_commit_pair(smem_u32(&bars->empty[it % MX_STAGES]));      // arrives in both CTAs
+        }
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&bars->done)) : "memory");
+        mbar_wait(smem_u32(&bars->done), 0, &bars->abort_flag, timeout_word, TO_MMA);
+    } else if (threadIdx.x == 32 && with_copies) {
+        bool ok = true;
+        uint32_t tile = blockIdx.x * 7u;
+        int issued = 0;
+        for (int it = 0; it < iters && ok; ++it) {
+            const int s = it % MX_STAGES;
+            const uint32_t bar = smem_u32(&bars->full[s]);
+            if (it >= MX_STAGES) {
+                const uint32_t par = (uint32_t)(it / MX_STAGES - 1) & 1u;
+                ok = mbar_wait_cluster(smem_u32(&bars->empty[s]), par, &bars->abort_flag, timeout_word, TO_PRODUCER) &&
+                     mbar_wait(bar, par, &bars->abort_flag, timeout_word, TO_PRODUCER);
+                if (!ok) break;
+            }
+            mbar_arrive_expect_tx(bar, 3 * TS_BOX);
+#pragma unroll
+            for (int b = 0; b < 3; ++b, ++tile)
+                tma_load_3d(smem_u32(sS + (size_t)(s * 3 + b) * TS_BOX), &tmap, bar, (int32_t)(tile & 63u) * 128,
+                            (int32_t)((tile >> 6) & 3u) * 128, 0);
+            ++issued;
+        }
+        // every armed stage lands before the CTA leaves (bounded)
+        for (int it = (issued > MX_STAGES ? issued - MX_STAGES : 0); it < issued; ++it)
+            if (!mbar_wait(smem_u32(&bars->full[it % MX_STAGES]), (uint32_t)(it / MX_STAGES) & 1u, &bars->abort_flag, timeout_word, TO_PRODUCER)) break;
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, 512);
     }
 }
 
@@ -162,7 +303,7 @@ extern "C" qless_status qless_microbench(int32_t what, int32_t iters, float* ms_
             if (what == 0) { QLESS_MB_LAUNCH(0) } else if (what == 1) { QLESS_MB_LAUNCH(1) } else { QLESS_MB_LAUNCH(2) }
 #undef QLESS_MB_LAUNCH
             ops = (double)sms * iters * 4.0 * 2.0 * 128 * 256 * (what == 2 ? 32 : 16);
-        } else if ((what >= 3 && what <= 5) || what == 7) {
+        } else if ((what >= 3 && what <= 5) || what == 7 || what == 8) {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3((unsigned)(sms / 2 * 2)); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = smem; cfg.stream = st;
             cudaLaunchAttribute attr; attr.id = cudaLaunchAttributeClusterDimension; attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
@@ -170,14 +311,35 @@ extern "C" qless_status qless_microbench(int32_t what, int32_t iters, float* ms_
 #define QLESS_MB_LAUNCH(K)                                                                                           \
             err = cudaFuncSetAttribute(mma_peak_kernel<K, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
             if (err == cudaSuccess) err = cudaLaunchKernelEx(&cfg, mma_peak_kernel<K, 1>, (int)iters, flag);
-            if (what == 3) { QLESS_MB_LAUNCH(0) } else if (what == 4) { QLESS_MB_LAUNCH(1) } else if (what == 5) { QLESS_MB_LAUNCH(2) } else { QLESS_MB_LAUNCH(3) }
+            if (what == 3) { QLESS_MB_LAUNCH(0) } else if (what == 4) { QLESS_MB_LAUNCH(1) } else if (what == 5) { QLESS_MB_LAUNCH(2) }
+            else if (what == 7) { QLESS_MB_LAUNCH(3) } else { QLESS_MB_LAUNCH(4) }
 #undef QLESS_MB_LAUNCH
-            ops = (double)(sms / 2) * iters * 4.0 * 2.0 * 256 * 256 * (what == 5 || what == 7 ? 32 : 16);
+            ops = (double)(sms / 2) * iters * 4.0 * 2.0 * 256 * (what == 8 ? 448 : 256) * (what == 5 || what == 7 || what == 8 ? 32 : 16);
         } else if (what == 6) {
             const size_t need = (size_t)sms * 8 * 256 * sizeof(uint32_t);
             QLESS_REQUIRE(scratch != nullptr && scratch_bytes >= need, QLESS_ERR_WORKSPACE, "scratch of %zu bytes required", need);
             popc_peak_kernel<<<sms * 8, 256, 0, st>>>(iters, 12345u, reinterpret_cast<uint32_t*>(scratch));
             ops = (double)sms * 8 * 256 * iters * 32.0;           // word operations: one XOR + POPC + IADD each
+        } else if (what == 9 || what == 10 || what == 11) {
+            const size_t need = (size_t)512 * 8192;
+            if (scratch == nullptr || scratch_bytes < need || (reinterpret_cast<uintptr_t>(scratch) % 16) != 0) {
+                cudaEventDestroy(e0); cudaEventDestroy(e1);
+                return fail(QLESS_ERR_WORKSPACE, "16-byte aligned scratch of %zu bytes required", need);
+            }
+            CUtensorMap tm;
+            const qless_status ts = make_tmap_3d_u8(&tm, scratch, 8192, 512, 1, 8192, need, 128, 128, true);
+            if (ts != QLESS_OK) { cudaEventDestroy(e0); cudaEventDestroy(e1); return ts; }
+            if (what == 9) {
+                const size_t ts_smem = 1024 + (size_t)TS_STAGES * 3 * TS_BOX + sizeof(TsBars);
+                err = cudaFuncSetAttribute(tma_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ts_smem);
+                if (err == cudaSuccess) tma_stream_kernel<<<sms, 128, ts_smem, st>>>(tm, iters, flag);
+                ops = (double)sms * iters * 3.0 * TS_BOX;             // bytes moved from L2 into shared memory
+            } else {
+                const size_t mx_smem = 1024 + 128 * 128 + 32 * 1024 + (size_t)MX_STAGES * 3 * TS_BOX + sizeof(MxBars);
+                err = cudaFuncSetAttribute(mma_tma_mix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mx_smem);
+                if (err == cudaSuccess) mma_tma_mix_kernel<<<sms / 2 * 2, 128, mx_smem, st>>>(tm, iters, what == 10 ? 1 : 0, flag);
+                ops = (double)(sms / 2) * iters * 4.0 * 2.0 * 256 * 448 * 32;
+            }
         } else {
             cudaEventDestroy(e0); cudaEventDestroy(e1);
             return fail(QLESS_ERR_INVALID_ARG, "unknown micro-benchmark %d", what);

@@ -667,3 +667,16 @@ def test_scoring_full_width_sampled(bits):
         assert np.abs(got[t0:t0 + 10] - want).max() <= SCORE_TOL * sum(eta)
     idx = _np(B.qless_select_topk(torch.from_numpy(got).to(DEV), 0.05))
     assert np.array_equal(idx, oracle.select_topk(got, 0.05))
+
+
+# ----------------------------------------------------------------------------------------------
+# Micro-benchmarks behind the roofline denominators: they run and report plausible rates
+# ----------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("what,lo,hi", [("i8_ss_pair", 1e15, 1e16), ("i8_ss_pair_n448", 1e15, 1e16),
+                                        ("tma_l2_stream", 1e12, 5e13), ("i8_n448_with_tma", 1e15, 1e16),
+                                        ("i8_n448_commit_per_block", 1e15, 1e16)])
+def test_microbenchmarks_run(what, lo, hi):
+    ms, ops = B.qless_microbench(what, 2000)
+    B.qless_check()
+    assert ms > 0 and lo <= ops / (ms * 1e-3) <= hi, (what, ms, ops)
