@@ -123,6 +123,14 @@ def test_bad_arguments_return_statuses_before_any_launch(L):
     for hook, bad in ((L.qless_set_projection_path, 2), (L.qless_set_score_path, -1), (L.qless_set_select_path, 3)):
         assert hook(bad) == B.ERR_INVALID_ARG
         assert hook(0) == B.QLESS_OK
+    # the matrix switch and the Gaussian entry hook
+    assert L.qless_set_projection_matrix(2) == B.ERR_INVALID_ARG and L.qless_set_projection_matrix(-1) == B.ERR_INVALID_ARG
+    assert L.qless_set_projection_matrix(B.GAUSSIAN) == B.QLESS_OK and L.qless_set_projection_matrix(B.RADEMACHER) == B.QLESS_OK
+    assert L.qless_gaussian_entries(1, 0, 2, 2, 8, fake, null) == B.ERR_INVALID_ARG          # j0 not a multiple of 4
+    assert L.qless_gaussian_entries(1, -1, 2, 0, 8, fake, null) == B.ERR_INVALID_ARG
+    assert L.qless_gaussian_entries(1, 0, 2, 1 << 39, 8, fake, null) == B.ERR_UNSUPPORTED
+    assert L.qless_gaussian_entries(1, 0, 2, 0, 8, null, null) == B.ERR_INVALID_ARG           # no output buffer
+    assert L.qless_gaussian_entries(1, 0, 0, 0, 8, null, null) == B.QLESS_OK                  # empty range
     # micro-benchmarks: unknown kind, missing outputs (checked before anything is launched)
     ms, ops = C.c_float(0), C.c_double(0)
     assert L.qless_microbench(0, 10, None, C.byref(ops), null, 0, null) == B.ERR_INVALID_ARG
