@@ -669,6 +669,48 @@ def test_scoring_full_width_sampled(bits):
     assert np.array_equal(idx, oracle.select_topk(got, 0.05))
 
 
+def _build_store_chunked(bits, C, N, V, d, seed):
+    """The benchmark's way of building a large store: features generated and quantised 16 384 rows at a time."""
+    rb = d * bits // 8
+    tc = torch.empty((C, N, rb), dtype=torch.uint8, device=DEV); vc = torch.empty((C, V, rb), dtype=torch.uint8, device=DEV)
+    ts = torch.empty((C, N), device=DEV); vs = torch.empty((C, V), device=DEV)
+    tq = torch.empty((C, N), dtype=torch.int32, device=DEV); vq = torch.empty((C, V), dtype=torch.int32, device=DEV)
+    for r0 in range(0, N, 16384):
+        r1 = min(N, r0 + 16384)
+        xs = W.lowrank_gaussian_features(r1 - r0, d, C, seed=seed + r0, device=DEV)
+        for i in range(C):
+            tc[i, r0:r1], ts[i, r0:r1], tq[i, r0:r1] = B.qless_quantize(xs[i], bits)
+    xs = W.lowrank_gaussian_features(V, d, C, seed=seed - 1, device=DEV)
+    for i in range(C):
+        vc[i], vs[i], vq[i] = B.qless_quantize(xs[i], bits)
+    return tc, vc, ts, vs, tq, vq
+
+
+@pytest.mark.parametrize("cfg_name,bits", [("c3_score_sweep", 8), ("c3_score_sweep", 4), ("c3_score_sweep", 2),
+                                           ("c4_onebit_scaleup", 1)])
+def test_scoring_full_size_sampled_rows(cfg_name, bits):
+    # configs 3 and 4 at their full sizes, in the launch configuration the benchmark times (every CTA pair walks
+    # many tiles, the last tile is ragged): the oracle scores sampled train rows one by one (a row's score depends
+    # on no other train row), and selects from the GPU's full score vector
+    cfg = W.CONFIGS[cfg_name]
+    N, d, C, V = cfg["N"], cfg["d"], cfg["C"], sum(cfg["tasks"])
+    off = W.task_offsets(cfg["tasks"]).tolist()
+    tc, vc, ts, vs, tq, vq = _build_store_chunked(bits, C, N, V, d, seed=7000)
+    scores = B.qless_score(tc, vc, ts, vs, cfg["lr"], off, d, bits, train_sumsq=tq, val_sumsq=vq)
+    B.qless_check()
+    last_full = (N // 256) * 256
+    rows = sorted({0, 1, 127, 128, 255, 256, N // 2, last_full - 1, min(last_full, N - 1), N - 1} |
+                  set(np.random.default_rng(5).integers(0, N, 22).tolist()))
+    r = torch.tensor(rows, device=DEV)
+    want = oracle.score(_np(tc[:, r]), _np(vc), _np(ts[:, r]), _np(vs), cfg["lr"], off, d, bits)
+    got = _np(scores)
+    assert np.abs(got[rows] - want).max() <= SCORE_TOL * sum(cfg["lr"])
+    assert np.isfinite(got).all() and np.abs(got).max() <= sum(cfg["lr"]) * (1 + 1e-5)      # a weighted mean of cosines
+    idx = _np(B.qless_select_topk(scores, cfg["frac"]))
+    assert idx.size == int(cfg["frac"] * N + 1e-6)
+    assert np.array_equal(idx, oracle.select_topk(got, cfg["frac"]))
+
+
 # ----------------------------------------------------------------------------------------------
 # Micro-benchmarks behind the roofline denominators: they run and report plausible rates
 # ----------------------------------------------------------------------------------------------
