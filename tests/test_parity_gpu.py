@@ -711,6 +711,46 @@ def test_scoring_full_size_sampled_rows(cfg_name, bits):
     assert np.array_equal(idx, oracle.select_topk(got, cfg["frac"]))
 
 
+def test_config5_pipeline_full_width_reduced_rows():
+    # config 5 with its real widths (P = 2^22 bf16 gradients, Adam on the train side only, d = 8192, 2-bit codes,
+    # 4 checkpoints, 448 validation gradients in 3 tasks) and 256 instead of 32 768 training rows per checkpoint:
+    # every stage against the oracle (projection on sampled rows and coordinates, codes from the GPU's own
+    # projection, scores from the GPU's own codes on sampled rows, selection from the GPU's own scores)
+    cfg = W.CONFIGS["c5_full_pipeline"]
+    P, d, C, bits, V, seed, n = cfg["P"], cfg["d"], cfg["C"], cfg["bits"], cfg["n_val"], 555, 256
+    off = W.task_offsets(cfg["tasks"]).tolist()
+    rb = d * bits // 8
+    tc = torch.empty((C, n, rb), dtype=torch.uint8, device=DEV); vc = torch.empty((C, V, rb), dtype=torch.uint8, device=DEV)
+    ts = torch.empty((C, n), device=DEV); vs = torch.empty((C, V), device=DEV)
+    tq = torch.empty((C, n), dtype=torch.int32, device=DEV); vq = torch.empty((C, V), dtype=torch.int32, device=DEV)
+    rows, coords = [0, 129, 255], [0, 127, 128, 5000, 8191]
+    for i in range(C):
+        m, v = W.adam_moments(P, seed=800 + i, device=DEV)
+        for side, count, codes, scales, sumsq in (("train", n, tc, ts, tq), ("val", V, vc, vs, vq)):
+            g = W.student_t_gradients(count, P, seed=900 + 10 * i + (side == "val"), device=DEV, dtype=torch.bfloat16)
+            adam = (m, v) if side == "train" else (None, None)
+            out = B.qless_project_quantize(g, d, seed, bits, adam[0], adam[1], want_proj=True)
+            codes[i], scales[i], sumsq[i] = out["codes"], out["scales"], out["sumsq"]
+            proj = _np(out["proj"])
+            if i in (0, C - 1):
+                gamma = oracle.adam_gamma(_np(g[rows].float()), *( (_np(m), _np(v)) if side == "train" else (None, None) ))
+                want = oracle.project_rows(gamma, d, seed, coords)
+                ref = np.abs(proj[rows]).max(axis=1, keepdims=True)
+                assert (np.abs(proj[np.ix_(rows, coords)] - want) / ref).max() <= PROJ_TOL
+            wc, wsc, wss = oracle.quantize_rows(proj, bits, normalize=True)
+            assert (_np(out["codes"]) == wc).all(axis=1).sum() >= count - 2
+            assert np.allclose(_np(out["scales"]), wsc, rtol=3e-7)
+            same = (_np(out["codes"]) == wc).all(axis=1)
+            assert np.array_equal(_np(out["sumsq"])[same], wss[same])
+    B.qless_check()
+    scores = B.qless_score(tc, vc, ts, vs, cfg["lr"], off, d, bits, train_sumsq=tq, val_sumsq=vq)
+    r = torch.arange(0, n, 8, device=DEV)
+    want = oracle.score(_np(tc[:, r]), _np(vc), _np(ts[:, r]), _np(vs), cfg["lr"], off, d, bits)
+    assert np.abs(_np(scores)[::8] - want).max() <= SCORE_TOL * sum(cfg["lr"])
+    idx = _np(B.qless_select_topk(scores, cfg["frac"]))
+    assert np.array_equal(idx, oracle.select_topk(_np(scores), cfg["frac"]))
+
+
 # ----------------------------------------------------------------------------------------------
 # Micro-benchmarks behind the roofline denominators: they run and report plausible rates
 # ----------------------------------------------------------------------------------------------
