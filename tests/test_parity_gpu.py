@@ -54,6 +54,17 @@ def test_adam_gamma_bit_exact(dtype, step, use_adam):
     assert np.array_equal(_np(got.float()).view(np.uint32), want.view(np.uint32))
 
 
+def test_adam_gamma_bit_exact_on_many_elements():
+    # 2^26 elements: the approximate-unit fast path must round to the oracle's bf16 everywhere, also for the few
+    # per ten thousand elements that fall next to a rounding boundary and take the exact sequence
+    n, P = 64, 1 << 20
+    g = W.student_t_gradients(n, P, seed=13, device=DEV, dtype=torch.bfloat16)
+    m, v = W.adam_moments(P, seed=14, device=DEV)
+    got = _np(B.qless_adam_gamma(g, m, v, dict(beta1=0.9, beta2=0.999, eps=1e-8, step=0)).float())
+    want = oracle.adam_gamma(_np(g.float()), _np(m), _np(v))
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
 def test_adam_gamma_strided_rows_and_extreme_values():
     n, P = 3, 256
     big = torch.zeros((n, P + 64), dtype=torch.float32, device=DEV)
