@@ -318,6 +318,8 @@ def stage_measurements(torch, B, W, dev, peaks):
         ts_ = _time_ms(torch, lambda: B.qless_score(st["tc"], st["vc"], st["ts"], st["vs"], cfg["lr"], off, d, b,
                                                     train_sumsq=st["tq"], val_sumsq=st["vq"], scores=sc, workspace=ws), 400, warm=0)
         ck = smp.stop()
+        if b == 1:
+            sc_1bit = sc.clone()        # for the selected-percentage sweep below
         e.update(ms_sustained=ts_, frac_of_int8_sustained=iops / ts_ / 1e9 / i8_sustained, sustained_clocks=ck)
         if ck.get("sm_mhz") and ck.get("sm_max_mhz"):
             # the micro-benchmark holds the maximum clock (its operands never change, so it draws little power); the
@@ -351,6 +353,17 @@ def stage_measurements(torch, B, W, dev, peaks):
     in16 = torch.zeros(N, dtype=torch.bool, device=dev)
     in16[top16] = True
     del t16, v16, ws16
+    # the selected-percentage sweep of the paper's Fig. 4 (0.1 to 10 % with the 1-bit store), on this synthetic store:
+    # how much of the 16-bit baseline's selection the 1-bit codes reproduce at each percentage, and the selection time
+    sweep = {}
+    for frac in (0.001, 0.005, 0.01, 0.02, 0.05, 0.10):
+        ref = torch.zeros(N, dtype=torch.bool, device=dev)
+        ref[B.qless_select_topk(sc16, frac)] = True
+        t = _time_ms(torch, lambda: B.qless_select_topk(sc_1bit, frac), 20)
+        sweep[str(frac)] = dict(k=int(frac * N + 1e-6), select_ms=t,
+                                overlap_with_16bit=float(ref[B.qless_select_topk(sc_1bit, frac)].float().mean()))
+    res["1bit_selected_percentage_sweep"] = sweep
+    del sc_1bit
     for b in cfg["bits"]:
         res[str(b)]["top5pct_overlap_with_16bit"] = float(in16[tops[b]].float().mean())
     out["score_c3_270000x448x4"] = res
