@@ -293,6 +293,24 @@ def test_gaussian_projection_matches_oracle(gaussian_matrix, n, P, d, dtype, use
     assert e_l2 <= 1e-5 and e_max <= 1e-5, (e_l2, e_max)
 
 
+def test_gaussian_host_entry_matches_device_entry(gaussian_matrix):
+    # the host-buffer entry projects column slabs with the Philox counters offset by the slab's first column: with
+    # the Gaussian matrix, too, it must give the device-buffer entry's bytes
+    n, P, d, bits = 70, 1 << 18, 256, 4
+    g = W.student_t_gradients(n, P, seed=63, device="cpu").to(torch.bfloat16)
+    host = g.clone().pin_memory()
+    m, v = W.adam_moments(P, seed=64, device=DEV)
+    dev_out = B.qless_project_quantize(g.to(DEV), d, 778, bits, adam_m=m, adam_v=v)
+    host_out = B.qless_project_quantize_host(host, d, 778, bits, adam_m=m, adam_v=v, device=DEV)
+    torch.cuda.synchronize()
+    assert np.array_equal(host_out["codes"].numpy(), _np(dev_out["codes"]))
+    assert np.array_equal(host_out["scales"].numpy(), _np(dev_out["scales"]))
+    # and it is not the Rademacher result
+    B.qless_set_projection_matrix(B.RADEMACHER)
+    rad = B.qless_project_quantize(g.to(DEV), d, 778, bits, adam_m=m, adam_v=v)
+    assert not np.array_equal(_np(rad["codes"]), _np(dev_out["codes"]))
+
+
 def test_gaussian_projection_of_basis_vectors_and_switch_back(gaussian_matrix):
     # e_j projects to column j of the matrix the entry hook returns, scaled by the fp32 value of 1/sqrt(d)
     P, d, seed = 1024, 256, 78
