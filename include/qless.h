@@ -200,9 +200,9 @@ qless_status qless_philox_entries(
  * row r in columns 4q .. 4q+3 come from one Philox4x32-10 call with counter (q mod 2^32, r, q div 2^32, 1) and
  * the same key; output words (w0, w1) give columns 4q, 4q+1 and (w2, w3) give 4q+2, 4q+3 by the Box-Muller
  * transform z_even = sqrt(-2 ln u1) cos(2 pi u2), z_odd = sqrt(-2 ln u1) sin(2 pi u2) with
- * u = (floor(w / 2^9) + 1/2) / 2^23. The logarithm, square root, sine and cosine are evaluated in fp32 on the GPU's approximate units, so an
- * entry may differ from the correctly rounded one by one bf16 step where it falls next to a rounding boundary.
- * The generator, not the tensor pipe, bounds this variant (about 100 times the instructions per entry).
+ * u = (floor(w / 2^9) + 1/2) / 2^23. The logarithm, square root, sine and cosine are evaluated in fp32 on the
+ * GPU's approximate units, so an entry may differ from the correctly rounded one by one bf16 step where it falls next to a rounding boundary.
+ * The generator, not the tensor pipe, bounds this variant (about 20 instructions per entry against one; the projection takes about 4.5 times as long).
  * Process-wide; stores built with different matrices (or seeds) must not be scored against each other.
  * Returns QLESS_ERR_INVALID_ARG for any other value. */
 enum { QLESS_MATRIX_RADEMACHER = 0, QLESS_MATRIX_GAUSSIAN = 1 };
