@@ -370,18 +370,21 @@ qless_status qless_project_quantize_host(const void* grads_host, qless_dtype dty
     cudaStream_t cs = nullptr;
     s = copy_stream(&cs);
     if (s != QLESS_OK) return s;
-    // about eight slabs, each a whole number of K chunks
+    // about eight slabs, each a whole number of K chunks; the copies take longer than the projection, so only the
+    // projection of the last slab is not hidden behind a copy: the last eighth is cut into slabs that halve in size
     int64_t chunks_per_slab = (w.plan.num_chunks + 7) / 8;
     if (chunks_per_slab < 1) chunks_per_slab = 1;
-    const int64_t slab = chunks_per_slab * w.plan.chunk;
     cudaEvent_t ev_entry = nullptr, ev_slab = nullptr;
     QLESS_CUDA_TRY(cudaEventCreateWithFlags(&ev_entry, cudaEventDisableTiming));
     cudaError_t ce = cudaEventRecord(ev_entry, st);
     if (ce == cudaSuccess) ce = cudaStreamWaitEvent(cs, ev_entry, 0);
     cudaEventDestroy(ev_entry);             // released once the recorded work has completed
     if (ce != cudaSuccess) return cuda_fail(ce, "event set-up of the host path");
-    for (int64_t j0 = 0; j0 < P; j0 += slab) {
-        const int64_t len = (P - j0 < slab) ? P - j0 : slab;
+    for (int64_t j0 = 0, len = 0; j0 < P; j0 += len) {
+        const int64_t chunks_left = (P - j0 + w.plan.chunk - 1) / w.plan.chunk;
+        const int64_t take = chunks_left > chunks_per_slab ? chunks_per_slab : (chunks_left + 1) / 2;
+        len = take * w.plan.chunk;
+        if (len > P - j0) len = P - j0;
         ce = cudaMemcpy2DAsync(reinterpret_cast<uint8_t*>(d_grads) + (size_t)j0 * esz, (size_t)P * esz,
                                reinterpret_cast<const uint8_t*>(grads_host) + (size_t)j0 * esz, (size_t)ld_grads * esz,
                                (size_t)len * esz, (size_t)n, cudaMemcpyHostToDevice, cs);
