@@ -589,6 +589,15 @@ def run_ours(args):
         d2h = n * rb + 2 * n * 4 + k_sel * 8
         e2e = dict(value=whole_job_rate(n, args.e2e_steps, world, ms_e2e), unit="grads/s", h2d_bytes_per_step=h2d,
                    d2h_bytes_per_step=d2h, steps=args.e2e_steps, ms_per_step=ms_e2e / args.e2e_steps)
+        # what bounds it: a plain pinned host-to-device copy of the same batch, nothing else running (outside the timed region)
+        g.copy_(g_host, non_blocking=True)
+        torch.cuda.synchronize()
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record()
+        g.copy_(g_host, non_blocking=True)
+        c1.record()
+        torch.cuda.synchronize()
+        e2e.update(plain_h2d_copy_ms=c0.elapsed_time(c1), plain_h2d_copy_gbs=n * P * 2 / c0.elapsed_time(c1) / 1e6)
 
     if rank == 0:
         peaks = load_peaks()
