@@ -293,6 +293,28 @@ def test_gaussian_projection_matches_oracle(gaussian_matrix, n, P, d, dtype, use
     assert e_l2 <= 1e-5 and e_max <= 1e-5, (e_l2, e_max)
 
 
+def test_gaussian_projection_full_width_sampled(gaussian_matrix):
+    # config 5's gradient width (P = 2^22, bf16, Adam), a full 256-row batch, d = 8192: the launch configuration of
+    # the large runs (64 K chunks, every CTA pair persistent); the oracle evaluates sampled rows and coordinates
+    n, P, d, seed = 256, 1 << 22, 8192, 4242
+    g = W.student_t_gradients(n, P, seed=46, device=DEV, dtype=torch.bfloat16)
+    m, v = W.adam_moments(P, seed=47, device=DEV)
+    out = B.qless_project_quantize(g, d, seed, 2, m, v, want_proj=True)
+    B.qless_check()
+    rows, coords = [0, 130, 255], [0, 129, 4096, 8191]
+    gamma = oracle.adam_gamma(_np(g[rows].float()), _np(m), _np(v)).astype(np.float64)
+    proj = _np(out["proj"])
+    ref = np.abs(proj[rows]).max(axis=1)
+    for b, r in enumerate(coords):
+        z = oracle.gaussian_rows(seed, r, 1, 0, P)[0].astype(np.float64)
+        want = (gamma @ z) * float(np.float32(1.0) / np.sqrt(np.float32(d)))
+        assert (np.abs(proj[rows, r] - want) / ref).max() <= PROJ_TOL
+    # JL for a Gaussian matrix: ||y||^2 / ||Gamma||^2 within 5 sigma of 1
+    g2 = (gamma ** 2).sum(1)
+    y2 = (proj[rows].astype(np.float64) ** 2).sum(1)
+    assert np.all(np.abs(y2 / g2 - 1) <= 5 * math.sqrt(2.0 / d))
+
+
 def test_gaussian_host_entry_matches_device_entry(gaussian_matrix):
     # the host-buffer entry projects column slabs with the Philox counters offset by the slab's first column: with
     # the Gaussian matrix, too, it must give the device-buffer entry's bytes
