@@ -93,73 +93,151 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm))
 
 
+def bench_config(cfg):
+    """The `config` object of the JSON line, the same for both arms."""
+    return dict(workload=WORKLOAD, batch_rows=cfg["batch_rows"], P=cfg["P"], d=cfg["d"], bits=cfg["bits"], val_rows=N_VAL,
+                tasks=TASKS, select_frac=FRAC, l2="inputs larger than L2 (4.3 GB batch), no flush")
+
+
+def host_cores():
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
+def _threaded(fn, pieces, threads):
+    """Runs fn(piece) for every piece on `threads` host threads. The oracle's C functions are called through ctypes,
+    which releases the interpreter lock for the duration of the call, so the pieces run on separate cores; each call
+    is the unchanged single-threaded oracle routine on its own rows or coordinates."""
+    if threads <= 1:
+        return [fn(p) for p in pieces]
+    from concurrent.futures import ThreadPoolExecutor
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        return list(ex.map(fn, pieces))
+
+
+class OracleProjectionSample:
+    """The oracle on a bounded sample of the benchmark's workload: n_rows gradient rows at full P through the Adam
+    prologue, the projection onto n_coords of the d output coordinates (the oracle regenerates a row of R per
+    coordinate, so its work is linear in the coordinates taken) and normalise + quantise of full rows. Both the
+    reference arm and the cpu_baseline leg time exactly this, so their figures agree."""
+
+    def __init__(self, threads, n_rows=2, coords_per_thread=8):
+        import numpy as np
+        import torch
+        from paper_2502_01703_b200 import workloads as W
+        cfg = W.CONFIGS[WORKLOAD]
+        self.P, self.d, self.bits = cfg["P"], cfg["d"], cfg["bits"]
+        self.threads, self.n_rows = threads, n_rows
+        self.n_coords = min(self.d, coords_per_thread * threads)
+        self.g = W.student_t_gradients(n_rows, self.P, seed=SEED, dtype=torch.bfloat16).float().numpy()
+        self.m, self.v = [t.numpy() for t in W.adam_moments(self.P, seed=SEED + 1)]
+        step = self.d // self.n_coords
+        self.coords = np.arange(self.n_coords, dtype=np.int32) * step
+        self.np = np
+
+    def run(self):
+        """One pass over the sample. Returns (seconds one gradient would take through the full path, seconds taken)."""
+        import oracle
+        np = self.np
+        t0 = time.perf_counter()
+        gam = np.concatenate(_threaded(lambda r: oracle.adam_gamma(self.g[r:r + 1], self.m, self.v), range(self.n_rows), self.threads))
+        t1 = time.perf_counter()
+        pieces = np.array_split(self.coords, min(self.threads, self.n_coords))
+        y = np.concatenate(_threaded(lambda c: oracle.project_rows(gam, self.d, SEED, c), pieces, self.threads), axis=1)
+        t2 = time.perf_counter()
+        full = np.resize(y, (self.n_rows, self.d)).astype(np.float32)
+        oracle.quantize_rows(full, self.bits, normalize=True)
+        t3 = time.perf_counter()
+        per_grad = ((t1 - t0) + (t2 - t1) * (self.d / self.n_coords) + (t3 - t2)) / self.n_rows
+        return per_grad, t3 - t0
+
+    def describe(self):
+        return (f"{self.n_rows} gradient rows at full P=2^23: Adam prologue, projection onto {self.n_coords} of {self.d} output "
+                f"coordinates (scaled x{self.d // self.n_coords}; the work is linear in d), normalise+quantise of full rows; "
+                f"{self.threads} thread(s) over coordinates")
+
+
 def run_reference(args):
-    """The CPU oracle timed as it stands on a bounded sample of the same workload (rank 0 only)."""
+    """The CPU oracle timed as it stands on a bounded sample of the same workload (rank 0 only; other ranks leave)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import numpy as np
-    import torch
-    import oracle
     from paper_2502_01703_b200 import workloads as W
     cfg = W.CONFIGS[WORKLOAD]
-    P, d, bits = cfg["P"], cfg["d"], cfg["bits"]
-    n_rows, n_coords = 1, 16
-    g = W.student_t_gradients(n_rows, P, seed=SEED, dtype=torch.bfloat16).float().numpy()
-    m, v = [t.numpy() for t in W.adam_moments(P, seed=SEED + 1)]
-    coords = np.arange(n_coords, dtype=np.int32) * (d // n_coords)
-
-    def step():
-        t0 = time.perf_counter()
-        gam = oracle.adam_gamma(g, m, v)
-        t1 = time.perf_counter()
-        y = oracle.project_rows(gam, d, SEED, coords)
-        t2 = time.perf_counter()
-        full = np.resize(y, (n_rows, d)).astype(np.float32)
-        oracle.quantize_rows(full, bits, normalize=True)
-        t3 = time.perf_counter()
-        # seconds one gradient would take through the full path (projection is linear in d)
-        return ((t1 - t0) + (t2 - t1) * (d / n_coords) + (t3 - t2)) / n_rows
-
+    cores = host_cores()
+    smp = OracleProjectionSample(cores)
     for _ in range(args.warmup):
-        step()
-    per_grad = [step() for _ in range(args.steps)]
-    sec = sum(per_grad) / len(per_grad)
+        smp.run()
+    runs = [smp.run() for _ in range(args.steps)]
+    sec = sum(r[0] for r in runs) / len(runs)               # seconds per gradient through the full path
+    step_s = sum(r[1] for r in runs) / len(runs)            # seconds a step (one pass over the sample) really took
     value = 1.0 / sec
-    sample = (f"{n_rows} gradient row(s) at full P=2^23 through Adam prologue, projection onto {n_coords} of {d} "
-              f"output coordinates (scaled x{d // n_coords}), normalise+quantise of a full row; single thread")
     line = dict(impl="reference", metric="grads projected+quantized/s (P=2^23,d=8192)", value=value, unit="grads/s",
-                n_gpus=args.gpus, steps=args.steps, warmup=args.warmup, ms_per_step=sec * cfg["batch_rows"] * 1e3,
+                n_gpus=args.gpus, steps=args.steps, warmup=args.warmup, ms_per_step=step_s * 1e3,
                 higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
-                config=dict(workload=WORKLOAD, batch_rows=cfg["batch_rows"], P=P, d=d, bits=bits),
-                cpu_baseline=dict(value=value, unit="grads/s", cores=1, kind="oracle", sample=sample),
+                config=bench_config(cfg),
+                gradients_per_step=step_s / sec,
+                cpu_baseline=dict(value=value, unit="grads/s", cores=cores, kind="oracle", sample=smp.describe()),
                 e2e=dict(value=value, unit="grads/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0),
                 gpu_launches=0)
     print(json.dumps(line))
 
 
 def cpu_baseline():
+    """The oracle, as it stands, on the host cores: the projection + quantisation sample of the reference arm (all
+    cores and one thread), scoring per code width on sampled train rows of configs 3 and 4 against all 448 x 4
+    validation vectors (one thread and all cores, rows split over threads), and selection at the full sizes."""
     import numpy as np
-    import torch
     import oracle
     from paper_2502_01703_b200 import workloads as W
-    cfg = W.CONFIGS[WORKLOAD]
-    P, d, bits = cfg["P"], cfg["d"], cfg["bits"]
-    n_rows, n_coords = 4, 512
-    g = W.student_t_gradients(n_rows, P, seed=SEED, dtype=torch.bfloat16).float().numpy()
-    m, v = [t.numpy() for t in W.adam_moments(P, seed=SEED + 1)]
-    coords = np.arange(n_coords, dtype=np.int32) * (d // n_coords)
-    t0 = time.perf_counter()
-    gam = oracle.adam_gamma(g, m, v)
-    t1 = time.perf_counter()
-    y = oracle.project_rows(gam, d, SEED, coords)
-    t2 = time.perf_counter()
-    oracle.quantize_rows(np.resize(y, (n_rows, d)).astype(np.float32), bits, normalize=True)
-    t3 = time.perf_counter()
-    sec_per_grad = ((t1 - t0) + (t2 - t1) * (d / n_coords) + (t3 - t2)) / n_rows
-    return dict(value=1.0 / sec_per_grad, unit="grads/s", cores=1, kind="oracle",
-                sample=(f"{n_rows} gradient rows at full P=2^23, projection onto {n_coords} of {d} output coordinates "
-                        f"(scaled x{d // n_coords}; the work is linear in d), {t3 - t0:.1f} s of CPU time, single thread"))
+    cores = host_cores()
+    t_begin = time.perf_counter()
+    smp = OracleProjectionSample(cores)
+    smp.run()
+    per_grad = min(smp.run()[0] for _ in range(2))
+    one = OracleProjectionSample(1, coords_per_thread=16)
+    per_grad_1 = one.run()[0]
+    out = dict(value=1.0 / per_grad, unit="grads/s", cores=cores, kind="oracle", sample=smp.describe(),
+               one_thread=dict(value=1.0 / per_grad_1, unit="grads/s", cores=1, sample=one.describe()))
+    # scoring: sampled train rows x all validation vectors x all checkpoints
+    cfg = W.CONFIGS["c3_score_sweep"]
+    d, C, V = cfg["d"], cfg["C"], sum(cfg["tasks"])
+    off = W.task_offsets(cfg["tasks"]).tolist()
+    n1, nall = 128, max(256, 16 * cores)
+    xt = W.lowrank_gaussian_features(nall, d, C, seed=SEED + 7).numpy()
+    xv = W.lowrank_gaussian_features(V, d, C, seed=SEED + 8).numpy()
+    scoring = {}
+    for b in cfg["bits"]:
+        tq = [oracle.quantize_rows(xt[i], b) for i in range(C)]
+        vq = [oracle.quantize_rows(xv[i], b) for i in range(C)]
+        tc, ts = np.stack([q[0] for q in tq]), np.stack([q[1] for q in tq])
+        vc, vs = np.stack([q[0] for q in vq]), np.stack([q[1] for q in vq])
+
+        def part(r, tc=tc, ts=ts, vc=vc, vs=vs, b=b):
+            return oracle.score(np.ascontiguousarray(tc[:, r[0]:r[1]]), vc, np.ascontiguousarray(ts[:, r[0]:r[1]]), vs, cfg["lr"], off, d, b)
+        t0 = time.perf_counter()
+        part((0, n1))
+        t1 = time.perf_counter()
+        edges = np.linspace(0, nall, cores + 1).astype(int)
+        _threaded(part, [(int(edges[k]), int(edges[k + 1])) for k in range(cores) if edges[k + 1] > edges[k]], cores)
+        t2 = time.perf_counter()
+        scoring[str(b)] = dict(scores_per_s_one_thread=n1 * V / (t1 - t0), scores_per_s_all_cores=nall * V / (t2 - t1),
+                               rows_one_thread=n1, rows_all_cores=nall)
+    out["scoring_c3_c4"] = dict(per_bits=scoring, cores=cores,
+                                sample=(f"{n1} (one thread) / {nall} (all cores) sampled train rows x {V} validation vectors x {C} "
+                                        f"checkpoints at d={d}; a score = one (train, validation) pair aggregated over the checkpoints; "
+                                        f"the oracle's time per train row does not depend on N, so config 4 (1-bit) has the 1-bit rate"))
+    sel = {}
+    for name, N, frac in (("c3_270000_top5pct", 270_000, 0.05), ("c4_2000000_top1pct", 2_000_000, 0.01)):
+        sc = np.random.default_rng(SEED).standard_normal(N).astype(np.float32)
+        t0 = time.perf_counter()
+        oracle.select_topk(sc, frac)
+        sel[name] = dict(ms=(time.perf_counter() - t0) * 1e3, cores=1)
+    out["select"] = dict(sizes=sel, note="full size; the oracle's selection is one sort, so one thread is all it uses")
+    out["seconds_spent"] = time.perf_counter() - t_begin
+    return out
 
 
 def max_over_ranks(ms_local, dist=None, device=None):
@@ -262,6 +340,22 @@ def stage_measurements(torch, B, W, dev, peaks):
     ck = smp.stop()
     i8_sustained = ops / ms / 1e9
     out["microbench"].update(int8_tops_sustained=i8_sustained, int8_sustained_clocks=ck)
+    # the int8 MMAs of 8-bit scoring reading, for every K block, operands that TMA has just streamed from a buffer of
+    # pseudo-random int8 values: the tensor pipe on data that changes, held for about two seconds with the clocks
+    # sampled. This is the sustained figure a scoring kernel can be held against: same shape, same data statistics,
+    # no epilogue, no HBM.
+    gen = torch.Generator(device=dev); gen.manual_seed(SEED + 11)
+    rnd = torch.randint(-127, 128, (4 << 20,), generator=gen, device=dev, dtype=torch.int8).view(torch.uint8)
+    B.qless_microbench("i8_n448_streamed_operands", 20000, device=dev, scratch=rnd)
+    smp = ClockSampler(torch.cuda.current_device())
+    smp.start()
+    ms, ops = B.qless_microbench("i8_n448_streamed_operands", 3_000_000, device=dev, scratch=rnd)
+    ck_rand = smp.stop()
+    i8_random = ops / ms / 1e9
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    out["microbench"].update(int8_tops_random_operands_sustained=i8_random, int8_random_operands_clocks=ck_rand,
+                             int8_random_operands_seconds=ms * 1e-3)
+    del rnd
     d = 8192
     # ---- quantise ----
     n = 65536
@@ -320,7 +414,11 @@ def stage_measurements(torch, B, W, dev, peaks):
         ck = smp.stop()
         if b == 1:
             sc_1bit = sc.clone()        # for the selected-percentage sweep below
-        e.update(ms_sustained=ts_, frac_of_int8_sustained=iops / ts_ / 1e9 / i8_sustained, sustained_clocks=ck)
+        e.update(ms_sustained=ts_, frac_of_int8_sustained=iops / ts_ / 1e9 / i8_sustained, sustained_clocks=ck,
+                 frac_of_int8_random_operands_sustained=iops / ts_ / 1e9 / i8_random)
+        if ck.get("sm_mhz"):
+            # against what the hardware's unit count allows at the SM clock this very loop was granted
+            e.update(frac_of_hw_int8_at_sampled_clock=iops / ts_ / 1e9 / (sms * HW_INT8_OP_PER_CLK_SM * ck["sm_mhz"] * 1e6 / 1e12))
         if ck.get("sm_mhz") and ck.get("sm_max_mhz"):
             # the micro-benchmark holds the maximum clock (its operands never change, so it draws little power); the
             # scoring kernel runs under the power cap: its rate against the tensor peak at the clock it actually had
@@ -418,7 +516,8 @@ def stage_measurements(torch, B, W, dev, peaks):
                                               scores=sc, workspace=ws), 2)
     iops = 2.0 * N * V * C * d
     out["score_c4_2000000x448x4_1bit"] = dict(ms=t, scores_per_s=N * V / (t * 1e-3), bound="tensor",
-                                              achieved_tops=iops / t / 1e9, frac_of_int8_peak=iops / t / 1e9 / i8_peak)
+                                              achieved_tops=iops / t / 1e9, frac_of_int8_peak=iops / t / 1e9 / i8_peak,
+                                              frac_of_int8_random_operands_sustained=iops / t / 1e9 / i8_random)
     # the same store through the XOR + population-count kernel (CUDA cores), against the integer-ALU peak
     B.qless_set_score_path(1)
     try:
@@ -450,22 +549,75 @@ def stage_measurements(torch, B, W, dev, peaks):
     ws = torch.empty(B.qless_project_quantize_workspace(n, P, d, 4), dtype=torch.uint8, device=dev)
     pq = {}
     for name, kind in (("rademacher", B.RADEMACHER), ("gaussian", B.GAUSSIAN)):
-        B.qless_set_projection_matrix(kind)
         try:
             B.qless_profile_collect()
             B.qless_profile_enable(True)
             for _ in range(4):
-                B.qless_project_quantize(g, d, SEED, 4, workspace=ws)
+                B.qless_project_quantize(g, d, SEED, 4, workspace=ws, matrix=kind)
             torch.cuda.synchronize()
             prof = B.qless_profile_collect()
         finally:
             B.qless_profile_enable(False)
-            B.qless_set_projection_matrix(B.RADEMACHER)
         t = prof["project"][0] / prof["project"][1]
         pq[name] = dict(ms=t, tflops=2.0 * n * P * d / t / 1e9, grads_per_s=n / (t * 1e-3))
     pq["note"] = "projection kernel alone, 256 bf16 rows, P = 2^20; the Gaussian matrix is bounded by its generator warps"
     out["project_256x2^20_by_matrix"] = pq
     B.qless_check()
+    return out
+
+
+# Tensor-pipe rates the hardware cannot exceed: dense bf16 (fp32 accumulation) 8192 flop and int8 16384 operations per
+# clock per SM (the unit counts behind the nominal 2.25 / 4.5 Pop/s at the nominal clock); times the SM count and a clock.
+HW_BF16_FLOP_PER_CLK_SM = 8192.0
+HW_INT8_OP_PER_CLK_SM = 16384.0
+
+
+def roofline_entry(achieved_tflops, peaks, clocks, sm_count=148):
+    """Roofline object of the projection kernel. `frac` is against the measured sustained library GEMM (the kernel is
+    timed inside a long step); a kernel can beat a library figure, so two denominators that it cannot beat stand
+    beside it: the hardware's unit count at the SM clock sampled while the timed region ran, and at the maximum clock."""
+    r = dict(bound="tensor", kernel="project", achieved=achieved_tflops, peak=peaks["bf16_sustained"], unit="TFLOP/s",
+             frac=(achieved_tflops / peaks["bf16_sustained"]) if achieved_tflops else None,
+             peak_source=f"{peaks['source']} (sustained bf16 GEMM of a library; burst {peaks['bf16_burst']})")
+    if achieved_tflops:
+        r["frac_of_burst_matmul"] = achieved_tflops / peaks["bf16_burst"]
+        mx = clocks.get("sm_max_mhz") or 1965.0
+        r["hw_peak_at_max_clock"] = sm_count * HW_BF16_FLOP_PER_CLK_SM * mx * 1e6 / 1e12
+        r["frac_of_hw_peak_at_max_clock"] = achieved_tflops / r["hw_peak_at_max_clock"]
+        if clocks.get("sm_mhz"):
+            r["hw_peak_at_sampled_clock"] = sm_count * HW_BF16_FLOP_PER_CLK_SM * clocks["sm_mhz"] * 1e6 / 1e12
+            r["frac_of_hw_peak_at_sampled_clock"] = achieved_tflops / r["hw_peak_at_sampled_clock"]
+    return r
+
+
+def summarize(stages, cpu, peaks, step_kernels_ms):
+    """Compact per-kernel figures taken from the stage measurements (and the oracle's rates beside them)."""
+    def pick(e, keys):
+        return {k: e[k] for k in keys if k in e}
+    c3 = stages.get("score_c3_270000x448x4", {})
+    scoring = {"c3": {}, "c4": {}}
+    keys = ("ms", "scores_per_s", "frac_of_int8_peak", "frac_of_int8_sustained", "frac_of_int8_random_operands_sustained",
+            "frac_of_hw_int8_at_sampled_clock", "frac_of_popc_peak", "frac_of_bf16_peak")
+    for b in ("8", "4", "2", "1", "1_popc", "16"):
+        if b in c3:
+            scoring["c3"][b] = pick(c3[b], keys)
+    if "score_c4_2000000x448x4_1bit" in stages:
+        scoring["c4"]["1"] = pick(stages["score_c4_2000000x448x4_1bit"], keys)
+    if "score_c4_2000000x448x4_1bit_popc" in stages:
+        scoring["c4"]["1_popc"] = pick(stages["score_c4_2000000x448x4_1bit_popc"], keys)
+    mb = stages.get("microbench", {})
+    out = dict(scoring=scoring,
+               peaks=dict(int8_tops_burst=mb.get("int8_tops"), int8_tops_sustained=mb.get("int8_tops_sustained"),
+                          int8_tops_random_operands_sustained=mb.get("int8_tops_random_operands_sustained"),
+                          popc_twordops=mb.get("popc_xor_add_twordops"), bf16_tcgen05_tflops=mb.get("bf16_tcgen05_tflops"),
+                          hbm_gbs=peaks["hbm_gbs"], source="library micro-benchmarks (tcgen05 int8, XOR+POPC+IADD); HBM: " + peaks["source"]),
+               quantize_65536x8192={b: pick(e, ("ms", "frac_of_hbm")) for b, e in stages.get("quantize_65536x8192", {}).items()},
+               step_kernels_ms=step_kernels_ms,
+               select={k: pick(stages[k], ("ms", "frac_of_hbm")) for k in ("select_c3_270000_top5pct", "select_c4_2000000_top1pct", "select_2^28_top5pct") if k in stages})
+    if cpu and "scoring_c3_c4" in cpu:
+        out["scoring_cpu_oracle_scores_per_s"] = {b: pick(e, ("scores_per_s_one_thread", "scores_per_s_all_cores"))
+                                                  for b, e in cpu["scoring_c3_c4"]["per_bits"].items()}
+        out["scoring_cpu_oracle_cores"] = cpu["scoring_c3_c4"]["cores"]
     return out
 
 
@@ -605,24 +757,28 @@ def run_ours(args):
         proj_ms, proj_cnt = prof.get("project", (0.0, 0))
         flops = 2.0 * n * P * d
         achieved = flops / (proj_ms / max(proj_cnt, 1) * 1e-3) / 1e12 if proj_cnt else None
-        roofline = dict(bound="tensor", kernel="project", achieved=achieved, peak=peaks["bf16_sustained"],
-                        unit="TFLOP/s", frac=(achieved / peaks["bf16_sustained"]) if achieved else None,
-                        traffic=PROJECT_TRAFFIC_BYTES_PER_P * P, traffic_source=PROJECT_TRAFFIC_SOURCE, peak_source=f"{peaks['source']} (sustained bf16; burst {peaks['bf16_burst']})",
+        roofline = roofline_entry(achieved, peaks, clocks, sm_count=torch.cuda.get_device_properties(dev).multi_processor_count)
+        roofline.update(traffic=PROJECT_TRAFFIC_BYTES_PER_P * P, traffic_source=PROJECT_TRAFFIC_SOURCE,
                         flops_per_launch=flops, ms_per_launch=proj_ms / max(proj_cnt, 1))
         line = dict(metric="grads projected+quantized/s (P=2^23,d=8192)", value=value, unit="grads/s",
                     n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=ms_total / args.steps,
                     higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
-                    config=dict(workload=WORKLOAD, batch_rows=n, P=P, d=d, bits=bits, val_rows=N_VAL, tasks=TASKS,
-                                select_frac=FRAC, l2="inputs larger than L2 (4.3 GB batch), no flush"),
+                    config=bench_config(cfg),
                     clocks=clocks, gpu_launches=launches, roofline=roofline,
                     stages_ms_per_step={k: ms / args.steps for k, (ms, c) in prof.items()},
                     e2e=e2e)
+        stages = None
         if world == 1 and not args.no_stages:
             del g, out
             torch.cuda.empty_cache()
-            line["stages"] = stage_measurements(torch, B, W, dev, peaks)
+            stages = stage_measurements(torch, B, W, dev, peaks)
+            line["stages"] = stages
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline()
+        if stages is not None:
+            # the second half of the metric (train x validation scores per second per code width) and the HBM-bound
+            # kernels, compact and last, so that a reader of the end of the line sees them
+            line["summary"] = summarize(stages, line.get("cpu_baseline"), peaks, line["stages_ms_per_step"])
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

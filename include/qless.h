@@ -67,6 +67,15 @@ const char* qless_last_error(void);
  * QLESS_ERR_TIMEOUT or QLESS_ERR_CUDA. */
 qless_status qless_check(void* cuda_stream);
 
+/* Self-test of that machinery (no counterpart in the paper). Enqueues a one-block kernel in which one thread waits,
+ * with the library's own bounded-wait routine and a limit of `polls` polls (256 .. 65536), on a barrier that nothing
+ * ever signals, while a second thread waits on another such barrier with a limit 256 times larger. The first gives
+ * up, records the producer code (0x1) in the device timeout word and raises the block-wide abort flag; the second
+ * must leave on seeing that flag without recording a code of its own; the kernel then returns normally. The next
+ * qless_check on the stream therefore returns QLESS_ERR_TIMEOUT (message: code 0x1) and the one after it QLESS_OK.
+ * No tensor memory is touched and no copy is started. Returns QLESS_ERR_INVALID_ARG for polls out of range. */
+qless_status qless_selftest_timeout(int32_t polls, void* cuda_stream);
+
 /* Per-kernel timing for benchmarks (no counterpart in the paper; measurement aid). While enabled on the
  * calling thread, every kernel the library launches is bracketed by CUDA events on the call's stream.
  * qless_profile_collect synchronises those events, writes "name=milliseconds*launches;..." (time summed
@@ -88,7 +97,10 @@ qless_status qless_profile_collect(char* buf /* host */, size_t buflen);
  * 16-byte aligned device buffer of >= 4 MiB, QLESS_ERR_WORKSPACE otherwise); 10 = 8 and 9 together as 8-bit
  * scoring runs them (the MMAs of one K block committed at once, one 48 KiB stage per K block streamed into other
  * shared memory three stages ahead, the MMAs never waiting for data; same scratch; operations counted are the
- * MMAs'); 11 = the kernel of 10 with the copies switched off. Runs the kernel twice and times
+ * MMAs'); 11 = the kernel of 10 with the copies switched off; 12 = the MMAs of 8 reading, for every K block, a
+ * stage that TMA has just brought from the scratch buffer (same scratch size; the CALLER fills it with the int8
+ * values the operands are to take, e.g. pseudo-random ones: the operands then change with every K block, which
+ * is what sets the power drawn and so the clock granted under the power cap). Runs the kernel twice and times
  * the second run with CUDA events on `cuda_stream` (synchronises it). *ms_out: milliseconds; *ops_out:
  * operations executed (2 x multiply-accumulates; word operations for 6; bytes moved for 9). Host pointers. */
 qless_status qless_microbench(int32_t what, int32_t iters, float* ms_out, double* ops_out, void* scratch,
@@ -98,8 +110,8 @@ qless_status qless_microbench(int32_t what, int32_t iters, float* ms_out, double
  * Stage 1 + 2: datastore construction (paper Sec. 2.2 Eq. 1-2, Sec. 3.1, Eq. 4-5).
  *
  * For each of the n gradient rows g (row-major [n, P], leading dimension ld_grads elements):
- *   Gamma = Adam direction of g given the checkpoint's moments (Sec. 2.2 "Adam training gradient
- *           Gamma(z; theta)"):  m' = b1 m + (1-b1) g, v' = b2 v + (1-b2) g^2, (bias-corrected if
+ *   Gamma = Adam direction of g given the checkpoint's moments (the training-side gradient of Sec. 2.2, which
+ *           the paper names without a formula):  m' = b1 m + (1-b1) g, v' = b2 v + (1-b2) g^2, (bias-corrected if
  *           step > 0), Gamma = m' / (sqrt(v') + eps), computed in fp32 and rounded to bf16.
  *           adam_m = adam_v = NULL selects the SGD (validation) gradient: Gamma = bf16(g).
  *   y     = R Gamma (Eq. 1), R in {+-1/sqrt(d)}^{d x P} Rademacher. R is never stored: entry
@@ -147,24 +159,64 @@ qless_status qless_project_quantize_host(
     void* codes_host, float* scales_host, int32_t* code_sumsq_host /* NULL to skip */,
     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* Test hook: which kernel computes the projection of Eq. 1 in qless_project_quantize. 0 (default): the
+/* The same two calls with the random matrix R of Eq. 1 chosen per call (Sec. 2.4 leaves its distribution open
+ * between Gaussian and Rademacher; R is a property of a datastore, fixed by (seed, matrix) for every vector that
+ * will be scored together, so it travels with the call and not in library state: two host threads may build a
+ * Rademacher and a Gaussian store at the same time). `projection` is a HOST pointer, NULL = defaults
+ * (QLESS_MATRIX_RADEMACHER, which is what qless_project_quantize and qless_project_quantize_host use).
+ *   QLESS_MATRIX_RADEMACHER: entries +-1/sqrt(d), entry map above.
+ *   QLESS_MATRIX_GAUSSIAN:   entries z/sqrt(d) with z standard normal, rounded to bf16 (the operand type of the
+ *     contraction): the four entries of row r in columns 4q .. 4q+3 come from one Philox4x32-10 call with counter
+ *     (q mod 2^32, r, q div 2^32, 1) and the same key; output words (w0, w1) give columns 4q, 4q+1 and (w2, w3)
+ *     give 4q+2, 4q+3 by the Box-Muller transform z_even = sqrt(-2 ln u1) cos(2 pi u2),
+ *     z_odd = sqrt(-2 ln u1) sin(2 pi u2) with u = (floor(w / 2^9) + 1/2) / 2^23. The logarithm, square root, sine
+ *     and cosine are evaluated in fp32 on the GPU's approximate units, so an entry may differ from the correctly
+ *     rounded one by one bf16 step where it falls next to a rounding boundary. The generator, not the tensor pipe,
+ *     bounds this variant.
+ * Every other argument, output, requirement and error is that of the call without the suffix; a matrix value other
+ * than the two above (or a non-zero reserved field) returns QLESS_ERR_INVALID_ARG. */
+enum { QLESS_MATRIX_RADEMACHER = 0, QLESS_MATRIX_GAUSSIAN = 1 };
+typedef struct {
+    int32_t matrix;      /* QLESS_MATRIX_RADEMACHER */
+    int32_t reserved[3]; /* must be 0 */
+} qless_projection_cfg;
+
+qless_status qless_project_quantize_ex(
+    const void* grads, qless_dtype dtype, int64_t n, int64_t ld_grads,
+    const float* adam_m, const float* adam_v, const qless_adam_cfg* adam /* host, NULL = defaults */,
+    int64_t P, int32_t d, uint64_t seed, const qless_projection_cfg* projection /* host, NULL = defaults */,
+    int32_t bits, void* codes, float* scales, int32_t* code_sumsq, float* proj_out,
+    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+qless_status qless_project_quantize_host_ex(
+    const void* grads_host, qless_dtype dtype, int64_t n, int64_t ld_grads,
+    const float* adam_m, const float* adam_v, const qless_adam_cfg* adam /* host, NULL = defaults */,
+    int64_t P, int32_t d, uint64_t seed, const qless_projection_cfg* projection /* host, NULL = defaults */,
+    int32_t bits, void* codes_host, float* scales_host, int32_t* code_sumsq_host /* NULL to skip */,
+    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---- Hooks for tests and measurements only. They select between kernels that compute the SAME result, are
+ * process-wide (every thread's later calls take the chosen kernel), and are not meant for production callers:
+ * leave them at 0. ---- */
+
+/* Which kernel computes the projection of Eq. 1 in qless_project_quantize. 0 (default): the
  * tcgen05 tensor-core kernel; 1: a plain CUDA-core kernel of the same definition, kept so that the
  * tensor-core result can be cross-checked on the device at sizes the CPU oracle only samples (it is
- * also what runs when P >= 2^31). Process-wide. */
+ * also what runs when P >= 2^31). */
 qless_status qless_set_projection_path(int32_t path);
 
-/* Test hook, as above, for the integer similarity in qless_score and qless_score_dots: 0 (default) the
+/* As above, for the integer similarity in qless_score and qless_score_dots: 0 (default) the
  * tcgen05 int8 kernel for every code width (used when T <= 8; sub-byte codes, sign bits included, are expanded
  * to int8 on the way), 1 the CUDA-core kernels (dp4a for 8-, 4- and 2-bit codes, XOR + population count for
- * 1-bit codes). Process-wide. */
+ * 1-bit codes). */
 qless_status qless_set_score_path(int32_t path);
 
-/* Test hook for qless_select_topk. 0 (default): up to 360 448 scores one launch of a thread-block cluster that
+/* As above, for qless_select_topk. 0 (default): up to 360 448 scores one launch of a thread-block cluster that
  * keeps the keys in shared memory (one read, no workspace used); up to 2^22 the multi-pass radix select (five
- * reads); above, a sampled lower bracket of the k-th largest key, one gather pass and a radix select on the
- * gathered candidates (two reads), with the multi-pass select enqueued behind it as a device-gated fallback.
+ * reads); above, a sampled bracket of the k-th largest key, one gather pass and a radix select on the
+ * gathered candidates, with the multi-pass select as the fallback when the bracket misses.
  * 1: multi-pass at every N. 2: as 0, with the bracket forced above every key, so that the fallback does the
- * work. The result is the same in all three. Process-wide. */
+ * work. The result is the same in all three. */
 qless_status qless_set_select_path(int32_t path);
 
 /* Stage 2 alone (Eq. 2, Eq. 4-5, packing) on fp32 rows x [n, d]; normalize = 0 skips Eq. 2 so that
@@ -193,21 +245,6 @@ qless_status qless_adam_gamma(
 qless_status qless_philox_entries(
     uint64_t seed, int64_t r0, int64_t nr, int64_t j0, int64_t nj, int8_t* out, void* cuda_stream);
 
-/* Which random matrix R the projection of Eq. 1 uses in qless_project_quantize and
- * qless_project_quantize_host (Sec. 2.4 leaves the distribution open between Gaussian and Rademacher).
- * QLESS_MATRIX_RADEMACHER (default): entries +-1/sqrt(d), entry map above. QLESS_MATRIX_GAUSSIAN: entries
- * z/sqrt(d) with z standard normal, rounded to bf16 (the operand type of the contraction): the four entries of
- * row r in columns 4q .. 4q+3 come from one Philox4x32-10 call with counter (q mod 2^32, r, q div 2^32, 1) and
- * the same key; output words (w0, w1) give columns 4q, 4q+1 and (w2, w3) give 4q+2, 4q+3 by the Box-Muller
- * transform z_even = sqrt(-2 ln u1) cos(2 pi u2), z_odd = sqrt(-2 ln u1) sin(2 pi u2) with
- * u = (floor(w / 2^9) + 1/2) / 2^23. The logarithm, square root, sine and cosine are evaluated in fp32 on the
- * GPU's approximate units, so an entry may differ from the correctly rounded one by one bf16 step where it falls next to a rounding boundary.
- * The generator, not the tensor pipe, bounds this variant (about 20 instructions per entry against one; the projection takes about 4.5 times as long).
- * Process-wide; stores built with different matrices (or seeds) must not be scored against each other.
- * Returns QLESS_ERR_INVALID_ARG for any other value. */
-enum { QLESS_MATRIX_RADEMACHER = 0, QLESS_MATRIX_GAUSSIAN = 1 };
-qless_status qless_set_projection_matrix(int32_t kind);
-
 /* Entries of the Gaussian matrix as the kernels generate them: out [nr, nj] fp32 (device; bf16-representable
  * values of sqrt(d) R) for rows r0 .. r0+nr-1 and columns j0 .. j0+nj-1; j0 must be a multiple of 4. */
 qless_status qless_gaussian_entries(
@@ -230,6 +267,10 @@ qless_status qless_gaussian_entries(
  * [C][N] / [C][V] int32 as produced by qless_project_quantize; NULL = recomputed from the codes.
  * lr_weights: host [C] (eta_i, used as given). task_offsets: host [T+1], strictly increasing,
  * [0] = 0, [T] = V. scores [N] fp32; per_task [N, T] fp32 or NULL.
+ * The two host arrays reach the device through copies from pageable memory enqueued on `cuda_stream`: the runtime
+ * stages them before the call returns (the arrays may be freed at once), but such a copy may wait for earlier work
+ * of the stream, so this call (and qless_score_16bit) can block for that long and must not be issued while the
+ * stream is being captured into a graph.
  * Requirements: d % 128 == 0, d <= 8192; 1 <= V <= 4096; 1 <= T <= 64; 1 <= C <= 64.
  * ------------------------------------------------------------------------------------------ */
 typedef enum { QLESS_SCORE_COSINE = 0, QLESS_SCORE_DEQUANT = 1 } qless_score_mode;

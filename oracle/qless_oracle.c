@@ -128,8 +128,8 @@ float qlo_round_to_bf16(float x)
 }
 
 /* ------------------------------------------------------------------------- */
-/* Adam training gradient Gamma(z; theta) (paper Sec. 2.2: "extracting Adam   */
-/* training gradient Gamma(z; theta) for each training sample z"). The paper  */
+/* Adam training gradient Gamma(z; theta) of a training example z (paper      */
+/* Sec. 2.2). The paper                                                        */
 /* names it without a formula; the reading taken is the Adam update direction */
 /* the optimiser would apply if the example's gradient g were the next one,   */
 /* given the checkpoint's moments m, v:                                       */

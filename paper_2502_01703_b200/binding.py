@@ -25,7 +25,7 @@ EXPORTS = [
     "qless_project_quantize_host_workspace", "qless_project_quantize_host", "qless_profile_enable",
     "qless_profile_collect", "qless_kernel_launches", "qless_select_topk_static",
     "qless_set_projection_path", "qless_set_score_path", "qless_set_select_path", "qless_microbench",
-    "qless_set_projection_matrix", "qless_gaussian_entries",
+    "qless_project_quantize_ex", "qless_project_quantize_host_ex", "qless_gaussian_entries", "qless_selftest_timeout",
 ]
 RADEMACHER, GAUSSIAN = 0, 1
 SELECT_STATIC_MAX_N = 1 << 22
@@ -33,6 +33,10 @@ SELECT_STATIC_MAX_N = 1 << 22
 
 class AdamCfg(C.Structure):
     _fields_ = [("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float), ("step", C.c_int64)]
+
+
+class ProjectionCfg(C.Structure):
+    _fields_ = [("matrix", C.c_int32), ("reserved", C.c_int32 * 3)]
 
 
 class QlessError(RuntimeError):
@@ -109,8 +113,14 @@ def lib():
         L.qless_set_select_path.argtypes = [i32]
         L.qless_set_projection_path.restype = C.c_int
         L.qless_set_projection_path.argtypes = [i32]
-        L.qless_set_projection_matrix.restype = C.c_int
-        L.qless_set_projection_matrix.argtypes = [i32]
+        L.qless_project_quantize_ex.restype = C.c_int
+        L.qless_project_quantize_ex.argtypes = [vp, C.c_int, i64, i64, vp, vp, C.POINTER(AdamCfg), i64, i32, u64,
+                                                C.POINTER(ProjectionCfg), i32, vp, vp, vp, vp, vp, sz, vp]
+        L.qless_project_quantize_host_ex.restype = C.c_int
+        L.qless_project_quantize_host_ex.argtypes = [vp, C.c_int, i64, i64, vp, vp, C.POINTER(AdamCfg), i64, i32, u64,
+                                                     C.POINTER(ProjectionCfg), i32, vp, vp, vp, vp, sz, vp]
+        L.qless_selftest_timeout.restype = C.c_int
+        L.qless_selftest_timeout.argtypes = [i32, vp]
         L.qless_gaussian_entries.restype = C.c_int
         L.qless_gaussian_entries.argtypes = [C.c_uint64, i64, i64, i64, i64, vp, vp]
         L.qless_select_topk_static.restype = C.c_int
@@ -148,6 +158,10 @@ def _adam(adam):
                            int(adam.get("step", 0))))
 
 
+def _projection(matrix):
+    return C.byref(ProjectionCfg(int(matrix), (C.c_int32 * 3)(0, 0, 0)))
+
+
 def _workspace(nbytes, device, workspace):
     if workspace is not None:
         return workspace
@@ -167,9 +181,11 @@ def qless_project_quantize_workspace(n, P, d, bits):
 
 
 def qless_project_quantize(grads, d, seed, bits, adam_m=None, adam_v=None, adam=None, want_sumsq=True,
-                           want_proj=False, out=None, workspace=None, stream=None):
+                           want_proj=False, out=None, workspace=None, stream=None, matrix=None):
     """grads [n, P] f32/bf16 (row stride allowed) -> dict(codes uint8 [n, d*bits/8], scales f32 [n],
-    sumsq i32 [n] | None, proj f32 [n, d] | None). `out` may pass preallocated tensors by those names."""
+    sumsq i32 [n] | None, proj f32 [n, d] | None). `out` may pass preallocated tensors by those names.
+    matrix = None calls qless_project_quantize; RADEMACHER / GAUSSIAN call qless_project_quantize_ex with that
+    matrix in its projection config."""
     n, P = grads.shape
     dev = grads.device
     out = out or {}
@@ -182,10 +198,16 @@ def qless_project_quantize(grads, d, seed, bits, adam_m=None, adam_v=None, adam=
     sumsq = out.get("sumsq", torch.empty(n, dtype=torch.int32, device=dev) if want_sumsq else None)
     proj = out.get("proj", torch.empty((n, d), dtype=torch.float32, device=dev) if want_proj else None)
     ws = _workspace(qless_project_quantize_workspace(n, P, d, bits), dev, workspace)
-    _check(lib().qless_project_quantize(_ptr(grads), _dtype_code(grads), n, grads.stride(0) if n > 0 else P,
-                                        _ptr(adam_m), _ptr(adam_v), _adam(adam), P, d, seed, bits,
-                                        _ptr(codes), _ptr(scales), _ptr(sumsq), _ptr(proj),
-                                        _ptr(ws), ws.numel(), _stream(stream)))
+    if matrix is None:
+        _check(lib().qless_project_quantize(_ptr(grads), _dtype_code(grads), n, grads.stride(0) if n > 0 else P,
+                                            _ptr(adam_m), _ptr(adam_v), _adam(adam), P, d, seed, bits,
+                                            _ptr(codes), _ptr(scales), _ptr(sumsq), _ptr(proj),
+                                            _ptr(ws), ws.numel(), _stream(stream)))
+    else:
+        _check(lib().qless_project_quantize_ex(_ptr(grads), _dtype_code(grads), n, grads.stride(0) if n > 0 else P,
+                                               _ptr(adam_m), _ptr(adam_v), _adam(adam), P, d, seed, _projection(matrix),
+                                               bits, _ptr(codes), _ptr(scales), _ptr(sumsq), _ptr(proj),
+                                               _ptr(ws), ws.numel(), _stream(stream)))
     return dict(codes=codes, scales=scales, sumsq=sumsq, proj=proj)
 
 
@@ -194,7 +216,7 @@ def qless_project_quantize_host_workspace(n, P, d, bits, dtype_code):
 
 
 def qless_project_quantize_host(grads_host, d, seed, bits, adam_m=None, adam_v=None, adam=None, out=None,
-                                workspace=None, device="cuda", stream=None):
+                                workspace=None, device="cuda", stream=None, matrix=None):
     """grads_host: CPU tensor [n, P] (pinned for asynchronous copies); adam_m / adam_v: device tensors.
     Returns dict(codes, scales, sumsq) of CPU tensors (pinned), valid once the stream has drained."""
     n, P = grads_host.shape
@@ -210,10 +232,16 @@ def qless_project_quantize_host(grads_host, d, seed, bits, adam_m=None, adam_v=N
         sumsq = torch.empty(n, dtype=torch.int32).pin_memory()
     code = _dtype_code(grads_host)
     ws = _workspace(qless_project_quantize_host_workspace(n, P, d, bits, code), device, workspace)
-    _check(lib().qless_project_quantize_host(_ptr(grads_host), code, n, grads_host.stride(0) if n > 0 else P,
-                                             _ptr(adam_m), _ptr(adam_v), _adam(adam), P, d, seed, bits,
-                                             _ptr(codes), _ptr(scales), _ptr(sumsq), _ptr(ws), ws.numel(),
-                                             _stream(stream)))
+    if matrix is None:
+        _check(lib().qless_project_quantize_host(_ptr(grads_host), code, n, grads_host.stride(0) if n > 0 else P,
+                                                 _ptr(adam_m), _ptr(adam_v), _adam(adam), P, d, seed, bits,
+                                                 _ptr(codes), _ptr(scales), _ptr(sumsq), _ptr(ws), ws.numel(),
+                                                 _stream(stream)))
+    else:
+        _check(lib().qless_project_quantize_host_ex(_ptr(grads_host), code, n, grads_host.stride(0) if n > 0 else P,
+                                                    _ptr(adam_m), _ptr(adam_v), _adam(adam), P, d, seed,
+                                                    _projection(matrix), bits, _ptr(codes), _ptr(scales), _ptr(sumsq),
+                                                    _ptr(ws), ws.numel(), _stream(stream)))
     return dict(codes=codes, scales=scales, sumsq=sumsq)
 
 
@@ -392,9 +420,9 @@ def qless_set_projection_path(path):
     _check(lib().qless_set_projection_path(int(path)))
 
 
-def qless_set_projection_matrix(kind):
-    """RADEMACHER (0, default: the method's matrix) or GAUSSIAN (1): the random matrix of the projection."""
-    _check(lib().qless_set_projection_matrix(int(kind)))
+def qless_selftest_timeout(polls=1024, stream=None):
+    """Enqueues the bounded-wait self-test kernel; the next qless_check() on the stream raises ERR_TIMEOUT."""
+    _check(lib().qless_selftest_timeout(int(polls), _stream(stream)))
 
 
 def qless_set_select_path(path):
@@ -408,13 +436,15 @@ def qless_set_score_path(path):
 
 
 MICROBENCH = {"bf16_ss": 0, "bf16_ts": 1, "i8_ss": 2, "bf16_ss_pair": 3, "bf16_ts_pair": 4, "i8_ss_pair": 5, "popc": 6, "i8_ts_pair": 7,
-              "i8_ss_pair_n448": 8, "tma_l2_stream": 9, "i8_n448_with_tma": 10, "i8_n448_commit_per_block": 11}
+              "i8_ss_pair_n448": 8, "tma_l2_stream": 9, "i8_n448_with_tma": 10, "i8_n448_commit_per_block": 11, "i8_n448_streamed_operands": 12}
 
 
-def qless_microbench(what, iters, device="cuda", stream=None):
-    """(milliseconds, operations) of one peak-rate micro-benchmark; `what` is a key of MICROBENCH."""
+def qless_microbench(what, iters, device="cuda", stream=None, scratch=None):
+    """(milliseconds, operations) of one peak-rate micro-benchmark; `what` is a key of MICROBENCH. `scratch`: a
+    uint8 device tensor of at least 4 MiB whose contents the streaming benchmarks read (default: uninitialised)."""
     ms, ops = C.c_float(0), C.c_double(0)
-    scratch = torch.empty(4 << 20, dtype=torch.uint8, device=device)
+    if scratch is None:
+        scratch = torch.empty(4 << 20, dtype=torch.uint8, device=device)
     _check(lib().qless_microbench(MICROBENCH[what], int(iters), C.byref(ms), C.byref(ops), _ptr(scratch), scratch.numel(),
                                   _stream(stream)))
     return ms.value, ops.value

@@ -83,7 +83,6 @@ ProfileScope::~ProfileScope()
 
 static std::atomic<int> g_score_path{0};        // 0 = tensor cores for 8/4/2-bit codes, 1 = CUDA cores
 static std::atomic<int> g_projection_path{0};   // 0 = tensor cores, 1 = CUDA cores (cross-check hook)
-static std::atomic<int> g_projection_matrix{0}; // 0 = Rademacher (the method), 1 = Gaussian
 
 static bool valid_bits(int b) { return b == 1 || b == 2 || b == 4 || b == 8; }
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -102,6 +101,19 @@ static qless_status make_adam(const qless_adam_cfg* cfg, AdamParams* ap)
         ap->c1 = (float)(1.0 - std::pow((double)c.beta1, (double)c.step));
         ap->c2 = (float)(1.0 - std::pow((double)c.beta2, (double)c.step));
     }
+    return QLESS_OK;
+}
+
+// The random matrix of Eq. 1 travels with the call: NULL = Rademacher.
+static qless_status matrix_kind(const qless_projection_cfg* cfg, bool* gaussian)
+{
+    *gaussian = false;
+    if (cfg == nullptr) return QLESS_OK;
+    QLESS_REQUIRE(cfg->matrix == QLESS_MATRIX_RADEMACHER || cfg->matrix == QLESS_MATRIX_GAUSSIAN, QLESS_ERR_INVALID_ARG,
+                  "projection->matrix must be QLESS_MATRIX_RADEMACHER (0) or QLESS_MATRIX_GAUSSIAN (1) (matrix=%d)", cfg->matrix);
+    QLESS_REQUIRE(cfg->reserved[0] == 0 && cfg->reserved[1] == 0 && cfg->reserved[2] == 0, QLESS_ERR_INVALID_ARG,
+                  "projection->reserved must be zero");
+    *gaussian = cfg->matrix == QLESS_MATRIX_GAUSSIAN;
     return QLESS_OK;
 }
 
@@ -140,7 +152,8 @@ static PqWorkspace pq_layout(int64_t n, int64_t P, int32_t d)
 // buffer [P/64][n][64], the partial sums to the chunks of that range. Everything is enqueued on st.
 static qless_status project_columns(const void* grads, qless_dtype dtype, int64_t n, int64_t ld_grads, const float* adam_m,
                                     const float* adam_v, const AdamParams& ap, const ProjectPlan& full, int64_t j0,
-                                    int64_t len, uint64_t seed, __nv_bfloat16* gamma, float* part, cudaStream_t st)
+                                    int64_t len, uint64_t seed, bool gaussian, __nv_bfloat16* gamma, float* part,
+                                    cudaStream_t st)
 {
     const size_t esz = (dtype == QLESS_BF16) ? 2 : 4;
     const void* g_slab = reinterpret_cast<const uint8_t*>(grads) + (size_t)j0 * esz;
@@ -151,7 +164,7 @@ static qless_status project_columns(const void* grads, qless_dtype dtype, int64_
                                        ap, len, gamma_slab, true, st)); }
     ProjectPlan pl = full;
     pl.P = len; pl.k_base = j0;
-    pl.gaussian = (g_projection_matrix == 1);
+    pl.gaussian = gaussian;
     pl.num_chunks = (int32_t)((len + full.chunk - 1) / full.chunk);
     float* part_slab = part + (j0 / full.chunk) * n * (int64_t)full.d;
     if (g_projection_path == 0 && (len / 64) * n < ((int64_t)1 << 31)) {
@@ -211,14 +224,6 @@ qless_status qless_set_projection_path(int32_t path)
 {
     QLESS_REQUIRE(path == 0 || path == 1, QLESS_ERR_INVALID_ARG, "path must be 0 (tensor cores) or 1 (CUDA cores)");
     g_projection_path.store(path);
-    return QLESS_OK;
-}
-
-qless_status qless_set_projection_matrix(int32_t kind)
-{
-    QLESS_REQUIRE(kind == QLESS_MATRIX_RADEMACHER || kind == QLESS_MATRIX_GAUSSIAN, QLESS_ERR_INVALID_ARG,
-                  "kind must be QLESS_MATRIX_RADEMACHER (0) or QLESS_MATRIX_GAUSSIAN (1)");
-    g_projection_matrix.store(kind);
     return QLESS_OK;
 }
 
@@ -295,8 +300,21 @@ qless_status qless_project_quantize(const void* grads, qless_dtype dtype, int64_
                                     int32_t* code_sumsq, float* proj_out, void* workspace, size_t workspace_bytes,
                                     void* cuda_stream)
 {
+    return qless_project_quantize_ex(grads, dtype, n, ld_grads, adam_m, adam_v, adam, P, d, seed, nullptr, bits, codes,
+                                     scales, code_sumsq, proj_out, workspace, workspace_bytes, cuda_stream);
+}
+
+qless_status qless_project_quantize_ex(const void* grads, qless_dtype dtype, int64_t n, int64_t ld_grads,
+                                       const float* adam_m, const float* adam_v, const qless_adam_cfg* adam,
+                                       int64_t P, int32_t d, uint64_t seed, const qless_projection_cfg* projection,
+                                       int32_t bits, void* codes, float* scales, int32_t* code_sumsq, float* proj_out,
+                                       void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     qless_status s = check_grads(grads, dtype, n, ld_grads, adam_m, adam_v, P);
+    if (s != QLESS_OK) return s;
+    bool gaussian = false;
+    s = matrix_kind(projection, &gaussian);
     if (s != QLESS_OK) return s;
     QLESS_REQUIRE(valid_bits(bits), QLESS_ERR_UNSUPPORTED, "bits must be 1, 2, 4 or 8 (bits=%d)", bits);
     QLESS_REQUIRE(d >= 128 && d <= 8192 && d % 128 == 0, QLESS_ERR_UNSUPPORTED, "d must be a multiple of 128 in [128, 8192] (d=%d)", d);
@@ -313,7 +331,7 @@ qless_status qless_project_quantize(const void* grads, qless_dtype dtype, int64_
     uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
     __nv_bfloat16* gamma = reinterpret_cast<__nv_bfloat16*>(ws + w.gamma_off);
     float* part = reinterpret_cast<float*>(ws + w.part_off);
-    s = project_columns(grads, dtype, n, ld_grads, adam_m, adam_v, ap, w.plan, 0, P, seed, gamma, part, st);
+    s = project_columns(grads, dtype, n, ld_grads, adam_m, adam_v, ap, w.plan, 0, P, seed, gaussian, gamma, part, st);
     if (s != QLESS_OK) return s;
     const float inv_sqrt_d = 1.0f / sqrtf((float)d);
     { ProfileScope ps("quantize", st);
@@ -335,7 +353,19 @@ qless_status qless_project_quantize_host(const void* grads_host, qless_dtype dty
                                          float* scales_host, int32_t* code_sumsq_host, void* workspace,
                                          size_t workspace_bytes, void* cuda_stream)
 {
+    return qless_project_quantize_host_ex(grads_host, dtype, n, ld_grads, adam_m, adam_v, adam, P, d, seed, nullptr, bits,
+                                          codes_host, scales_host, code_sumsq_host, workspace, workspace_bytes, cuda_stream);
+}
+
+qless_status qless_project_quantize_host_ex(const void* grads_host, qless_dtype dtype, int64_t n, int64_t ld_grads,
+                                            const float* adam_m, const float* adam_v, const qless_adam_cfg* adam,
+                                            int64_t P, int32_t d, uint64_t seed, const qless_projection_cfg* projection,
+                                            int32_t bits, void* codes_host, float* scales_host, int32_t* code_sumsq_host,
+                                            void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    bool gaussian = false;
+    { const qless_status ms = matrix_kind(projection, &gaussian); if (ms != QLESS_OK) return ms; }
     QLESS_REQUIRE(n >= 0 && P > 0 && d > 0, QLESS_ERR_INVALID_ARG, "n >= 0, P > 0, d > 0 required");
     QLESS_REQUIRE(dtype == QLESS_F32 || dtype == QLESS_BF16, QLESS_ERR_INVALID_ARG, "dtype must be QLESS_F32 or QLESS_BF16");
     QLESS_REQUIRE(valid_bits(bits), QLESS_ERR_UNSUPPORTED, "bits must be 1, 2, 4 or 8 (bits=%d)", bits);
@@ -394,7 +424,7 @@ qless_status qless_project_quantize_host(const void* grads_host, qless_dtype dty
         if (ce == cudaSuccess) ce = cudaStreamWaitEvent(st, ev_slab, 0);
         cudaEventDestroy(ev_slab);
         if (ce != cudaSuccess) return cuda_fail(ce, "ordering a column slab before its projection");
-        s = project_columns(d_grads, dtype, n, P, adam_m, adam_v, ap, w.plan, j0, len, seed, gamma, part, st);
+        s = project_columns(d_grads, dtype, n, P, adam_m, adam_v, ap, w.plan, j0, len, seed, gaussian, gamma, part, st);
         if (s != QLESS_OK) return s;
     }
     { ProfileScope ps("quantize", st);

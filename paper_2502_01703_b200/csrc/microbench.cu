@@ -241,6 +241,93 @@ mma_tma_mix_kernel(const __grid_constant__ CUtensorMap tmap, int iters, int with
     }
 }
 
+// The int8 tensor pipe on operands that change: the leader of a CTA pair issues the MMAs of 8-bit scoring at 448
+// validation vectors (per K block four K steps of one N = 256 and one N = 192 MMA on the same A), and every K block
+// reads a stage that TMA has just brought from a 4 MiB buffer the caller filled with pseudo-random int8 values (256
+// distinct 16 KiB boxes, taken in a sequence that differs from CTA to CTA), MC_STAGES stages ahead. TMA streams four
+// times faster than the MMAs consume (micro-benchmark 9), so in steady state the MMAs never wait: what this adds to
+// micro-benchmark 8 is data that toggles the operand paths, i.e. the power the tensor pipe draws on real codes, and
+// with it the clock the power cap grants. The accumulator restarts every 64 K blocks, as a checkpoint of d = 8192 does.
+constexpr int MC_STAGES = 4;
+struct __align__(8) McBars { uint64_t done, full[MC_STAGES], empty[MC_STAGES]; uint32_t tmem_base; uint32_t abort_flag; };
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128, 1)
+mma_stream_consume_kernel(const __grid_constant__ CUtensorMap tmap, int iters, unsigned int* timeout_word)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    constexpr int STAGE = 3 * TS_BOX;                       // A (128 rows) | B rows of the N = 256 MMA | B rows of the N = 192 MMA
+    McBars* bars = reinterpret_cast<McBars*>(smem + (size_t)MC_STAGES * STAGE);
+    const int warp = threadIdx.x >> 5;
+    const uint32_t rank = cluster_ctarank();
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars->done), 1);
+        for (int s = 0; s < MC_STAGES; ++s) { mbar_init(smem_u32(&bars->full[s]), 1); mbar_init(smem_u32(&bars->empty[s]), 1); }
+        bars->abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tmap);
+    }
+    if (warp == 0) { tmem_alloc_pair(smem_u32(&bars->tmem_base), 512); tmem_relinquish_pair(); }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = bars->tmem_base;
+
+    if (threadIdx.x == 0 && rank == 0) {
+        const uint32_t idesc = make_idesc(2, 1, 1, 256, 256), idesc192 = make_idesc(2, 1, 1, 256, 192);
+        bool ok = true;
+        for (int it = 0; it < iters && ok; ++it) {
+            const int s = it % MC_STAGES;
+            ok = mbar_wait(smem_u32(&bars->full[s]), (uint32_t)(it / MC_STAGES) & 1u, &bars->abort_flag, timeout_word, TO_MMA);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t st = smem_u32(smem + (size_t)s * STAGE);
+            const uint64_t adesc = make_smem_desc_sw128(st);
+            const uint64_t bdesc = make_smem_desc_sw128(st + TS_BOX);
+            const uint64_t bdesc192 = make_smem_desc_sw128(st + 2 * TS_BOX);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t acc = ((it & 63) > 0 || k > 0) ? 1u : 0u;
+                mma_i8_ss_pair(tmem_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, acc);
+                mma_i8_ss_pair(tmem_base + 256, adesc + (uint64_t)(2 * k), bdesc192 + (uint64_t)(2 * k), idesc192, acc);
+            }
+            mma_commit_pair(smem_u32(&bars->empty[s]));      // arrives in both CTAs
+        }
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&bars->done)) : "memory");
+        mbar_wait_quiet(smem_u32(&bars->done), 0u);
+    } else if (threadIdx.x == 32) {
+        // both CTAs: this CTA's three boxes of every stage; all of a stage's bytes complete on the leader's barrier
+        bool ok = true;
+        uint32_t tile = blockIdx.x * 37u;
+        uint32_t issued = 0;
+        for (int it = 0; it < iters && ok; ++it) {
+            const int s = it % MC_STAGES;
+            if (it >= MC_STAGES) {
+                ok = mbar_wait_cluster(smem_u32(&bars->empty[s]), (uint32_t)(it / MC_STAGES - 1) & 1u, &bars->abort_flag, timeout_word, TO_PRODUCER);
+                if (!ok) break;
+            }
+            const uint32_t full = map_to_cta(smem_u32(&bars->full[s]), 0);
+            if (rank == 0) mbar_arrive_expect_tx(smem_u32(&bars->full[s]), 2 * STAGE);
+#pragma unroll
+            for (int b = 0; b < 3; ++b, ++tile)
+                tma_load_3d_pair(smem_u32(smem + (size_t)s * STAGE + (size_t)b * TS_BOX), &tmap, full, (int32_t)(tile & 63u) * 128,
+                                 (int32_t)((tile >> 6) & 3u) * 128, 0);
+            ++issued;
+        }
+        if (!ok && rank == 0)       // a failed wait: let the stages armed last land before the CTA leaves (bounded)
+            for (uint32_t j = (issued > (uint32_t)MC_STAGES ? issued - MC_STAGES : 0u); j < issued; ++j)
+                if (!mbar_wait_quiet(smem_u32(&bars->full[j % MC_STAGES]), (j / MC_STAGES) & 1u)) break;
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, 512);
+    }
+}
+
 // 1-bit scoring instruction mix: acc += popc(a ^ b), 32 independent accumulators per thread.
 __global__ void __launch_bounds__(256)
 popc_peak_kernel(int iters, uint32_t seed, uint32_t* out)
@@ -320,7 +407,7 @@ extern "C" qless_status qless_microbench(int32_t what, int32_t iters, float* ms_
             QLESS_REQUIRE(scratch != nullptr && scratch_bytes >= need, QLESS_ERR_WORKSPACE, "scratch of %zu bytes required", need);
             popc_peak_kernel<<<sms * 8, 256, 0, st>>>(iters, 12345u, reinterpret_cast<uint32_t*>(scratch));
             ops = (double)sms * 8 * 256 * iters * 32.0;           // word operations: one XOR + POPC + IADD each
-        } else if (what == 9 || what == 10 || what == 11) {
+        } else if (what == 9 || what == 10 || what == 11 || what == 12) {
             const size_t need = (size_t)512 * 8192;
             if (scratch == nullptr || scratch_bytes < need || (reinterpret_cast<uintptr_t>(scratch) % 16) != 0) {
                 cudaEventDestroy(e0); cudaEventDestroy(e1);
@@ -334,6 +421,11 @@ extern "C" qless_status qless_microbench(int32_t what, int32_t iters, float* ms_
                 err = cudaFuncSetAttribute(tma_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ts_smem);
                 if (err == cudaSuccess) tma_stream_kernel<<<sms, 128, ts_smem, st>>>(tm, iters, flag);
                 ops = (double)sms * iters * 3.0 * TS_BOX;             // bytes moved from L2 into shared memory
+            } else if (what == 12) {
+                const size_t mc_smem = 1024 + (size_t)MC_STAGES * 3 * TS_BOX + sizeof(McBars);
+                err = cudaFuncSetAttribute(mma_stream_consume_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mc_smem);
+                if (err == cudaSuccess) mma_stream_consume_kernel<<<sms / 2 * 2, 128, mc_smem, st>>>(tm, iters, flag);
+                ops = (double)(sms / 2) * iters * 4.0 * 2.0 * 256 * 448 * 32;
             } else {
                 const size_t mx_smem = 1024 + 128 * 128 + 32 * 1024 + (size_t)MX_STAGES * 3 * TS_BOX + sizeof(MxBars);
                 err = cudaFuncSetAttribute(mma_tma_mix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mx_smem);

@@ -41,7 +41,7 @@ constexpr int NTHREADS = 448;
 constexpr uint32_t IDESC = make_idesc(/*D=F32*/ 1, /*A=BF16*/ 1, /*B=BF16*/ 1, 2 * BM, BN);
 
 struct __align__(8) Barriers {
-    uint64_t b_full[SB], b_empty[SB], a_full[SA], a_empty[SA], d_full, d_empty;
+    uint64_t b_full[SB], b_empty[SB], a_full[SA], a_empty[SA], d_full, d_empty, drain;
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -74,6 +74,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
         for (int s = 0; s < SA; ++s) { mbar_init(smem_u32(&bars->a_full[s]), 8); mbar_init(smem_u32(&bars->a_empty[s]), 1); }
         mbar_init(smem_u32(&bars->d_full), 1);
         mbar_init(smem_u32(&bars->d_empty), 8);
+        mbar_init(smem_u32(&bars->drain), 1);
         bars->abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmap_gamma);
@@ -116,11 +117,16 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 }
             }
             if (!ok) {
-                // leave no copy in flight behind us: give every armed stage a bounded chance to land
-                for (int s = 0; s < SB; ++s)
-                    for (uint32_t t = 0; t < (1u << 16); ++t)
-                        if (mbar_try_wait(smem_u32(&bars->b_full[s]), 0) || mbar_try_wait(smem_u32(&bars->b_full[s]), 1)) break;
-                for (volatile int spin = 0; spin < (1 << 16); ++spin) { }    // the peer's barrier sees our copies: give them time to land
+                // Leave no copy in flight behind us. Stages 0 .. it-1 have been armed; all but the last SB of them were
+                // consumed before their slot was armed again. Every copy of the pair completes on the leader's barrier,
+                // so the leader waits (bounded) for the phases of those last stages; the peer cannot see that barrier
+                // and idles instead, and leaves only after the leader does (the cluster barrier at the end).
+                if (rank == 0) {
+                    for (uint32_t j = (it > (uint32_t)SB ? it - SB : 0u); j < it; ++j)
+                        if (!mbar_wait_quiet(smem_u32(&bars->b_full[j % SB]), (j / SB) & 1u)) break;
+                } else {
+                    for (uint32_t t = 0; t < (1u << 14); ++t) __nanosleep(64);
+                }
             }
         }
     } else if (warp == 1) {
@@ -156,6 +162,11 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 }
                 if (ok) mma_commit_pair(smem_u32(&bars->d_full));
             }
+            // Whatever ended the loop, every MMA issued above completes before tensor memory is freed: one more commit
+            // on a barrier of its own and a bounded wait for it (after the last item this is the wait for that item's
+            // MMAs, which the drain warps need anyway; after a failed wait it covers MMAs that no commit had followed).
+            mma_commit_pair(smem_u32(&bars->drain));
+            mbar_wait_quiet(smem_u32(&bars->drain), 0u);
         }
     } else if (warp < 6 || warp >= 10) {
         // ------------------------------- sign generators -------------------------------

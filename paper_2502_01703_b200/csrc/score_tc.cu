@@ -63,7 +63,7 @@ struct ScoreTcParams {
 
 struct __align__(8) ScoreBars {
     uint64_t full[MAX_STAGES], empty[MAX_STAGES];
-    uint64_t p_full[MAX_STAGES], p_empty[MAX_STAGES], d_full, d_empty;
+    uint64_t p_full[MAX_STAGES], p_empty[MAX_STAGES], d_full, d_empty, drain;
     uint32_t tmem_base, abort_flag;
     int32_t task_off[65];
     __align__(16) float mv[512];
@@ -133,6 +133,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
         }
         mbar_init(smem_u32(&bars->d_full), 1);
         mbar_init(smem_u32(&bars->d_empty), 8 * p.epi_groups);     // one arrival per epilogue warp of both CTAs
+        mbar_init(smem_u32(&bars->drain), 1);
         bars->abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmap_train); prefetch_tmap(&tmap_val1); prefetch_tmap(&tmap_val2);
@@ -200,6 +201,22 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                                 tma_load_3d_pair(smem_u32(st + A_SMEM + bh1), &tmap_val2, full, kb * KB, vt * p.vpad + p.n1 + (int)rank * (p.n2 / 2), i);
                         }
             }
+            if (!ok) {
+                // Leave no copy in flight behind us. Packed loads 0 .. pq-1 have been issued into this CTA's own ring
+                // (barriers of its own: wait, bounded, for the phases of the last nP of them). Operand stages 0 .. it-1
+                // have been armed; their copies complete on the leader's barriers, whose phases also need the unpack
+                // warps' arrivals at the sub-byte widths and may therefore never close: the leader gives them a bounded
+                // wait, the peer idles, and neither leaves before the other (the cluster barrier at the end).
+                if (!DIRECT)
+                    for (int64_t j = (pq > p.nP ? pq - p.nP : 0); j < pq; ++j)
+                        if (!mbar_wait_quiet(smem_u32(&bars->p_full[j % p.nP]), (uint32_t)(j / p.nP) & 1u)) break;
+                if (rank == 0) {
+                    for (uint32_t j = (it > (uint32_t)p.nS ? it - (uint32_t)p.nS : 0u); j < it; ++j)
+                        if (!mbar_wait_quiet(smem_u32(&bars->full[j % (uint32_t)p.nS]), (j / (uint32_t)p.nS) & 1u, 1u << 14)) break;
+                } else {
+                    for (uint32_t t = 0; t < (1u << 14); ++t) __nanosleep(64);
+                }
+            }
         }
     } else if (warp == 1) {
         // ------------------------------- MMA issuer (leader CTA) -------------------------------
@@ -238,6 +255,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         }
                         if (ok) mma_commit_pair(smem_u32(&bars->d_full));
                     }
+            // Whatever ended the loops, every MMA issued above completes before tensor memory is freed: one more commit
+            // on a barrier of its own and a bounded wait for it (after a failed wait this covers MMAs that no commit had
+            // followed; otherwise it is the wait for the last accumulator, which the epilogue needs anyway).
+            mma_commit_pair(smem_u32(&bars->drain));
+            mbar_wait_quiet(smem_u32(&bars->drain), 0u);
         }
     } else if (!DIRECT && (warp < 6 || warp >= 10)) {
         // ------------------------------- unpack warps (4- and 2-bit train codes) -------------------------------

@@ -62,14 +62,25 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
 // Bounded wait. Returns false if the wait gave up or another role already aborted; the first thread to
 // give up records `code` in the device timeout word and raises the CTA-wide abort flag.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          unsigned int* timeout_word, uint32_t code)
+                                          unsigned int* timeout_word, uint32_t code, uint32_t limit = kWaitLimit)
 {
-    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 255u && *abort_flag) return false;
     }
     *abort_flag = 1u;
     atomicOr(timeout_word, code);
+    return false;
+}
+
+// Bounded wait of the abort path: a role that is leaving after a failed wait uses it to let work it has already
+// started (tensor-core instructions issued, copies armed) finish before tensor memory is freed and the CTA exits.
+// It records nothing: the timeout word already says which wait gave up.
+constexpr uint32_t kDrainLimit = 1u << 18;
+__device__ __forceinline__ bool mbar_wait_quiet(uint32_t bar, uint32_t parity, uint32_t limit = kDrainLimit)
+{
+    for (uint32_t it = 0; it < limit; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
 

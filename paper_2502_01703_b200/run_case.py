@@ -32,11 +32,11 @@ def main():
     a = ap.parse_args()
     dev = "cuda"
     if a.stage == "project":
-        B.qless_set_projection_matrix(B.GAUSSIAN if a.matrix == "gaussian" else B.RADEMACHER)
+        matrix = B.GAUSSIAN if a.matrix == "gaussian" else B.RADEMACHER
         g = W.student_t_gradients(a.n, a.P, seed=1, device=dev, dtype=torch.bfloat16)
         m, v = (None, None) if a.no_adam else W.adam_moments(a.P, seed=2, device=dev)
         ws = torch.empty(B.qless_project_quantize_workspace(a.n, a.P, a.d, a.bits), dtype=torch.uint8, device=dev)
-        fn = lambda: B.qless_project_quantize(g, a.d, 7, a.bits, m, v, workspace=ws)
+        fn = lambda: B.qless_project_quantize(g, a.d, 7, a.bits, m, v, workspace=ws, matrix=matrix)
     elif a.stage == "quantize":
         x = torch.randn((a.n, a.d), device=dev)
         fn = lambda: B.qless_quantize(x, a.bits)

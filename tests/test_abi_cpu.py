@@ -123,9 +123,21 @@ def test_bad_arguments_return_statuses_before_any_launch(L):
     for hook, bad in ((L.qless_set_projection_path, 2), (L.qless_set_score_path, -1), (L.qless_set_select_path, 3)):
         assert hook(bad) == B.ERR_INVALID_ARG
         assert hook(0) == B.QLESS_OK
-    # the matrix switch and the Gaussian entry hook
-    assert L.qless_set_projection_matrix(2) == B.ERR_INVALID_ARG and L.qless_set_projection_matrix(-1) == B.ERR_INVALID_ARG
-    assert L.qless_set_projection_matrix(B.GAUSSIAN) == B.QLESS_OK and L.qless_set_projection_matrix(B.RADEMACHER) == B.QLESS_OK
+    # the matrix travels with the call: only the two documented kinds, reserved fields zero; checked before anything else
+    def pq_ex(cfg, host=False):
+        fn = L.qless_project_quantize_host_ex if host else L.qless_project_quantize_ex
+        tail = (fake, fake, null, null, 0, null) if host else (fake, fake, null, null, null, 0, null)
+        return fn(fake, B.F32, 2, 1024, null, null, None, 1024, 512, 1, C.byref(cfg) if cfg is not None else None, 8, *tail)
+    zero3 = (C.c_int32 * 3)(0, 0, 0)
+    for host in (False, True):
+        assert pq_ex(B.ProjectionCfg(2, zero3), host) == B.ERR_INVALID_ARG and b"matrix" in L.qless_last_error()
+        assert pq_ex(B.ProjectionCfg(-1, zero3), host) == B.ERR_INVALID_ARG
+        assert pq_ex(B.ProjectionCfg(B.GAUSSIAN, (C.c_int32 * 3)(0, 1, 0)), host) == B.ERR_INVALID_ARG
+        assert pq_ex(B.ProjectionCfg(B.GAUSSIAN, zero3), host) == B.ERR_WORKSPACE        # valid: stops at the missing workspace
+        assert pq_ex(None, host) == B.ERR_WORKSPACE
+    assert not hasattr(L, "qless_set_projection_matrix")     # no process-wide matrix state
+    # the bounded-wait self-test takes a poll limit in a documented range
+    assert L.qless_selftest_timeout(10, null) == B.ERR_INVALID_ARG and L.qless_selftest_timeout(1 << 20, null) == B.ERR_INVALID_ARG
     assert L.qless_gaussian_entries(1, 0, 2, 2, 8, fake, null) == B.ERR_INVALID_ARG          # j0 not a multiple of 4
     assert L.qless_gaussian_entries(1, -1, 2, 0, 8, fake, null) == B.ERR_INVALID_ARG
     assert L.qless_gaussian_entries(1, 0, 2, 1 << 39, 8, fake, null) == B.ERR_UNSUPPORTED

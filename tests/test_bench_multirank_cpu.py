@@ -50,3 +50,30 @@ def test_reference_arm_is_silent_on_other_ranks():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
                           "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_roofline_fractions_against_denominators_the_kernel_cannot_beat():
+    # figures of the kind a run produces: 1560 TFLOP/s achieved at a sampled SM clock of 1627 MHz (maximum 1965)
+    import bench
+    peaks = dict(hbm_gbs=6448.4, bf16_burst=1654.2, bf16_sustained=1380.5, source="measured")
+    r = bench.roofline_entry(1560.3, peaks, dict(sm_mhz=1627.0, sm_max_mhz=1965.0), sm_count=148)
+    assert r["peak"] == 1380.5 and abs(r["frac"] - 1560.3 / 1380.5) < 1e-12         # the library GEMM a kernel may beat
+    hw_sampled = 148 * 8192 * 1627.0e6 / 1e12
+    hw_max = 148 * 8192 * 1965.0e6 / 1e12
+    assert abs(r["hw_peak_at_sampled_clock"] - hw_sampled) < 1e-9 and abs(r["hw_peak_at_max_clock"] - hw_max) < 1e-9
+    assert abs(r["frac_of_hw_peak_at_sampled_clock"] - 1560.3 / hw_sampled) < 1e-12
+    assert r["frac_of_hw_peak_at_max_clock"] < r["frac_of_hw_peak_at_sampled_clock"] <= 1.0
+    # the unit-count peak lies above every measured figure it is compared with: the library GEMMs and the nominal 2.25 PFLOP/s
+    assert hw_max > 2250.0 > peaks["bf16_burst"] > peaks["bf16_sustained"]
+    # without clock samples only the maximum-clock fraction is given; without a measurement, none
+    r = bench.roofline_entry(1560.3, peaks, dict(sm_mhz=None, sm_max_mhz=None))
+    assert "frac_of_hw_peak_at_sampled_clock" not in r and r["frac_of_hw_peak_at_max_clock"] < 1.0
+    assert bench.roofline_entry(None, peaks, {})["frac"] is None
+
+
+def test_config_object_is_the_same_for_both_arms():
+    import bench
+    from paper_2502_01703_b200 import workloads as W
+    c = bench.bench_config(W.CONFIGS[bench.WORKLOAD])
+    assert c["workload"] == "c2_project_quantize" and c["P"] == 1 << 23 and c["d"] == 8192 and c["bits"] == 4
+    assert "model" not in c

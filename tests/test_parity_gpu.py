@@ -22,6 +22,34 @@ def _np(t):
     return t.detach().cpu().numpy()
 
 
+def _audit_codes_against_oracle_quantiser(proj, codes, scales, sumsq, bits, max_rows=2):
+    """Stage 2 of the GPU path against the oracle's stage 2 on the SAME fp32 projection (the GPU's own). Scales agree
+    to the last bits of the norm (reduced in another order, both in fp64). A row's codes may differ from the oracle's
+    only through that last bit: every differing code is audited, it must be one level away and alpha * yhat / S must
+    lie within 1e-5 of the rounding boundary between the two levels. At 1 bit (a sign) nothing may differ. Rows
+    without a differing code have the oracle's code norm. At most `max_rows` rows may need the audit at all."""
+    d = proj.shape[1]
+    wc, ws, wss = oracle.quantize_rows(proj, bits, normalize=True)
+    assert np.allclose(scales, ws, rtol=3e-7, atol=0)
+    bad_rows = np.where((codes != wc).any(axis=1))[0]
+    assert len(bad_rows) <= max_rows, f"{len(bad_rows)} rows differ from the oracle's codes"
+    alpha = 2 ** (bits - 1) - 1 if bits > 1 else 1
+    for r in bad_rows:
+        assert bits > 1, f"row {r}: sign codes differ"
+        qa = oracle.unpack(codes[r], d, bits).astype(np.int32)
+        qb = oracle.unpack(wc[r], d, bits).astype(np.int32)
+        diff = np.where(qa != qb)[0]
+        assert np.abs(qa - qb).max() == 1, f"row {r}: a code differs by more than one level"
+        yh = oracle.normalize(proj[r])[0].astype(np.float64)
+        pos = alpha * yh[diff] / float(ws[r])
+        boundary = (qa[diff] + qb[diff]) / 2.0                  # the half-integer between the two codes
+        assert np.all(np.abs(pos - boundary) < 1e-5), f"row {r}: a differing code is not at a rounding boundary"
+    if sumsq is not None:
+        ok = np.setdiff1d(np.arange(proj.shape[0]), bad_rows)
+        assert np.array_equal(sumsq[ok], wss[ok])
+    return len(bad_rows)
+
+
 # ----------------------------------------------------------------------------------------------
 # Projection-matrix entries (bit-exact)
 # ----------------------------------------------------------------------------------------------
@@ -203,11 +231,9 @@ def test_projection_matches_oracle(n, P, d, dtype, use_adam):
     want = oracle.project(gamma, d, seed)
     rel_l2, rel_max = _proj_err(_np(out["proj"]), want)
     assert rel_l2 <= PROJ_TOL and rel_max <= PROJ_TOL, (rel_l2, rel_max)
-    # downstream of the GPU's own projection the integer stages are exact: oracle quantiser on proj_out
-    wc, ws, wss = oracle.quantize_rows(_np(out["proj"]), 8, normalize=True)
-    same = (_np(out["codes"]) == wc).all(axis=1)
-    assert same.sum() >= n - 1          # a row may sit on a rounding tie through the norm's last bit
-    assert np.allclose(_np(out["scales"]), ws, rtol=3e-7)
+    # downstream of the GPU's own projection the integer stages are exact: oracle quantiser on proj_out (a row
+    # may sit on a rounding tie through the norm's last bit: audited code by code)
+    _audit_codes_against_oracle_quantiser(_np(out["proj"]), _np(out["codes"]), _np(out["scales"]), _np(out["sumsq"]), 8, max_rows=1)
 
 
 def test_projection_of_basis_vectors_is_exact():
@@ -239,12 +265,10 @@ def test_projection_is_deterministic_and_handles_empty_batch():
 # ----------------------------------------------------------------------------------------------
 
 @pytest.fixture
-def gaussian_matrix():
-    B.qless_set_projection_matrix(B.GAUSSIAN)
+def restore_projection_path():
     try:
         yield
     finally:
-        B.qless_set_projection_matrix(B.RADEMACHER)
         B.qless_set_projection_path(0)
 
 
@@ -272,34 +296,32 @@ def test_gaussian_entries_match_oracle(seed, r0, nr, j0, nj):
     (5, 2048 + 128, 512, torch.bfloat16, False),
     (64, 1 << 16, 256, torch.bfloat16, True),
 ])
-def test_gaussian_projection_matches_oracle(gaussian_matrix, n, P, d, dtype, use_adam):
+def test_gaussian_projection_matches_oracle(restore_projection_path, n, P, d, dtype, use_adam):
     seed = 0xBADC0DE
     g = W.student_t_gradients(n, P, seed=44, device=DEV, dtype=dtype)
     m, v = W.adam_moments(P, seed=45, device=DEV)
-    out = B.qless_project_quantize(g, d, seed, 4, m if use_adam else None, v if use_adam else None, want_proj=True)
+    out = B.qless_project_quantize(g, d, seed, 4, m if use_adam else None, v if use_adam else None, want_proj=True, matrix=B.GAUSSIAN)
     B.qless_check()
     gamma = oracle.adam_gamma(_np(g.float()), _np(m) if use_adam else None, _np(v) if use_adam else None)
     want = oracle.project_gaussian(gamma, d, seed)
     rel_l2, rel_max = _proj_err(_np(out["proj"]), want)
     assert rel_l2 <= PROJ_TOL and rel_max <= PROJ_TOL, (rel_l2, rel_max)
     # the integer stages downstream are the same kernels: oracle quantiser on the GPU's own projection
-    wc, ws, _ = oracle.quantize_rows(_np(out["proj"]), 4, normalize=True)
-    assert (_np(out["codes"]) == wc).all(axis=1).sum() >= n - 1
-    assert np.allclose(_np(out["scales"]), ws, rtol=3e-7)
+    _audit_codes_against_oracle_quantiser(_np(out["proj"]), _np(out["codes"]), _np(out["scales"]), _np(out["sumsq"]), 4, max_rows=1)
     # the CUDA-core kernel generates the same entries: only the fp32 summation order differs
     B.qless_set_projection_path(1)
-    ref = B.qless_project_quantize(g, d, seed, 4, m if use_adam else None, v if use_adam else None, want_proj=True)
+    ref = B.qless_project_quantize(g, d, seed, 4, m if use_adam else None, v if use_adam else None, want_proj=True, matrix=B.GAUSSIAN)
     e_l2, e_max = _proj_err(_np(out["proj"]), _np(ref["proj"]))
     assert e_l2 <= 1e-5 and e_max <= 1e-5, (e_l2, e_max)
 
 
-def test_gaussian_projection_full_width_sampled(gaussian_matrix):
+def test_gaussian_projection_full_width_sampled():
     # config 5's gradient width (P = 2^22, bf16, Adam), a full 256-row batch, d = 8192: the launch configuration of
     # the large runs (64 K chunks, every CTA pair persistent); the oracle evaluates sampled rows and coordinates
     n, P, d, seed = 256, 1 << 22, 8192, 4242
     g = W.student_t_gradients(n, P, seed=46, device=DEV, dtype=torch.bfloat16)
     m, v = W.adam_moments(P, seed=47, device=DEV)
-    out = B.qless_project_quantize(g, d, seed, 2, m, v, want_proj=True)
+    out = B.qless_project_quantize(g, d, seed, 2, m, v, want_proj=True, matrix=B.GAUSSIAN)
     B.qless_check()
     rows, coords = [0, 130, 255], [0, 129, 4096, 8191]
     gamma = oracle.adam_gamma(_np(g[rows].float()), _np(m), _np(v)).astype(np.float64)
@@ -315,42 +337,42 @@ def test_gaussian_projection_full_width_sampled(gaussian_matrix):
     assert np.all(np.abs(y2 / g2 - 1) <= 5 * math.sqrt(2.0 / d))
 
 
-def test_gaussian_host_entry_matches_device_entry(gaussian_matrix):
+def test_gaussian_host_entry_matches_device_entry():
     # the host-buffer entry projects column slabs with the Philox counters offset by the slab's first column: with
     # the Gaussian matrix, too, it must give the device-buffer entry's bytes
     n, P, d, bits = 70, 1 << 18, 256, 4
     g = W.student_t_gradients(n, P, seed=63, device="cpu").to(torch.bfloat16)
     host = g.clone().pin_memory()
     m, v = W.adam_moments(P, seed=64, device=DEV)
-    dev_out = B.qless_project_quantize(g.to(DEV), d, 778, bits, adam_m=m, adam_v=v)
-    host_out = B.qless_project_quantize_host(host, d, 778, bits, adam_m=m, adam_v=v, device=DEV)
+    dev_out = B.qless_project_quantize(g.to(DEV), d, 778, bits, adam_m=m, adam_v=v, matrix=B.GAUSSIAN)
+    host_out = B.qless_project_quantize_host(host, d, 778, bits, adam_m=m, adam_v=v, device=DEV, matrix=B.GAUSSIAN)
     torch.cuda.synchronize()
     assert np.array_equal(host_out["codes"].numpy(), _np(dev_out["codes"]))
     assert np.array_equal(host_out["scales"].numpy(), _np(dev_out["scales"]))
-    # and it is not the Rademacher result
-    B.qless_set_projection_matrix(B.RADEMACHER)
+    # and it is not the Rademacher result, which the plain call and an explicit RADEMACHER both give
     rad = B.qless_project_quantize(g.to(DEV), d, 778, bits, adam_m=m, adam_v=v)
+    rad2 = B.qless_project_quantize(g.to(DEV), d, 778, bits, adam_m=m, adam_v=v, matrix=B.RADEMACHER)
+    assert torch.equal(rad["codes"], rad2["codes"])
     assert not np.array_equal(_np(rad["codes"]), _np(dev_out["codes"]))
 
 
-def test_gaussian_projection_of_basis_vectors_and_switch_back(gaussian_matrix):
+def test_gaussian_projection_of_basis_vectors():
     # e_j projects to column j of the matrix the entry hook returns, scaled by the fp32 value of 1/sqrt(d)
     P, d, seed = 1024, 256, 78
     js = [0, 1, 2, 3, 127, 128, 1023]
     g = torch.zeros((len(js), P), dtype=torch.bfloat16, device=DEV)
     for a, j in enumerate(js):
         g[a, j] = 1.0
-    proj = _np(B.qless_project_quantize(g, d, seed, 8, want_proj=True)["proj"])
+    proj = _np(B.qless_project_quantize(g, d, seed, 8, want_proj=True, matrix=B.GAUSSIAN)["proj"])
     for a, j in enumerate(js):
         col = _np(B.qless_gaussian_entries(seed, 0, d, j - j % 4, 4))[:, j % 4]
         assert np.array_equal(proj[a], col * np.float32(1.0 / np.sqrt(np.float32(d))))
-    # switching back restores the Rademacher matrix
-    B.qless_set_projection_matrix(B.RADEMACHER)
+    # the matrix is an argument, not a state: the next plain call uses the Rademacher matrix
     proj = _np(B.qless_project_quantize(g, d, seed, 8, want_proj=True)["proj"])
     col = oracle.rademacher_rows(seed, 0, d, 0, 1)[:, 0].astype(np.float32)
     assert np.array_equal(proj[0], col * np.float32(1.0 / np.sqrt(np.float32(d))))
     with pytest.raises(B.QlessError):
-        B.qless_set_projection_matrix(2)
+        B.qless_project_quantize(g, d, seed, 8, matrix=2)
 
 
 # ----------------------------------------------------------------------------------------------
@@ -399,6 +421,47 @@ def test_scores_match_oracle(bits, mode):
     # sumsq recomputed inside the library gives the same scores
     got2 = B.qless_score(tc, vc, ts, vs, eta, off, d, bits, mode=mode)
     assert torch.equal(got2, got)
+
+
+# More validation vectors than one accumulator tile holds (512 at 8 bits, 448 at the sub-byte widths): the kernel walks
+# several validation tiles per train tile, finds the task that each tile starts in and carries a task that straddles
+# two tiles in its running sum. Task boundaries are placed across 448 and 512 and off every multiple of 32.
+@pytest.mark.parametrize("bits", [8, 4, 2, 1])
+@pytest.mark.parametrize("V,off", [(600, [0, 100, 470, 600]), (1100, [0, 100, 470, 530, 1000, 1100]),
+                                   (1024, [0, 448, 512, 1024]), (449, [0, 449])])
+def test_scores_with_several_validation_tiles(bits, V, off):
+    C, N, d = 2, 300, 256
+    eta = [1.0, 0.5]
+    tc, vc, ts, vs, tss, vss = _make_store(bits, C, N, V, d, seed=160 + V)
+    got, got_pt = B.qless_score(tc, vc, ts, vs, eta, off, d, bits, train_sumsq=tss, val_sumsq=vss, want_per_task=True)
+    B.qless_check()
+    want, want_pt = oracle.score(_np(tc), _np(vc), _np(ts), _np(vs), eta, off, d, bits, want_per_task=True)
+    assert np.abs(_np(got) - want).max() <= SCORE_TOL * sum(eta)
+    assert np.abs(_np(got_pt) - want_pt).max() <= SCORE_TOL * sum(eta)
+    # the integer numerators of every tile, bit for bit
+    dots = _np(B.qless_score_dots(tc[0], vc[0], d, bits))
+    assert np.array_equal(dots, oracle.dots(_np(tc[0]), _np(vc[0]), d, bits))
+
+
+# More tasks than the tensor-core epilogue keeps in registers (8): the call takes the CUDA-core kernel.
+@pytest.mark.parametrize("bits", [8, 4, 2, 1])
+@pytest.mark.parametrize("T", [9, 64])
+def test_scores_with_many_tasks(bits, T):
+    C, N, V, d = 2, 200, 5 * T + 3, 256
+    eta = [1.0, 0.25]
+    sizes = [5] * (T - 1) + [8]
+    off = np.concatenate([[0], np.cumsum(sizes)]).tolist()
+    tc, vc, ts, vs, tss, vss = _make_store(bits, C, N, V, d, seed=170 + T)
+    got, got_pt = B.qless_score(tc, vc, ts, vs, eta, off, d, bits, train_sumsq=tss, val_sumsq=vss, want_per_task=True)
+    want, want_pt = oracle.score(_np(tc), _np(vc), _np(ts), _np(vs), eta, off, d, bits, want_per_task=True)
+    assert np.abs(_np(got) - want).max() <= SCORE_TOL * sum(eta)
+    assert np.abs(_np(got_pt) - want_pt).max() <= SCORE_TOL * sum(eta)
+    # T = 8 is the last count the tensor-core kernel takes: same store, the first eight tasks
+    if T == 9:
+        off8 = off[:8] + [V]
+        got8 = B.qless_score(tc, vc, ts, vs, eta, off8, d, bits)
+        want8 = oracle.score(_np(tc), _np(vc), _np(ts), _np(vs), eta, off8, d, bits)
+        assert np.abs(_np(got8) - want8).max() <= SCORE_TOL * sum(eta)
 
 
 # The CUDA-core kernels (dp4a for 8/4/2-bit codes, XOR + population count for 1-bit codes) stay in the library as
@@ -627,6 +690,32 @@ def test_topk_2pow28_properties():
 # lr [1, 0.5], 2 tasks of 32, top 5 %)
 # ----------------------------------------------------------------------------------------------
 
+def _audit_codes_of_two_pipelines(codes_gpu, codes_or, proj_or, eps, bits):
+    """Codes of the GPU pipeline against codes of the oracle's own pipeline (different fp32 / fp64 projections).
+    alpha * yhat_m / S = alpha * y_m / max|y| does not depend on the norm, and a projection error of at most eps
+    (relative to max|y|, as measured for this batch) moves it by at most 2 alpha eps (the element and the maximum each
+    move by eps max|y|). So a code may differ from the oracle's only by one level and only where the oracle's own
+    position lies within 2 alpha eps (+ 1e-6 for the fp32 steps of both quantisers) of the boundary between the two
+    levels; at 1 bit only where |y_m| <= eps max|y|. Returns the number of differing codes per row."""
+    d = proj_or.shape[1]
+    alpha = 2 ** (bits - 1) - 1 if bits > 1 else 1
+    flips = np.zeros(codes_gpu.shape[0], np.int64)
+    for r in np.where((codes_gpu != codes_or).any(axis=1))[0]:
+        qa = oracle.unpack(codes_gpu[r], d, bits).astype(np.int32)
+        qb = oracle.unpack(codes_or[r], d, bits).astype(np.int32)
+        diff = np.where(qa != qb)[0]
+        flips[r] = diff.size
+        y = proj_or[r].astype(np.float64)
+        ymax = np.abs(y).max()
+        if bits == 1:
+            assert np.all(np.abs(y[diff]) <= eps * ymax * (1 + 1e-6))
+        else:
+            assert np.abs(qa - qb).max() == 1
+            pos = alpha * y[diff] / ymax
+            assert np.all(np.abs(pos - (qa[diff] + qb[diff]) / 2.0) <= 2 * alpha * eps + 1e-6)
+    return flips
+
+
 @pytest.mark.parametrize("bits", [8, 1])
 def test_config1_end_to_end(bits):
     cfg = W.CONFIGS["c1_tiny_e2e"]
@@ -639,6 +728,7 @@ def test_config1_end_to_end(bits):
     tss = torch.empty((C, nt), dtype=torch.int32, device=DEV); vss = torch.empty((C, nv), dtype=torch.int32, device=DEV)
     o_tc = np.empty((C, nt, rb), np.uint8); o_vc = np.empty((C, nv, rb), np.uint8)
     o_ts = np.empty((C, nt), np.float32); o_vs = np.empty((C, nv), np.float32)
+    flips_t = np.zeros((C, nt), np.int64); flips_v = np.zeros((C, nv), np.int64)
     for i in range(C):
         g_tr = W.student_t_gradients(nt, P, seed=100 + i, device=DEV)
         g_va = W.student_t_gradients(nv, P, seed=200 + i, device=DEV)
@@ -648,33 +738,42 @@ def test_config1_end_to_end(bits):
         tc[i], ts[i], tss[i] = a["codes"], a["scales"], a["sumsq"]
         vc[i], vs[i], vss[i] = b["codes"], b["scales"], b["sumsq"]
         # oracle, stage by stage
-        oc, os_, _, op = oracle.project_quantize(_np(g_tr), d, seed, bits, m=_np(m), v=_np(v), want_proj=True)
-        rel_l2, rel_max = _proj_err(_np(a["proj"]), op)
-        assert rel_l2 <= PROJ_TOL and rel_max <= PROJ_TOL
-        o_tc[i], o_ts[i] = oc, os_
-        oc, os_, _, op = oracle.project_quantize(_np(g_va), d, seed, bits, want_proj=True)
-        rel_l2, rel_max = _proj_err(_np(b["proj"]), op)
-        assert rel_l2 <= PROJ_TOL and rel_max <= PROJ_TOL
-        o_vc[i], o_vs[i] = oc, os_
-        # codes: the two pipelines may differ where the fp32-accumulated projection lands on the other
-        # side of a rounding boundary; that must be rare and by one level
-        frac_diff = float((_np(a["codes"]) != o_tc[i]).mean())
-        assert frac_diff < 0.02, frac_diff
-    scores = B.qless_score(tc, vc, ts, vs, cfg["lr"], off, d, bits, train_sumsq=tss, val_sumsq=vss)
+        for out, g, mv, o_codes, o_scales, flips in ((a, g_tr, (_np(m), _np(v)), o_tc, o_ts, flips_t),
+                                                     (b, g_va, (None, None), o_vc, o_vs, flips_v)):
+            oc, os_, _, op = oracle.project_quantize(_np(g), d, seed, bits, m=mv[0], v=mv[1], want_proj=True)
+            rel_l2, rel_max = _proj_err(_np(out["proj"]), op)
+            assert rel_l2 <= PROJ_TOL and rel_max <= PROJ_TOL
+            o_codes[i], o_scales[i] = oc, os_
+            # stage 2 on the GPU's own projection: the oracle's codes up to the audited last-bit ties
+            _audit_codes_against_oracle_quantiser(_np(out["proj"]), _np(out["codes"]), _np(out["scales"]), _np(out["sumsq"]), bits)
+            # the two pipelines' codes: they differ only where the measured projection error allows it
+            flips[i] = _audit_codes_of_two_pipelines(_np(out["codes"]), oc, op, rel_max, bits)
+    eta = cfg["lr"]
+    scores = B.qless_score(tc, vc, ts, vs, eta, off, d, bits, train_sumsq=tss, val_sumsq=vss)
     # (a) same codes in, same scores out
-    want_same = oracle.score(_np(tc), _np(vc), _np(ts), _np(vs), cfg["lr"], off, d, bits)
-    assert np.abs(_np(scores) - want_same).max() <= SCORE_TOL * sum(cfg["lr"])
-    # (b) whole pipeline against the oracle's own pipeline: scores close, selections agree up to near-ties
-    want_full = oracle.score(o_tc, o_vc, o_ts, o_vs, cfg["lr"], off, d, bits)
-    assert np.abs(_np(scores) - want_full).max() <= 2e-3 * sum(cfg["lr"])
+    want_same = oracle.score(_np(tc), _np(vc), _np(ts), _np(vs), eta, off, d, bits)
+    assert np.abs(_np(scores) - want_same).max() <= SCORE_TOL * sum(eta)
     idx = _np(B.qless_select_topk(scores, cfg["frac"]))
     assert idx.size == 50
     assert np.array_equal(idx, oracle.select_topk(_np(scores), cfg["frac"]))     # bit-exact given the same scores
+    # (b) whole pipeline against the oracle's own pipeline. The bar follows from the code differences counted above:
+    # a code vector q with f codes moved by one level (by two, at 1 bit: -1 <-> +1) turns by an angle of at most
+    # asin(step sqrt(f) / ||q||), and a cosine moves by at most the sum of the angles its two vectors turn by
+    # (triangle inequality on the sphere). Summed with |eta| and with the worst validation vector of each checkpoint:
+    step = 2.0 if bits == 1 else 1.0
+    nrm_t = np.sqrt(_np(tss).astype(np.float64)); nrm_v = np.sqrt(_np(vss).astype(np.float64))
+    ang_t = np.arcsin(np.minimum(1.0, step * np.sqrt(flips_t) / np.maximum(nrm_t - step * np.sqrt(flips_t), 1.0)))
+    ang_v = np.arcsin(np.minimum(1.0, step * np.sqrt(flips_v) / np.maximum(nrm_v - step * np.sqrt(flips_v), 1.0)))
+    bound = sum(abs(eta[i]) * (ang_t[i] + ang_v[i].max()) for i in range(C)) + SCORE_TOL * sum(eta)     # [nt]
+    want_full = oracle.score(o_tc, o_vc, o_ts, o_vs, eta, off, d, bits)
+    assert np.all(np.abs(_np(scores) - want_full) <= bound), float((np.abs(_np(scores) - want_full) / bound).max())
+    assert bound.max() <= 2e-2 * sum(eta)            # the bound itself stays small: few codes differ
+    # selections agree up to near-ties: a score moves by at most bmax, hence so does the 50th largest, so an index in
+    # one set only has an oracle score within 2 bmax of the oracle's threshold
     o_idx = oracle.select_topk(want_full, cfg["frac"])
     thr = np.sort(want_full)[-50]
     for t in set(idx.tolist()) ^ set(o_idx.tolist()):
-        assert abs(want_full[t] - thr) <= 2e-3 * sum(cfg["lr"])
-    assert len(set(idx.tolist()) & set(o_idx.tolist())) >= 45
+        assert abs(want_full[t] - thr) <= 2 * bound.max()
 
 
 # ----------------------------------------------------------------------------------------------
@@ -682,27 +781,39 @@ def test_config1_end_to_end(bits):
 # ----------------------------------------------------------------------------------------------
 
 def test_projection_full_size_sampled():
-    # config 2 shape: 256 bf16 rows, P = 2^23, d = 8192, 4-bit; the oracle evaluates sampled outputs
+    # config 2 shape: 256 bf16 rows, P = 2^23, d = 8192, 4-bit, in the launch configuration the benchmark times
+    # (128 K chunks x 32 tiles of 256 coordinates = 4096 work items walked by 74 persistent CTA pairs).
     cfg = W.CONFIGS["c2_project_quantize"]
     n, P, d, bits, seed = cfg["batch_rows"], cfg["P"], cfg["d"], cfg["bits"], 31337
     g = W.student_t_gradients(n, P, seed=500, device=DEV, dtype=torch.bfloat16)
     m, v = W.adam_moments(P, seed=501, device=DEV)
     out = B.qless_project_quantize(g, d, seed, bits, m, v, want_proj=True)
     B.qless_check()
+    proj = _np(out["proj"])
+    # (1) the oracle evaluates one coordinate in each of the 64 halves (one CTA of a pair each) of the 32 coordinate
+    # tiles, at an offset that walks through the half, plus the first and last coordinates, for rows of both row halves
     rows = [0, 100, 255]
-    coords = [0, 1, 127, 128, 4095, 8191]
+    coords = sorted({128 * h + (37 * h + 5) % 128 for h in range(64)} | {0, 1, 127, 128, 8191})
     gamma = oracle.adam_gamma(_np(g[rows].float()), _np(m), _np(v))
     want = oracle.project_rows(gamma, d, seed, coords)
-    got = _np(out["proj"])[np.ix_(rows, coords)]
-    ref_scale = np.abs(_np(out["proj"])[rows]).max(axis=1, keepdims=True)
+    got = proj[np.ix_(rows, coords)]
+    ref_scale = np.abs(proj[rows]).max(axis=1, keepdims=True)
     assert (np.abs(got - want) / ref_scale).max() <= PROJ_TOL
-    # properties that hold at any size: oracle stage 2 on the GPU's projection reproduces the codes
-    wc, ws, wss = oracle.quantize_rows(_np(out["proj"]), bits, normalize=True)
-    assert ((_np(out["codes"]) == wc).all(axis=1)).sum() >= n - 2
-    assert np.allclose(_np(out["scales"]), ws, rtol=3e-7)
+    # (2) all 256 x 8192 outputs against the CUDA-core kernel of the same definition (another summation order inside
+    # a K chunk, both in fp32): a misplaced (K chunk, tile) work item would move its outputs by about 1/sqrt(128) of
+    # their size; rounding differences stay far below the bar
+    try:
+        B.qless_set_projection_path(1)
+        ref = B.qless_project_quantize(g, d, seed, bits, m, v, want_proj=True)
+    finally:
+        B.qless_set_projection_path(0)
+    rel_l2, rel_max = _proj_err(proj, _np(ref["proj"]))
+    assert rel_l2 <= PROJ_TOL / 2 and rel_max <= PROJ_TOL / 2, (rel_l2, rel_max)
+    # (3) properties that hold at any size: oracle stage 2 on the GPU's projection reproduces the codes (audited)
+    _audit_codes_against_oracle_quantiser(proj, _np(out["codes"]), _np(out["scales"]), _np(out["sumsq"]), bits)
     # JL: the projection keeps the norm of Gamma within 5 sigma
     g2 = (gamma.astype(np.float64) ** 2).sum(1)
-    y2 = (_np(out["proj"])[rows].astype(np.float64) ** 2).sum(1)
+    y2 = (proj[rows].astype(np.float64) ** 2).sum(1)
     assert np.all(np.abs(y2 / g2 - 1) <= 5 * math.sqrt(2.0 / d))
 
 
@@ -788,11 +899,7 @@ def test_config5_pipeline_full_width_reduced_rows():
                 want = oracle.project_rows(gamma, d, seed, coords)
                 ref = np.abs(proj[rows]).max(axis=1, keepdims=True)
                 assert (np.abs(proj[np.ix_(rows, coords)] - want) / ref).max() <= PROJ_TOL
-            wc, wsc, wss = oracle.quantize_rows(proj, bits, normalize=True)
-            assert (_np(out["codes"]) == wc).all(axis=1).sum() >= count - 2
-            assert np.allclose(_np(out["scales"]), wsc, rtol=3e-7)
-            same = (_np(out["codes"]) == wc).all(axis=1)
-            assert np.array_equal(_np(out["sumsq"])[same], wss[same])
+            _audit_codes_against_oracle_quantiser(proj, _np(out["codes"]), _np(out["scales"]), _np(out["sumsq"]), bits)
     B.qless_check()
     scores = B.qless_score(tc, vc, ts, vs, cfg["lr"], off, d, bits, train_sumsq=tq, val_sumsq=vq)
     r = torch.arange(0, n, 8, device=DEV)
@@ -800,6 +907,99 @@ def test_config5_pipeline_full_width_reduced_rows():
     assert np.abs(_np(scores)[::8] - want).max() <= SCORE_TOL * sum(cfg["lr"])
     idx = _np(B.qless_select_topk(scores, cfg["frac"]))
     assert np.array_equal(idx, oracle.select_topk(_np(scores), cfg["frac"]))
+
+
+def test_config5_pipeline_full_size():
+    # config 5 at its own size: 4 checkpoints x (32 768 training + 448 validation) bf16 gradients of width 2^22, Adam on
+    # the training side, d = 8192, 2-bit codes, scoring of the 32 768-row store against 448 validation vectors in 3
+    # tasks, top 5 %. Training batches of 256 rows are distinct: four generated batches per checkpoint, each used 32
+    # times with its columns rotated by another multiple of 1024 (a rotation changes every projected value). Against
+    # the oracle: the projection of sampled batches on sampled rows and coordinates, the codes of whole sampled batches
+    # from the GPU's own projection, the scores of sampled rows of the final store, the selection from the GPU's scores.
+    cfg = W.CONFIGS["c5_full_pipeline"]
+    N, V, P, d, C, bits, seed = cfg["n_train"], cfg["n_val"], cfg["P"], cfg["d"], cfg["C"], cfg["bits"], 5150
+    off = W.task_offsets(cfg["tasks"]).tolist()
+    rb = d * bits // 8
+    tc = torch.empty((C, N, rb), dtype=torch.uint8, device=DEV); vc = torch.empty((C, V, rb), dtype=torch.uint8, device=DEV)
+    ts = torch.empty((C, N), device=DEV); vs = torch.empty((C, V), device=DEV)
+    tq = torch.empty((C, N), dtype=torch.int32, device=DEV); vq = torch.empty((C, V), dtype=torch.int32, device=DEV)
+    ws = torch.empty(B.qless_project_quantize_workspace(256, P, d, bits), dtype=torch.uint8, device=DEV)
+    proj = torch.empty((256, d), device=DEV)
+    rolled = torch.empty((256, P), dtype=torch.bfloat16, device=DEV)
+    rows, coords = [0, 127, 128, 255], [0, 127, 128, 4097, 8191]
+    nb = N // 256
+    checked = {(0, 0), (0, nb - 1), (C - 1, 37), (C - 1, nb - 1)}           # (checkpoint, batch) pairs the oracle looks into
+
+    def check_batch(g, m, v, out, count):
+        p_np = _np(out["proj"])[:count]
+        gamma = oracle.adam_gamma(_np(g[rows].float()), None if m is None else _np(m), None if v is None else _np(v))
+        want = oracle.project_rows(gamma, d, seed, coords)
+        ref = np.abs(p_np[rows]).max(axis=1, keepdims=True)
+        assert (np.abs(p_np[np.ix_(rows, coords)] - want) / ref).max() <= PROJ_TOL
+        _audit_codes_against_oracle_quantiser(p_np, _np(out["codes"]), _np(out["scales"]), _np(out["sumsq"]), bits)
+
+    for i in range(C):
+        m, v = W.adam_moments(P, seed=1800 + i, device=DEV)
+        pool = [W.student_t_gradients(256, P, seed=1900 + 8 * i + j, device=DEV, dtype=torch.bfloat16) for j in range(4)]
+        for b in range(nb):
+            shift = (b // 4) * 1024
+            g = pool[b % 4]
+            if shift:
+                rolled[:, shift:] = g[:, :P - shift]; rolled[:, :shift] = g[:, P - shift:]
+                g = rolled
+            r0 = b * 256
+            look = (i, b) in checked
+            out = B.qless_project_quantize(g, d, seed, bits, m, v, workspace=ws,
+                                           out=dict(codes=tc[i, r0:r0 + 256], scales=ts[i, r0:r0 + 256], sumsq=tq[i, r0:r0 + 256],
+                                                    proj=proj if look else None))
+            if look:
+                check_batch(g, m, v, out, 256)
+        del pool
+        gv = W.student_t_gradients(V, P, seed=2000 + i, device=DEV, dtype=torch.bfloat16)
+        for r0 in range(0, V, 256):
+            r1 = min(V, r0 + 256)
+            out = B.qless_project_quantize(gv[r0:r1], d, seed, bits, workspace=ws,
+                                           out=dict(codes=vc[i, r0:r1], scales=vs[i, r0:r1], sumsq=vq[i, r0:r1], proj=proj[:r1 - r0]))
+            if i in (0, C - 1) and r0 == 0:
+                check_batch(gv[r0:r1], None, None, out, r1 - r0)
+        del gv, m, v
+    B.qless_check()
+    scores = B.qless_score(tc, vc, ts, vs, cfg["lr"], off, d, bits, train_sumsq=tq, val_sumsq=vq)
+    B.qless_check()
+    got = _np(scores)
+    sample = sorted({0, 1, 127, 128, 255, 256, 257, N // 2, N - 257, N - 256, N - 255, N - 2, N - 1} |
+                    set(np.random.default_rng(55).integers(0, N, 27).tolist()))
+    r = torch.tensor(sample, device=DEV)
+    want = oracle.score(_np(tc[:, r]), _np(vc), _np(ts[:, r]), _np(vs), cfg["lr"], off, d, bits)
+    assert np.abs(got[sample] - want).max() <= SCORE_TOL * sum(cfg["lr"])
+    assert np.isfinite(got).all() and np.abs(got).max() <= sum(cfg["lr"]) * (1 + 1e-5)
+    assert np.unique(got).size > N // 2                    # the rotated batches gave distinct rows, not 32 copies of four
+    idx = _np(B.qless_select_topk(scores, cfg["frac"]))
+    assert idx.size == 1638
+    assert np.array_equal(idx, oracle.select_topk(got, cfg["frac"]))
+
+
+# ----------------------------------------------------------------------------------------------
+# Bounded device-side waits: a wait that nothing satisfies gives up, the kernel returns, the host reads the status
+# ----------------------------------------------------------------------------------------------
+
+def test_bounded_wait_times_out_and_reports():
+    B.qless_check()                                  # start from a clear flag
+    s = torch.randn(10_000, device=DEV)
+    before = _np(B.qless_select_topk(s, 0.1))
+    B.qless_selftest_timeout(1024)                   # returns: the launch only enqueues the kernel
+    with pytest.raises(B.QlessError) as e:
+        B.qless_check()
+    assert e.value.status == B.ERR_TIMEOUT
+    assert "0x1)" in str(e.value)                    # the producer role's code alone: the second waiter left on the abort flag
+    B.qless_check()                                  # the flag was cleared by the failing check
+    # the context is intact: the library still computes, and no later check trips
+    assert np.array_equal(_np(B.qless_select_topk(s, 0.1)), before)
+    x = W.student_t_gradients(8, 1024, seed=3, device=DEV, dtype=torch.bfloat16)
+    B.qless_project_quantize(x, 256, 1, 4)
+    B.qless_check()
+    with pytest.raises(B.QlessError):
+        B.qless_selftest_timeout(10)                 # poll limit out of range: refused on the host
 
 
 # ----------------------------------------------------------------------------------------------

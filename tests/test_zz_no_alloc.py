@@ -3,8 +3,8 @@
 Some callers cannot hand the library a workspace: they run inside a process whose device memory is a
 fixed arena owned by someone else, or on a path where an allocation would synchronise the device.
 qless_select_topk_static keeps its scratch in a fixed array inside the library instead. This test calls
-it through the C ABI twice in a row (the second call sees whatever the first left in the shared
-array) and requires the same indices, bit for bit, as qless_select_topk. The file name sorts last so a
+it through the C ABI twice in a row, at sizes whose kernels do use that array (the second call sees
+whatever the first left in it), and requires the same indices, bit for bit, as qless_select_topk. The file name sorts last so a
 run that stops at the first failure has already run every other test.
 """
 import ctypes as C
@@ -29,22 +29,43 @@ def _scores(N, seed, ties):
 
 
 def test_static_select_matches_workspace_select_on_two_calls_in_a_row():
-    cases = [(270_000, 0.05, 1, False), (1_000, 0.5, 2, True)]      # large first, small second: stale
-    outs = []                                                       # per-block scratch must not leak
+    # Both sizes lie above what the one-launch cluster kernel takes (360 448 scores), so both calls run the multi-pass
+    # select, the path that keeps its histograms, selection state and per-block counts and offsets in the library's
+    # fixed array. Large first, smaller second: the second call finds the first one's 2048 block entries and full
+    # histograms in the array and must not be misled by them. The calls are enqueued back to back on one stream.
+    cases = [(B.SELECT_STATIC_MAX_N, 0.05, 1, False), (400_000, 0.3, 2, True)]
+    outs = []
     for N, frac, seed, ties in cases:
         s = _scores(N, seed, ties)
         idx = torch.full((N,), -1, dtype=torch.int64, device=DEV)   # caller-owned output
         got = B.qless_select_topk_static(s, frac, idx)
-        outs.append((s, frac, got.clone()))
+        outs.append((s, frac, got))
     torch.cuda.synchronize()
     for s, frac, got in outs:
         want = B.qless_select_topk(s, frac)
         assert got.numel() == want.numel() == int(frac * s.numel() + 1e-6)
         assert torch.equal(got, want)
-    # and once more with the first input: same answer after the array has been reused
+    # and once more with the first input: same answer after the array has been reused by a smaller problem
     s, frac, first = outs[0]
     idx = torch.empty(s.numel(), dtype=torch.int64, device=DEV)
     assert torch.equal(B.qless_select_topk_static(s, frac, idx), first)
+
+
+def test_static_select_allocates_nothing():
+    # Neither the driver's view of free device memory nor torch's allocator moves across warmed-up calls, whichever
+    # kernel path the size selects (the one-launch cluster kernel below 360 448 scores, the multi-pass select above).
+    for N in (100_000, 1_000_000):
+        s = _scores(N, 7, False)
+        idx = torch.empty(N, dtype=torch.int64, device=DEV)
+        B.qless_select_topk_static(s, 0.05, idx)                    # first call on the device: resolves the array's address
+        torch.cuda.synchronize()
+        free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+        for _ in range(3):
+            got = B.qless_select_topk_static(s, 0.05, idx)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] >= free0                # a device allocation would have lowered it
+        assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+        assert torch.equal(got, B.qless_select_topk(s, 0.05))
 
 
 def test_static_select_edge_cases_and_limit():
