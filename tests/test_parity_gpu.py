@@ -801,14 +801,14 @@ def test_projection_full_size_sampled():
     assert (np.abs(got - want) / ref_scale).max() <= PROJ_TOL
     # (2) all 256 x 8192 outputs against the CUDA-core kernel of the same definition (another summation order inside
     # a K chunk, both in fp32): a misplaced (K chunk, tile) work item would move its outputs by about 1/sqrt(128) of
-    # their size; rounding differences stay far below the bar
+    # their size; rounding differences of two fp32 summations of exact products (measured: 1.5e-6) stay below 2e-5
     try:
         B.qless_set_projection_path(1)
         ref = B.qless_project_quantize(g, d, seed, bits, m, v, want_proj=True)
     finally:
         B.qless_set_projection_path(0)
     rel_l2, rel_max = _proj_err(proj, _np(ref["proj"]))
-    assert rel_l2 <= PROJ_TOL / 2 and rel_max <= PROJ_TOL / 2, (rel_l2, rel_max)
+    assert rel_l2 <= 2e-5 and rel_max <= 2e-5, (rel_l2, rel_max)
     # (3) properties that hold at any size: oracle stage 2 on the GPU's projection reproduces the codes (audited)
     _audit_codes_against_oracle_quantiser(proj, _np(out["codes"]), _np(out["scales"]), _np(out["sumsq"]), bits)
     # JL: the projection keeps the norm of Gamma within 5 sigma
