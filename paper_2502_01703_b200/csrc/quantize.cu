@@ -141,8 +141,12 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
 #pragma unroll
                     for (int u = 0; u < 4; ++u) nib |= (S > 0.0f && e[u] < 0.0f) ? (1u << u) : 0u;
                     ss += (S > 0.0f) ? 4 : 0;
-                    const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, nib, 1);
-                    if ((lane & 1) == 0) s_out[c >> 1] = (uint8_t)(nib | (hi << 4));
+                    // eight lanes' nibbles -> one 32-bit word (three butterfly steps), stored by every eighth lane: whole
+                    // words, no byte stores of neighbouring lanes into the same bank
+                    uint32_t w = nib | (__shfl_down_sync(0xFFFFFFFFu, nib, 1) << 4);
+                    w |= __shfl_down_sync(0xFFFFFFFFu, w, 2) << 8;
+                    w |= __shfl_down_sync(0xFFFFFFFFu, w, 4) << 16;
+                    if ((lane & 7) == 0) reinterpret_cast<uint32_t*>(s_out)[c >> 3] = w;
                 } else {
                     // round-half-even to an integer by adding 1.5 * 2^23: the sum's low mantissa bits are the
                     // two's-complement code (|yhat r| <= alpha (1 + 2^-23), so no clamp is needed)

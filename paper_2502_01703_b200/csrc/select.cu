@@ -1,7 +1,9 @@
 // Stage 4: top-k by radix select on order-preserving 32-bit keys, then an index-ordered compaction.
-// Three histogram passes (11 + 11 + 10 bits) fix the k-th largest key T exactly and the number of
-// keys equal to T that are admitted (smallest indices first); the compaction writes the indices of
-// {key > T} and of the admitted ties in ascending order.
+// The k-th largest key T and the number of keys equal to T that are admitted (smallest indices first) are
+// found exactly; the compaction writes the indices of {key > T} and of the admitted ties in ascending order.
+// Three designs by size: one cluster launch that keeps the keys in shared memory (up to 360 448 scores), a
+// multi-pass radix select on the scores (up to 2^22), and above that a sampled two-sided bracket of T with one
+// streaming pass over the scores.
 #include <cmath>
 #include <mutex>
 
@@ -14,20 +16,22 @@ namespace {
 
 constexpr int SEL_T = 256;
 constexpr int SEL_EPT = 8;                       // elements per thread in the compaction
-constexpr int SEL_CHUNK = SEL_T * SEL_EPT;       // 2048 elements per block
+constexpr int SEL_CHUNK = SEL_T * SEL_EPT;       // 2048 elements per unit of the compaction
+constexpr int SEL_MAX_GRID = 1024;               // blocks of the count and write kernels (one total per block)
 
 struct SelectState {
     uint32_t prefix;      // key bits fixed so far (right-aligned)
     uint32_t pad;
     int64_t k_rem;        // how many more to take from the current bucket
+    uint32_t ticket[4];   // blocks that have finished each histogram round (the last one scans)
 };
 
-// Workspace: [0, 3*2048*4) histograms | state | block counts (2 x int32 per block) | block offsets (2 x int64)
+// Workspace: histograms | state (256 B) | block totals | unit counts (2 x int32 per 2048-score unit)
 struct SelectWs {
     uint32_t* hist;       // [3][2048]
     SelectState* state;
-    int32_t* blk_cnt;     // [nblk][2]  (gt, eq)
-    int64_t* blk_off;     // [nblk][2]  exclusive prefix (gt, eq)
+    int64_t* blk_tot;     // [SEL_MAX_GRID][2]  totals (gt, eq) of each block's range of units
+    int32_t* blk_cnt;     // [nblk][2]  (gt, eq) per unit
 };
 
 // A kernel whose gate is closed returns at once: the launches of the bracketed path and of its
@@ -40,13 +44,86 @@ struct Gate {
 
 __host__ __device__ inline int64_t sel_nblk(int64_t N) { return (N + SEL_CHUNK - 1) / SEL_CHUNK; }
 
+// Programmatic dependent launch: a kernel launched with launch_after() may be set up on the GPU while the kernel before
+// it in the stream is still draining; its first statement, dep_wait(), returns only when that kernel has completed and
+// its writes are visible, so nothing it reads can be stale. dep_release() right after lets the launch behind start
+// its own set-up in the same way. (Both are no-ops in a kernel launched the ordinary way.)
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_after(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// The block (256 threads) that finishes a histogram round last finds the bin that holds the k_rem-th largest key,
+// counting from the top bin down: thread t owns NB / 256 consecutive bins from the top. Returns false if the
+// histogram holds fewer than k_rem keys. hist is read around L1 (other blocks' atomics filled it).
+template <int NB>
+__device__ __forceinline__ bool block_find_bin(const uint32_t* hist, int64_t k_rem, uint32_t* bin_out, int64_t* krem_out)
+{
+    constexpr int PER = NB / SEL_T;
+    __shared__ int64_t s_w[SEL_T / 32];
+    __shared__ uint32_t s_bin;
+    __shared__ int64_t s_krem;
+    __shared__ int s_found;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) s_found = 0;
+    uint32_t c[PER];
+    int64_t mine = 0;
+#pragma unroll
+    for (int u = 0; u < PER; ++u) { c[u] = __ldcg(hist + (NB - 1 - (tid * PER + u))); mine += c[u]; }
+    int64_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int64_t a = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += a;
+    }
+    if (lane == 31) s_w[warp] = inc;
+    __syncthreads();
+    int64_t pre = inc - mine;
+    for (int w = 0; w < warp; ++w) pre += s_w[w];
+#pragma unroll
+    for (int u = 0; u < PER; ++u) {
+        if (pre < k_rem && k_rem <= pre + c[u]) {       // at most one (thread, u) satisfies this
+            s_bin = (uint32_t)(NB - 1 - (tid * PER + u));
+            s_krem = k_rem - pre;
+            s_found = 1;
+        }
+        pre += c[u];
+    }
+    __syncthreads();
+    *bin_out = s_bin; *krem_out = s_krem;
+    return s_found != 0;
+}
+
+// All threads of a block call this after their last global atomic of a round: true in every thread of the block
+// that arrives last (its reads then see every other block's contributions).
+__device__ __forceinline__ bool last_block_done(uint32_t* ticket)
+{
+    __shared__ int s_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    const bool last = s_last != 0;
+    if (last) __threadfence();
+    return last;
+}
+
+// One radix round on the scores (11 + 11 + 10 bits of the key); the last block to finish fixes the round's bits.
 template <int PASS>
-__global__ void __launch_bounds__(SEL_T)
-select_hist_kernel(const float* __restrict__ scores, int64_t N, const SelectState* __restrict__ state,
-                   uint32_t* __restrict__ hist, Gate gate)
+__device__ __forceinline__ void select_hist_body(const float* __restrict__ scores, int64_t N, int64_t k, SelectState* __restrict__ state,
+                                                 uint32_t* __restrict__ hist)
 {
     __shared__ uint32_t s_h[2048];
-    if (gate.closed()) return;
     for (int i = threadIdx.x; i < 2048; i += SEL_T) s_h[i] = 0;
     __syncthreads();
     const uint32_t prefix = (PASS == 0) ? 0u : state->prefix;
@@ -55,307 +132,214 @@ select_hist_kernel(const float* __restrict__ scores, int64_t N, const SelectStat
     const int64_t n4 = N >> 2;
     for (int64_t i = (int64_t)blockIdx.x * SEL_T + threadIdx.x; i < n4; i += stride) {
         const uint4 raw = __ldg(reinterpret_cast<const uint4*>(scores) + i);
-        const uint32_t k[4] = {order_key(raw.x), order_key(raw.y), order_key(raw.z), order_key(raw.w)};
+        const uint32_t kk[4] = {order_key(raw.x), order_key(raw.y), order_key(raw.z), order_key(raw.w)};
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            if (PASS == 0) atomicAdd(&s_h[k[u] >> 21], 1u);
-            else if (PASS == 1) { if ((k[u] >> 21) == prefix) atomicAdd(&s_h[(k[u] >> 10) & 0x7FFu], 1u); }
-            else { if ((k[u] >> 10) == prefix) atomicAdd(&s_h[k[u] & 0x3FFu], 1u); }
+            if (PASS == 0) atomicAdd(&s_h[kk[u] >> 21], 1u);
+            else if (PASS == 1) { if ((kk[u] >> 21) == prefix) atomicAdd(&s_h[(kk[u] >> 10) & 0x7FFu], 1u); }
+            else { if ((kk[u] >> 10) == prefix) atomicAdd(&s_h[kk[u] & 0x3FFu], 1u); }
         }
     }
     for (int64_t i = (n4 << 2) + (int64_t)blockIdx.x * SEL_T + threadIdx.x; i < N; i += stride) {
-        const uint32_t k = order_key(__float_as_uint(scores[i]));
-        if (PASS == 0) atomicAdd(&s_h[k >> 21], 1u);
-        else if (PASS == 1) { if ((k >> 21) == prefix) atomicAdd(&s_h[(k >> 10) & 0x7FFu], 1u); }
-        else { if ((k >> 10) == prefix) atomicAdd(&s_h[k & 0x3FFu], 1u); }
+        const uint32_t kk = order_key(__float_as_uint(scores[i]));
+        if (PASS == 0) atomicAdd(&s_h[kk >> 21], 1u);
+        else if (PASS == 1) { if ((kk >> 21) == prefix) atomicAdd(&s_h[(kk >> 10) & 0x7FFu], 1u); }
+        else { if ((kk >> 10) == prefix) atomicAdd(&s_h[kk & 0x3FFu], 1u); }
     }
     __syncthreads();
     for (int i = threadIdx.x; i < 2048; i += SEL_T)
         if (s_h[i]) atomicAdd(&hist[i], s_h[i]);
-}
-
-// One block of 1024 threads: find the bin that holds the k_rem-th largest key, counting from the top bin
-// down (block-wide prefix sum over the reversed histogram).
-template <int PASS>
-__global__ void __launch_bounds__(1024)
-select_scan_kernel(const uint32_t* __restrict__ hist, SelectState* __restrict__ state, int64_t k, Gate gate,
-                   uint32_t* __restrict__ short_flag)
-{
-    if (gate.closed()) return;
-    constexpr int NB = (PASS == 2) ? 1024 : 2048;
+    if (!last_block_done(&state->ticket[PASS])) return;
     constexpr int SHIFT = (PASS == 2) ? 10 : 11;
-    constexpr int PER = NB / 1024;
-    __shared__ int64_t s_w[32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t k_rem = (PASS == 0) ? k : state->k_rem;
-    const uint32_t prefix = (PASS == 0) ? 0u : state->prefix;
-    int64_t c[PER];
-    int64_t mine = 0;
-#pragma unroll
-    for (int u = 0; u < PER; ++u) { c[u] = hist[NB - 1 - (tid * PER + u)]; mine += c[u]; }
-    int64_t inc = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int64_t a = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-        if (lane >= o) inc += a;
-    }
-    if (lane == 31) s_w[warp] = inc;
-    __syncthreads();            // also orders every thread's read of *state before the single write below
-    int64_t pre = inc - mine;
-    for (int w = 0; w < warp; ++w) pre += s_w[w];
-#pragma unroll
-    for (int u = 0; u < PER; ++u) {
-        if (pre < k_rem && k_rem <= pre + c[u]) {       // exactly one (thread, u) satisfies this
-            const int b = NB - 1 - (tid * PER + u);
-            state->prefix = (prefix << SHIFT) | (uint32_t)b;
-            state->k_rem = k_rem - pre;
-        }
-        pre += c[u];
-    }
-    // fewer than k_rem keys in the whole histogram: no bin was chosen; tell the caller
-    if (short_flag != nullptr && tid == 1023 && pre < k_rem) *short_flag = 1u;
+    uint32_t bin; int64_t krem;
+    bool found;
+    if constexpr (PASS == 2) found = block_find_bin<1024>(hist, k_rem, &bin, &krem);
+    else found = block_find_bin<2048>(hist, k_rem, &bin, &krem);
+    if (found && threadIdx.x == 0) { state->prefix = (prefix << SHIFT) | bin; state->k_rem = krem; }
+}
+template <int PASS>
+__global__ void __launch_bounds__(SEL_T)
+select_hist_kernel(const float* __restrict__ scores, int64_t N, int64_t k, SelectState* __restrict__ state,
+                   uint32_t* __restrict__ hist)
+{
+    select_hist_body<PASS>(scores, N, k, state, hist);
 }
 
-__global__ void __launch_bounds__(SEL_T)
-select_count_kernel(const float* __restrict__ scores, int64_t N, int64_t nblk, const SelectState* __restrict__ state,
-                    int32_t* __restrict__ blk_cnt, Gate gate)
+// Counts of {key > T} and {key == T} per 2048-score unit. Block b owns the units [b R, (b + 1) R) and leaves their
+// totals, so that the write kernel needs no prefix-sum pass in between.
+__device__ __forceinline__ void select_count_body(const float* __restrict__ scores, int64_t N, int64_t nblk, int64_t R, int64_t G,
+                                                  const SelectState* __restrict__ state, int32_t* __restrict__ blk_cnt,
+                                                  int64_t* __restrict__ blk_tot)
 {
     __shared__ int s_gt[SEL_T / 32], s_eq[SEL_T / 32];
-    if (gate.closed()) return;
+    if ((int64_t)blockIdx.x >= G) return;            // the launch may be wider than the partition
     const uint32_t T = state->prefix;
-    for (int64_t blk = blockIdx.x; blk < nblk; blk += gridDim.x) {
-    const int64_t base = blk * SEL_CHUNK + threadIdx.x * SEL_EPT;
-    int gt = 0, eq = 0;
+    const int64_t u0 = (int64_t)blockIdx.x * R, u1 = (u0 + R < nblk) ? u0 + R : nblk;
+    int64_t tot_gt = 0, tot_eq = 0;
+    for (int64_t blk = u0; blk < u1; ++blk) {
+        const int64_t base = blk * SEL_CHUNK + threadIdx.x * SEL_EPT;
+        int gt = 0, eq = 0;
+        if (base + SEL_EPT <= N) {
+            const uint4 r0 = __ldg(reinterpret_cast<const uint4*>(scores + base)), r1 = __ldg(reinterpret_cast<const uint4*>(scores + base) + 1);
+            const uint32_t r[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
 #pragma unroll
-    for (int u = 0; u < SEL_EPT; ++u) {
-        const int64_t i = base + u;
-        if (i < N) {
-            const uint32_t k = order_key(__float_as_uint(scores[i]));
-            gt += (k > T); eq += (k == T);
-        }
-    }
+            for (int u = 0; u < SEL_EPT; ++u) { const uint32_t kk = order_key(r[u]); gt += (kk > T); eq += (kk == T); }
+        } else {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) { gt += __shfl_xor_sync(0xFFFFFFFFu, gt, o); eq += __shfl_xor_sync(0xFFFFFFFFu, eq, o); }
-    if ((threadIdx.x & 31) == 0) { s_gt[threadIdx.x >> 5] = gt; s_eq[threadIdx.x >> 5] = eq; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int a = 0, b = 0;
-        for (int w = 0; w < SEL_T / 32; ++w) { a += s_gt[w]; b += s_eq[w]; }
-        blk_cnt[2 * blk] = a; blk_cnt[2 * blk + 1] = b;
-    }
-    __syncthreads();
-    }
-}
-
-// Exclusive prefix sums over blocks: one block of 32 warps. Warp w scans its run of consecutive entries
-// in coalesced tiles of 32 (shuffle scan, running total carried along) and writes run-local prefixes;
-// after the 32 run totals are combined, a second sweep adds each run's base.
-__global__ void __launch_bounds__(1024)
-select_block_scan_kernel(const int32_t* __restrict__ blk_cnt, int64_t nblk, int64_t* __restrict__ blk_off, Gate gate)
-{
-    if (gate.closed()) return;
-    __shared__ int64_t s_w[2][32];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t per = ((nblk + 31) / 32 + 31) / 32 * 32;          // entries per warp, a multiple of 32
-    const int64_t b0 = warp * per, b1 = (b0 + per < nblk) ? b0 + per : nblk;
-    const int2* cnt2 = reinterpret_cast<const int2*>(blk_cnt);
-    longlong2* off2 = reinterpret_cast<longlong2*>(blk_off);
-    int64_t run0 = 0, run1 = 0;
-    constexpr int NB = 8;                           // tiles fetched together: one memory round trip per batch
-    for (int64_t t = b0; t < b1; t += 32 * NB) {
-        int2 c[NB];
-#pragma unroll
-        for (int q = 0; q < NB; ++q) {
-            const int64_t b = t + q * 32 + lane;
-            c[q] = (b < b1) ? cnt2[b] : make_int2(0, 0);
-        }
-#pragma unroll
-        for (int q = 0; q < NB; ++q) {
-            const int64_t b = t + q * 32 + lane;
-            int i0 = c[q].x, i1 = c[q].y;           // a tile sums to at most 32 * 4096
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int a0 = __shfl_up_sync(0xFFFFFFFFu, i0, o), a1 = __shfl_up_sync(0xFFFFFFFFu, i1, o);
-                if (lane >= o) { i0 += a0; i1 += a1; }
+            for (int u = 0; u < SEL_EPT; ++u) {
+                const int64_t i = base + u;
+                if (i < N) { const uint32_t kk = order_key(__float_as_uint(scores[i])); gt += (kk > T); eq += (kk == T); }
             }
-            if (b < b1) off2[b] = make_longlong2(run0 + (i0 - c[q].x), run1 + (i1 - c[q].y));
-            run0 += __shfl_sync(0xFFFFFFFFu, i0, 31);
-            run1 += __shfl_sync(0xFFFFFFFFu, i1, 31);
-        }
-    }
-    if (lane == 0) { s_w[0][warp] = run0; s_w[1][warp] = run1; }
-    __syncthreads();
-    if (warp == 0) return;
-    int64_t base0 = 0, base1 = 0;
-    for (int w = 0; w < warp; ++w) { base0 += s_w[0][w]; base1 += s_w[1][w]; }
-    for (int64_t t = b0; t < b1; t += 32 * NB) {
-        longlong2 v[NB];
-#pragma unroll
-        for (int q = 0; q < NB; ++q) {
-            const int64_t b = t + q * 32 + lane;
-            if (b < b1) v[q] = off2[b];             // this lane's own writes of the first sweep
         }
 #pragma unroll
-        for (int q = 0; q < NB; ++q) {
-            const int64_t b = t + q * 32 + lane;
-            if (b < b1) { v[q].x += base0; v[q].y += base1; off2[b] = v[q]; }
+        for (int o = 16; o > 0; o >>= 1) { gt += __shfl_xor_sync(0xFFFFFFFFu, gt, o); eq += __shfl_xor_sync(0xFFFFFFFFu, eq, o); }
+        if ((threadIdx.x & 31) == 0) { s_gt[threadIdx.x >> 5] = gt; s_eq[threadIdx.x >> 5] = eq; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int a = 0, b = 0;
+            for (int w = 0; w < SEL_T / 32; ++w) { a += s_gt[w]; b += s_eq[w]; }
+            blk_cnt[2 * blk] = a; blk_cnt[2 * blk + 1] = b;
+            tot_gt += a; tot_eq += b;
         }
+        __syncthreads();
     }
+    if (threadIdx.x == 0) { blk_tot[2 * blockIdx.x] = tot_gt; blk_tot[2 * blockIdx.x + 1] = tot_eq; }
+}
+__global__ void __launch_bounds__(SEL_T)
+select_count_kernel(const float* __restrict__ scores, int64_t N, int64_t nblk, int64_t R, int64_t G, const SelectState* __restrict__ state,
+                    int32_t* __restrict__ blk_cnt, int64_t* __restrict__ blk_tot)
+{
+    select_count_body(scores, N, nblk, R, G, state, blk_cnt, blk_tot);
 }
 
-// The same prefix sums for many blocks, spread over the GPU (one SM alone is bound by its own memory
-// bandwidth): tiles of 1024 entries are scanned by a block each, which also leaves the tile's total;
-// a second launch adds to every tile the sum of the totals of the tiles before it.
-__global__ void __launch_bounds__(1024)
-select_tile_scan_kernel(const int32_t* __restrict__ blk_cnt, int64_t nblk, int64_t* __restrict__ blk_off,
-                        int64_t* __restrict__ tile_tot, Gate gate)
+// Sum of the totals of the blocks before this one (every thread gets both sums).
+__device__ __forceinline__ void block_base_before(const int64_t* __restrict__ blk_tot, int64_t& base0, int64_t& base1)
 {
-    if (gate.closed()) return;
-    __shared__ int s_w[2][32];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t b = (int64_t)blockIdx.x * 1024 + threadIdx.x;
-    int2 c = make_int2(0, 0);
-    if (b < nblk) c = reinterpret_cast<const int2*>(blk_cnt)[b];
-    int i0 = c.x, i1 = c.y;                         // a tile sums to at most 1024 * 4096
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int a0 = __shfl_up_sync(0xFFFFFFFFu, i0, o), a1 = __shfl_up_sync(0xFFFFFFFFu, i1, o);
-        if (lane >= o) { i0 += a0; i1 += a1; }
-    }
-    if (lane == 31) { s_w[0][warp] = i0; s_w[1][warp] = i1; }
-    __syncthreads();
-    const int w0 = s_w[0][lane], w1 = s_w[1][lane];
-    int p0 = w0, p1 = w1;                           // every warp scans the 32 warp totals
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int a0 = __shfl_up_sync(0xFFFFFFFFu, p0, o), a1 = __shfl_up_sync(0xFFFFFFFFu, p1, o);
-        if (lane >= o) { p0 += a0; p1 += a1; }
-    }
-    const int base0 = __shfl_sync(0xFFFFFFFFu, p0 - w0, warp), base1 = __shfl_sync(0xFFFFFFFFu, p1 - w1, warp);
-    if (b < nblk) reinterpret_cast<longlong2*>(blk_off)[b] = make_longlong2((int64_t)(base0 + i0 - c.x), (int64_t)(base1 + i1 - c.y));
-    if (threadIdx.x == 1023)
-        reinterpret_cast<longlong2*>(tile_tot)[blockIdx.x] = make_longlong2((int64_t)(base0 + i0), (int64_t)(base1 + i1));
-}
-
-__global__ void __launch_bounds__(1024)
-select_tile_add_kernel(int64_t nblk, int64_t* __restrict__ blk_off, const int64_t* __restrict__ tile_tot, Gate gate)
-{
-    if (gate.closed()) return;
-    if (blockIdx.x == 0) return;
-    __shared__ int64_t s_w[2][32];
+    __shared__ int64_t s_b[2][SEL_T / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int64_t a0 = 0, a1 = 0;
-    for (int64_t t = threadIdx.x; t < (int64_t)blockIdx.x; t += 1024) {
-        const longlong2 v = reinterpret_cast<const longlong2*>(tile_tot)[t];
-        a0 += v.x; a1 += v.y;
-    }
+    for (int b = threadIdx.x; b < (int)blockIdx.x; b += SEL_T) { a0 += __ldcg(blk_tot + 2 * b); a1 += __ldcg(blk_tot + 2 * b + 1); }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) { a0 += __shfl_xor_sync(0xFFFFFFFFu, a0, o); a1 += __shfl_xor_sync(0xFFFFFFFFu, a1, o); }
-    if (lane == 0) { s_w[0][warp] = a0; s_w[1][warp] = a1; }
+    if (lane == 0) { s_b[0][warp] = a0; s_b[1][warp] = a1; }
     __syncthreads();
-    int64_t base0 = 0, base1 = 0;
+    base0 = 0; base1 = 0;
 #pragma unroll
-    for (int w = 0; w < 32; ++w) { base0 += s_w[0][w]; base1 += s_w[1][w]; }
-    const int64_t b = (int64_t)blockIdx.x * 1024 + threadIdx.x;
-    if (b < nblk) {
-        longlong2 v = reinterpret_cast<longlong2*>(blk_off)[b];
-        v.x += base0; v.y += base1;
-        reinterpret_cast<longlong2*>(blk_off)[b] = v;
-    }
-}
-
-// Prefix sums over the per-block counts: one launch for a few thousand blocks, two beyond.
-inline void launch_block_scan(const int32_t* blk_cnt, int64_t nblk, int64_t* blk_off, int64_t* tile_tot, Gate gate,
-                              cudaStream_t st)
-{
-    if (tile_tot == nullptr || nblk <= 4096) {
-        select_block_scan_kernel<<<1, 1024, 0, st>>>(blk_cnt, nblk, blk_off, gate);
-        count_launches(1);
-    } else {
-        const unsigned tiles = (unsigned)((nblk + 1023) / 1024);
-        select_tile_scan_kernel<<<tiles, 1024, 0, st>>>(blk_cnt, nblk, blk_off, tile_tot, gate);
-        select_tile_add_kernel<<<tiles, 1024, 0, st>>>(nblk, blk_off, tile_tot, gate);
-        count_launches(2);
-    }
+    for (int w = 0; w < SEL_T / 32; ++w) { base0 += s_b[0][w]; base1 += s_b[1][w]; }
+    __syncthreads();
 }
 
 __global__ void __launch_bounds__(SEL_T)
-select_write_kernel(const float* __restrict__ scores, int64_t N, int64_t nblk, const SelectState* __restrict__ state,
-                    const int64_t* __restrict__ blk_off, int64_t* __restrict__ indices, Gate gate)
+select_write_kernel(const float* __restrict__ scores, int64_t N, int64_t nblk, int64_t R, const SelectState* __restrict__ state,
+                    const int32_t* __restrict__ blk_cnt, const int64_t* __restrict__ blk_tot, int64_t* __restrict__ indices, Gate gate)
 {
+    dep_wait();
     __shared__ int s_gt[SEL_T / 32], s_eq[SEL_T / 32];
     if (gate.closed()) return;
     const uint32_t T = state->prefix;
     const int64_t k_ties = state->k_rem;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int64_t blk = blockIdx.x; blk < nblk; blk += gridDim.x) {
-    const int64_t base = blk * SEL_CHUNK + threadIdx.x * SEL_EPT;
-    uint32_t fgt = 0, feq = 0;
+    int64_t gt_run, eq_run;                   // selected-larger and tied scores before the current unit
+    block_base_before(blk_tot, gt_run, eq_run);
+    const int64_t u0 = (int64_t)blockIdx.x * R, u1 = (u0 + R < nblk) ? u0 + R : nblk;
+    for (int64_t blk = u0; blk < u1; ++blk) {
+        const int64_t base = blk * SEL_CHUNK + threadIdx.x * SEL_EPT;
+        uint32_t fgt = 0, feq = 0;
 #pragma unroll
-    for (int u = 0; u < SEL_EPT; ++u) {
-        const int64_t i = base + u;
-        if (i < N) {
-            const uint32_t k = order_key(__float_as_uint(scores[i]));
-            fgt |= (uint32_t)(k > T) << u; feq |= (uint32_t)(k == T) << u;
+        for (int u = 0; u < SEL_EPT; ++u) {
+            const int64_t i = base + u;
+            if (i < N) {
+                const uint32_t kk = order_key(__float_as_uint(scores[i]));
+                fgt |= (uint32_t)(kk > T) << u; feq |= (uint32_t)(kk == T) << u;
+            }
         }
-    }
-    const int gt = __popc(fgt), eq = __popc(feq);
-    int igt = gt, ieq = eq;
+        const int gt = __popc(fgt), eq = __popc(feq);
+        int igt = gt, ieq = eq;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int a = __shfl_up_sync(0xFFFFFFFFu, igt, o), b = __shfl_up_sync(0xFFFFFFFFu, ieq, o);
-        if (lane >= o) { igt += a; ieq += b; }
-    }
-    if (lane == 31) { s_gt[warp] = igt; s_eq[warp] = ieq; }
-    __syncthreads();
-    int64_t gt_before = blk_off[2 * blk] + igt - gt;
-    int64_t eq_before = blk_off[2 * blk + 1] + ieq - eq;
-    for (int w = 0; w < warp; ++w) { gt_before += s_gt[w]; eq_before += s_eq[w]; }
-#pragma unroll
-    for (int u = 0; u < SEL_EPT; ++u) {
-        const bool g = (fgt >> u) & 1u, e = (feq >> u) & 1u;
-        if (g || (e && eq_before < k_ties)) {
-            const int64_t pos = gt_before + (eq_before < k_ties ? eq_before : k_ties);
-            indices[pos] = base + u;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int a = __shfl_up_sync(0xFFFFFFFFu, igt, o), b = __shfl_up_sync(0xFFFFFFFFu, ieq, o);
+            if (lane >= o) { igt += a; ieq += b; }
         }
-        gt_before += g; eq_before += e;
-    }
-    __syncthreads();
+        if (lane == 31) { s_gt[warp] = igt; s_eq[warp] = ieq; }
+        __syncthreads();
+        int64_t gt_before = gt_run + igt - gt;
+        int64_t eq_before = eq_run + ieq - eq;
+        for (int w = 0; w < warp; ++w) { gt_before += s_gt[w]; eq_before += s_eq[w]; }
+#pragma unroll
+        for (int u = 0; u < SEL_EPT; ++u) {
+            const bool g = (fgt >> u) & 1u, e = (feq >> u) & 1u;
+            if (g || (e && eq_before < k_ties)) {
+                const int64_t pos = gt_before + (eq_before < k_ties ? eq_before : k_ties);
+                indices[pos] = base + u;
+            }
+            gt_before += g; eq_before += e;
+        }
+        gt_run += blk_cnt[2 * blk]; eq_run += blk_cnt[2 * blk + 1];
+        __syncthreads();
     }
 }
 
 // ------------------------------------------------------------------------------------------------
-// Large N: two reads of the scores instead of five. A stratified sample brackets the k-th largest
-// key from below (lo); one pass over the scores copies every key >= lo, in index order, into the
-// segment of its 4096-score chunk; the radix select and the ordered compaction then run on those
-// candidates alone (a few per cent of N, resident in L2). If fewer than k candidates turn up (the
-// bracket was too high: probability below 1e-8 for scores in any order, since the offset inside
-// each stratum is hashed) a flag opens the gates of the exact multi-pass path enqueued behind.
+// Large N: the scores are read once. A stratified sample (offset inside each stratum hashed) brackets the
+// k-th largest key T from both sides: lo <= T <= hi except with probability below 1e-8 per side, for scores in
+// any order. One streaming pass over the scores then classifies each key: above hi it is selected for sure,
+// inside [lo, hi] it may be (about 2 % of N for a 5 % selection), below lo it is dropped. Per 4096-score chunk
+// the pass leaves the offsets of both classes in index order (16 bits each, the class in the top bit) and, for
+// the second class, (key, offset) pairs; it also counts the first class and histograms the second. T is then
+// found by a radix select on the pairs alone (their keys span hi - lo, usually some 2^21 values: 8 + 12 (+ 12)
+// bits), and the final write walks each chunk's ordered list, looks the second class up in a bitmap built from
+// the chunk's pairs, and writes the selected indices in ascending order. If T falls outside the bracket (the
+// counts show it), a flag opens the gates of the exact multi-pass path enqueued behind.
 // ------------------------------------------------------------------------------------------------
 
 constexpr int SG_T = 256;
-constexpr int SG_CH = 4096;                     // scores per chunk = capacity of its candidate segment
-constexpr int SG_SAMPLE = 16384;                // strata (one sampled score each)
+constexpr int SG_CH = 4096;                     // scores per chunk = capacity of its lists
+constexpr int SG_SAMPLE = 1 << 18;              // strata (one sampled score each): the bracket holds about 0.5 % of N at a 5 % selection
 constexpr int64_t SG_MIN_N = (int64_t)1 << 22;  // above this the bracketed path is used
+constexpr int B1_BINS = 256, B23_BINS = 4096;   // bins of the first round (in the streaming pass) and of the later ones
 
 struct BracketState {
-    uint32_t lo_key;              // candidates are the keys >= lo_key
-    uint32_t fallback;            // 1: fewer than k candidates, the exact path must run
-    unsigned long long n_cand;
+    uint32_t lo_key, hi_key;      // second class: lo <= key <= hi; first class: key > hi
+    uint32_t b[3], sh[3];         // bits and right shift of the three radix rounds on rel = key - lo
+    uint32_t rel_prefix;          // bits of T - lo fixed so far
+    uint32_t fallback;            // 1: T lies outside the bracket, the exact path must run
+    uint32_t T, pad;              // the k-th largest key, once known
+    int64_t k_rem;                // rank still to find inside the current bucket; ties admitted, at the end
+    unsigned long long n_sure, n_maybe;
+    uint32_t s_bin[2], s_rem[2];  // sample: first-level bin of the two bracket ranks and the ranks left inside it
+    uint32_t ticket[6];           // blocks that have finished: sample levels 1, 2; streaming pass; pair rounds 2, 3
+};
+
+// What the streaming pass leaves per 4096-score chunk: a bitmap of the first class (one bit per score, 512 bytes,
+// consecutive chunks side by side), and the (key, offset) pairs of the second class in two levels. A chunk usually
+// yields some twenty pairs but may yield 4096 (constant scores): the first PP pairs of every chunk live in dense arrays
+// (the passes that read them stream through memory); whatever comes after goes to full-size segments, pair i at slot
+// i, that typical inputs never touch.
+constexpr int PG = 16, PU = 1;                  // pair lists a warp walks together, and loads in flight per lane and list
+constexpr int PP = 32 * PU;                     // dense capacity per chunk: pairs
+constexpr int BMW = SG_CH / 32;                 // bitmap words per chunk
+struct ChunkLists {
+    uint32_t* sure_bm;            // [nchunk][BMW]  bit (o & 31) of word o >> 5: score o of the chunk is above hi
+    uint32_t* key_p;              // [nchunk][PP]   keys of the pairs (any order)
+    uint32_t* key_o;              // [nchunk][SG_CH]
+    uint16_t* off_p;              // [nchunk][PP]   offsets of the pairs
+    uint16_t* off_o;              // [nchunk][SG_CH]
+    __device__ __forceinline__ uint32_t* key(int64_t c, uint32_t i) const { return i < (uint32_t)PP ? key_p + c * PP + i : key_o + c * SG_CH + i; }
+    __device__ __forceinline__ uint16_t* off(int64_t c, uint32_t i) const { return i < (uint32_t)PP ? off_p + c * PP + i : off_o + c * SG_CH + i; }
 };
 
 struct BracketWs {
-    uint32_t* hist;               // [6][2048]: 0..2 candidates, 3..5 fallback
-    SelectState* state;           // 256-byte region; BracketState sits 64 bytes in
-    BracketState* bstate;
-    int64_t* blk_off;             // sized for the fallback's 2048-score blocks
-    int32_t* blk_cnt;
-    int64_t* tile_tot;            // [ceil(nblk / 1024)][2] totals of the block-count tiles
+    uint32_t* hist;               // [B1_BINS + 2 * B23_BINS] rounds of the bracketed path, [3][2048] of the fallback, [3][4096] of the sample
+    BracketState* bstate;         // 256-byte region
+    SelectState* fstate;          // 256-byte region (fallback)
+    int64_t* blk_tot;             // [SEL_MAX_GRID][2]
+    int32_t* blk_cnt;             // [max(chunks, fallback units)][2]
     uint32_t* sample_key;         // [SG_SAMPLE]
-    uint32_t* chunk_cnt;          // [nchunk]
-    uint16_t* seg_off;            // [nchunk][SG_CH] offset of the candidate inside its chunk
-    uint32_t* seg_key;            // [nchunk][SG_CH]
+    uint32_t* chunk_cnt;          // [nchunk]  scores above hi | pairs << 16
+    ChunkLists L;
 };
+constexpr int BR_HIST_WORDS = B1_BINS + 2 * B23_BINS + 3 * 2048 + 3 * 4096;
 
 __host__ __device__ inline int64_t sg_nchunk(int64_t N) { return (N + SG_CH - 1) / SG_CH; }
 
@@ -365,65 +349,113 @@ __device__ __forceinline__ uint32_t mix32(uint32_t x)
     return x;
 }
 
-// First launch of the bracketed path, spread over the GPU: clears the histograms and the state, and
-// fetches one score per stratum (16384 scattered reads: far too many misses for one SM to keep in flight).
-__global__ void __launch_bounds__(256)
-select_init_kernel(const float* __restrict__ scores, int64_t N, uint32_t* __restrict__ clear, int clear_words,
-                   uint32_t* __restrict__ sample_key)
+// The bracket from the sample: the sampled keys of ranks r_lo = ceil(k S / N) + w and r_hi = ceil(k S / N) - w
+// (counted from the largest), w = 6 standard deviations of that rank + 8, by two radix levels of 12 bits each on the
+// 262144 sampled keys, spread over 64 blocks whose last one scans. The remaining 8 bits are rounded outwards (lo
+// down, hi up), which keeps both bounds valid and widens the bracket by at most 2^-15 of T's magnitude.
+constexpr int SS_BLOCKS = 64, SS_PER = SG_SAMPLE / (SS_BLOCKS * SEL_T);     // blocks of the two level kernels, keys per thread
+struct SampleRanks { int r_lo, r_hi; bool all_lo, no_hi; };
+__device__ __forceinline__ SampleRanks sample_ranks(int64_t N, int64_t k)
 {
-    const int j = blockIdx.x * 256 + threadIdx.x;           // grid covers SG_SAMPLE threads
-    for (int i = j; i < clear_words; i += SG_SAMPLE) clear[i] = 0u;
-    const int64_t per = N / SG_SAMPLE;                      // >= 256 for every N this path takes
-    // offset inside the stratum: hash scaled to [0, per) (per < 2^32 for every N below 2^46)
-    const int64_t pos = (int64_t)j * per + (int64_t)(((uint64_t)mix32(0x9E3779B9u * (uint32_t)j + 0x85EBCA6Bu) * (uint64_t)per) >> 32);
-    sample_key[j] = order_key(__float_as_uint(__ldg(scores + pos)));
-}
-
-// One block: the r-th largest sampled key by bisection on the key's bits, largest t with
-// #{key >= t} >= r: 32 block-wide counts over 16 keys per thread held in registers.
-// r = expected rank of the k-th largest + 6 standard deviations + 8.
-__global__ void __launch_bounds__(1024)
-select_sample_kernel(const uint32_t* __restrict__ sample_key, int64_t N, int64_t k, BracketState* __restrict__ bs,
-                     int force_short)
-{
-    constexpr int PER_T = SG_SAMPLE / 1024;
-    __shared__ int s_cnt[2][32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const double p = (double)k / (double)N;
     const double ks = ceil(p * (double)SG_SAMPLE);
-    const double rr = ks + ceil(6.0 * sqrt(ks * (1.0 - p))) + 8.0;
-    if (force_short) { if (tid == 0) bs->lo_key = 0xFF800000u; return; }      // key of +inf
-    if (rr >= (double)SG_SAMPLE) { if (tid == 0) bs->lo_key = 0u; return; }     // every score is a candidate
-    const int r = (int)rr;
-    uint32_t v[PER_T];
-#pragma unroll
-    for (int i = 0; i < PER_T; ++i) v[i] = sample_key[tid + i * 1024];
-    uint32_t t = 0;
-#pragma unroll 1
-    for (int bit = 31; bit >= 0; --bit) {
-        const uint32_t cand = t | (1u << bit);
-        int c = 0;
-#pragma unroll
-        for (int i = 0; i < PER_T; ++i) c += (v[i] >= cand);
-        c = __reduce_add_sync(0xFFFFFFFFu, c);
-        if (lane == 0) s_cnt[bit & 1][warp] = c;
-        __syncthreads();                    // the two count buffers alternate: one barrier per bit
-        const int total = __reduce_add_sync(0xFFFFFFFFu, s_cnt[bit & 1][lane]);
-        if (total >= r) t = cand;
-    }
-    if (tid == 0) bs->lo_key = t;
+    const double w = ceil(6.0 * sqrt(ks * (1.0 - p))) + 8.0;
+    SampleRanks r;
+    r.all_lo = ks + w >= (double)SG_SAMPLE;        // every score is a candidate
+    r.no_hi = ks - w < 1.0;                        // no score is selected for sure
+    r.r_lo = r.all_lo ? SG_SAMPLE : (int)(ks + w);
+    r.r_hi = r.no_hi ? 1 : (int)(ks - w);
+    return r;
 }
 
-// The second (and last) read of the scores: the candidates of each 4096-score chunk go to the chunk's
-// segment (key and offset inside the chunk, in no particular order: the final write restores index
-// order from the offsets), and their top-11-bit histogram feeds the first round of the radix select.
-// The test runs on s = key ^ 0x80000000 read as a signed integer: lo_s <= s <= s(+inf), one subtraction
-// and one unsigned compare. For a bracket above zero (POS) s is the raw bit pattern itself: negative
-// scores and NaNs fall outside the range by themselves. Otherwise s takes two more operations per score.
-// A warp owns whole chunks and walks each in eight steps of 512 scores (16 per lane, as four 16-byte
-// pieces 128 scores apart), with no block-wide barrier; a warp scan of the per-lane counts gives each
-// lane its run in the segment. Each lane fetches its own pieces with cp.async into a ring of three
-// steps, two steps ahead of the one it works on: enough bytes in flight per SM without registers.
+// Level 1 also draws the sample: one score per stratum of N / 262144 scores, at a hashed offset inside it.
+__global__ void __launch_bounds__(SEL_T)
+sample_level1_kernel(const float* __restrict__ scores, uint32_t* __restrict__ sample_key, int64_t N, int64_t k,
+                     BracketState* __restrict__ bs, uint32_t* __restrict__ hist)
+{
+    dep_wait();
+    dep_release();
+    __shared__ uint32_t s_h[4096];
+    for (int i = threadIdx.x; i < 4096; i += SEL_T) s_h[i] = 0;
+    const int64_t per = N / SG_SAMPLE;                      // >= 16 for every N this path takes
+    uint32_t key[SS_PER];
+#pragma unroll
+    for (int i = 0; i < SS_PER; ++i) {                      // grid covers SG_SAMPLE keys; all scattered reads in flight together
+        const int j = (blockIdx.x * SS_PER + i) * SEL_T + threadIdx.x;
+        // offset inside the stratum: hash scaled to [0, per) (per < 2^32 for every N below 2^50)
+        const int64_t pos = (int64_t)j * per + (int64_t)(((uint64_t)mix32(0x9E3779B9u * (uint32_t)j + 0x85EBCA6Bu) * (uint64_t)per) >> 32);
+        key[i] = order_key(__float_as_uint(__ldg(scores + pos)));
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < SS_PER; ++i) {
+        sample_key[(blockIdx.x * SS_PER + i) * SEL_T + threadIdx.x] = key[i];
+        atomicAdd(&s_h[key[i] >> 20], 1u);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 4096; i += SEL_T)
+        if (s_h[i]) atomicAdd(&hist[i], s_h[i]);
+    if (!last_block_done(&bs->ticket[0])) return;
+    const SampleRanks r = sample_ranks(N, k);
+    uint32_t bin; int64_t rem;
+    block_find_bin<4096>(hist, r.r_lo, &bin, &rem);
+    if (threadIdx.x == 0) { bs->s_bin[0] = bin; bs->s_rem[0] = (uint32_t)rem; }
+    __syncthreads();
+    block_find_bin<4096>(hist, r.r_hi, &bin, &rem);
+    if (threadIdx.x == 0) { bs->s_bin[1] = bin; bs->s_rem[1] = (uint32_t)rem; }
+}
+
+__global__ void __launch_bounds__(SEL_T)
+sample_level2_kernel(const uint32_t* __restrict__ sample_key, int64_t N, int64_t k, BracketState* __restrict__ bs,
+                     uint32_t* __restrict__ hist_lo, uint32_t* __restrict__ hist_hi, int force_short)
+{
+    dep_wait();
+    dep_release();
+    __shared__ uint32_t s_h[2][4096];
+    for (int i = threadIdx.x; i < 2 * 4096; i += SEL_T) (&s_h[0][0])[i] = 0;
+    __syncthreads();
+    const uint32_t bin_lo = bs->s_bin[0], bin_hi = bs->s_bin[1];
+    for (int i = 0; i < SS_PER; ++i) {
+        const uint32_t key = sample_key[(blockIdx.x * SS_PER + i) * SEL_T + threadIdx.x];
+        if ((key >> 20) == bin_lo) atomicAdd(&s_h[0][(key >> 8) & 0xFFFu], 1u);
+        if ((key >> 20) == bin_hi) atomicAdd(&s_h[1][(key >> 8) & 0xFFFu], 1u);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 4096; i += SEL_T) {
+        if (s_h[0][i]) atomicAdd(&hist_lo[i], s_h[0][i]);
+        if (s_h[1][i]) atomicAdd(&hist_hi[i], s_h[1][i]);
+    }
+    if (!last_block_done(&bs->ticket[1])) return;
+    const SampleRanks r = sample_ranks(N, k);
+    uint32_t sub_lo, sub_hi; int64_t rem;
+    block_find_bin<4096>(hist_lo, (int64_t)bs->s_rem[0], &sub_lo, &rem);
+    __syncthreads();
+    block_find_bin<4096>(hist_hi, (int64_t)bs->s_rem[1], &sub_hi, &rem);
+    if (threadIdx.x == 0) {
+        uint32_t lo = r.all_lo ? 0u : ((bin_lo << 20) | (sub_lo << 8));
+        uint32_t hi = r.no_hi ? 0xFFFFFFFFu : ((bin_hi << 20) | (sub_hi << 8) | 0xFFu);
+        if (force_short) lo = hi = 0xFF800000u;             // key of +inf: (almost) nothing qualifies
+        if (hi < lo) hi = lo;                               // cannot happen (r_hi <= r_lo); keeps the plan below sane
+        // plan of the radix rounds on key - lo, which lies in [0, hi - lo]: 8 bits in the streaming pass, then 12 and 12
+        const uint32_t range = hi - lo;
+        const uint32_t nbits = range ? 32u - (uint32_t)__clz((int)range) : 0u;
+        const uint32_t b1 = nbits < 8u ? nbits : 8u, rest = nbits - b1, b2 = rest < 12u ? rest : 12u, b3 = rest - b2;
+        bs->lo_key = lo; bs->hi_key = hi;
+        bs->b[0] = b1; bs->b[1] = b2; bs->b[2] = b3;
+        bs->sh[0] = nbits - b1; bs->sh[1] = nbits - b1 - b2; bs->sh[2] = 0u;
+    }
+}
+
+// The one read of the scores. A warp owns whole chunks and walks each in eight steps of 512 scores, with no
+// block-wide barrier. Each lane fetches four 16-byte pieces of a step with cp.async into a ring of three steps, two
+// steps ahead of the one the warp works on: enough bytes in flight per SM without registers. A step is then read back
+// as 16 slots of 32 consecutive scores (lane = score): two ballots per slot are the slot's words of the two class
+// bitmaps, with no scan and no divergence. The first-class words go to memory as they are (64 bytes per step); the
+// few set bits of the second-class words (2 % of the scores) are then turned into pairs, half a word per lane.
+// The class test runs on s = key ^ 0x80000000 read as a signed integer: for a bracket above zero (MODE 0) s is the raw
+// bit pattern itself, and negative scores and NaNs fall outside the range by themselves; for other brackets (MODE 1)
+// s takes two more operations per score; if every score is a candidate (MODE 2, lo = 0) the key is formed in full,
+// so that NaNs (key 0) land in the second class.
 constexpr int SG_RING = 3;
 constexpr int SG_STEP = 512;                    // scores per warp step
 constexpr int SG_STEPS = SG_CH / SG_STEP;       // 8
@@ -435,15 +467,15 @@ __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc, 
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int KEEP> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(KEEP) : "memory"); }
 
-template <bool POS>
-__device__ __forceinline__ void gather_chunks(const float* __restrict__ scores, int64_t N, uint32_t lo,
-                                              uint32_t* __restrict__ seg_key, uint16_t* __restrict__ seg_off,
-                                              uint32_t* __restrict__ chunk_cnt, uint32_t* s_h, uint32_t* __restrict__ hist0,
-                                              uint32_t* s_ring /* this warp's [SG_RING][SG_STEP] */, unsigned long long& mine)
+template <int MODE>
+__device__ __forceinline__ void gather_chunks(const float* __restrict__ scores, int64_t N, uint32_t lo, uint32_t hi, uint32_t sh1,
+                                              const ChunkLists& L, uint32_t* __restrict__ chunk_cnt, uint32_t* s_h, uint32_t* s_mc /* this warp's pair counter */,
+                                              uint32_t* s_w /* this warp's 32 ballot words */, uint32_t* s_ring /* this warp's [SG_RING][SG_STEP] */,
+                                              unsigned long long& sure_total, unsigned long long& maybe_total)
 {
     const int lane = threadIdx.x & 31;
-    const uint32_t lo_s = lo ^ 0x80000000u;
-    const uint32_t range = (lo == 0u) ? 0xFFFFFFFFu : (0x7F800000u - lo_s);     // lo == 0: NaNs are candidates too
+    const uint32_t lo_s = lo ^ 0x80000000u, hi_s = hi ^ 0x80000000u;
+    const uint32_t range = 0x7F800000u - lo_s;                     // up to the image of +inf (MODE 0, 1)
     const int64_t nchunk = sg_nchunk(N);
     const int64_t gwarp = (int64_t)blockIdx.x * (SG_T / 32) + (threadIdx.x >> 5);
     const int64_t nwarp = (int64_t)gridDim.x * (SG_T / 32);
@@ -476,272 +508,416 @@ __device__ __forceinline__ void gather_chunks(const float* __restrict__ scores, 
     fetch();
     int slot = 0;
     for (int64_t c = gwarp; c < nchunk; c += nwarp) {
-        uint32_t* kp = seg_key + c * SG_CH;
-        uint16_t* op = seg_off + c * SG_CH;
-        uint32_t run = 0;
+        if (lane == 0) *s_mc = 0u;
+        __syncwarp();
+        uint32_t* bm_out = L.sure_bm + c * BMW;
+        uint32_t n_sure = 0;                                          // lanes 0..15: set bits of the words they stored
 #pragma unroll 1
         for (int sub = 0; sub < SG_STEPS; ++sub) {
             fetch();
-            cp_async_wait<2>();                                       // this lane's pieces of the step have landed
-            const uint32_t* mine_s = s_ring + slot * SG_STEP + lane * 4;
+            cp_async_wait<2>();                                       // this lane's pieces of the step have landed ...
+            __syncwarp();                                             // ... and so have the other lanes'
+            const uint32_t* step_s = s_ring + slot * SG_STEP;
             const int64_t i0 = c * SG_CH + sub * SG_STEP;
-            uint32_t F = 0;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint4 raw = *reinterpret_cast<const uint4*>(mine_s + j * 128);
-                const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const uint32_t sv = POS ? r[u] : (r[u] ^ ((uint32_t)((int32_t)r[u] >> 31) & 0x7FFFFFFFu));
-                    if (sv - lo_s <= range) F |= 1u << (4 * j + u);
+            for (int sl = 0; sl < SG_STEP / 32; ++sl) {
+                const uint32_t r = step_s[sl * 32 + lane];
+                bool sure, cand;
+                if (MODE == 2) {
+                    cand = true; sure = order_key(r) > hi;
+                } else {
+                    const uint32_t sv = (MODE == 0) ? r : (r ^ ((uint32_t)((int32_t)r >> 31) & 0x7FFFFFFFu));
+                    cand = sv - lo_s <= range;
+                    sure = cand && (int32_t)sv > (int32_t)hi_s;
                 }
+                const uint32_t bs = __ballot_sync(0xFFFFFFFFu, sure), bc = __ballot_sync(0xFFFFFFFFu, cand);
+                if (lane == 0) { s_w[sl] = bs; s_w[16 + sl] = bc; }   // the slot's words of the two bitmaps
             }
+            __syncwarp();
+            uint32_t w_sure = 0, w_may = 0;                           // lane s < 16: the two bitmap words of slot s
+            if (lane < SG_STEP / 32) { w_sure = s_w[lane]; w_may = s_w[16 + lane] & ~w_sure; }
             if (N - i0 < SG_STEP) {                                   // ragged end: drop what lies beyond N
-                uint32_t valid = 0;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int64_t left = N - (i0 + lane * 4 + j * 128);
-                    valid |= (left >= 4 ? 0xFu : (left > 0 ? (1u << (int)left) - 1u : 0u)) << (4 * j);
-                }
-                F &= valid;
+                const int64_t left = N - (i0 + lane * 32);            // scores of slot `lane` that exist
+                const uint32_t valid = left >= 32 ? 0xFFFFFFFFu : (left > 0 ? (1u << (int)left) - 1u : 0u);
+                w_sure &= valid; w_may &= valid;
             }
-            const uint32_t cnt = (uint32_t)__popc(F);
-            uint32_t inc = cnt;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t a = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-                if (lane >= o) inc += a;
+            if (lane < SG_STEP / 32) { bm_out[sub * (SG_STEP / 32) + lane] = w_sure; n_sure += (uint32_t)__popc(w_sure); }
+            // second class: lane L takes half L & 1 of word L >> 1
+            uint32_t half = (__shfl_sync(0xFFFFFFFFu, w_may, lane >> 1) >> ((lane & 1) * 16)) & 0xFFFFu;
+            while (half) {
+                const int b = __ffs((int)half) - 1;
+                half &= half - 1u;
+                const uint32_t idx = (uint32_t)(lane * 16 + b);       // score of the step
+                const uint32_t r = step_s[idx];
+                const uint32_t key = (MODE == 0) ? (r | 0x80000000u) : order_key(r);
+                const uint32_t slot_m = atomicAdd(s_mc, 1u);          // pairs: any order
+                *L.key(c, slot_m) = key;
+                *L.off(c, slot_m) = (uint16_t)(sub * SG_STEP + idx);
+                atomicAdd(&s_h[(key - lo) >> sh1], 1u);
             }
-            const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31);
-            uint32_t pos = run + inc - cnt;
-            const uint32_t obase = (uint32_t)(sub * SG_STEP + lane * 4);
-            while (F) {
-                const int b = __ffs((int)F) - 1;
-                F &= F - 1u;
-                const uint32_t e = (uint32_t)((b >> 2) * 128 + (b & 3));
-                const uint32_t r = mine_s[e];
-                // the key; a NaN (only reachable with lo == 0) has key 0
-                const uint32_t key = POS ? (r | 0x80000000u) : order_key(r);
-                kp[pos] = key;
-                op[pos] = (uint16_t)(obase + e);
-                if (POS || key >= 0x80000000u) atomicAdd(&s_h[(key >> 21) - 1024u], 1u);
-                else atomicAdd(&hist0[key >> 21], 1u);          // negative scores and NaNs: rare as candidates
-                ++pos;
-            }
-            run += tot;
+            __syncwarp();                                             // every lane is done with the step before its slot is refilled
             slot = (slot == SG_RING - 1) ? 0 : slot + 1;
         }
-        if (lane == 0) { chunk_cnt[c] = run; mine += run; }
+        n_sure = __reduce_add_sync(0xFFFFFFFFu, n_sure);
+        if (lane == 0) {
+            const uint32_t m = *s_mc;
+            chunk_cnt[c] = n_sure | (m << 16);
+            sure_total += n_sure; maybe_total += m;
+        }
+        __syncwarp();
     }
     cp_async_wait<0>();
 }
 
 __global__ void __launch_bounds__(SG_T, 4)
-select_gather_kernel(const float* __restrict__ scores, int64_t N, BracketState* __restrict__ bs,
-                     uint32_t* __restrict__ seg_key, uint16_t* __restrict__ seg_off,
-                     uint32_t* __restrict__ chunk_cnt, uint32_t* __restrict__ hist0)
+select_gather_kernel(const float* __restrict__ scores, int64_t N, int64_t k, BracketState* __restrict__ bs,
+                     const ChunkLists L, uint32_t* __restrict__ chunk_cnt, uint32_t* __restrict__ hist1)
 {
+    dep_wait();
+    dep_release();
     extern __shared__ __align__(16) uint8_t s_dyn[];      // per warp: ring of SG_RING steps of raw scores
-    __shared__ uint32_t s_h[1024];           // bins 1024..2047: keys of scores with the sign bit clear
+    __shared__ uint32_t s_h[B1_BINS];
+    __shared__ uint32_t s_mc[SG_T / 32];
+    __shared__ uint32_t s_bw[SG_T / 32][32];
     const int tid = threadIdx.x;
-    for (int i = tid; i < 1024; i += SG_T) s_h[i] = 0;
+    for (int i = tid; i < B1_BINS; i += SG_T) s_h[i] = 0;
     __syncthreads();
-    const uint32_t lo = bs->lo_key;
-    unsigned long long mine = 0;
+    const uint32_t lo = bs->lo_key, hi = bs->hi_key, sh1 = bs->sh[0];
+    unsigned long long sure_total = 0, maybe_total = 0;
     uint32_t* s_ring = reinterpret_cast<uint32_t*>(s_dyn) + (tid >> 5) * (SG_RING * SG_STEP);
-    if (lo > 0x80000000u) gather_chunks<true>(scores, N, lo, seg_key, seg_off, chunk_cnt, s_h, hist0, s_ring, mine);
-    else gather_chunks<false>(scores, N, lo, seg_key, seg_off, chunk_cnt, s_h, hist0, s_ring, mine);
+    if (lo > 0x80000000u) gather_chunks<0>(scores, N, lo, hi, sh1, L, chunk_cnt, s_h, &s_mc[tid >> 5], s_bw[tid >> 5], s_ring, sure_total, maybe_total);
+    else if (lo > 0u) gather_chunks<1>(scores, N, lo, hi, sh1, L, chunk_cnt, s_h, &s_mc[tid >> 5], s_bw[tid >> 5], s_ring, sure_total, maybe_total);
+    else gather_chunks<2>(scores, N, lo, hi, sh1, L, chunk_cnt, s_h, &s_mc[tid >> 5], s_bw[tid >> 5], s_ring, sure_total, maybe_total);
     __syncthreads();
-    for (int i = tid; i < 1024; i += SG_T)
-        if (s_h[i]) atomicAdd(&hist0[1024 + i], s_h[i]);
-    if ((tid & 31) == 0 && mine) atomicAdd(&bs->n_cand, mine);
+    for (int i = tid; i < B1_BINS; i += SG_T)
+        if (s_h[i]) atomicAdd(&hist1[i], s_h[i]);
+    if ((tid & 31) == 0) {
+        if (sure_total) atomicAdd(&bs->n_sure, sure_total);
+        if (maybe_total) atomicAdd(&bs->n_maybe, maybe_total);
+    }
+    if (!last_block_done(&bs->ticket[2])) return;
+    // the last block: is T inside the bracket? then the first radix round on key - lo
+    const unsigned long long n_sure = *reinterpret_cast<volatile unsigned long long*>(&bs->n_sure);
+    const unsigned long long n_maybe = *reinterpret_cast<volatile unsigned long long*>(&bs->n_maybe);
+    const bool inside = n_sure < (unsigned long long)k && (unsigned long long)k <= n_sure + n_maybe;
+    uint32_t bin = 0; int64_t krem = 0;
+    const bool found = inside && block_find_bin<B1_BINS>(hist1, k - (int64_t)n_sure, &bin, &krem);
+    if (tid == 0) {
+        if (found) { bs->rel_prefix = bin; bs->k_rem = krem; bs->T = lo + (bin << sh1); }
+        else bs->fallback = 1u;
+    }
 }
 
-// The kernels below walk the candidate segments with one warp per chunk. A segment holds a few hundred
-// entries, so the walk is bound by memory round trips, not bytes: each warp fetches the first CB * 32
-// keys of its NEXT chunk (and the count of the one after) before it works on the current one.
-constexpr int CB = 8;
-
-struct SegCursor {
-    const uint32_t* __restrict__ seg_key;
-    const uint32_t* __restrict__ chunk_cnt;
-    int64_t nchunk, nwarp, c;
-    int lane;
-    int cnt, cnt_next;                  // of chunk c and of chunk c + nwarp
-    uint32_t k[CB], k_next[CB];         // first batch of chunk c / c + nwarp (lanes beyond the count: unspecified)
-
-    __device__ __forceinline__ void fetch_keys(int64_t chunk, int n, uint32_t (&dst)[CB]) const
-    {
-        const uint32_t* seg = seg_key + chunk * SG_CH;
+// Radix rounds 2 and 3 on the pairs: keys whose higher bits of key - lo equal the prefix fixed so far are
+// histogrammed on the round's bits; the last block to finish fixes them. A round of zero bits does nothing.
+template <int ROUND>
+__device__ __forceinline__ void pair_hist_body(const ChunkLists& L, const uint32_t* __restrict__ chunk_cnt, int64_t nchunk,
+                                               BracketState* __restrict__ bs, uint32_t* __restrict__ hist)
+{
+    __shared__ uint32_t s_h[B23_BINS];
+    const uint32_t b = bs->b[ROUND];
+    if (b == 0u) return;
+    for (int i = threadIdx.x; i < B23_BINS; i += SG_T) s_h[i] = 0;
+    __syncthreads();
+    const uint32_t lo = bs->lo_key, prefix = bs->rel_prefix, sh_prev = bs->sh[ROUND - 1], sh = bs->sh[ROUND], mask = (1u << b) - 1u;
+    const int lane = threadIdx.x & 31;
+    const int64_t nwarp = (int64_t)gridDim.x * (SG_T / 32);
+    auto add = [&](uint32_t key) {
+        const uint32_t rel = key - lo;
+        if ((rel >> sh_prev) == prefix) atomicAdd(&s_h[(rel >> sh) & mask], 1u);
+    };
+    // a warp takes PG consecutive chunks at a time: their counts in one load, then the first 128 pairs of every one
+    // of them in flight together (a chunk holds some 90 pairs; a list is too short to hide a memory round trip)
+    for (int64_t c0 = ((int64_t)blockIdx.x * (SG_T / 32) + (threadIdx.x >> 5)) * PG; c0 < nchunk; c0 += nwarp * PG) {
+        const int nc = (int)((nchunk - c0 < PG) ? nchunk - c0 : PG);
+        const uint32_t cnt_l = (lane < nc) ? __ldg(chunk_cnt + c0 + lane) >> 16 : 0u;
+        uint32_t v[PG][PU];
 #pragma unroll
-        for (int q = 0; q < CB; ++q) {
-            const int j = q * 32 + lane;
-            if (j < n) dst[q] = __ldg(seg + j);
+        for (int q = 0; q < PG; ++q) {
+            const int m = (int)__shfl_sync(0xFFFFFFFFu, cnt_l, q);
+            const uint32_t* seg = L.key_p + (c0 + q) * PP;
+#pragma unroll
+            for (int t = 0; t < PU; ++t) v[q][t] = (lane + 32 * t < m) ? __ldg(seg + lane + 32 * t) : 0u;
+        }
+#pragma unroll
+        for (int q = 0; q < PG; ++q) {
+            const int m = (int)__shfl_sync(0xFFFFFFFFu, cnt_l, q);
+#pragma unroll
+            for (int t = 0; t < PU; ++t) if (lane + 32 * t < m) add(v[q][t]);
+            if (m > PP) {
+                const uint32_t* seg = L.key_o + (c0 + q) * SG_CH;
+                for (int j = PP + lane; j < m; j += 32) add(__ldg(seg + j));
+            }
         }
     }
-    __device__ __forceinline__ void start(const uint32_t* sk, const uint32_t* cc, int64_t n)
-    {
-        seg_key = sk; chunk_cnt = cc; nchunk = n;
-        lane = threadIdx.x & 31;
-        nwarp = (int64_t)gridDim.x * (blockDim.x >> 5);
-        c = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-        cnt = (c < nchunk) ? (int)__ldg(chunk_cnt + c) : 0;
-        cnt_next = (c + nwarp < nchunk) ? (int)__ldg(chunk_cnt + c + nwarp) : 0;
-        if (c < nchunk) fetch_keys(c, cnt, k);
+    __syncthreads();
+    for (int i = threadIdx.x; i < B23_BINS; i += SG_T)
+        if (s_h[i]) atomicAdd(&hist[i], s_h[i]);
+    if (!last_block_done(&bs->ticket[2 + ROUND])) return;
+    uint32_t bin = 0; int64_t krem = 0;
+    const bool found = block_find_bin<B23_BINS>(hist, bs->k_rem, &bin, &krem);
+    if (threadIdx.x == 0) {
+        if (found) { const uint32_t np = (prefix << b) | bin; bs->rel_prefix = np; bs->k_rem = krem; bs->T = lo + (np << sh); }
+        else bs->fallback = 1u;          // cannot happen for counts that are consistent; fail safe
     }
-    __device__ __forceinline__ bool valid() const { return c < nchunk; }
-    // issue the loads for the chunks ahead; call before working on chunk c
-    __device__ __forceinline__ int prefetch()
-    {
-        const int cnt_after = (c + 2 * nwarp < nchunk) ? (int)__ldg(chunk_cnt + c + 2 * nwarp) : 0;
-        if (c + nwarp < nchunk) fetch_keys(c + nwarp, cnt_next, k_next);
-        return cnt_after;
-    }
-    __device__ __forceinline__ void advance(int cnt_after)
-    {
-        c += nwarp; cnt = cnt_next; cnt_next = cnt_after;
+}
+
+// Per chunk: how many of its scores are larger than T (the first class, counted by the streaming pass, and the pairs above T) and how many equal
+// T. Block b owns the chunks [b R, (b + 1) R) and leaves their totals for the write kernel.
+__device__ __forceinline__ void pair_count_body(const ChunkLists& L, const uint32_t* __restrict__ chunk_cnt, int64_t nchunk, int64_t R,
+                                                int64_t G, const BracketState* __restrict__ bs, int32_t* __restrict__ blk_cnt,
+                                                int64_t* __restrict__ blk_tot)
+{
+    __shared__ int64_t s_t[2][SG_T / 32];
+    if ((int64_t)blockIdx.x >= G) return;            // the launch may be wider than the partition
+    const uint32_t T = bs->T;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t c_lo = (int64_t)blockIdx.x * R, c_hi = (c_lo + R < nchunk) ? c_lo + R : nchunk;
+    int64_t tot_gt = 0, tot_eq = 0;
+    for (int64_t c0 = c_lo + warp * PG; c0 < c_hi; c0 += (SG_T / 32) * PG) {
+        const int nc = (int)((c_hi - c0 < PG) ? c_hi - c0 : PG);
+        const uint32_t cw = (lane < nc) ? __ldg(chunk_cnt + c0 + lane) : 0u;
+        uint32_t v[PG][PU];
 #pragma unroll
-        for (int q = 0; q < CB; ++q) k[q] = k_next[q];
+        for (int q = 0; q < PG; ++q) {
+            const int m = (int)(__shfl_sync(0xFFFFFFFFu, cw, q) >> 16);
+            const uint32_t* seg = L.key_p + (c0 + q) * PP;
+#pragma unroll
+            for (int t = 0; t < PU; ++t) v[q][t] = (lane + 32 * t < m) ? __ldg(seg + lane + 32 * t) : 0u;
+        }
+        int my_gt = 0, my_eq = 0;                   // lane q ends up with the counts of chunk c0 + q
+#pragma unroll
+        for (int q = 0; q < PG; ++q) {
+            const uint32_t w = __shfl_sync(0xFFFFFFFFu, cw, q);
+            const int n = (int)(w & 0xFFFFu), m = (int)(w >> 16);
+            int gt = 0, eq = 0;
+#pragma unroll
+            for (int t = 0; t < PU; ++t) if (lane + 32 * t < m) { gt += (v[q][t] > T); eq += (v[q][t] == T); }
+            if (m > PP) {
+                const uint32_t* seg = L.key_o + (c0 + q) * SG_CH;
+                for (int j = PP + lane; j < m; j += 32) { const uint32_t key = __ldg(seg + j); gt += (key > T); eq += (key == T); }
+            }
+            gt = __reduce_add_sync(0xFFFFFFFFu, gt);
+            eq = __reduce_add_sync(0xFFFFFFFFu, eq);
+            if (lane == q) { my_gt = gt + n; my_eq = eq; }      // n: the chunk's scores above hi
+        }
+        if (lane < nc) *reinterpret_cast<int2*>(blk_cnt + 2 * (c0 + lane)) = make_int2(my_gt, my_eq);
+        tot_gt += my_gt; tot_eq += my_eq;
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { tot_gt += __shfl_xor_sync(0xFFFFFFFFu, tot_gt, o); tot_eq += __shfl_xor_sync(0xFFFFFFFFu, tot_eq, o); }
+    if (lane == 0) { s_t[0][warp] = tot_gt; s_t[1][warp] = tot_eq; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int64_t a = 0, b = 0;
+        for (int w = 0; w < SG_T / 32; ++w) { a += s_t[0][w]; b += s_t[1][w]; }
+        blk_tot[2 * blockIdx.x] = a; blk_tot[2 * blockIdx.x + 1] = b;
+    }
+}
+
+// Final write. Block b owns the chunks [b R, (b + 1) R) (the partition of the count kernel), its warps consecutive
+// runs of them. For a chunk the warp marks, in a 4096-bit map in shared memory, the offsets of the pairs that are
+// selected: key above T, or equal to T while ties are still admitted (ties by ascending offset, ranked through a
+// second map if the chunk holds the last admitted tie). OR-ed with the chunk's first-class bitmap this is the bitmap
+// of the selected scores; a lane owns four of its words, a warp scan of their population counts gives the lane its
+// place in the output, and it writes the indices of its set bits in ascending order.
+__device__ __forceinline__ void pair_write_body(const ChunkLists& L, const uint32_t* __restrict__ chunk_cnt, int64_t nchunk, int64_t R,
+                                                int64_t G, const BracketState* __restrict__ bs, const int32_t* __restrict__ blk_cnt,
+                                                const int64_t* __restrict__ blk_tot, int64_t* __restrict__ indices)
+{
+    __shared__ __align__(16) uint32_t s_bm[SG_T / 32][2][BMW];
+    __shared__ uint16_t s_stage[SG_T / 32][SG_CH / 4];
+    __shared__ int64_t s_w[2][SG_T / 32];
+    if ((int64_t)blockIdx.x >= G) return;            // the launch may be wider than the partition
+    const uint32_t T = bs->T;
+    const int64_t k_ties = bs->k_rem;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint16_t* stage = s_stage[warp];
+    int64_t gt_run, eq_run;
+    block_base_before(blk_tot, gt_run, eq_run);
+    const int64_t c_lo = (int64_t)blockIdx.x * R, c_hi = (c_lo + R < nchunk) ? c_lo + R : nchunk;
+    // this warp's run of chunks, and what the warps before it in the block contribute
+    const int64_t per_w = (c_hi - c_lo + SG_T / 32 - 1) / (SG_T / 32);
+    const int64_t w_lo = (c_lo + warp * per_w < c_hi) ? c_lo + warp * per_w : c_hi;
+    const int64_t w_hi = (w_lo + per_w < c_hi) ? w_lo + per_w : c_hi;
+    {
+        int64_t a = 0, b = 0;
+        for (int64_t c = w_lo + lane; c < w_hi; c += 32) { const int2 v = *reinterpret_cast<const int2*>(blk_cnt + 2 * c); a += v.x; b += v.y; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { a += __shfl_xor_sync(0xFFFFFFFFu, a, o); b += __shfl_xor_sync(0xFFFFFFFFu, b, o); }
+        if (lane == 0) { s_w[0][warp] = a; s_w[1][warp] = b; }
+        __syncthreads();
+        for (int w = 0; w < warp; ++w) { gt_run += s_w[0][w]; eq_run += s_w[1][w]; }
+    }
+    uint32_t* bm_sel = s_bm[warp][0];
+    uint32_t* bm_tie = s_bm[warp][1];
+    static_assert(BMW == 128, "a lane owns four bitmap words");
+    // everything the next chunk needs is requested while the current one is worked on
+    uint32_t cw_n = 0; int2 ge_n = make_int2(0, 0); uint4 sure_n = make_uint4(0u, 0u, 0u, 0u);
+    uint32_t pk_n[PU], po_n[PU];
+    auto request = [&](int64_t c) {
+        cw_n = __ldg(chunk_cnt + c);
+        ge_n = *reinterpret_cast<const int2*>(blk_cnt + 2 * c);
+        sure_n = __ldg(reinterpret_cast<const uint4*>(L.sure_bm + c * BMW) + lane);
+        // the first PP pairs: slots beyond the chunk's count hold stale data and are ignored below
+#pragma unroll
+        for (int t = 0; t < PU; ++t) { pk_n[t] = __ldg(L.key_p + c * PP + lane + 32 * t); po_n[t] = (uint32_t)__ldg(L.off_p + c * PP + lane + 32 * t); }
+    };
+    if (w_lo < w_hi) request(w_lo);
+    for (int64_t c = w_lo; c < w_hi; ++c) {
+        const uint32_t cw = cw_n;
+        const int2 ge = ge_n;
+        uint4 f4 = sure_n;
+        uint32_t pk[PU], po[PU];
+#pragma unroll
+        for (int t = 0; t < PU; ++t) { pk[t] = pk_n[t]; po[t] = po_n[t]; }
+        if (c + 1 < w_hi) request(c + 1);
+        const int m = (int)(cw >> 16);
+        if (m > 0) {
+            reinterpret_cast<uint4*>(bm_sel)[lane] = make_uint4(0u, 0u, 0u, 0u);
+            reinterpret_cast<uint4*>(bm_tie)[lane] = make_uint4(0u, 0u, 0u, 0u);
+            __syncwarp();
+#pragma unroll
+            for (int t = 0; t < PU; ++t)
+                if (lane + 32 * t < m && pk[t] >= T) atomicOr((pk[t] > T ? bm_sel : bm_tie) + (po[t] >> 5), 1u << (po[t] & 31u));
+            for (int j = PP + lane; j < m; j += 32) {
+                const uint32_t key = __ldg(L.key_o + c * SG_CH + j);
+                if (key >= T) { const uint32_t o = __ldg(L.off_o + c * SG_CH + j); atomicOr((key > T ? bm_sel : bm_tie) + (o >> 5), 1u << (o & 31u)); }
+            }
+            __syncwarp();
+            uint4 s4 = reinterpret_cast<const uint4*>(bm_sel)[lane];
+            if (ge.y > 0) {
+                const int64_t room64 = k_ties - eq_run;                               // ties this chunk may still admit
+                const uint4 t4 = reinterpret_cast<const uint4*>(bm_tie)[lane];
+                if (room64 >= (int64_t)ge.y) {                                        // all of them
+                    s4.x |= t4.x; s4.y |= t4.y; s4.z |= t4.z; s4.w |= t4.w;
+                } else if (room64 > 0) {                                              // the first room64 by offset
+                    const uint32_t tw[4] = {t4.x, t4.y, t4.z, t4.w};
+                    const int cnt = __popc(tw[0]) + __popc(tw[1]) + __popc(tw[2]) + __popc(tw[3]);
+                    int incl = cnt;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) { const int a = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += a; }
+                    int rank = incl - cnt;                                            // ties before this lane's words
+                    const int room = (int)room64;
+                    uint32_t keep[4];
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t word = tw[q];
+                        keep[q] = 0u;
+                        while (word && rank < room) { const uint32_t low = word & (0u - word); keep[q] |= low; word ^= low; ++rank; }
+                        rank += __popc(word);
+                    }
+                    s4.x |= keep[0]; s4.y |= keep[1]; s4.z |= keep[2]; s4.w |= keep[3];
+                }
+            }
+            f4.x |= s4.x; f4.y |= s4.y; f4.z |= s4.z; f4.w |= s4.w;
+            __syncwarp();       // the maps are read: they may be cleared for the next chunk
+        }
+        // The selected scores of the chunk, in index order: a lane's four words cover offsets [128 lane, 128 lane + 128); a
+        // warp scan of the lanes' population counts ranks their set bits, which are staged as 16-bit offsets and then
+        // leave as consecutive 64-bit indices, 32 per store (a lane writing its own indices one by one touched a
+        // 32-byte sector per 8 bytes written). The staging area holds a quarter of a chunk; a chunk with more selected
+        // scores than that goes through it quarter by quarter.
+        int64_t* out = indices + gt_run + (eq_run < k_ties ? eq_run : k_ties);
+        const int64_t ibase = c * SG_CH;
+        {
+            const uint32_t fw[4] = {f4.x, f4.y, f4.z, f4.w};
+            const int cnt = __popc(fw[0]) + __popc(fw[1]) + __popc(fw[2]) + __popc(fw[3]);
+            int incl = cnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int a = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += a; }
+            const int tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            if (tot <= SG_CH / 4) {
+                int pos = incl - cnt;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t word = fw[q];
+                    const uint32_t obase = (uint32_t)(lane * 128 + q * 32);
+                    while (word) {
+                        const int b = __ffs((int)word) - 1;
+                        word &= word - 1u;
+                        stage[pos++] = (uint16_t)(obase + (uint32_t)b);
+                    }
+                }
+                __syncwarp();
+                for (int i = lane; i < tot; i += 32) out[i] = ibase + stage[i];
+                __syncwarp();       // the staging area is rewritten by the next chunk
+                gt_run += ge.x; eq_run += ge.y;
+                continue;
+            }
+        }
+        reinterpret_cast<uint4*>(bm_sel)[lane] = f4;
+        __syncwarp();
+#pragma unroll 1
+        for (int qt = 0; qt < 4; ++qt) {
+            uint32_t word = bm_sel[qt * 32 + lane];
+            const int cnt = __popc(word);
+            int incl = cnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int a = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += a; }
+            const int tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            if (tot == 0) continue;
+            int pos = incl - cnt;
+            const uint32_t obase = (uint32_t)((qt * 32 + lane) * 32);
+            while (word) {
+                const int b = __ffs((int)word) - 1;
+                word &= word - 1u;
+                stage[pos++] = (uint16_t)(obase + (uint32_t)b);
+            }
+            __syncwarp();
+            for (int i = lane; i < tot; i += 32) out[i] = ibase + stage[i];
+            out += tot;
+            __syncwarp();       // the staging area is rewritten by the next quarter
+        }
+        gt_run += ge.x; eq_run += ge.y;
+    }
+}
+
+// The launches behind the streaming pass. Each does its step of the bracketed path or, if the bracket missed T (the
+// flag the streaming pass left), the matching step of the exact multi-pass path on the scores: one launch serves
+// both, so that the rare path costs one extra launch (its final write) instead of five that return at once.
+struct FallbackArgs {
+    const float* scores; int64_t N, k;
+    SelectState* state; uint32_t* hist;          // three cleared histograms
+    int64_t nblk, R, G;                          // units of 2048 scores and their partition over blocks
 };
 
-// Radix-select rounds 2 and 3 on the candidates.
-template <int PASS>
 __global__ void __launch_bounds__(SG_T)
-cand_hist_kernel(const uint32_t* __restrict__ seg_key, const uint32_t* __restrict__ chunk_cnt, int64_t nchunk,
-                 const SelectState* __restrict__ state, uint32_t* __restrict__ hist, Gate gate)
+bracket_round2_kernel(const ChunkLists L, const uint32_t* __restrict__ chunk_cnt, int64_t nchunk, BracketState* __restrict__ bs,
+                      uint32_t* __restrict__ hist, const FallbackArgs fb)
 {
-    __shared__ uint32_t s_h[2048];
-    if (gate.closed()) return;
-    for (int i = threadIdx.x; i < 2048; i += blockDim.x) s_h[i] = 0;
-    __syncthreads();
-    const uint32_t prefix = state->prefix;
-    auto add = [&](uint32_t key) {
-        if (PASS == 1) { if ((key >> 21) == prefix) atomicAdd(&s_h[(key >> 10) & 0x7FFu], 1u); }
-        else { if ((key >> 10) == prefix) atomicAdd(&s_h[key & 0x3FFu], 1u); }
-    };
-    SegCursor cur;
-    for (cur.start(seg_key, chunk_cnt, nchunk); cur.valid();) {
-        const int after = cur.prefetch();
-#pragma unroll
-        for (int q = 0; q < CB; ++q)
-            if (q * 32 + cur.lane < cur.cnt) add(cur.k[q]);
-        const uint32_t* seg = seg_key + cur.c * SG_CH;
-        for (int j = CB * 32 + cur.lane; j < cur.cnt; j += 32) add(seg[j]);       // segments longer than a batch
-        cur.advance(after);
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < 2048; i += blockDim.x)
-        if (s_h[i]) atomicAdd(&hist[i], s_h[i]);
+    dep_wait();
+    dep_release();
+    if (bs->fallback != 0u) select_hist_body<0>(fb.scores, fb.N, fb.k, fb.state, fb.hist);
+    else pair_hist_body<1>(L, chunk_cnt, nchunk, bs, hist);
 }
-
 __global__ void __launch_bounds__(SG_T)
-cand_count_kernel(const uint32_t* __restrict__ seg_key, const uint32_t* __restrict__ chunk_cnt, int64_t nchunk,
-                  const SelectState* __restrict__ state, int32_t* __restrict__ blk_cnt, Gate gate)
+bracket_round3_kernel(const ChunkLists L, const uint32_t* __restrict__ chunk_cnt, int64_t nchunk, BracketState* __restrict__ bs,
+                      uint32_t* __restrict__ hist, const FallbackArgs fb)
 {
-    if (gate.closed()) return;
-    const uint32_t T = state->prefix;
-    SegCursor cur;
-    for (cur.start(seg_key, chunk_cnt, nchunk); cur.valid();) {
-        const int after = cur.prefetch();
-        int gt = 0, eq = 0;
-#pragma unroll
-        for (int q = 0; q < CB; ++q)
-            if (q * 32 + cur.lane < cur.cnt) { gt += (cur.k[q] > T); eq += (cur.k[q] == T); }
-        const uint32_t* seg = seg_key + cur.c * SG_CH;
-        for (int j = CB * 32 + cur.lane; j < cur.cnt; j += 32) { const uint32_t key = seg[j]; gt += (key > T); eq += (key == T); }
-        gt = __reduce_add_sync(0xFFFFFFFFu, gt);
-        eq = __reduce_add_sync(0xFFFFFFFFu, eq);
-        if (cur.lane == 0) *reinterpret_cast<int2*>(blk_cnt + 2 * cur.c) = make_int2(gt, eq);
-        cur.advance(after);
-    }
+    dep_wait();
+    dep_release();
+    if (bs->fallback != 0u) select_hist_body<1>(fb.scores, fb.N, fb.k, fb.state, fb.hist + 2048);
+    else pair_hist_body<2>(L, chunk_cnt, nchunk, bs, hist);
 }
-
-// Final write: a warp per chunk marks the offsets of {key > T} and of {key == T} in two 4096-bit maps
-// in shared memory, which puts the segment's unordered candidates back in index order: the number of
-// set bits below a candidate's offset (a per-word prefix plus a masked population count) is how many
-// of the chunk's larger or equal-key scores come before it, and with the chunk's offsets that is its
-// place in the output.
 __global__ void __launch_bounds__(SG_T)
-cand_write_kernel(const uint32_t* __restrict__ seg_key, const uint16_t* __restrict__ seg_off,
-                  const uint32_t* __restrict__ chunk_cnt, int64_t nchunk, const SelectState* __restrict__ state,
-                  const int64_t* __restrict__ blk_off, int64_t* __restrict__ indices, Gate gate)
+bracket_count_kernel(const ChunkLists L, const uint32_t* __restrict__ chunk_cnt, int64_t nchunk, int64_t R, int64_t G,
+                     const BracketState* __restrict__ bs, int32_t* __restrict__ blk_cnt, int64_t* __restrict__ blk_tot,
+                     const FallbackArgs fb)
 {
-    __shared__ __align__(16) uint32_t s_bm[SG_T / 32][2][SG_CH / 32];
-    __shared__ __align__(16) uint16_t s_pre[SG_T / 32][2][SG_CH / 32];      // set bits in the words before
-    if (gate.closed()) return;
-    const uint32_t T = state->prefix;
-    const int64_t k_ties = state->k_rem;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t* bm_gt = s_bm[warp][0];
-    uint32_t* bm_eq = s_bm[warp][1];
-    uint16_t* pre_gt = s_pre[warp][0];
-    uint16_t* pre_eq = s_pre[warp][1];
-    SegCursor cur;
-    for (cur.start(seg_key, chunk_cnt, nchunk); cur.valid();) {
-        const int after = cur.prefetch();
-        const int64_t c = cur.c;
-        const int cnt = cur.cnt;
-        if (cnt == 0) { cur.advance(after); continue; }
-        const uint32_t* seg = seg_key + c * SG_CH;
-        const uint16_t* off = seg_off + c * SG_CH;
-        const longlong2 base2 = *reinterpret_cast<const longlong2*>(blk_off + 2 * c);
-        // offsets of the first batch, for the entries that are selected or tied (all loads issued together)
-        uint32_t o[CB];
-#pragma unroll
-        for (int q = 0; q < CB; ++q) {
-            const int j = q * 32 + lane;
-            o[q] = (j < cnt && cur.k[q] >= T) ? (uint32_t)off[j] : 0xFFFFFFFFu;
-        }
-        reinterpret_cast<uint4*>(bm_gt)[lane] = make_uint4(0u, 0u, 0u, 0u);
-        reinterpret_cast<uint4*>(bm_eq)[lane] = make_uint4(0u, 0u, 0u, 0u);
-        __syncwarp();
-#pragma unroll
-        for (int q = 0; q < CB; ++q)
-            if (o[q] != 0xFFFFFFFFu) atomicOr((cur.k[q] > T ? bm_gt : bm_eq) + (o[q] >> 5), 1u << (o[q] & 31u));
-        for (int j = CB * 32 + lane; j < cnt; j += 32) {                 // segments longer than a batch
-            const uint32_t key = seg[j];
-            if (key >= T) { const uint32_t oo = off[j]; atomicOr((key > T ? bm_gt : bm_eq) + (oo >> 5), 1u << (oo & 31u)); }
-        }
-        __syncwarp();
-        const uint4 g4 = reinterpret_cast<const uint4*>(bm_gt)[lane];
-        const uint4 e4 = reinterpret_cast<const uint4*>(bm_eq)[lane];
-        const int pg[4] = {__popc(g4.x), __popc(g4.y), __popc(g4.z), __popc(g4.w)};
-        const int pe[4] = {__popc(e4.x), __popc(e4.y), __popc(e4.z), __popc(e4.w)};
-        const int cg = pg[0] + pg[1] + pg[2] + pg[3], ce = pe[0] + pe[1] + pe[2] + pe[3];
-        int ig = cg, ie = ce;
-#pragma unroll
-        for (int sh = 1; sh < 32; sh <<= 1) {
-            const int a2 = __shfl_up_sync(0xFFFFFFFFu, ig, sh), b2 = __shfl_up_sync(0xFFFFFFFFu, ie, sh);
-            if (lane >= sh) { ig += a2; ie += b2; }
-        }
-        ig -= cg; ie -= ce;
-        reinterpret_cast<uint2*>(pre_gt)[lane] = make_uint2((uint32_t)ig | ((uint32_t)(ig + pg[0]) << 16),
-                                                            (uint32_t)(ig + pg[0] + pg[1]) | ((uint32_t)(ig + pg[0] + pg[1] + pg[2]) << 16));
-        reinterpret_cast<uint2*>(pre_eq)[lane] = make_uint2((uint32_t)ie | ((uint32_t)(ie + pe[0]) << 16),
-                                                            (uint32_t)(ie + pe[0] + pe[1]) | ((uint32_t)(ie + pe[0] + pe[1] + pe[2]) << 16));
-        __syncwarp();
-        // place = (larger keys before) + min(ties before, k_ties): the chunk's own part of both in 32 bits
-        const int64_t room64 = k_ties - base2.y;                                  // ties this chunk may still admit
-        const uint32_t room = room64 <= 0 ? 0u : (room64 >= SG_CH ? (uint32_t)SG_CH : (uint32_t)room64);
-        int64_t* out = indices + base2.x + (base2.y < k_ties ? base2.y : k_ties);
-        const int64_t ibase = c * SG_CH;
-        auto place = [&](uint32_t key, uint32_t oo) {
-            const uint32_t w = oo >> 5, below = (1u << (oo & 31u)) - 1u;
-            const uint32_t g_loc = pre_gt[w] + __popc(bm_gt[w] & below);
-            const uint32_t e_loc = pre_eq[w] + __popc(bm_eq[w] & below);
-            if (key > T || e_loc < room) out[g_loc + (e_loc < room ? e_loc : room)] = ibase + oo;
-        };
-#pragma unroll
-        for (int q = 0; q < CB; ++q)
-            if (o[q] != 0xFFFFFFFFu) place(cur.k[q], o[q]);
-        for (int j = CB * 32 + lane; j < cnt; j += 32) {
-            const uint32_t key = seg[j];
-            if (key >= T) place(key, off[j]);
-        }
-        __syncwarp();       // the maps are cleared again for the warp's next chunk
-        cur.advance(after);
-    }
+    dep_wait();
+    dep_release();
+    if (bs->fallback != 0u) select_hist_body<2>(fb.scores, fb.N, fb.k, fb.state, fb.hist + 4096);
+    else pair_count_body(L, chunk_cnt, nchunk, R, G, bs, blk_cnt, blk_tot);
+}
+__global__ void __launch_bounds__(SG_T, 6)
+bracket_write_kernel(const ChunkLists L, const uint32_t* __restrict__ chunk_cnt, int64_t nchunk, int64_t R, int64_t G,
+                     const BracketState* __restrict__ bs, int32_t* __restrict__ blk_cnt, int64_t* __restrict__ blk_tot,
+                     int64_t* __restrict__ indices, const FallbackArgs fb)
+{
+    dep_wait();
+    dep_release();
+    if (bs->fallback != 0u) select_count_body(fb.scores, fb.N, fb.nblk, fb.R, fb.G, fb.state, blk_cnt, blk_tot);
+    else pair_write_body(L, chunk_cnt, nchunk, R, G, bs, blk_cnt, blk_tot, indices);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -871,16 +1047,16 @@ SelectWs carve(void* ws, int64_t N)
     uint8_t* p = reinterpret_cast<uint8_t*>(ws);
     w.hist = reinterpret_cast<uint32_t*>(p); p += 3 * 2048 * sizeof(uint32_t);
     w.state = reinterpret_cast<SelectState*>(p); p += 256;
-    const int64_t nblk = sel_nblk(N);
-    w.blk_off = reinterpret_cast<int64_t*>(p); p += align_up((size_t)nblk * 2 * sizeof(int64_t), 256);
+    w.blk_tot = reinterpret_cast<int64_t*>(p); p += (size_t)SEL_MAX_GRID * 2 * sizeof(int64_t);
     w.blk_cnt = reinterpret_cast<int32_t*>(p);
+    (void)N;
     return w;
 }
 
 size_t compact_workspace_bytes(int64_t N)
 {
     const int64_t nblk = sel_nblk(N > 0 ? N : 1);
-    return 3 * 2048 * sizeof(uint32_t) + 256 + align_up((size_t)nblk * 2 * sizeof(int64_t), 256) +
+    return 3 * 2048 * sizeof(uint32_t) + 256 + (size_t)SEL_MAX_GRID * 2 * sizeof(int64_t) +
            align_up((size_t)nblk * 2 * sizeof(int32_t), 256);
 }
 
@@ -888,50 +1064,51 @@ BracketWs carve_bracket(void* ws, int64_t N)
 {
     BracketWs w;
     uint8_t* p = reinterpret_cast<uint8_t*>(ws);
-    w.hist = reinterpret_cast<uint32_t*>(p); p += 6 * 2048 * sizeof(uint32_t);
-    w.state = reinterpret_cast<SelectState*>(p);
-    w.bstate = reinterpret_cast<BracketState*>(p + 64); p += 256;
+    w.hist = reinterpret_cast<uint32_t*>(p); p += (size_t)BR_HIST_WORDS * sizeof(uint32_t);
+    w.bstate = reinterpret_cast<BracketState*>(p); p += 256;
+    w.fstate = reinterpret_cast<SelectState*>(p); p += 256;
     const int64_t nblk = sel_nblk(N), nchunk = sg_nchunk(N);
-    w.blk_off = reinterpret_cast<int64_t*>(p); p += align_up((size_t)nblk * 2 * sizeof(int64_t), 256);
+    w.blk_tot = reinterpret_cast<int64_t*>(p); p += (size_t)SEL_MAX_GRID * 2 * sizeof(int64_t);
     w.blk_cnt = reinterpret_cast<int32_t*>(p); p += align_up((size_t)nblk * 2 * sizeof(int32_t), 256);
-    w.tile_tot = reinterpret_cast<int64_t*>(p); p += align_up((size_t)((nblk + 1023) / 1024) * 2 * sizeof(int64_t), 256);
     w.sample_key = reinterpret_cast<uint32_t*>(p); p += SG_SAMPLE * sizeof(uint32_t);
     w.chunk_cnt = reinterpret_cast<uint32_t*>(p); p += align_up((size_t)nchunk * sizeof(uint32_t), 256);
-    w.seg_off = reinterpret_cast<uint16_t*>(p); p += align_up((size_t)nchunk * SG_CH * sizeof(uint16_t), 256);
-    w.seg_key = reinterpret_cast<uint32_t*>(p);
+    w.L.sure_bm = reinterpret_cast<uint32_t*>(p); p += align_up((size_t)nchunk * BMW * sizeof(uint32_t), 256);
+    w.L.key_p = reinterpret_cast<uint32_t*>(p); p += align_up((size_t)nchunk * PP * sizeof(uint32_t), 256);
+    w.L.off_p = reinterpret_cast<uint16_t*>(p); p += align_up((size_t)nchunk * PP * sizeof(uint16_t), 256);
+    w.L.off_o = reinterpret_cast<uint16_t*>(p); p += align_up((size_t)nchunk * SG_CH * sizeof(uint16_t), 256);
+    w.L.key_o = reinterpret_cast<uint32_t*>(p);
     return w;
 }
 
 size_t bracket_workspace_bytes(int64_t N)
 {
     const int64_t nblk = sel_nblk(N), nchunk = sg_nchunk(N);
-    return 6 * 2048 * sizeof(uint32_t) + 256 + align_up((size_t)nblk * 2 * sizeof(int64_t), 256) +
-           align_up((size_t)nblk * 2 * sizeof(int32_t), 256) + align_up((size_t)((nblk + 1023) / 1024) * 2 * sizeof(int64_t), 256) +
-           SG_SAMPLE * sizeof(uint32_t) + align_up((size_t)nchunk * sizeof(uint32_t), 256) +
+    return (size_t)BR_HIST_WORDS * sizeof(uint32_t) + 512 + (size_t)SEL_MAX_GRID * 2 * sizeof(int64_t) +
+           align_up((size_t)nblk * 2 * sizeof(int32_t), 256) + SG_SAMPLE * sizeof(uint32_t) +
+           align_up((size_t)nchunk * sizeof(uint32_t), 256) + align_up((size_t)nchunk * BMW * sizeof(uint32_t), 256) +
+           align_up((size_t)nchunk * PP * sizeof(uint32_t), 256) + align_up((size_t)nchunk * PP * sizeof(uint16_t), 256) +
            align_up((size_t)nchunk * SG_CH * sizeof(uint16_t), 256) + (size_t)nchunk * SG_CH * sizeof(uint32_t);
 }
+static_assert(sizeof(BracketState) <= 256 && sizeof(SelectState) <= 256, "state regions are 256 bytes");
 
-// The exact multi-pass path on the scores themselves (five reads). hist: three cleared histograms.
+// The exact multi-pass path on the scores themselves (five reads, five launches). hist: three cleared histograms;
+// state: cleared.
 cudaError_t launch_multipass(const float* scores, int64_t N, int64_t k, int64_t* indices, uint32_t* hist,
-                             SelectState* state, int32_t* blk_cnt, int64_t* blk_off, int64_t* tile_tot, Gate gate, cudaStream_t st)
+                             SelectState* state, int32_t* blk_cnt, int64_t* blk_tot, cudaStream_t st)
 {
     int64_t hb = (N / 4 + SEL_T - 1) / SEL_T;
     const int64_t cap = (int64_t)sm_count() * 8;
     if (hb > cap) hb = cap;
     if (hb < 1) hb = 1;
-    select_hist_kernel<0><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, state, hist, gate);
-    select_scan_kernel<0><<<1, 1024, 0, st>>>(hist, state, k, gate, nullptr);
-    select_hist_kernel<1><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, state, hist + 2048, gate);
-    select_scan_kernel<1><<<1, 1024, 0, st>>>(hist + 2048, state, k, gate, nullptr);
-    select_hist_kernel<2><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, state, hist + 4096, gate);
-    select_scan_kernel<2><<<1, 1024, 0, st>>>(hist + 4096, state, k, gate, nullptr);
+    select_hist_kernel<0><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, k, state, hist);
+    select_hist_kernel<1><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, k, state, hist + 2048);
+    select_hist_kernel<2><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, k, state, hist + 4096);
     const int64_t nblk = sel_nblk(N);
-    const int64_t cap2 = (int64_t)sm_count() * 32;
-    const unsigned cg = (unsigned)(nblk < cap2 ? nblk : cap2);
-    select_count_kernel<<<cg, SEL_T, 0, st>>>(scores, N, nblk, state, blk_cnt, gate);
-    launch_block_scan(blk_cnt, nblk, blk_off, tile_tot, gate, st);
-    select_write_kernel<<<cg, SEL_T, 0, st>>>(scores, N, nblk, state, blk_off, indices, gate);
-    count_launches(8);
+    const int64_t G = nblk < SEL_MAX_GRID ? nblk : SEL_MAX_GRID;
+    const int64_t R = (nblk + G - 1) / G;
+    select_count_kernel<<<(unsigned)G, SEL_T, 0, st>>>(scores, N, nblk, R, G, state, blk_cnt, blk_tot);
+    select_write_kernel<<<(unsigned)G, SEL_T, 0, st>>>(scores, N, nblk, R, state, blk_cnt, blk_tot, indices, Gate{nullptr, 0u});
+    count_launches(5);
     return cudaGetLastError();
 }
 
@@ -946,32 +1123,47 @@ cudaError_t launch_bracketed(const float* scores, int64_t N, int64_t k, int64_t*
     });
     if (attr_err != cudaSuccess) return attr_err;
     BracketWs w = carve_bracket(ws, N);
-    cudaError_t e = cudaSuccess;
     const int64_t nchunk = sg_nchunk(N);
-    const int64_t cap = (int64_t)sm_count() * 8;
     const int64_t gcap = (int64_t)sm_count() * 4;          // the gather kernel's resident blocks (48 KiB ring each)
     const int64_t gneed = (nchunk + SG_T / 32 - 1) / (SG_T / 32);       // a warp per chunk
     const unsigned gb = (unsigned)(gneed < gcap ? gneed : gcap);
-    const int64_t wb = (nchunk + SG_T / 32 - 1) / (SG_T / 32);
-    const unsigned cb = (unsigned)(wb < cap ? wb : cap);
-    const Gate none{nullptr, 0u};
-    const Gate ok{&w.bstate->fallback, 0u};          // enough candidates: select among them
-    const Gate fb{&w.bstate->fallback, 1u};          // too few: exact path on the scores
-    select_init_kernel<<<SG_SAMPLE / 256, 256, 0, st>>>(scores, N, w.hist, 6 * 2048 + 64, w.sample_key);     // histograms + state
-    select_sample_kernel<<<1, 1024, 0, st>>>(w.sample_key, N, k, w.bstate, force_short ? 1 : 0);
-    select_gather_kernel<<<gb, SG_T, (SG_T / 32) * SG_RING * SG_STEP * sizeof(uint32_t), st>>>(scores, N, w.bstate, w.seg_key, w.seg_off, w.chunk_cnt, w.hist);
-    select_scan_kernel<0><<<1, 1024, 0, st>>>(w.hist, w.state, k, none, &w.bstate->fallback);
-    cand_hist_kernel<1><<<cb, SG_T, 0, st>>>(w.seg_key, w.chunk_cnt, nchunk, w.state, w.hist + 2048, ok);
-    select_scan_kernel<1><<<1, 1024, 0, st>>>(w.hist + 2048, w.state, k, ok, nullptr);
-    cand_hist_kernel<2><<<cb, SG_T, 0, st>>>(w.seg_key, w.chunk_cnt, nchunk, w.state, w.hist + 4096, ok);
-    select_scan_kernel<2><<<1, 1024, 0, st>>>(w.hist + 4096, w.state, k, ok, nullptr);
-    cand_count_kernel<<<cb, SG_T, 0, st>>>(w.seg_key, w.chunk_cnt, nchunk, w.state, w.blk_cnt, ok);
-    launch_block_scan(w.blk_cnt, nchunk, w.blk_off, w.tile_tot, ok, st);
-    cand_write_kernel<<<cb, SG_T, 0, st>>>(w.seg_key, w.seg_off, w.chunk_cnt, nchunk, w.state, w.blk_off, indices, ok);
-    count_launches(10);          // the prefix-sum launches count themselves
-    e = cudaGetLastError();
+    const int64_t hneed = (nchunk + (SG_T / 32) * PG - 1) / ((SG_T / 32) * PG);     // a warp per PG chunks
+    const int64_t hcap = (int64_t)sm_count() * 8;
+    const int64_t hb = hneed < hcap ? hneed : hcap;
+    // count and write: contiguous runs of chunks, every block resident at once (six per SM)
+    int64_t G = (int64_t)sm_count() * 6;
+    if (G > SEL_MAX_GRID) G = SEL_MAX_GRID;
+    if (G > gneed) G = gneed;
+    const int64_t R = (nchunk + G - 1) / G;
+    uint32_t* hist1 = w.hist;
+    uint32_t* hist2 = w.hist + B1_BINS;
+    uint32_t* hist3 = hist2 + B23_BINS;
+    uint32_t* hist_s = hist3 + B23_BINS + 3 * 2048;      // sample: first level, second level of lo, of hi
+    // the exact multi-pass path, should the bracket miss: its grids, and its steps riding in the launches below
+    FallbackArgs fb;
+    fb.scores = scores; fb.N = N; fb.k = k; fb.state = w.fstate; fb.hist = hist3 + B23_BINS;
+    fb.nblk = sel_nblk(N);
+    fb.G = fb.nblk < SEL_MAX_GRID ? fb.nblk : SEL_MAX_GRID;
+    fb.R = (fb.nblk + fb.G - 1) / fb.G;
+    int64_t fhb = (N / 4 + SEL_T - 1) / SEL_T;
+    if (fhb > hcap) fhb = hcap;
+    const unsigned g_round = (unsigned)(hb > fhb ? hb : fhb), g_count = (unsigned)(G > fhb ? G : fhb), g_write = (unsigned)(G > fb.G ? G : fb.G);
+    // histograms and both states are contiguous: one clear
+    cudaError_t e = cudaMemsetAsync(w.hist, 0, (size_t)(BR_HIST_WORDS + 128) * sizeof(uint32_t), st);
     if (e != cudaSuccess) return e;
-    return launch_multipass(scores, N, k, indices, w.hist + 3 * 2048, w.state, w.blk_cnt, w.blk_off, w.tile_tot, fb, st);
+    const size_t ring_bytes = (SG_T / 32) * SG_RING * SG_STEP * sizeof(uint32_t);
+    const int fs = force_short ? 1 : 0;
+    if ((e = launch_after(sample_level1_kernel, SS_BLOCKS, SEL_T, 0, st, scores, w.sample_key, N, k, w.bstate, hist_s)) != cudaSuccess) return e;
+    if ((e = launch_after(sample_level2_kernel, SS_BLOCKS, SEL_T, 0, st, w.sample_key, N, k, w.bstate, hist_s + 4096, hist_s + 8192, fs)) != cudaSuccess) return e;
+    if ((e = launch_after(select_gather_kernel, gb, SG_T, ring_bytes, st, scores, N, k, w.bstate, w.L, w.chunk_cnt, hist1)) != cudaSuccess) return e;
+    if ((e = launch_after(bracket_round2_kernel, g_round, SG_T, 0, st, w.L, w.chunk_cnt, nchunk, w.bstate, hist2, fb)) != cudaSuccess) return e;
+    if ((e = launch_after(bracket_round3_kernel, g_round, SG_T, 0, st, w.L, w.chunk_cnt, nchunk, w.bstate, hist3, fb)) != cudaSuccess) return e;
+    if ((e = launch_after(bracket_count_kernel, g_count, SG_T, 0, st, w.L, w.chunk_cnt, nchunk, R, G, w.bstate, w.blk_cnt, w.blk_tot, fb)) != cudaSuccess) return e;
+    if ((e = launch_after(bracket_write_kernel, g_write, SG_T, 0, st, w.L, w.chunk_cnt, nchunk, R, G, w.bstate, w.blk_cnt, w.blk_tot, indices, fb)) != cudaSuccess) return e;
+    if ((e = launch_after(select_write_kernel, (unsigned)fb.G, SEL_T, 0, st, scores, N, fb.nblk, fb.R, w.fstate, w.blk_cnt, w.blk_tot, indices,
+                          Gate{&w.bstate->fallback, 1u})) != cudaSuccess) return e;
+    count_launches(8);
+    return cudaGetLastError();
 }
 
 int g_select_path = 0;     // 0: by size; 1: multi-pass always; 2: bracketed with a bracket that is too high
@@ -1005,9 +1197,9 @@ cudaError_t launch_select_topk(const float* scores, int64_t N, int64_t k, int64_
     }
     if (use_bracket(N)) return launch_bracketed(scores, N, k, indices, ws, g_select_path == 2, st);
     SelectWs w = carve(ws, N);
-    cudaError_t e = cudaMemsetAsync(w.hist, 0, 3 * 2048 * sizeof(uint32_t), st);
+    cudaError_t e = cudaMemsetAsync(w.hist, 0, 3 * 2048 * sizeof(uint32_t) + 256, st);      // histograms and state
     if (e != cudaSuccess) return e;
-    return launch_multipass(scores, N, k, indices, w.hist, w.state, w.blk_cnt, w.blk_off, nullptr, Gate{nullptr, 0u}, st);
+    return launch_multipass(scores, N, k, indices, w.hist, w.state, w.blk_cnt, w.blk_tot, st);
 }
 
 }  // namespace qless
@@ -1019,8 +1211,8 @@ cudaError_t launch_select_topk(const float* scores, int64_t N, int64_t k, int64_
 namespace qless {
 namespace {
 
-// 3 histograms (24 KiB) + state (256 B) + per-block offsets and counts for MAX_N / 2048 = 2048 blocks
-// (32 KiB + 16 KiB) = 73 984 bytes; rounded up. Resident on every GPU that loads the library.
+// 3 histograms (24 KiB) + state (256 B) + block totals (16 KiB) + counts of the MAX_N / 2048 = 2048 units
+// (16 KiB) = 57 600 bytes; the array keeps its 74 KiB. Resident on every GPU that loads the library.
 constexpr size_t kStaticScratchBytes = 74 * 1024;
 static __device__ __align__(256) unsigned char g_select_scratch[kStaticScratchBytes];
 
@@ -1068,7 +1260,7 @@ extern "C" qless_status qless_select_topk_static(const float* scores, int64_t N,
     if (k > 0) {
         QLESS_REQUIRE(scores != nullptr && indices != nullptr, QLESS_ERR_INVALID_ARG, "scores and indices are required");
         QLESS_REQUIRE((reinterpret_cast<uintptr_t>(scores) % 16) == 0, QLESS_ERR_INVALID_ARG, "scores must be 16-byte aligned");
-        static_assert(kStaticScratchBytes >= 3 * 2048 * 4 + 256 + 2048 * 16 + 2048 * 8, "scratch array too small");
+        static_assert(kStaticScratchBytes >= 3 * 2048 * 4 + 256 + SEL_MAX_GRID * 16 + 2048 * 8, "scratch array too small");
         QLESS_REQUIRE(select_workspace_bytes(N) <= kStaticScratchBytes, QLESS_ERR_UNSUPPORTED, "internal: scratch array too small");
     }
     *k_out = k;
@@ -1076,8 +1268,8 @@ extern "C" qless_status qless_select_topk_static(const float* scores, int64_t N,
     void* scratch = nullptr;
     qless_status s = static_scratch(&scratch);
     if (s != QLESS_OK) return s;
-    // The histograms are cleared inside; the state and the per-block arrays are rewritten in full for
-    // this N before they are read, so nothing of the previous call's contents is used.
+    // The histograms and the selection state are cleared inside; the block totals and the unit counts are
+    // rewritten in full for this N before they are read, so nothing of the previous call's contents is used.
     QLESS_CUDA_TRY(launch_select_topk(scores, N, k, indices, scratch, st));
     return QLESS_OK;
 }
