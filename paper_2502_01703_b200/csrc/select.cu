@@ -163,6 +163,8 @@ __global__ void __launch_bounds__(SEL_T)
 select_hist_kernel(const float* __restrict__ scores, int64_t N, int64_t k, SelectState* __restrict__ state,
                    uint32_t* __restrict__ hist)
 {
+    dep_wait();
+    dep_release();
     select_hist_body<PASS>(scores, N, k, state, hist);
 }
 
@@ -210,6 +212,8 @@ __global__ void __launch_bounds__(SEL_T)
 select_count_kernel(const float* __restrict__ scores, int64_t N, int64_t nblk, int64_t R, int64_t G, const SelectState* __restrict__ state,
                     int32_t* __restrict__ blk_cnt, int64_t* __restrict__ blk_tot)
 {
+    dep_wait();
+    dep_release();
     select_count_body(scores, N, nblk, R, G, state, blk_cnt, blk_tot);
 }
 
@@ -821,7 +825,8 @@ __device__ __forceinline__ void pair_write_body(const ChunkLists& L, const uint3
         const int64_t ibase = c * SG_CH;
         {
             const uint32_t fw[4] = {f4.x, f4.y, f4.z, f4.w};
-            const int cnt = __popc(fw[0]) + __popc(fw[1]) + __popc(fw[2]) + __popc(fw[3]);
+            const int pc[4] = {__popc(fw[0]), __popc(fw[1]), __popc(fw[2]), __popc(fw[3])};
+            const int cnt = pc[0] + pc[1] + pc[2] + pc[3];
             int incl = cnt;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) { const int a = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += a; }
@@ -830,12 +835,16 @@ __device__ __forceinline__ void pair_write_body(const ChunkLists& L, const uint3
                 int pos = incl - cnt;
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
+                    // a word's bits from the top down into the end of its run: one leading-zero count per bit
+                    // (bit scans run on the quarter-rate unit; finding the lowest bit takes two of them)
                     uint32_t word = fw[q];
                     const uint32_t obase = (uint32_t)(lane * 128 + q * 32);
+                    pos += pc[q];
+                    int pe = pos;
                     while (word) {
-                        const int b = __ffs((int)word) - 1;
-                        word &= word - 1u;
-                        stage[pos++] = (uint16_t)(obase + (uint32_t)b);
+                        const int b = 31 - __clz((int)word);
+                        word ^= 1u << b;
+                        stage[--pe] = (uint16_t)(obase + (uint32_t)b);
                     }
                 }
                 __syncwarp();
@@ -1100,14 +1109,15 @@ cudaError_t launch_multipass(const float* scores, int64_t N, int64_t k, int64_t*
     const int64_t cap = (int64_t)sm_count() * 8;
     if (hb > cap) hb = cap;
     if (hb < 1) hb = 1;
-    select_hist_kernel<0><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, k, state, hist);
-    select_hist_kernel<1><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, k, state, hist + 2048);
-    select_hist_kernel<2><<<(unsigned)hb, SEL_T, 0, st>>>(scores, N, k, state, hist + 4096);
     const int64_t nblk = sel_nblk(N);
     const int64_t G = nblk < SEL_MAX_GRID ? nblk : SEL_MAX_GRID;
     const int64_t R = (nblk + G - 1) / G;
-    select_count_kernel<<<(unsigned)G, SEL_T, 0, st>>>(scores, N, nblk, R, G, state, blk_cnt, blk_tot);
-    select_write_kernel<<<(unsigned)G, SEL_T, 0, st>>>(scores, N, nblk, R, state, blk_cnt, blk_tot, indices, Gate{nullptr, 0u});
+    cudaError_t e;
+    if ((e = launch_after(select_hist_kernel<0>, (unsigned)hb, SEL_T, 0, st, scores, N, k, state, hist)) != cudaSuccess) return e;
+    if ((e = launch_after(select_hist_kernel<1>, (unsigned)hb, SEL_T, 0, st, scores, N, k, state, hist + 2048)) != cudaSuccess) return e;
+    if ((e = launch_after(select_hist_kernel<2>, (unsigned)hb, SEL_T, 0, st, scores, N, k, state, hist + 4096)) != cudaSuccess) return e;
+    if ((e = launch_after(select_count_kernel, (unsigned)G, SEL_T, 0, st, scores, N, nblk, R, G, state, blk_cnt, blk_tot)) != cudaSuccess) return e;
+    if ((e = launch_after(select_write_kernel, (unsigned)G, SEL_T, 0, st, scores, N, nblk, R, state, blk_cnt, blk_tot, indices, Gate{nullptr, 0u})) != cudaSuccess) return e;
     count_launches(5);
     return cudaGetLastError();
 }
