@@ -25,9 +25,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 # DRAM bytes of one projection launch per projected coordinate (dram__bytes_read.sum + dram__bytes_write.sum of
-# project_tc_kernel): one ncu capture at n = 256, d = 8192, P = 2^20 gave 734.2 MB + 120.3 MB; both parts grow in
+# project_tc_kernel): one ncu capture at n = 256, d = 8192, P = 2^20 gave 735.7 MB + 120.0 MB; both parts grow in
 # proportion to P (the Gamma batch read, and one fp32 partial per 65 536-coordinate chunk written).
-PROJECT_TRAFFIC_BYTES_PER_P = (734.219520e6 + 120.312064e6) / 1048576.0
+PROJECT_TRAFFIC_BYTES_PER_P = (735.706624e6 + 120.043008e6) / 1048576.0
 PROJECT_TRAFFIC_SOURCE = "ncu capture at n=256, d=8192, P=2^20, scaled by P (profiles/project_tc_kernel__n256_P2e20_d8192.md)"
 WORKLOAD = "c2_project_quantize"
 N_VAL, TASKS, FRAC = 448, [64, 128, 256], 0.05
@@ -539,7 +539,7 @@ def stage_measurements(torch, B, W, dev, peaks):
     s = torch.randn(N, device=dev)
     idx = torch.empty(N // 16, dtype=torch.int64, device=dev)
     wsel = torch.empty(B.qless_select_topk_workspace(N), dtype=torch.uint8, device=dev)
-    t = _time_ms(torch, lambda: B.qless_select_topk(s, 0.05, indices=idx, workspace=wsel), 3)
+    t = _time_ms(torch, lambda: B.qless_select_topk(s, 0.05, indices=idx, workspace=wsel), 20, warm=2)
     out["select_2^28_top5pct"] = dict(ms=t, gbs_algorithmic=4.0 * N / t / 1e6, frac_of_hbm=4.0 * N / t / 1e6 / peaks["hbm_gbs"],
                                       note="algorithmic bytes = 4N (every score read once)")
     del s, idx, wsel

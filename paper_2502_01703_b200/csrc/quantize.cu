@@ -139,7 +139,7 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
                 if (BITS == 1) {
                     uint32_t nib = 0;
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) nib |= (S > 0.0f && e[u] < 0.0f) ? (1u << u) : 0u;
+                    for (int u = 0; u < 4; ++u) nib |= (e[u] < 0.0f) ? (1u << u) : 0u;     // a zero vector (S = 0) has no negative entry
                     ss += (S > 0.0f) ? 4 : 0;
                     // eight lanes' nibbles -> one 32-bit word (three butterfly steps), stored by every eighth lane: whole
                     // words, no byte stores of neighbouring lanes into the same bank
