@@ -39,6 +39,7 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
     __shared__ double s_d[QT / 32];
     __shared__ float s_f[QT / 32];
     __shared__ int s_i[QT / 32];
+    __shared__ float s_par[3];            // the row's scalars: 1 / norm, scale S, multiplier of Eq. 5
     __shared__ __align__(16) uint8_t s_out[8192];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -90,24 +91,33 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
         mx = warp_max(mx);
         if (lane == 0) { s_d[warp] = acc; s_f[warp] = mx; }
         __syncthreads();
-        double tot = 0.0;
-        float S = 0.0f;
+        // One thread finishes the reduction and derives the row's scalars (the fp64 square root and the two IEEE
+        // divisions are long instruction sequences: done by all 256 threads they were a tenth of the kernel's
+        // instructions); the others pick them up behind a barrier.
+        constexpr int ALPHA = (BITS == 1) ? 1 : ((1 << (BITS - 1)) - 1);
+        if (tid == 0) {
+            double tot = 0.0;
+            float S0 = 0.0f;
 #pragma unroll
-        for (int w = 0; w < QT / 32; ++w) { tot += s_d[w]; S = fmaxf(S, s_f[w]); }
-        float rn = 1.0f;
-        if (normalize) {
-            const float nrm = (float)sqrt(tot);
-            if (nrm == 0.0f) {
-                S = 0.0f;                               // zero vector
-            } else {
-                rn = __fdiv_rn(1.0f, nrm);
-                S = __fmul_rn(S, rn);
+            for (int w = 0; w < QT / 32; ++w) { tot += s_d[w]; S0 = fmaxf(S0, s_f[w]); }
+            float rn0 = 1.0f;
+            if (normalize) {
+                const float nrm = (float)sqrt(tot);
+                if (nrm == 0.0f) {
+                    S0 = 0.0f;                              // zero vector
+                } else {
+                    rn0 = __fdiv_rn(1.0f, nrm);
+                    S0 = __fmul_rn(S0, rn0);
+                }
             }
+            s_par[0] = rn0; s_par[1] = S0;
+            s_par[2] = (S0 > 0.0f) ? __fdiv_rn((float)ALPHA, S0) : 0.0f;       // Eq. 5: alpha / S
         }
+        __syncthreads();
+        const float rn = s_par[0];
+        float S = s_par[1], r = s_par[2];
 
         // ---- Eq. 5 + pack into shared memory ----
-        constexpr int ALPHA = (BITS == 1) ? 1 : ((1 << (BITS - 1)) - 1);
-        float r = (S > 0.0f) ? __fdiv_rn((float)ALPHA, S) : 0.0f;
         if (ABSMEAN) {
             // gamma = mean |yhat| (sum in double), Delta = gamma * c_b (c_2 = 1, c_4 = 1/2, c_8 = 1/32),
             // q = clamp(rne(yhat / Delta), -alpha, alpha); the stored scale alpha * Delta dequantises like an absmax one
@@ -118,17 +128,20 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
                 sa += (double)fabsf(__fmul_rn(x[k].z, rn)); sa += (double)fabsf(__fmul_rn(x[k].w, rn));
             }
             sa = warp_sum(sa);
-            __syncthreads();                 // everyone has read s_d of the first reduction
-            if (lane == 0) s_d[warp] = sa;
+            if (lane == 0) s_d[warp] = sa;       // s_d of the first reduction was read before the barrier above
             __syncthreads();
-            double ta = 0.0;
+            if (tid == 0) {
+                double ta = 0.0;
 #pragma unroll
-            for (int w = 0; w < QT / 32; ++w) ta += s_d[w];
-            const float gamma = (float)(ta / (double)d);
-            constexpr float CB = (BITS == 2) ? 1.0f : (BITS == 4) ? 0.5f : 0.03125f;
-            const float delta = __fmul_rn(gamma, CB);
-            r = (gamma > 0.0f) ? __fdiv_rn(1.0f, delta) : 0.0f;
-            S = (gamma > 0.0f) ? __fmul_rn((float)ALPHA, delta) : 0.0f;
+                for (int w = 0; w < QT / 32; ++w) ta += s_d[w];
+                const float gamma = (float)(ta / (double)d);
+                constexpr float CB = (BITS == 2) ? 1.0f : (BITS == 4) ? 0.5f : 0.03125f;
+                const float delta = __fmul_rn(gamma, CB);
+                s_par[2] = (gamma > 0.0f) ? __fdiv_rn(1.0f, delta) : 0.0f;
+                s_par[1] = (gamma > 0.0f) ? __fmul_rn((float)ALPHA, delta) : 0.0f;
+            }
+            __syncthreads();
+            S = s_par[1]; r = s_par[2];
         }
         int ss = 0;
 #pragma unroll
@@ -140,13 +153,8 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
                     uint32_t nib = 0;
 #pragma unroll
                     for (int u = 0; u < 4; ++u) nib |= (e[u] < 0.0f) ? (1u << u) : 0u;     // a zero vector (S = 0) has no negative entry
-                    ss += (S > 0.0f) ? 4 : 0;
-                    // eight lanes' nibbles -> one 32-bit word (three butterfly steps), stored by every eighth lane: whole
-                    // words, no byte stores of neighbouring lanes into the same bank
-                    uint32_t w = nib | (__shfl_down_sync(0xFFFFFFFFu, nib, 1) << 4);
-                    w |= __shfl_down_sync(0xFFFFFFFFu, w, 2) << 8;
-                    w |= __shfl_down_sync(0xFFFFFFFFu, w, 4) << 16;
-                    if ((lane & 7) == 0) reinterpret_cast<uint32_t*>(s_out)[c >> 3] = w;
+                    const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, nib, 1);
+                    if ((lane & 1) == 0) s_out[c >> 1] = (uint8_t)(nib | (hi << 4));
                 } else {
                     // round-half-even to an integer by adding 1.5 * 2^23: the sum's low mantissa bits are the
                     // two's-complement code (|yhat r| <= alpha (1 + 2^-23), so no clamp is needed)
@@ -175,13 +183,18 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
                 }
             }
         }
-        ss = warp_sum_i(ss);
-        if (lane == 0) s_i[warp] = ss;
+        if (BITS > 1) {
+            ss = warp_sum_i(ss);
+            if (lane == 0) s_i[warp] = ss;
+        }
         __syncthreads();       // s_out and s_i complete
         if (tid == 0) {
-            int tot = 0;
+            int tot = (S > 0.0f) ? d : 0;         // sign codes: every q^2 is 1, unless the vector is the zero vector
+            if (BITS > 1) {
+                tot = 0;
 #pragma unroll
-            for (int w = 0; w < QT / 32; ++w) tot += s_i[w];
+                for (int w = 0; w < QT / 32; ++w) tot += s_i[w];
+            }
             scales[row] = S;
             if (sumsq) sumsq[row] = tot;
         }
