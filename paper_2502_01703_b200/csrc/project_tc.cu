@@ -10,7 +10,8 @@
 // Gamma ([P/64][n][64], so that each 128 x 64 operand tile is one contiguous 16 KiB span) into
 // 128-byte-swizzled shared memory: pairing halves the bytes every SM pulls from L2 and the shared-memory
 // traffic of the gradient operand. In each CTA the accumulator (128 x 256 fp32) occupies TMEM columns
-// 0..255 and four 128-deep stages of the sign operand occupy columns 256..511. Pairs are persistent and
+// 0..255 and two 256-deep stages of the sign operand occupy columns 256..511 (one barrier round of the MMA-issuing
+// thread covers 256 columns of both operands: 16 MMAs per two waits and two commits). Pairs are persistent and
 // walk work items (gradient tile, K-chunk, r tile) K-chunk-major, so that at any time all pairs read the
 // same slab of Gamma (L2 reuse); after each K-chunk the accumulator is drained to a per-chunk partial,
 // which bounds the length of any fp32 accumulation chain and makes the final sum order fixed.
@@ -32,7 +33,7 @@ constexpr int BM = 128;                 // projected coordinates per CTA (UMMA M
 constexpr int BN = 256;                 // gradient rows per tile (UMMA N), 128 of them staged by each CTA
 constexpr int BK = 256;                 // K per shared-memory stage: four 64-column (128-byte) swizzle panels
 constexpr int SB = 3;                   // shared-memory stages of the gradient operand
-constexpr int SA = 4;                   // TMEM stages of the sign operand, 128 K each (64 columns)
+constexpr int SA = 2;                   // TMEM stages of the sign operand, 256 K each (128 columns): one per generator group
 constexpr int B_PANEL_BYTES = (BN / 2) * 64 * 2;      // 16 KiB: 128 rows x 64 columns
 constexpr int B_STAGE_BYTES = (BK / 64) * B_PANEL_BYTES;      // 64 KiB per CTA
 constexpr int TMEM_COLS = 512;
@@ -132,7 +133,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
     } else if (warp == 1) {
         // ------------------------------- MMA issuer -------------------------------
         if (lane == 0 && rank == 0) {
-            uint32_t itb = 0, ita = 0, n_item = 0;
+            uint32_t itb = 0, n_item = 0;
             bool ok = true;
             for (int64_t item = pair; item < num_items && ok; item += num_pairs, ++n_item) {
                 const int kc = (int)((item / num_dt) % num_chunks);
@@ -144,20 +145,20 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 for (int kb = 0; kb < nkb; ++kb, ++itb) {
                     const int sb = itb % SB;
                     if (!mbar_wait(smem_u32(&bars->b_full[sb]), (itb / SB) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
+                    // the sign operand of the same 256 columns (a chunk may end on half a stage: 8 MMAs instead of 16)
                     const int nh = (int)min((int64_t)(BK / 128), (klen - (int64_t)kb * BK) >> 7);
-                    for (int h = 0; h < nh && ok; ++h, ++ita) {                // one 128-deep sign stage at a time
-                        const int sa = ita % SA;
-                        if (!mbar_wait(smem_u32(&bars->a_full[sa]), (ita / SA) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
-                        tc_fence_after();
-                        const uint32_t a_addr = tmem_base + A_COL + sa * 64;
+                    const int sa = itb % SA;
+                    if (!mbar_wait(smem_u32(&bars->a_full[sa]), (itb / SA) & 1u, abort_flag, timeout_word, TO_MMA)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = tmem_base + A_COL + sa * 128;
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            const uint64_t bdesc = make_smem_desc_sw128(smem_u32(smem + (size_t)sb * B_STAGE_BYTES + (2 * h + (k >> 2)) * B_PANEL_BYTES));
-                            mma_f16_ts_pair(tmem_base + D_COL, a_addr + k * 8, bdesc + (uint64_t)((k & 3) * 2), IDESC, (kb > 0 || h > 0 || k > 0) ? 1u : 0u);
+                    for (int k = 0; k < 16; ++k) {
+                        if (k < 8 * nh) {
+                            const uint64_t bdesc = make_smem_desc_sw128(smem_u32(smem + (size_t)sb * B_STAGE_BYTES + (k >> 2) * B_PANEL_BYTES));
+                            mma_f16_ts_pair(tmem_base + D_COL, a_addr + k * 8, bdesc + (uint64_t)((k & 3) * 2), IDESC, (kb > 0 || k > 0) ? 1u : 0u);
                         }
-                        mma_commit_pair(smem_u32(&bars->a_empty[sa]));
                     }
-                    if (!ok) break;
+                    mma_commit_pair(smem_u32(&bars->a_empty[sa]));
                     mma_commit_pair(smem_u32(&bars->b_empty[sb]));
                 }
                 if (ok) mma_commit_pair(smem_u32(&bars->d_full));
@@ -170,8 +171,8 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
         }
     } else if (warp < 6 || warp >= 10) {
         // ------------------------------- sign generators -------------------------------
-        // two groups of four warps (2-5 and 10-13) take alternate 128-deep stages, so that the latency of one
-        // stage (Philox chain, TMEM store, barrier round trip) overlaps the next
+        // two groups of four warps (2-5 and 10-13) take alternate 256-deep stages (each group owns one of the two
+        // TMEM stages), so that the latency of one stage (Philox chains, TMEM stores, barrier round trip) overlaps the next
         const int q = warp & 3;                                  // TMEM lane quadrant this warp may access
         const uint32_t grp = (warp >= 10) ? 1u : 0u;
         uint32_t ita = 0;
@@ -180,39 +181,54 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
             const int dt = (int)(item % num_dt) * 2 + (int)rank;           // this CTA's 128 projected coordinates
             const int kc = (int)((item / num_dt) % num_chunks);
             const int64_t k0 = (int64_t)kc * chunk;
-            const int nka = (int)((min(P, k0 + chunk) - k0) / 128);
+            const int64_t klen = min(P, k0 + chunk) - k0;                  // multiple of 128
+            const int nka = (int)((klen + BK - 1) / BK);                   // 256-deep stages of the chunk
             const uint32_t r = (uint32_t)(dt * BM + q * 32 + lane);
             for (int ka = 0; ka < nka; ++ka, ++ita) {
                 if ((ita & 1u) != grp) continue;
-                const int sa = ita % SA;
-                const uint32_t blk = kblk_base + (uint32_t)((k0 >> 7) + ka);      // 128-column block of the matrix
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + A_COL + sa * 64;
+                const int sa = ita % SA;                                   // = grp: each group owns one stage
+                const int nh = (int)min((int64_t)2, (klen - (int64_t)ka * BK) >> 7);      // halves of 128 columns (a chunk may end on one)
+                const uint32_t blk = kblk_base + (uint32_t)((k0 >> 7) + 2 * ka);          // first 128-column block of the stage
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + A_COL + sa * 128;
                 if constexpr (GAUSS) {
-                    uint32_t v[4][16];                                            // generated before the slot is waited for
+#pragma unroll 1
+                    for (int h = 0; h < nh; ++h) {
+                        const uint32_t bh = blk + (uint32_t)h;
+                        uint32_t v[4][16];                                        // generated before the slot is waited for
 #pragma unroll
-                    for (int wi = 0; wi < 4; ++wi)
+                        for (int wi = 0; wi < 4; ++wi)
 #pragma unroll
-                        for (int c = 0; c < 8; ++c)
-                            gaussian_quad_bf16x2(seed, r, (blk << 5) | (uint32_t)(wi * 8 + c), blk >> 27, v[wi][2 * c], v[wi][2 * c + 1]);
-                    ok = mbar_wait_cluster(smem_u32(&bars->a_empty[sa]), ((ita / SA) & 1u) ^ 1u, abort_flag, timeout_word, TO_GENERATOR);
-                    ok = __all_sync(0xFFFFFFFFu, ok);
+                            for (int c = 0; c < 8; ++c)
+                                gaussian_quad_bf16x2(seed, r, (bh << 5) | (uint32_t)(wi * 8 + c), bh >> 27, v[wi][2 * c], v[wi][2 * c + 1]);
+                        if (h == 0) {
+                            ok = mbar_wait_cluster(smem_u32(&bars->a_empty[sa]), ((ita / SA) & 1u) ^ 1u, abort_flag, timeout_word, TO_GENERATOR);
+                            ok = __all_sync(0xFFFFFFFFu, ok);
+                            if (!ok) break;
+                            tc_fence_after();
+                        }
+#pragma unroll
+                        for (int wi = 0; wi < 4; ++wi) tmem_st_x16(taddr + h * 64 + wi * 16, v[wi]);
+                    }
                     if (!ok) break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int wi = 0; wi < 4; ++wi) tmem_st_x16(taddr + wi * 16, v[wi]);
                 } else {
-                    uint32_t w[4];
-                    rademacher_block(seed, r, blk, w);     // overlaps with the wait below
+                    uint32_t w[2][4];
+                    rademacher_block(seed, r, blk, w[0]);     // overlaps with the wait below
+                    if (nh == 2) rademacher_block(seed, r, blk + 1u, w[1]);
                     ok = mbar_wait_cluster(smem_u32(&bars->a_empty[sa]), ((ita / SA) & 1u) ^ 1u, abort_flag, timeout_word, TO_GENERATOR);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll
-                    for (int wi = 0; wi < 4; ++wi) {
-                        uint32_t v[16];
+                    for (int h = 0; h < 2; ++h) {
+                        if (h < nh) {
 #pragma unroll
-                        for (int p = 0; p < 16; ++p) v[p] = rademacher_bf16x2(w[wi], p);
-                        tmem_st_x16(taddr + wi * 16, v);
+                            for (int wi = 0; wi < 4; ++wi) {
+                                uint32_t v[16];
+#pragma unroll
+                                for (int p = 0; p < 16; ++p) v[p] = rademacher_bf16x2(w[h][wi], p);
+                                tmem_st_x16(taddr + h * 64 + wi * 16, v);
+                            }
+                        }
                     }
                 }
                 tmem_wait_st();
