@@ -126,7 +126,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_STAGES; ++s) {
             // leader's full[s]: the producer's expect_tx arrival (+ one arrival per unpack warp of both CTAs)
-            mbar_init(smem_u32(&bars->full[s]), DIRECT ? 1 : 9);
+            // (8-bit codes and bf16 rows: one barrier per PAIR of stages, at the even slot, collects both stages' arrivals,
+            // so that the MMA-issuing thread waits once per 16 MMAs)
+            mbar_init(smem_u32(&bars->full[s]), DIRECT ? 2 : 9);
             mbar_init(smem_u32(&bars->empty[s]), 1);
             mbar_init(smem_u32(&bars->p_full[s]), 1);
             mbar_init(smem_u32(&bars->p_empty[s]), 4);
@@ -191,8 +193,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                             }
                             const int s = (int)st_ring.slot;
                             if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), st_ring.parity ^ 1u, abort_flag, p.timeout_word, TO_PRODUCER)) { ok = false; break; }
-                            const uint32_t full = map_to_cta(smem_u32(&bars->full[s]), 0);
-                            if (rank == 0) mbar_arrive_expect_tx(smem_u32(&bars->full[s]), tx_total);
+                            const int fs = DIRECT ? (s & ~1) : s;                 // the pair's barrier
+                            const uint32_t full = map_to_cta(smem_u32(&bars->full[fs]), 0);
+                            if (rank == 0) mbar_arrive_expect_tx(smem_u32(&bars->full[fs]), tx_total);
                             uint8_t* st = sS + (size_t)s * stage_bytes;
                             if (DIRECT) tma_load_3d_pair(smem_u32(st), &tmap_train, full, kb * KB, row0, i);
                             // this CTA's rows of the validation operand of each MMA half
@@ -201,6 +204,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                                 tma_load_3d_pair(smem_u32(st + A_SMEM + bh1), &tmap_val2, full, kb * KB, vt * p.vpad + p.n1 + (int)rank * (p.n2 / 2), i);
                         }
             }
+            // an odd number of stages in all: the last pair's barrier still lacks its second arrival
+            if (DIRECT && ok && (it & 1u) && rank == 0) mbar_arrive(smem_u32(&bars->full[st_ring.slot & ~1u]));
             if (!ok) {
                 // Leave no copy in flight behind us. Packed loads 0 .. pq-1 have been issued into this CTA's own ring
                 // (barriers of its own: wait, bounded, for the phases of the last nP of them). Operand stages 0 .. it-1
@@ -212,7 +217,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         if (!mbar_wait_quiet(smem_u32(&bars->p_full[j % p.nP]), (uint32_t)(j / p.nP) & 1u)) break;
                 if (rank == 0) {
                     for (uint32_t j = (it > (uint32_t)p.nS ? it - (uint32_t)p.nS : 0u); j < it; ++j)
-                        if (!mbar_wait_quiet(smem_u32(&bars->full[j % (uint32_t)p.nS]), (j / (uint32_t)p.nS) & 1u, 1u << 14)) break;
+                        if (!mbar_wait_quiet(smem_u32(&bars->full[(j % (uint32_t)p.nS) & (DIRECT ? ~1u : ~0u)]), (j / (uint32_t)p.nS) & 1u, 1u << 14)) break;
                 } else {
                     for (uint32_t t = 0; t < (1u << 14); ++t) __nanosleep(64);
                 }
@@ -230,8 +235,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         if (!mbar_wait_cluster(smem_u32(&bars->d_empty), (n_acc & 1u) ^ 1u, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
                         for (int kb = 0; kb < nkb; ++kb, ++it, st_ring.next((uint32_t)p.nS)) {
                             const int s = (int)st_ring.slot;
-                            if (!mbar_wait(smem_u32(&bars->full[s]), st_ring.parity, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
-                            tc_fence_after();
+                            if (!DIRECT || (s & 1) == 0) {       // DIRECT: the barrier at the even slot covers this stage and the next
+                                if (!mbar_wait(smem_u32(&bars->full[s]), st_ring.parity, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
+                                tc_fence_after();
+                            }
                             const uint32_t st = smem_u32(sS + (size_t)s * stage_bytes);
                             const uint64_t adesc = make_smem_desc_sw128(st);
                             const uint64_t bdesc1 = make_smem_desc_sw128(st + A_SMEM);
@@ -507,6 +514,7 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     int nP = a.bits >= 8 ? 0 : 4;
     int nS = (int)((budget - (size_t)nP * p_stage) / stage);
     if (nS > MAX_STAGES) nS = MAX_STAGES;
+    if (a.bits >= 8) nS &= ~1;                              // stages are handed to the MMAs in pairs
     QLESS_REQUIRE(nS >= 3, QLESS_ERR_UNSUPPORTED, "internal: not enough shared memory for two pipeline stages");
     p.nS = nS; p.nP = nP > 0 ? nP : 1;
     p.epi_groups = (a.bits >= 8 && a.T <= 6) ? 2 : 1;
