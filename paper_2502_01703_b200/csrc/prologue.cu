@@ -8,30 +8,36 @@ namespace qless {
 // bm = fl(b1 m), bv = fl(b2 v) are passed in because they are the same for every row of the batch.
 //
 // The IEEE square root and division are the expensive part, and the result only keeps 8 bits. So the
-// quotient is first formed with the approximate reciprocal units (a few ulp of error); unless that value
+// quotient is first formed with the approximate reciprocal-square-root unit (a few ulp of error); unless that value
 // lies close to a bf16 rounding boundary (or outside the normal range) its bf16 rounding is already the one
 // the exact sequence gives, and the exact sequence runs only for the rare remaining elements. The value
 // returned always rounds to the same bf16 as the exact one.
 __device__ __forceinline__ float adam_dir(float g, float bm, float bv, const AdamParams& ap)
 {
     float m1 = __fadd_rn(bm, __fmul_rn(ap.omb1, g));
-    float v1 = __fadd_rn(bv, __fmul_rn(ap.omb2, __fmul_rn(g, g)));
     if (!ap.bias_correct) {
-        float rs, rc;
-        asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rs) : "f"(v1));
-        const float den_a = __fadd_rn(__fmul_rn(v1, rs), ap.eps);          // v1 = 0 gives NaN: handled below
-        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(den_a));
-        const float q = __fmul_rn(m1, rc);
-        // Safe if q is well inside the normal range (biased exponent in [28, 226]: zeros, subnormals, infinities
-        // and NaNs all fall outside; so does every case in which den_a or its reciprocal left the normal range,
-        // since q is then 0, infinite or NaN) and its low 16 bits are more than 32 away from the bf16 tie 0x8000.
+        // Fast path, about 16 instructions and one special-function operation per element (the kernel is bound by
+        // instruction issue, then by that unit at 16 lanes per clock per SM). v' is a sum of non-negative terms, so
+        // forming it with one fused multiply-add moves it by an ulp; m' may cancel and keeps the exact roundings.
+        // With rs = 1 / sqrt(v'), 1 / (sqrt(v') + eps) = rs / (1 + t), t = eps rs, and for t < 2^-8 the series
+        // 1 - t + t^2 is within t^3 < 2^-24 of 1 / (1 + t). All roundings and the unit's error (2^-22.9) add up to
+        // less than 7 fp32 ulps between this quotient and the exact sequence's, 13 steps of its significand.
+        const float v1f = fmaf(ap.omb2, __fmul_rn(g, g), bv);
+        float rs;
+        asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rs) : "f"(v1f));
+        const float t = ap.eps * rs;
+        const float q = (m1 * rs) * fmaf(t, t, 1.0f - t);
+        // Safe if t is small (a larger one, v' tiny or zero, rs huge or infinite, t possibly NaN, fails the test), q
+        // is well inside the normal range (biased exponent in [28, 226]: zeros, subnormals, infinities and NaNs all
+        // fall outside; so does every case in which rs or a product left the normal range, since q is then 0,
+        // infinite or NaN) and its low 16 bits are more than 32 away from the bf16 tie 0x8000.
         const uint32_t qb = __float_as_uint(q);
-        const bool in_range = (((qb >> 23) & 0xFFu) - 28u) <= 198u;
-        const bool off_tie = ((qb - 0x7FE0u) & 0xFFFFu) > 0x40u;
-        if (in_range && off_tie) return q;
-    } else {
-        m1 = __fdiv_rn(m1, ap.c1); v1 = __fdiv_rn(v1, ap.c2);
+        const bool in_range = (qb * 2u - (28u << 24)) <= ((198u << 24) | 0xFFFFFFu);
+        const bool off_tie = ((qb << 16) - (0x7FE0u << 16)) > (0x40u << 16);
+        if (t < 0.00390625f && in_range && off_tie) return q;
     }
+    float v1 = __fadd_rn(bv, __fmul_rn(ap.omb2, __fmul_rn(g, g)));
+    if (ap.bias_correct) { m1 = __fdiv_rn(m1, ap.c1); v1 = __fdiv_rn(v1, ap.c2); }
     const float den = __fadd_rn(__fsqrt_rn(v1), ap.eps);
     return __fdiv_rn(m1, den);
 }

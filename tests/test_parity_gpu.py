@@ -93,6 +93,21 @@ def test_adam_gamma_bit_exact_on_many_elements():
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
 
 
+@pytest.mark.parametrize("v_scale,eps", [(1e-12, 1e-8), (1e-10, 1e-8), (1e-14, 1e-8), (1e-6, 0.0), (1e-6, 1e-3), (1e-30, 1e-8)])
+def test_adam_gamma_bit_exact_across_eps_over_sqrt_v(v_scale, eps):
+    # eps / sqrt(v') from far below to far above the bound under which the kernel's one-unit fast path is used:
+    # both sides of that bound, and the elements next to it, must round to the oracle's bf16
+    n, P = 16, 1 << 16
+    g = W.student_t_gradients(n, P, seed=15, device=DEV, dtype=torch.bfloat16) * (v_scale ** 0.5 * 30)
+    m, v = W.adam_moments(P, seed=16, device=DEV)
+    v = v * (v_scale / 1e-6)
+    v *= torch.logspace(-2, 2, P, device=DEV)                   # four decades of v across the coordinates
+    cfg = dict(beta1=0.9, beta2=0.999, eps=eps, step=0)
+    got = _np(B.qless_adam_gamma(g, m, v, cfg).float())
+    want = oracle.adam_gamma(_np(g.float()), _np(m), _np(v), **cfg)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
 def test_adam_gamma_strided_rows_and_extreme_values():
     n, P = 3, 256
     big = torch.zeros((n, P + 64), dtype=torch.float32, device=DEV)
