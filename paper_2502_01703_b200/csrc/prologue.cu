@@ -10,36 +10,57 @@ namespace qless {
 // The IEEE square root and division are the expensive part, and the result only keeps 8 bits. So the
 // quotient is first formed with the approximate reciprocal-square-root unit (a few ulp of error); unless that value
 // lies close to a bf16 rounding boundary (or outside the normal range) its bf16 rounding is already the one
-// the exact sequence gives, and the exact sequence runs only for the rare remaining elements. The value
-// returned always rounds to the same bf16 as the exact one.
-__device__ __forceinline__ float adam_dir(float g, float bm, float bv, const AdamParams& ap)
+// the exact sequence gives, and the exact sequence runs only for the rare remaining elements.
+
+// The exact sequence. Not inlined: it is long, runs for about one element in a thousand, and the kernel holds 32
+// call sites. c1 = c2 = 1 without bias correction (a division by 1 is exact).
+__device__ __noinline__ float adam_dir_exact(float g, float bm, float bv, float omb1, float omb2, float eps, float c1, float c2)
 {
-    float m1 = __fadd_rn(bm, __fmul_rn(ap.omb1, g));
-    if (!ap.bias_correct) {
-        // Fast path, about 16 instructions and one special-function operation per element (the kernel is bound by
-        // instruction issue, then by that unit at 16 lanes per clock per SM). v' is a sum of non-negative terms, so
-        // forming it with one fused multiply-add moves it by an ulp; m' may cancel and keeps the exact roundings.
-        // With rs = 1 / sqrt(v'), 1 / (sqrt(v') + eps) = rs / (1 + t), t = eps rs, and for t < 2^-8 the series
-        // 1 - t + t^2 is within t^3 < 2^-24 of 1 / (1 + t). All roundings and the unit's error (2^-22.9) add up to
-        // less than 7 fp32 ulps between this quotient and the exact sequence's, 13 steps of its significand.
-        const float v1f = fmaf(ap.omb2, __fmul_rn(g, g), bv);
-        float rs;
-        asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rs) : "f"(v1f));
-        const float t = ap.eps * rs;
-        const float q = (m1 * rs) * fmaf(t, t, 1.0f - t);
-        // Safe if t is small (a larger one, v' tiny or zero, rs huge or infinite, t possibly NaN, fails the test), q
-        // is well inside the normal range (biased exponent in [28, 226]: zeros, subnormals, infinities and NaNs all
-        // fall outside; so does every case in which rs or a product left the normal range, since q is then 0,
-        // infinite or NaN) and its low 16 bits are more than 32 away from the bf16 tie 0x8000.
-        const uint32_t qb = __float_as_uint(q);
-        const bool in_range = (qb * 2u - (28u << 24)) <= ((198u << 24) | 0xFFFFFFu);
-        const bool off_tie = ((qb << 16) - (0x7FE0u << 16)) > (0x40u << 16);
-        if (t < 0.00390625f && in_range && off_tie) return q;
-    }
-    float v1 = __fadd_rn(bv, __fmul_rn(ap.omb2, __fmul_rn(g, g)));
-    if (ap.bias_correct) { m1 = __fdiv_rn(m1, ap.c1); v1 = __fdiv_rn(v1, ap.c2); }
-    const float den = __fadd_rn(__fsqrt_rn(v1), ap.eps);
+    float m1 = __fadd_rn(bm, __fmul_rn(omb1, g));
+    float v1 = __fadd_rn(bv, __fmul_rn(omb2, __fmul_rn(g, g)));
+    if (c1 != 1.0f || c2 != 1.0f) { m1 = __fdiv_rn(m1, c1); v1 = __fdiv_rn(v1, c2); }
+    const float den = __fadd_rn(__fsqrt_rn(v1), eps);
     return __fdiv_rn(m1, den);
+}
+
+// Fast path (no bias correction): one special-function operation per element (the kernel is bound by instruction
+// issue, then by that unit at 16 lanes per clock per SM). v' is a sum of non-negative terms, so forming it with one
+// fused multiply-add moves it by an ulp; m' may cancel and keeps the exact roundings. With rs = 1 / sqrt(v'),
+// 1 / (sqrt(v') + eps) = rs / (1 + t), t = eps rs, and for t < 2^-8 the series 1 - t + t^2 is within t^3 < 2^-24 of
+// 1 / (1 + t): q = u - u (t - t^2), u = m' rs. All roundings and the unit's error (2^-22.9) add up to less than 7 fp32
+// ulps between this quotient and the exact sequence's, 13 steps of its significand.
+// ok: t is small (a larger one, v' tiny or zero, rs huge or infinite, t possibly NaN, fails the test), q is well inside
+// the normal range (biased exponent in [28, 226]: zeros, subnormals, infinities and NaNs all fall outside; so does
+// every case in which rs or a product left the normal range, since q is then 0, infinite or NaN) and its low 16 bits
+// are more than 32 away from the bf16 tie 0x8000. Then q rounds to the same bf16 as the exact quotient.
+__device__ __forceinline__ float adam_dir_fast(float g, float bm, float bv, const AdamParams& ap, bool& ok)
+{
+    const float m1 = __fadd_rn(bm, __fmul_rn(ap.omb1, g));
+    const float v1f = fmaf(ap.omb2, __fmul_rn(g, g), bv);
+    float rs;
+    asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rs) : "f"(v1f));
+    const float t = ap.eps * rs;
+    const float u = m1 * rs;
+    const float q = fmaf(-u, fmaf(-t, t, t), u);
+    const uint32_t qb = __float_as_uint(q);
+    const bool in_range = (qb * 2u - (28u << 24)) <= ((198u << 24) | 0xFFFFFFu);
+    const bool off_tie = ((qb << 16) - (0x7FE0u << 16)) > (0x40u << 16);
+    ok = t < 0.00390625f && in_range && off_tie;
+    return q;
+}
+
+// Two neighbouring elements share one branch to the exact sequence.
+__device__ __forceinline__ void adam_dir2(float& g0, float& g1, float bm0, float bm1, float bv0, float bv1, const AdamParams& ap)
+{
+    bool ok0 = false, ok1 = false;
+    float q0 = 0.0f, q1 = 0.0f;
+    if (!ap.bias_correct) { q0 = adam_dir_fast(g0, bm0, bv0, ap, ok0); q1 = adam_dir_fast(g1, bm1, bv1, ap, ok1); }
+    if (!(ok0 && ok1)) {
+        const float c1 = ap.bias_correct ? ap.c1 : 1.0f, c2 = ap.bias_correct ? ap.c2 : 1.0f;
+        if (!ok0) q0 = adam_dir_exact(g0, bm0, bv0, ap.omb1, ap.omb2, ap.eps, c1, c2);
+        if (!ok1) q1 = adam_dir_exact(g1, bm1, bv1, ap.omb1, ap.omb2, ap.eps, c1, c2);
+    }
+    g0 = q0; g1 = q1;
 }
 
 // One thread handles 8 consecutive columns (16-byte bf16 accesses); AG_ROWS is the number of consecutive
@@ -105,7 +126,7 @@ adam_gamma_kernel(const void* __restrict__ grads, int64_t n, int64_t ld, const f
                 }
                 if (ADAM) {
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) g[k] = adam_dir(g[k], mm[k], vv[k], ap);
+                    for (int k = 0; k < 8; k += 2) adam_dir2(g[k], g[k + 1], mm[k], mm[k + 1], vv[k], vv[k + 1], ap);
                 }
                 uint32_t o[4];
 #pragma unroll
