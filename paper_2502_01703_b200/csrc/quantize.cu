@@ -15,23 +15,24 @@ __device__ __forceinline__ double warp_sum(double x)
     for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
     return x;
 }
+// x >= 0 and not NaN (a running fmaxf that starts at 0): such floats order like their bit patterns, so the
+// warp-wide integer maximum (one instruction) is their maximum.
 __device__ __forceinline__ float warp_max(float x)
 {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xFFFFFFFFu, x, o));
-    return x;
+    return __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(x)));
 }
 __device__ __forceinline__ int warp_sum_i(int x)
 {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
-    return x;
+    return __reduce_add_sync(0xFFFFFFFFu, x);
 }
 
 // ABSMEAN: the scale comes from the mean absolute value of the row instead of its maximum (see the absmean
-// branch below); BITS = 1 has no scale and is always instantiated with ABSMEAN = false.
-template <int BITS, bool ABSMEAN = false>
-__global__ void __launch_bounds__(QT, 5)
+// branch below); BITS = 1 has no scale and is always instantiated with ABSMEAN = false. FULL: d = 8192, every
+// thread owns eight whole float4 chunks and the per-chunk bounds tests compile away (the kernel is bound by
+// instruction issue: those tests and the per-chunk tests of the call's options were a tenth of its instructions).
+// MULTI: the row is the sum of num_parts > 1 partial rows (fewer resident blocks, more registers: eight loads in flight).
+template <int BITS, bool ABSMEAN = false, bool FULL = false, bool MULTI = false>
+__global__ void __launch_bounds__(QT, MULTI ? 3 : 5)
 quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale, int64_t n, int32_t d,
                 int normalize, uint8_t* __restrict__ codes, float* __restrict__ scales,
                 int32_t* __restrict__ sumsq, float* __restrict__ proj_out)
@@ -54,40 +55,70 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
                 asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(parts + s * part_stride + (row + gridDim.x) * d), "r"(d * 4) : "memory");
         }
         float4 x[QMAX_V4];
-        // ---- load + fixed-order sum of partials, scaled once ----
+        // ---- load + fixed-order sum of partials (part 0, 1, 2, ... for every element), scaled once ----
+        if (!MULTI) {
+            const float4* p = reinterpret_cast<const float4*>(parts + row * d) + tid;
 #pragma unroll
-        for (int k = 0; k < QMAX_V4; ++k) {
-            const int c = tid + k * QT;
-            float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (c < nv4) {
-                const float4* p = reinterpret_cast<const float4*>(parts + row * d) + c;
-                a = __ldcs(p);
-                for (int s = 1; s < num_parts; ++s) {
-                    const float4 b = __ldcs(reinterpret_cast<const float4*>(parts + s * part_stride + row * d) + c);
-                    a.x = __fadd_rn(a.x, b.x); a.y = __fadd_rn(a.y, b.y);
-                    a.z = __fadd_rn(a.z, b.z); a.w = __fadd_rn(a.w, b.w);
+            for (int k = 0; k < QMAX_V4; ++k)
+                x[k] = (FULL || tid + k * QT < nv4) ? __ldcs(p + k * QT) : make_float4(0.f, 0.f, 0.f, 0.f);
+        } else {
+            // many parts (the projection's K chunks), usually few rows: a thread keeps eight loads of one chunk's
+            // column in flight and adds them in part order
+            const int64_t ps4 = part_stride >> 2;
+#pragma unroll
+            for (int k = 0; k < QMAX_V4; ++k) {
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (FULL || tid + k * QT < nv4) {
+                    const float4* p = reinterpret_cast<const float4*>(parts + row * d) + tid + k * QT;
+                    a = __ldcs(p);
+                    int s = 1;
+                    for (; s + 8 <= num_parts; s += 8) {
+                        float4 b[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) b[u] = __ldcs(p + (s + u) * ps4);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            a.x = __fadd_rn(a.x, b[u].x); a.y = __fadd_rn(a.y, b[u].y);
+                            a.z = __fadd_rn(a.z, b[u].z); a.w = __fadd_rn(a.w, b[u].w);
+                        }
+                    }
+                    for (; s < num_parts; ++s) {
+                        const float4 b = __ldcs(p + s * ps4);
+                        a.x = __fadd_rn(a.x, b.x); a.y = __fadd_rn(a.y, b.y);
+                        a.z = __fadd_rn(a.z, b.z); a.w = __fadd_rn(a.w, b.w);
+                    }
                 }
-                if (scale != 1.0f) {
-                    a.x = __fmul_rn(a.x, scale); a.y = __fmul_rn(a.y, scale);
-                    a.z = __fmul_rn(a.z, scale); a.w = __fmul_rn(a.w, scale);
-                }
-                if (proj_out) __stcs(reinterpret_cast<float4*>(proj_out + row * d) + c, a);
+                x[k] = a;
             }
-            x[k] = a;
+        }
+        if (scale != 1.0f) {
+#pragma unroll
+            for (int k = 0; k < QMAX_V4; ++k) {
+                x[k].x = __fmul_rn(x[k].x, scale); x[k].y = __fmul_rn(x[k].y, scale);
+                x[k].z = __fmul_rn(x[k].z, scale); x[k].w = __fmul_rn(x[k].w, scale);
+            }
+        }
+        if (proj_out) {
+            float4* o = reinterpret_cast<float4*>(proj_out + row * d) + tid;
+#pragma unroll
+            for (int k = 0; k < QMAX_V4; ++k)
+                if (FULL || tid + k * QT < nv4) __stcs(o + k * QT, x[k]);
         }
         // ---- one block reduction for both Eq. 2 and Eq. 4: sum of squares (double) and max |x| of the raw row.
         // yhat_m = fl(x_m * rn) is monotone in |x_m|, so max_m |yhat_m| = fl(max_m |x_m| * rn) exactly.
         double acc = 0.0;
         float mx = 0.0f;
+        if (normalize) {
 #pragma unroll
-        for (int k = 0; k < QMAX_V4; ++k) {
-            if (normalize) {
+            for (int k = 0; k < QMAX_V4; ++k) {
                 acc += (double)x[k].x * (double)x[k].x; acc += (double)x[k].y * (double)x[k].y;
                 acc += (double)x[k].z * (double)x[k].z; acc += (double)x[k].w * (double)x[k].w;
             }
-            mx = fmaxf(fmaxf(mx, fmaxf(fabsf(x[k].x), fabsf(x[k].y))), fmaxf(fabsf(x[k].z), fabsf(x[k].w)));
+            acc = warp_sum(acc);
         }
-        if (normalize) acc = warp_sum(acc);
+#pragma unroll
+        for (int k = 0; k < QMAX_V4; ++k)
+            mx = fmaxf(fmaxf(mx, fmaxf(fabsf(x[k].x), fabsf(x[k].y))), fmaxf(fabsf(x[k].z), fabsf(x[k].w)));
         mx = warp_max(mx);
         if (lane == 0) { s_d[warp] = acc; s_f[warp] = mx; }
         __syncthreads();
@@ -147,7 +178,7 @@ quantize_kernel(const float* __restrict__ parts, int32_t num_parts, float scale,
 #pragma unroll
         for (int k = 0; k < QMAX_V4; ++k) {
             const int c = tid + k * QT;
-            if (c < nv4) {      // warp-uniform: nv4 is a multiple of 32
+            if (FULL || c < nv4) {      // warp-uniform: nv4 is a multiple of 32
                 const float e[4] = {__fmul_rn(x[k].x, rn), __fmul_rn(x[k].y, rn), __fmul_rn(x[k].z, rn), __fmul_rn(x[k].w, rn)};
                 if (BITS == 1) {
                     uint32_t nib = 0;
@@ -216,12 +247,15 @@ cudaError_t launch_quantize_absmean(const float* x, int64_t n, int32_t d, int no
     const int64_t cap = (int64_t)sm_count() * 8 * 4;
     if (blocks > cap) blocks = cap;
     uint8_t* c = reinterpret_cast<uint8_t*>(codes);
+#define QLESS_QA(B, F) quantize_kernel<B, (B > 1), F><<<(unsigned)blocks, QT, 0, st>>>(x, 1, 1.0f, n, d, normalize, c, scales, sumsq, nullptr)
+    const bool full = (d == QT * QMAX_V4 * 4);
     switch (bits) {
-        case 8: quantize_kernel<8, true><<<(unsigned)blocks, QT, 0, st>>>(x, 1, 1.0f, n, d, normalize, c, scales, sumsq, nullptr); break;
-        case 4: quantize_kernel<4, true><<<(unsigned)blocks, QT, 0, st>>>(x, 1, 1.0f, n, d, normalize, c, scales, sumsq, nullptr); break;
-        case 2: quantize_kernel<2, true><<<(unsigned)blocks, QT, 0, st>>>(x, 1, 1.0f, n, d, normalize, c, scales, sumsq, nullptr); break;
-        default: quantize_kernel<1><<<(unsigned)blocks, QT, 0, st>>>(x, 1, 1.0f, n, d, normalize, c, scales, sumsq, nullptr); break;
+        case 8: if (full) QLESS_QA(8, true); else QLESS_QA(8, false); break;
+        case 4: if (full) QLESS_QA(4, true); else QLESS_QA(4, false); break;
+        case 2: if (full) QLESS_QA(2, true); else QLESS_QA(2, false); break;
+        default: if (full) QLESS_QA(1, true); else QLESS_QA(1, false); break;
     }
+#undef QLESS_QA
     count_launches(1);
     return cudaGetLastError();
 }
@@ -235,12 +269,18 @@ cudaError_t launch_quantize(const float* parts, int32_t num_parts, float scale, 
     const int64_t cap = (int64_t)sm_count() * 8 * 4;
     if (blocks > cap) blocks = cap;
     uint8_t* c = reinterpret_cast<uint8_t*>(codes);
+#define QLESS_Q(B, F, M) quantize_kernel<B, false, F, M><<<(unsigned)blocks, QT, 0, st>>>(parts, num_parts, scale, n, d, normalize, c, scales, sumsq, proj_out)
+#define QLESS_QB(B) do { if (full && multi) QLESS_Q(B, true, true); else if (full) QLESS_Q(B, true, false); \
+                         else if (multi) QLESS_Q(B, false, true); else QLESS_Q(B, false, false); } while (0)
+    const bool full = (d == QT * QMAX_V4 * 4), multi = (num_parts > 1);
     switch (bits) {
-        case 8: quantize_kernel<8><<<(unsigned)blocks, QT, 0, st>>>(parts, num_parts, scale, n, d, normalize, c, scales, sumsq, proj_out); break;
-        case 4: quantize_kernel<4><<<(unsigned)blocks, QT, 0, st>>>(parts, num_parts, scale, n, d, normalize, c, scales, sumsq, proj_out); break;
-        case 2: quantize_kernel<2><<<(unsigned)blocks, QT, 0, st>>>(parts, num_parts, scale, n, d, normalize, c, scales, sumsq, proj_out); break;
-        default: quantize_kernel<1><<<(unsigned)blocks, QT, 0, st>>>(parts, num_parts, scale, n, d, normalize, c, scales, sumsq, proj_out); break;
+        case 8: QLESS_QB(8); break;
+        case 4: QLESS_QB(4); break;
+        case 2: QLESS_QB(2); break;
+        default: QLESS_QB(1); break;
     }
+#undef QLESS_QB
+#undef QLESS_Q
     count_launches(1);
     return cudaGetLastError();
 }
