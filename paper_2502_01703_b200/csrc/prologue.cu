@@ -45,7 +45,7 @@ __device__ __forceinline__ float adam_dir_fast(float g, float bm, float bv, cons
     const uint32_t qb = __float_as_uint(q);
     const bool in_range = (qb * 2u - (28u << 24)) <= ((198u << 24) | 0xFFFFFFu);
     const bool off_tie = ((qb << 16) - (0x7FE0u << 16)) > (0x40u << 16);
-    ok = t < 0.00390625f && in_range && off_tie;
+    ok = (t < 0.00390625f) & in_range & off_tie;          // no short circuit: three compares, no branch
     return q;
 }
 
@@ -55,7 +55,7 @@ __device__ __forceinline__ void adam_dir2(float& g0, float& g1, float bm0, float
     bool ok0 = false, ok1 = false;
     float q0 = 0.0f, q1 = 0.0f;
     if (!ap.bias_correct) { q0 = adam_dir_fast(g0, bm0, bv0, ap, ok0); q1 = adam_dir_fast(g1, bm1, bv1, ap, ok1); }
-    if (!(ok0 && ok1)) {
+    if (!(ok0 & ok1)) {
         const float c1 = ap.bias_correct ? ap.c1 : 1.0f, c2 = ap.bias_correct ? ap.c2 : 1.0f;
         if (!ok0) q0 = adam_dir_exact(g0, bm0, bv0, ap.omb1, ap.omb2, ap.eps, c1, c2);
         if (!ok1) q1 = adam_dir_exact(g1, bm1, bv1, ap.omb1, ap.omb2, ap.eps, c1, c2);
