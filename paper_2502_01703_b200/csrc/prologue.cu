@@ -12,13 +12,28 @@ namespace qless {
 // lies close to a bf16 rounding boundary (or outside the normal range) its bf16 rounding is already the one
 // the exact sequence gives, and the exact sequence runs only for the rare remaining elements.
 
-// The exact sequence. Not inlined: it is long, runs for about one element in a thousand, and the kernel holds 32
-// call sites. c1 = c2 = 1 without bias correction (a division by 1 is exact).
-__device__ __noinline__ float adam_dir_exact(float g, float bm, float bv, float omb1, float omb2, float eps, float c1, float c2)
+// Elements the fast path below gave up on (about one in a thousand on typical moments; all of them where
+// eps / sqrt(v') is not small). Not inlined: it is long and the kernel holds 16 call sites. Without bias correction
+// (c1 = c2 = 1) a second approximation is tried first, good for any eps / sqrt(v'): sqrt(v') as v' rs, the quotient
+// by the approximate reciprocal (two special-function operations, a few ulp of error), accepted under the same two
+// tests as the fast path; what is left takes the exact sequence.
+__device__ __noinline__ float adam_dir_slow(float g, float bm, float bv, float omb1, float omb2, float eps, float c1, float c2)
 {
     float m1 = __fadd_rn(bm, __fmul_rn(omb1, g));
     float v1 = __fadd_rn(bv, __fmul_rn(omb2, __fmul_rn(g, g)));
-    if (c1 != 1.0f || c2 != 1.0f) { m1 = __fdiv_rn(m1, c1); v1 = __fdiv_rn(v1, c2); }
+    if (c1 == 1.0f && c2 == 1.0f) {
+        float rs, rc;
+        asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rs) : "f"(v1));
+        const float den_a = __fadd_rn(__fmul_rn(v1, rs), eps);          // v1 = 0 gives NaN: fails the range test
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(den_a));
+        const float q = __fmul_rn(m1, rc);
+        const uint32_t qb = __float_as_uint(q);
+        const bool in_range = (((qb >> 23) & 0xFFu) - 28u) <= 198u;
+        const bool off_tie = ((qb - 0x7FE0u) & 0xFFFFu) > 0x40u;
+        if (in_range && off_tie) return q;
+    } else {
+        m1 = __fdiv_rn(m1, c1); v1 = __fdiv_rn(v1, c2);                 // bias correction
+    }
     const float den = __fadd_rn(__fsqrt_rn(v1), eps);
     return __fdiv_rn(m1, den);
 }
@@ -49,7 +64,7 @@ __device__ __forceinline__ float adam_dir_fast(float g, float bm, float bv, cons
     return q;
 }
 
-// Two neighbouring elements share one branch to the exact sequence.
+// Two neighbouring elements share one branch to the slow path.
 __device__ __forceinline__ void adam_dir2(float& g0, float& g1, float bm0, float bm1, float bv0, float bv1, const AdamParams& ap)
 {
     bool ok0 = false, ok1 = false;
@@ -57,8 +72,8 @@ __device__ __forceinline__ void adam_dir2(float& g0, float& g1, float bm0, float
     if (!ap.bias_correct) { q0 = adam_dir_fast(g0, bm0, bv0, ap, ok0); q1 = adam_dir_fast(g1, bm1, bv1, ap, ok1); }
     if (!(ok0 & ok1)) {
         const float c1 = ap.bias_correct ? ap.c1 : 1.0f, c2 = ap.bias_correct ? ap.c2 : 1.0f;
-        if (!ok0) q0 = adam_dir_exact(g0, bm0, bv0, ap.omb1, ap.omb2, ap.eps, c1, c2);
-        if (!ok1) q1 = adam_dir_exact(g1, bm1, bv1, ap.omb1, ap.omb2, ap.eps, c1, c2);
+        if (!ok0) q0 = adam_dir_slow(g0, bm0, bv0, ap.omb1, ap.omb2, ap.eps, c1, c2);
+        if (!ok1) q1 = adam_dir_slow(g1, bm1, bv1, ap.omb1, ap.omb2, ap.eps, c1, c2);
     }
     g0 = q0; g1 = q1;
 }
