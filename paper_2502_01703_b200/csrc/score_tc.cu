@@ -76,13 +76,6 @@ __device__ __forceinline__ void unpack4(uint32_t w, uint32_t& lo, uint32_t& hi)
     lo = __vsub4((w & 0x0F0F0F0Fu) ^ 0x08080808u, 0x08080808u);
     hi = __vsub4(((w >> 4) & 0x0F0F0F0Fu) ^ 0x08080808u, 0x08080808u);
 }
-// 16 packed 2-bit codes -> four words of four int8 (field f of every byte -> word f)
-__device__ __forceinline__ void unpack2(uint32_t w, uint32_t (&o)[4])
-{
-#pragma unroll
-    for (int f = 0; f < 4; ++f) o[f] = __vsub4(((w >> (2 * f)) & 0x03030303u) ^ 0x02020202u, 0x02020202u);
-}
-
 // Position in a ring of n slots: slot index and the parity of its current use. Advanced by comparison, not by
 // division: the role loops below run on single threads whose every instruction is on the critical path.
 struct Ring {
@@ -90,10 +83,50 @@ struct Ring {
     __device__ __forceinline__ void next(uint32_t n) { if (++slot == n) { slot = 0; parity ^= 1u; } }
 };
 
-// 4 sign bits (bit set = negative) -> one word of four int8 +-1: the multiply copies bit i to byte i
-__device__ __forceinline__ uint32_t unpack1_nibble(uint32_t nib)
+// 16 sign bits (bit set = negative) -> two words of eight e2m1 codes (+1 = 0x2, -1 = 0xA), code j of the sixteen in
+// nibble j: the bits are spread into eight 2-bit byte selectors, and a byte permute looks each pair of codes up.
+__device__ __forceinline__ uint32_t spread2_to_nibbles(uint32_t h)          // 2-bit field j of 16 bits -> nibble j
 {
-    return 0x01010101u + ((nib * 0x00204081u) & 0x01010101u) * 0xFEu;
+    uint32_t x = (h | (h << 8)) & 0x00FF00FFu;
+    x = (x | (x << 4)) & 0x0F0F0F0Fu;
+    return (x | (x << 2)) & 0x33333333u;
+}
+__device__ __forceinline__ void fp4_from_signs16(uint32_t h, uint32_t& lo, uint32_t& hi)
+{
+    const uint32_t sel = spread2_to_nibbles(h);
+    lo = __byte_perm(0xAAA22A22u, 0u, sel);              // selector 0..3 -> 0x22, 0x2A, 0xA2, 0xAA
+    hi = __byte_perm(0xAAA22A22u, 0u, sel >> 16);
+}
+// 16 two-bit codes (two's complement) -> two words of eight e2m1 codes: 00 -> 0, 01 -> +1 (0x2), 11 -> -1 (0xA), 10 -> -2 (0xC)
+__device__ __forceinline__ uint32_t fp4_from_nibble_codes2(uint32_t y)     // nibbles 00 c1 c0
+{
+    const uint32_t c0 = (y & 0x11111111u) << 1, c1 = y & 0x22222222u;
+    return c0 | (c1 << 2) | ((c1 & ~c0) << 1);
+}
+__device__ __forceinline__ void fp4_from_codes2(uint32_t w, uint32_t& lo, uint32_t& hi)
+{
+    lo = fp4_from_nibble_codes2(spread2_to_nibbles(w & 0xFFFFu));
+    hi = fp4_from_nibble_codes2(spread2_to_nibbles(w >> 16));
+}
+
+// Pair MMA on e2m1 operands (kind::mxf4, block-scaled, 64 codes per instruction, fp32 accumulation), both operands from
+// shared memory. The scale factors (one UE8M0 byte per 32 codes of a row) are all 2^0: every byte of the tensor-memory
+// columns at sf_tmem is 0x7F, so the layout in which the instruction reads them does not matter.
+__device__ __forceinline__ void mma_mxf4_ss_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t sf_tmem,
+                                                 uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%5], p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sf_tmem)
+        : "memory");
+}
+// Instruction descriptor of kind::mxf4: A and B format e2m1 (1) at bits [7,10) and [10,13), K-major, N/8 at [17,23),
+// scale format UE8M0 (1) at bit 23, M/16 at [24,29), scale-factor byte offsets 0.
+__host__ __device__ constexpr uint32_t make_idesc_mxf4(uint32_t M, uint32_t N)
+{
+    return (1u << 7) | (1u << 10) | ((N >> 3) << 17) | (1u << 23) | ((M >> 4) << 24);
 }
 
 template <int BITS>
@@ -105,9 +138,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);    // 1 KiB aligned, still a shared pointer
     const int bh1 = (p.n1 / 2) * KB, bh2 = (p.n2 / 2) * KB;      // bytes of this CTA's rows of the two MMA halves
     constexpr bool DIRECT = (BITS >= 8);                           // 8-bit codes and bf16 rows feed the MMA as stored
-    constexpr int A_SMEM = DIRECT ? A_STAGE : 0;                   // sub-byte widths keep A in tensor memory
+    constexpr bool FP4 = (BITS <= 2);                              // 2- and 1-bit codes run as e2m1 (kind::mxf4): 256 codes per K block
+    constexpr int A_SMEM = (DIRECT || FP4) ? A_STAGE : 0;         // 4-bit codes keep A in tensor memory
     const int stage_bytes = A_SMEM + bh1 + bh2;                   // multiple of 1024
-    constexpr int P_STAGE = DIRECT ? 0 : TM * 16 * BITS;          // packed staging bytes per stage
+    constexpr int PROW = DIRECT ? 0 : (FP4 ? 32 : 16) * BITS;     // packed bytes of one row's K block
+    constexpr int P_STAGE = TM * PROW;                            // packed staging bytes per stage
     uint8_t* sS = smem;                                           // stage s: [A 16 KiB][B half 1][B half 2]
     uint8_t* sP = sS + (size_t)p.nS * stage_bytes;
     ScoreBars* bars = reinterpret_cast<ScoreBars*>(sP + (size_t)p.nP * P_STAGE);
@@ -116,12 +151,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     const int64_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-    const int nkb = (BITS == 16) ? (2 * p.d) / KB : p.d / KB;      // K blocks of 128 bytes per row
+    const int nkb = (BITS == 16) ? (2 * p.d) / KB : FP4 ? (p.d + 2 * KB - 1) / (2 * KB) : p.d / KB;      // K blocks of 128 operand bytes per row
     const int num_vt = (p.V + p.vpad - 1) / p.vpad;
     const int64_t num_tiles = (p.N + 2 * TM - 1) / (2 * TM);      // tiles of 256 train rows
     // int8: D = S32 (2), A = B = S8 (1); 16-bit baseline: D = F32 (1), A = B = BF16 (1)
-    const uint32_t idesc1 = make_idesc(BITS == 16 ? 1 : 2, 1, 1, 2 * TM, p.n1);
-    const uint32_t idesc2 = make_idesc(BITS == 16 ? 1 : 2, 1, 1, 2 * TM, p.n2 > 0 ? p.n2 : 16);
+    const uint32_t idesc1 = FP4 ? make_idesc_mxf4(2 * TM, p.n1) : make_idesc(BITS == 16 ? 1 : 2, 1, 1, 2 * TM, p.n1);
+    const uint32_t idesc2 = FP4 ? make_idesc_mxf4(2 * TM, p.n2 > 0 ? p.n2 : 16) : make_idesc(BITS == 16 ? 1 : 2, 1, 1, 2 * TM, p.n2 > 0 ? p.n2 : 16);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_STAGES; ++s) {
@@ -151,13 +186,26 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
     cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
+    if (FP4) {
+        // unit scale factors: 0x7F in every byte of 16 tensor-memory columns behind the accumulator, all 128 lanes
+        if (warp >= 6 && warp < 10) {
+            uint32_t v[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) v[k] = 0x7F7F7F7Fu;
+            tmem_st_x16(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + A_TMEM_COL, v);
+            tmem_wait_st();
+            tc_fence_before();
+        }
+        __syncthreads();         // the unpack warps' first arrival (which the first MMA waits for) comes after this
+        tc_fence_after();
+    }
 
     if (warp == 0) {
         // ------------------------------- TMA producer -------------------------------
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            const uint32_t tx_total = 2u * (uint32_t)(A_SMEM + bh1 + bh2);   // both CTAs
+            const uint32_t tx_total = 2u * (uint32_t)((DIRECT ? A_STAGE : 0) + bh1 + bh2);   // both CTAs (TMA bytes only)
             const int64_t my_tiles = (num_tiles > pair) ? (num_tiles - pair + num_pairs - 1) / num_pairs : 0;
             const int64_t total = my_tiles * num_vt * p.C * nkb;
             // Packed train codes run ahead of the operand stages in their own ring: the load for iteration q is
@@ -173,7 +221,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 else if (!mbar_test_wait(smem_u32(&bars->p_empty[sp]), pring.parity ^ 1u)) return false;
                 const uint32_t pfull = smem_u32(&bars->p_full[sp]);
                 mbar_arrive_expect_tx(pfull, P_STAGE);
-                tma_load_3d(smem_u32(sP + (size_t)sp * P_STAGE), &tmap_train, pfull, p_kb * 16 * BITS, (int32_t)(p_tile * 2 * TM + rank * TM), p_i);
+                tma_load_3d(smem_u32(sP + (size_t)sp * P_STAGE), &tmap_train, pfull, p_kb * PROW, (int32_t)(p_tile * 2 * TM + rank * TM), p_i);
                 ++pq; pring.next((uint32_t)p.nP);
                 if (++p_kb == nkb) { p_kb = 0; if (++p_i == p.C) { p_i = 0; if (++p_vt == num_vt) { p_vt = 0; p_tile += num_pairs; } } }
                 return true;
@@ -236,7 +284,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         for (int kb = 0; kb < nkb; ++kb, ++it, st_ring.next((uint32_t)p.nS)) {
                             const int s = (int)st_ring.slot;
                             if (!DIRECT || (s & 1) == 0) {       // DIRECT: the barrier at the even slot covers this stage and the next
-                                if (!mbar_wait(smem_u32(&bars->full[s]), st_ring.parity, abort_flag, p.timeout_word, TO_MMA)) { ok = false; break; }
+                                // e2m1 path: the peer's unpack warps wrote their rows of A into the peer's shared memory and
+                                // released them at cluster scope; tensor-memory operands are ordered by the tcgen05 fences
+                                const bool okw = FP4 ? mbar_wait_cluster(smem_u32(&bars->full[s]), st_ring.parity, abort_flag, p.timeout_word, TO_MMA)
+                                                     : mbar_wait(smem_u32(&bars->full[s]), st_ring.parity, abort_flag, p.timeout_word, TO_MMA);
+                                if (!okw) { ok = false; break; }
                                 tc_fence_after();
                             }
                             const uint32_t st = smem_u32(sS + (size_t)s * stage_bytes);
@@ -253,6 +305,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                                 } else if (BITS == 8) {
                                     mma_i8_ss_pair(tmem_base, adesc + (uint64_t)(k * 2), bdesc1 + (uint64_t)(k * 2), idesc1, acc);
                                     if (p.n2 > 0) mma_i8_ss_pair(tmem_base + p.n1, adesc + (uint64_t)(k * 2), bdesc2 + (uint64_t)(k * 2), idesc2, acc);
+                                } else if (FP4) {
+                                    mma_mxf4_ss_pair(tmem_base, adesc + (uint64_t)(k * 2), bdesc1 + (uint64_t)(k * 2), idesc1, tmem_base + A_TMEM_COL, acc);
+                                    if (p.n2 > 0) mma_mxf4_ss_pair(tmem_base + p.n1, adesc + (uint64_t)(k * 2), bdesc2 + (uint64_t)(k * 2), idesc2, tmem_base + A_TMEM_COL, acc);
                                 } else {
                                     mma_i8_ts_pair(tmem_base, a_tmem + k * 8, bdesc1 + (uint64_t)(k * 2), idesc1, acc);
                                     if (p.n2 > 0) mma_i8_ts_pair(tmem_base + p.n1, a_tmem + k * 8, bdesc2 + (uint64_t)(k * 2), idesc2, acc);
@@ -288,24 +343,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 // unpack into registers first: this needs only the packed bytes, not the TMEM slot
-                const uint4* src = reinterpret_cast<const uint4*>(sP + (size_t)sp * P_STAGE + (size_t)row * (16 * BITS));
+                const uint4* src = reinterpret_cast<const uint4*>(sP + (size_t)sp * P_STAGE + (size_t)row * PROW);
                 uint32_t out[32];
 #pragma unroll
-                for (int c = 0; c < (16 * BITS) / 16; ++c) {
+                for (int c = 0; c < PROW / 16; ++c) {
                     const uint4 w = src[c];
                     const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         if (BITS == 4) {
                             unpack4(ww[u], out[(c * 4 + u) * 2], out[(c * 4 + u) * 2 + 1]);
-                        } else if (BITS == 1) {
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) out[u * 8 + j] = unpack1_nibble((ww[u] >> (4 * j)) & 0xFu);
-                        } else {
-                            uint32_t o4[4];
-                            unpack2(ww[u], o4);
-#pragma unroll
-                            for (int f = 0; f < 4; ++f) out[(c * 4 + u) * 4 + f] = o4[f];
+                        } else if (BITS == 1) {          // 32 sign bits -> four words of eight e2m1 codes, in order
+                            fp4_from_signs16(ww[u] & 0xFFFFu, out[(c * 4 + u) * 4], out[(c * 4 + u) * 4 + 1]);
+                            fp4_from_signs16(ww[u] >> 16, out[(c * 4 + u) * 4 + 2], out[(c * 4 + u) * 4 + 3]);
+                        } else {                         // 16 two-bit codes -> two words of eight e2m1 codes, in order
+                            fp4_from_codes2(ww[u], out[(c * 4 + u) * 2], out[(c * 4 + u) * 2 + 1]);
                         }
                     }
                 }
@@ -314,6 +366,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bars->p_empty[sp]));      // staging slot read: the producer may refill it
+                if (FP4) {
+                    // The row goes into operand stage s of this CTA's shared memory as the MMA reads a K-major operand with
+                    // the 128-byte swizzle (what a TMA load would have written): 16-byte piece j of row r at piece j ^ (r & 7).
+                    // The stage is free once the MMAs of its previous use have completed (the commit arrives in both CTAs).
+                    ok = mbar_wait(smem_u32(&bars->empty[s]), st_ring.parity ^ 1u, abort_flag, p.timeout_word, TO_UNPACK);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    uint4* dst = reinterpret_cast<uint4*>(sS + (size_t)s * stage_bytes + (size_t)row * KB);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) dst[j ^ (row & 7)] = make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+                    fence_proxy_async_smem();      // generic-proxy writes, read by the tensor core through the async proxy
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (rank == 0) mbar_arrive(smem_u32(&bars->full[s]));
+                        else mbar_arrive_cluster(map_to_cta(smem_u32(&bars->full[s]), 0));      // release at cluster scope
+                    }
+                    continue;
+                }
                 // TMEM slot it % 2 is free once the MMAs of K block it - 2 have completed, which is what releases
                 // operand stage (it - 2) % nS (nS > 2, so that barrier cannot run a whole phase ahead of us)
                 if (it >= 2)
@@ -389,7 +459,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                             if (t < p.N) {
 #pragma unroll
                                 for (int k = 0; k < 32; ++k)
-                                    if (c0 + k < vcount) p.dots[t * p.V + v0 + c0 + k] = (int32_t)v[k];
+                                    if (c0 + k < vcount) p.dots[t * p.V + v0 + c0 + k] = FP4 ? (int32_t)__uint_as_float(v[k]) : (int32_t)v[k];
                             }
                         } else {
                             // columns >= vcount carry a zero multiplier, so they add nothing
@@ -397,8 +467,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
 #pragma unroll
                             for (int k4 = 0; k4 < 8; ++k4) {
                                 const float4 m4 = *reinterpret_cast<const float4*>(&bars->mv[c0 + 4 * k4]);
-                                // the accumulator holds int32 dots, or fp32 inner products for the 16-bit baseline
-                                auto acc_f = [](uint32_t raw) { return BITS == 16 ? __uint_as_float(raw) : (float)(int32_t)raw; };
+                                // the accumulator holds int32 dots; fp32 inner products for the 16-bit baseline; fp32 values that
+                                // are exact integers (at most 4 d in magnitude) for the e2m1 path
+                                auto acc_f = [](uint32_t raw) { return (BITS == 16 || BITS <= 2) ? __uint_as_float(raw) : (float)(int32_t)raw; };
                                 x[4 * k4 + 0] = __fmul_rn(acc_f(v[4 * k4 + 0]), m4.x);
                                 x[4 * k4 + 1] = __fmul_rn(acc_f(v[4 * k4 + 1]), m4.y);
                                 x[4 * k4 + 2] = __fmul_rn(acc_f(v[4 * k4 + 2]), m4.z);
@@ -475,13 +546,17 @@ __global__ void unpack_val_kernel(const uint8_t* __restrict__ codes, int64_t ckp
         const int wq = (int)(idx - rowid * words_per_row);
         const int64_t i = rowid / V, v = rowid - i * V;
         const uint32_t w = *reinterpret_cast<const uint32_t*>(codes + i * ckpt_stride + v * (int64_t)(d * BITS / 8) + 4 * wq);
-        uint32_t* o = reinterpret_cast<uint32_t*>(out + rowid * d) + wq * (8 / BITS);
-        if (BITS == 4) { unpack4(w, o[0], o[1]); }
-        else if (BITS == 1) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) o[j] = unpack1_nibble((w >> (4 * j)) & 0xFu);
+        if (BITS == 4) {
+            uint32_t* o = reinterpret_cast<uint32_t*>(out + rowid * d) + wq * 2;
+            unpack4(w, o[0], o[1]);
+        } else if (BITS == 1) {      // e2m1, two codes per byte: d / 2 bytes per row
+            uint32_t* o = reinterpret_cast<uint32_t*>(out + rowid * (d / 2)) + wq * 4;
+            fp4_from_signs16(w & 0xFFFFu, o[0], o[1]);
+            fp4_from_signs16(w >> 16, o[2], o[3]);
+        } else {
+            uint32_t* o = reinterpret_cast<uint32_t*>(out + rowid * (d / 2)) + wq * 2;
+            fp4_from_codes2(w, o[0], o[1]);
         }
-        else { uint32_t o4[4]; unpack2(w, o4); o[0] = o4[0]; o[1] = o4[1]; o[2] = o4[2]; o[3] = o4[3]; }
     }
 }
 
@@ -509,8 +584,9 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
 
     // shared-memory plan: as many operand stages as fit (each: 16 KiB of train rows + this CTA's validation rows)
     const size_t budget = 227 * 1024 - 1024 - sizeof(ScoreBars) - 64;
-    const size_t stage = (a.bits >= 8 ? (size_t)A_STAGE : 0) + (size_t)(p.vpad / 2) * KB;
-    const size_t p_stage = a.bits >= 8 ? 0 : (size_t)TM * 16 * a.bits;
+    const bool fp4 = a.bits <= 2;                          // 2- and 1-bit codes: e2m1 operands, both from shared memory
+    const size_t stage = ((a.bits >= 8 || fp4) ? (size_t)A_STAGE : 0) + (size_t)(p.vpad / 2) * KB;
+    const size_t p_stage = a.bits >= 8 ? 0 : (size_t)TM * (fp4 ? 32 : 16) * a.bits;
     int nP = a.bits >= 8 ? 0 : 4;
     int nS = (int)((budget - (size_t)nP * p_stage) / stage);
     if (nS > MAX_STAGES) nS = MAX_STAGES;
@@ -533,13 +609,14 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
         else if (a.bits == 1) unpack_val_kernel<1><<<(unsigned)blocks, 256, 0, st>>>(a.val, a.val_stride, a.V, a.C, a.d, val_unpacked);
         else unpack_val_kernel<2><<<(unsigned)blocks, 256, 0, st>>>(a.val, a.val_stride, a.V, a.C, a.d, val_unpacked);
         count_launches(1);
-        val_src = val_unpacked; val_row = a.d; val_stride = (int64_t)a.V * a.d;
+        val_row = fp4 ? a.d / 2 : a.d;
+        val_src = val_unpacked; val_stride = (int64_t)a.V * val_row;
     }
     CUtensorMap tm_train, tm_v1, tm_v2;
     qless_status s;
     const int64_t tstride = a.C > 1 ? a.train_stride : (int64_t)a.N * row_bytes;
     s = make_tmap_3d_u8(&tm_train, a.train, (uint64_t)row_bytes, (uint64_t)a.N, (uint64_t)a.C, (uint64_t)row_bytes,
-                        (uint64_t)tstride, a.bits >= 8 ? 128 : 16 * a.bits, TM, a.bits >= 8);     // this CTA's 128 rows
+                        (uint64_t)tstride, a.bits >= 8 ? 128 : (fp4 ? 32 : 16) * a.bits, TM, a.bits >= 8);     // this CTA's 128 rows
     if (s != QLESS_OK) return s;
     const int64_t vstride = a.C > 1 ? val_stride : (int64_t)a.V * val_row;
     s = make_tmap_3d_u8(&tm_v1, val_src, (uint64_t)val_row, (uint64_t)a.V, (uint64_t)a.C, (uint64_t)val_row, (uint64_t)vstride, 128, p.n1 / 2, true);
