@@ -51,6 +51,8 @@ struct ScoreTcParams {
     int32_t n1, n2;             // MMA N of the two halves (n1 + n2 = vpad)
     int32_t nS, nP;             // pipeline depths: operand stages (A + B), packed staging
     int32_t epi_groups;         // 1 or 2 groups of four epilogue warps (2: each takes half of the columns)
+    const uint8_t* train_codes; // packed train codes (read directly by the unpack warps of the 2- and 1-bit path)
+    int64_t train_stride;       // bytes between checkpoints
     const float* train_mult;    // [C][N]
     const float* val_mult;      // [C][V]
     const float* eta_over_cnt;  // [C][T]
@@ -142,7 +144,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
     constexpr int A_SMEM = (DIRECT || FP4) ? A_STAGE : 0;         // 4-bit codes keep A in tensor memory
     const int stage_bytes = A_SMEM + bh1 + bh2;                   // multiple of 1024
     constexpr int PROW = DIRECT ? 0 : (FP4 ? 32 : 16) * BITS;     // packed bytes of one row's K block
-    constexpr int P_STAGE = TM * PROW;                            // packed staging bytes per stage
+    constexpr int P_STAGE = (DIRECT || FP4) ? 0 : TM * PROW;      // packed staging bytes per stage (4-bit codes only)
     uint8_t* sS = smem;                                           // stage s: [A 16 KiB][B half 1][B half 2]
     uint8_t* sP = sS + (size_t)p.nS * stage_bytes;
     ScoreBars* bars = reinterpret_cast<ScoreBars*>(sP + (size_t)p.nP * P_STAGE);
@@ -233,7 +235,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 for (int vt = 0; vt < num_vt && ok; ++vt)
                     for (int i = 0; i < p.C && ok; ++i)
                         for (int kb = 0; kb < nkb; ++kb, ++it, st_ring.next((uint32_t)p.nS)) {
-                            if (!DIRECT) {
+                            if (!DIRECT && !FP4) {
                                 // the packed codes of this iteration must be on their way; those of the next few if a slot is free
                                 while (pq <= (int64_t)it && ok) ok = issue_packed(true);
                                 if (!ok) break;
@@ -260,7 +262,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 // have been armed; their copies complete on the leader's barriers, whose phases also need the unpack
                 // warps' arrivals at the sub-byte widths and may therefore never close: the leader gives them a bounded
                 // wait, the peer idles, and neither leaves before the other (the cluster barrier at the end).
-                if (!DIRECT)
+                if (!DIRECT && !FP4)
                     for (int64_t j = (pq > p.nP ? pq - p.nP : 0); j < pq; ++j)
                         if (!mbar_wait_quiet(smem_u32(&bars->p_full[j % p.nP]), (uint32_t)(j / p.nP) & 1u)) break;
                 if (rank == 0) {
@@ -327,7 +329,82 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
         // ------------------------------- unpack warps (4- and 2-bit train codes) -------------------------------
         // two groups of four warps (2-5 and 10-13) take alternate K blocks, so that the barrier round trips of
         // one block overlap the unpacking of the next
-        if (!DIRECT) {
+        if (FP4) {
+            // 2- and 1-bit codes. A thread owns a row of the half tile and takes its packed codes straight from global memory
+            // (32 or 64 bytes per K block: whole sectors), two of its group's K blocks ahead in registers; it expands them to
+            // e2m1 and writes the row into operand stage s of this CTA's shared memory as the MMA reads a K-major operand
+            // with the 128-byte swizzle (what a TMA load would have written): 16-byte piece j of row r at piece j ^ (r & 7).
+            const int row = (warp & 3) * 32 + lane;
+            const uint32_t grp = (warp >= 10) ? 1u : 0u;
+            constexpr int NV = PROW >= 16 ? PROW / 16 : 1;       // (this branch is compiled for every width)
+            const int64_t my_tiles = (num_tiles > pair) ? (num_tiles - pair + num_pairs - 1) / num_pairs : 0;
+            const int64_t total = my_tiles * num_vt * p.C * nkb;
+            const int64_t row_bytes = (int64_t)p.d * BITS / 8;
+            struct Pos { int kb, i, vt; int64_t tile; };
+            auto advance = [&](Pos& q, int n) {
+                q.kb += n;
+                while (q.kb >= nkb) { q.kb -= nkb; if (++q.i == p.C) { q.i = 0; if (++q.vt == num_vt) { q.vt = 0; q.tile += num_pairs; } } }
+            };
+            auto fetch = [&](const Pos& q, uint4 (&r)[NV]) {
+                const int64_t t = q.tile * 2 * TM + rank * TM + row;
+                const uint8_t* src = p.train_codes + (int64_t)q.i * p.train_stride + t * row_bytes + (int64_t)q.kb * PROW;
+#pragma unroll
+                for (int c = 0; c < NV; ++c)
+                    r[c] = (t < p.N && (int64_t)q.kb * PROW + 16 * c < row_bytes) ? __ldcs(reinterpret_cast<const uint4*>(src) + c)
+                                                                                  : make_uint4(0u, 0u, 0u, 0u);
+            };
+            Pos pf{0, 0, 0, pair};
+            advance(pf, (int)grp);
+            Ring st_ring;
+            if (grp) st_ring.next((uint32_t)p.nS);
+            uint4 ra[NV], rb[NV];
+            int64_t g = grp;                                      // K block (in this pair's sequence) of the registers ra
+            if (g < total) { fetch(pf, ra); advance(pf, 2); }
+            if (g + 2 < total) { fetch(pf, rb); advance(pf, 2); }
+            bool ok = true;
+            auto emit = [&](const uint4 (&r)[NV]) -> bool {
+                uint32_t out[32];
+#pragma unroll
+                for (int c = 0; c < NV; ++c) {
+                    const uint32_t ww[4] = {r[c].x, r[c].y, r[c].z, r[c].w};
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (BITS == 1) {                 // 32 sign bits -> four words of eight e2m1 codes, in order
+                            fp4_from_signs16(ww[u] & 0xFFFFu, out[(c * 4 + u) * 4], out[(c * 4 + u) * 4 + 1]);
+                            fp4_from_signs16(ww[u] >> 16, out[(c * 4 + u) * 4 + 2], out[(c * 4 + u) * 4 + 3]);
+                        } else {                         // 16 two-bit codes -> two words of eight e2m1 codes, in order
+                            fp4_from_codes2(ww[u], out[(c * 4 + u) * 2], out[(c * 4 + u) * 2 + 1]);
+                        }
+                    }
+                }
+                const int s = (int)st_ring.slot;
+                // the stage is free once the MMAs of its previous use have completed (the commit arrives in both CTAs)
+                bool w = mbar_wait(smem_u32(&bars->empty[s]), st_ring.parity ^ 1u, abort_flag, p.timeout_word, TO_UNPACK);
+                w = __all_sync(0xFFFFFFFFu, w);
+                if (!w) return false;
+                uint4* dst = reinterpret_cast<uint4*>(sS + (size_t)s * stage_bytes + (size_t)row * KB);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) dst[j ^ (row & 7)] = make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+                fence_proxy_async_smem();      // generic-proxy writes, read by the tensor core through the async proxy
+                __syncwarp();
+                if (lane == 0) {
+                    if (rank == 0) mbar_arrive(smem_u32(&bars->full[s]));
+                    else mbar_arrive_cluster(map_to_cta(smem_u32(&bars->full[s]), 0));      // release at cluster scope
+                }
+                st_ring.next((uint32_t)p.nS); st_ring.next((uint32_t)p.nS);
+                return true;
+            };
+            for (; g < total && ok; g += 4) {
+                ok = emit(ra);
+                if (!ok) break;
+                if (g + 4 < total) { fetch(pf, ra); advance(pf, 2); }
+                if (g + 2 < total) {
+                    ok = emit(rb);
+                    if (!ok) break;
+                    if (g + 6 < total) { fetch(pf, rb); advance(pf, 2); }
+                }
+            }
+        } else if (!DIRECT) {
             const int row = (warp & 3) * 32 + lane;               // row of this CTA's 128-row half tile = TMEM lane
             const uint32_t grp = (warp >= 10) ? 1u : 0u;
             uint32_t it = 0;
@@ -353,11 +430,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                     for (int u = 0; u < 4; ++u) {
                         if (BITS == 4) {
                             unpack4(ww[u], out[(c * 4 + u) * 2], out[(c * 4 + u) * 2 + 1]);
-                        } else if (BITS == 1) {          // 32 sign bits -> four words of eight e2m1 codes, in order
-                            fp4_from_signs16(ww[u] & 0xFFFFu, out[(c * 4 + u) * 4], out[(c * 4 + u) * 4 + 1]);
-                            fp4_from_signs16(ww[u] >> 16, out[(c * 4 + u) * 4 + 2], out[(c * 4 + u) * 4 + 3]);
-                        } else {                         // 16 two-bit codes -> two words of eight e2m1 codes, in order
-                            fp4_from_codes2(ww[u], out[(c * 4 + u) * 2], out[(c * 4 + u) * 2 + 1]);
                         }
                     }
                 }
@@ -366,24 +438,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bars->p_empty[sp]));      // staging slot read: the producer may refill it
-                if (FP4) {
-                    // The row goes into operand stage s of this CTA's shared memory as the MMA reads a K-major operand with
-                    // the 128-byte swizzle (what a TMA load would have written): 16-byte piece j of row r at piece j ^ (r & 7).
-                    // The stage is free once the MMAs of its previous use have completed (the commit arrives in both CTAs).
-                    ok = mbar_wait(smem_u32(&bars->empty[s]), st_ring.parity ^ 1u, abort_flag, p.timeout_word, TO_UNPACK);
-                    ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (!ok) break;
-                    uint4* dst = reinterpret_cast<uint4*>(sS + (size_t)s * stage_bytes + (size_t)row * KB);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) dst[j ^ (row & 7)] = make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
-                    fence_proxy_async_smem();      // generic-proxy writes, read by the tensor core through the async proxy
-                    __syncwarp();
-                    if (lane == 0) {
-                        if (rank == 0) mbar_arrive(smem_u32(&bars->full[s]));
-                        else mbar_arrive_cluster(map_to_cta(smem_u32(&bars->full[s]), 0));      // release at cluster scope
-                    }
-                    continue;
-                }
                 // TMEM slot it % 2 is free once the MMAs of K block it - 2 have completed, which is what releases
                 // operand stage (it - 2) % nS (nS > 2, so that barrier cannot run a whole phase ahead of us)
                 if (it >= 2)
@@ -586,8 +640,8 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     const size_t budget = 227 * 1024 - 1024 - sizeof(ScoreBars) - 64;
     const bool fp4 = a.bits <= 2;                          // 2- and 1-bit codes: e2m1 operands, both from shared memory
     const size_t stage = ((a.bits >= 8 || fp4) ? (size_t)A_STAGE : 0) + (size_t)(p.vpad / 2) * KB;
-    const size_t p_stage = a.bits >= 8 ? 0 : (size_t)TM * (fp4 ? 32 : 16) * a.bits;
-    int nP = a.bits >= 8 ? 0 : 4;
+    const size_t p_stage = (a.bits >= 8 || fp4) ? 0 : (size_t)TM * 16 * a.bits;      // packed staging ring: 4-bit codes only
+    int nP = (a.bits >= 8 || fp4) ? 0 : 4;
     int nS = (int)((budget - (size_t)nP * p_stage) / stage);
     if (nS > MAX_STAGES) nS = MAX_STAGES;
     if (a.bits >= 8) nS &= ~1;                              // stages are handed to the MMAs in pairs
@@ -596,6 +650,7 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     p.epi_groups = (a.bits >= 8 && a.T <= 6) ? 2 : 1;
     const size_t smem = 1024 + (size_t)nS * stage + (size_t)nP * p_stage + sizeof(ScoreBars);
 
+    p.train_codes = a.train; p.train_stride = a.C > 1 ? a.train_stride : 0;
     p.train_mult = a.train_mult; p.val_mult = a.val_mult; p.eta_over_cnt = a.eta_over_cnt; p.task_off = a.task_off;
     p.scores = a.scores; p.per_task = a.per_task; p.dots = a.dots; p.timeout_word = timeout_word;
 
