@@ -41,6 +41,7 @@ constexpr int KB = 128;                    // codes (= unpacked bytes) per row p
 constexpr int A_STAGE = TM * KB;           // 16 KiB
 constexpr int MAX_STAGES = 8;
 constexpr int NTHREADS = 448;
+constexpr int NTHREADS_FP4 = 576;          // 2- and 1-bit codes: a third group of four unpack warps (14-17)
 constexpr int TMAX = 8;                    // tasks held in registers by the epilogue
 constexpr int A_TMEM_COL = 448;            // sub-byte widths: two 32-column slots of unpacked train codes
 
@@ -132,7 +133,7 @@ __host__ __device__ constexpr uint32_t make_idesc_mxf4(uint32_t M, uint32_t N)
 }
 
 template <int BITS>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(BITS <= 2 ? NTHREADS_FP4 : NTHREADS, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_constant__ CUtensorMap tmap_val1,
                 const __grid_constant__ CUtensorMap tmap_val2, const ScoreTcParams p)
 {
@@ -178,7 +179,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
         prefetch_tmap(&tmap_train); prefetch_tmap(&tmap_val1); prefetch_tmap(&tmap_val2);
     }
     if (p.task_off != nullptr)
-        for (int j = threadIdx.x; j <= p.T; j += NTHREADS) bars->task_off[j] = p.task_off[j];
+        for (int j = threadIdx.x; j <= p.T; j += (int)blockDim.x) bars->task_off[j] = p.task_off[j];
     if (warp == 1) {
         tmem_alloc_pair(smem_u32(&bars->tmem_base), 512);
         tmem_relinquish_pair();
@@ -334,8 +335,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
             // (32 or 64 bytes per K block: whole sectors), two of its group's K blocks ahead in registers; it expands them to
             // e2m1 and writes the row into operand stage s of this CTA's shared memory as the MMA reads a K-major operand
             // with the 128-byte swizzle (what a TMA load would have written): 16-byte piece j of row r at piece j ^ (r & 7).
-            const int row = (warp & 3) * 32 + lane;
-            const uint32_t grp = (warp >= 10) ? 1u : 0u;
+            const int row = ((warp - 2) & 3) * 32 + lane;
+            constexpr int NG = 3;                                 // groups of four warps: 2-5, 10-13, 14-17; group g takes K blocks g, g + 3, ...
+            const uint32_t grp = (warp >= 14) ? 2u : (warp >= 10) ? 1u : 0u;
             constexpr int NV = PROW >= 16 ? PROW / 16 : 1;       // (this branch is compiled for every width)
             const int64_t my_tiles = (num_tiles > pair) ? (num_tiles - pair + num_pairs - 1) / num_pairs : 0;
             const int64_t total = my_tiles * num_vt * p.C * nkb;
@@ -356,11 +358,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
             Pos pf{0, 0, 0, pair};
             advance(pf, (int)grp);
             Ring st_ring;
-            if (grp) st_ring.next((uint32_t)p.nS);
+            for (uint32_t j = 0; j < grp; ++j) st_ring.next((uint32_t)p.nS);
             uint4 ra[NV], rb[NV];
             int64_t g = grp;                                      // K block (in this pair's sequence) of the registers ra
-            if (g < total) { fetch(pf, ra); advance(pf, 2); }
-            if (g + 2 < total) { fetch(pf, rb); advance(pf, 2); }
+            if (g < total) { fetch(pf, ra); advance(pf, NG); }
+            if (g + NG < total) { fetch(pf, rb); advance(pf, NG); }
             bool ok = true;
             auto emit = [&](const uint4 (&r)[NV]) -> bool {
                 uint32_t out[32];
@@ -391,17 +393,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                     if (rank == 0) mbar_arrive(smem_u32(&bars->full[s]));
                     else mbar_arrive_cluster(map_to_cta(smem_u32(&bars->full[s]), 0));      // release at cluster scope
                 }
-                st_ring.next((uint32_t)p.nS); st_ring.next((uint32_t)p.nS);
+#pragma unroll
+                for (int j = 0; j < NG; ++j) st_ring.next((uint32_t)p.nS);
                 return true;
             };
-            for (; g < total && ok; g += 4) {
+            for (; g < total && ok; g += 2 * NG) {
                 ok = emit(ra);
                 if (!ok) break;
-                if (g + 4 < total) { fetch(pf, ra); advance(pf, 2); }
-                if (g + 2 < total) {
+                if (g + 2 * NG < total) { fetch(pf, ra); advance(pf, NG); }
+                if (g + NG < total) {
                     ok = emit(rb);
                     if (!ok) break;
-                    if (g + 6 < total) { fetch(pf, rb); advance(pf, 2); }
+                    if (g + 3 * NG < total) { fetch(pf, rb); advance(pf, NG); }
                 }
             }
         } else if (!DIRECT) {
@@ -685,7 +688,7 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     if (grid > 2 * tiles) grid = 2 * tiles;
 #define QLESS_LAUNCH_SCORE_TC(B)                                                                                    \
     QLESS_CUDA_TRY(cudaFuncSetAttribute(score_tc_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-    score_tc_kernel<B><<<(unsigned)grid, NTHREADS, smem, st>>>(tm_train, tm_v1, tm_v2, p);
+    score_tc_kernel<B><<<(unsigned)grid, (B <= 2 ? NTHREADS_FP4 : NTHREADS), smem, st>>>(tm_train, tm_v1, tm_v2, p);
     if (a.bits == 16) { QLESS_LAUNCH_SCORE_TC(16) }
     else if (a.bits == 8) { QLESS_LAUNCH_SCORE_TC(8) }
     else if (a.bits == 4) { QLESS_LAUNCH_SCORE_TC(4) }
