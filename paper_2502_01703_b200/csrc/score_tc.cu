@@ -41,7 +41,9 @@ constexpr int KB = 128;                    // codes (= unpacked bytes) per row p
 constexpr int A_STAGE = TM * KB;           // 16 KiB
 constexpr int MAX_STAGES = 8;
 constexpr int NTHREADS = 448;
-constexpr int NTHREADS_FP4 = 576;          // 2- and 1-bit codes: a third group of four unpack warps (14-17)
+// 2- and 1-bit codes: NG groups of four unpack warps (2-5, 10-13, 14-17, ...) and, behind them, four more epilogue warps
+__host__ __device__ constexpr int fp4_groups(int bits) { return bits == 1 ? 3 : 4; }
+__host__ __device__ constexpr int fp4_threads(int bits) { return NTHREADS + 128 * (fp4_groups(bits) - 2) + 128; }
 constexpr int TMAX = 8;                    // tasks held in registers by the epilogue
 constexpr int A_TMEM_COL = 448;            // sub-byte widths: two 32-column slots of unpacked train codes
 
@@ -133,7 +135,7 @@ __host__ __device__ constexpr uint32_t make_idesc_mxf4(uint32_t M, uint32_t N)
 }
 
 template <int BITS>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(BITS <= 2 ? NTHREADS_FP4 : NTHREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(BITS <= 2 ? fp4_threads(BITS) : NTHREADS, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_constant__ CUtensorMap tmap_val1,
                 const __grid_constant__ CUtensorMap tmap_val2, const ScoreTcParams p)
 {
@@ -326,7 +328,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
             mma_commit_pair(smem_u32(&bars->drain));
             mbar_wait_quiet(smem_u32(&bars->drain), 0u);
         }
-    } else if (!DIRECT && (warp < 6 || warp >= 10)) {
+    } else if (!DIRECT && (warp < 6 || (warp >= 10 && (!FP4 || warp < 10 + 4 * (fp4_groups(BITS) - 1))))) {
         // ------------------------------- unpack warps (4- and 2-bit train codes) -------------------------------
         // two groups of four warps (2-5 and 10-13) take alternate K blocks, so that the barrier round trips of
         // one block overlap the unpacking of the next
@@ -336,8 +338,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
             // e2m1 and writes the row into operand stage s of this CTA's shared memory as the MMA reads a K-major operand
             // with the 128-byte swizzle (what a TMA load would have written): 16-byte piece j of row r at piece j ^ (r & 7).
             const int row = ((warp - 2) & 3) * 32 + lane;
-            constexpr int NG = 3;                                 // groups of four warps: 2-5, 10-13, 14-17; group g takes K blocks g, g + 3, ...
-            const uint32_t grp = (warp >= 14) ? 2u : (warp >= 10) ? 1u : 0u;
+            constexpr int NG = fp4_groups(BITS);                  // groups of four warps: 2-5, 10-13, 14-17, ...; group g takes K blocks g, g + NG, ...
+            const uint32_t grp = (warp >= 10) ? (uint32_t)((warp - 6) >> 2) : 0u;
             constexpr int NV = PROW >= 16 ? PROW / 16 : 1;       // (this branch is compiled for every width)
             const int64_t my_tiles = (num_tiles > pair) ? (num_tiles - pair + num_pairs - 1) / num_pairs : 0;
             const int64_t total = my_tiles * num_vt * p.C * nkb;
@@ -463,13 +465,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 if (lane == 0) mbar_arrive_leader_tmem(smem_u32(&bars->full[s]), rank);
             }
         }
-    } else if (warp >= 6 && warp < 10 || (warp < 6 && p.epi_groups == 2)) {
+    } else if ((warp >= 6 && warp < 10) || ((FP4 ? warp >= 10 : warp < 6) && p.epi_groups == 2)) {
         // ------------------------------- epilogue -------------------------------
         // warps 6-9 (group 0) and, for 8-bit codes where they have nothing to unpack, warps 2-5 (group 1): with two
         // groups each reads half of the accumulator's columns, which halves the time the tensor pipe waits for it
         const int q = warp & 3;
         const int tl = q * 32 + lane;                        // row of the tile = TMEM lane
-        const int eg = (warp >= 6) ? 0 : 1;
+        const int eg = (warp >= 6 && warp < 10) ? 0 : 1;
         const int et = eg * 128 + tl;                        // index among the epilogue threads
         const int nthr_e = 128 * p.epi_groups;
         const int nch = (p.vpad + 31) / 32;                  // 32-column chunks of the accumulator
@@ -650,7 +652,7 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     if (a.bits >= 8) nS &= ~1;                              // stages are handed to the MMAs in pairs
     QLESS_REQUIRE(nS >= 3, QLESS_ERR_UNSUPPORTED, "internal: not enough shared memory for two pipeline stages");
     p.nS = nS; p.nP = nP > 0 ? nP : 1;
-    p.epi_groups = (a.bits >= 8 && a.T <= 6) ? 2 : 1;
+    p.epi_groups = ((a.bits >= 8 || fp4) && a.T <= 6) ? 2 : 1;      // the second group: idle unpack warps (8-bit), four more warps (2-, 1-bit)
     const size_t smem = 1024 + (size_t)nS * stage + (size_t)nP * p_stage + sizeof(ScoreBars);
 
     p.train_codes = a.train; p.train_stride = a.C > 1 ? a.train_stride : 0;
@@ -688,7 +690,7 @@ qless_status launch_score_tc(const ScoreArgs& a, uint8_t* val_unpacked, unsigned
     if (grid > 2 * tiles) grid = 2 * tiles;
 #define QLESS_LAUNCH_SCORE_TC(B)                                                                                    \
     QLESS_CUDA_TRY(cudaFuncSetAttribute(score_tc_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-    score_tc_kernel<B><<<(unsigned)grid, (B <= 2 ? NTHREADS_FP4 : NTHREADS), smem, st>>>(tm_train, tm_v1, tm_v2, p);
+    score_tc_kernel<B><<<(unsigned)grid, (B <= 2 ? fp4_threads(B) : NTHREADS), smem, st>>>(tm_train, tm_v1, tm_v2, p);
     if (a.bits == 16) { QLESS_LAUNCH_SCORE_TC(16) }
     else if (a.bits == 8) { QLESS_LAUNCH_SCORE_TC(8) }
     else if (a.bits == 4) { QLESS_LAUNCH_SCORE_TC(4) }
