@@ -328,10 +328,17 @@ def stage_measurements(torch, B, W, dev, peaks):
     bf16_peak = ops / ms / 1e9          # TFLOP/s
     ms, ops = B.qless_microbench("i8_ss_pair_n448", 20000, device=dev)
     i8_n448 = ops / ms / 1e9            # Tops/s in the two-MMA shape of 8-bit scoring at 448 validation vectors
+    # e2m1 operands (kind::mxf4, unit scale factors), the path of 2- and 1-bit scoring: the two-MMA shape with both operands
+    # in shared memory (what the kernel issues), and with A in tensor memory (for which a 448-column accumulator leaves no room)
+    ms, ops = B.qless_microbench("fp4_ss_pair_n448", 20000, device=dev)
+    fp4_n448 = ops / ms / 1e9
+    ms, ops = B.qless_microbench("fp4_ts_pair", 20000, device=dev)
+    fp4_ts = ops / ms / 1e9
     ms, byts = B.qless_microbench("tma_l2_stream", 20000, device=dev)
     l2_gbs = byts / ms / 1e6            # GB/s from L2 into shared memory, TMA alone
     out["microbench"] = dict(int8_tops=i8_peak, popc_xor_add_twordops=popc_peak, bf16_tcgen05_tflops=bf16_peak,
-                             int8_tops_scoring_shape_n448=i8_n448, tma_l2_to_smem_gbs=l2_gbs,
+                             int8_tops_scoring_shape_n448=i8_n448, fp4_tops_scoring_shape_n448=fp4_n448,
+                             fp4_tops_a_in_tensor_memory=fp4_ts, tma_l2_to_smem_gbs=l2_gbs,
                              note="back-to-back tcgen05.mma / XOR+POPC+IADD on all SMs, burst; TMA streaming from an L2-resident buffer")
     # the same int8 micro-benchmark held for about two seconds, clocks sampled: the tensor pipe under the power cap
     smp = ClockSampler(torch.cuda.current_device())
@@ -340,6 +347,12 @@ def stage_measurements(torch, B, W, dev, peaks):
     ck = smp.stop()
     i8_sustained = ops / ms / 1e9
     out["microbench"].update(int8_tops_sustained=i8_sustained, int8_sustained_clocks=ck)
+    smp = ClockSampler(torch.cuda.current_device())
+    smp.start()
+    ms, ops = B.qless_microbench("fp4_ss_pair_n448", 2_000_000, device=dev)
+    ck4 = smp.stop()
+    fp4_sustained = ops / ms / 1e9
+    out["microbench"].update(fp4_tops_scoring_shape_sustained=fp4_sustained, fp4_sustained_clocks=ck4)
     # the int8 MMAs of 8-bit scoring reading, for every K block, operands that TMA has just streamed from a buffer of
     # pseudo-random int8 values: the tensor pipe on data that changes, held for about two seconds with the clocks
     # sampled. This is the sustained figure a scoring kernel can be held against: same shape, same data statistics,
@@ -405,7 +418,10 @@ def stage_measurements(torch, B, W, dev, peaks):
         e = dict(ms=t, scores_per_s=N * V / (t * 1e-3), pair_dots_per_s=N * V * C / (t * 1e-3))
         iops = 2.0 * N * V * C * d
         e.update(bound="tensor", achieved_tops=iops / t / 1e9, frac_of_int8_peak=iops / t / 1e9 / i8_peak,
+                 tensor_path="e2m1 (kind::mxf4, unit scales)" if b <= 2 else "int8 (kind::i8)",
                  store_gb=C * (N + V) * (d * b // 8 + 8) / 1e9)
+        if b <= 2:
+            e.update(frac_of_fp4_peak=iops / t / 1e9 / fp4_n448)
         # the same call repeated for over a second with the clocks sampled, against the sustained micro-benchmark
         smp = ClockSampler(torch.cuda.current_device())
         smp.start()
@@ -416,9 +432,13 @@ def stage_measurements(torch, B, W, dev, peaks):
             sc_1bit = sc.clone()        # for the selected-percentage sweep below
         e.update(ms_sustained=ts_, frac_of_int8_sustained=iops / ts_ / 1e9 / i8_sustained, sustained_clocks=ck,
                  frac_of_int8_random_operands_sustained=iops / ts_ / 1e9 / i8_random)
+        if b <= 2:
+            e.update(frac_of_fp4_sustained=iops / ts_ / 1e9 / fp4_sustained)
         if ck.get("sm_mhz"):
             # against what the hardware's unit count allows at the SM clock this very loop was granted
-            e.update(frac_of_hw_int8_at_sampled_clock=iops / ts_ / 1e9 / (sms * HW_INT8_OP_PER_CLK_SM * ck["sm_mhz"] * 1e6 / 1e12))
+            hw_ops = HW_FP4_OP_PER_CLK_SM if b <= 2 else HW_INT8_OP_PER_CLK_SM
+            e.update({"frac_of_hw_fp4_at_sampled_clock" if b <= 2 else "frac_of_hw_int8_at_sampled_clock":
+                      iops / ts_ / 1e9 / (sms * hw_ops * ck["sm_mhz"] * 1e6 / 1e12)})
         if ck.get("sm_mhz") and ck.get("sm_max_mhz"):
             # the micro-benchmark holds the maximum clock (its operands never change, so it draws little power); the
             # scoring kernel runs under the power cap: its rate against the tensor peak at the clock it actually had
@@ -517,6 +537,8 @@ def stage_measurements(torch, B, W, dev, peaks):
     iops = 2.0 * N * V * C * d
     out["score_c4_2000000x448x4_1bit"] = dict(ms=t, scores_per_s=N * V / (t * 1e-3), bound="tensor",
                                               achieved_tops=iops / t / 1e9, frac_of_int8_peak=iops / t / 1e9 / i8_peak,
+                                              frac_of_fp4_peak=iops / t / 1e9 / fp4_n448, frac_of_fp4_sustained=iops / t / 1e9 / fp4_sustained,
+                                              tensor_path="e2m1 (kind::mxf4, unit scales)",
                                               frac_of_int8_random_operands_sustained=iops / t / 1e9 / i8_random)
     # the same store through the XOR + population-count kernel (CUDA cores), against the integer-ALU peak
     B.qless_set_score_path(1)
@@ -570,6 +592,7 @@ def stage_measurements(torch, B, W, dev, peaks):
 # clock per SM (the unit counts behind the nominal 2.25 / 4.5 Pop/s at the nominal clock); times the SM count and a clock.
 HW_BF16_FLOP_PER_CLK_SM = 8192.0
 HW_INT8_OP_PER_CLK_SM = 16384.0
+HW_FP4_OP_PER_CLK_SM = 32768.0         # block-scaled e2m1: twice the int8 count (nominal 9 Pop/s dense)
 
 
 def roofline_entry(achieved_tflops, peaks, clocks, sm_count=148):
@@ -596,8 +619,9 @@ def summarize(stages, cpu, peaks, step_kernels_ms):
         return {k: e[k] for k in keys if k in e}
     c3 = stages.get("score_c3_270000x448x4", {})
     scoring = {"c3": {}, "c4": {}}
-    keys = ("ms", "scores_per_s", "frac_of_int8_peak", "frac_of_int8_sustained", "frac_of_int8_random_operands_sustained",
-            "frac_of_hw_int8_at_sampled_clock", "frac_of_popc_peak", "frac_of_bf16_peak")
+    keys = ("ms", "scores_per_s", "tensor_path", "frac_of_int8_peak", "frac_of_int8_sustained", "frac_of_int8_random_operands_sustained",
+            "frac_of_hw_int8_at_sampled_clock", "frac_of_fp4_peak", "frac_of_fp4_sustained", "frac_of_hw_fp4_at_sampled_clock",
+            "frac_of_popc_peak", "frac_of_bf16_peak")
     for b in ("8", "4", "2", "1", "1_popc", "16"):
         if b in c3:
             scoring["c3"][b] = pick(c3[b], keys)
@@ -609,6 +633,8 @@ def summarize(stages, cpu, peaks, step_kernels_ms):
     out = dict(scoring=scoring,
                peaks=dict(int8_tops_burst=mb.get("int8_tops"), int8_tops_sustained=mb.get("int8_tops_sustained"),
                           int8_tops_random_operands_sustained=mb.get("int8_tops_random_operands_sustained"),
+                          fp4_tops_scoring_shape=mb.get("fp4_tops_scoring_shape_n448"), fp4_tops_scoring_shape_sustained=mb.get("fp4_tops_scoring_shape_sustained"),
+                          fp4_tops_a_in_tensor_memory=mb.get("fp4_tops_a_in_tensor_memory"),
                           popc_twordops=mb.get("popc_xor_add_twordops"), bf16_tcgen05_tflops=mb.get("bf16_tcgen05_tflops"),
                           hbm_gbs=peaks["hbm_gbs"], source="library micro-benchmarks (tcgen05 int8, XOR+POPC+IADD); HBM: " + peaks["source"]),
                quantize_65536x8192={b: pick(e, ("ms", "frac_of_hbm")) for b, e in stages.get("quantize_65536x8192", {}).items()},

@@ -100,7 +100,9 @@ qless_status qless_profile_collect(char* buf /* host */, size_t buflen);
  * MMAs'); 11 = the kernel of 10 with the copies switched off; 12 = the MMAs of 8 reading, for every K block, a
  * stage that TMA has just brought from the scratch buffer (same scratch size; the CALLER fills it with the int8
  * values the operands are to take, e.g. pseudo-random ones: the operands then change with every K block, which
- * is what sets the power drawn and so the clock granted under the power cap). Runs the kernel twice and times
+ * is what sets the power drawn and so the clock granted under the power cap); 13 = the shape of 8 on e2m1 operands
+ * (tcgen05.mma kind::mxf4 with unit scale factors, 64 codes per MMA, both operands in shared memory), which is what
+ * 2- and 1-bit scoring issues; 14 = e2m1 on CTA pairs with A in tensor memory, N = 256. Runs the kernel twice and times
  * the second run with CUDA events on `cuda_stream` (synchronises it). *ms_out: milliseconds; *ops_out:
  * operations executed (2 x multiply-accumulates; word operations for 6; bytes moved for 9). Host pointers. */
 qless_status qless_microbench(int32_t what, int32_t iters, float* ms_out, double* ops_out, void* scratch,
@@ -206,8 +208,8 @@ qless_status qless_project_quantize_host_ex(
 qless_status qless_set_projection_path(int32_t path);
 
 /* As above, for the integer similarity in qless_score and qless_score_dots: 0 (default) the
- * tcgen05 int8 kernel for every code width (used when T <= 8; sub-byte codes, sign bits included, are expanded
- * to int8 on the way), 1 the CUDA-core kernels (dp4a for 8-, 4- and 2-bit codes, XOR + population count for
+ * tcgen05 kernel for every code width (used when T <= 8; int8 operands for 8- and 4-bit codes, e2m1 operands with
+ * unit scale factors for 2-bit codes and sign bits, whose values e2m1 holds exactly), 1 the CUDA-core kernels (dp4a for 8-, 4- and 2-bit codes, XOR + population count for
  * 1-bit codes). */
 qless_status qless_set_score_path(int32_t path);
 

@@ -436,7 +436,8 @@ def qless_set_score_path(path):
 
 
 MICROBENCH = {"bf16_ss": 0, "bf16_ts": 1, "i8_ss": 2, "bf16_ss_pair": 3, "bf16_ts_pair": 4, "i8_ss_pair": 5, "popc": 6, "i8_ts_pair": 7,
-              "i8_ss_pair_n448": 8, "tma_l2_stream": 9, "i8_n448_with_tma": 10, "i8_n448_commit_per_block": 11, "i8_n448_streamed_operands": 12}
+              "i8_ss_pair_n448": 8, "tma_l2_stream": 9, "i8_n448_with_tma": 10, "i8_n448_commit_per_block": 11, "i8_n448_streamed_operands": 12,
+              "fp4_ss_pair_n448": 13, "fp4_ts_pair": 14}
 
 
 def qless_microbench(what, iters, device="cuda", stream=None, scratch=None):

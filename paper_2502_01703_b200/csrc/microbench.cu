@@ -16,7 +16,9 @@ struct __align__(8) MbBars { uint64_t done; uint32_t tmem_base; uint32_t abort_f
 
 // KIND: 0 = bf16 A,B in shared memory; 1 = bf16 A in tensor memory; 2 = int8 A,B in shared memory;
 //       3 = int8 A in tensor memory; 4 = int8 A,B in shared memory in the shape the 8-bit scoring kernel issues
-//       for 448 validation vectors (pair only): per K step one MMA of N = 256 and one of N = 192 on the same A.
+//       for 448 validation vectors (pair only): per K step one MMA of N = 256 and one of N = 192 on the same A;
+//       5 = e2m1 (kind::mxf4, unit scale factors, 64 codes per MMA) A,B in shared memory in the same two-MMA shape, as the
+//       2- and 1-bit scoring kernel issues them (pair only); 6 = e2m1 with A in tensor memory, N = 256 (pair only).
 // PAIR: 0 = one CTA per 128 x 256 tile; 1 = CTA pair per 256 x 256 tile (cta_group::2).
 template <int KIND, int PAIR>
 __global__ void __launch_bounds__(128, 1)
@@ -25,7 +27,8 @@ mma_peak_kernel(int iters, unsigned int* timeout_word)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     constexpr int A_BYTES = 128 * 128;                      // 128 rows x 128 bytes (one swizzle panel)
-    constexpr int B_BYTES = (KIND == 4 ? 224 : PAIR ? 128 : 256) * 128;
+    constexpr int B_BYTES = ((KIND == 4 || KIND == 5) ? 224 : PAIR ? 128 : 256) * 128;
+    constexpr uint32_t SF_COL = 448;                        // e2m1 kinds: 16 columns of unit scale factors (0x7F in every byte)
     uint8_t* sA = smem;
     uint8_t* sB = smem + A_BYTES;
     MbBars* bars = reinterpret_cast<MbBars*>(sB + B_BYTES);
@@ -33,8 +36,9 @@ mma_peak_kernel(int iters, unsigned int* timeout_word)
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
 
     for (int i = threadIdx.x; i < (A_BYTES + B_BYTES) / 4; i += blockDim.x)
-        reinterpret_cast<uint32_t*>(smem)[i] = (KIND >= 2) ? (0x01FF02FEu ^ (uint32_t)(i * 0x01010101u & 0x03030303u))
-                                                            : ((i & 1) ? 0x3F80BF80u : 0xBF803F80u);
+        reinterpret_cast<uint32_t*>(smem)[i] = (KIND >= 5) ? ((i & 1) ? 0x2AA2A22Au : 0xA22A2AA2u)      // e2m1 codes +-1
+                                               : (KIND >= 2) ? (0x01FF02FEu ^ (uint32_t)(i * 0x01010101u & 0x03030303u))
+                                                             : ((i & 1) ? 0x3F80BF80u : 0xBF803F80u);
     if (threadIdx.x == 0) { mbar_init(smem_u32(&bars->done), 1); bars->abort_flag = 0; fence_barrier_init(); }
     if (warp == 0) {
         if (PAIR) { tmem_alloc_pair(smem_u32(&bars->tmem_base), 512); tmem_relinquish_pair(); }
@@ -46,14 +50,23 @@ mma_peak_kernel(int iters, unsigned int* timeout_word)
     if (PAIR) cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
-    if (KIND == 1 || KIND == 3) {                           // A operand: 64 columns (bf16 +-1.0 pairs, or small int8) in every lane
+    if (KIND >= 5) {
+        uint32_t v[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) v[k] = 0x7F7F7F7Fu;
+        tmem_st_x16(tmem_base + ((uint32_t)(warp * 32) << 16) + SF_COL, v);
+        tmem_wait_st();
+        tc_fence_before();
+    }
+    if (KIND == 1 || KIND == 3 || KIND == 6) {              // A operand: 64 columns (bf16 +-1.0 pairs, small int8, or e2m1 +-1) in every lane
         const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + 256;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             uint32_t v[16];
 #pragma unroll
-            for (int k = 0; k < 16; ++k) v[k] = (KIND == 3) ? (0x01FF02FEu ^ (uint32_t)((lane + k) & 3) * 0x01010101u)
-                                                            : (((lane + k) & 1) ? 0x3F80BF80u : 0xBF803F80u);
+            for (int k = 0; k < 16; ++k) v[k] = (KIND == 6) ? (((lane + k) & 1) ? 0x2AA2A22Au : 0xA22A2AA2u)
+                                                : (KIND == 3) ? (0x01FF02FEu ^ (uint32_t)((lane + k) & 3) * 0x01010101u)
+                                                              : (((lane + k) & 1) ? 0x3F80BF80u : 0xBF803F80u);
             tmem_st_x16(taddr + c * 16, v);
         }
         tmem_wait_st();
@@ -84,6 +97,13 @@ mma_peak_kernel(int iters, unsigned int* timeout_word)
                     else mma_f16_ts(tmem_base, tmem_base + 256 + 8 * k, bdesc + (uint64_t)(2 * k), idesc, acc);
                 } else if (KIND == 3) {
                     if (PAIR) mma_i8_ts_pair(tmem_base, tmem_base + 256 + 8 * k, bdesc + (uint64_t)(2 * k), idesc, acc);
+                } else if (KIND == 5) {
+                    if (PAIR) {
+                        mma_mxf4_ss_pair(tmem_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), make_idesc_mxf4(256, 256), tmem_base + SF_COL, acc);
+                        mma_mxf4_ss_pair(tmem_base + 256, adesc + (uint64_t)(2 * k), bdesc192 + (uint64_t)(2 * k), make_idesc_mxf4(256, 192), tmem_base + SF_COL, acc);
+                    }
+                } else if (KIND == 6) {
+                    if (PAIR) mma_mxf4_ts_pair(tmem_base, tmem_base + 256 + 8 * k, bdesc + (uint64_t)(2 * k), make_idesc_mxf4(256, 256), tmem_base + SF_COL, acc);
                 } else if (KIND == 4) {
                     if (PAIR) {
                         mma_i8_ss_pair(tmem_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, acc);
@@ -390,7 +410,7 @@ extern "C" qless_status qless_microbench(int32_t what, int32_t iters, float* ms_
             if (what == 0) { QLESS_MB_LAUNCH(0) } else if (what == 1) { QLESS_MB_LAUNCH(1) } else { QLESS_MB_LAUNCH(2) }
 #undef QLESS_MB_LAUNCH
             ops = (double)sms * iters * 4.0 * 2.0 * 128 * 256 * (what == 2 ? 32 : 16);
-        } else if ((what >= 3 && what <= 5) || what == 7 || what == 8) {
+        } else if ((what >= 3 && what <= 5) || what == 7 || what == 8 || what == 13 || what == 14) {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3((unsigned)(sms / 2 * 2)); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = smem; cfg.stream = st;
             cudaLaunchAttribute attr; attr.id = cudaLaunchAttributeClusterDimension; attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
@@ -399,9 +419,11 @@ extern "C" qless_status qless_microbench(int32_t what, int32_t iters, float* ms_
             err = cudaFuncSetAttribute(mma_peak_kernel<K, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
             if (err == cudaSuccess) err = cudaLaunchKernelEx(&cfg, mma_peak_kernel<K, 1>, (int)iters, flag);
             if (what == 3) { QLESS_MB_LAUNCH(0) } else if (what == 4) { QLESS_MB_LAUNCH(1) } else if (what == 5) { QLESS_MB_LAUNCH(2) }
-            else if (what == 7) { QLESS_MB_LAUNCH(3) } else { QLESS_MB_LAUNCH(4) }
+            else if (what == 7) { QLESS_MB_LAUNCH(3) } else if (what == 8) { QLESS_MB_LAUNCH(4) } else if (what == 13) { QLESS_MB_LAUNCH(5) }
+            else { QLESS_MB_LAUNCH(6) }
 #undef QLESS_MB_LAUNCH
-            ops = (double)(sms / 2) * iters * 4.0 * 2.0 * 256 * (what == 8 ? 448 : 256) * (what == 5 || what == 7 || what == 8 ? 32 : 16);
+            ops = (double)(sms / 2) * iters * 4.0 * 2.0 * 256 * ((what == 8 || what == 13) ? 448 : 256) *
+                  (what >= 13 ? 64 : (what == 5 || what == 7 || what == 8) ? 32 : 16);
         } else if (what == 6) {
             const size_t need = (size_t)sms * 8 * 256 * sizeof(uint32_t);
             QLESS_REQUIRE(scratch != nullptr && scratch_bytes >= need, QLESS_ERR_WORKSPACE, "scratch of %zu bytes required", need);

@@ -1,32 +1,41 @@
-// Stage 3 on the tensor cores (tcgen05.mma kind::i8, int32 accumulators in TMEM) for every code width: 8-bit
-// codes as they are, 4-, 2- and 1-bit codes (sign bits as +-1) expanded to int8 on the way.
+// Stage 3 on the tensor cores for every code width. 8- and 4-bit codes: tcgen05.mma kind::i8, int32 accumulators in
+// TMEM (4-bit codes expanded to int8 on the way). 2- and 1-bit codes: the codes -2 .. 1 and the signs +-1 are exact
+// e2m1 values, so they run on the block-scaled fp4 path (kind::mxf4 with every scale factor 2^0, 64 codes per
+// instruction instead of 32, fp32 accumulation of integers no larger than 4 d: exact), at twice the int8 rate.
 //
 // Two CTAs on neighbouring SMs form a pair (cta_group::2) and own a tile of 256 train rows (UMMA M), 128
 // per CTA. For each checkpoint the pair streams the tile's codes and the validation codes K-block by
-// K-block (128 codes = 128 bytes per row per block, 128-byte-swizzled K-major operands) and accumulates
-// D[t, v] = sum_m q_t,m q_v,m for up to 512 validation vectors at once (two MMAs of N <= 256 per K step);
-// each CTA stages only half of the validation rows of every MMA, which halves what an SM pulls from L2.
-// After the last K block of a checkpoint the epilogue warps of each CTA read their half of the accumulator
-// (thread = train row), apply the per-vector multipliers (Eq. 6), form the per-task means and add
+// K-block (128 operand bytes per row per block: 128 int8 codes or 256 e2m1 codes, 128-byte-swizzled K-major
+// operands) and accumulates D[t, v] = sum_m q_t,m q_v,m for up to 512 validation vectors at once (two MMAs of
+// N <= 256 per K step); each CTA stages only half of the validation rows of every MMA, which halves what an SM
+// pulls from L2. After the last K block of a checkpoint the epilogue warps of each CTA read their half of the
+// accumulator (thread = train row), apply the per-vector multipliers (Eq. 6), form the per-task means and add
 // eta_i * mean to the running per-task sums; after the last checkpoint they take the max over tasks.
 // The N x V x C similarity tensor never exists in memory.
 //
-// 8-bit train codes go from global memory to the MMA operand buffer by TMA. 4-, 2- and 1-bit train codes
-// arrive packed (TMA, no swizzle) in a staging ring; unpack warps (thread = train row = TMEM lane)
-// sign-extend them to int8 and store them straight into tensor memory, from where the MMA takes its A
-// operand: no shared-memory write, no swizzle, no proxy fence. The accumulator leaves 64 of the 512 TMEM
-// columns free, enough for two 128-code blocks of A, so at these widths a validation tile holds at most 448
-// vectors. Validation codes are unpacked once per call into a workspace (they are a few MB and stay in L2).
-// Inside a 128-code block the unpackers place the codes in a fixed permutation, the same for both
-// operands, which an inner product does not see.
+// 8-bit train codes go from global memory to the MMA operand buffer by TMA. 4-bit train codes arrive packed (TMA,
+// no swizzle) in a staging ring; unpack warps (thread = train row = TMEM lane) sign-extend them to int8 and store
+// them straight into tensor memory, from where the MMA takes its A operand: no shared-memory write, no swizzle, no
+// proxy fence. The accumulator leaves 64 of the 512 TMEM columns free, enough for two 128-code blocks of A, so at
+// the sub-byte widths a validation tile holds at most 448 vectors. 2- and 1-bit train codes: the block-scaled MMA
+// also reads its scale factors from tensor memory (8 columns), which a 448-column accumulator and two A slots leave
+// no room for, so the unpack warps (three or four groups of four, each thread a row) take the packed codes straight
+// from global memory (32 or 64 bytes per row and K block, whole sectors, two blocks ahead in registers), expand
+// them to e2m1 and write the row into the operand stage in shared memory in the swizzled layout a TMA load would
+// have produced (a proxy fence and, from the peer CTA, a cluster-scope release per warp and block).
+// Validation codes are expanded once per call into a workspace (they are a few MB and stay in L2). Inside a
+// 128-code block the 4-bit unpackers place the codes in a fixed permutation, the same for both operands, which an
+// inner product does not see; the e2m1 codes stay in order.
 //
 // One barrier per pipeline stage on the leader CTA collects everything the MMAs of that stage need (TMA
 // bytes of both CTAs, and the unpack warps' arrivals); one tcgen05.commit releases the stage in both CTAs:
 // the single MMA-issuing thread runs at the tensor pipe's own pace, so every other instruction it executes
 // is lost tensor time.
 //
-// Warp roles (448 threads per CTA): warp 0 TMA producer, warp 1 MMA issuer (leader only; + TMEM
-// allocation), warps 2-5 and 10-13 unpack (idle for 8-bit), warps 6-9 epilogue. All waits are bounded.
+// Warp roles (448 threads per CTA; 704 / 832 for 1- / 2-bit codes): warp 0 TMA producer, warp 1 MMA issuer (leader
+// only; + TMEM allocation), warps 2-5 and 10-13 unpack (idle for 8-bit, where 2-5 form a second epilogue group),
+// warps 6-9 epilogue; 2- and 1-bit codes add unpack warps 14-17 (and 18-21 at 2 bits) and behind them four more
+// epilogue warps that take half of the accumulator's columns. All waits are bounded.
 #include "qless_kernels.h"
 #include "tc_common.cuh"
 
@@ -112,26 +121,6 @@ __device__ __forceinline__ void fp4_from_codes2(uint32_t w, uint32_t& lo, uint32
 {
     lo = fp4_from_nibble_codes2(spread2_to_nibbles(w & 0xFFFFu));
     hi = fp4_from_nibble_codes2(spread2_to_nibbles(w >> 16));
-}
-
-// Pair MMA on e2m1 operands (kind::mxf4, block-scaled, 64 codes per instruction, fp32 accumulation), both operands from
-// shared memory. The scale factors (one UE8M0 byte per 32 codes of a row) are all 2^0: every byte of the tensor-memory
-// columns at sf_tmem is 0x7F, so the layout in which the instruction reads them does not matter.
-__device__ __forceinline__ void mma_mxf4_ss_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t sf_tmem,
-                                                 uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%5], p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sf_tmem)
-        : "memory");
-}
-// Instruction descriptor of kind::mxf4: A and B format e2m1 (1) at bits [7,10) and [10,13), K-major, N/8 at [17,23),
-// scale format UE8M0 (1) at bit 23, M/16 at [24,29), scale-factor byte offsets 0.
-__host__ __device__ constexpr uint32_t make_idesc_mxf4(uint32_t M, uint32_t N)
-{
-    return (1u << 7) | (1u << 10) | ((N >> 3) << 17) | (1u << 23) | ((M >> 4) << 24);
 }
 
 template <int BITS>

@@ -217,6 +217,37 @@ __device__ __forceinline__ void mma_i8_ts_pair(uint32_t d_tmem, uint32_t a_tmem,
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// Pair MMA on e2m1 operands (kind::mxf4, block-scaled, 64 codes per instruction, fp32 accumulation), both operands from
+// shared memory. The scale factors (one UE8M0 byte per 32 codes of a row) are all 2^0: every byte of the tensor-memory
+// columns at sf_tmem is 0x7F, so the layout in which the instruction reads them does not matter.
+__device__ __forceinline__ void mma_mxf4_ss_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t sf_tmem,
+                                                 uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%5], p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sf_tmem)
+        : "memory");
+}
+// Instruction descriptor of kind::mxf4: A and B format e2m1 (1) at bits [7,10) and [10,13), K-major, N/8 at [17,23),
+// scale format UE8M0 (1) at bit 23, M/16 at [24,29), scale-factor byte offsets 0.
+__host__ __device__ constexpr uint32_t make_idesc_mxf4(uint32_t M, uint32_t N)
+{
+    return (1u << 7) | (1u << 10) | ((N >> 3) << 17) | (1u << 23) | ((M >> 4) << 24);
+}
+
+// The same with A in tensor memory (lane = row, eight codes per 32-bit column, code j of them in bits [4j, 4j + 4)).
+__device__ __forceinline__ void mma_mxf4_ts_pair(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t sf_tmem,
+                                                 uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], [%1], %2, %3, [%5], [%5], p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sf_tmem)
+        : "memory");
+}
 // Arrive, once every MMA issued so far has completed, on the barrier at this offset in BOTH CTAs of the pair.
 __device__ __forceinline__ void mma_commit_pair(uint32_t bar)
 {

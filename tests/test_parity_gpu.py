@@ -420,6 +420,19 @@ def test_score_dots_bit_exact(bits, N, V, d):
 
 
 @pytest.mark.parametrize("bits", [8, 4, 2, 1])
+@pytest.mark.parametrize("N,V,d", [(300, 449, 8192), (77, 33, 384)])
+def test_score_dots_of_arbitrary_code_bytes(bits, N, V, d):
+    # every bit pattern is a code: the most negative value of each width (-2 at 2 bits, which the quantiser never emits
+    # and the e2m1 operand path has to map to its own -2), d not a multiple of the 256-code K block, two validation tiles
+    gen = torch.Generator(device=DEV); gen.manual_seed(77 + bits)
+    tc = torch.randint(0, 256, (N, d * bits // 8), generator=gen, device=DEV, dtype=torch.uint8)
+    vc = torch.randint(0, 256, (V, d * bits // 8), generator=gen, device=DEV, dtype=torch.uint8)
+    got = _np(B.qless_score_dots(tc, vc, d, bits))
+    want = oracle.dots(_np(tc), _np(vc), d, bits)
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("bits", [8, 4, 2, 1])
 @pytest.mark.parametrize("mode", [B.COSINE, B.DEQUANT])
 def test_scores_match_oracle(bits, mode):
     C, N, V, d = 3, 333, 100, 512
