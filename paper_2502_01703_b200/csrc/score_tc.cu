@@ -51,7 +51,7 @@ constexpr int A_STAGE = TM * KB;           // 16 KiB
 constexpr int MAX_STAGES = 8;
 constexpr int NTHREADS = 448;
 // 2- and 1-bit codes: NG groups of four unpack warps (2-5, 10-13, 14-17, ...) and, behind them, four more epilogue warps
-__host__ __device__ constexpr int fp4_groups(int bits) { return bits == 1 ? 3 : 4; }
+__host__ __device__ constexpr int fp4_groups(int bits) { return 3; }
 __host__ __device__ constexpr int fp4_threads(int bits) { return NTHREADS + 128 * (fp4_groups(bits) - 2) + 128; }
 constexpr int TMAX = 8;                    // tasks held in registers by the epilogue
 constexpr int A_TMEM_COL = 448;            // sub-byte widths: two 32-column slots of unpacked train codes
@@ -81,6 +81,7 @@ struct __align__(8) ScoreBars {
     uint32_t tmem_base, abort_flag;
     int32_t task_off[65];
     __align__(16) float mv[512];
+    float eta_s[TMAX];          // this checkpoint's eta_i / |task j|
     float comb[TM][6];          // per-task partial sums handed from the second epilogue group to the first
 };
 
@@ -372,7 +373,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                 }
                 const int s = (int)st_ring.slot;
                 // the stage is free once the MMAs of its previous use have completed (the commit arrives in both CTAs)
-                bool w = mbar_wait(smem_u32(&bars->empty[s]), st_ring.parity ^ 1u, abort_flag, p.timeout_word, TO_UNPACK);
+                bool w = mbar_wait_parked(smem_u32(&bars->empty[s]), st_ring.parity ^ 1u, abort_flag, p.timeout_word, TO_UNPACK);
                 w = __all_sync(0xFFFFFFFFu, w);
                 if (!w) return false;
                 uint4* dst = reinterpret_cast<uint4*>(sS + (size_t)s * stage_bytes + (size_t)row * KB);
@@ -481,14 +482,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                         // this checkpoint's validation multipliers -> shared memory (epilogue threads only)
                         asm volatile("bar.sync 1, %0;" ::"r"(nthr_e) : "memory");
                         for (int v = et; v < p.vpad; v += nthr_e) bars->mv[v] = (v < vcount) ? p.val_mult[(int64_t)i * p.V + v0 + v] : 0.0f;
+                        if (et < p.T) bars->eta_s[et] = p.eta_over_cnt[i * p.T + et];
                         asm volatile("bar.sync 1, %0;" ::"r"(nthr_e) : "memory");
                     }
+                    // this row's multiplier: requested before the wait for the accumulator, so that its latency is not added
+                    // to the time the tensor pipe waits for the accumulator to be read (the task weights are in shared memory)
+                    const float mt = (p.dots == nullptr && t < p.N) ? p.train_mult[(int64_t)i * p.N + t] : 0.0f;
                     ok = mbar_wait_cluster(smem_u32(&bars->d_full), n_acc & 1u, abort_flag, p.timeout_word, TO_EPILOGUE);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-                    const float mt = (p.dots == nullptr && t < p.N) ? p.train_mult[(int64_t)i * p.N + t] : 0.0f;
                     int j = 0;
                     if (p.dots == nullptr) while (j < p.T - 1 && bars->task_off[j + 1] <= v0 + ch_lo * 32) ++j;
                     int next_b = (p.dots == nullptr) ? bars->task_off[j + 1] - v0 : 0x7FFFFFFF;   // first column of task j+1
@@ -523,27 +527,36 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_train, const __grid_con
                                 x[4 * k4 + 2] = __fmul_rn(acc_f(v[4 * k4 + 2]), m4.z);
                                 x[4 * k4 + 3] = __fmul_rn(acc_f(v[4 * k4 + 3]), m4.w);
                             }
-                            if (next_b >= c0 + 32) {          // whole chunk inside task j (the common case)
+                            // Sums in column order. A task that ends inside this chunk (or exactly at its start) closes
+                            // with the columns before its end; the passes are straight-line code with predicated adds (a
+                            // branch per column made such a chunk five times as slow as the others).
+                            int k_lo = 0;
+                            while (next_b < c0 + 32 && j < p.T) {
+                                const int k_hi = next_b - c0;          // 0 .. 31
+#pragma unroll
+                                for (int k = 0; k < 32; ++k) if (k >= k_lo && k < k_hi) task_sum += x[k];
+#pragma unroll
+                                {
+                                    const float add = task_sum * mt * bars->eta_s[j];
+#pragma unroll
+                                    for (int jj = 0; jj < TMAX; ++jj) if (jj == j) A[jj] += add;
+                                }
+                                task_sum = 0.0f;
+                                ++j;
+                                next_b = (j < p.T) ? bars->task_off[j + 1] - v0 : 0x7FFFFFFF;
+                                k_lo = k_hi;
+                            }
+                            if (k_lo == 0) {
 #pragma unroll
                                 for (int k = 0; k < 32; ++k) task_sum += x[k];
                             } else {
 #pragma unroll
-                                for (int k = 0; k < 32; ++k) {
-                                    if (c0 + k == next_b && j < p.T) {   // task j complete
-                                        const float add = task_sum * mt * p.eta_over_cnt[i * p.T + j];
-#pragma unroll
-                                        for (int jj = 0; jj < TMAX; ++jj) if (jj == j) A[jj] += add;
-                                        task_sum = 0.0f;
-                                        ++j;
-                                        next_b = (j < p.T) ? bars->task_off[j + 1] - v0 : 0x7FFFFFFF;
-                                    }
-                                    task_sum += x[k];
-                                }
+                                for (int k = 0; k < 32; ++k) if (k >= k_lo) task_sum += x[k];
                             }
                         }
                     }
                     if (p.dots == nullptr && j < p.T) {
-                        const float add = task_sum * mt * p.eta_over_cnt[i * p.T + j];
+                        const float add = task_sum * mt * bars->eta_s[j];
 #pragma unroll
                         for (int jj = 0; jj < TMAX; ++jj) if (jj == j) A[jj] += add;
                     }

@@ -45,6 +45,32 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
+// try_wait that lets the hardware park the thread for up to hint_ns while the phase is open (it wakes when the phase
+// closes): for waits of roles that share their scheduler with warps that have work to do.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t hint_ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait built on it (same contract as mbar_wait).
+__device__ __forceinline__ bool mbar_wait_parked(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                 unsigned int* timeout_word, uint32_t code, uint32_t hint_ns = 2000u)
+{
+    for (uint32_t it = 0; it < (1u << 22); ++it) {
+        if (mbar_try_wait_parked(bar, parity, hint_ns)) return true;
+        if ((it & 15u) == 15u && *abort_flag) return false;
+    }
+    *abort_flag = 1u;
+    atomicOr(timeout_word, code);
+    return false;
+}
 // One look at the barrier, never suspending the thread (try_wait may park it for a while when the phase is
 // still open): for opportunistic checks on a path that has other work to do.
 __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
