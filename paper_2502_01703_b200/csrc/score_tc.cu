@@ -51,7 +51,7 @@ constexpr int A_STAGE = TM * KB;           // 16 KiB
 constexpr int MAX_STAGES = 8;
 constexpr int NTHREADS = 448;
 // 2- and 1-bit codes: NG groups of four unpack warps (2-5, 10-13, 14-17, ...) and, behind them, four more epilogue warps
-__host__ __device__ constexpr int fp4_groups(int bits) { return 3; }
+__host__ __device__ constexpr int fp4_groups(int bits) { return bits == 1 ? 3 : 4; }
 __host__ __device__ constexpr int fp4_threads(int bits) { return NTHREADS + 128 * (fp4_groups(bits) - 2) + 128; }
 constexpr int TMAX = 8;                    // tasks held in registers by the epilogue
 constexpr int A_TMEM_COL = 448;            // sub-byte widths: two 32-column slots of unpacked train codes
