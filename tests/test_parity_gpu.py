@@ -471,9 +471,10 @@ def test_scores_with_several_validation_tiles(bits, V, off):
     assert np.array_equal(dots, oracle.dots(_np(tc[0]), _np(vc[0]), d, bits))
 
 
-# More tasks than the tensor-core epilogue keeps in registers (8): the call takes the CUDA-core kernel.
+# 7 and 8 tasks: the tensor-core kernels with one epilogue group (two groups exchange six per-task sums). More tasks
+# than the tensor-core epilogue keeps in registers (8): the call takes the CUDA-core kernel.
 @pytest.mark.parametrize("bits", [8, 4, 2, 1])
-@pytest.mark.parametrize("T", [9, 64])
+@pytest.mark.parametrize("T", [7, 8, 9, 64])
 def test_scores_with_many_tasks(bits, T):
     C, N, V, d = 2, 200, 5 * T + 3, 256
     eta = [1.0, 0.25]
