@@ -25,10 +25,11 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 # DRAM bytes of one projection launch per projected coordinate (dram__bytes_read.sum + dram__bytes_write.sum of
-# project_tc_kernel): one ncu capture at n = 256, d = 8192, P = 2^20 gave 735.8 MB + 122.2 MB; both parts grow in
-# proportion to P (the Gamma batch read, and one fp32 partial per 65 536-coordinate chunk written).
-PROJECT_TRAFFIC_BYTES_PER_P = (735.820032e6 + 122.241536e6) / 1048576.0
-PROJECT_TRAFFIC_SOURCE = "ncu capture at n=256, d=8192, P=2^20, scaled by P (profiles/project_tc_kernel__n256_P2e20_d8192.md)"
+# project_tc_kernel): one ncu capture at n = 256, d = 8192, P = 2^22 (the smallest P with the K-chunk length of the
+# benchmark's P = 2^23) gave 2.9665 GB + 120.6 MB; both parts grow in proportion to P (the Gamma batch read, and one fp32
+# partial per 262 144-coordinate chunk written).
+PROJECT_TRAFFIC_BYTES_PER_P = (2.966501e9 + 120.602368e6) / 4194304.0
+PROJECT_TRAFFIC_SOURCE = "ncu capture at n=256, d=8192, P=2^22, scaled by P (profiles/project_tc_kernel__n256_P2e22_d8192.md)"
 WORKLOAD = "c2_project_quantize"
 N_VAL, TASKS, FRAC = 448, [64, 128, 256], 0.05
 SEED = 20250203
