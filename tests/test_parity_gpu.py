@@ -1037,7 +1037,8 @@ def test_bounded_wait_times_out_and_reports():
 
 @pytest.mark.parametrize("what,lo,hi", [("i8_ss_pair", 1e15, 1e16), ("i8_ss_pair_n448", 1e15, 1e16),
                                         ("tma_l2_stream", 1e12, 5e13), ("i8_n448_with_tma", 1e15, 1e16),
-                                        ("i8_n448_commit_per_block", 1e15, 1e16)])
+                                        ("i8_n448_commit_per_block", 1e15, 1e16),
+                                        ("fp4_ss_pair_n448", 2e15, 2e16), ("fp4_ts_pair", 2e15, 2e16)])
 def test_microbenchmarks_run(what, lo, hi):
     ms, ops = B.qless_microbench(what, 2000)
     B.qless_check()
