@@ -16,8 +16,9 @@
 // same slab of Gamma (L2 reuse); after each K-chunk the accumulator is drained to a per-chunk partial,
 // which bounds the length of any fp32 accumulation chain and makes the final sum order fixed.
 //
-// Warp roles (448 threads per CTA): warp 0 TMA producer, warp 1 MMA issuer (leader CTA only; + TMEM
-// allocation in both), warps 2-5 and 10-13 sign generators, warps 6-9 accumulator drain. The leader's barriers
+// Warp roles (448 threads per CTA; 704 for the Gaussian matrix, whose generator has eight more warps, 14-21): warp 0
+// TMA producer, warp 1 MMA issuer (leader CTA only; + TMEM allocation in both), warps 2-5 and 10-13 sign generators,
+// warps 6-9 accumulator drain. The leader's barriers
 // collect the arrivals of both CTAs; tcgen05.commit releases stages in both CTAs at once. All waits are
 // bounded; a wait that gives up raises the device timeout word and every role leaves its loop.
 #include "qless_kernels.h"
@@ -39,6 +40,7 @@ constexpr int B_STAGE_BYTES = (BK / 64) * B_PANEL_BYTES;      // 64 KiB per CTA
 constexpr int TMEM_COLS = 512;
 constexpr int D_COL = 0, A_COL = 256;
 constexpr int NTHREADS = 448;
+constexpr int NTHREADS_GAUSS = 704;     // the Gaussian matrix: eight more generator warps (14-21)
 constexpr uint32_t IDESC = make_idesc(/*D=F32*/ 1, /*A=BF16*/ 1, /*B=BF16*/ 1, 2 * BM, BN);
 
 struct __align__(8) Barriers {
@@ -52,7 +54,7 @@ constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)SB * B_STAGE_BY
 // GAUSS = false: the Rademacher matrix of the method; true: Gaussian entries (Box-Muller on Philox words, bf16),
 // which cost the generator warps about twenty instructions per entry instead of one.
 template <bool GAUSS>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GAUSS ? NTHREADS_GAUSS : NTHREADS, 1)
 project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int32_t d, int64_t P, int64_t chunk,
                   int32_t num_chunks, uint32_t kblk_base, uint64_t seed, float* __restrict__ part,
                   unsigned int* __restrict__ timeout_word)
@@ -72,7 +74,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
     if (threadIdx.x == 0) {
         for (int s = 0; s < SB; ++s) { mbar_init(smem_u32(&bars->b_full[s]), 1); mbar_init(smem_u32(&bars->b_empty[s]), 1); }
         // a_full / d_empty of the leader collect one arrival per generator / drain warp of both CTAs
-        for (int s = 0; s < SA; ++s) { mbar_init(smem_u32(&bars->a_full[s]), 8); mbar_init(smem_u32(&bars->a_empty[s]), 1); }
+        for (int s = 0; s < SA; ++s) { mbar_init(smem_u32(&bars->a_full[s]), GAUSS ? 16 : 8); mbar_init(smem_u32(&bars->a_empty[s]), 1); }
         mbar_init(smem_u32(&bars->d_full), 1);
         mbar_init(smem_u32(&bars->d_empty), 8);
         mbar_init(smem_u32(&bars->drain), 1);
@@ -173,8 +175,11 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
         // ------------------------------- sign generators -------------------------------
         // two groups of four warps (2-5 and 10-13) take alternate 256-deep stages (each group owns one of the two
         // TMEM stages), so that the latency of one stage (Philox chains, TMEM stores, barrier round trip) overlaps the next
+        // (Gaussian matrix: the entries cost twenty times as many instructions, so each stage has eight warps, two per
+        // quadrant: warps 2-5 and 10-13 generate the first 128 columns of their group's stage, warps 14-17 and 18-21 the second)
         const int q = warp & 3;                                  // TMEM lane quadrant this warp may access
-        const uint32_t grp = (warp >= 10) ? 1u : 0u;
+        const uint32_t grp = (warp >= 18) ? 1u : (warp >= 14) ? 0u : (warp >= 10) ? 1u : 0u;
+        const int my_half = (warp >= 14) ? 1 : 0;
         uint32_t ita = 0;
         bool ok = true;
         for (int64_t item = pair; item < num_items && ok; item += num_pairs) {
@@ -191,25 +196,26 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmap_gamma, int64_t n, int
                 const uint32_t blk = kblk_base + (uint32_t)((k0 >> 7) + 2 * ka);          // first 128-column block of the stage
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + A_COL + sa * 128;
                 if constexpr (GAUSS) {
-#pragma unroll 1
-                    for (int h = 0; h < nh; ++h) {
+                    const int h = my_half;
+                    uint32_t v[4][16];                                            // generated before the slot is waited for
+                    if (h < nh) {
                         const uint32_t bh = blk + (uint32_t)h;
-                        uint32_t v[4][16];                                        // generated before the slot is waited for
 #pragma unroll
                         for (int wi = 0; wi < 4; ++wi)
 #pragma unroll
                             for (int c = 0; c < 8; ++c)
                                 gaussian_quad_bf16x2(seed, r, (bh << 5) | (uint32_t)(wi * 8 + c), bh >> 27, v[wi][2 * c], v[wi][2 * c + 1]);
-                        if (h == 0) {
-                            ok = mbar_wait_cluster(smem_u32(&bars->a_empty[sa]), ((ita / SA) & 1u) ^ 1u, abort_flag, timeout_word, TO_GENERATOR);
-                            ok = __all_sync(0xFFFFFFFFu, ok);
-                            if (!ok) break;
-                            tc_fence_after();
-                        }
+                    }
+                    // a warp with nothing to generate (the chunk ends on half a stage) still waits before it arrives: its
+                    // arrival must not land in the stage's previous phase
+                    ok = mbar_wait_cluster(smem_u32(&bars->a_empty[sa]), ((ita / SA) & 1u) ^ 1u, abort_flag, timeout_word, TO_GENERATOR);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (h < nh) {
 #pragma unroll
                         for (int wi = 0; wi < 4; ++wi) tmem_st_x16(taddr + h * 64 + wi * 16, v[wi]);
                     }
-                    if (!ok) break;
                 } else {
                     uint32_t w[2][4];
                     rademacher_block(seed, r, blk, w[0]);     // overlaps with the wait below
@@ -294,7 +300,7 @@ cudaError_t launch_project_tc(const CUtensorMap& tmap, const ProjectPlan& pl, ui
     int64_t grid = (sm_count() / 2) * 2;               // CTA pairs
     if (grid > 2 * items) grid = 2 * items;
     if (pl.gaussian)
-        project_tc_kernel<true><<<(unsigned)grid, NTHREADS, SMEM_BYTES, st>>>(tmap, pl.n, pl.d, pl.P, pl.chunk, pl.num_chunks,
+        project_tc_kernel<true><<<(unsigned)grid, NTHREADS_GAUSS, SMEM_BYTES, st>>>(tmap, pl.n, pl.d, pl.P, pl.chunk, pl.num_chunks,
                                                                               (uint32_t)(pl.k_base >> 7), seed, part, timeout_word);
     else
         project_tc_kernel<false><<<(unsigned)grid, NTHREADS, SMEM_BYTES, st>>>(tmap, pl.n, pl.d, pl.P, pl.chunk, pl.num_chunks,
